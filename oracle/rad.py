@@ -1,0 +1,333 @@
+"""Activation-sampling RAD for fully connected nets: oracle (numpy, float64).
+
+TEST INFRASTRUCTURE ONLY; see the package docstring.
+
+What is computed (paper, Sec. 4.2).  For a linear layer Z = A W + b with
+A in R^{B x D} the weight gradient of exact backprop is dW = A^T dZ.  The only
+Jacobian RAD samples is dh/dW, i.e. the layer input A: it is replaced by
+A_hat = A P with a random P, E[P] = I (Sec. 3.2, the random matrix injection
+S_P[J] = J P and its two required properties).  Everything else on the
+backward path (the loss Jacobian, W, the ReLU derivative bits) is kept exact,
+so only dW is random.
+
+Reading of the sampling law used here.  The paper draws k of d coordinates
+with replacement, P = (d/k) sum_s e_s e_s^T; it also notes that sampling
+without replacement makes fraction 1.0 identical to exact backprop.  This
+oracle uses independent Bernoulli keeps: P = diag(m) / p_eff with
+m_i ~ Bernoulli(p_eff), which has E[P] = I and P = R R^T for
+R = diag(sqrt(m / p_eff)) restricted to kept columns.  "different sample"
+draws m per minibatch row, "same sample" draws one m per layer and step
+(Sec. 4.3).
+
+The keep decision for (row b, column d) compares a 16-bit lane of a
+Philox-4x32-10 output with a threshold T = round(p * 2^16) clipped to
+[1, 2^16]; p_eff = T / 2^16 and stored values are scaled by fl32(2^16 / T) so
+the estimator is exactly unbiased for the probability actually sampled.
+"""
+from dataclasses import dataclass, field
+from typing import List, Optional
+
+import numpy as np
+from scipy.special import erf
+
+from .philox import philox4x32_10
+
+STREAM_DIFFERENT = 0     # counter stream of per-row masks
+STREAM_SAME = 1          # counter stream of masks shared by the minibatch
+LANE_BITS = 16
+LANES_PER_CALL = 8       # 128 output bits / 16
+
+
+# --------------------------------------------------------------------------
+# mask (Sec. 3.2: E[P] = I; Sec. 4.3: "same sample" / "different sample")
+# --------------------------------------------------------------------------
+def keep_threshold(p) -> int:
+    """T such that a 16-bit lane u is kept iff u < T."""
+    p32 = float(np.float32(p))
+    if not (0.0 < p32 <= 1.0):
+        raise ValueError("p must be in (0, 1]")
+    return int(min(max(np.rint(p32 * 65536.0), 1.0), 65536.0))
+
+
+def effective_p(p) -> float:
+    return keep_threshold(p) / 65536.0
+
+
+def scale_factor(p) -> np.float32:
+    """s = fl32(1 / p_eff), one correctly rounded float32 division."""
+    return np.float32(65536.0) / np.float32(keep_threshold(p))
+
+
+def keep_mask(variant: str, B: int, D: int, p, seed: int, layer: int, step: int) -> np.ndarray:
+    """Boolean B x D keep mask.
+
+    Counter = (d // 8, row, layer | stream << 24, step), key = (seed low word,
+    seed high word).  Output word j holds the lanes of columns 8*(d//8) + 2j
+    (low half) and 8*(d//8) + 2j + 1 (high half).  For "same" the row field is
+    0 and the single row of decisions is shared by every minibatch element.
+    """
+    T = keep_threshold(p)
+    groups = (D + LANES_PER_CALL - 1) // LANES_PER_CALL
+    if variant == "different":
+        rows, stream = np.arange(B, dtype=np.uint64)[:, None], STREAM_DIFFERENT
+    elif variant == "same":
+        rows, stream = np.zeros((1, 1), dtype=np.uint64), STREAM_SAME
+    else:
+        raise ValueError(variant)
+    c0 = np.arange(groups, dtype=np.uint64)[None, :]
+    c2 = np.uint64((layer & 0xFFFFFF) | (stream << 24))
+    words = philox4x32_10(c0, rows, c2, np.uint64(step & 0xFFFFFFFF),
+                          np.uint64(seed & 0xFFFFFFFF), np.uint64((seed >> 32) & 0xFFFFFFFF))
+    lanes = np.empty(words[0].shape + (LANES_PER_CALL,), dtype=np.uint32)
+    for j, w in enumerate(words):
+        lanes[..., 2 * j] = w & np.uint32(0xFFFF)
+        lanes[..., 2 * j + 1] = w >> np.uint32(16)
+    m = (lanes < T).reshape(lanes.shape[0], groups * LANES_PER_CALL)[:, :D]
+    if variant == "same":
+        m = np.broadcast_to(m, (B, D))
+    return np.ascontiguousarray(m)
+
+
+# --------------------------------------------------------------------------
+# number formats
+# --------------------------------------------------------------------------
+def round_bf16(x) -> np.ndarray:
+    """float32 -> nearest bf16 (ties to even), returned as float32.  Finite inputs."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    u = x.view(np.uint32).astype(np.uint64)
+    u = (u + np.uint64(0x7FFF) + ((u >> np.uint64(16)) & np.uint64(1))) >> np.uint64(16)
+    return (u << np.uint64(16)).astype(np.uint32).view(np.float32).reshape(x.shape)
+
+
+def bf16_bits(x) -> np.ndarray:
+    """bf16 bit patterns (uint16) of float32 values that already lie on the bf16 grid."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    return (x.view(np.uint32) >> np.uint32(16)).astype(np.uint16).reshape(x.shape)
+
+
+def pack_bits(m: np.ndarray) -> np.ndarray:
+    """Boolean B x D -> uint32 B x ceil(D/32), bit (d % 32) of word d // 32, LSB first."""
+    B, D = m.shape
+    W = (D + 31) // 32
+    padded = np.zeros((B, W * 32), dtype=np.uint64)
+    padded[:, :D] = m
+    weights = (np.uint64(1) << np.arange(32, dtype=np.uint64))
+    return (padded.reshape(B, W, 32) * weights).sum(axis=2).astype(np.uint32)
+
+
+def unpack_bits(words: np.ndarray, D: int) -> np.ndarray:
+    B, W = words.shape
+    bits = (words[:, :, None] >> np.arange(32, dtype=np.uint32)) & np.uint32(1)
+    return bits.reshape(B, W * 32)[:, :D].astype(bool)
+
+
+# --------------------------------------------------------------------------
+# the compact store (Sec. 3.2 "sparsify the input vectors"; App. A memory model)
+# --------------------------------------------------------------------------
+@dataclass
+class Store:
+    variant: str
+    dtype: str
+    B: int
+    D: int
+    T: int
+    scale: np.float32
+    keepbits: np.ndarray                 # uint32; different: B x ceil(D/32); same: 1 x ceil(D/32)
+    values: np.ndarray                   # float32, canonical order (row-major, ascending column)
+    row_ptr: Optional[np.ndarray] = None  # different: int64 B+1
+    idx: Optional[np.ndarray] = None      # same: kept columns ascending
+    relubits: Optional[np.ndarray] = None  # uint32 B x ceil(D/32): (A > 0)
+
+    @property
+    def nnz(self) -> int:
+        return int(self.values.size)
+
+
+def forward_store(A, dtype: str, variant: str, p, seed: int, layer: int, step: int,
+                  mask: Optional[np.ndarray] = None, with_relu_bits: bool = True) -> Store:
+    """What the forward pass keeps of a layer input A (B x D).
+
+    A_hat[b, d] = m[b, d] * round_dtype(fl32(A[b, d] * s)); only the kept
+    entries are emitted.  `mask` replaces the Philox mask (test hook for
+    exhaustive enumeration).  The ReLU derivative of the layer that produced A
+    is (A > 0), one bit per entry (Sec. 4.2; -0.0 and 0.0 give 0).
+    """
+    A = np.ascontiguousarray(A, dtype=np.float32)
+    B, D = A.shape
+    T = keep_threshold(p)
+    s = scale_factor(p)
+    m = keep_mask(variant, B, D, p, seed, layer, step) if mask is None else np.asarray(mask, bool)
+    scaled = A * s                                   # float32 x float32, one rounding
+    if dtype == "bf16":
+        scaled = round_bf16(scaled)
+    elif dtype != "f32":
+        raise ValueError(dtype)
+    relubits = pack_bits(A > 0) if with_relu_bits else None
+    if variant == "different":
+        counts = m.sum(axis=1)
+        row_ptr = np.concatenate([[0], np.cumsum(counts)]).astype(np.int64)
+        return Store(variant, dtype, B, D, T, s, pack_bits(m), scaled[m], row_ptr=row_ptr,
+                     relubits=relubits)
+    if not (m == m[0:1]).all():
+        raise ValueError("same-sample mask must not depend on the row")
+    idx = np.flatnonzero(m[0]).astype(np.int64)
+    return Store(variant, dtype, B, D, T, s, pack_bits(m[0:1]),
+                 np.ascontiguousarray(scaled[:, idx]).reshape(-1), idx=idx, relubits=relubits)
+
+
+def densify(st: Store) -> np.ndarray:
+    """A_hat (B x D, float64) rebuilt from the compact form alone."""
+    Ah = np.zeros((st.B, st.D), dtype=np.float64)
+    if st.variant == "different":
+        m = unpack_bits(st.keepbits, st.D)
+        for b in range(st.B):
+            Ah[b, m[b]] = st.values[st.row_ptr[b]:st.row_ptr[b + 1]]
+    else:
+        Ah[:, st.idx] = st.values.reshape(st.B, st.idx.size)
+    return Ah
+
+
+def weight_grad(st: Store, dZ) -> np.ndarray:
+    """dW_hat = A_hat^T dZ (D x H, float64), using nothing but the store and dZ.
+
+    For "same" only the kept rows of dW_hat can be non-zero (Sec. 4.3: only
+    part of the weight matrix is updated).
+    """
+    dZ = np.asarray(dZ, dtype=np.float64)
+    if st.variant == "same":
+        dW = np.zeros((st.D, dZ.shape[1]), dtype=np.float64)
+        Ac = st.values.reshape(st.B, st.idx.size).astype(np.float64)
+        dW[st.idx, :] = Ac.T @ dZ
+        return dW
+    return densify(st).T @ dZ
+
+
+# --------------------------------------------------------------------------
+# exact pieces of the step (never sampled: Sec. 4.2)
+# --------------------------------------------------------------------------
+def act_forward(Z, act: str):
+    if act == "relu":
+        return np.maximum(Z, 0.0)
+    if act == "gelu":
+        return 0.5 * Z * (1.0 + erf(Z / np.sqrt(2.0)))
+    if act == "none":
+        return Z
+    raise ValueError(act)
+
+
+def gelu_grad(Z):
+    return 0.5 * (1.0 + erf(Z / np.sqrt(2.0))) + Z * np.exp(-0.5 * Z * Z) / np.sqrt(2.0 * np.pi)
+
+
+def softmax_xent(Z, labels):
+    """Mean cross-entropy of softmax(Z) and its Jacobian dZ = (softmax - onehot) / B."""
+    Z = np.asarray(Z, dtype=np.float64)
+    B = Z.shape[0]
+    zmax = Z.max(axis=1, keepdims=True)
+    e = np.exp(Z - zmax)
+    ssum = e.sum(axis=1, keepdims=True)
+    logp = Z - zmax - np.log(ssum)
+    loss = -logp[np.arange(B), labels].mean()
+    dZ = e / ssum
+    dZ[np.arange(B), labels] -= 1.0
+    return loss, dZ / B
+
+
+def input_grad(dZ, W, relubits_prev=None, Z_prev=None, act="relu", dtype="f32"):
+    """Exact dA = dZ W^T, masked by the derivative of the activation that produced A; db = sum_b dZ."""
+    dZ = np.asarray(dZ, dtype=np.float64)
+    dA = dZ @ np.asarray(W, dtype=np.float64).T
+    if act == "relu" and relubits_prev is not None:
+        dA = dA * unpack_bits(relubits_prev, dA.shape[1])
+    elif act == "gelu" and Z_prev is not None:
+        dA = dA * gelu_grad(np.asarray(Z_prev, dtype=np.float64))
+    if dtype == "bf16":
+        dA = round_bf16(dA.astype(np.float32)).astype(np.float64)
+    elif dtype == "f32":
+        dA = dA.astype(np.float32).astype(np.float64)
+    return dA, dZ.sum(axis=0)
+
+
+@dataclass
+class StepResult:
+    loss: float
+    Z: List[np.ndarray]
+    A: List[np.ndarray]                 # A[0] = X, A[l] = act(Z[l-1])
+    dZ: List[np.ndarray]
+    dW: List[np.ndarray]
+    db: List[np.ndarray]
+    stores: List[Optional[Store]] = field(default_factory=list)
+
+
+def mlp_step(X, labels, Ws, bs, act="relu", dtype="f32", variant=None, p=1.0, seed=0, step=0,
+             masks=None) -> StepResult:
+    """One forward + backward pass of a fully connected net with softmax cross-entropy.
+
+    variant None: exact backprop (dW_l = A_{l-1}^T dZ_l).  Otherwise the input
+    of every linear layer, the network input included, goes through
+    forward_store and dW_l comes from the store; the softmax input is not
+    sampled (App. A).  The tensors that live on the device in the working type
+    (activations, stored pre-activations, dZ: float32 or bf16) are rounded to
+    it at those points and nowhere else; accumulations stay in float64.
+    """
+    L = len(Ws)
+    W64 = [np.asarray(W, dtype=np.float64) for W in Ws]
+    b64 = [np.asarray(b, dtype=np.float64) for b in bs]
+    if dtype == "bf16":
+        rnd = lambda v: round_bf16(np.asarray(v, np.float32)).astype(np.float64)
+    elif dtype == "f32":
+        rnd = lambda v: np.asarray(v, np.float32).astype(np.float64)
+    elif dtype == "f64" and variant is None:         # no rounding at all: for pins of the exact net
+        rnd = lambda v: np.asarray(v, np.float64)
+    else:
+        raise ValueError(dtype)
+    A = [np.asarray(X, dtype=np.float64)]
+    Z, stores = [], []
+    for l in range(L):
+        if variant is not None:
+            stores.append(forward_store(A[l].astype(np.float32), dtype, variant, p, seed, l, step,
+                                        mask=None if masks is None else masks[l]))
+        else:
+            stores.append(None)
+        z = A[l] @ W64[l] + b64[l]
+        if l < L - 1:
+            Z.append(rnd(z) if act == "gelu" else z)   # a GELU net keeps Z (bf16) for the backward
+            A.append(rnd(act_forward(z, act)))
+        else:
+            Z.append(z)
+    loss, dz = softmax_xent(Z[-1], labels)
+    dZ = [None] * L
+    dW = [None] * L
+    db = [None] * L
+    dZ[L - 1] = rnd(dz)
+    for l in range(L - 1, -1, -1):
+        dW[l] = A[l].T @ dZ[l] if variant is None else weight_grad(stores[l], dZ[l])
+        if l > 0:
+            if act == "relu":
+                dA, db[l] = input_grad(dZ[l], W64[l], relubits_prev=pack_bits(A[l] > 0), dtype=dtype)
+            else:
+                dA, db[l] = input_grad(dZ[l], W64[l], Z_prev=Z[l - 1], act=act, dtype=dtype)
+            dZ[l - 1] = dA
+        else:
+            db[l] = dZ[l].sum(axis=0)
+    return StepResult(loss, Z, A, dZ, dW, db, stores)
+
+
+# --------------------------------------------------------------------------
+# bytes held between forward and backward (App. A, "Calculation of memory saved")
+# --------------------------------------------------------------------------
+def stored_bytes(stores: List[Store], logits_shape, elem_bytes: int):
+    """Bytes the compact stores really hold, split by kind, and the full-backprop figure."""
+    value_bytes = sum(st.nnz * elem_bytes for st in stores)
+    index_bytes = 0
+    relu_bytes = 0
+    full = 0
+    for i, st in enumerate(stores):
+        words = (st.D + 31) // 32
+        index_bytes += 4 * words * (st.B if st.variant == "different" else 1)
+        if i > 0:                                   # the network input is not a ReLU output
+            relu_bytes += 4 * words * st.B
+        full += st.B * st.D * elem_bytes
+    unsampled = int(np.prod(logits_shape)) * 4
+    return dict(value_bytes=value_bytes, index_bytes=index_bytes, relu_bytes=relu_bytes,
+                unsampled_bytes=unsampled, full_backprop_bytes=full + unsampled)

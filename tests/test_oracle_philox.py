@@ -1,0 +1,81 @@
+"""Pins for the oracle's Philox-4x32-10 (host only).
+
+The generator's published known-answer vectors are not available offline, so
+conformance to them is unpinned.  What is pinned: agreement with an
+independent restatement in Python big integers, invertibility of each round
+(multiplication by an odd constant is a bijection mod 2^32), sensitivity to
+every counter/key word, and lane uniformity.
+"""
+import numpy as np
+
+from oracle import philox as ph
+
+M0, M1, W0, W1 = 0xD2511F53, 0xCD9E8D57, 0x9E3779B9, 0xBB67AE85
+MASK = (1 << 32) - 1
+
+
+def bigint_philox(ctr, key, rounds=10):
+    c = list(ctr)
+    k = list(key)
+    for r in range(rounds):
+        if r:
+            k = [(k[0] + W0) & MASK, (k[1] + W1) & MASK]
+        p0, p1 = M0 * c[0], M1 * c[2]
+        c = [(p1 >> 32) ^ c[1] ^ k[0], p1 & MASK, (p0 >> 32) ^ c[3] ^ k[1], p0 & MASK]
+    return c
+
+
+def inverse_round(c, k):
+    """Undo one round: word 1 and 3 are the low product halves, so the inputs follow by modular inverse."""
+    inv0, inv1 = pow(M0, -1, 1 << 32), pow(M1, -1, 1 << 32)
+    c0 = (c[3] * inv0) & MASK
+    c2 = (c[1] * inv1) & MASK
+    c1 = c[0] ^ ((M1 * c2) >> 32) ^ k[0]
+    c3 = c[2] ^ ((M0 * c0) >> 32) ^ k[1]
+    return [c0, c1, c2, c3]
+
+
+def test_matches_bigint_restatement():
+    rng = np.random.default_rng(7)
+    n = 20000
+    ctr = rng.integers(0, 1 << 32, size=(n, 4), dtype=np.uint64)
+    key = rng.integers(0, 1 << 32, size=(n, 2), dtype=np.uint64)
+    # include the corners where carries and masks matter
+    ctr[:4] = [[0, 0, 0, 0], [MASK] * 4, [1, 0, 0, 0], [0, 0, MASK, 1]]
+    key[:4] = [[0, 0], [MASK, MASK], [0, 1], [MASK, 0]]
+    out = ph.philox4x32_10(ctr[:, 0], ctr[:, 1], ctr[:, 2], ctr[:, 3], key[:, 0], key[:, 1])
+    out = np.stack(out, axis=1)
+    for i in range(0, n, 7):
+        assert list(out[i]) == bigint_philox([int(v) for v in ctr[i]], [int(v) for v in key[i]])
+    for i in range(4):
+        assert list(out[i]) == bigint_philox([int(v) for v in ctr[i]], [int(v) for v in key[i]])
+
+
+def test_round_is_invertible():
+    rng = np.random.default_rng(11)
+    for _ in range(200):
+        c = [int(v) for v in rng.integers(0, 1 << 32, size=4, dtype=np.uint64)]
+        k = [int(v) for v in rng.integers(0, 1 << 32, size=2, dtype=np.uint64)]
+        out = ph.philox4x32_round(*(np.uint64(v) for v in c), *(np.uint64(v) for v in k))
+        assert inverse_round([int(v) for v in out], k) == c
+
+
+def test_every_input_word_matters():
+    base = [3, 5, 7, 11, 13, 17]
+    ref = np.stack(ph.philox4x32_10(*[np.uint64(v) for v in base]))
+    for i in range(6):
+        alt = list(base)
+        alt[i] ^= 1
+        out = np.stack(ph.philox4x32_10(*[np.uint64(v) for v in alt]))
+        assert (out != ref).all()
+
+
+def test_lane_uniformity_chi_square():
+    n = 1 << 16
+    words = ph.philox4x32_10(np.arange(n, dtype=np.uint64), 9, 2, 0, 42, 0)
+    lanes = np.concatenate([w & np.uint32(0xFFFF) for w in words] + [w >> np.uint32(16) for w in words])
+    hist = np.bincount(lanes >> 8, minlength=256).astype(np.float64)
+    expected = lanes.size / 256.0
+    chi2 = ((hist - expected) ** 2 / expected).sum()
+    # 255 degrees of freedom: mean 255, sd ~22.6; 6 sigma band
+    assert abs(chi2 - 255.0) < 6 * 22.6

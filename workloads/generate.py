@@ -1,0 +1,70 @@
+"""Seeded generators for inputs, labels and weights (numpy PCG64 streams).
+
+Every array is returned as float32 (labels as int32).  For bf16 workloads the
+float32 values already lie on the bf16 grid, so converting them to bf16 on
+either side of a comparison is exact.
+"""
+import numpy as np
+
+
+def to_bf16_grid(x: np.ndarray) -> np.ndarray:
+    """Round float32 values to the nearest bf16 value (ties to even), kept as float32."""
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32))
+    return t.to(torch.bfloat16).to(torch.float32).numpy()
+
+
+def uniform_labels(rng: np.random.Generator, batch: int, classes: int) -> np.ndarray:
+    return rng.integers(0, classes, size=batch, dtype=np.int64).astype(np.int32)
+
+
+def _draw(rng, shape, dist):
+    if dist == "uniform01":
+        return rng.random(shape, dtype=np.float32)
+    if dist == "normal":
+        return rng.standard_normal(shape, dtype=np.float32)
+    raise ValueError(dist)
+
+
+def mlp_inputs(dims, batch, dtype="f32", x_dist="uniform01", seed=1234, bias_zero=True):
+    """Inputs of one training step of a fully connected net.
+
+    X is batch x dims[0]; weight l is dims[l] x dims[l+1] (fan-in major, the
+    paper's h = W^T x written row-wise as Z = A W), Kaiming-normal with
+    std sqrt(2 / fan_in); biases are zero unless bias_zero is False, in which
+    case they are small normals so bias paths are exercised.
+    """
+    rng = np.random.default_rng(seed)
+    X = _draw(rng, (batch, dims[0]), x_dist)
+    labels = uniform_labels(rng, batch, dims[-1])
+    Ws, bs = [], []
+    for l in range(len(dims) - 1):
+        std = np.float32(np.sqrt(2.0 / dims[l]))
+        Ws.append(rng.standard_normal((dims[l], dims[l + 1]), dtype=np.float32) * std)
+        if bias_zero:
+            bs.append(np.zeros(dims[l + 1], dtype=np.float32))
+        else:
+            bs.append(rng.standard_normal(dims[l + 1], dtype=np.float32) * np.float32(0.1))
+    if dtype == "bf16":
+        X = to_bf16_grid(X)
+        Ws = [to_bf16_grid(W) for W in Ws]
+    return X, labels, Ws, bs
+
+
+def layer_inputs(B, D, H, dtype="f32", x_dist="normal", seed=1234, relu_like=False):
+    """Inputs of the per-layer calls: activations A (B x D) and output gradient dZ (B x H).
+
+    With relu_like=True about half of A is exactly zero and a few entries are
+    -0.0, as after a ReLU, so the sign-bit cases of the 1-bit derivative store
+    are covered.
+    """
+    rng = np.random.default_rng(seed)
+    A = _draw(rng, (B, D), x_dist)
+    if relu_like:
+        A = np.maximum(A, np.float32(0))
+        neg0 = rng.random((B, D)) < 0.01
+        A = np.where(neg0 & (A == 0), np.float32(-0.0), A).astype(np.float32)
+    dZ = rng.standard_normal((B, H), dtype=np.float32) * np.float32(1.0 / max(B, 1))
+    if dtype == "bf16":
+        A, dZ = to_bf16_grid(A), to_bf16_grid(dZ)
+    return A, dZ
