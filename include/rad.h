@@ -1,0 +1,246 @@
+/*
+ * rad.h - C ABI of the RAD activation-sampling library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the neural-network instance of Randomized Automatic
+ * Differentiation (Oktay et al., ICLR 2021, Sec. 4.2): for every linear layer
+ * Z = A W + b the forward pass keeps only a random subsample of the layer input
+ * A (B x D), rescaled so that it is an unbiased stand-in for A, and the backward
+ * pass forms the weight gradient from that subsample, dW_hat = A_hat^T dZ, while
+ * dX = dZ W^T, the bias gradient and the ReLU derivative stay exact.
+ *
+ * Conventions for every entry point
+ *   - "device" pointers are CUDA global-memory addresses owned by the caller; the
+ *     library allocates nothing the caller must free and keeps no pointer after
+ *     the call returns.  "host" pointers are ordinary process memory.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*); no call
+ *     synchronises the device.  Outputs are valid once the stream reaches the end
+ *     of the enqueued work.
+ *   - Return value: RAD_OK or a negative host-detected error; nothing is enqueued
+ *     when an error is returned unless stated otherwise.
+ *   - `dev_status` (device int32, may be NULL) receives conditions only the device
+ *     can see (RAD_DEV_*).  It is sticky: the first non-zero code wins and the
+ *     library never clears it.  A kernel that raises one finishes without
+ *     touching memory outside the caller's buffers.
+ *   - Matrices are row-major with a leading dimension in elements.
+ *   - bf16 paths need D and H to be multiples of 8 and all bf16 pointers and
+ *     leading dimensions to be 16-byte aligned (TMA); otherwise
+ *     RAD_EUNSUPPORTED.  f32 paths have no alignment rule beyond 4 bytes.
+ */
+#ifndef RAD_H_
+#define RAD_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define RAD_OK            0
+#define RAD_EINVAL       (-1)  /* bad argument (null pointer, size, p outside (0,1], enum)   */
+#define RAD_EUNSUPPORTED (-2)  /* not an sm_100 device, or an alignment rule is not met      */
+#define RAD_ECUDA        (-3)  /* a CUDA runtime or driver call failed                       */
+#define RAD_EWORKSPACE   (-4)  /* workspace_bytes is smaller than the matching *_workspace   */
+
+#define RAD_DEV_OK        0
+#define RAD_DEV_ECAPACITY 1    /* the compact store did not fit values_capacity / values_ld  */
+#define RAD_DEV_ETIMEOUT  2    /* a bounded device-side wait expired                         */
+
+typedef enum { RAD_F32 = 0, RAD_BF16 = 1 } rad_dtype;
+typedef enum { RAD_DIFFERENT_SAMPLE = 0, RAD_SAME_SAMPLE = 1 } rad_variant;
+typedef enum { RAD_ACT_NONE = 0, RAD_ACT_RELU = 1, RAD_ACT_GELU = 2 } rad_act;
+
+/* Geometry of the compact store (fixed; part of the data layout). */
+#define RAD_TILE_ROWS   64     /* minibatch rows per tile                                    */
+#define RAD_TILE_COLS   128    /* layer-input columns per tile                               */
+#define RAD_VALUE_ALIGN 8      /* every tile's values start at a multiple of 8 elements      */
+
+/*
+ * The mask (Sec. 3.2: a random P with E[P] = I; Sec. 4.3: "same sample" /
+ * "different sample").  Entry (b, d) is kept iff a 16-bit lane of
+ * Philox-4x32-10 is below T = clamp(rint(p * 65536), 1, 65536):
+ *   key     = (seed & 0xffffffff, seed >> 32)
+ *   counter = (d / 8, row, layer | stream << 24, step), row = b and stream = 0
+ *             for different-sample; row = 0 and stream = 1 for same-sample
+ *   lane of column d = 16-bit half (d & 1) of output word (d % 8) / 2.
+ * p_eff = T / 65536 is the probability actually sampled and kept values are
+ * multiplied by fl32(65536 / T) = 1 / p_eff, so E[A_hat] = A exactly.
+ */
+uint32_t rad_keep_threshold(float p);   /* T; 0 if p is outside (0, 1]                        */
+float    rad_effective_p(float p);      /* T / 65536                                          */
+float    rad_scale(float p);            /* fl32(65536 / T)                                    */
+
+/*
+ * One layer's compact store: plain data, all buffers device memory of the caller.
+ *
+ * different-sample layout.  Rows are cut into slabs of RAD_TILE_ROWS, columns
+ * into blocks of RAD_TILE_COLS; tile t = slab * ceil(D / 128) + block.
+ *   keepbits : 256 words per tile, word (r * 4 + w) of tile t holds the keep bits
+ *              of row slab*64 + r, columns block*128 + 32*w .. +31, LSB first.
+ *              Bits of rows >= B or columns >= D are 0.
+ *   values   : the kept entries of tile t, A[b,d] * scale rounded once to `dtype`,
+ *              in (row, column) order, start at element offsets[t]; the tile is
+ *              padded with zeros to a multiple of RAD_VALUE_ALIGN elements.
+ *   offsets  : ntiles + 1 words; offsets[ntiles] = elements used in `values`.
+ *   nnz      : nnz[0] = number of kept entries, nnz[1] = offsets[ntiles].
+ * same-sample layout.
+ *   keepbits : ceil(D / 32) words, bit d%32 of word d/32.
+ *   offsets  : kept columns in ascending order (k' entries, room for D).
+ *   values   : B x values_ld row-major; values[b, j] = A[b, offsets[j]] * scale
+ *              for j < k', zero for k' <= j < values_ld.
+ *   nnz      : nnz[0] = k', nnz[1] = B * k'.
+ * relubits (optional, either variant): B x ceil(D / 32) words row-major,
+ *   bit = (A[b,d] > 0): the 1-bit ReLU derivative of the layer that produced A
+ *   (Sec. 4.2).  Zero of either sign gives 0.  NULL skips it.
+ */
+typedef struct rad_store {
+  int32_t   variant;          /* rad_variant */
+  int32_t   dtype;            /* rad_dtype of A and of `values` */
+  int64_t   B, D;
+  float     p;                /* requested keep probability, 0 < p <= 1 */
+  uint32_t  layer, step;
+  uint64_t  seed;
+  void*     values;
+  int64_t   values_capacity;  /* elements available in `values` */
+  int64_t   values_ld;        /* same-sample: leading dimension (multiple of 8); else ignored */
+  uint32_t* keepbits;
+  uint32_t* offsets;
+  int64_t*  nnz;              /* 2 device int64 */
+  uint32_t* relubits;         /* or NULL */
+} rad_store;
+
+typedef struct rad_store_sizes {
+  int64_t values_worst;       /* elements that always suffice (p_eff = 1 plus padding)        */
+  int64_t values_typical;     /* mean + 8 sigma of the kept count plus padding                */
+  int64_t values_ld_worst;    /* same-sample leading dimension that always suffices           */
+  int64_t values_ld_typical;  /* same-sample: mean + 8 sigma of k', rounded up to 64          */
+  int64_t keepbits_words, offsets_words, relubits_words;
+  int64_t workspace_bytes;    /* scratch rad_linear_forward_store needs                        */
+} rad_store_sizes;
+
+/* Buffer sizes for a store of the given shape (host only, nothing is launched). */
+int rad_store_size_query(int32_t variant, int32_t dtype, int64_t B, int64_t D, float p,
+                         rad_store_sizes* out /* host */);
+
+/*
+ * Forward-pass store of one layer input (Sec. 3.2 "sparsify the input vectors";
+ * Sec. 4.2 sampling of dh/dW).  Reads A (device, B x D, leading dimension lda,
+ * type st->dtype), draws the mask, and fills st->keepbits / values / offsets /
+ * nnz (and relubits).  `st` is a host struct read during the call.  `workspace`
+ * is device scratch of at least rad_store_sizes.workspace_bytes, 256-byte
+ * aligned, contents irrelevant on entry.  If the kept entries do not fit the
+ * capacity, RAD_DEV_ECAPACITY is raised, the overflowing values are dropped and
+ * nnz still reports the exact counts.
+ */
+int rad_linear_forward_store(const void* A /* device */, int64_t lda, const rad_store* st /* host */,
+                             void* workspace /* device */, int64_t workspace_bytes,
+                             int32_t* dev_status /* device or NULL */, void* stream);
+
+/* Scratch rad_linear_weight_grad needs for this store and H (host only). */
+int rad_weight_grad_workspace(const rad_store* st /* host */, int64_t H, int64_t* bytes /* host */);
+
+/*
+ * Backward-pass weight gradient from the store alone (Sec. 4.2, the sampled
+ * Jacobian S_P[dh/dW] in the chain): dW[d, h] = sum_b A_hat[b, d] dZ[b, h].
+ * dZ is device, B x H, type st->dtype; dW is device float32, D x H, overwritten
+ * (for same-sample the rows of columns that were not kept are set to zero,
+ * Sec. 4.3).  Accumulation is in float32 in a fixed order: results are
+ * bit-reproducible run to run.
+ */
+int rad_linear_weight_grad(const rad_store* st /* host */, const void* dZ /* device */, int64_t ldz,
+                           int64_t H, float* dW /* device */, int64_t ldw,
+                           void* workspace /* device */, int64_t workspace_bytes,
+                           int32_t* dev_status, void* stream);
+
+/*
+ * Exact forward of one layer (never sampled: Sec. 3, the original graph is used
+ * for the forward pass): Z = A W + bias, out = act(Z).
+ *   A device B x D (dtype), W device D x H (dtype), bias device float32[H] or NULL.
+ *   out_act  device B x H (dtype) or NULL: act(Z) rounded to dtype.
+ *   out_z    device B x H float32 or NULL: Z before the activation (the softmax input).
+ *   out_zlow device B x H (dtype) or NULL: Z rounded to dtype (kept by GELU nets).
+ *   relubits device B x ceil(H/32) words or NULL: (act(Z) > 0) packed as in rad_store.
+ */
+int rad_linear_forward(int32_t dtype, int32_t act, int64_t B, int64_t D, int64_t H,
+                       const void* A, int64_t lda, const void* W, int64_t ldw, const float* bias,
+                       void* out_act, int64_t ld_act, float* out_z, int64_t ld_z,
+                       void* out_zlow, int64_t ld_zlow, uint32_t* relubits,
+                       int32_t* dev_status, void* stream);
+
+/*
+ * Loss Jacobian (exact, Sec. 4.2: not a memory bottleneck, never sampled):
+ * loss = mean_b CE(softmax(logits_b), label_b), dZ = (softmax - onehot) / B.
+ *   logits device float32 B x C; labels device int32[B]; loss device float32[1];
+ *   dZ device B x C (dtype).  `workspace`: device, at least 4 * B bytes.
+ */
+int rad_softmax_xent(int32_t dtype, int64_t B, int64_t C, const float* logits, int64_t ldl,
+                     const int32_t* labels, float* loss, void* dZ, int64_t ldz,
+                     void* workspace, int64_t workspace_bytes, void* stream);
+
+/*
+ * Exact input gradient and bias gradient (Sec. 4.2: W is batch-independent, the
+ * activation derivative is stored exactly):
+ *   dA = dZ W^T; dZ_prev = dA * act'(.) ; db[h] = sum_b dZ[b, h].
+ *   dZ device B x H (dtype); W device D x H (dtype).
+ *   relubits_prev device B x ceil(D/32) words (ReLU nets) or NULL.
+ *   z_prev device B x D (dtype), pre-activation of the producing layer (GELU nets) or NULL.
+ *   dZ_prev device B x D (dtype) or NULL (first layer: no input gradient wanted).
+ *   db device float32[H] or NULL.  `workspace`: device scratch for the column
+ *   sums, at least rad_input_grad_workspace bytes.
+ */
+int rad_input_grad_workspace(int64_t B, int64_t H, int64_t* bytes /* host */);
+int rad_linear_input_grad(int32_t dtype, int64_t B, int64_t D, int64_t H,
+                          const void* dZ, int64_t ldz, const void* W, int64_t ldw,
+                          const uint32_t* relubits_prev, const void* z_prev, int64_t ld_zprev,
+                          void* dZ_prev, int64_t ldp, float* db,
+                          void* workspace, int64_t workspace_bytes,
+                          int32_t* dev_status, void* stream);
+
+/* One training step of a fully connected net with softmax cross-entropy. */
+typedef struct rad_mlp_desc {
+  int32_t  L;                 /* linear layers */
+  int32_t  act;               /* rad_act between layers (none after the last) */
+  int32_t  dtype;             /* rad_dtype of X, W, activations, dZ */
+  int32_t  variant;           /* rad_variant */
+  const int64_t* dims;        /* host, L + 1 entries: fan-in of layer 1 .. fan-out of layer L */
+  int64_t  B;
+  float    p;
+  uint32_t step;
+  uint64_t seed;
+} rad_mlp_desc;
+
+typedef struct rad_step_stats {   /* bytes held between forward and backward (App. A accounting) */
+  int64_t value_bytes;            /* capacity reserved for kept values (mean + 8 sigma)          */
+  int64_t index_bytes;            /* keep bitmasks / kept-column lists and tile offsets          */
+  int64_t relu_bytes;             /* 1-bit ReLU derivatives                                      */
+  int64_t preact_bytes;           /* pre-activations kept whole (GELU nets only)                 */
+  int64_t unsampled_bytes;        /* the softmax input, stored whole                             */
+  int64_t full_backprop_bytes;    /* what exact backprop would hold: every layer input + logits  */
+} rad_step_stats;
+
+int rad_mlp_workspace(const rad_mlp_desc* net /* host */, int64_t* bytes /* host */,
+                      rad_step_stats* stats /* host or NULL */);
+
+/*
+ * Forward, loss and RAD backward of the whole net on one stream (Sec. 4.2 for
+ * arbitrary depth): every layer input, the network input included, is stored
+ * through the mask of (seed, layer l, step); the softmax input is kept whole;
+ * dW_l comes from store l, everything else is exact.
+ *   X device B x dims[0] (dtype, dense); labels device int32[B];
+ *   W[l] device dims[l] x dims[l+1] (dtype, dense); b[l] device float32 or NULL entries;
+ *   dW[l] device float32 dims[l] x dims[l+1]; db[l] device float32; loss device float32[1].
+ *   W, b, dW, db are host arrays of L device pointers.
+ *   nnz_out device int64[2*L] or NULL: the nnz pair of every layer's store.
+ */
+int rad_mlp_step(const rad_mlp_desc* net /* host */, const void* X, const int32_t* labels,
+                 const void* const* W, const float* const* b,
+                 float* const* dW, float* const* db, float* loss, int64_t* nnz_out,
+                 void* workspace, int64_t workspace_bytes,
+                 int32_t* dev_status, void* stream);
+
+const char* rad_strerror(int code);
+const char* rad_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RAD_H_ */

@@ -1,0 +1,268 @@
+"""ctypes binding of librad_b200.so: argument marshalling only.
+
+Every function here has the name of the C entry point it calls (include/rad.h)
+and passes torch tensors by data pointer plus the current CUDA stream.  torch
+is used for device memory and streams; no arithmetic of the method happens in
+Python.  There is no CPU fallback: a missing library or a negative return code
+raises.
+"""
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "librad_b200.so")
+
+RAD_F32, RAD_BF16 = 0, 1
+RAD_DIFFERENT_SAMPLE, RAD_SAME_SAMPLE = 0, 1
+RAD_ACT_NONE, RAD_ACT_RELU, RAD_ACT_GELU = 0, 1, 2
+RAD_DEV_ECAPACITY, RAD_DEV_ETIMEOUT = 1, 2
+TILE_ROWS, TILE_COLS, VALUE_ALIGN = 64, 128, 8
+
+DTYPES = {"f32": RAD_F32, "bf16": RAD_BF16, torch.float32: RAD_F32, torch.bfloat16: RAD_BF16}
+VARIANTS = {"different": RAD_DIFFERENT_SAMPLE, "same": RAD_SAME_SAMPLE}
+ACTS = {"none": RAD_ACT_NONE, "relu": RAD_ACT_RELU, "gelu": RAD_ACT_GELU}
+TORCH_DTYPE = {RAD_F32: torch.float32, RAD_BF16: torch.bfloat16}
+
+
+class RadError(RuntimeError):
+    pass
+
+
+class rad_store(C.Structure):
+    _fields_ = [("variant", C.c_int32), ("dtype", C.c_int32), ("B", C.c_int64), ("D", C.c_int64),
+                ("p", C.c_float), ("layer", C.c_uint32), ("step", C.c_uint32), ("seed", C.c_uint64),
+                ("values", C.c_void_p), ("values_capacity", C.c_int64), ("values_ld", C.c_int64),
+                ("keepbits", C.c_void_p), ("offsets", C.c_void_p), ("nnz", C.c_void_p),
+                ("relubits", C.c_void_p)]
+
+
+class rad_store_sizes(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in ("values_worst", "values_typical", "values_ld_worst",
+                                         "values_ld_typical", "keepbits_words", "offsets_words",
+                                         "relubits_words", "workspace_bytes")]
+
+
+class rad_mlp_desc(C.Structure):
+    _fields_ = [("L", C.c_int32), ("act", C.c_int32), ("dtype", C.c_int32), ("variant", C.c_int32),
+                ("dims", C.POINTER(C.c_int64)), ("B", C.c_int64), ("p", C.c_float), ("step", C.c_uint32),
+                ("seed", C.c_uint64)]
+
+
+class rad_step_stats(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in ("value_bytes", "index_bytes", "relu_bytes", "preact_bytes",
+                                         "unsampled_bytes", "full_backprop_bytes")]
+
+
+EXPORTS = ["rad_keep_threshold", "rad_effective_p", "rad_scale", "rad_store_size_query",
+           "rad_linear_forward_store", "rad_weight_grad_workspace", "rad_linear_weight_grad",
+           "rad_linear_forward", "rad_softmax_xent", "rad_input_grad_workspace", "rad_linear_input_grad",
+           "rad_mlp_workspace", "rad_mlp_step", "rad_strerror", "rad_version"]
+
+_lib = None
+
+
+def lib():
+    """The loaded shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RadError(f"{LIB_PATH} is missing: run `python -m paper_2007_10412_b200.build`")
+        L = C.CDLL(LIB_PATH)
+        L.rad_keep_threshold.restype = C.c_uint32
+        L.rad_keep_threshold.argtypes = [C.c_float]
+        L.rad_effective_p.restype = C.c_float
+        L.rad_effective_p.argtypes = [C.c_float]
+        L.rad_scale.restype = C.c_float
+        L.rad_scale.argtypes = [C.c_float]
+        L.rad_strerror.restype = C.c_char_p
+        L.rad_strerror.argtypes = [C.c_int]
+        L.rad_version.restype = C.c_char_p
+        i32, i64, f32, vp = C.c_int32, C.c_int64, C.c_float, C.c_void_p
+        L.rad_store_size_query.argtypes = [i32, i32, i64, i64, f32, C.POINTER(rad_store_sizes)]
+        L.rad_linear_forward_store.argtypes = [vp, i64, C.POINTER(rad_store), vp, i64, vp, vp]
+        L.rad_weight_grad_workspace.argtypes = [C.POINTER(rad_store), i64, C.POINTER(i64)]
+        L.rad_linear_weight_grad.argtypes = [C.POINTER(rad_store), vp, i64, i64, vp, i64, vp, i64, vp, vp]
+        L.rad_linear_forward.argtypes = [i32, i32, i64, i64, i64, vp, i64, vp, i64, vp, vp, i64, vp, i64,
+                                         vp, i64, vp, vp, vp]
+        L.rad_softmax_xent.argtypes = [i32, i64, i64, vp, i64, vp, vp, vp, i64, vp, i64, vp]
+        L.rad_input_grad_workspace.argtypes = [i64, i64, C.POINTER(i64)]
+        L.rad_linear_input_grad.argtypes = [i32, i64, i64, i64, vp, i64, vp, i64, vp, vp, i64, vp, i64, vp,
+                                            vp, i64, vp, vp]
+        L.rad_mlp_workspace.argtypes = [C.POINTER(rad_mlp_desc), C.POINTER(i64), C.POINTER(rad_step_stats)]
+        L.rad_mlp_step.argtypes = [C.POINTER(rad_mlp_desc), vp, vp, C.POINTER(vp), C.POINTER(vp),
+                                   C.POINTER(vp), C.POINTER(vp), vp, vp, vp, i64, vp, vp]
+        for name in EXPORTS:
+            fn = getattr(L, name)
+            if fn.restype is C.c_int:
+                fn.restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _check(rc, what):
+    if rc != 0:
+        raise RadError(f"{what} failed: {lib().rad_strerror(rc).decode()} ({rc})")
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _ld(t):
+    return 0 if t is None else t.stride(0)
+
+
+def rad_keep_threshold(p):
+    return int(lib().rad_keep_threshold(p))
+
+
+def rad_effective_p(p):
+    return float(lib().rad_effective_p(p))
+
+
+def rad_scale(p):
+    return float(lib().rad_scale(p))
+
+
+def rad_version():
+    return lib().rad_version().decode()
+
+
+def rad_store_size_query(variant, dtype, B, D, p):
+    out = rad_store_sizes()
+    _check(lib().rad_store_size_query(VARIANTS[variant], DTYPES[dtype], B, D, p, C.byref(out)),
+           "rad_store_size_query")
+    return out
+
+
+class Store:
+    """Device buffers of one layer's compact store plus the host struct that describes them."""
+
+    def __init__(self, variant, dtype, B, D, p, seed=0, layer=0, step=0, relu_bits=True, capacity="typical",
+                 device="cuda"):
+        self.variant, self.dtype, self.B, self.D, self.p = variant, dtype, B, D, p
+        sz = rad_store_size_query(variant, dtype, B, D, p)
+        self.sizes = sz
+        cap = {"typical": sz.values_typical, "worst": sz.values_worst}.get(capacity, capacity)
+        ld = 0
+        if variant == "same":
+            ld = {"typical": sz.values_ld_typical, "worst": sz.values_ld_worst}.get(capacity, capacity)
+            cap = B * ld
+        tdt = TORCH_DTYPE[DTYPES[dtype]]
+        self.values = torch.empty(max(int(cap), 8), dtype=tdt, device=device)
+        self.keepbits = torch.empty(sz.keepbits_words, dtype=torch.int32, device=device)
+        self.offsets = torch.empty(sz.offsets_words, dtype=torch.int32, device=device)
+        self.nnz = torch.zeros(2, dtype=torch.int64, device=device)
+        self.relubits = torch.empty(sz.relubits_words, dtype=torch.int32, device=device) if relu_bits else None
+        self.workspace = torch.empty(sz.workspace_bytes, dtype=torch.uint8, device=device)
+        self.c = rad_store(VARIANTS[variant], DTYPES[dtype], B, D, p, layer, step, seed,
+                           self.values.data_ptr(), int(cap), int(ld), self.keepbits.data_ptr(),
+                           self.offsets.data_ptr(), self.nnz.data_ptr(),
+                           self.relubits.data_ptr() if relu_bits else None)
+
+    def held_bytes(self):
+        """Bytes this store holds between forward and backward (values as reserved, indices, ReLU bits)."""
+        es = self.values.element_size()
+        return dict(value_bytes=int(self.c.values_capacity) * es,
+                    index_bytes=(self.keepbits.numel() + self.offsets.numel()) * 4,
+                    relu_bytes=0 if self.relubits is None else self.relubits.numel() * 4)
+
+
+def rad_linear_forward_store(A, store, dev_status=None):
+    _check(lib().rad_linear_forward_store(_ptr(A), A.stride(0), C.byref(store.c), _ptr(store.workspace),
+                                          store.workspace.numel(), _ptr(dev_status), _stream()),
+           "rad_linear_forward_store")
+
+
+def rad_weight_grad_workspace(store, H):
+    out = C.c_int64(0)
+    _check(lib().rad_weight_grad_workspace(C.byref(store.c), H, C.byref(out)), "rad_weight_grad_workspace")
+    return out.value
+
+
+def rad_linear_weight_grad(store, dZ, dW, workspace=None, dev_status=None):
+    H = dZ.shape[1]
+    if workspace is None:
+        workspace = torch.empty(max(rad_weight_grad_workspace(store, H), 256), dtype=torch.uint8, device=dZ.device)
+    _check(lib().rad_linear_weight_grad(C.byref(store.c), _ptr(dZ), dZ.stride(0), H, _ptr(dW), dW.stride(0),
+                                        _ptr(workspace), workspace.numel(), _ptr(dev_status), _stream()),
+           "rad_linear_weight_grad")
+    return dW
+
+
+def rad_linear_forward(A, W, bias, act, out_act=None, out_z=None, out_zlow=None, relubits=None, dev_status=None):
+    B, D = A.shape
+    H = W.shape[1]
+    _check(lib().rad_linear_forward(DTYPES[A.dtype], ACTS[act], B, D, H, _ptr(A), A.stride(0), _ptr(W),
+                                    W.stride(0), _ptr(bias), _ptr(out_act), _ld(out_act), _ptr(out_z),
+                                    _ld(out_z), _ptr(out_zlow), _ld(out_zlow), _ptr(relubits),
+                                    _ptr(dev_status), _stream()), "rad_linear_forward")
+
+
+def rad_softmax_xent(logits, labels, loss, dZ, workspace=None):
+    B, Cn = logits.shape
+    if workspace is None:
+        workspace = torch.empty(B * 4, dtype=torch.uint8, device=logits.device)
+    _check(lib().rad_softmax_xent(DTYPES[dZ.dtype], B, Cn, _ptr(logits), logits.stride(0), _ptr(labels),
+                                  _ptr(loss), _ptr(dZ), dZ.stride(0), _ptr(workspace), workspace.numel(),
+                                  _stream()), "rad_softmax_xent")
+
+
+def rad_input_grad_workspace(B, H):
+    out = C.c_int64(0)
+    _check(lib().rad_input_grad_workspace(B, H, C.byref(out)), "rad_input_grad_workspace")
+    return out.value
+
+
+def rad_linear_input_grad(dZ, W, relubits_prev=None, z_prev=None, dZ_prev=None, db=None, workspace=None,
+                          dev_status=None):
+    B, H = dZ.shape
+    D = W.shape[0]
+    if workspace is None:
+        workspace = torch.empty(rad_input_grad_workspace(B, H), dtype=torch.uint8, device=dZ.device)
+    _check(lib().rad_linear_input_grad(DTYPES[dZ.dtype], B, D, H, _ptr(dZ), dZ.stride(0), _ptr(W), W.stride(0),
+                                       _ptr(relubits_prev), _ptr(z_prev), _ld(z_prev), _ptr(dZ_prev),
+                                       _ld(dZ_prev), _ptr(db), _ptr(workspace), workspace.numel(),
+                                       _ptr(dev_status), _stream()), "rad_linear_input_grad")
+
+
+class MLPStep:
+    """Owns the workspace and pointer tables of rad_mlp_step for one net shape."""
+
+    def __init__(self, dims, B, dtype="f32", act="relu", variant="different", p=0.1, device="cuda"):
+        self.dims, self.B, self.L = list(dims), B, len(dims) - 1
+        self._dims = (C.c_int64 * len(dims))(*dims)
+        self.desc = rad_mlp_desc(self.L, ACTS[act], DTYPES[dtype], VARIANTS[variant], self._dims, B, p, 0, 0)
+        nbytes = C.c_int64(0)
+        self.stats = rad_step_stats()
+        _check(lib().rad_mlp_workspace(C.byref(self.desc), C.byref(nbytes), C.byref(self.stats)),
+               "rad_mlp_workspace")
+        self.workspace = torch.empty(nbytes.value, dtype=torch.uint8, device=device)
+        self.dW = [torch.empty(dims[l], dims[l + 1], dtype=torch.float32, device=device) for l in range(self.L)]
+        self.db = [torch.empty(dims[l + 1], dtype=torch.float32, device=device) for l in range(self.L)]
+        self.loss = torch.zeros(1, dtype=torch.float32, device=device)
+        self.nnz = torch.zeros(2 * self.L, dtype=torch.int64, device=device)
+        self.dev_status = torch.zeros(1, dtype=torch.int32, device=device)
+        arr = C.c_void_p * self.L
+        self._dW = arr(*[t.data_ptr() for t in self.dW])
+        self._db = arr(*[t.data_ptr() for t in self.db])
+
+    def __call__(self, X, labels, Ws, bs, seed=0, step=0):
+        return rad_mlp_step(self, X, labels, Ws, bs, seed, step)
+
+
+def rad_mlp_step(ctx, X, labels, Ws, bs, seed=0, step=0):
+    ctx.desc.seed, ctx.desc.step = seed, step
+    arr = C.c_void_p * ctx.L
+    W = arr(*[w.data_ptr() for w in Ws])
+    b = arr(*[(None if t is None else t.data_ptr()) for t in bs])
+    _check(lib().rad_mlp_step(C.byref(ctx.desc), _ptr(X), _ptr(labels), W, b, ctx._dW, ctx._db,
+                              _ptr(ctx.loss), _ptr(ctx.nnz), _ptr(ctx.workspace), ctx.workspace.numel(),
+                              _ptr(ctx.dev_status), _stream()), "rad_mlp_step")
+    return ctx

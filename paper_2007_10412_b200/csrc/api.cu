@@ -1,0 +1,270 @@
+// C ABI entry points that route to the kernels, and the whole-net step (Sec. 4.2 for arbitrary
+// depth: every layer input is stored through its own mask, dW_l comes from store l, the rest of
+// backprop is exact).
+#include "common.cuh"
+
+namespace rad {
+
+int check_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return RAD_ECUDA;
+  static int cached_dev = -1, cached_rc = RAD_ECUDA;
+  if (dev == cached_dev) return cached_rc;
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return RAD_ECUDA;
+  cached_rc = (major == 10) ? RAD_OK : RAD_EUNSUPPORTED;
+  cached_dev = dev;
+  return cached_rc;
+}
+
+namespace {
+
+bool valid_dtype(int d) { return d == RAD_F32 || d == RAD_BF16; }
+int64_t esize(int dtype) { return dtype == RAD_BF16 ? 2 : 4; }
+
+bool store_args_ok(const rad_store* st) {
+  if (st == nullptr || st->B <= 0 || st->D <= 0) return false;
+  if (st->variant != RAD_DIFFERENT_SAMPLE && st->variant != RAD_SAME_SAMPLE) return false;
+  if (!valid_dtype(st->dtype)) return false;
+  if (st->values == nullptr || st->keepbits == nullptr || st->offsets == nullptr || st->nnz == nullptr) return false;
+  if (keep_threshold_host(st->p) == 0) return false;
+  if (st->variant == RAD_SAME_SAMPLE && (st->values_ld <= 0 || st->values_ld % 8 != 0)) return false;
+  return true;
+}
+
+// ---- workspace plan of rad_mlp_step ---------------------------------------------------------------
+struct LayerPlan {
+  int64_t values, keepbits, offsets, nnz, relubits, preact;   // byte offsets; -1 if absent
+  int64_t capacity, values_ld;
+};
+struct StepPlan {
+  LayerPlan layer[64];
+  int64_t act[2], dz[2], logits, scratch, status_unused;
+  int64_t scratch_bytes, total;
+  rad_step_stats stats;
+};
+
+int make_plan(const rad_mlp_desc* net, StepPlan* plan) {
+  if (net == nullptr || net->dims == nullptr || net->L < 1 || net->L > 64 || net->B <= 0) return RAD_EINVAL;
+  if (!valid_dtype(net->dtype)) return RAD_EINVAL;
+  if (net->variant != RAD_DIFFERENT_SAMPLE && net->variant != RAD_SAME_SAMPLE) return RAD_EINVAL;
+  if (net->act != RAD_ACT_RELU && net->act != RAD_ACT_GELU) return RAD_EINVAL;
+  if (keep_threshold_host(net->p) == 0) return RAD_EINVAL;
+  const int64_t B = net->B, es = esize(net->dtype);
+  int64_t off = 0;
+  auto take = [&](int64_t bytes) { const int64_t at = off; off += round_up(bytes, 256); return at; };
+  rad_step_stats st = {};
+  int64_t max_hidden = 8, max_out = 8, scratch = B * 4;
+  for (int l = 0; l < net->L; ++l) {
+    const int64_t D = net->dims[l], H = net->dims[l + 1];
+    if (D <= 0 || H <= 0) return RAD_EINVAL;
+    rad_store_sizes sz;
+    int rc = rad_store_size_query(net->variant, net->dtype, B, D, net->p, &sz);
+    if (rc != RAD_OK) return rc;
+    LayerPlan& lp = plan->layer[l];
+    lp.capacity = sz.values_typical;
+    lp.values_ld = sz.values_ld_typical;
+    lp.values = take(lp.capacity * es);
+    lp.keepbits = take(sz.keepbits_words * 4);
+    lp.offsets = take(sz.offsets_words * 4);
+    lp.nnz = take(16);
+    lp.relubits = (l > 0 && net->act == RAD_ACT_RELU) ? take(sz.relubits_words * 4) : -1;
+    lp.preact = (l > 0 && net->act == RAD_ACT_GELU) ? take(B * D * es) : -1;
+    st.value_bytes += lp.capacity * es;
+    st.index_bytes += (sz.keepbits_words + sz.offsets_words) * 4;
+    if (lp.relubits >= 0) st.relu_bytes += sz.relubits_words * 4;
+    if (lp.preact >= 0) st.preact_bytes += B * D * es;
+    st.full_backprop_bytes += B * D * es;
+    if (l > 0) max_hidden = max(max_hidden, D);
+    max_out = max(max_out, H);
+    scratch = max(scratch, sz.workspace_bytes);
+    scratch = max(scratch, column_sums_workspace(B, H));
+    rad_store tmp = {};
+    tmp.variant = net->variant; tmp.dtype = net->dtype; tmp.B = B; tmp.D = D; tmp.p = net->p;
+    tmp.values_ld = lp.values_ld; tmp.values_capacity = lp.capacity;
+    scratch = max(scratch, tc_weight_grad_workspace(&tmp, H));
+  }
+  st.unsampled_bytes = B * net->dims[net->L] * 4;
+  st.full_backprop_bytes += st.unsampled_bytes;
+  plan->act[0] = take(B * max_hidden * es);
+  plan->act[1] = take(B * max_hidden * es);
+  plan->dz[0] = take(B * max_out * es);
+  plan->dz[1] = take(B * max_out * es);
+  plan->logits = take(B * net->dims[net->L] * 4);
+  plan->scratch_bytes = round_up(scratch, 256);
+  plan->scratch = take(plan->scratch_bytes);
+  plan->total = off;
+  plan->stats = st;
+  return RAD_OK;
+}
+
+}  // namespace
+}  // namespace rad
+
+using namespace rad;
+
+extern "C" const char* rad_version(void) { return "rad-b200 0.1 (sm_100a)"; }
+
+extern "C" const char* rad_strerror(int code) {
+  switch (code) {
+    case RAD_OK: return "ok";
+    case RAD_EINVAL: return "invalid argument";
+    case RAD_EUNSUPPORTED: return "unsupported device or alignment";
+    case RAD_ECUDA: return "CUDA call failed";
+    case RAD_EWORKSPACE: return "workspace too small";
+    case RAD_DEV_ECAPACITY: return "device: compact store capacity exceeded";
+    case RAD_DEV_ETIMEOUT: return "device: bounded wait expired";
+    default: return "unknown code";
+  }
+}
+
+extern "C" int rad_weight_grad_workspace(const rad_store* st, int64_t H, int64_t* bytes) {
+  if (st == nullptr || bytes == nullptr || H <= 0 || st->B <= 0 || st->D <= 0) return RAD_EINVAL;
+  *bytes = round_up(tc_weight_grad_workspace(st, H), 256);
+  return RAD_OK;
+}
+
+extern "C" int rad_linear_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H, float* dW,
+                                      int64_t ldw, void* workspace, int64_t workspace_bytes,
+                                      int32_t* dev_status, void* stream) {
+  if (!store_args_ok(st) || dZ == nullptr || dW == nullptr || H <= 0 || ldz < H || ldw < H) return RAD_EINVAL;
+  int rc = check_device();
+  if (rc != RAD_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (st->dtype == RAD_BF16 && tc_shape_ok(st->B, st->D, H, dZ, ldz, st->values, 8) &&
+      ((uintptr_t)dW & 15) == 0 && ldw % 4 == 0) {
+    if (workspace_bytes < tc_weight_grad_workspace(st, H) || (workspace == nullptr && tc_weight_grad_workspace(st, H) > 0))
+      return RAD_EWORKSPACE;
+    return tc_weight_grad(st, dZ, ldz, H, dW, ldw, workspace, workspace_bytes, dev_status, s);
+  }
+  return simt_weight_grad(st, dZ, ldz, H, dW, ldw, dev_status, s);
+}
+
+extern "C" int rad_linear_forward(int32_t dtype, int32_t act, int64_t B, int64_t D, int64_t H, const void* A,
+                                  int64_t lda, const void* W, int64_t ldw, const float* bias, void* out_act,
+                                  int64_t ld_act, float* out_z, int64_t ld_z, void* out_zlow, int64_t ld_zlow,
+                                  uint32_t* relubits, int32_t* dev_status, void* stream) {
+  if (!valid_dtype(dtype) || B <= 0 || D <= 0 || H <= 0 || A == nullptr || W == nullptr) return RAD_EINVAL;
+  if (act != RAD_ACT_NONE && act != RAD_ACT_RELU && act != RAD_ACT_GELU) return RAD_EINVAL;
+  if (lda < D || ldw < H) return RAD_EINVAL;
+  if (out_act == nullptr && out_z == nullptr && out_zlow == nullptr) return RAD_EINVAL;
+  if ((out_act != nullptr && ld_act < H) || (out_z != nullptr && ld_z < H) || (out_zlow != nullptr && ld_zlow < H))
+    return RAD_EINVAL;
+  if (relubits != nullptr && out_act == nullptr) return RAD_EINVAL;
+  int rc = check_device();
+  if (rc != RAD_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (dtype == RAD_BF16 && tc_shape_ok(B, D, H, A, lda, W, ldw) &&
+      (out_act == nullptr || (((uintptr_t)out_act & 15) == 0 && ld_act % 8 == 0)) &&
+      (out_zlow == nullptr || (((uintptr_t)out_zlow & 15) == 0 && ld_zlow % 8 == 0)) &&
+      (out_z == nullptr || (((uintptr_t)out_z & 15) == 0 && ld_z % 4 == 0)))
+    return tc_forward(act, B, D, H, A, lda, W, ldw, bias, out_act, ld_act, out_z, ld_z, out_zlow, ld_zlow,
+                      relubits, dev_status, s);
+  return simt_forward(dtype, act, B, D, H, A, lda, W, ldw, bias, out_act, ld_act, out_z, ld_z, out_zlow,
+                      ld_zlow, relubits, s);
+}
+
+extern "C" int rad_input_grad_workspace(int64_t B, int64_t H, int64_t* bytes) {
+  if (bytes == nullptr || B <= 0 || H <= 0) return RAD_EINVAL;
+  *bytes = column_sums_workspace(B, H);
+  return RAD_OK;
+}
+
+extern "C" int rad_linear_input_grad(int32_t dtype, int64_t B, int64_t D, int64_t H, const void* dZ, int64_t ldz,
+                                     const void* W, int64_t ldw, const uint32_t* relubits_prev,
+                                     const void* z_prev, int64_t ld_zprev, void* dZ_prev, int64_t ldp,
+                                     float* db, void* workspace, int64_t workspace_bytes,
+                                     int32_t* dev_status, void* stream) {
+  if (!valid_dtype(dtype) || B <= 0 || D <= 0 || H <= 0 || dZ == nullptr || W == nullptr) return RAD_EINVAL;
+  if (ldz < H || ldw < H) return RAD_EINVAL;
+  if (dZ_prev == nullptr && db == nullptr) return RAD_EINVAL;
+  if (dZ_prev != nullptr && ldp < D) return RAD_EINVAL;
+  if (z_prev != nullptr && ld_zprev < D) return RAD_EINVAL;
+  int rc = check_device();
+  if (rc != RAD_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (db != nullptr) {
+    rc = column_sums(dtype, B, H, dZ, ldz, db, workspace, workspace_bytes, s);
+    if (rc != RAD_OK) return rc;
+  }
+  if (dZ_prev == nullptr) return RAD_OK;
+  if (dtype == RAD_BF16 && tc_shape_ok(B, D, H, dZ, ldz, W, ldw) && ((uintptr_t)dZ_prev & 15) == 0 &&
+      ldp % 8 == 0 && (z_prev == nullptr || (((uintptr_t)z_prev & 15) == 0 && ld_zprev % 8 == 0)))
+    return tc_input_grad(B, D, H, dZ, ldz, W, ldw, relubits_prev, z_prev, ld_zprev, dZ_prev, ldp, dev_status, s);
+  return simt_input_grad(dtype, B, D, H, dZ, ldz, W, ldw, relubits_prev, z_prev, ld_zprev, dZ_prev, ldp, s);
+}
+
+extern "C" int rad_mlp_workspace(const rad_mlp_desc* net, int64_t* bytes, rad_step_stats* stats) {
+  if (bytes == nullptr) return RAD_EINVAL;
+  StepPlan plan;
+  int rc = make_plan(net, &plan);
+  if (rc != RAD_OK) return rc;
+  *bytes = plan.total;
+  if (stats != nullptr) *stats = plan.stats;
+  return RAD_OK;
+}
+
+extern "C" int rad_mlp_step(const rad_mlp_desc* net, const void* X, const int32_t* labels, const void* const* W,
+                            const float* const* b, float* const* dW, float* const* db, float* loss,
+                            int64_t* nnz_out, void* workspace, int64_t workspace_bytes, int32_t* dev_status,
+                            void* stream) {
+  StepPlan plan;
+  int rc = make_plan(net, &plan);
+  if (rc != RAD_OK) return rc;
+  if (X == nullptr || labels == nullptr || W == nullptr || dW == nullptr || db == nullptr || loss == nullptr)
+    return RAD_EINVAL;
+  if (workspace == nullptr || workspace_bytes < plan.total) return RAD_EWORKSPACE;
+  if (((uintptr_t)workspace & 255) != 0) return RAD_EINVAL;
+  rc = check_device();
+  if (rc != RAD_OK) return rc;
+  char* ws = static_cast<char*>(workspace);
+  const int L = net->L;
+  const int64_t B = net->B;
+  rad_store st[64];
+  const void* a_in = X;
+  int64_t ld_in = net->dims[0];
+  for (int l = 0; l < L; ++l) {
+    const int64_t D = net->dims[l], H = net->dims[l + 1];
+    if (W[l] == nullptr || dW[l] == nullptr || db[l] == nullptr) return RAD_EINVAL;
+    const LayerPlan& lp = plan.layer[l];
+    rad_store& s = st[l];
+    s.variant = net->variant; s.dtype = net->dtype; s.B = B; s.D = D; s.p = net->p;
+    s.layer = (uint32_t)l; s.step = net->step; s.seed = net->seed;
+    s.values = ws + lp.values; s.values_capacity = lp.capacity; s.values_ld = lp.values_ld;
+    s.keepbits = reinterpret_cast<uint32_t*>(ws + lp.keepbits);
+    s.offsets = reinterpret_cast<uint32_t*>(ws + lp.offsets);
+    s.nnz = nnz_out != nullptr ? nnz_out + 2 * l : reinterpret_cast<int64_t*>(ws + lp.nnz);
+    s.relubits = lp.relubits >= 0 ? reinterpret_cast<uint32_t*>(ws + lp.relubits) : nullptr;
+    rc = rad_linear_forward_store(a_in, ld_in, &s, ws + plan.scratch, plan.scratch_bytes, dev_status, stream);
+    if (rc != RAD_OK) return rc;
+    const bool last = (l == L - 1);
+    void* a_out = last ? nullptr : ws + plan.act[l & 1];
+    // a GELU net keeps the pre-activation of layer l for the backward of layer l + 1's input
+    void* zlow = (!last && net->act == RAD_ACT_GELU) ? ws + plan.layer[l + 1].preact : nullptr;
+    rc = rad_linear_forward(net->dtype, last ? RAD_ACT_NONE : net->act, B, D, H, a_in, ld_in, W[l], H,
+                            b != nullptr ? b[l] : nullptr, a_out, H,
+                            last ? reinterpret_cast<float*>(ws + plan.logits) : nullptr, H, zlow, H, nullptr,
+                            dev_status, stream);
+    if (rc != RAD_OK) return rc;
+    a_in = a_out;
+    ld_in = H;
+  }
+  const int64_t C = net->dims[L];
+  void* dz = ws + plan.dz[(L - 1) & 1];
+  rc = rad_softmax_xent(net->dtype, B, C, reinterpret_cast<const float*>(ws + plan.logits), C, labels, loss, dz,
+                        C, ws + plan.scratch, plan.scratch_bytes, stream);
+  if (rc != RAD_OK) return rc;
+  for (int l = L - 1; l >= 0; --l) {
+    const int64_t D = net->dims[l], H = net->dims[l + 1];
+    rc = rad_linear_weight_grad(&st[l], dz, H, H, dW[l], H, ws + plan.scratch, plan.scratch_bytes, dev_status,
+                                stream);
+    if (rc != RAD_OK) return rc;
+    void* dz_prev = l > 0 ? ws + plan.dz[(l - 1) & 1] : nullptr;
+    rc = rad_linear_input_grad(net->dtype, B, D, H, dz, H, W[l], H, st[l].relubits,
+                               plan.layer[l].preact >= 0 ? ws + plan.layer[l].preact : nullptr, D, dz_prev, D,
+                               db[l], ws + plan.scratch, plan.scratch_bytes, dev_status, stream);
+    if (rc != RAD_OK) return rc;
+    dz = dz_prev;
+  }
+  return RAD_OK;
+}

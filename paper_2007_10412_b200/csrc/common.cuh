@@ -1,0 +1,149 @@
+// Shared device/host helpers of the RAD library (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/rad.h"
+
+#if defined(__CUDA_ARCH__) && (__CUDA_ARCH__ < 1000)
+#error "this library is written for sm_100a only"
+#endif
+
+namespace rad {
+
+typedef __nv_bfloat16 bf16;
+
+constexpr int kTileRows = RAD_TILE_ROWS;
+constexpr int kTileCols = RAD_TILE_COLS;
+constexpr int kTileWords = kTileRows * kTileCols / 32;   // 256 keep-bit words per tile
+constexpr int kValueAlign = RAD_VALUE_ALIGN;
+
+// ---------------------------------------------------------------------------------------------
+// Philox-4x32-10 (Salmon et al., SC'11): counter (c0..c3), key (k0,k1); per round the counter
+// becomes (hi(M1*c2)^c1^k0, lo(M1*c2), hi(M0*c0)^c3^k1, lo(M0*c0)); the key advances by the
+// Weyl constants between rounds.  The ten round keys depend on the seed only, so the host
+// expands them once and kernels take them by value.
+// ---------------------------------------------------------------------------------------------
+constexpr uint32_t kPhiloxM0 = 0xD2511F53u;
+constexpr uint32_t kPhiloxM1 = 0xCD9E8D57u;
+constexpr uint32_t kPhiloxW0 = 0x9E3779B9u;
+constexpr uint32_t kPhiloxW1 = 0xBB67AE85u;
+
+struct PhiloxKeys {
+  uint32_t k0[10];
+  uint32_t k1[10];
+};
+
+inline PhiloxKeys philox_expand_key(uint64_t seed) {
+  PhiloxKeys ks;
+  uint32_t a = (uint32_t)(seed & 0xffffffffu), b = (uint32_t)(seed >> 32);
+  for (int r = 0; r < 10; ++r) {
+    ks.k0[r] = a;
+    ks.k1[r] = b;
+    a += kPhiloxW0;
+    b += kPhiloxW1;
+  }
+  return ks;
+}
+
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                              const PhiloxKeys& ks, uint32_t out[4]) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint64_t p0 = (uint64_t)kPhiloxM0 * c0;
+    const uint64_t p1 = (uint64_t)kPhiloxM1 * c2;
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ ks.k0[r];
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ ks.k1[r];
+    c1 = (uint32_t)p1;
+    c3 = (uint32_t)p0;
+    c0 = n0;
+    c2 = n2;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// Keep bits of the 8 columns of one counter: bit i set iff the 16-bit lane of column i is < T.
+__device__ __forceinline__ uint32_t philox_keep8(uint32_t group, uint32_t row, uint32_t c2, uint32_t c3,
+                                                 const PhiloxKeys& ks, uint32_t T) {
+  uint32_t w[4];
+  philox4x32_10(group, row, c2, c3, ks, w);
+  uint32_t m = 0;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    m |= ((w[j] & 0xffffu) < T ? 1u : 0u) << (2 * j);
+    m |= ((w[j] >> 16) < T ? 1u : 0u) << (2 * j + 1);
+  }
+  return m;
+}
+
+// Host-side twins of the threshold arithmetic (double rint, one float32 division).
+uint32_t keep_threshold_host(float p);
+inline uint32_t counter_word2(uint32_t layer, int variant) {
+  return (layer & 0xffffffu) | ((variant == RAD_SAME_SAMPLE ? 1u : 0u) << 24);
+}
+
+// ---------------------------------------------------------------------------------------------
+// element access
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float to_float(float v) { return v; }
+__device__ __forceinline__ float to_float(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_float(float v);
+template <> __device__ __forceinline__ float from_float<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_float<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ void raise_status(int32_t* dev_status, int32_t code) {
+  if (dev_status != nullptr) atomicCAS(dev_status, 0, code);
+}
+
+__device__ __forceinline__ float gelu_f(float z) {
+  return 0.5f * z * (1.0f + erff(z * 0.70710678118654752440f));
+}
+__device__ __forceinline__ float gelu_grad_f(float z) {
+  return 0.5f * (1.0f + erff(z * 0.70710678118654752440f)) +
+         z * 0.39894228040143267794f * __expf(-0.5f * z * z);
+}
+
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+inline int64_t round_up(int64_t a, int64_t b) { return ceil_div(a, b) * b; }
+
+#define RAD_CUDA_TRY(expr)                          \
+  do {                                              \
+    cudaError_t e__ = (expr);                       \
+    if (e__ != cudaSuccess) return RAD_ECUDA;       \
+  } while (0)
+
+// internal launchers shared across translation units --------------------------------------------
+int check_device();   // RAD_OK on an sm_100 device
+
+// f32/bf16 CUDA-core kernels (small or unaligned problems)
+int simt_forward(int dtype, int act, int64_t B, int64_t D, int64_t H, const void* A, int64_t lda,
+                 const void* W, int64_t ldw, const float* bias, void* out_act, int64_t ld_act,
+                 float* out_z, int64_t ld_z, void* out_zlow, int64_t ld_zlow, uint32_t* relubits,
+                 cudaStream_t s);
+int simt_input_grad(int dtype, int64_t B, int64_t D, int64_t H, const void* dZ, int64_t ldz,
+                    const void* W, int64_t ldw, const uint32_t* relubits_prev, const void* z_prev,
+                    int64_t ld_zprev, void* dZ_prev, int64_t ldp, cudaStream_t s);
+int simt_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H, float* dW,
+                     int64_t ldw, int32_t* dev_status, cudaStream_t s);
+int column_sums(int dtype, int64_t B, int64_t H, const void* dZ, int64_t ldz, float* db,
+                void* workspace, int64_t workspace_bytes, cudaStream_t s);
+int64_t column_sums_workspace(int64_t B, int64_t H);
+
+// tcgen05 kernels (bf16, aligned)
+bool tc_shape_ok(int64_t B, int64_t D, int64_t H, const void* p0, int64_t ld0, const void* p1,
+                 int64_t ld1);
+int tc_forward(int act, int64_t B, int64_t D, int64_t H, const void* A, int64_t lda, const void* W,
+               int64_t ldw, const float* bias, void* out_act, int64_t ld_act, float* out_z,
+               int64_t ld_z, void* out_zlow, int64_t ld_zlow, uint32_t* relubits,
+               int32_t* dev_status, cudaStream_t s);
+int tc_input_grad(int64_t B, int64_t D, int64_t H, const void* dZ, int64_t ldz, const void* W,
+                  int64_t ldw, const uint32_t* relubits_prev, const void* z_prev, int64_t ld_zprev,
+                  void* dZ_prev, int64_t ldp, int32_t* dev_status, cudaStream_t s);
+int tc_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H, float* dW,
+                   int64_t ldw, void* workspace, int64_t workspace_bytes, int32_t* dev_status,
+                   cudaStream_t s);
+int64_t tc_weight_grad_workspace(const rad_store* st, int64_t H);
+
+}  // namespace rad

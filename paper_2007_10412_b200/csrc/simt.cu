@@ -1,0 +1,335 @@
+// CUDA-core (FFMA) kernels: the float32 nets, whose 1e-5 tolerance rules out tensor-core input
+// rounding, and bf16 problems whose shapes the TMA path cannot take.  These problems are small
+// and latency-bound; the kernels favour exact float32 accumulation in a fixed order over speed.
+#include <algorithm>
+#include <cmath>
+
+#include "common.cuh"
+
+namespace rad {
+namespace {
+
+constexpr int kBM = 64, kBN = 64, kBK = 16;
+
+enum Epilogue { kEpiForward = 0, kEpiInputGrad = 1, kEpiScatterRows = 2 };
+
+struct GemmParams {
+  // C(m, n) = sum_k A(m, k) * Bm(k, n); element (m, k) of A at A[m * sam + k * sak], etc.
+  const void* A; int64_t sam, sak;
+  const void* Bm; int64_t sbk, sbn;
+  int64_t M, N, K;
+  const int64_t* M_dev;        // optional: M read from device memory (clamped to M)
+  // forward epilogue
+  const float* bias; int act;
+  void* out_act; int64_t ld_act;
+  float* out_z; int64_t ld_z;
+  void* out_zlow; int64_t ld_zlow;
+  // input-grad epilogue
+  const uint32_t* relubits; int64_t w32;
+  const void* z_prev; int64_t ld_zprev;
+  void* out_low; int64_t ld_low;
+  // scatter-rows epilogue (same-sample dW): row m goes to row idx[m] of out_f32
+  const uint32_t* row_idx;
+  float* out_f32; int64_t ld_f32;
+};
+
+template <typename T, int EPI>
+__global__ void __launch_bounds__(256) gemm_kernel(const GemmParams p) {
+  __shared__ float sA[kBK][kBM + 4];
+  __shared__ float sB[kBK][kBN + 4];
+  int64_t M = p.M;
+  if (p.M_dev != nullptr) M = min(M, *p.M_dev);
+  const int64_t m0 = (int64_t)blockIdx.y * kBM, n0 = (int64_t)blockIdx.x * kBN;
+  if (m0 >= M) return;
+  const int tid = threadIdx.x;
+  const int tm = (tid >> 4) * 4, tn = (tid & 15) * 4;
+  const T* A = static_cast<const T*>(p.A);
+  const T* Bm = static_cast<const T*>(p.Bm);
+  float acc[4][4] = {};
+  for (int64_t k0 = 0; k0 < p.K; k0 += kBK) {
+    // 64 x 16 elements of each operand, 4 per thread; whichever index is contiguous in memory
+    // is made the fast thread index
+    for (int i = tid; i < kBM * kBK; i += 256) {
+      int mm, kk;
+      if (p.sak == 1) { kk = i % kBK; mm = i / kBK; } else { mm = i % kBM; kk = i / kBM; }
+      const int64_t m = m0 + mm, k = k0 + kk;
+      sA[kk][mm] = (m < M && k < p.K) ? to_float(A[m * p.sam + k * p.sak]) : 0.0f;
+    }
+    for (int i = tid; i < kBN * kBK; i += 256) {
+      int nn, kk;
+      if (p.sbk == 1) { kk = i % kBK; nn = i / kBK; } else { nn = i % kBN; kk = i / kBN; }
+      const int64_t n = n0 + nn, k = k0 + kk;
+      sB[kk][nn] = (n < p.N && k < p.K) ? to_float(Bm[k * p.sbk + n * p.sbn]) : 0.0f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < kBK; ++kk) {
+      float a[4], b[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { a[i] = sA[kk][tm + i]; b[i] = sB[kk][tn + i]; }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int64_t m = m0 + tm + i;
+    if (m >= M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int64_t n = n0 + tn + j;
+      if (n >= p.N) continue;
+      float v = acc[i][j];
+      if (EPI == kEpiForward) {
+        if (p.bias != nullptr) v += p.bias[n];
+        if (p.out_z != nullptr) p.out_z[m * p.ld_z + n] = v;
+        if (p.out_zlow != nullptr) static_cast<T*>(p.out_zlow)[m * p.ld_zlow + n] = from_float<T>(v);
+        if (p.out_act != nullptr) {
+          const float a = p.act == RAD_ACT_RELU ? fmaxf(v, 0.0f) : p.act == RAD_ACT_GELU ? gelu_f(v) : v;
+          static_cast<T*>(p.out_act)[m * p.ld_act + n] = from_float<T>(a);
+        }
+      } else if (EPI == kEpiInputGrad) {
+        if (p.relubits != nullptr) {
+          if (((p.relubits[m * p.w32 + (n >> 5)] >> (n & 31)) & 1u) == 0) v = 0.0f;
+        } else if (p.z_prev != nullptr) {
+          v *= gelu_grad_f(to_float(static_cast<const T*>(p.z_prev)[m * p.ld_zprev + n]));
+        }
+        static_cast<T*>(p.out_low)[m * p.ld_low + n] = from_float<T>(v);
+      } else {
+        p.out_f32[(int64_t)p.row_idx[m] * p.ld_f32 + n] = v;
+      }
+    }
+  }
+}
+
+template <int EPI>
+int launch_gemm(int dtype, const GemmParams& p, int64_t Mgrid, cudaStream_t s) {
+  dim3 grid((unsigned)ceil_div(p.N, kBN), (unsigned)ceil_div(Mgrid, kBM));
+  if (grid.x == 0 || grid.y == 0) return RAD_OK;
+  if (dtype == RAD_BF16)
+    gemm_kernel<bf16, EPI><<<grid, 256, 0, s>>>(p);
+  else
+    gemm_kernel<float, EPI><<<grid, 256, 0, s>>>(p);
+  return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
+}
+
+// relubits[b, w] = bits of (X[b, 32w..] > 0)
+template <typename T>
+__global__ void __launch_bounds__(256) relu_bits_rows_kernel(const T* X, int64_t ld, int64_t B, int64_t H,
+                                                             int64_t w32, uint32_t* out) {
+  const int64_t n = B * w32;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n;
+       i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t b = i / w32, w = i % w32;
+    const T* rowp = X + b * ld + w * 32;
+    const int nv = (int)min((int64_t)32, H - w * 32);
+    uint32_t m = 0;
+    for (int c = 0; c < nv; ++c) m |= (to_float(rowp[c]) > 0.0f ? 1u : 0u) << c;
+    out[i] = m;
+  }
+}
+
+// ---- different-sample dW on CUDA cores ----------------------------------------------------------
+// One CTA owns 128 columns d of the layer input (one column block) and 32 outputs h.  Per row slab
+// it rebuilds the 64 x 128 tile of A_hat in shared memory from keep bits and packed values
+// (per-word popcount prefix), then accumulates A_hat^T dZ.
+constexpr int kSparseBN = 32;
+struct SparseDwParams {
+  const void* values; const uint32_t* keepbits; const uint32_t* offsets;
+  int64_t capacity;
+  int64_t B, D, H; int32_t ncb, nslabs;
+  const void* dZ; int64_t ldz;
+  float* dW; int64_t ldw;
+};
+
+template <typename T>
+__global__ void __launch_bounds__(256) sparse_dw_kernel(const SparseDwParams p) {
+  __shared__ float sAh[kTileRows][kTileCols + 1];
+  __shared__ float sZ[kTileRows][kSparseBN + 1];
+  __shared__ uint32_t s_scan[256];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int cb = blockIdx.x;
+  const int64_t h0 = (int64_t)blockIdx.y * kSparseBN;
+  const T* vals = static_cast<const T*>(p.values);
+  const T* dZ = static_cast<const T*>(p.dZ);
+  // 128 x 32 outputs over 256 threads: 4 columns d x 4 outputs h each
+  const int td = (tid >> 3) * 4, th = (tid & 7) * 4;
+  float acc[4][4] = {};
+  for (int slab = 0; slab < p.nslabs; ++slab) {
+    const int64_t tile = (int64_t)slab * p.ncb + cb;
+    const uint32_t word = p.keepbits[tile * kTileWords + tid];    // row tid/4, word tid%4
+    const uint32_t cnt = __popc(word);
+    // exclusive scan of the 256 per-word counts
+    uint32_t incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t n = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += n;
+    }
+    if (lane == 31) s_scan[warp] = incl;
+    __syncthreads();
+    uint32_t wbase = 0;
+    for (int w = 0; w < warp; ++w) wbase += s_scan[w];
+    uint32_t pos = wbase + incl - cnt;
+    const int64_t base = p.offsets[tile];
+    const int r = tid >> 2, c0 = (tid & 3) * 32;
+#pragma unroll 4
+    for (int b = 0; b < 32; ++b) {
+      float v = 0.0f;
+      if ((word >> b) & 1u) {                       // a store that overflowed is never read past
+        const int64_t at = base + pos++;
+        if (at < p.capacity) v = to_float(vals[at]);
+      }
+      sAh[r][c0 + b] = v;
+    }
+    for (int i = tid; i < kTileRows * kSparseBN; i += 256) {
+      const int rr = i / kSparseBN, hh = i % kSparseBN;
+      const int64_t row = (int64_t)slab * kTileRows + rr, h = h0 + hh;
+      sZ[rr][hh] = (row < p.B && h < p.H) ? to_float(dZ[row * p.ldz + h]) : 0.0f;
+    }
+    __syncthreads();
+#pragma unroll 4
+    for (int rr = 0; rr < kTileRows; ++rr) {
+      float a[4], z[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) a[i] = sAh[rr][td + i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) z[j] = sZ[rr][th + j];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], z[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int64_t d = (int64_t)cb * kTileCols + td + i;
+    if (d >= p.D) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int64_t h = h0 + th + j;
+      if (h < p.H) p.dW[d * p.ldw + h] = acc[i][j];
+    }
+  }
+}
+
+__global__ void zero_rows_kernel(float* dW, int64_t ldw, int64_t D, int64_t H) {
+  const int64_t n = D * H;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n;
+       i += (int64_t)gridDim.x * blockDim.x)
+    dW[(i / H) * ldw + (i % H)] = 0.0f;
+}
+
+// ---- column sums (bias gradient), two fixed-order stages ------------------------------------------
+constexpr int kColChunkRows = 128;
+template <typename T>
+__global__ void __launch_bounds__(256) colsum_partial_kernel(const T* dZ, int64_t ldz, int64_t B, int64_t H,
+                                                             float* partial) {
+  const int64_t h = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (h >= H) return;
+  const int64_t b0 = (int64_t)blockIdx.y * kColChunkRows, b1 = min(B, b0 + kColChunkRows);
+  float s = 0.0f;
+  for (int64_t b = b0; b < b1; ++b) s += to_float(dZ[b * ldz + h]);
+  partial[(int64_t)blockIdx.y * H + h] = s;
+}
+__global__ void __launch_bounds__(256) colsum_final_kernel(const float* partial, int64_t chunks, int64_t H,
+                                                           float* db) {
+  const int64_t h = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (h >= H) return;
+  float s = 0.0f;
+  for (int64_t c = 0; c < chunks; ++c) s += partial[c * H + h];
+  db[h] = s;
+}
+
+}  // namespace
+
+int simt_forward(int dtype, int act, int64_t B, int64_t D, int64_t H, const void* A, int64_t lda,
+                 const void* W, int64_t ldw, const float* bias, void* out_act, int64_t ld_act,
+                 float* out_z, int64_t ld_z, void* out_zlow, int64_t ld_zlow, uint32_t* relubits,
+                 cudaStream_t s) {
+  GemmParams p = {};
+  p.A = A; p.sam = lda; p.sak = 1;
+  p.Bm = W; p.sbk = ldw; p.sbn = 1;
+  p.M = B; p.N = H; p.K = D;
+  p.bias = bias; p.act = act;
+  p.out_act = out_act; p.ld_act = ld_act; p.out_z = out_z; p.ld_z = ld_z;
+  p.out_zlow = out_zlow; p.ld_zlow = ld_zlow;
+  int rc = launch_gemm<kEpiForward>(dtype, p, B, s);
+  if (rc != RAD_OK) return rc;
+  if (relubits != nullptr) {
+    if (out_act == nullptr) return RAD_EINVAL;
+    const int64_t w32 = ceil_div(H, 32), n = B * w32;
+    const int g = (int)std::min<int64_t>(ceil_div(n, 256), 148 * 16);
+    if (dtype == RAD_BF16)
+      relu_bits_rows_kernel<bf16><<<g, 256, 0, s>>>(static_cast<const bf16*>(out_act), ld_act, B, H, w32, relubits);
+    else
+      relu_bits_rows_kernel<float><<<g, 256, 0, s>>>(static_cast<const float*>(out_act), ld_act, B, H, w32, relubits);
+    if (cudaGetLastError() != cudaSuccess) return RAD_ECUDA;
+  }
+  return RAD_OK;
+}
+
+int simt_input_grad(int dtype, int64_t B, int64_t D, int64_t H, const void* dZ, int64_t ldz,
+                    const void* W, int64_t ldw, const uint32_t* relubits_prev, const void* z_prev,
+                    int64_t ld_zprev, void* dZ_prev, int64_t ldp, cudaStream_t s) {
+  GemmParams p = {};
+  p.A = dZ; p.sam = ldz; p.sak = 1;          // (b, h)
+  p.Bm = W; p.sbk = 1; p.sbn = ldw;          // Bm(h, d) = W[d, h]
+  p.M = B; p.N = D; p.K = H;
+  p.relubits = relubits_prev; p.w32 = ceil_div(D, 32);
+  p.z_prev = z_prev; p.ld_zprev = ld_zprev;
+  p.out_low = dZ_prev; p.ld_low = ldp;
+  return launch_gemm<kEpiInputGrad>(dtype, p, B, s);
+}
+
+int simt_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H, float* dW,
+                     int64_t ldw, int32_t* dev_status, cudaStream_t s) {
+  (void)dev_status;
+  if (st->variant == RAD_SAME_SAMPLE) {
+    const int g = (int)std::min<int64_t>(ceil_div(st->D * H, 256), 148 * 16);
+    zero_rows_kernel<<<g, 256, 0, s>>>(dW, ldw, st->D, H);
+    GemmParams p = {};
+    p.A = st->values; p.sam = 1; p.sak = st->values_ld;     // A(j, b) = values[b, j]
+    p.Bm = dZ; p.sbk = ldz; p.sbn = 1;
+    p.M = min(st->values_ld, st->D); p.N = H; p.K = st->B;
+    p.M_dev = st->nnz;
+    p.row_idx = st->offsets; p.out_f32 = dW; p.ld_f32 = ldw;
+    return launch_gemm<kEpiScatterRows>(st->dtype, p, p.M, s);
+  }
+  SparseDwParams p;
+  p.values = st->values; p.keepbits = st->keepbits; p.offsets = st->offsets;
+  p.capacity = st->values_capacity;
+  p.B = st->B; p.D = st->D; p.H = H;
+  p.ncb = (int32_t)ceil_div(st->D, kTileCols); p.nslabs = (int32_t)ceil_div(st->B, kTileRows);
+  p.dZ = dZ; p.ldz = ldz; p.dW = dW; p.ldw = ldw;
+  dim3 grid((unsigned)p.ncb, (unsigned)ceil_div(H, kSparseBN));
+  if (st->dtype == RAD_BF16)
+    sparse_dw_kernel<bf16><<<grid, 256, 0, s>>>(p);
+  else
+    sparse_dw_kernel<float><<<grid, 256, 0, s>>>(p);
+  return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
+}
+
+int64_t column_sums_workspace(int64_t B, int64_t H) {
+  return round_up(ceil_div(B, kColChunkRows) * H * 4, 256);
+}
+
+int column_sums(int dtype, int64_t B, int64_t H, const void* dZ, int64_t ldz, float* db, void* workspace,
+                int64_t workspace_bytes, cudaStream_t s) {
+  if (workspace == nullptr || workspace_bytes < column_sums_workspace(B, H)) return RAD_EWORKSPACE;
+  const int64_t chunks = ceil_div(B, kColChunkRows);
+  dim3 grid((unsigned)ceil_div(H, 256), (unsigned)chunks);
+  float* partial = static_cast<float*>(workspace);
+  if (dtype == RAD_BF16)
+    colsum_partial_kernel<bf16><<<grid, 256, 0, s>>>(static_cast<const bf16*>(dZ), ldz, B, H, partial);
+  else
+    colsum_partial_kernel<float><<<grid, 256, 0, s>>>(static_cast<const float*>(dZ), ldz, B, H, partial);
+  colsum_final_kernel<<<(unsigned)ceil_div(H, 256), 256, 0, s>>>(partial, chunks, H, db);
+  return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
+}
+
+}  // namespace rad

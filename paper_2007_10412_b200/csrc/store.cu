@@ -1,0 +1,519 @@
+// Forward-pass store kernels: Philox keep mask, scale, compaction (Sec. 3.2 / 4.2 of the paper:
+// the layer input is what gets sampled, never the Jacobian itself).
+//
+// different-sample: one pass over A.  A CTA takes one 64 x 128 tile (ticket order), draws the
+// keep bits of its entries, counts them, and learns where its values start from a decoupled
+// look-back over the tiles before it (each tile publishes first its own count, then its
+// inclusive prefix, in a 64-bit status word).  Kept values are staged in shared memory in
+// (row, column) order and leave as 16-byte stores.  The order of tiles in `values` is fixed by the
+// tile index, so the layout does not depend on scheduling.
+//
+// same-sample: the column mask is drawn once (one CTA), then rows are gathered.
+#include <algorithm>
+#include <cmath>
+
+#include "common.cuh"
+
+namespace rad {
+
+uint32_t keep_threshold_host(float p) {
+  if (!(p > 0.0f) || !(p <= 1.0f)) return 0;
+  double t = rint((double)p * 65536.0);
+  if (t < 1.0) t = 1.0;
+  if (t > 65536.0) t = 65536.0;
+  return (uint32_t)t;
+}
+
+namespace {
+
+// ---- look-back status word ---------------------------------------------------------------------
+// bits 63..62 flag, 61..32 padded prefix in granules of 8 elements, 31..0 exact kept count.
+constexpr uint64_t kFlagShift = 62;
+constexpr uint64_t kFlagAggregate = 1, kFlagPrefix = 2, kFlagPoison = 3;
+constexpr uint64_t kValueMask = (1ull << kFlagShift) - 1;
+constexpr int kSpinLimit = 1 << 20;   // bounded wait: about a second with the back-off below
+
+__device__ __forceinline__ uint64_t pack_counts(uint32_t granules, uint32_t exact) {
+  return ((uint64_t)granules << 32) | exact;
+}
+__device__ __forceinline__ uint64_t load_status(const uint64_t* p) {
+  uint64_t v;
+  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void store_status(uint64_t* p, uint64_t v) {
+  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ uint64_t warp_sum_u64(uint64_t v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+struct StoreParams {
+  const void* A;
+  int64_t lda;
+  int64_t B, D;
+  int32_t ncb;        // column blocks
+  int32_t ntiles;
+  uint32_t T;         // keep threshold
+  float scale;
+  uint32_t c2, c3;    // counter words 2 and 3
+  void* values;
+  int64_t capacity;
+  uint32_t* keepbits;
+  uint32_t* offsets;
+  int64_t* nnz;
+  uint32_t* relubits;
+  int32_t w32;        // relu-bit words per row
+  uint64_t* status;   // ntiles look-back words (zeroed before launch)
+  uint32_t* ticket;   // zeroed before launch
+  int32_t* dev_status;
+  int32_t vec_ok;     // rows are 16-byte aligned: 8-element vector loads allowed
+};
+
+template <typename T> struct Raw8;   // eight consecutive elements of one row
+template <> struct Raw8<float> { float v[8]; };
+template <> struct Raw8<bf16> { uint4 q; };
+
+template <typename T>
+__device__ __forceinline__ void load8(const T* rowp, int64_t col0, int nvalid, bool vec, Raw8<T>& out);
+
+template <>
+__device__ __forceinline__ void load8<float>(const float* rowp, int64_t col0, int nvalid, bool vec,
+                                             Raw8<float>& out) {
+  if (vec && nvalid == 8) {
+    const float4 a = __ldcs(reinterpret_cast<const float4*>(rowp + col0));
+    const float4 b = __ldcs(reinterpret_cast<const float4*>(rowp + col0 + 4));
+    out.v[0] = a.x; out.v[1] = a.y; out.v[2] = a.z; out.v[3] = a.w;
+    out.v[4] = b.x; out.v[5] = b.y; out.v[6] = b.z; out.v[7] = b.w;
+  } else {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) out.v[i] = (i < nvalid) ? rowp[col0 + i] : 0.0f;
+  }
+}
+template <>
+__device__ __forceinline__ void load8<bf16>(const bf16* rowp, int64_t col0, int nvalid, bool vec,
+                                            Raw8<bf16>& out) {
+  if (vec && nvalid == 8) {
+    out.q = __ldcs(reinterpret_cast<const uint4*>(rowp + col0));
+  } else {
+    const unsigned short* p = reinterpret_cast<const unsigned short*>(rowp) + col0;
+    uint32_t w[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      if (i < nvalid) w[i >> 1] |= (uint32_t)p[i] << (16 * (i & 1));
+    out.q = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
+__device__ __forceinline__ float elem(const Raw8<float>& r, int i) { return r.v[i]; }
+__device__ __forceinline__ float elem(const Raw8<bf16>& r, int i) {
+  const uint32_t w = (i < 2) ? r.q.x : (i < 4) ? r.q.y : (i < 6) ? r.q.z : r.q.w;
+  return __uint_as_float((i & 1) ? (w & 0xffff0000u) : (w << 16));
+}
+
+// (a > 0) for the eight entries; zero of either sign gives 0.
+template <typename T> __device__ __forceinline__ uint32_t positive8(const Raw8<T>& r) {
+  uint32_t m = 0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) m |= (elem(r, i) > 0.0f ? 1u : 0u) << i;
+  return m;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) store_different_kernel(const StoreParams p, const PhiloxKeys ks) {
+  __shared__ uint32_t s_rowcnt[kTileRows];
+  __shared__ uint32_t s_rowoff[kTileRows];
+  __shared__ uint32_t s_tile;
+  __shared__ uint32_t s_total;
+  __shared__ int64_t s_base;        // first element of this tile in `values`, or -1: do not write
+  __shared__ __align__(16) T s_stage[kTileRows * kTileCols];
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) s_tile = atomicAdd(p.ticket, 1u);
+  __syncthreads();
+  const uint32_t tile = s_tile;
+  if (tile >= (uint32_t)p.ntiles) return;
+  const int64_t slab = tile / p.ncb;
+  const int cb = tile % p.ncb;
+  const int half = lane >> 4, cg = lane & 15;
+  const int64_t col0 = (int64_t)cb * kTileCols + cg * 8;
+  const int nvalid = (int)max((int64_t)0, min((int64_t)8, p.D - col0));
+  const T* Abase = static_cast<const T*>(p.A);
+
+  Raw8<T> raw[4];
+  uint32_t mask[4], pre[4];
+#pragma unroll
+  for (int it = 0; it < 4; ++it) {
+    const int r = warp * 8 + it * 2 + half;
+    const int64_t row = slab * kTileRows + r;
+    const bool live = (row < p.B) && (nvalid > 0);
+    uint32_t m = 0, rb = 0;
+    if (live) {
+      load8<T>(Abase + row * p.lda, col0, nvalid, p.vec_ok != 0, raw[it]);
+      m = philox_keep8((uint32_t)(col0 >> 3), (uint32_t)row, p.c2, p.c3, ks, p.T) & ((1u << nvalid) - 1u);
+      if (p.relubits != nullptr) rb = positive8(raw[it]) & ((1u << nvalid) - 1u);
+    }
+    mask[it] = m;
+    // exclusive prefix of the kept count inside the row (16 lanes per row)
+    const uint32_t c = __popc(m);
+    uint32_t incl = c;
+#pragma unroll
+    for (int o = 1; o < 16; o <<= 1) {
+      const uint32_t n = __shfl_up_sync(0xffffffffu, incl, o, 16);
+      if (cg >= o) incl += n;
+    }
+    pre[it] = incl - c;
+    if (cg == 15) s_rowcnt[r] = incl;
+    // four lanes make one 32-bit word of keep bits (and of ReLU bits)
+    uint32_t kw = m << (8 * (cg & 3));
+    kw |= __shfl_xor_sync(0xffffffffu, kw, 1);
+    kw |= __shfl_xor_sync(0xffffffffu, kw, 2);
+    uint32_t rw = rb << (8 * (cg & 3));
+    rw |= __shfl_xor_sync(0xffffffffu, rw, 1);
+    rw |= __shfl_xor_sync(0xffffffffu, rw, 2);
+    if ((cg & 3) == 0) {
+      p.keepbits[(int64_t)tile * kTileWords + r * 4 + (cg >> 2)] = kw;
+      const int word = cb * 4 + (cg >> 2);
+      if (p.relubits != nullptr && row < p.B && word < p.w32) p.relubits[row * p.w32 + word] = rw;
+    }
+  }
+  __syncthreads();
+
+  // row offsets inside the tile and the tile total (warp 0)
+  if (warp == 0) {
+    const uint32_t v0 = s_rowcnt[2 * lane], v1 = s_rowcnt[2 * lane + 1];
+    uint32_t incl = v0 + v1;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t n = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += n;
+    }
+    const uint32_t ex = incl - (v0 + v1);
+    s_rowoff[2 * lane] = ex;
+    s_rowoff[2 * lane + 1] = ex + v0;
+    const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
+    if (lane == 0) {
+      s_total = total;
+      const uint32_t gran = (total + kValueAlign - 1) / kValueAlign;
+      // the first tile knows its prefix at once; the others publish their own count first
+      store_status(p.status + tile, ((tile == 0 ? kFlagPrefix : kFlagAggregate) << kFlagShift) |
+                                        pack_counts(gran, total));
+    }
+  }
+  __syncthreads();
+
+  // stage the kept values of the tile in (row, column) order
+  const uint32_t total = s_total;
+  const uint32_t padded = (total + kValueAlign - 1) / kValueAlign * kValueAlign;
+#pragma unroll
+  for (int it = 0; it < 4; ++it) {
+    const int r = warp * 8 + it * 2 + half;
+    uint32_t pos = s_rowoff[r] + pre[it];
+    const uint32_t m = mask[it];
+    if (m != 0) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        if ((m >> i) & 1u) s_stage[pos++] = from_float<T>(elem(raw[it], i) * p.scale);
+    }
+  }
+  if (tid < (int)(padded - total)) s_stage[total + tid] = from_float<T>(0.0f);
+
+  // look-back (warp 0): sum the counts of earlier tiles until one with a known prefix is met
+  if (warp == 0) {
+    uint64_t excl = 0;
+    bool failed = false;
+    if (tile != 0) {
+      int64_t idx = (int64_t)tile - 1;
+      bool done = false;
+      while (!done) {
+        const int64_t j = idx - lane;
+        uint64_t w = kFlagPrefix << kFlagShift;          // before the first tile: prefix 0
+        if (j >= 0) {
+          int spins = 0;
+          w = load_status(p.status + j);
+          while ((w >> kFlagShift) == 0 && spins < kSpinLimit) {
+            __nanosleep(spins < 64 ? 32 : 256);
+            w = load_status(p.status + j);
+            ++spins;
+          }
+        }
+        const uint64_t flag = w >> kFlagShift;
+        if (__any_sync(0xffffffffu, flag == 0 || flag == kFlagPoison)) { failed = true; break; }
+        const uint32_t pm = __ballot_sync(0xffffffffu, flag == kFlagPrefix);
+        uint64_t contrib = w & kValueMask;
+        if (pm != 0) {
+          const int first = __ffs(pm) - 1;
+          if (lane > first) contrib = 0;
+          done = true;
+        }
+        excl += warp_sum_u64(contrib);
+        idx -= 32;
+      }
+    }
+    if (lane == 0) {
+      if (failed) {
+        store_status(p.status + tile, kFlagPoison << kFlagShift);   // later tiles stop waiting too
+        raise_status(p.dev_status, RAD_DEV_ETIMEOUT);
+        s_base = -1;
+      } else {
+        const uint64_t incl = excl + pack_counts(padded / kValueAlign, total);
+        if (tile != 0) store_status(p.status + tile, (kFlagPrefix << kFlagShift) | incl);
+        const int64_t base = (int64_t)(excl >> 32) * kValueAlign;
+        p.offsets[tile] = (uint32_t)base;
+        if (tile == (uint32_t)p.ntiles - 1) {
+          p.offsets[p.ntiles] = (uint32_t)((incl >> 32) * kValueAlign);
+          p.nnz[0] = (int64_t)(incl & 0xffffffffu);
+          p.nnz[1] = (int64_t)(incl >> 32) * kValueAlign;
+        }
+        if (base + padded > p.capacity) {
+          raise_status(p.dev_status, RAD_DEV_ECAPACITY);
+          s_base = -1;
+        } else {
+          s_base = base;
+        }
+      }
+    }
+  }
+  __syncthreads();
+  const int64_t base = s_base;
+  if (base < 0) return;
+  // 16-byte stores: base and padded are multiples of 8 elements
+  constexpr int kPerVec = 16 / (int)sizeof(T);
+  uint4* dst = reinterpret_cast<uint4*>(static_cast<T*>(p.values) + base);
+  const uint4* src = reinterpret_cast<const uint4*>(s_stage);
+  for (int i = tid; i < (int)(padded / kPerVec); i += 256) dst[i] = src[i];
+}
+
+// ---- same-sample ---------------------------------------------------------------------------------
+struct SameParams {
+  const void* A;
+  int64_t lda;
+  int64_t B, D;
+  uint32_t T;
+  float scale;
+  uint32_t c2, c3;
+  void* values;
+  int64_t ld;
+  uint32_t* keepbits;
+  uint32_t* idx;
+  int64_t* nnz;
+  int32_t* dev_status;
+};
+
+// One CTA draws the D column decisions and writes the ascending kept-column list.
+__global__ void __launch_bounds__(1024) same_mask_kernel(const SameParams p, const PhiloxKeys ks) {
+  __shared__ uint32_t s_warp[32];
+  __shared__ uint32_t s_running;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) s_running = 0;
+  __syncthreads();
+  const int64_t groups = (p.D + 7) / 8;
+  for (int64_t g0 = 0; g0 < groups; g0 += 1024) {
+    const int64_t g = g0 + tid;
+    uint32_t m = 0;
+    if (g < groups) {
+      const int nvalid = (int)min((int64_t)8, p.D - g * 8);
+      m = philox_keep8((uint32_t)g, 0u, p.c2, p.c3, ks, p.T) & ((1u << nvalid) - 1u);
+    }
+    uint32_t kw = m << (8 * (lane & 3));
+    kw |= __shfl_xor_sync(0xffffffffu, kw, 1);
+    kw |= __shfl_xor_sync(0xffffffffu, kw, 2);
+    if ((lane & 3) == 0 && g < groups) p.keepbits[g >> 2] = kw;
+    const uint32_t c = __popc(m);
+    uint32_t incl = c;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t n = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += n;
+    }
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      const uint32_t v = s_warp[lane];
+      uint32_t wi = v;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t n = __shfl_up_sync(0xffffffffu, wi, o);
+        if (lane >= o) wi += n;
+      }
+      s_warp[lane] = wi - v;
+    }
+    __syncthreads();
+    uint32_t pos = s_running + s_warp[warp] + incl - c;
+    for (int i = 0; i < 8; ++i)
+      if ((m >> i) & 1u) p.idx[pos++] = (uint32_t)(g * 8 + i);
+    __syncthreads();
+    if (tid == 1023) s_running = pos;   // last thread's end position is the running total
+    __syncthreads();
+  }
+  if (tid == 0) {
+    const int64_t k = s_running;
+    p.nnz[0] = k;
+    p.nnz[1] = k * p.B;
+    if (k > p.ld) raise_status(p.dev_status, RAD_DEV_ECAPACITY);
+  }
+}
+
+// values[b, j] = A[b, idx[j]] * scale for j < k', zero up to ld.  One warp per row at a time.
+template <typename T>
+__global__ void __launch_bounds__(256) same_gather_kernel(const SameParams p) {
+  const int64_t k = min(p.nnz[0], p.ld);
+  const int lane = threadIdx.x & 31;
+  const int64_t warp0 = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int64_t nwarps = (int64_t)gridDim.x * 8;
+  const T* A = static_cast<const T*>(p.A);
+  T* out = static_cast<T*>(p.values);
+  for (int64_t b = warp0; b < p.B; b += nwarps) {
+    const T* rowp = A + b * p.lda;
+    T* orow = out + b * p.ld;
+    for (int64_t j = lane; j < p.ld; j += 32) {
+      float v = 0.0f;
+      if (j < k) v = to_float(rowp[__ldg(p.idx + j)]) * p.scale;
+      orow[j] = from_float<T>(v);
+    }
+  }
+}
+
+// relubits[b, w] = bits of (A[b, 32w .. 32w+31] > 0).  One thread per output word.
+template <typename T>
+__global__ void __launch_bounds__(256) relu_bits_kernel(const T* A, int64_t lda, int64_t B, int64_t D,
+                                                        int64_t w32, uint32_t* out) {
+  const int64_t n = B * w32;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n;
+       i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t b = i / w32, w = i % w32;
+    const T* rowp = A + b * lda + w * 32;
+    const int nv = (int)min((int64_t)32, D - w * 32);
+    uint32_t m = 0;
+    for (int c = 0; c < nv; ++c) m |= (to_float(rowp[c]) > 0.0f ? 1u : 0u) << c;
+    out[i] = m;
+  }
+}
+
+int64_t store_workspace_bytes(int variant, int64_t B, int64_t D) {
+  if (variant == RAD_SAME_SAMPLE) return 256;
+  const int64_t ntiles = ceil_div(B, kTileRows) * ceil_div(D, kTileCols);
+  return round_up(ntiles * 8 + 256, 256);
+}
+
+}  // namespace
+}  // namespace rad
+
+using namespace rad;
+
+extern "C" uint32_t rad_keep_threshold(float p) { return keep_threshold_host(p); }
+extern "C" float rad_effective_p(float p) { return (float)keep_threshold_host(p) / 65536.0f; }
+extern "C" float rad_scale(float p) {
+  const uint32_t T = keep_threshold_host(p);
+  return T == 0 ? 0.0f : 65536.0f / (float)T;
+}
+
+extern "C" int rad_store_size_query(int32_t variant, int32_t dtype, int64_t B, int64_t D, float p,
+                                    rad_store_sizes* out) {
+  if (out == nullptr || B <= 0 || D <= 0) return RAD_EINVAL;
+  if (variant != RAD_DIFFERENT_SAMPLE && variant != RAD_SAME_SAMPLE) return RAD_EINVAL;
+  if (dtype != RAD_F32 && dtype != RAD_BF16) return RAD_EINVAL;
+  const uint32_t T = keep_threshold_host(p);
+  if (T == 0) return RAD_EINVAL;
+  if ((double)B * (double)D >= 4294967296.0 * 0.75) return RAD_EINVAL;   // 32-bit tile offsets
+  const double pe = T / 65536.0;
+  const int64_t w32 = ceil_div(D, 32);
+  out->relubits_words = B * w32;
+  if (variant == RAD_DIFFERENT_SAMPLE) {
+    const int64_t ntiles = ceil_div(B, kTileRows) * ceil_div(D, kTileCols);
+    const double n = (double)B * (double)D;
+    const int64_t pad = ntiles * (kValueAlign - 1);
+    out->values_worst = B * D + pad;
+    const double typ = n * pe + 8.0 * sqrt(n * pe * (1.0 - pe)) + 64.0;
+    out->values_typical = round_up((int64_t)fmin(typ, n) + pad, kValueAlign);
+    if (out->values_typical > out->values_worst) out->values_typical = out->values_worst;
+    out->values_ld_worst = out->values_ld_typical = 0;
+    out->keepbits_words = ntiles * kTileWords;
+    out->offsets_words = ntiles + 1;
+  } else {
+    const double n = (double)D;
+    const int64_t ldw = round_up(D, 64);
+    int64_t ldt = round_up((int64_t)(n * pe + 8.0 * sqrt(n * pe * (1.0 - pe)) + 8.0), 64);
+    if (ldt > ldw) ldt = ldw;
+    out->values_ld_worst = ldw;
+    out->values_ld_typical = ldt;
+    out->values_worst = B * ldw;
+    out->values_typical = B * ldt;
+    out->keepbits_words = w32;
+    out->offsets_words = D;
+  }
+  out->workspace_bytes = store_workspace_bytes(variant, B, D);
+  return RAD_OK;
+}
+
+extern "C" int rad_linear_forward_store(const void* A, int64_t lda, const rad_store* st, void* workspace,
+                                        int64_t workspace_bytes, int32_t* dev_status, void* stream) {
+  if (A == nullptr || st == nullptr) return RAD_EINVAL;
+  if (st->B <= 0 || st->D <= 0 || lda < st->D) return RAD_EINVAL;
+  if (st->variant != RAD_DIFFERENT_SAMPLE && st->variant != RAD_SAME_SAMPLE) return RAD_EINVAL;
+  if (st->dtype != RAD_F32 && st->dtype != RAD_BF16) return RAD_EINVAL;
+  if (st->values == nullptr || st->keepbits == nullptr || st->offsets == nullptr || st->nnz == nullptr)
+    return RAD_EINVAL;
+  const uint32_t T = keep_threshold_host(st->p);
+  if (T == 0) return RAD_EINVAL;
+  if ((double)st->B * (double)st->D >= 4294967296.0 * 0.75) return RAD_EINVAL;
+  if (((uintptr_t)st->values & 15) != 0) return RAD_EUNSUPPORTED;
+  int rc = check_device();
+  if (rc != RAD_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t esz = st->dtype == RAD_BF16 ? 2 : 4;
+  const PhiloxKeys ks = philox_expand_key(st->seed);
+  const int64_t w32 = ceil_div(st->D, 32);
+
+  if (st->variant == RAD_DIFFERENT_SAMPLE) {
+    const int64_t need = store_workspace_bytes(st->variant, st->B, st->D);
+    if (workspace == nullptr || workspace_bytes < need) return RAD_EWORKSPACE;
+    if (((uintptr_t)workspace & 7) != 0) return RAD_EINVAL;
+    StoreParams p;
+    p.A = A; p.lda = lda; p.B = st->B; p.D = st->D;
+    p.ncb = (int32_t)ceil_div(st->D, kTileCols);
+    p.ntiles = (int32_t)(ceil_div(st->B, kTileRows) * p.ncb);
+    p.T = T; p.scale = 65536.0f / (float)T;
+    p.c2 = counter_word2(st->layer, RAD_DIFFERENT_SAMPLE); p.c3 = st->step;
+    p.values = st->values; p.capacity = st->values_capacity;
+    p.keepbits = st->keepbits; p.offsets = st->offsets; p.nnz = st->nnz;
+    p.relubits = st->relubits; p.w32 = (int32_t)w32;
+    p.ticket = static_cast<uint32_t*>(workspace);
+    p.status = reinterpret_cast<uint64_t*>(static_cast<char*>(workspace) + 256);
+    p.dev_status = dev_status;
+    p.vec_ok = (((uintptr_t)A & 15) == 0 && (lda * esz) % 16 == 0) ? 1 : 0;
+    RAD_CUDA_TRY(cudaMemsetAsync(workspace, 0, (size_t)need, s));
+    if (st->dtype == RAD_BF16)
+      store_different_kernel<bf16><<<p.ntiles, 256, 0, s>>>(p, ks);
+    else
+      store_different_kernel<float><<<p.ntiles, 256, 0, s>>>(p, ks);
+    RAD_CUDA_TRY(cudaGetLastError());
+    return RAD_OK;
+  }
+
+  if (st->values_ld <= 0 || st->values_ld % 8 != 0 || st->values_capacity < st->B * st->values_ld)
+    return RAD_EINVAL;
+  SameParams p;
+  p.A = A; p.lda = lda; p.B = st->B; p.D = st->D; p.T = T; p.scale = 65536.0f / (float)T;
+  p.c2 = counter_word2(st->layer, RAD_SAME_SAMPLE); p.c3 = st->step;
+  p.values = st->values; p.ld = st->values_ld; p.keepbits = st->keepbits; p.idx = st->offsets;
+  p.nnz = st->nnz; p.dev_status = dev_status;
+  same_mask_kernel<<<1, 1024, 0, s>>>(p, ks);
+  const int grid = (int)std::min<int64_t>(ceil_div(st->B, 8), 148 * 8);
+  if (st->dtype == RAD_BF16)
+    same_gather_kernel<bf16><<<grid, 256, 0, s>>>(p);
+  else
+    same_gather_kernel<float><<<grid, 256, 0, s>>>(p);
+  if (st->relubits != nullptr) {
+    const int64_t n = st->B * w32;
+    const int g2 = (int)std::min<int64_t>(ceil_div(n, 256), 148 * 16);
+    if (st->dtype == RAD_BF16)
+      relu_bits_kernel<bf16><<<g2, 256, 0, s>>>(static_cast<const bf16*>(A), lda, st->B, st->D, w32, st->relubits);
+    else
+      relu_bits_kernel<float><<<g2, 256, 0, s>>>(static_cast<const float*>(A), lda, st->B, st->D, w32, st->relubits);
+  }
+  RAD_CUDA_TRY(cudaGetLastError());
+  return RAD_OK;
+}
