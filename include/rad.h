@@ -44,6 +44,7 @@ extern "C" {
 #define RAD_DEV_OK        0
 #define RAD_DEV_ECAPACITY 1    /* the compact store did not fit values_capacity / values_ld  */
 #define RAD_DEV_ETIMEOUT  2    /* a bounded device-side wait expired                         */
+#define RAD_DEV_EINTERNAL 3    /* an index left its buffer; the access was skipped (a bug)   */
 
 typedef enum { RAD_F32 = 0, RAD_BF16 = 1 } rad_dtype;
 typedef enum { RAD_DIFFERENT_SAMPLE = 0, RAD_SAME_SAMPLE = 1 } rad_variant;

@@ -114,6 +114,7 @@ extern "C" const char* rad_strerror(int code) {
     case RAD_EWORKSPACE: return "workspace too small";
     case RAD_DEV_ECAPACITY: return "device: compact store capacity exceeded";
     case RAD_DEV_ETIMEOUT: return "device: bounded wait expired";
+    case RAD_DEV_EINTERNAL: return "device: index out of range, access skipped";
     default: return "unknown code";
   }
 }
@@ -154,7 +155,7 @@ extern "C" int rad_linear_forward(int32_t dtype, int32_t act, int64_t B, int64_t
   int rc = check_device();
   if (rc != RAD_OK) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (dtype == RAD_BF16 && tc_shape_ok(B, D, H, A, lda, W, ldw) &&
+  if (dtype == RAD_BF16 && tc_shape_ok(B, D, H, A, lda, W, ldw) && ((uintptr_t)bias & 15) == 0 &&
       (out_act == nullptr || (((uintptr_t)out_act & 15) == 0 && ld_act % 8 == 0)) &&
       (out_zlow == nullptr || (((uintptr_t)out_zlow & 15) == 0 && ld_zlow % 8 == 0)) &&
       (out_z == nullptr || (((uintptr_t)out_z & 15) == 0 && ld_z % 4 == 0)))
@@ -234,16 +235,20 @@ extern "C" int rad_mlp_step(const rad_mlp_desc* net, const void* X, const int32_
     s.keepbits = reinterpret_cast<uint32_t*>(ws + lp.keepbits);
     s.offsets = reinterpret_cast<uint32_t*>(ws + lp.offsets);
     s.nnz = nnz_out != nullptr ? nnz_out + 2 * l : reinterpret_cast<int64_t*>(ws + lp.nnz);
-    s.relubits = lp.relubits >= 0 ? reinterpret_cast<uint32_t*>(ws + lp.relubits) : nullptr;
+    // the ReLU bits of this layer's input were written by the epilogue of the layer that produced it
+    s.relubits = nullptr;
     rc = rad_linear_forward_store(a_in, ld_in, &s, ws + plan.scratch, plan.scratch_bytes, dev_status, stream);
     if (rc != RAD_OK) return rc;
+    s.relubits = lp.relubits >= 0 ? reinterpret_cast<uint32_t*>(ws + lp.relubits) : nullptr;
     const bool last = (l == L - 1);
     void* a_out = last ? nullptr : ws + plan.act[l & 1];
     // a GELU net keeps the pre-activation of layer l for the backward of layer l + 1's input
     void* zlow = (!last && net->act == RAD_ACT_GELU) ? ws + plan.layer[l + 1].preact : nullptr;
     rc = rad_linear_forward(net->dtype, last ? RAD_ACT_NONE : net->act, B, D, H, a_in, ld_in, W[l], H,
                             b != nullptr ? b[l] : nullptr, a_out, H,
-                            last ? reinterpret_cast<float*>(ws + plan.logits) : nullptr, H, zlow, H, nullptr,
+                            last ? reinterpret_cast<float*>(ws + plan.logits) : nullptr, H, zlow, H,
+                            (!last && plan.layer[l + 1].relubits >= 0)
+                                ? reinterpret_cast<uint32_t*>(ws + plan.layer[l + 1].relubits) : nullptr,
                             dev_status, stream);
     if (rc != RAD_OK) return rc;
     a_in = a_out;

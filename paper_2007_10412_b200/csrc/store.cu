@@ -370,7 +370,11 @@ __global__ void __launch_bounds__(256) same_gather_kernel(const SameParams p) {
     T* orow = out + b * p.ld;
     for (int64_t j = lane; j < p.ld; j += 32) {
       float v = 0.0f;
-      if (j < k) v = to_float(rowp[__ldg(p.idx + j)]) * p.scale;
+      if (j < k) {
+        const uint32_t col = __ldg(p.idx + j);
+        if (col < (uint32_t)p.D) v = to_float(rowp[col]) * p.scale;
+        else raise_status(p.dev_status, RAD_DEV_EINTERNAL);
+      }
       orow[j] = from_float<T>(v);
     }
   }

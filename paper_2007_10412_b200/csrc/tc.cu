@@ -1,12 +1,768 @@
-// placeholder until the tcgen05 engine lands
+// tcgen05 GEMM engine (bf16 in, float32 accumulate in tensor memory) for the four contractions of
+// a RAD step on large aligned layers:
+//   forward      Z = A W + b                 (exact; Sec. 3: the forward pass is the original graph)
+//   input grad   dA = dZ W^T                 (exact; Sec. 4.2)
+//   dW, same     dW[idx, :] = A_c^T dZ       (column-compacted dense GEMM; Sec. 4.3 "same sample")
+//   dW, diff.    dW = A_hat^T dZ             (A_hat tiles rebuilt in shared memory from keep bits
+//                                             and packed values; Sec. 4.2 / 4.3 "different sample")
+//
+// One CTA per SM, persistent.  A CTA owns a 256 x 256 output tile held as two 128 x 256
+// accumulators that fill all 512 tensor-memory columns; per 64-deep K block it issues eight
+// 128x256x16 MMAs.  Operands arrive by TMA (128-byte swizzle, no multicast) through a 3-stage
+// mbarrier ring; for the different-sample dW the A operand is written by eight "expander" warps
+// instead.  Warp roles: 0 TMA producer, 1 MMA issuer and tensor-memory owner, 2-5 epilogue,
+// 6-13 expanders (sparse A only).  Long contractions can be split along K; partial tiles are
+// summed in split order by a second kernel, so results are reproducible.
+// Every mbarrier wait is bounded: on expiry the CTA raises RAD_DEV_ETIMEOUT, all roles leave
+// their loops, tensor memory is released and the kernel returns.
+#include <cuda.h>
+
+#include <algorithm>
+#include <cmath>
+
 #include "common.cuh"
+
 namespace rad {
-bool tc_shape_ok(int64_t, int64_t, int64_t, const void*, int64_t, const void*, int64_t) { return false; }
-int tc_forward(int, int64_t, int64_t, int64_t, const void*, int64_t, const void*, int64_t, const float*, void*,
-               int64_t, float*, int64_t, void*, int64_t, uint32_t*, int32_t*, cudaStream_t) { return RAD_EUNSUPPORTED; }
-int tc_input_grad(int64_t, int64_t, int64_t, const void*, int64_t, const void*, int64_t, const uint32_t*,
-                  const void*, int64_t, void*, int64_t, int32_t*, cudaStream_t) { return RAD_EUNSUPPORTED; }
-int tc_weight_grad(const rad_store*, const void*, int64_t, int64_t, float*, int64_t, void*, int64_t, int32_t*,
-                   cudaStream_t) { return RAD_EUNSUPPORTED; }
-int64_t tc_weight_grad_workspace(const rad_store*, int64_t) { return 0; }
+namespace {
+
+constexpr int BM = 256, BN = 256, BK = 64;
+constexpr int kHalfM = 128;
+constexpr int kAStageBytes = BM * BK * 2;      // 32 KB
+constexpr int kBStageBytes = BN * BK * 2;      // 32 KB
+constexpr int kNumSMsDefault = 148;
+constexpr int kMaxSplits = 16;
+constexpr int kRasterGroup = 8;                // m-tiles per raster group
+
+enum AKind { kAK = 0, kAMN = 1, kASparse = 2 };
+enum BKind { kBK_ = 0, kBMN = 1 };
+enum EpiKind { kFwd = 0, kDx = 1, kDw = 2 };
+
+struct TcParams {
+  int64_t M, N, K;
+  const int64_t* M_dev;      // same-sample dW: M = number of kept columns, read on the device
+  int32_t splits;            // K splits (1: epilogue writes final results)
+  int32_t num_stages;
+  // sparse A (different-sample store)
+  const bf16* values; const uint32_t* keepbits; const uint32_t* offsets;
+  int64_t values_capacity; int32_t ncb; int32_t comp_cap;   // comp_cap: value bytes per half-stage
+  // forward epilogue
+  const float* bias; int32_t act;
+  bf16* out_act; int64_t ld_act; float* out_z; int64_t ld_z; bf16* out_zlow; int64_t ld_zlow;
+  uint32_t* relubits; int64_t w32;
+  // input-grad epilogue
+  const uint32_t* relubits_prev; const bf16* z_prev; int64_t ld_zprev; bf16* out_dx; int64_t ld_dx;
+  // dW epilogue
+  float* out_dw; int64_t ld_dw; int64_t dw_rows; const uint32_t* row_idx; float* partial; int64_t partial_rows;
+  int32_t* dev_status;
+};
+
+// ---- PTX wrappers ---------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any legitimate wait here
+
+// Bounded wait.  Returns false if the CTA is aborting (this or another role timed out).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  while (true) {
+#pragma unroll 1
+    for (int i = 0; i < 32; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag != 0) return false;
+    if (global_timer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  K-major: rows of 64 elements (128 B), eight
+// rows form a 1024 B swizzle atom, SBO = 1024 B between atoms along M/N.  MN-major: rows of 64
+// M/N elements (one per K index), SBO = 1024 B between groups of eight K rows, LBO = distance to
+// the next 64 M/N elements.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
+         ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// Instruction descriptor: D = f32, A = B = bf16, M = 128, N = 256, operand major-ness as given.
+__host__ __device__ constexpr uint32_t make_idesc(bool a_mn, bool b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+         ((256u >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+// ---- work decomposition ---------------------------------------------------------------------------
+struct Unit {
+  int64_t m0, n0;
+  int32_t kb0, kb1;    // K blocks [kb0, kb1)
+  int32_t split;
+  int32_t halves;      // 1 or 2 active 128-row halves
+};
+
+struct Schedule {
+  int64_t M, m_tiles, n_tiles, ntiles, units;
+  int32_t kblocks, splits;
+  __device__ Schedule(int64_t M_, int64_t N_, int64_t K_, int32_t splits_) {
+    M = M_;
+    m_tiles = (M + BM - 1) / BM;
+    n_tiles = (N_ + BN - 1) / BN;
+    ntiles = m_tiles * n_tiles;
+    kblocks = (int32_t)((K_ + BK - 1) / BK);
+    splits = splits_;
+    units = ntiles * splits;
+  }
+  // split-major order: CTAs of one wave work on the same K range, so operand panels shared by
+  // tiles of a row or column of the grid are read from L2 at about the same time.
+  __device__ Unit unit(int64_t u) const {
+    Unit w;
+    const int64_t s = u / ntiles, t = u % ntiles;
+    const int64_t per_group = kRasterGroup * n_tiles;
+    const int64_t g = t / per_group, r = t % per_group;
+    const int64_t first_m = g * kRasterGroup;
+    const int64_t gm = min((int64_t)kRasterGroup, m_tiles - first_m);
+    w.m0 = (first_m + r % gm) * BM;
+    w.n0 = (r / gm) * BN;
+    w.split = (int32_t)s;
+    w.kb0 = (int32_t)(s * kblocks / splits);
+    w.kb1 = (int32_t)((s + 1) * kblocks / splits);
+    w.halves = (w.m0 + kHalfM < M) ? 2 : 1;
+    return w;
+  }
+};
+
+// ---- shared memory layout -------------------------------------------------------------------------
+struct SmemCtl {
+  uint64_t full[4], empty[4], comp_full[4], tmem_full, tmem_empty;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+template <int AK> __host__ __device__ constexpr int threads_for() { return AK == kASparse ? 448 : 192; }
+
+template <int AK, int BKIND, int EPI>
+__global__ void __launch_bounds__(threads_for<AK>(), 1)
+tc_gemm_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB) {
+  extern __shared__ uint8_t smem_raw[];
+  // 1024-byte alignment for the 128-byte swizzle atoms
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int stages = p.num_stages;
+  const int comp_half = (AK == kASparse) ? (1024 + p.comp_cap) : 0;          // bits + values of one half
+  const int stage_bytes = (kAStageBytes + kBStageBytes + 2 * comp_half + 1023) & ~1023;   // swizzle atoms need 1024 B
+  SmemCtl* ctl = reinterpret_cast<SmemCtl*>(smem + (size_t)stages * stage_bytes);
+  volatile int* abort_flag = &ctl->abort_flag;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // rows of the problem: for the same-sample dW the number of kept columns lives in device memory
+  int64_t m_rows = p.M;
+  if (p.M_dev != nullptr) {
+    int64_t md;
+    asm volatile("ld.global.cg.s64 %0, [%1];" : "=l"(md) : "l"(p.M_dev) : "memory");
+    m_rows = md < m_rows ? md : m_rows;
+  }
+  const Schedule sched(m_rows, p.N, p.K, p.splits);
+  if (tid == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(smem_u32(&ctl->full[s]), AK == kASparse ? 1 + 8 : 1);
+      mbar_init(smem_u32(&ctl->empty[s]), 1);
+      mbar_init(smem_u32(&ctl->comp_full[s]), 1);
+    }
+    mbar_init(smem_u32(&ctl->tmem_full), 1);
+    mbar_init(smem_u32(&ctl->tmem_empty), 128);
+    ctl->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {   // tensor memory: all 512 columns (two 128 x 256 float32 accumulators)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(&ctl->tmem_base)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = ctl->tmem_base;
+  const uint32_t smem_base = smem_u32(smem);
+
+  if (warp == 0) {
+    // ===== TMA producer (one lane issues; for sparse A all lanes prefetch tile offsets) =====
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int64_t u = blockIdx.x; u < sched.units && ok; u += gridDim.x) {
+      const Unit w = sched.unit(u);
+      uint32_t off_lo = 0, off_mid = 0, off_hi = 0;   // sparse: offsets of the 2 tiles of k-block (base + lane)
+      for (int kb = w.kb0; kb < w.kb1; ++kb) {
+        if (AK == kASparse && ((kb - w.kb0) & 31) == 0) {
+          const int kbl = kb + lane;
+          if (kbl < w.kb1) {
+            const int64_t cb0 = w.m0 / kTileCols;
+            const int64_t t0 = (int64_t)kbl * p.ncb + cb0;
+            off_lo = __ldg(p.offsets + t0);
+            off_mid = __ldg(p.offsets + t0 + 1);
+            off_hi = (w.halves == 2) ? __ldg(p.offsets + t0 + 2) : off_mid;
+          }
+        }
+        uint32_t o0 = 0, o1 = 0, o2 = 0;
+        if (AK == kASparse) {
+          const int src = (kb - w.kb0) & 31;
+          o0 = __shfl_sync(0xffffffffu, off_lo, src);
+          o1 = __shfl_sync(0xffffffffu, off_mid, src);
+          o2 = __shfl_sync(0xffffffffu, off_hi, src);
+        }
+        if (lane == 0) {
+          ok = mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag);
+          if (ok) {
+            const uint32_t sA = smem_base + stage * stage_bytes;
+            const uint32_t sB = sA + kAStageBytes;
+            const uint32_t full = smem_u32(&ctl->full[stage]);
+            const int k0 = kb * BK;
+            if (AK == kASparse) {
+              mbar_arrive_expect_tx(full, kBStageBytes);
+            } else {
+              mbar_arrive_expect_tx(full, kAStageBytes + kBStageBytes);
+              if (AK == kAK) {
+                tma_load_2d(sA, &tmA, k0, (int)w.m0, full);                       // 64 (K) x 256 rows
+              } else {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) tma_load_2d(sA + c * 8192, &tmA, (int)w.m0 + c * 64, k0, full);
+              }
+            }
+            if (BKIND == kBK_) {
+              tma_load_2d(sB, &tmB, k0, (int)w.n0, full);
+            } else {
+#pragma unroll
+              for (int c = 0; c < 4; ++c) tma_load_2d(sB + c * 8192, &tmB, (int)w.n0 + c * 64, k0, full);
+            }
+            if (AK == kASparse) {
+              // keep bits (1 KB per tile) and packed values of the one or two store tiles
+              const uint32_t cfull = smem_u32(&ctl->comp_full[stage]);
+              const uint32_t sC = sB + kBStageBytes;
+              const int64_t t0 = (int64_t)kb * p.ncb + w.m0 / kTileCols;
+              uint32_t vb0 = (o1 - o0) * 2u, vb1 = (o2 - o1) * 2u;
+              bool bad = false;
+              if (vb0 > (uint32_t)p.comp_cap || (int64_t)o1 > p.values_capacity) { vb0 = 0; bad = true; }
+              if (vb1 > (uint32_t)p.comp_cap || (int64_t)o2 > p.values_capacity) { vb1 = 0; bad = true; }
+              if (bad) raise_status(p.dev_status, RAD_DEV_ECAPACITY);
+              mbar_arrive_expect_tx(cfull, 1024u * w.halves + vb0 + (w.halves == 2 ? vb1 : 0u));
+              bulk_load(sC, p.keepbits + t0 * kTileWords, 1024, cfull);
+              if (vb0 != 0) bulk_load(sC + 1024, p.values + o0, vb0, cfull);
+              if (w.halves == 2) {
+                bulk_load(sC + comp_half, p.keepbits + (t0 + 1) * kTileWords, 1024, cfull);
+                if (vb1 != 0) bulk_load(sC + comp_half + 1024, p.values + o1, vb1, cfull);
+              }
+            }
+          }
+        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) break;
+        if (++stage == stages) { stage = 0; phase ^= 1u; }
+      }
+    }
+  } else if (warp == 1) {
+    // ===== MMA issuer =====
+    constexpr uint32_t idesc = make_idesc(AK != kAK, BKIND == kBMN);
+    int stage = 0;
+    uint32_t phase = 0, unit_phase = 0;
+    bool ok = true;
+    for (int64_t u = blockIdx.x; u < sched.units && ok; u += gridDim.x) {
+      const Unit w = sched.unit(u);
+      if (lane == 0) ok = mbar_wait(smem_u32(&ctl->tmem_empty), unit_phase ^ 1u, abort_flag);
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) break;
+      tc_fence_after();
+      for (int kb = w.kb0; kb < w.kb1; ++kb) {
+        if (lane == 0) {
+          ok = mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag);
+          if (ok) {
+            tc_fence_after();
+            const uint32_t sA = smem_base + stage * stage_bytes;
+            const uint32_t sB = sA + kAStageBytes;
+#pragma unroll
+            for (int k = 0; k < BK / 16; ++k) {
+              const uint64_t bdesc = (BKIND == kBK_) ? make_desc(sB + k * 32, 16, 1024)
+                                                     : make_desc(sB + k * 2048, 8192, 1024);
+              for (int h = 0; h < w.halves; ++h) {
+                const uint64_t adesc = (AK == kAK) ? make_desc(sA + h * 16384 + k * 32, 16, 1024)
+                                                   : make_desc(sA + h * 16384 + k * 2048, 8192, 1024);
+                tc_mma(tmem_base + h * 256, adesc, bdesc, idesc, (kb > w.kb0 || k > 0) ? 1u : 0u);
+              }
+            }
+            tc_commit(smem_u32(&ctl->empty[stage]));            // frees the stage when the MMAs retire
+            if (kb == w.kb1 - 1) tc_commit(smem_u32(&ctl->tmem_full));
+          }
+        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) break;
+        if (++stage == stages) { stage = 0; phase ^= 1u; }
+      }
+      unit_phase ^= 1u;
+    }
+  } else if (warp < 6) {
+    // ===== epilogue: thread = one accumulator row (tensor-memory lane) =====
+    const int q = warp & 3;                      // lanes 32q .. 32q+31 are the ones this warp may read
+    uint32_t unit_phase = 0;
+    bool ok = true;
+    for (int64_t u = blockIdx.x; u < sched.units && ok; u += gridDim.x) {
+      const Unit w = sched.unit(u);
+      ok = mbar_wait(smem_u32(&ctl->tmem_full), unit_phase, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      for (int h = 0; h < w.halves; ++h) {
+        const int64_t m = w.m0 + h * kHalfM + q * 32 + lane;
+        const bool row_ok = m < sched.M;
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          const int64_t n = w.n0 + c0;
+          if (n >= p.N) break;                  // warp-uniform
+          uint32_t r[32];
+          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * 256 + c0), r);
+          tmem_ld_wait();
+          const int nvalid = (int)min((int64_t)32, p.N - n);      // multiple of 8
+          if (EPI == kFwd) {
+            float v[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+            if (p.bias != nullptr) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4) {
+                if (j < nvalid) {
+                  const float4 b4 = __ldg(reinterpret_cast<const float4*>(p.bias + n + j));
+                  v[j] += b4.x; v[j + 1] += b4.y; v[j + 2] += b4.z; v[j + 3] += b4.w;
+                }
+              }
+            }
+            if (row_ok) {
+              if (p.out_z != nullptr) {
+                float4* dst = reinterpret_cast<float4*>(p.out_z + m * p.ld_z + n);
+#pragma unroll
+                for (int j = 0; j < 32; j += 4)
+                  if (j < nvalid) dst[j >> 2] = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+              }
+              if (p.out_zlow != nullptr) {
+                uint4* dst = reinterpret_cast<uint4*>(p.out_zlow + m * p.ld_zlow + n);
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) {
+                  if (j < nvalid) {
+                    __nv_bfloat162 a = __floats2bfloat162_rn(v[j], v[j + 1]), b = __floats2bfloat162_rn(v[j + 2], v[j + 3]);
+                    __nv_bfloat162 c = __floats2bfloat162_rn(v[j + 4], v[j + 5]), d = __floats2bfloat162_rn(v[j + 6], v[j + 7]);
+                    dst[j >> 3] = make_uint4(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b),
+                                             *reinterpret_cast<uint32_t*>(&c), *reinterpret_cast<uint32_t*>(&d));
+                  }
+                }
+              }
+              if (p.out_act != nullptr) {
+                uint32_t bits = 0;
+                uint4* dst = reinterpret_cast<uint4*>(p.out_act + m * p.ld_act + n);
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) {
+                  if (j < nvalid) {
+                    uint32_t pk[4];
+#pragma unroll
+                    for (int e = 0; e < 8; e += 2) {
+                      float a0 = v[j + e], a1 = v[j + e + 1];
+                      if (p.act == RAD_ACT_RELU) { a0 = fmaxf(a0, 0.0f); a1 = fmaxf(a1, 0.0f); }
+                      else if (p.act == RAD_ACT_GELU) { a0 = gelu_f(a0); a1 = gelu_f(a1); }
+                      const __nv_bfloat162 h2 = __floats2bfloat162_rn(a0, a1);
+                      pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+                      // the bit is taken from the rounded activation, the tensor the backward sees
+                      bits |= (__bfloat162float(h2.x) > 0.0f ? 1u : 0u) << (j + e);
+                      bits |= (__bfloat162float(h2.y) > 0.0f ? 1u : 0u) << (j + e + 1);
+                    }
+                    dst[j >> 3] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                  }
+                }
+                if (p.relubits != nullptr) p.relubits[m * p.w32 + (n >> 5)] = bits;
+              }
+            }
+          } else if (EPI == kDx) {
+            if (row_ok) {
+              uint32_t bits = 0xffffffffu;
+              if (p.relubits_prev != nullptr) bits = __ldg(p.relubits_prev + m * ((p.N + 31) / 32) + (n >> 5));
+              uint4* dst = reinterpret_cast<uint4*>(p.out_dx + m * p.ld_dx + n);
+#pragma unroll
+              for (int j = 0; j < 32; j += 8) {
+                if (j < nvalid) {
+                  float g[8];
+#pragma unroll
+                  for (int e = 0; e < 8; ++e) g[e] = ((bits >> (j + e)) & 1u) ? __uint_as_float(r[j + e]) : 0.0f;
+                  if (p.z_prev != nullptr) {
+                    const uint4 zq = __ldg(reinterpret_cast<const uint4*>(p.z_prev + m * p.ld_zprev + n + j));
+                    const uint32_t zw[4] = {zq.x, zq.y, zq.z, zq.w};
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                      const float z = __uint_as_float((e & 1) ? (zw[e >> 1] & 0xffff0000u) : (zw[e >> 1] << 16));
+                      g[e] *= gelu_grad_f(z);
+                    }
+                  }
+                  uint32_t pk[4];
+#pragma unroll
+                  for (int e = 0; e < 8; e += 2) {
+                    const __nv_bfloat162 h2 = __floats2bfloat162_rn(g[e], g[e + 1]);
+                    pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+                  }
+                  dst[j >> 3] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                }
+              }
+            }
+          } else {
+            if (row_ok) {
+              float* dst;
+              if (p.splits > 1) {
+                dst = p.partial + ((int64_t)w.split * p.partial_rows + m) * p.N + n;
+              } else {
+                const int64_t row = (p.row_idx != nullptr) ? (int64_t)__ldg(p.row_idx + m) : m;
+                if (row >= p.dw_rows) { raise_status(p.dev_status, RAD_DEV_EINTERNAL); continue; }
+                dst = p.out_dw + row * p.ld_dw + n;
+              }
+              float4* d4 = reinterpret_cast<float4*>(dst);
+#pragma unroll
+              for (int j = 0; j < 32; j += 4)
+                if (j < nvalid)
+                  d4[j >> 2] = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
+                                           __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(smem_u32(&ctl->tmem_empty));
+      unit_phase ^= 1u;
+    }
+  } else if (AK == kASparse) {
+    // ===== expanders: rebuild the A_hat tile (64 K rows x 256 columns, M-major, swizzled) =====
+    const int et = tid - 192;            // 0..255: keep-bit word et of each half (row et/4, word et%4)
+    const int ew = et >> 5;              // expander warp 0..7
+    const int r = et >> 2, wq = et & 3;
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int64_t u = blockIdx.x; u < sched.units && ok; u += gridDim.x) {
+      const Unit w = sched.unit(u);
+      for (int kb = w.kb0; kb < w.kb1; ++kb) {
+        ok = mbar_wait(smem_u32(&ctl->comp_full[stage]), phase, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        uint8_t* sA = smem + (size_t)stage * stage_bytes;
+        const uint8_t* sC = sA + kAStageBytes + kBStageBytes;
+        for (int h = 0; h < w.halves; ++h) {
+          const uint32_t* bits = reinterpret_cast<const uint32_t*>(sC + (size_t)h * comp_half);
+          const unsigned short* vals = reinterpret_cast<const unsigned short*>(sC + (size_t)h * comp_half + 1024);
+          const uint32_t word = bits[et];
+          const uint32_t cnt = __popc(word);
+          uint32_t incl = cnt;
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t nb = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += nb;
+          }
+          // kept entries before this warp's 32 words: every warp counts them itself, so the eight
+          // expander warps never wait on one another
+          uint32_t before = 0;
+          for (int j = 0; j < ew; ++j) before += __popc(bits[j * 32 + lane]);
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
+          uint32_t pos = before + incl - cnt;
+          // this thread's 32 columns: zero them, then drop the kept values in place
+          uint8_t* rowp = sA + h * 16384 + (wq >> 1) * 8192 + r * 128;
+          const int j0 = (wq & 1) * 4;
+#pragma unroll
+          for (int jj = 0; jj < 4; ++jj)
+            *reinterpret_cast<uint4*>(rowp + (((j0 + jj) ^ (r & 7)) << 4)) = make_uint4(0, 0, 0, 0);
+          uint32_t rest = word;
+          const uint32_t limit = (uint32_t)p.comp_cap >> 1;
+          while (rest != 0) {
+            const int b = __ffs(rest) - 1;
+            rest &= rest - 1;
+            const unsigned short v = (pos < limit) ? vals[pos] : (unsigned short)0;
+            ++pos;
+            const int j = j0 + (b >> 3);
+            *reinterpret_cast<unsigned short*>(rowp + ((j ^ (r & 7)) << 4) + ((b & 7) << 1)) = v;
+          }
+        }
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ctl->full[stage]));
+        if (++stage == stages) { stage = 0; phase ^= 1u; }
+      }
+    }
+  }
+
+  // ===== teardown =====
+  tc_fence_before();
+  __syncthreads();
+  if (tid == 0 && ctl->abort_flag != 0) raise_status(p.dev_status, RAD_DEV_ETIMEOUT);
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+// Sum of the K-split partial tiles in split order; rows may be scattered (same-sample).
+__global__ void __launch_bounds__(256) dw_reduce_kernel(const float* partial, int64_t partial_rows, int splits,
+                                                        int64_t M, const int64_t* M_dev, int64_t N,
+                                                        const uint32_t* row_idx, float* out, int64_t ldw) {
+  if (M_dev != nullptr) M = min(M, *M_dev);
+  const int64_t n4 = N / 4, total = M * n4;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t m = i / n4, c = i % n4;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < splits; ++s) {
+      const float4 v = __ldcs(reinterpret_cast<const float4*>(partial + ((int64_t)s * partial_rows + m) * N) + c);
+      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    const int64_t row = row_idx != nullptr ? (int64_t)row_idx[m] : m;
+    reinterpret_cast<float4*>(out + row * ldw)[c] = acc;
+  }
+}
+
+__global__ void __launch_bounds__(256) zero_f32_kernel(float* out, int64_t rows, int64_t cols, int64_t ld) {
+  const int64_t c4 = cols / 4, total = rows * c4;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x)
+    reinterpret_cast<float4*>(out + (i / c4) * ld)[i % c4] = make_float4(0.f, 0.f, 0.f, 0.f);
+}
+
+// ---- host side -------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(sym);
+  }
+  return fn;
+}
+
+// bf16 matrix, `inner` contiguous elements per row, `outer` rows of `ld` elements; box = 64 x box_outer.
+int make_map(CUtensorMap* map, const void* ptr, int64_t inner, int64_t outer, int64_t ld, int box_outer) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return RAD_ECUDA;
+  const cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+  const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)box_outer};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? RAD_OK : RAD_ECUDA;
+}
+
+int num_sms() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+      n = kNumSMsDefault;
+  }
+  return n;
+}
+
+// K splits for a dW contraction: fewest "waves x K blocks per unit", with a small charge per split
+// for the partial-tile traffic.  Pure function of the shapes, so the workspace query and the launch agree.
+int choose_splits(int64_t m_tiles, int64_t n_tiles, int64_t kblocks) {
+  const int64_t sms = kNumSMsDefault;
+  int best = 1;
+  double best_cost = 1e300;
+  for (int s = 1; s <= kMaxSplits && s <= kblocks; ++s) {
+    const int64_t units = m_tiles * n_tiles * s;
+    const double cost = (double)ceil_div(units, sms) * (double)ceil_div(kblocks, s) + (s > 1 ? 4.0 * s : 0.0);
+    if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
+  }
+  return best;
+}
+
+struct DwPlan { int splits; int64_t partial_rows; int64_t bytes; int comp_cap; int stages; };
+
+DwPlan plan_dw(const rad_store* st, int64_t H) {
+  DwPlan d;
+  const int64_t kblocks = ceil_div(st->B, BK);
+  int64_t m_expect;
+  if (st->variant == RAD_SAME_SAMPLE) {
+    m_expect = std::max<int64_t>(1, (int64_t)std::llround((double)st->D * keep_threshold_host(st->p) / 65536.0));
+    d.partial_rows = round_up(std::min(st->values_ld, round_up(st->D, 8)), BM);
+    d.comp_cap = 0;
+    d.stages = 3;
+  } else {
+    m_expect = st->D;
+    d.partial_rows = round_up(st->D, BM);
+    // per-tile value staging: mean + 8 sigma of Binomial(8192, p_eff), padded, in bytes
+    const double pe = keep_threshold_host(st->p) / 65536.0, n = (double)kTileRows * kTileCols;
+    int64_t cap = (int64_t)(n * pe + 8.0 * std::sqrt(n * pe * (1.0 - pe)) + 16.0);
+    cap = std::min<int64_t>(round_up(cap, 8), (int64_t)n) * 2;
+    d.comp_cap = (int)round_up(cap, 128);
+    const int stage_bytes = (int)round_up(kAStageBytes + kBStageBytes + 2 * (1024 + d.comp_cap), 1024);
+    d.stages = std::min(3, (int)((227 * 1024 - 2048) / stage_bytes));
+  }
+  d.splits = choose_splits(ceil_div(m_expect, BM), ceil_div(H, BN), kblocks);
+  d.bytes = d.splits > 1 ? (int64_t)d.splits * d.partial_rows * H * 4 : 0;
+  return d;
+}
+
+template <int AK, int BKIND, int EPI>
+int launch(const TcParams& p, const CUtensorMap& ta, const CUtensorMap& tb, int64_t max_units, cudaStream_t s) {
+  const int comp_half = (AK == kASparse) ? (1024 + p.comp_cap) : 0;
+  const int stage_bytes = (int)round_up(kAStageBytes + kBStageBytes + 2 * comp_half, 1024);
+  const size_t smem = (size_t)p.num_stages * stage_bytes + sizeof(SmemCtl) + 1024;
+  auto kernel = tc_gemm_kernel<AK, BKIND, EPI>;
+  static bool configured = false;
+  static size_t configured_smem = 0;
+  if (!configured || smem > configured_smem) {
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+      return RAD_ECUDA;
+    configured = true;
+    configured_smem = 227 * 1024;
+  }
+  if (smem > 227 * 1024) return RAD_EUNSUPPORTED;
+  const int grid = (int)std::max<int64_t>(1, std::min<int64_t>(max_units, num_sms()));
+  kernel<<<grid, threads_for<AK>(), smem, s>>>(p, ta, tb);
+  return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
+}
+
+bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+
+}  // namespace
+
+bool tc_shape_ok(int64_t B, int64_t D, int64_t H, const void* p0, int64_t ld0, const void* p1, int64_t ld1) {
+  if (B < 64 || D < 64 || H < 64) return false;                    // tiny layers stay on CUDA cores
+  if (D % 8 != 0 || H % 8 != 0) return false;
+  if (!aligned16(p0) || !aligned16(p1) || ld0 % 8 != 0 || ld1 % 8 != 0) return false;
+  if (B >= (1ll << 31) || D >= (1ll << 31) || H >= (1ll << 31)) return false;
+  return encode_fn() != nullptr;
+}
+
+int tc_forward(int act, int64_t B, int64_t D, int64_t H, const void* A, int64_t lda, const void* W, int64_t ldw,
+               const float* bias, void* out_act, int64_t ld_act, float* out_z, int64_t ld_z, void* out_zlow,
+               int64_t ld_zlow, uint32_t* relubits, int32_t* dev_status, cudaStream_t s) {
+  CUtensorMap ta, tb;
+  int rc = make_map(&ta, A, D, B, lda, 256);          // K-major A: box 64 (K) x 256 rows
+  if (rc != RAD_OK) return rc;
+  rc = make_map(&tb, W, H, D, ldw, 64);               // MN-major B: box 64 (N) x 64 K rows
+  if (rc != RAD_OK) return rc;
+  TcParams p = {};
+  p.M = B; p.N = H; p.K = D; p.splits = 1; p.num_stages = 3;
+  p.bias = bias; p.act = act;
+  p.out_act = static_cast<bf16*>(out_act); p.ld_act = ld_act; p.out_z = out_z; p.ld_z = ld_z;
+  p.out_zlow = static_cast<bf16*>(out_zlow); p.ld_zlow = ld_zlow; p.relubits = relubits; p.w32 = ceil_div(H, 32);
+  p.dev_status = dev_status;
+  return launch<kAK, kBMN, kFwd>(p, ta, tb, ceil_div(B, BM) * ceil_div(H, BN), s);
+}
+
+int tc_input_grad(int64_t B, int64_t D, int64_t H, const void* dZ, int64_t ldz, const void* W, int64_t ldw,
+                  const uint32_t* relubits_prev, const void* z_prev, int64_t ld_zprev, void* dZ_prev, int64_t ldp,
+                  int32_t* dev_status, cudaStream_t s) {
+  CUtensorMap ta, tb;
+  int rc = make_map(&ta, dZ, H, B, ldz, 256);         // K-major A (K = H)
+  if (rc != RAD_OK) return rc;
+  rc = make_map(&tb, W, H, D, ldw, 256);              // K-major B: rows d (N), K = H contiguous
+  if (rc != RAD_OK) return rc;
+  TcParams p = {};
+  p.M = B; p.N = D; p.K = H; p.splits = 1; p.num_stages = 3;
+  p.relubits_prev = relubits_prev; p.z_prev = static_cast<const bf16*>(z_prev); p.ld_zprev = ld_zprev;
+  p.out_dx = static_cast<bf16*>(dZ_prev); p.ld_dx = ldp;
+  p.dev_status = dev_status;
+  return launch<kAK, kBK_, kDx>(p, ta, tb, ceil_div(B, BM) * ceil_div(D, BN), s);
+}
+
+int64_t tc_weight_grad_workspace(const rad_store* st, int64_t H) {
+  if (st->dtype != RAD_BF16 || st->D % 8 != 0 || H % 8 != 0 || st->B < 64 || st->D < 64 || H < 64) return 0;
+  return plan_dw(st, H).bytes;
+}
+
+int tc_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H, float* dW, int64_t ldw,
+                   void* workspace, int64_t workspace_bytes, int32_t* dev_status, cudaStream_t s) {
+  const DwPlan d = plan_dw(st, H);
+  if (d.bytes > 0 && (workspace == nullptr || workspace_bytes < d.bytes || !aligned16(workspace))) return RAD_EWORKSPACE;
+  if (!aligned16(st->keepbits) || !aligned16(st->values)) return RAD_EUNSUPPORTED;
+  CUtensorMap ta, tb;
+  int rc = make_map(&tb, dZ, H, st->B, ldz, 64);      // MN-major B: box 64 (N = h) x 64 K rows (b)
+  if (rc != RAD_OK) return rc;
+  TcParams p = {};
+  p.N = H; p.K = st->B; p.splits = d.splits; p.num_stages = d.stages;
+  p.out_dw = dW; p.ld_dw = ldw; p.dw_rows = st->D; p.partial = static_cast<float*>(workspace); p.partial_rows = d.partial_rows;
+  p.dev_status = dev_status;
+  const int grid_z = (int)std::min<int64_t>(ceil_div(st->D * H / 4, 256), 148 * 16);
+  if (st->variant == RAD_SAME_SAMPLE) {
+    const int64_t mmax = std::min(st->values_ld, round_up(st->D, 8));
+    rc = make_map(&ta, st->values, st->values_ld, st->B, st->values_ld, 64);   // MN-major A: A_c is B x ld
+    if (rc != RAD_OK) return rc;
+    p.M = mmax; p.M_dev = st->nnz; p.row_idx = st->offsets;
+    zero_f32_kernel<<<grid_z, 256, 0, s>>>(dW, st->D, H, ldw);
+    rc = launch<kAMN, kBMN, kDw>(p, ta, tb, ceil_div(mmax, BM) * ceil_div(H, BN) * d.splits, s);
+  } else {
+    ta = tb;                                           // unused by the sparse-A kernel
+    p.M = st->D;
+    p.values = static_cast<const bf16*>(st->values); p.keepbits = st->keepbits; p.offsets = st->offsets;
+    p.values_capacity = st->values_capacity; p.ncb = (int32_t)ceil_div(st->D, kTileCols); p.comp_cap = d.comp_cap;
+    rc = launch<kASparse, kBMN, kDw>(p, ta, tb, ceil_div(st->D, BM) * ceil_div(H, BN) * d.splits, s);
+  }
+  if (rc != RAD_OK) return rc;
+  if (d.splits > 1) {
+    const int64_t work = p.M * (H / 4);
+    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>(ceil_div(work, 256), 148 * 16));
+    dw_reduce_kernel<<<grid, 256, 0, s>>>(p.partial, d.partial_rows, d.splits, p.M, p.M_dev, H, p.row_idx, dW, ldw);
+  }
+  return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
+}
+
+}  // namespace rad
