@@ -1,0 +1,435 @@
+#!/usr/bin/env python
+"""Benchmark of the RAD training step on the wide bf16 MLP (8192 x 4 -> 1000, batch 65536).
+
+A step is one pass of the whole hot path over one synthetic batch: for every layer the
+Philox-masked compact store and the exact forward, then the loss, then per layer the weight
+gradient from the store, the bias gradient and the exact input gradient.  The timed region
+issues the per-layer C-ABI calls (the same launches rad_mlp_step makes) so CUDA events can
+bracket each kernel family; the end-to-end figure goes through rad_mlp_step with the batch
+coming from pinned host memory each step.
+
+    python bench.py --gpus 1 --steps 5 --warmup 3
+    python -m torch.distributed.run --nnodes=1 --nproc-per-node N --master-addr 127.0.0.1 \
+        --master-port P bench.py --gpus N --steps K --warmup W
+    python bench.py --impl reference      # the CPU oracle on a row slab of the same workload
+
+With N > 1 every rank runs an independent replica on its own batch (the path has no exchange
+step: masks are keyed on global row indices and a real data-parallel job would only add one
+all-reduce of dW); the reported value is all ranks' samples over the slowest rank's time.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "rad_train_step_samples_per_s"
+UNIT = "samples/s"
+DIMS = (8192, 8192, 8192, 8192, 8192, 1000)
+BATCH = 65536
+CPU_SLAB_ROWS = 2048         # rows of the workload the CPU oracle is timed on (10-30 s per step on 16 cores)
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--variant", default="different", choices=["different", "same"])
+    ap.add_argument("--p", type=float, default=0.1)
+    ap.add_argument("--act", default="gelu", choices=["gelu", "relu"])
+    ap.add_argument("--batch", type=int, default=BATCH)
+    ap.add_argument("--no-sweep", action="store_true", help="skip the per-kernel p sweep")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    return ap.parse_args()
+
+
+# --------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands, on a bounded row slab of the same workload
+# --------------------------------------------------------------------------------------------
+def _oracle_inputs(rows, seed=1234):
+    from workloads import mlp_inputs
+    return mlp_inputs(DIMS, rows, "bf16", "normal", seed)
+
+
+def time_oracle(args, steps, warmup):
+    import numpy as np
+    from oracle import rad as orc
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    X, y, Ws, bs = _oracle_inputs(CPU_SLAB_ROWS)
+    times = []
+    for i in range(warmup + steps):
+        t0 = time.perf_counter()
+        r = orc.mlp_step(X, y, Ws, bs, act=args.act, dtype="bf16", variant=args.variant, p=args.p, seed=0, step=i)
+        dt = time.perf_counter() - t0
+        if i >= warmup:
+            times.append(dt)
+        assert np.isfinite(r.loss)
+    mean = sum(times) / len(times)
+    return dict(value=CPU_SLAB_ROWS / mean, unit=UNIT, cores=int(cores), kind="oracle",
+                sample=f"row slab of {CPU_SLAB_ROWS} rows of the same net (full D and H), "
+                       f"{len(times)} step(s) of {mean:.2f} s"), mean
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps, warmup = max(1, min(args.steps, 3)), min(args.warmup, 1)
+    base, mean = time_oracle(args, steps, warmup)
+    line = dict(impl="reference", metric=METRIC, value=base["value"], unit=UNIT, n_gpus=args.gpus, steps=steps,
+                warmup=warmup, ms_per_step=mean * 1e3, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="f64", data="synthetic",
+                config=dict(workload="mlp_wide 8192x4->1000 bf16 grid, oracle on a row slab", dims=list(DIMS),
+                            batch=CPU_SLAB_ROWS, variant=args.variant, p=args.p, act=args.act),
+                cpu_baseline=base,
+                e2e=dict(value=base["value"], unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------------------
+# our arm
+# --------------------------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc = index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["no samples"])
+        return dict(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), power_w_max=max(power), samples=len(sm),
+                    reasons=sorted(reasons))
+
+
+class LayerwiseStep:
+    """The launches of rad_mlp_step issued call by call, with CUDA events around each kernel family."""
+
+    def __init__(self, rad, torch, dims, B, act, variant, p):
+        self.rad, self.torch, self.dims, self.B, self.act, self.variant, self.p = rad, torch, dims, B, act, variant, p
+        L = self.L = len(dims) - 1
+        dev, bf = "cuda", torch.bfloat16
+        self.stores = [rad.Store(variant, "bf16", B, dims[l], p, layer=l, relu_bits=False) for l in range(L)]
+        hid = max(dims[1:L]) if L > 1 else 8
+        self.acts = [torch.empty(B, hid, dtype=bf, device=dev) for _ in range(2)]
+        self.dzs = [torch.empty(B, max(dims[1:]), dtype=bf, device=dev) for _ in range(2)]
+        self.logits = torch.empty(B, dims[L], dtype=torch.float32, device=dev)
+        self.relubits = [None] + [torch.empty(B * ((dims[l] + 31) // 32), dtype=torch.int32, device=dev)
+                                  if act == "relu" else None for l in range(1, L)]
+        self.preact = [None] + [torch.empty(B, dims[l], dtype=bf, device=dev) if act == "gelu" else None
+                                for l in range(1, L)]
+        self.dW = [torch.empty(dims[l], dims[l + 1], dtype=torch.float32, device=dev) for l in range(L)]
+        self.db = [torch.empty(dims[l + 1], dtype=torch.float32, device=dev) for l in range(L)]
+        self.loss = torch.zeros(1, dtype=torch.float32, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        ws = max([rad.rad_weight_grad_workspace(self.stores[l], dims[l + 1]) for l in range(L)] +
+                 [rad.rad_input_grad_workspace(B, dims[l + 1]) for l in range(L)] + [B * 4, 256])
+        self.ws = torch.empty(ws, dtype=torch.uint8, device=dev)
+        self.events = []          # (family, layer, start, stop)
+
+    def _timed(self, family, layer, fn):
+        e0, e1 = self.torch.cuda.Event(enable_timing=True), self.torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        self.events.append((family, layer, e0, e1))
+
+    def __call__(self, X, labels, Ws, bs, seed, step, record):
+        rad, L, dims = self.rad, self.L, self.dims
+        run = self._timed if record else (lambda fam, l, fn: fn())
+        a_in = X
+        for l in range(L):
+            st = self.stores[l]
+            st.c.seed, st.c.step = seed, step
+            run("store", l, lambda: rad.rad_linear_forward_store(a_in, st, self.status))
+            last = l == L - 1
+            if last:
+                run("forward", l, lambda: rad.rad_linear_forward(a_in, Ws[l], bs[l], "none", out_z=self.logits,
+                                                                 dev_status=self.status))
+            else:
+                out = self.acts[l & 1][:, :dims[l + 1]]
+                run("forward", l, lambda: rad.rad_linear_forward(a_in, Ws[l], bs[l], self.act, out_act=out,
+                                                                 out_zlow=self.preact[l + 1],
+                                                                 relubits=self.relubits[l + 1],
+                                                                 dev_status=self.status))
+                a_in = out
+        dz = self.dzs[(L - 1) & 1][:, :dims[L]]
+        run("loss", L - 1, lambda: rad.rad_softmax_xent(self.logits, labels, self.loss, dz, self.ws))
+        for l in range(L - 1, -1, -1):
+            st = self.stores[l]
+            run("dW", l, lambda: rad.rad_linear_weight_grad(st, dz, self.dW[l], self.ws, self.status))
+            dz_prev = self.dzs[(l - 1) & 1][:, :dims[l]] if l > 0 else None
+            run("dX+db", l, lambda: rad.rad_linear_input_grad(dz, Ws[l], relubits_prev=self.relubits[l],
+                                                              z_prev=self.preact[l], dZ_prev=dz_prev, db=self.db[l],
+                                                              workspace=self.ws, dev_status=self.status))
+            dz = dz_prev
+
+    def family_ms(self):
+        out = {}
+        for fam, layer, e0, e1 in self.events:
+            out.setdefault((fam, layer), []).append(e0.elapsed_time(e1))
+        return out
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return dict(hbm_gbs=d["hbm_gbs"], tflops_burst=d["bf16_tflops"], tflops_sustained=d["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, source="fallback")
+
+
+def kernel_sweep(rad, torch, A, dZ, H, ps):
+    """Store GB/s and dW TFLOP/s of one 8192 x 8192 layer for both variants over the p sweep."""
+    B, D = A.shape
+    rows = []
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dW = torch.empty(D, H, dtype=torch.float32, device="cuda")
+
+    def timed(fn, n=5):
+        fn(); fn()
+        torch.cuda.synchronize()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
+        ev[0].record()
+        for i in range(n):
+            fn()
+            ev[i + 1].record()
+        torch.cuda.synchronize()
+        return statistics.median(ev[i].elapsed_time(ev[i + 1]) for i in range(n))
+
+    for variant in ("different", "same"):
+        for p in ps:
+            st = rad.Store(variant, "bf16", B, D, p, relu_bits=False)
+            ms_store = timed(lambda: rad.rad_linear_forward_store(A, st, status))
+            nnz = st.nnz.cpu().numpy()
+            ws = torch.empty(max(rad.rad_weight_grad_workspace(st, H), 256), dtype=torch.uint8, device="cuda")
+            ms_dw = timed(lambda: rad.rad_linear_weight_grad(st, dZ, dW, ws, status), n=3)
+            if variant == "different":
+                store_bytes = B * D * 2 + int(nnz[1]) * 2 + B * D // 8 + 4 * (len(st.offsets))
+                flops, kind = 2.0 * B * D * H, "dense-tile"
+            else:
+                store_bytes = B * D * 2 + int(nnz[1]) * 2 + 4 * int(nnz[0])
+                flops, kind = 2.0 * B * int(nnz[0]) * H, "kept-columns"
+            rows.append(dict(variant=variant, p=p, store_ms=round(ms_store, 4),
+                             store_gbs=round(store_bytes / ms_store / 1e6, 1),
+                             dW_ms=round(ms_dw, 4), dW_tflops=round(flops / ms_dw / 1e9, 1), dW_flops=kind,
+                             nnz=int(nnz[0])))
+            del st, ws
+    assert status.item() == 0, f"device status {status.item()}"
+    return rows
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2007_10412_b200 as rad
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    B, dims, L = args.batch, DIMS, len(DIMS) - 1
+    bf = torch.bfloat16
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(1234 + rank)                       # every rank its own batch (weak scaling)
+    X = torch.randn(B, dims[0], generator=gen, device="cuda", dtype=torch.float32).to(bf)
+    labels = torch.randint(0, dims[L], (B,), generator=gen, device="cuda", dtype=torch.int32)
+    wgen = torch.Generator(device="cuda")
+    wgen.manual_seed(99)                               # same weights on every rank
+    Ws = [(torch.randn(dims[l], dims[l + 1], generator=wgen, device="cuda") * (2.0 / dims[l]) ** 0.5).to(bf)
+          for l in range(L)]
+    bs = [torch.zeros(dims[l + 1], device="cuda") for l in range(L)]
+
+    lw = LayerwiseStep(rad, torch, dims, B, args.act, args.variant, args.p)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        lw(X, labels, Ws, bs, seed=0, step=i, record=False)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = rad.rad_launch_count()
+    t_start, t_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    for i in range(args.steps):
+        lw(X, labels, Ws, bs, seed=0, step=args.warmup + i, record=True)
+    t_stop.record()
+    barrier()
+    launches = (rad.rad_launch_count() - launches0) // max(args.steps, 1)
+    clocks = sampler.stop()
+    ms_total = t_start.elapsed_time(t_stop)
+    if world > 1:
+        t = torch.tensor([ms_total], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = t.item()
+    assert lw.status.item() == 0, f"device status {lw.status.item()}"
+    ms_step = ms_total / args.steps
+    value = world * B * args.steps / (ms_total / 1e3)
+
+    # per-family device time inside the timed region, and the roofline of the dominant kernel
+    fam = lw.family_ms()
+    by_family = {}
+    for (f, l), v in fam.items():
+        by_family.setdefault(f, 0.0)
+        by_family[f] += sum(v) / args.steps
+    pk = peaks()
+    dw_big = [(l, sum(v) / len(v)) for (f, l), v in fam.items() if f == "dW" and dims[l] == 8192 and dims[l + 1] == 8192]
+    fwd_big = [(l, sum(v) / len(v)) for (f, l), v in fam.items() if f == "forward" and dims[l + 1] == 8192]
+    dominant = max(by_family, key=by_family.get)
+    if dominant == "dW":
+        ms_k = sum(t for _, t in dw_big) / len(dw_big)
+        if args.variant == "different":
+            flops, what = 2.0 * B * 8192 * 8192, "tc_gemm_kernel<sparse A> dW, dense-tile flops 2*B*D*H"
+        else:
+            k = int(lw.stores[1].nnz[0].item())
+            flops, what = 2.0 * B * k * 8192, "tc_gemm_kernel<MN,MN> dW, flops 2*B*k'*H on kept columns"
+    else:
+        ms_k = sum(t for _, t in fwd_big) / len(fwd_big)
+        flops, what = 2.0 * B * 8192 * 8192, "tc_gemm_kernel forward, flops 2*B*D*H"
+    achieved = flops / ms_k / 1e9
+    roofline = dict(bound="tensor", kernel=what, achieved=round(achieved, 1), peak=pk["tflops_sustained"],
+                    unit="TFLOP/s", frac=round(achieved / pk["tflops_sustained"], 4), traffic=None,
+                    peak_source=pk["source"] + " (sustained cuBLAS bf16)", ms_per_launch=round(ms_k, 4),
+                    how="CUDA events around the call on the launching stream, inside the timed steps")
+    store_big = [sum(v) / len(v) for (f, l), v in fam.items() if f == "store" and dims[l] == 8192]
+    nnz1 = lw.stores[1].nnz.cpu().numpy()
+    if args.variant == "different":
+        sbytes = B * 8192 * 2 + int(nnz1[1]) * 2 + B * 8192 // 8 + 4 * len(lw.stores[1].offsets)
+    else:
+        sbytes = B * 8192 * 2 + int(nnz1[1]) * 2 + 4 * int(nnz1[0])
+    ms_s = sum(store_big) / len(store_big)
+    store_roofline = dict(bound="hbm", kernel="store kernel, one 8192-wide layer input",
+                          achieved=round(sbytes / ms_s / 1e6, 1), peak=pk["hbm_gbs"], unit="GB/s",
+                          frac=round(sbytes / ms_s / 1e6 / pk["hbm_gbs"], 4), traffic=None,
+                          ms_per_launch=round(ms_s, 4), algorithmic_bytes=sbytes)
+
+    # stored activation bytes versus full backprop (from the whole-net entry point's plan)
+    ctx = rad.MLPStep(dims, B, "bf16", args.act, args.variant, args.p)
+    s = ctx.stats
+    held = s.value_bytes + s.index_bytes + s.relu_bytes + s.preact_bytes + s.unsampled_bytes
+    memory = dict(value_bytes=s.value_bytes, index_bytes=s.index_bytes, relu_bytes=s.relu_bytes,
+                  preact_bytes=s.preact_bytes, unsampled_bytes=s.unsampled_bytes, held_bytes=held,
+                  full_backprop_bytes=s.full_backprop_bytes, ratio=round(s.full_backprop_bytes / held, 3))
+
+    # end to end through rad_mlp_step: the batch comes from pinned host memory every step
+    Xh = torch.empty(X.shape, dtype=bf).pin_memory()
+    Xh.copy_(X)
+    yh = torch.empty(labels.shape, dtype=torch.int32).pin_memory()
+    yh.copy_(labels)
+    Xd, yd = torch.empty_like(X), torch.empty_like(labels)
+    del lw
+    torch.cuda.empty_cache()
+
+    def e2e_step(i):
+        Xd.copy_(Xh, non_blocking=True)
+        yd.copy_(yh, non_blocking=True)
+        ctx(Xd, yd, Ws, bs, seed=0, step=i)
+        return ctx.loss.cpu().item()
+
+    for i in range(min(args.warmup, 2)):
+        e2e_step(i)
+    barrier()
+    t0 = time.perf_counter()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        loss = e2e_step(100 + i)
+    e1.record()
+    barrier()
+    e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3 if world == 1 else 0.0)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = t.item()
+    assert ctx.dev_status.item() == 0
+    e2e = dict(value=world * B * args.steps / (e2e_ms / 1e3), unit=UNIT,
+               h2d_bytes_per_step=Xh.numel() * 2 + yh.numel() * 4, d2h_bytes_per_step=4,
+               ms_per_step=round(e2e_ms / args.steps, 3), api="rad_mlp_step", last_loss=round(loss, 5))
+
+    sweep = None
+    if rank == 0 and world == 1 and not args.no_sweep:
+        dZ = (torch.randn(B, 8192, generator=gen, device="cuda") / B).to(bf)
+        sweep = kernel_sweep(rad, torch, X, dZ, 8192, (0.01, 0.05, 0.1, 0.5))
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        cpu, _ = time_oracle(args, 1, 0)
+
+    if rank == 0:
+        line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+                    ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
+                    data="synthetic",
+                    config=dict(workload="mlp_wide: 8192->8192x4->1000, bf16, batch 65536 per GPU, N(0,1) inputs",
+                                dims=list(dims), global_batch=world * B, act=args.act, variant=args.variant, p=args.p,
+                                parallelism="replicas" if world > 1 else "1 GPU",
+                                l2="inputs larger than L2 (1 GiB activations per layer)"),
+                    clocks=clocks, e2e=e2e, gpu_launches=int(launches), roofline=roofline,
+                    store_roofline=store_roofline, family_ms={k: round(v, 3) for k, v in by_family.items()},
+                    activation_memory=memory, cpu_baseline=cpu, kernel_sweep=sweep)
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -238,6 +238,9 @@ int rad_mlp_step(const rad_mlp_desc* net /* host */, const void* X, const int32_
                  void* workspace, int64_t workspace_bytes,
                  int32_t* dev_status, void* stream);
 
+/* Kernels this library has launched since it was loaded (host-side tally; memsets not counted). */
+int64_t rad_launch_count(void);
+
 const char* rad_strerror(int code);
 const char* rad_version(void);
 

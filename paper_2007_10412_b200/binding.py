@@ -58,7 +58,7 @@ class rad_step_stats(C.Structure):
 EXPORTS = ["rad_keep_threshold", "rad_effective_p", "rad_scale", "rad_store_size_query",
            "rad_linear_forward_store", "rad_weight_grad_workspace", "rad_linear_weight_grad",
            "rad_linear_forward", "rad_softmax_xent", "rad_input_grad_workspace", "rad_linear_input_grad",
-           "rad_mlp_workspace", "rad_mlp_step", "rad_strerror", "rad_version"]
+           "rad_mlp_workspace", "rad_mlp_step", "rad_launch_count", "rad_strerror", "rad_version"]
 
 _lib = None
 
@@ -79,6 +79,7 @@ def lib():
         L.rad_strerror.restype = C.c_char_p
         L.rad_strerror.argtypes = [C.c_int]
         L.rad_version.restype = C.c_char_p
+        L.rad_launch_count.restype = C.c_int64
         i32, i64, f32, vp = C.c_int32, C.c_int64, C.c_float, C.c_void_p
         L.rad_store_size_query.argtypes = [i32, i32, i64, i64, f32, C.POINTER(rad_store_sizes)]
         L.rad_linear_forward_store.argtypes = [vp, i64, C.POINTER(rad_store), vp, i64, vp, vp]
@@ -128,6 +129,10 @@ def rad_effective_p(p):
 
 def rad_scale(p):
     return float(lib().rad_scale(p))
+
+
+def rad_launch_count():
+    return int(lib().rad_launch_count())
 
 
 def rad_version():

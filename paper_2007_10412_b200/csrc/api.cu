@@ -17,6 +17,9 @@ int check_device() {
   return cached_rc;
 }
 
+static int64_t g_launches = 0;
+void count_launch(int n) { g_launches += n; }
+
 namespace {
 
 bool valid_dtype(int d) { return d == RAD_F32 || d == RAD_BF16; }
@@ -102,6 +105,8 @@ int make_plan(const rad_mlp_desc* net, StepPlan* plan) {
 }  // namespace rad
 
 using namespace rad;
+
+extern "C" int64_t rad_launch_count(void) { return g_launches; }
 
 extern "C" const char* rad_version(void) { return "rad-b200 0.1 (sm_100a)"; }
 

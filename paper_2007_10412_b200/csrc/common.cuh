@@ -116,6 +116,7 @@ inline int64_t round_up(int64_t a, int64_t b) { return ceil_div(a, b) * b; }
 
 // internal launchers shared across translation units --------------------------------------------
 int check_device();   // RAD_OK on an sm_100 device
+void count_launch(int n = 1);   // host-side tally of kernels this library has launched
 
 // f32/bf16 CUDA-core kernels (small or unaligned problems)
 int simt_forward(int dtype, int act, int64_t B, int64_t D, int64_t H, const void* A, int64_t lda,

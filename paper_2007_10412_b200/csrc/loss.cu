@@ -63,6 +63,7 @@ extern "C" int rad_softmax_xent(int32_t dtype, int64_t B, int64_t C, const float
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   float* rows = static_cast<float*>(workspace);
   const unsigned grid = (unsigned)ceil_div(B, 8);
+  count_launch(2);
   if (dtype == RAD_BF16)
     xent_rows_kernel<bf16><<<grid, 256, 0, s>>>(logits, ldl, labels, B, C, static_cast<bf16*>(dZ), ldz, rows);
   else

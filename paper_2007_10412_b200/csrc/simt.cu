@@ -109,6 +109,7 @@ template <int EPI>
 int launch_gemm(int dtype, const GemmParams& p, int64_t Mgrid, cudaStream_t s) {
   dim3 grid((unsigned)ceil_div(p.N, kBN), (unsigned)ceil_div(Mgrid, kBM));
   if (grid.x == 0 || grid.y == 0) return RAD_OK;
+  count_launch();
   if (dtype == RAD_BF16)
     gemm_kernel<bf16, EPI><<<grid, 256, 0, s>>>(p);
   else
@@ -264,6 +265,7 @@ int simt_forward(int dtype, int act, int64_t B, int64_t D, int64_t H, const void
     if (out_act == nullptr) return RAD_EINVAL;
     const int64_t w32 = ceil_div(H, 32), n = B * w32;
     const int g = (int)std::min<int64_t>(ceil_div(n, 256), 148 * 16);
+    count_launch();
     if (dtype == RAD_BF16)
       relu_bits_rows_kernel<bf16><<<g, 256, 0, s>>>(static_cast<const bf16*>(out_act), ld_act, B, H, w32, relubits);
     else
@@ -291,6 +293,7 @@ int simt_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H
   (void)dev_status;
   if (st->variant == RAD_SAME_SAMPLE) {
     const int g = (int)std::min<int64_t>(ceil_div(st->D * H, 256), 148 * 16);
+    count_launch();
     zero_rows_kernel<<<g, 256, 0, s>>>(dW, ldw, st->D, H);
     GemmParams p = {};
     p.A = st->values; p.sam = 1; p.sak = st->values_ld;     // A(j, b) = values[b, j]
@@ -307,6 +310,7 @@ int simt_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H
   p.ncb = (int32_t)ceil_div(st->D, kTileCols); p.nslabs = (int32_t)ceil_div(st->B, kTileRows);
   p.dZ = dZ; p.ldz = ldz; p.dW = dW; p.ldw = ldw;
   dim3 grid((unsigned)p.ncb, (unsigned)ceil_div(H, kSparseBN));
+  count_launch();
   if (st->dtype == RAD_BF16)
     sparse_dw_kernel<bf16><<<grid, 256, 0, s>>>(p);
   else
@@ -324,6 +328,7 @@ int column_sums(int dtype, int64_t B, int64_t H, const void* dZ, int64_t ldz, fl
   const int64_t chunks = ceil_div(B, kColChunkRows);
   dim3 grid((unsigned)ceil_div(H, 256), (unsigned)chunks);
   float* partial = static_cast<float*>(workspace);
+  count_launch(2);
   if (dtype == RAD_BF16)
     colsum_partial_kernel<bf16><<<grid, 256, 0, s>>>(static_cast<const bf16*>(dZ), ldz, B, H, partial);
   else

@@ -489,6 +489,7 @@ extern "C" int rad_linear_forward_store(const void* A, int64_t lda, const rad_st
     p.dev_status = dev_status;
     p.vec_ok = (((uintptr_t)A & 15) == 0 && (lda * esz) % 16 == 0) ? 1 : 0;
     RAD_CUDA_TRY(cudaMemsetAsync(workspace, 0, (size_t)need, s));
+    count_launch();
     if (st->dtype == RAD_BF16)
       store_different_kernel<bf16><<<p.ntiles, 256, 0, s>>>(p, ks);
     else
@@ -504,6 +505,7 @@ extern "C" int rad_linear_forward_store(const void* A, int64_t lda, const rad_st
   p.c2 = counter_word2(st->layer, RAD_SAME_SAMPLE); p.c3 = st->step;
   p.values = st->values; p.ld = st->values_ld; p.keepbits = st->keepbits; p.idx = st->offsets;
   p.nnz = st->nnz; p.dev_status = dev_status;
+  count_launch(2);
   same_mask_kernel<<<1, 1024, 0, s>>>(p, ks);
   const int grid = (int)std::min<int64_t>(ceil_div(st->B, 8), 148 * 8);
   if (st->dtype == RAD_BF16)
@@ -513,6 +515,7 @@ extern "C" int rad_linear_forward_store(const void* A, int64_t lda, const rad_st
   if (st->relubits != nullptr) {
     const int64_t n = st->B * w32;
     const int g2 = (int)std::min<int64_t>(ceil_div(n, 256), 148 * 16);
+    count_launch();
     if (st->dtype == RAD_BF16)
       relu_bits_kernel<bf16><<<g2, 256, 0, s>>>(static_cast<const bf16*>(A), lda, st->B, st->D, w32, st->relubits);
     else

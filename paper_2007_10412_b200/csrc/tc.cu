@@ -618,15 +618,20 @@ int num_sms() {
   return n;
 }
 
-// K splits for a dW contraction: fewest "waves x K blocks per unit", with a small charge per split
-// for the partial-tile traffic.  Pure function of the shapes, so the workspace query and the launch agree.
+// K splits for a dW contraction.  Cost model in units of one CTA working through one K block
+// (about 1024 tensor-pipe clocks): waves x K blocks per unit, plus what writing and re-reading the
+// float32 partial tiles costs at HBM speed.  Pure function of the shapes, so the workspace query
+// and the launch agree.
 int choose_splits(int64_t m_tiles, int64_t n_tiles, int64_t kblocks) {
   const int64_t sms = kNumSMsDefault;
+  const double kblock_us = 0.55;                                            // 1024 clk at ~1.9 GHz
+  const double partial_us = (double)(m_tiles * BM) * (double)(n_tiles * BN) * 8.0 / 6.5e6;   // per split
   int best = 1;
   double best_cost = 1e300;
   for (int s = 1; s <= kMaxSplits && s <= kblocks; ++s) {
     const int64_t units = m_tiles * n_tiles * s;
-    const double cost = (double)ceil_div(units, sms) * (double)ceil_div(kblocks, s) + (s > 1 ? 4.0 * s : 0.0);
+    const double cost = (double)ceil_div(units, sms) * (double)ceil_div(kblocks, s) * kblock_us +
+                        (s > 1 ? partial_us * s + 5.0 : 0.0);
     if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
   }
   return best;
@@ -675,6 +680,7 @@ int launch(const TcParams& p, const CUtensorMap& ta, const CUtensorMap& tb, int6
   }
   if (smem > 227 * 1024) return RAD_EUNSUPPORTED;
   const int grid = (int)std::max<int64_t>(1, std::min<int64_t>(max_units, num_sms()));
+  count_launch();
   kernel<<<grid, threads_for<AK>(), smem, s>>>(p, ta, tb);
   return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
 }
@@ -747,6 +753,7 @@ int tc_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H, 
     rc = make_map(&ta, st->values, st->values_ld, st->B, st->values_ld, 64);   // MN-major A: A_c is B x ld
     if (rc != RAD_OK) return rc;
     p.M = mmax; p.M_dev = st->nnz; p.row_idx = st->offsets;
+    count_launch();
     zero_f32_kernel<<<grid_z, 256, 0, s>>>(dW, st->D, H, ldw);
     rc = launch<kAMN, kBMN, kDw>(p, ta, tb, ceil_div(mmax, BM) * ceil_div(H, BN) * d.splits, s);
   } else {
@@ -760,6 +767,7 @@ int tc_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H, 
   if (d.splits > 1) {
     const int64_t work = p.M * (H / 4);
     const int grid = (int)std::max<int64_t>(1, std::min<int64_t>(ceil_div(work, 256), 148 * 16));
+    count_launch();
     dw_reduce_kernel<<<grid, 256, 0, s>>>(p.partial, d.partial_rows, d.splits, p.M, p.M_dev, H, p.row_idx, dW, ldw);
   }
   return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
