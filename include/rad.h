@@ -54,6 +54,8 @@ typedef enum { RAD_ACT_NONE = 0, RAD_ACT_RELU = 1, RAD_ACT_GELU = 2 } rad_act;
 #define RAD_TILE_ROWS   64     /* minibatch rows per tile                                    */
 #define RAD_TILE_COLS   128    /* layer-input columns per tile                               */
 #define RAD_VALUE_ALIGN 8      /* every tile's values start at a multiple of 8 elements      */
+#define RAD_TILE_WORDS  288    /* 32-bit words of index data per tile: 256 keep-bit words    */
+                               /* followed by 64 16-bit row offsets                          */
 
 /*
  * The mask (Sec. 3.2: a random P with E[P] = I; Sec. 4.3: "same sample" /
@@ -75,9 +77,13 @@ float    rad_scale(float p);            /* fl32(65536 / T)                      
  *
  * different-sample layout.  Rows are cut into slabs of RAD_TILE_ROWS, columns
  * into blocks of RAD_TILE_COLS; tile t = slab * ceil(D / 128) + block.
- *   keepbits : 256 words per tile, word (r * 4 + w) of tile t holds the keep bits
- *              of row slab*64 + r, columns block*128 + 32*w .. +31, LSB first.
- *              Bits of rows >= B or columns >= D are 0.
+ *   keepbits : RAD_TILE_WORDS words per tile.  Word (r * 4 + w), r < 64, w < 4, of
+ *              tile t holds the keep bits of row slab*64 + r, columns
+ *              block*128 + 32*w .. +31, LSB first; bits of rows >= B or columns
+ *              >= D are 0.  Words 256..287 hold 64 unsigned 16-bit numbers
+ *              (little endian, row r in half-word r): how many kept entries of
+ *              the tile lie in rows before r, i.e. where row r starts inside
+ *              the tile's values.
  *   values   : the kept entries of tile t, A[b,d] * scale rounded once to `dtype`,
  *              in (row, column) order, start at element offsets[t]; the tile is
  *              padded with zeros to a multiple of RAD_VALUE_ALIGN elements.

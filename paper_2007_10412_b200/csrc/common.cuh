@@ -17,7 +17,8 @@ typedef __nv_bfloat16 bf16;
 
 constexpr int kTileRows = RAD_TILE_ROWS;
 constexpr int kTileCols = RAD_TILE_COLS;
-constexpr int kTileWords = kTileRows * kTileCols / 32;   // 256 keep-bit words per tile
+constexpr int kBitWords = kTileRows * kTileCols / 32;    // 256 keep-bit words per tile
+constexpr int kTileWords = RAD_TILE_WORDS;               // plus 64 16-bit row offsets
 constexpr int kValueAlign = RAD_VALUE_ALIGN;
 
 // ---------------------------------------------------------------------------------------------

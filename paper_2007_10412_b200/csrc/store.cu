@@ -193,6 +193,8 @@ __global__ void __launch_bounds__(256) store_different_kernel(const StoreParams 
     const uint32_t ex = incl - (v0 + v1);
     s_rowoff[2 * lane] = ex;
     s_rowoff[2 * lane + 1] = ex + v0;
+    // row offsets travel with the keep bits: the dW kernel finds a row's values without a scan
+    p.keepbits[(int64_t)tile * kTileWords + kBitWords + lane] = ex | ((ex + v0) << 16);
     const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
     if (lane == 0) {
       s_total = total;

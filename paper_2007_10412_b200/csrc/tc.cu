@@ -9,9 +9,9 @@
 // One CTA per SM, persistent.  A CTA owns a 256 x 256 output tile held as two 128 x 256
 // accumulators that fill all 512 tensor-memory columns; per 64-deep K block it issues eight
 // 128x256x16 MMAs.  Operands arrive by TMA (128-byte swizzle, no multicast) through a 3-stage
-// mbarrier ring; for the different-sample dW the A operand is written by eight "expander" warps
+// mbarrier ring; for the different-sample dW the A operand is written by sixteen "expander" warps
 // instead.  Warp roles: 0 TMA producer, 1 MMA issuer and tensor-memory owner, 2-5 epilogue,
-// 6-13 expanders (sparse A only).  Long contractions can be split along K; partial tiles are
+// 6 producer of the compressed ring and 7-22 expanders (sparse A only).  Long contractions can be split along K; partial tiles are
 // summed in split order by a second kernel, so results are reproducible.
 // Every mbarrier wait is bounded: on expiry the CTA raises RAD_DEV_ETIMEOUT, all roles leave
 // their loops, tensor memory is released and the kernel returns.
@@ -42,6 +42,7 @@ struct TcParams {
   const int64_t* M_dev;      // same-sample dW: M = number of kept columns, read on the device
   int32_t splits;            // K splits (1: epilogue writes final results)
   int32_t num_stages;
+  int32_t comp_depth;        // sparse A: depth of the ring of compressed (index + values) buffers
   // sparse A (different-sample store)
   const bf16* values; const uint32_t* keepbits; const uint32_t* offsets;
   int64_t values_capacity; int32_t ncb; int32_t comp_cap;   // comp_cap: value bytes per half-stage
@@ -187,12 +188,15 @@ struct Schedule {
 
 // ---- shared memory layout -------------------------------------------------------------------------
 struct SmemCtl {
-  uint64_t full[4], empty[4], comp_full[4], tmem_full, tmem_empty;
+  uint64_t full[4], empty[4], comp_full[8], comp_empty[8], tmem_full, tmem_empty;
   uint32_t tmem_base;
   int abort_flag;
 };
 
-template <int AK> __host__ __device__ constexpr int threads_for() { return AK == kASparse ? 448 : 192; }
+constexpr int kIndexBytes = kTileWords * 4;   // keep bits + row offsets of one store tile (1152 B)
+constexpr int kExpanderWarps = 16;            // one thread per keep-bit word of the two halves
+constexpr int kFirstExpanderWarp = 7;        // warp 6 feeds the compressed ring
+template <int AK> __host__ __device__ constexpr int threads_for() { return AK == kASparse ? 32 * (kFirstExpanderWarp + kExpanderWarps) : 192; }
 
 template <int AK, int BKIND, int EPI>
 __global__ void __launch_bounds__(threads_for<AK>(), 1)
@@ -201,9 +205,11 @@ tc_gemm_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, const 
   // 1024-byte alignment for the 128-byte swizzle atoms
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int stages = p.num_stages;
-  const int comp_half = (AK == kASparse) ? (1024 + p.comp_cap) : 0;          // bits + values of one half
-  const int stage_bytes = (kAStageBytes + kBStageBytes + 2 * comp_half + 1023) & ~1023;   // swizzle atoms need 1024 B
-  SmemCtl* ctl = reinterpret_cast<SmemCtl*>(smem + (size_t)stages * stage_bytes);
+  const int comp_half = (AK == kASparse) ? (kIndexBytes + p.comp_cap) : 0;   // index data + values of one half
+  constexpr int stage_bytes = kAStageBytes + kBStageBytes;      // 64 KB: swizzle atoms stay 1024-byte aligned
+  const int comp_slot = 2 * comp_half;                           // compressed data of one K block (two halves)
+  uint8_t* comp_base = smem + (size_t)stages * stage_bytes;
+  SmemCtl* ctl = reinterpret_cast<SmemCtl*>(comp_base + (size_t)p.comp_depth * comp_slot);
   volatile int* abort_flag = &ctl->abort_flag;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -217,9 +223,12 @@ tc_gemm_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, const 
   const Schedule sched(m_rows, p.N, p.K, p.splits);
   if (tid == 0) {
     for (int s = 0; s < stages; ++s) {
-      mbar_init(smem_u32(&ctl->full[s]), AK == kASparse ? 1 + 8 : 1);
+      mbar_init(smem_u32(&ctl->full[s]), AK == kASparse ? 1 + kExpanderWarps : 1);
       mbar_init(smem_u32(&ctl->empty[s]), 1);
-      mbar_init(smem_u32(&ctl->comp_full[s]), 1);
+    }
+    for (int c = 0; c < p.comp_depth; ++c) {
+      mbar_init(smem_u32(&ctl->comp_full[c]), 1);
+      mbar_init(smem_u32(&ctl->comp_empty[c]), kExpanderWarps);
     }
     mbar_init(smem_u32(&ctl->tmem_full), 1);
     mbar_init(smem_u32(&ctl->tmem_empty), 128);
@@ -238,31 +247,13 @@ tc_gemm_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, const 
   const uint32_t smem_base = smem_u32(smem);
 
   if (warp == 0) {
-    // ===== TMA producer (one lane issues; for sparse A all lanes prefetch tile offsets) =====
+    // ===== TMA producer for the A and B tiles (one lane issues) =====
     int stage = 0;
     uint32_t phase = 0;
     bool ok = true;
     for (int64_t u = blockIdx.x; u < sched.units && ok; u += gridDim.x) {
       const Unit w = sched.unit(u);
-      uint32_t off_lo = 0, off_mid = 0, off_hi = 0;   // sparse: offsets of the 2 tiles of k-block (base + lane)
       for (int kb = w.kb0; kb < w.kb1; ++kb) {
-        if (AK == kASparse && ((kb - w.kb0) & 31) == 0) {
-          const int kbl = kb + lane;
-          if (kbl < w.kb1) {
-            const int64_t cb0 = w.m0 / kTileCols;
-            const int64_t t0 = (int64_t)kbl * p.ncb + cb0;
-            off_lo = __ldg(p.offsets + t0);
-            off_mid = __ldg(p.offsets + t0 + 1);
-            off_hi = (w.halves == 2) ? __ldg(p.offsets + t0 + 2) : off_mid;
-          }
-        }
-        uint32_t o0 = 0, o1 = 0, o2 = 0;
-        if (AK == kASparse) {
-          const int src = (kb - w.kb0) & 31;
-          o0 = __shfl_sync(0xffffffffu, off_lo, src);
-          o1 = __shfl_sync(0xffffffffu, off_mid, src);
-          o2 = __shfl_sync(0xffffffffu, off_hi, src);
-        }
         if (lane == 0) {
           ok = mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag);
           if (ok) {
@@ -286,24 +277,6 @@ tc_gemm_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, const 
             } else {
 #pragma unroll
               for (int c = 0; c < 4; ++c) tma_load_2d(sB + c * 8192, &tmB, (int)w.n0 + c * 64, k0, full);
-            }
-            if (AK == kASparse) {
-              // keep bits (1 KB per tile) and packed values of the one or two store tiles
-              const uint32_t cfull = smem_u32(&ctl->comp_full[stage]);
-              const uint32_t sC = sB + kBStageBytes;
-              const int64_t t0 = (int64_t)kb * p.ncb + w.m0 / kTileCols;
-              uint32_t vb0 = (o1 - o0) * 2u, vb1 = (o2 - o1) * 2u;
-              bool bad = false;
-              if (vb0 > (uint32_t)p.comp_cap || (int64_t)o1 > p.values_capacity) { vb0 = 0; bad = true; }
-              if (vb1 > (uint32_t)p.comp_cap || (int64_t)o2 > p.values_capacity) { vb1 = 0; bad = true; }
-              if (bad) raise_status(p.dev_status, RAD_DEV_ECAPACITY);
-              mbar_arrive_expect_tx(cfull, 1024u * w.halves + vb0 + (w.halves == 2 ? vb1 : 0u));
-              bulk_load(sC, p.keepbits + t0 * kTileWords, 1024, cfull);
-              if (vb0 != 0) bulk_load(sC + 1024, p.values + o0, vb0, cfull);
-              if (w.halves == 2) {
-                bulk_load(sC + comp_half, p.keepbits + (t0 + 1) * kTileWords, 1024, cfull);
-                if (vb1 != 0) bulk_load(sC + comp_half + 1024, p.values + o1, vb1, cfull);
-              }
             }
           }
         }
@@ -483,61 +456,129 @@ tc_gemm_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, const 
       mbar_arrive(smem_u32(&ctl->tmem_empty));
       unit_phase ^= 1u;
     }
+  } else if (AK == kASparse && warp == 6) {
+    // ===== producer of the compressed ring: keep bits + row offsets (1152 B) and packed values of
+    // the one or two store tiles of each K block.  It runs ahead of the A/B ring: a slot is free as
+    // soon as the expanders have read it, long before the MMAs of that K block retire. =====
+    int slot = 0;
+    uint32_t cphase = 0;
+    bool ok = true;
+    for (int64_t u = blockIdx.x; u < sched.units && ok; u += gridDim.x) {
+      const Unit w = sched.unit(u);
+      uint32_t off_lo = 0, off_mid = 0, off_hi = 0;   // tile offsets of K block (base + lane)
+      for (int kb = w.kb0; kb < w.kb1; ++kb) {
+        if (((kb - w.kb0) & 31) == 0) {
+          const int kbl = kb + lane;
+          if (kbl < w.kb1) {
+            const int64_t t0 = (int64_t)kbl * p.ncb + w.m0 / kTileCols;
+            off_lo = __ldg(p.offsets + t0);
+            off_mid = __ldg(p.offsets + t0 + 1);
+            off_hi = (w.halves == 2) ? __ldg(p.offsets + t0 + 2) : off_mid;
+          }
+        }
+        const int src = (kb - w.kb0) & 31;
+        const uint32_t o0 = __shfl_sync(0xffffffffu, off_lo, src);
+        const uint32_t o1 = __shfl_sync(0xffffffffu, off_mid, src);
+        const uint32_t o2 = __shfl_sync(0xffffffffu, off_hi, src);
+        if (lane == 0) {
+          ok = mbar_wait(smem_u32(&ctl->comp_empty[slot]), cphase ^ 1u, abort_flag);
+          if (ok) {
+            const uint32_t cfull = smem_u32(&ctl->comp_full[slot]);
+            const uint32_t sC = smem_u32(comp_base) + slot * comp_slot;
+            const int64_t t0 = (int64_t)kb * p.ncb + w.m0 / kTileCols;
+            uint32_t vb0 = (o1 - o0) * 2u, vb1 = (o2 - o1) * 2u;
+            bool bad = false;
+            if (vb0 > (uint32_t)p.comp_cap || (int64_t)o1 > p.values_capacity) { vb0 = 0; bad = true; }
+            if (vb1 > (uint32_t)p.comp_cap || (int64_t)o2 > p.values_capacity) { vb1 = 0; bad = true; }
+            if (bad) raise_status(p.dev_status, RAD_DEV_ECAPACITY);
+            mbar_arrive_expect_tx(cfull, (uint32_t)kIndexBytes * w.halves + vb0 + (w.halves == 2 ? vb1 : 0u));
+            bulk_load(sC, p.keepbits + t0 * kTileWords, kIndexBytes, cfull);
+            if (vb0 != 0) bulk_load(sC + kIndexBytes, p.values + o0, vb0, cfull);
+            if (w.halves == 2) {
+              bulk_load(sC + comp_half, p.keepbits + (t0 + 1) * kTileWords, kIndexBytes, cfull);
+              if (vb1 != 0) bulk_load(sC + comp_half + kIndexBytes, p.values + o1, vb1, cfull);
+            }
+          }
+        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) break;
+        if (++slot == p.comp_depth) { slot = 0; cphase ^= 1u; }
+      }
+    }
   } else if (AK == kASparse) {
     // ===== expanders: rebuild the A_hat tile (64 K rows x 256 columns, M-major, swizzled) =====
-    const int et = tid - 192;            // 0..255: keep-bit word et of each half (row et/4, word et%4)
-    const int ew = et >> 5;              // expander warp 0..7
-    const int r = et >> 2, wq = et & 3;
-    int stage = 0;
-    uint32_t phase = 0;
+    // One thread per keep-bit word: half h = columns 128h..128h+127 of the tile (one store tile),
+    // row r of the slab, columns 32*wq..32*wq+31 of that half.  The row's first value is given by
+    // the stored row offset; the words before this one in the row are counted with popc.
+    const int et = tid - 32 * kFirstExpanderWarp;            // 0..511
+    const int h = et >> 8, wi = et & 255;
+    const int r = wi >> 2, wq = wi & 3;
+    int stage = 0, slot = 0;
+    uint32_t phase = 0, cphase = 0;
     bool ok = true;
     for (int64_t u = blockIdx.x; u < sched.units && ok; u += gridDim.x) {
       const Unit w = sched.unit(u);
       for (int kb = w.kb0; kb < w.kb1; ++kb) {
-        ok = mbar_wait(smem_u32(&ctl->comp_full[stage]), phase, abort_flag);
+        ok = mbar_wait(smem_u32(&ctl->comp_full[slot]), cphase, abort_flag) &&
+             mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag);     // A tile of this stage is free
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
-        uint8_t* sA = smem + (size_t)stage * stage_bytes;
-        const uint8_t* sC = sA + kAStageBytes + kBStageBytes;
-        for (int h = 0; h < w.halves; ++h) {
-          const uint32_t* bits = reinterpret_cast<const uint32_t*>(sC + (size_t)h * comp_half);
-          const unsigned short* vals = reinterpret_cast<const unsigned short*>(sC + (size_t)h * comp_half + 1024);
-          const uint32_t word = bits[et];
-          const uint32_t cnt = __popc(word);
-          uint32_t incl = cnt;
-#pragma unroll
-          for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t nb = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += nb;
-          }
-          // kept entries before this warp's 32 words: every warp counts them itself, so the eight
-          // expander warps never wait on one another
-          uint32_t before = 0;
-          for (int j = 0; j < ew; ++j) before += __popc(bits[j * 32 + lane]);
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
-          uint32_t pos = before + incl - cnt;
-          // this thread's 32 columns: zero them, then drop the kept values in place
+        if (h < w.halves) {
+          uint8_t* sA = smem + (size_t)stage * stage_bytes;
+          const uint8_t* sC = comp_base + (size_t)slot * comp_slot + (size_t)h * comp_half;
+          const uint32_t* bits = reinterpret_cast<const uint32_t*>(sC);
+          const unsigned short* rowoff = reinterpret_cast<const unsigned short*>(sC + kBitWords * 4);
+          const unsigned short* vals = reinterpret_cast<const unsigned short*>(sC + kIndexBytes);
+          const uint4 rowbits = *reinterpret_cast<const uint4*>(bits + r * 4);
+          const uint32_t word = wq == 0 ? rowbits.x : wq == 1 ? rowbits.y : wq == 2 ? rowbits.z : rowbits.w;
+          uint32_t pos = rowoff[r];
+          if (wq > 0) pos += __popc(rowbits.x);
+          if (wq > 1) pos += __popc(rowbits.y);
+          if (wq > 2) pos += __popc(rowbits.z);
           uint8_t* rowp = sA + h * 16384 + (wq >> 1) * 8192 + r * 128;
           const int j0 = (wq & 1) * 4;
-#pragma unroll
-          for (int jj = 0; jj < 4; ++jj)
-            *reinterpret_cast<uint4*>(rowp + (((j0 + jj) ^ (r & 7)) << 4)) = make_uint4(0, 0, 0, 0);
-          uint32_t rest = word;
           const uint32_t limit = (uint32_t)p.comp_cap >> 1;
-          while (rest != 0) {
-            const int b = __ffs(rest) - 1;
-            rest &= rest - 1;
-            const unsigned short v = (pos < limit) ? vals[pos] : (unsigned short)0;
-            ++pos;
-            const int j = j0 + (b >> 3);
-            *reinterpret_cast<unsigned short*>(rowp + ((j ^ (r & 7)) << 4) + ((b & 7) << 1)) = v;
+          if (__popc(word) <= 10) {
+            // sparse word: zero this thread's 32 columns, then drop the kept values in place
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj)
+              *reinterpret_cast<uint4*>(rowp + (((j0 + jj) ^ (r & 7)) << 4)) = make_uint4(0, 0, 0, 0);
+            uint32_t rest = word;
+            while (rest != 0) {
+              const int b = __ffs(rest) - 1;
+              rest &= rest - 1;
+              const unsigned short v = (pos < limit) ? vals[pos] : (unsigned short)0;
+              ++pos;
+              const int j = j0 + (b >> 3);
+              *reinterpret_cast<unsigned short*>(rowp + ((j ^ (r & 7)) << 4) + ((b & 7) << 1)) = v;
+            }
+          } else {
+            // dense word: every column's value position follows from a popcount of the bits below
+            // it, so the 32 loads are independent; each 16-byte chunk is written once
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) {
+              uint32_t pk[4];
+#pragma unroll
+              for (int e = 0; e < 8; e += 2) {
+                const int b0 = jj * 8 + e;
+                const uint32_t p0 = pos + __popc(word & ((1u << b0) - 1u));
+                const uint32_t p1 = pos + __popc(word & ((2u << b0) - 1u));
+                const uint32_t v0 = ((word >> b0) & 1u) && p0 < limit ? vals[p0] : 0u;
+                const uint32_t v1 = ((word >> (b0 + 1)) & 1u) && p1 < limit ? vals[p1] : 0u;
+                pk[e >> 1] = v0 | (v1 << 16);
+              }
+              *reinterpret_cast<uint4*>(rowp + (((j0 + jj) ^ (r & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            }
           }
+          fence_proxy_async();
         }
-        fence_proxy_async();
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&ctl->full[stage]));
+        if (lane == 0) {
+          mbar_arrive(smem_u32(&ctl->full[stage]));
+          mbar_arrive(smem_u32(&ctl->comp_empty[slot]));
+        }
         if (++stage == stages) { stage = 0; phase ^= 1u; }
+        if (++slot == p.comp_depth) { slot = 0; cphase ^= 1u; }
       }
     }
   }
@@ -637,7 +678,7 @@ int choose_splits(int64_t m_tiles, int64_t n_tiles, int64_t kblocks) {
   return best;
 }
 
-struct DwPlan { int splits; int64_t partial_rows; int64_t bytes; int comp_cap; int stages; };
+struct DwPlan { int splits; int64_t partial_rows; int64_t bytes; int comp_cap; int stages; int comp_depth; };
 
 DwPlan plan_dw(const rad_store* st, int64_t H) {
   DwPlan d;
@@ -648,6 +689,7 @@ DwPlan plan_dw(const rad_store* st, int64_t H) {
     d.partial_rows = round_up(std::min(st->values_ld, round_up(st->D, 8)), BM);
     d.comp_cap = 0;
     d.stages = 3;
+    d.comp_depth = 0;
   } else {
     m_expect = st->D;
     d.partial_rows = round_up(st->D, BM);
@@ -656,8 +698,12 @@ DwPlan plan_dw(const rad_store* st, int64_t H) {
     int64_t cap = (int64_t)(n * pe + 8.0 * std::sqrt(n * pe * (1.0 - pe)) + 16.0);
     cap = std::min<int64_t>(round_up(cap, 8), (int64_t)n) * 2;
     d.comp_cap = (int)round_up(cap, 128);
-    const int stage_bytes = (int)round_up(kAStageBytes + kBStageBytes + 2 * (1024 + d.comp_cap), 1024);
-    d.stages = std::min(3, (int)((227 * 1024 - 2048) / stage_bytes));
+    // shared memory: 64 KB per A/B stage plus a ring of compressed slots, at least one deeper than
+    // the A/B ring when it fits
+    const int64_t budget = 227 * 1024 - 2048 - (int64_t)sizeof(SmemCtl);
+    const int64_t slot = 2 * (kIndexBytes + d.comp_cap);
+    d.stages = (3 * 65536 + 3 * slot <= budget) ? 3 : 2;
+    d.comp_depth = (int)std::max<int64_t>(2, std::min<int64_t>(6, (budget - d.stages * 65536) / slot));
   }
   d.splits = choose_splits(ceil_div(m_expect, BM), ceil_div(H, BN), kblocks);
   d.bytes = d.splits > 1 ? (int64_t)d.splits * d.partial_rows * H * 4 : 0;
@@ -666,9 +712,9 @@ DwPlan plan_dw(const rad_store* st, int64_t H) {
 
 template <int AK, int BKIND, int EPI>
 int launch(const TcParams& p, const CUtensorMap& ta, const CUtensorMap& tb, int64_t max_units, cudaStream_t s) {
-  const int comp_half = (AK == kASparse) ? (1024 + p.comp_cap) : 0;
-  const int stage_bytes = (int)round_up(kAStageBytes + kBStageBytes + 2 * comp_half, 1024);
-  const size_t smem = (size_t)p.num_stages * stage_bytes + sizeof(SmemCtl) + 1024;
+  const int comp_half = (AK == kASparse) ? (kIndexBytes + p.comp_cap) : 0;
+  const size_t smem = (size_t)p.num_stages * (kAStageBytes + kBStageBytes) + (size_t)p.comp_depth * 2 * comp_half +
+                      sizeof(SmemCtl) + 1024;
   auto kernel = tc_gemm_kernel<AK, BKIND, EPI>;
   static bool configured = false;
   static size_t configured_smem = 0;
@@ -744,7 +790,7 @@ int tc_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H, 
   int rc = make_map(&tb, dZ, H, st->B, ldz, 64);      // MN-major B: box 64 (N = h) x 64 K rows (b)
   if (rc != RAD_OK) return rc;
   TcParams p = {};
-  p.N = H; p.K = st->B; p.splits = d.splits; p.num_stages = d.stages;
+  p.N = H; p.K = st->B; p.splits = d.splits; p.num_stages = d.stages; p.comp_depth = d.comp_depth;
   p.out_dw = dW; p.ld_dw = ldw; p.dw_rows = st->D; p.partial = static_cast<float*>(workspace); p.partial_rows = d.partial_rows;
   p.dev_status = dev_status;
   const int grid_z = (int)std::min<int64_t>(ceil_div(st->D * H / 4, 256), 148 * 16);

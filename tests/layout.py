@@ -25,6 +25,8 @@ def tile_major(st):
             sub = mask[s * TILE_ROWS:(s + 1) * TILE_ROWS, c * TILE_COLS:(c + 1) * TILE_COLS]
             m[:sub.shape[0], :sub.shape[1]] = sub
             bits.append(rad.pack_bits(m).reshape(-1))
+            rowoff = np.concatenate([[0], np.cumsum(m.sum(axis=1))[:-1]]).astype(np.uint16)
+            bits.append(rowoff.view(np.uint32))
             v = dense[s * TILE_ROWS:(s + 1) * TILE_ROWS, c * TILE_COLS:(c + 1) * TILE_COLS][sub]
             pad = (-v.size) % ALIGN
             vals.append(np.concatenate([v, np.zeros(pad, np.float32)]))

@@ -44,7 +44,7 @@ def test_host_only_entry_points():
     assert b.rad_keep_threshold(0.0) == 0 and b.rad_keep_threshold(1.5) == 0
     sz = b.rad_store_size_query("different", "bf16", 65536, 8192, 0.1)
     ntiles = 1024 * 64
-    assert sz.keepbits_words == ntiles * 256 and sz.offsets_words == ntiles + 1
+    assert sz.keepbits_words == ntiles * 288 and sz.offsets_words == ntiles + 1
     assert sz.relubits_words == 65536 * 256
     assert sz.values_worst == 65536 * 8192 + 7 * ntiles
     assert 0.1 * 65536 * 8192 < sz.values_typical < 0.102 * 65536 * 8192
