@@ -70,11 +70,13 @@ __device__ __forceinline__ uint32_t philox_keep8(uint32_t group, uint32_t row, u
                                                  const PhiloxKeys& ks, uint32_t T) {
   uint32_t w[4];
   philox4x32_10(group, row, c2, c3, ks, w);
+  // lane - T is negative exactly when lane < T (both below 2^17); a funnel shift moves each sign
+  // bit into the mask, last column first
   uint32_t m = 0;
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    m |= ((w[j] & 0xffffu) < T ? 1u : 0u) << (2 * j);
-    m |= ((w[j] >> 16) < T ? 1u : 0u) << (2 * j + 1);
+  for (int j = 3; j >= 0; --j) {
+    m = __funnelshift_l((w[j] >> 16) - T, m, 1);
+    m = __funnelshift_l((w[j] & 0xffffu) - T, m, 1);
   }
   return m;
 }

@@ -121,6 +121,16 @@ template <typename T> __device__ __forceinline__ uint32_t positive8(const Raw8<T
   return m;
 }
 
+// Four lanes each hold one byte per item (4 items); afterwards lane k of the four holds the
+// 32-bit word of item k: byte j = what lane j held for item k.
+__device__ __forceinline__ uint32_t transpose4x4_bytes(uint32_t v, int k) {
+  uint32_t x = __shfl_xor_sync(0xffffffffu, v, 1);
+  v = (k & 1) ? __byte_perm(v, x, 0x3715) : __byte_perm(v, x, 0x6240);
+  x = __shfl_xor_sync(0xffffffffu, v, 2);
+  v = (k & 2) ? __byte_perm(v, x, 0x3276) : __byte_perm(v, x, 0x5410);
+  return v;
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256) store_different_kernel(const StoreParams p, const PhiloxKeys ks) {
   __shared__ uint32_t s_rowcnt[kTileRows];
@@ -143,40 +153,41 @@ __global__ void __launch_bounds__(256) store_different_kernel(const StoreParams 
   const T* Abase = static_cast<const T*>(p.A);
 
   Raw8<T> raw[4];
-  uint32_t mask[4], pre[4];
+  uint32_t masks = 0, relus = 0, counts = 0;     // one byte per item: keep bits, ReLU bits, kept count
 #pragma unroll
   for (int it = 0; it < 4; ++it) {
-    const int r = warp * 8 + it * 2 + half;
-    const int64_t row = slab * kTileRows + r;
-    const bool live = (row < p.B) && (nvalid > 0);
-    uint32_t m = 0, rb = 0;
-    if (live) {
+    const int64_t row = slab * kTileRows + warp * 8 + it * 2 + half;
+    if (row < p.B && nvalid > 0) {
       load8<T>(Abase + row * p.lda, col0, nvalid, p.vec_ok != 0, raw[it]);
-      m = philox_keep8((uint32_t)(col0 >> 3), (uint32_t)row, p.c2, p.c3, ks, p.T) & ((1u << nvalid) - 1u);
-      if (p.relubits != nullptr) rb = positive8(raw[it]) & ((1u << nvalid) - 1u);
+      const uint32_t m = philox_keep8((uint32_t)(col0 >> 3), (uint32_t)row, p.c2, p.c3, ks, p.T) & ((1u << nvalid) - 1u);
+      masks |= m << (8 * it);
+      counts |= __popc(m) << (8 * it);
+      if (p.relubits != nullptr) relus |= (positive8(raw[it]) & ((1u << nvalid) - 1u)) << (8 * it);
     }
-    mask[it] = m;
-    // exclusive prefix of the kept count inside the row (16 lanes per row)
-    const uint32_t c = __popc(m);
-    uint32_t incl = c;
+  }
+  // exclusive prefix of the kept count inside each row (16 lanes per row); the four items scan as
+  // one word, a byte each (a row holds at most 128 kept entries)
+  uint32_t incl = counts;
 #pragma unroll
-    for (int o = 1; o < 16; o <<= 1) {
-      const uint32_t n = __shfl_up_sync(0xffffffffu, incl, o, 16);
-      if (cg >= o) incl += n;
-    }
-    pre[it] = incl - c;
-    if (cg == 15) s_rowcnt[r] = incl;
-    // four lanes make one 32-bit word of keep bits (and of ReLU bits)
-    uint32_t kw = m << (8 * (cg & 3));
-    kw |= __shfl_xor_sync(0xffffffffu, kw, 1);
-    kw |= __shfl_xor_sync(0xffffffffu, kw, 2);
-    uint32_t rw = rb << (8 * (cg & 3));
-    rw |= __shfl_xor_sync(0xffffffffu, rw, 1);
-    rw |= __shfl_xor_sync(0xffffffffu, rw, 2);
-    if ((cg & 3) == 0) {
-      p.keepbits[(int64_t)tile * kTileWords + r * 4 + (cg >> 2)] = kw;
+  for (int o = 1; o < 16; o <<= 1) {
+    const uint32_t n = __shfl_up_sync(0xffffffffu, incl, o, 16);
+    if (cg >= o) incl += n;
+  }
+  const uint32_t pres = incl - counts;
+  if (cg == 15) {
+#pragma unroll
+    for (int it = 0; it < 4; ++it) s_rowcnt[warp * 8 + it * 2 + half] = (incl >> (8 * it)) & 0xffu;
+  }
+  {
+    // four lanes make one 32-bit word of keep bits (and of ReLU bits) per item
+    const int k = cg & 3;
+    const int r = warp * 8 + k * 2 + half;
+    p.keepbits[(int64_t)tile * kTileWords + r * 4 + (cg >> 2)] = transpose4x4_bytes(masks, k);
+    if (p.relubits != nullptr) {
+      const uint32_t rw = transpose4x4_bytes(relus, k);
+      const int64_t row = slab * kTileRows + r;
       const int word = cb * 4 + (cg >> 2);
-      if (p.relubits != nullptr && row < p.B && word < p.w32) p.relubits[row * p.w32 + word] = rw;
+      if (row < p.B && word < p.w32) p.relubits[row * p.w32 + word] = rw;
     }
   }
   __syncthreads();
@@ -212,8 +223,8 @@ __global__ void __launch_bounds__(256) store_different_kernel(const StoreParams 
 #pragma unroll
   for (int it = 0; it < 4; ++it) {
     const int r = warp * 8 + it * 2 + half;
-    uint32_t pos = s_rowoff[r] + pre[it];
-    const uint32_t m = mask[it];
+    uint32_t pos = s_rowoff[r] + ((pres >> (8 * it)) & 0xffu);
+    const uint32_t m = (masks >> (8 * it)) & 0xffu;
     if (m != 0) {
 #pragma unroll
       for (int i = 0; i < 8; ++i)
