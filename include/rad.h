@@ -40,6 +40,7 @@ extern "C" {
 #define RAD_EUNSUPPORTED (-2)  /* not an sm_100 device, or an alignment rule is not met      */
 #define RAD_ECUDA        (-3)  /* a CUDA runtime or driver call failed                       */
 #define RAD_EWORKSPACE   (-4)  /* workspace_bytes is smaller than the matching *_workspace   */
+#define RAD_ELIMIT       (-5)  /* the problem is larger than a fixed built-in buffer          */
 
 #define RAD_DEV_OK        0
 #define RAD_DEV_ECAPACITY 1    /* the compact store did not fit values_capacity / values_ld  */
@@ -141,6 +142,37 @@ int rad_store_size_query(int32_t variant, int32_t dtype, int64_t B, int64_t D, f
 int rad_linear_forward_store(const void* A /* device */, int64_t lda, const rad_store* st /* host */,
                              void* workspace /* device */, int64_t workspace_bytes,
                              int32_t* dev_status /* device or NULL */, void* stream);
+
+/*
+ * rad_linear_forward_store without a workspace argument (the paper has no
+ * counterpart: this entry point exists for the sake of callers, not of the
+ * method).  It is meant for programs that must not allocate device memory
+ * while they run: a trainer that hands every byte of the GPU to its own pool
+ * at start-up and treats a later cudaMalloc as a bug, or a step loop in which
+ * an allocation would stall the device.  Such a caller still owns A and every
+ * buffer of `st`, but has nowhere to take the kernel's scratch from, so the
+ * scratch (one claim counter and one 8-byte word per tile) lives in a
+ * fixed array inside the library: 256 + 8 * RAD_STATIC_STORE_MAX_TILES bytes
+ * (about 1 MiB), held by every GPU that has loaded the library until the
+ * process exits.  The call itself allocates nothing and frees nothing.
+ *
+ *   - different-sample stores only (the same-sample path of
+ *     rad_linear_forward_store needs no scratch; pass it a NULL workspace);
+ *     RAD_EUNSUPPORTED otherwise.
+ *   - ceil(B / 64) * ceil(D / 128) must not exceed RAD_STATIC_STORE_MAX_TILES,
+ *     else RAD_ELIMIT and nothing is enqueued.
+ *   - The first call on a device looks up the array's device address (with
+ *     that device current) and remembers it; make that first call outside any
+ *     stream capture.
+ *   - All calls on one device share the array.  Each call clears the part it
+ *     uses before its kernel runs, in stream order, so back-to-back calls on
+ *     one stream are fine; two calls whose kernels may overlap on the GPU
+ *     (different streams, no dependency) race on it and give wrong offsets.
+ * Outputs are bit for bit those of rad_linear_forward_store.
+ */
+#define RAD_STATIC_STORE_MAX_TILES 131072
+int rad_linear_forward_store_static(const void* A /* device */, int64_t lda, const rad_store* st /* host */,
+                                    int32_t* dev_status /* device or NULL */, void* stream);
 
 /* Scratch rad_linear_weight_grad needs for this store and H (host only). */
 int rad_weight_grad_workspace(const rad_store* st /* host */, int64_t H, int64_t* bytes /* host */);

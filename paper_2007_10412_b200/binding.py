@@ -56,7 +56,7 @@ class rad_step_stats(C.Structure):
 
 
 EXPORTS = ["rad_keep_threshold", "rad_effective_p", "rad_scale", "rad_store_size_query",
-           "rad_linear_forward_store", "rad_weight_grad_workspace", "rad_linear_weight_grad",
+           "rad_linear_forward_store", "rad_linear_forward_store_static", "rad_weight_grad_workspace", "rad_linear_weight_grad",
            "rad_linear_forward", "rad_softmax_xent", "rad_input_grad_workspace", "rad_linear_input_grad",
            "rad_mlp_workspace", "rad_mlp_step", "rad_launch_count", "rad_strerror", "rad_version"]
 
@@ -83,6 +83,7 @@ def lib():
         i32, i64, f32, vp = C.c_int32, C.c_int64, C.c_float, C.c_void_p
         L.rad_store_size_query.argtypes = [i32, i32, i64, i64, f32, C.POINTER(rad_store_sizes)]
         L.rad_linear_forward_store.argtypes = [vp, i64, C.POINTER(rad_store), vp, i64, vp, vp]
+        L.rad_linear_forward_store_static.argtypes = [vp, i64, C.POINTER(rad_store), vp, vp]
         L.rad_weight_grad_workspace.argtypes = [C.POINTER(rad_store), i64, C.POINTER(i64)]
         L.rad_linear_weight_grad.argtypes = [C.POINTER(rad_store), vp, i64, i64, vp, i64, vp, i64, vp, vp]
         L.rad_linear_forward.argtypes = [i32, i32, i64, i64, i64, vp, i64, vp, i64, vp, vp, i64, vp, i64,
@@ -183,6 +184,21 @@ def rad_linear_forward_store(A, store, dev_status=None):
     _check(lib().rad_linear_forward_store(_ptr(A), A.stride(0), C.byref(store.c), _ptr(store.workspace),
                                           store.workspace.numel(), _ptr(dev_status), _stream()),
            "rad_linear_forward_store")
+
+
+STATIC_STORE_MAX_TILES = 131072
+
+
+def rad_linear_forward_store_static(A, store, dev_status=None):
+    """The different-sample store for callers that may not allocate device memory while running.
+
+    Same inputs and outputs as rad_linear_forward_store, but the kernel's scratch comes from a
+    fixed array inside the library (at most STATIC_STORE_MAX_TILES tiles of 64 x 128), so nothing
+    is allocated by the call; `store.workspace` is not used.  Calls on one device share that array:
+    issue them on one stream, or otherwise ordered, never concurrently.
+    """
+    _check(lib().rad_linear_forward_store_static(_ptr(A), A.stride(0), C.byref(store.c), _ptr(dev_status),
+                                                 _stream()), "rad_linear_forward_store_static")
 
 
 def rad_weight_grad_workspace(store, H):

@@ -117,6 +117,7 @@ extern "C" const char* rad_strerror(int code) {
     case RAD_EUNSUPPORTED: return "unsupported device or alignment";
     case RAD_ECUDA: return "CUDA call failed";
     case RAD_EWORKSPACE: return "workspace too small";
+    case RAD_ELIMIT: return "problem larger than the built-in scratch buffer";
     case RAD_DEV_ECAPACITY: return "device: compact store capacity exceeded";
     case RAD_DEV_ETIMEOUT: return "device: bounded wait expired";
     case RAD_DEV_EINTERNAL: return "device: index out of range, access skipped";

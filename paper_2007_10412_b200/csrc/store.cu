@@ -537,3 +537,73 @@ extern "C" int rad_linear_forward_store(const void* A, int64_t lda, const rad_st
   RAD_CUDA_TRY(cudaGetLastError());
   return RAD_OK;
 }
+
+// ---- the store without a caller-provided workspace ------------------------------------------------
+// Scratch of the different-sample kernel for callers that cannot allocate: a claim counter (first
+// 256 bytes) and one status word per tile.  The name below is only a handle in host code; the
+// device address is looked up once per device.
+static __device__ __align__(256) unsigned char g_static_store_scratch[256 + 8 * RAD_STATIC_STORE_MAX_TILES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_ptr[kMaxDevices] = {};
+
+int static_scratch_address(void** out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return RAD_ECUDA;
+  if (dev < 0 || dev >= kMaxDevices) return RAD_EUNSUPPORTED;
+  if (g_static_scratch_ptr[dev] == nullptr) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_store_scratch) != cudaSuccess || ptr == nullptr) return RAD_ECUDA;
+    g_static_scratch_ptr[dev] = ptr;
+  }
+  *out = g_static_scratch_ptr[dev];
+  return RAD_OK;
+}
+}  // namespace
+
+extern "C" int rad_linear_forward_store_static(const void* A, int64_t lda, const rad_store* st,
+                                               int32_t* dev_status, void* stream) {
+  if (A == nullptr || st == nullptr) return RAD_EINVAL;
+  if (st->B <= 0 || st->D <= 0 || lda < st->D) return RAD_EINVAL;
+  if (st->variant != RAD_DIFFERENT_SAMPLE) return RAD_EUNSUPPORTED;
+  if (st->dtype != RAD_F32 && st->dtype != RAD_BF16) return RAD_EINVAL;
+  if (st->values == nullptr || st->keepbits == nullptr || st->offsets == nullptr || st->nnz == nullptr)
+    return RAD_EINVAL;
+  const uint32_t T = keep_threshold_host(st->p);
+  if (T == 0) return RAD_EINVAL;
+  if ((double)st->B * (double)st->D >= 4294967296.0 * 0.75) return RAD_EINVAL;
+  if (((uintptr_t)st->values & 15) != 0) return RAD_EUNSUPPORTED;
+  const int64_t ntiles = ceil_div(st->B, kTileRows) * ceil_div(st->D, kTileCols);
+  if (ntiles > RAD_STATIC_STORE_MAX_TILES) return RAD_ELIMIT;
+  int rc = check_device();
+  if (rc != RAD_OK) return rc;
+  void* scratch = nullptr;
+  rc = static_scratch_address(&scratch);
+  if (rc != RAD_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t esz = st->dtype == RAD_BF16 ? 2 : 4;
+  const PhiloxKeys ks = philox_expand_key(st->seed);
+  StoreParams p;
+  p.A = A; p.lda = lda; p.B = st->B; p.D = st->D;
+  p.ncb = (int32_t)ceil_div(st->D, kTileCols);
+  p.ntiles = (int32_t)ntiles;
+  p.T = T; p.scale = 65536.0f / (float)T;
+  p.c2 = counter_word2(st->layer, RAD_DIFFERENT_SAMPLE); p.c3 = st->step;
+  p.values = st->values; p.capacity = st->values_capacity;
+  p.keepbits = st->keepbits; p.offsets = st->offsets; p.nnz = st->nnz;
+  p.relubits = st->relubits; p.w32 = (int32_t)ceil_div(st->D, 32);
+  p.ticket = static_cast<uint32_t*>(scratch);
+  p.status = reinterpret_cast<uint64_t*>(static_cast<char*>(scratch) + 256);
+  p.dev_status = dev_status;
+  p.vec_ok = (((uintptr_t)A & 15) == 0 && (lda * esz) % 16 == 0) ? 1 : 0;
+  // the array keeps what the last call left: the counter and this call's status words start at zero
+  RAD_CUDA_TRY(cudaMemsetAsync(scratch, 0, 256 + 8 * (size_t)ntiles, s));
+  count_launch();
+  if (st->dtype == RAD_BF16)
+    store_different_kernel<bf16><<<p.ntiles, 256, 0, s>>>(p, ks);
+  else
+    store_different_kernel<float><<<p.ntiles, 256, 0, s>>>(p, ks);
+  RAD_CUDA_TRY(cudaGetLastError());
+  return RAD_OK;
+}
