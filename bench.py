@@ -101,6 +101,22 @@ def run_reference(args):
 # --------------------------------------------------------------------------------------------
 # our arm
 # --------------------------------------------------------------------------------------------
+def max_over_ranks(ms, device="cpu"):
+    """Slowest rank's time: every rank contributes its own device time, all get the maximum."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world, batch_per_rank, steps, ms_total):
+    """Samples per second of the whole job: all ranks' samples over the slowest rank's time."""
+    return world * batch_per_rank * steps / (ms_total / 1e3)
+
+
 class ClockSampler:
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -311,13 +327,10 @@ def run_ours(args):
     launches = (rad.rad_launch_count() - launches0) // max(args.steps, 1)
     clocks = sampler.stop()
     ms_total = t_start.elapsed_time(t_stop)
-    if world > 1:
-        t = torch.tensor([ms_total], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = t.item()
+    ms_total = max_over_ranks(ms_total, "cuda")
     assert lw.status.item() == 0, f"device status {lw.status.item()}"
     ms_step = ms_total / args.steps
-    value = world * B * args.steps / (ms_total / 1e3)
+    value = whole_job_value(world, B, args.steps, ms_total)
 
     # per-family device time inside the timed region, and the roofline of the dominant kernel
     fam = lw.family_ms()
@@ -390,12 +403,9 @@ def run_ours(args):
     e1.record()
     barrier()
     e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3 if world == 1 else 0.0)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = t.item()
+    e2e_ms = max_over_ranks(e2e_ms, "cuda")
     assert ctx.dev_status.item() == 0
-    e2e = dict(value=world * B * args.steps / (e2e_ms / 1e3), unit=UNIT,
+    e2e = dict(value=whole_job_value(world, B, args.steps, e2e_ms), unit=UNIT,
                h2d_bytes_per_step=Xh.numel() * 2 + yh.numel() * 4, d2h_bytes_per_step=4,
                ms_per_step=round(e2e_ms / args.steps, 3), api="rad_mlp_step", last_loss=round(loss, 5))
 
