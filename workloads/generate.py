@@ -68,3 +68,28 @@ def layer_inputs(B, D, H, dtype="f32", x_dist="normal", seed=1234, relu_like=Fal
     if dtype == "bf16":
         A, dZ = to_bf16_grid(A), to_bf16_grid(dZ)
     return A, dZ
+
+
+def irnn_inputs(batch, steps, hidden=100, classes=10, seed=1234, identity=True):
+    """Inputs of the sequential-pixel IRNN (paper, App. A, "RNN training details"): x in [0, 1) fed
+    one scalar per step, recurrent matrix initialised to the identity, input and output weights
+    N(0, 0.001) (read as standard deviation 0.001), zero biases.  identity=False draws a random
+    recurrent matrix of spectral norm about 0.9 and larger weights, so that tests exercise every term.
+    """
+    rng = np.random.default_rng(seed)
+    x = rng.random((batch, steps), dtype=np.float32)
+    labels = uniform_labels(rng, batch, classes)
+    if identity:
+        W_hh = np.eye(hidden, dtype=np.float32)
+        W_ih = rng.standard_normal(hidden, dtype=np.float32) * np.float32(0.001)
+        W_out = rng.standard_normal((hidden, classes), dtype=np.float32) * np.float32(0.001)
+        b_ih = np.zeros(hidden, np.float32)
+        b_hh = np.zeros(hidden, np.float32)
+    else:
+        W_hh = rng.standard_normal((hidden, hidden), dtype=np.float32) * np.float32(0.45 / np.sqrt(hidden))
+        W_ih = rng.standard_normal(hidden, dtype=np.float32) * np.float32(0.5)
+        W_out = rng.standard_normal((hidden, classes), dtype=np.float32) * np.float32(0.3)
+        b_ih = rng.standard_normal(hidden, dtype=np.float32) * np.float32(0.1)
+        b_hh = rng.standard_normal(hidden, dtype=np.float32) * np.float32(0.1)
+    b_out = np.zeros(classes, np.float32)
+    return x, labels, W_ih, b_ih, W_hh, b_hh, W_out, b_out
