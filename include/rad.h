@@ -276,6 +276,38 @@ int rad_mlp_step(const rad_mlp_desc* net /* host */, const void* X, const int32_
                  void* workspace, int64_t workspace_bytes,
                  int32_t* dev_status, void* stream);
 
+/*
+ * One training step of a ReLU recurrent net fed one scalar per time step (the paper's IRNN,
+ * App. A "Architectures Used"): h_t = relu(x_t W_ih + b_ih + h_{t-1} W_hh + b_hh), h_0 = 0,
+ * logits = h_T W_out + b_out, softmax cross-entropy.  RAD as in Sec. 4.3 / App. A: the hidden
+ * state entering step t is stored through the mask of (seed, layer 0, step0 + t), a fresh sample
+ * every step; the state entering the output layer through (seed, layer 1, step0); the scalar
+ * inputs and the softmax input are kept whole; ReLU derivatives take one bit.  dW_hh and dW_out
+ * come from the stores, everything else is exact.  float32 only, Hd <= 128.
+ *   x device B x T; labels device int32[B]; W_ih, b_ih, b_hh device float32[Hd];
+ *   W_hh device Hd x Hd (row = input unit, column = output unit); W_out device Hd x C; b_out [C].
+ *   dW_ih, db (gradient of b_ih and of b_hh) device [Hd]; dW_hh device Hd x Hd; dW_out Hd x C;
+ *   db_out [C]; loss device float32[1].
+ *   nnz_out device int64[2] or NULL: kept hidden entries over all steps, kept entries of h_T.
+ * If a row keeps more entries than its reserved share (mean + 8 sigma), RAD_DEV_ECAPACITY is raised.
+ */
+typedef struct rad_irnn_desc {
+  int64_t  B, T, Hd, C;
+  int32_t  variant;           /* rad_variant */
+  float    p;
+  uint64_t seed;
+  uint32_t step0;             /* added to the time index in the Philox counter */
+} rad_irnn_desc;
+
+int rad_irnn_workspace(const rad_irnn_desc* net /* host */, int64_t* bytes /* host */,
+                       rad_step_stats* stats /* host or NULL */);
+int rad_irnn_step(const rad_irnn_desc* net /* host */, const float* x, const int32_t* labels,
+                  const float* W_ih, const float* b_ih, const float* W_hh, const float* b_hh,
+                  const float* W_out, const float* b_out,
+                  float* dW_ih, float* db, float* dW_hh, float* dW_out, float* db_out, float* loss,
+                  int64_t* nnz_out, void* workspace, int64_t workspace_bytes,
+                  int32_t* dev_status, void* stream);
+
 /* Kernels this library has launched since it was loaded (host-side tally; memsets not counted). */
 int64_t rad_launch_count(void);
 

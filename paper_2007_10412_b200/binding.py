@@ -50,6 +50,11 @@ class rad_mlp_desc(C.Structure):
                 ("seed", C.c_uint64)]
 
 
+class rad_irnn_desc(C.Structure):
+    _fields_ = [("B", C.c_int64), ("T", C.c_int64), ("Hd", C.c_int64), ("C", C.c_int64), ("variant", C.c_int32),
+                ("p", C.c_float), ("seed", C.c_uint64), ("step0", C.c_uint32)]
+
+
 class rad_step_stats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in ("value_bytes", "index_bytes", "relu_bytes", "preact_bytes",
                                          "unsampled_bytes", "full_backprop_bytes")]
@@ -58,7 +63,7 @@ class rad_step_stats(C.Structure):
 EXPORTS = ["rad_keep_threshold", "rad_effective_p", "rad_scale", "rad_store_size_query",
            "rad_linear_forward_store", "rad_linear_forward_store_static", "rad_weight_grad_workspace", "rad_linear_weight_grad",
            "rad_linear_forward", "rad_softmax_xent", "rad_input_grad_workspace", "rad_linear_input_grad",
-           "rad_mlp_workspace", "rad_mlp_step", "rad_launch_count", "rad_strerror", "rad_version"]
+           "rad_mlp_workspace", "rad_mlp_step", "rad_irnn_workspace", "rad_irnn_step", "rad_launch_count", "rad_strerror", "rad_version"]
 
 _lib = None
 
@@ -93,6 +98,8 @@ def lib():
         L.rad_linear_input_grad.argtypes = [i32, i64, i64, i64, vp, i64, vp, i64, vp, vp, i64, vp, i64, vp,
                                             vp, i64, vp, vp]
         L.rad_mlp_workspace.argtypes = [C.POINTER(rad_mlp_desc), C.POINTER(i64), C.POINTER(rad_step_stats)]
+        L.rad_irnn_workspace.argtypes = [C.POINTER(rad_irnn_desc), C.POINTER(i64), C.POINTER(rad_step_stats)]
+        L.rad_irnn_step.argtypes = [C.POINTER(rad_irnn_desc)] + [vp] * 15 + [vp, i64, vp, vp]
         L.rad_mlp_step.argtypes = [C.POINTER(rad_mlp_desc), vp, vp, C.POINTER(vp), C.POINTER(vp),
                                    C.POINTER(vp), C.POINTER(vp), vp, vp, vp, i64, vp, vp]
         for name in EXPORTS:
@@ -286,4 +293,33 @@ def rad_mlp_step(ctx, X, labels, Ws, bs, seed=0, step=0):
     _check(lib().rad_mlp_step(C.byref(ctx.desc), _ptr(X), _ptr(labels), W, b, ctx._dW, ctx._db,
                               _ptr(ctx.loss), _ptr(ctx.nnz), _ptr(ctx.workspace), ctx.workspace.numel(),
                               _ptr(ctx.dev_status), _stream()), "rad_mlp_step")
+    return ctx
+
+
+class IRNNStep:
+    """Owns the workspace and gradient buffers of rad_irnn_step for one shape."""
+
+    def __init__(self, B, T, hidden, classes, variant="different", p=0.1, device="cuda"):
+        self.desc = rad_irnn_desc(B, T, hidden, classes, VARIANTS[variant], p, 0, 0)
+        nbytes = C.c_int64(0)
+        self.stats = rad_step_stats()
+        _check(lib().rad_irnn_workspace(C.byref(self.desc), C.byref(nbytes), C.byref(self.stats)), "rad_irnn_workspace")
+        f32 = dict(dtype=torch.float32, device=device)
+        self.workspace = torch.empty(nbytes.value, dtype=torch.uint8, device=device)
+        self.dW_ih, self.db = torch.empty(hidden, **f32), torch.empty(hidden, **f32)
+        self.dW_hh, self.dW_out = torch.empty(hidden, hidden, **f32), torch.empty(hidden, classes, **f32)
+        self.db_out, self.loss = torch.empty(classes, **f32), torch.zeros(1, **f32)
+        self.nnz = torch.zeros(2, dtype=torch.int64, device=device)
+        self.dev_status = torch.zeros(1, dtype=torch.int32, device=device)
+
+    def __call__(self, x, labels, W_ih, b_ih, W_hh, b_hh, W_out, b_out, seed=0, step0=0):
+        return rad_irnn_step(self, x, labels, W_ih, b_ih, W_hh, b_hh, W_out, b_out, seed, step0)
+
+
+def rad_irnn_step(ctx, x, labels, W_ih, b_ih, W_hh, b_hh, W_out, b_out, seed=0, step0=0):
+    ctx.desc.seed, ctx.desc.step0 = seed, step0
+    _check(lib().rad_irnn_step(C.byref(ctx.desc), _ptr(x), _ptr(labels), _ptr(W_ih), _ptr(b_ih), _ptr(W_hh),
+                               _ptr(b_hh), _ptr(W_out), _ptr(b_out), _ptr(ctx.dW_ih), _ptr(ctx.db), _ptr(ctx.dW_hh),
+                               _ptr(ctx.dW_out), _ptr(ctx.db_out), _ptr(ctx.loss), _ptr(ctx.nnz), _ptr(ctx.workspace),
+                               ctx.workspace.numel(), _ptr(ctx.dev_status), _stream()), "rad_irnn_step")
     return ctx
