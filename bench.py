@@ -280,6 +280,47 @@ def kernel_sweep(rad, torch, A, dZ, H, ps):
     return rows
 
 
+def small_workloads(rad, torch):
+    """Samples/s of the two small float32 workloads (launch-latency bound; no roofline claim)."""
+    import numpy as np
+    from workloads import irnn_inputs, mlp_inputs
+    out = {}
+
+    def rate(fn, batch, reps):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(reps):
+            fn(i)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        return dict(samples_per_s=round(batch / ms * 1e3, 1), ms_per_step=round(ms, 4))
+
+    X, y, Ws, bs = mlp_inputs((784, 300, 300, 10), 150, "f32", "uniform01", 1234)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    Xd, yd, Wd, bd = dev(X), dev(y), [dev(W) for W in Ws], [dev(b) for b in bs]
+    for variant in ("different", "same"):
+        ctx = rad.MLPStep((784, 300, 300, 10), 150, "f32", "relu", variant, 0.1)
+        r = rate(lambda i=0: ctx(Xd, yd, Wd, bd, seed=0, step=i), 150, 50)
+        st = ctx.stats
+        r["held_bytes"] = st.value_bytes + st.index_bytes + st.relu_bytes + st.unsampled_bytes
+        r["full_backprop_bytes"] = st.full_backprop_bytes
+        assert ctx.dev_status.item() == 0
+        out["mlp_784_300_300_10_b150_f32_" + variant] = r
+    args = [dev(a) for a in irnn_inputs(150, 784, 100, 10, 1234, True)]
+    ctx = rad.IRNNStep(150, 784, 100, 10, "different", 0.1)
+    r = rate(lambda i=0: ctx(*args, seed=0, step0=784 * i), 150, 20)
+    st = ctx.stats
+    r["held_bytes"] = st.value_bytes + st.index_bytes + st.relu_bytes + st.unsampled_bytes
+    r["full_backprop_bytes"] = st.full_backprop_bytes
+    assert ctx.dev_status.item() == 0
+    out["irnn_h100_t784_b150_f32_different"] = r
+    return out
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -413,6 +454,7 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_sweep:
         dZ = (torch.randn(B, 8192, generator=gen, device="cuda") / B).to(bf)
         sweep = kernel_sweep(rad, torch, X, dZ, 8192, (0.01, 0.05, 0.1, 0.5))
+    small = small_workloads(rad, torch) if (rank == 0 and world == 1 and not args.no_sweep) else None
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
         cpu, _ = time_oracle(args, 1, 0)
@@ -427,7 +469,7 @@ def run_ours(args):
                                 l2="inputs larger than L2 (1 GiB activations per layer)"),
                     clocks=clocks, e2e=e2e, gpu_launches=int(launches), roofline=roofline,
                     store_roofline=store_roofline, family_ms={k: round(v, 3) for k, v in by_family.items()},
-                    activation_memory=memory, cpu_baseline=cpu, kernel_sweep=sweep)
+                    activation_memory=memory, cpu_baseline=cpu, kernel_sweep=sweep, small_workloads=small)
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

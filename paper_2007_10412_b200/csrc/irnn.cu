@@ -97,13 +97,15 @@ __global__ void __launch_bounds__(kRnnThreads) irnn_forward_kernel(const RnnPara
       off += total;
     } else {
       // z_j = x_t W_ih[j] + b_ih[j] + b_hh[j] + sum_k h_{t-1}[k] W_hh[k][j]
-      float z = fmaf(s_x[t - 1], wih, bias);
+      // four partial sums keep the FMA pipe busy; they are combined in a fixed order
+      float z0 = fmaf(s_x[t - 1], wih, bias), z1 = 0.0f, z2 = 0.0f, z3 = 0.0f;
 #pragma unroll
       for (int k = 0; k < kHdMax; k += 4) {
         const float4 h4 = *reinterpret_cast<const float4*>(hc + k);
-        z = fmaf(h4.x, wcol[k], z); z = fmaf(h4.y, wcol[k + 1], z);
-        z = fmaf(h4.z, wcol[k + 2], z); z = fmaf(h4.w, wcol[k + 3], z);
+        z0 = fmaf(h4.x, wcol[k], z0); z1 = fmaf(h4.y, wcol[k + 1], z1);
+        z2 = fmaf(h4.z, wcol[k + 2], z2); z3 = fmaf(h4.w, wcol[k + 3], z3);
       }
+      const float z = (z0 + z1) + (z2 + z3);
       const float hn = (j < Hd) ? fmaxf(z, 0.0f) : 0.0f;
       s_h[t & 1][j] = hn;
       const uint32_t bits = __ballot_sync(0xffffffffu, hn > 0.0f);
@@ -115,23 +117,35 @@ __global__ void __launch_bounds__(kRnnThreads) irnn_forward_kernel(const RnnPara
   if (warp == 4 && lane == 0) p.nnz_rows[b] = off;
 }
 
+constexpr int kRing = 8;             // steps of kept entries in flight in the backward kernel
+
 __global__ void __launch_bounds__(kRnnThreads) irnn_backward_kernel(const RnnParams p) {
   extern __shared__ float sm[];
   const int Hd = p.Hd;
   const int S = Hd + 1;                               // odd stride: conflict-free rows and columns
+  const int64_t Tp = (p.T + 3) & ~(int64_t)3;
   float* s_x = sm;                                    // T
-  float* s_dw = s_x + ((p.T + 3) & ~(int64_t)3);      // Hd x S: this row's share of dW_hh
+  float* s_dw = s_x + Tp;                             // Hd x S: this row's share of dW_hh
+  uint32_t* s_keep = reinterpret_cast<uint32_t*>(s_dw + ((Hd * S + 3) & ~3));   // T x w32 keep bits of the row
+  uint32_t* s_rl = s_keep + p.T * p.w32;              // T x w32 ReLU bits
+  uint32_t* s_off = s_rl + p.T * p.w32;               // T value offsets
   __shared__ __align__(16) float s_dz[kHdMax];
-  __shared__ uint32_t s_kidx[2][kHdMax];
-  __shared__ float s_kval[2][kHdMax];
-  __shared__ uint32_t s_kcnt[2];
-  __shared__ uint32_t s_relu[2][4];
+  __shared__ uint32_t s_kidx[kRing][kHdMax];
+  __shared__ float s_kval[kRing][kHdMax];
+  __shared__ uint32_t s_kcnt[kRing];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int64_t b = blockIdx.x;
-  for (int64_t t = tid; t < p.T; t += kRnnThreads) s_x[t] = p.x[b * p.T + t];
+  for (int64_t t = tid; t < p.T; t += kRnnThreads) {
+    s_x[t] = p.x[b * p.T + t];
+    s_off[t] = p.offsets[t * p.B + b];
+  }
+  for (int64_t i = tid; i < p.T * p.w32; i += kRnnThreads) {
+    const int64_t at = ((i / p.w32) * p.B + b) * p.w32 + (i % p.w32);
+    s_keep[i] = p.keepbits[at];
+    s_rl[i] = p.relubits[at];
+  }
   for (int i = tid; i < Hd * S; i += kRnnThreads) s_dw[i] = 0.0f;
   if (tid < kHdMax) s_dz[tid] = 0.0f;
-  if (tid < 8) s_relu[tid >> 2][tid & 3] = 0u;
   const int k = tid;                                  // unit k: row k of W_hh in registers
   float wrow[kHdMax];
   float dh = 0.0f, dwih = 0.0f, dbs = 0.0f, dwih_c = 0.0f, dbs_c = 0.0f;
@@ -140,44 +154,54 @@ __global__ void __launch_bounds__(kRnnThreads) irnn_backward_kernel(const RnnPar
     for (int jj = 0; jj < kHdMax; ++jj) wrow[jj] = (k < Hd && jj < Hd) ? p.W_hh[(int64_t)k * Hd + jj] : 0.0f;
     if (k < Hd) dh = p.dh_last[b * Hd + k];
   }
-  // helper: kept entries of h_{t-1} and ReLU bits of h_t for step t, into buffer t & 1
+  __syncthreads();
+  // helper warp: list of the kept units of step t and an asynchronous copy of their values into
+  // ring slot t % kRing; one commit group per call, so groups can be counted
   auto prefetch = [&](int64_t t) {
-    const int buf = (int)(t & 1);
-    const int64_t sb = (t - 1) * p.B + b;
-    uint32_t m = 0;
-    if (lane < p.ngroups) m = (p.keepbits[sb * p.w32 + (lane >> 2)] >> (8 * (lane & 3))) & 0xffu;
-    const uint32_t c = __popc(m);
-    uint32_t incl = c;
+    if (t >= 1) {
+      const int slot = (int)(t % kRing);
+      uint32_t m = 0;
+      if (lane < p.ngroups) m = (s_keep[(t - 1) * p.w32 + (lane >> 2)] >> (8 * (lane & 3))) & 0xffu;
+      const uint32_t c = __popc(m);
+      uint32_t incl = c;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t n = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += n;
-    }
-    const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
-    const uint32_t off = p.offsets[sb];
-    uint32_t pos = incl - c;
-    const bool fits = (int64_t)off + total <= p.cap_row;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      if ((m >> i) & 1u) {
-        s_kidx[buf][pos] = (uint32_t)(lane * 8 + i);
-        s_kval[buf][pos] = fits ? p.values[b * p.cap_row + off + pos] : 0.0f;
-        ++pos;
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t n = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += n;
       }
+      const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
+      const uint32_t off = s_off[t - 1];
+      uint32_t pos = incl - c;
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        if ((m >> i) & 1u) s_kidx[slot][pos++] = (uint32_t)(lane * 8 + i);
+      const bool fits = (int64_t)off + total <= p.cap_row;
+      for (uint32_t i = lane; i < total; i += 32) {
+        if (fits) {
+          asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(&s_kval[slot][i])),
+                       "l"(p.values + b * p.cap_row + off + i) : "memory");
+        } else {
+          s_kval[slot][i] = 0.0f;
+        }
+      }
+      if (lane == 0) s_kcnt[slot] = total;
     }
-    if (lane < p.w32) s_relu[buf][lane] = p.relubits[sb * p.w32 + lane];
-    if (lane == 0) s_kcnt[buf] = total;
+    asm volatile("cp.async.commit_group;" ::: "memory");
   };
-  __syncthreads();                  // the zero fills above must not land on what the helper prefetches
-  if (warp == 4) prefetch(p.T);
+  if (warp == 4) {
+    for (int d = 0; d < kRing - 1; ++d) prefetch(p.T - d);
+    asm volatile("cp.async.wait_group %0;" ::"n"(kRing - 2) : "memory");      // step T has landed
+  }
   __syncthreads();
   for (int64_t t = p.T; t >= 1; --t) {
-    const int buf = (int)(t & 1);
+    const int slot = (int)(t % kRing);
     if (warp == 4) {
-      if (t > 1) prefetch(t - 1);
+      prefetch(t - (kRing - 1));
+      asm volatile("cp.async.wait_group %0;" ::"n"(kRing - 2) : "memory");    // step t - 1 has landed
     } else {
       // dz_t = dh_t * relu'(h_t); exact gradients of the input weights and biases
-      const float dz = ((s_relu[buf][warp] >> lane) & 1u) ? dh : 0.0f;
+      const uint32_t rbits = warp < p.w32 ? s_rl[(t - 1) * p.w32 + warp] : 0u;
+      const float dz = ((rbits >> lane) & 1u) ? dh : 0.0f;
       s_dz[k] = dz;
       // compensated sums: T terms of one sign would otherwise drift past the float32 tolerance
       const float yi = fmaf(s_x[t - 1], dz, -dwih_c), ti = dwih + yi;
@@ -188,19 +212,22 @@ __global__ void __launch_bounds__(kRnnThreads) irnn_backward_kernel(const RnnPar
     __syncthreads();
     if (warp < 4) {
       // dh_{t-1}[k] = sum_j dz[j] W_hh[k][j]
-      float acc = 0.0f;
+      float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
 #pragma unroll
       for (int jj = 0; jj < kHdMax; jj += 4) {
         const float4 d4 = *reinterpret_cast<const float4*>(s_dz + jj);
-        acc = fmaf(d4.x, wrow[jj], acc); acc = fmaf(d4.y, wrow[jj + 1], acc);
-        acc = fmaf(d4.z, wrow[jj + 2], acc); acc = fmaf(d4.w, wrow[jj + 3], acc);
+        a0 = fmaf(d4.x, wrow[jj], a0); a1 = fmaf(d4.y, wrow[jj + 1], a1);
+        a2 = fmaf(d4.z, wrow[jj + 2], a2); a3 = fmaf(d4.w, wrow[jj + 3], a3);
       }
-      dh = acc;
-      // dW_hh[kept column d, j] += h_hat_{t-1}[d] * dz[j]: thread j owns column j of every row
+      dh = (a0 + a1) + (a2 + a3);
+      // dW_hh[kept unit d, j] += h_hat_{t-1}[d] * dz[j]: thread j owns column j of every row
       if (k < Hd) {
         const float dzj = s_dz[k];
-        const uint32_t cnt = s_kcnt[buf];
-        for (uint32_t n = 0; n < cnt; ++n) s_dw[s_kidx[buf][n] * S + k] = fmaf(s_kval[buf][n], dzj, s_dw[s_kidx[buf][n] * S + k]);
+        const uint32_t cnt = s_kcnt[slot];
+        for (uint32_t n = 0; n < cnt; ++n) {
+          float* cell = s_dw + s_kidx[slot][n] * S + k;
+          *cell = fmaf(s_kval[slot][n], dzj, *cell);
+        }
       }
     }
     __syncthreads();
@@ -333,7 +360,9 @@ extern "C" int rad_irnn_step(const rad_irnn_desc* d, const float* x, const int32
   p.dev_status = dev_status;
   const PhiloxKeys ks = philox_expand_key(d->seed);
   const size_t smem_f = (size_t)d->T * 4;
-  const size_t smem_b = (size_t)((d->T + 3) & ~(int64_t)3) * 4 + (size_t)d->Hd * (d->Hd + 1) * 4;
+  const int64_t w32s = ceil_div(d->Hd, 32);
+  const size_t smem_b = (size_t)((d->T + 3) & ~(int64_t)3) * 4 + (size_t)((d->Hd * (d->Hd + 1) + 3) & ~3) * 4 +
+                        (size_t)d->T * (2 * w32s + 1) * 4;
   if (smem_f > 200 * 1024 || smem_b > 200 * 1024) return RAD_ELIMIT;
   RAD_CUDA_TRY(cudaFuncSetAttribute(irnn_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)std::max<size_t>(smem_f, 1024)));
   RAD_CUDA_TRY(cudaFuncSetAttribute(irnn_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_b));
