@@ -17,4 +17,4 @@ Parity status
     answer vectors distributed with the generator's reference code is
     "parity unpinned": those vectors are not available offline.
 """
-from . import philox, rad, memory_model, irnn  # noqa: F401
+from . import philox, rad, memory_model, irnn, cnn  # noqa: F401

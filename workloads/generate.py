@@ -93,3 +93,29 @@ def irnn_inputs(batch, steps, hidden=100, classes=10, seed=1234, identity=True):
         b_hh = rng.standard_normal(hidden, dtype=np.float32) * np.float32(0.1)
     b_out = np.zeros(classes, np.float32)
     return x, labels, W_ih, b_ih, W_hh, b_hh, W_out, b_out
+
+
+def cnn_inputs(batch, hw=32, cin=3, channels=(16, 32, 64), fc=(128, 10), dtype="bf16", seed=1234, bias_zero=True):
+    """Inputs of the small convolutional net: N(0,1) images (NHWC), 3x3 filters and linear weights
+    Kaiming-normal (std sqrt(2 / fan_in)), zero biases (or small normal ones for tests).  Filters are
+    3 x 3 x Cin x Cout; each conv is followed by ReLU and 2x2 average pooling, so the first linear layer
+    sees (hw / 2^n)^2 * channels[-1] features."""
+    rng = np.random.default_rng(seed)
+    X = rng.standard_normal((batch, hw, hw, cin), dtype=np.float32)
+    labels = uniform_labels(rng, batch, fc[-1])
+    conv_Ws, conv_bs, c = [], [], cin
+    for co in channels:
+        conv_Ws.append(rng.standard_normal((3, 3, c, co), dtype=np.float32) * np.float32(np.sqrt(2.0 / (9 * c))))
+        conv_bs.append(np.zeros(co, np.float32) if bias_zero else rng.standard_normal(co, dtype=np.float32) * np.float32(0.1))
+        c = co
+    feat = (hw >> len(channels)) ** 2 * c
+    fc_Ws, fc_bs, d = [], [], feat
+    for h in fc:
+        fc_Ws.append(rng.standard_normal((d, h), dtype=np.float32) * np.float32(np.sqrt(2.0 / d)))
+        fc_bs.append(np.zeros(h, np.float32) if bias_zero else rng.standard_normal(h, dtype=np.float32) * np.float32(0.1))
+        d = h
+    if dtype == "bf16":
+        X = to_bf16_grid(X)
+        conv_Ws = [to_bf16_grid(W) for W in conv_Ws]
+        fc_Ws = [to_bf16_grid(W) for W in fc_Ws]
+    return X, labels, conv_Ws, conv_bs, fc_Ws, fc_bs
