@@ -318,6 +318,17 @@ def small_workloads(rad, torch):
     r["full_backprop_bytes"] = st.full_backprop_bytes
     assert ctx.dev_status.item() == 0
     out["irnn_h100_t784_b150_f32_different"] = r
+    from workloads import cnn_inputs
+    X, y, cW, cb, fW, fb = cnn_inputs(128, 32, 3, (16, 32, 64), (128, 10), "bf16", 1234)
+    bf = lambda a: dev(a).to(torch.bfloat16)
+    cargs = (bf(X), dev(y), [bf(w) for w in cW], [dev(b) for b in cb], [bf(w) for w in fW], [dev(b) for b in fb])
+    ctx = rad.CNNStep(128, 32, 3, (16, 32, 64), (128, 10), "bf16", "different", 0.1)
+    r = rate(lambda i=0: ctx(*cargs, seed=0, step=i), 128, 20)
+    st = ctx.stats
+    r["held_bytes"] = st.value_bytes + st.index_bytes + st.relu_bytes + st.unsampled_bytes
+    r["full_backprop_bytes"] = st.full_backprop_bytes
+    assert ctx.dev_status.item() == 0
+    out["cnn_32x32x3_c16_32_64_fc128_10_b128_bf16_different"] = r
     return out
 
 

@@ -308,6 +308,42 @@ int rad_irnn_step(const rad_irnn_desc* net /* host */, const float* x, const int
                   int64_t* nnz_out, void* workspace, int64_t workspace_bytes,
                   int32_t* dev_status, void* stream);
 
+/*
+ * One training step of a small convolutional net (paper, Fig. "Convnet activation sampling",
+ * Sec. 4.2): n_conv blocks of [3x3 convolution, zero padding 1, stride 1, + bias, ReLU, 2x2
+ * average pooling], then n_fc linear layers (ReLU between them, none after the last) and softmax
+ * cross-entropy.  NHWC.  The input of every convolution and of every linear layer is stored
+ * through the mask of (seed, layer, step), layers numbered conv blocks first: one keep decision per
+ * input entry, shared by every filter tap that reads it.  ReLU derivatives take one bit per conv
+ * output, average pooling and biases need nothing.  Filter and weight gradients come from the
+ * stores, everything else is exact.
+ *   X device B x H x W x Cin (dtype); labels device int32[B];
+ *   conv_W[l] device 3 x 3 x Cin_l x Cout_l (dtype), Cout_l multiple of 8; conv_b[l] device float32 or NULL;
+ *   fc_W[l] device fc_in_l x fc_dims[l] (dtype) with fc_in_0 = (H / 2^n_conv)(W / 2^n_conv) Cout_last, the
+ *   pooled map flattened in (y, x, c) order; fc_b[l] device float32 or NULL;
+ *   dconv_W[l], dfc_W[l] device float32, same shapes; dconv_b[l], dfc_b[l] device float32; loss float32[1].
+ *   The pointer tables are host arrays.  nnz_out device int64[2 * (n_conv + n_fc)] or NULL.
+ */
+typedef struct rad_cnn_desc {
+  int64_t  B, H, W, Cin;
+  int32_t  n_conv, n_fc;
+  const int64_t* conv_channels;   /* host, n_conv entries */
+  const int64_t* fc_dims;         /* host, n_fc entries: outputs of the linear layers */
+  int32_t  dtype, variant;
+  float    p;
+  uint32_t step;
+  uint64_t seed;
+} rad_cnn_desc;
+
+int rad_cnn_workspace(const rad_cnn_desc* net /* host */, int64_t* bytes /* host */,
+                      rad_step_stats* stats /* host or NULL */);
+int rad_cnn_step(const rad_cnn_desc* net /* host */, const void* X, const int32_t* labels,
+                 const void* const* conv_W, const float* const* conv_b,
+                 const void* const* fc_W, const float* const* fc_b,
+                 float* const* dconv_W, float* const* dconv_b, float* const* dfc_W, float* const* dfc_b,
+                 float* loss, int64_t* nnz_out, void* workspace, int64_t workspace_bytes,
+                 int32_t* dev_status, void* stream);
+
 /* Kernels this library has launched since it was loaded (host-side tally; memsets not counted). */
 int64_t rad_launch_count(void);
 

@@ -55,6 +55,13 @@ class rad_irnn_desc(C.Structure):
                 ("p", C.c_float), ("seed", C.c_uint64), ("step0", C.c_uint32)]
 
 
+class rad_cnn_desc(C.Structure):
+    _fields_ = [("B", C.c_int64), ("H", C.c_int64), ("W", C.c_int64), ("Cin", C.c_int64), ("n_conv", C.c_int32),
+                ("n_fc", C.c_int32), ("conv_channels", C.POINTER(C.c_int64)), ("fc_dims", C.POINTER(C.c_int64)),
+                ("dtype", C.c_int32), ("variant", C.c_int32), ("p", C.c_float), ("step", C.c_uint32),
+                ("seed", C.c_uint64)]
+
+
 class rad_step_stats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in ("value_bytes", "index_bytes", "relu_bytes", "preact_bytes",
                                          "unsampled_bytes", "full_backprop_bytes")]
@@ -63,7 +70,7 @@ class rad_step_stats(C.Structure):
 EXPORTS = ["rad_keep_threshold", "rad_effective_p", "rad_scale", "rad_store_size_query",
            "rad_linear_forward_store", "rad_linear_forward_store_static", "rad_weight_grad_workspace", "rad_linear_weight_grad",
            "rad_linear_forward", "rad_softmax_xent", "rad_input_grad_workspace", "rad_linear_input_grad",
-           "rad_mlp_workspace", "rad_mlp_step", "rad_irnn_workspace", "rad_irnn_step", "rad_launch_count", "rad_strerror", "rad_version"]
+           "rad_mlp_workspace", "rad_mlp_step", "rad_irnn_workspace", "rad_irnn_step", "rad_cnn_workspace", "rad_cnn_step", "rad_launch_count", "rad_strerror", "rad_version"]
 
 _lib = None
 
@@ -100,6 +107,8 @@ def lib():
         L.rad_mlp_workspace.argtypes = [C.POINTER(rad_mlp_desc), C.POINTER(i64), C.POINTER(rad_step_stats)]
         L.rad_irnn_workspace.argtypes = [C.POINTER(rad_irnn_desc), C.POINTER(i64), C.POINTER(rad_step_stats)]
         L.rad_irnn_step.argtypes = [C.POINTER(rad_irnn_desc)] + [vp] * 15 + [vp, i64, vp, vp]
+        L.rad_cnn_workspace.argtypes = [C.POINTER(rad_cnn_desc), C.POINTER(i64), C.POINTER(rad_step_stats)]
+        L.rad_cnn_step.argtypes = [C.POINTER(rad_cnn_desc), vp, vp] + [C.POINTER(vp)] * 8 + [vp, vp, vp, i64, vp, vp]
         L.rad_mlp_step.argtypes = [C.POINTER(rad_mlp_desc), vp, vp, C.POINTER(vp), C.POINTER(vp),
                                    C.POINTER(vp), C.POINTER(vp), vp, vp, vp, i64, vp, vp]
         for name in EXPORTS:
@@ -322,4 +331,45 @@ def rad_irnn_step(ctx, x, labels, W_ih, b_ih, W_hh, b_hh, W_out, b_out, seed=0, 
                                _ptr(b_hh), _ptr(W_out), _ptr(b_out), _ptr(ctx.dW_ih), _ptr(ctx.db), _ptr(ctx.dW_hh),
                                _ptr(ctx.dW_out), _ptr(ctx.db_out), _ptr(ctx.loss), _ptr(ctx.nnz), _ptr(ctx.workspace),
                                ctx.workspace.numel(), _ptr(ctx.dev_status), _stream()), "rad_irnn_step")
+    return ctx
+
+
+class CNNStep:
+    """Owns the workspace, gradient buffers and pointer tables of rad_cnn_step for one net shape."""
+
+    def __init__(self, B, hw, cin, channels, fc, dtype="bf16", variant="different", p=0.1, device="cuda"):
+        self.channels, self.fc = list(channels), list(fc)
+        self._ch = (C.c_int64 * len(channels))(*channels)
+        self._fc = (C.c_int64 * len(fc))(*fc)
+        self.desc = rad_cnn_desc(B, hw, hw, cin, len(channels), len(fc), self._ch, self._fc, DTYPES[dtype],
+                                 VARIANTS[variant], p, 0, 0)
+        nbytes = C.c_int64(0)
+        self.stats = rad_step_stats()
+        _check(lib().rad_cnn_workspace(C.byref(self.desc), C.byref(nbytes), C.byref(self.stats)), "rad_cnn_workspace")
+        f32 = dict(dtype=torch.float32, device=device)
+        self.workspace = torch.empty(nbytes.value, dtype=torch.uint8, device=device)
+        cs = [cin] + self.channels
+        self.dconv_W = [torch.empty(3, 3, cs[l], cs[l + 1], **f32) for l in range(len(channels))]
+        self.dconv_b = [torch.empty(cs[l + 1], **f32) for l in range(len(channels))]
+        fs = [(hw >> len(channels)) ** 2 * cs[-1]] + self.fc
+        self.dfc_W = [torch.empty(fs[l], fs[l + 1], **f32) for l in range(len(fc))]
+        self.dfc_b = [torch.empty(fs[l + 1], **f32) for l in range(len(fc))]
+        self.loss = torch.zeros(1, **f32)
+        self.nnz = torch.zeros(2 * (len(channels) + len(fc)), dtype=torch.int64, device=device)
+        self.dev_status = torch.zeros(1, dtype=torch.int32, device=device)
+
+    def __call__(self, X, labels, conv_W, conv_b, fc_W, fc_b, seed=0, step=0):
+        return rad_cnn_step(self, X, labels, conv_W, conv_b, fc_W, fc_b, seed, step)
+
+
+def _table(tensors):
+    return (C.c_void_p * len(tensors))(*[(None if t is None else t.data_ptr()) for t in tensors])
+
+
+def rad_cnn_step(ctx, X, labels, conv_W, conv_b, fc_W, fc_b, seed=0, step=0):
+    ctx.desc.seed, ctx.desc.step = seed, step
+    _check(lib().rad_cnn_step(C.byref(ctx.desc), _ptr(X), _ptr(labels), _table(conv_W), _table(conv_b), _table(fc_W),
+                              _table(fc_b), _table(ctx.dconv_W), _table(ctx.dconv_b), _table(ctx.dfc_W),
+                              _table(ctx.dfc_b), _ptr(ctx.loss), _ptr(ctx.nnz), _ptr(ctx.workspace),
+                              ctx.workspace.numel(), _ptr(ctx.dev_status), _stream()), "rad_cnn_step")
     return ctx

@@ -135,6 +135,17 @@ int column_sums(int dtype, int64_t B, int64_t H, const void* dZ, int64_t ldz, fl
                 void* workspace, int64_t workspace_bytes, cudaStream_t s);
 int64_t column_sums_workspace(int64_t B, int64_t H);
 
+// 3x3 convolution layers (conv.cu)
+int conv_forward_pool(int dtype, int64_t B, int H, int W, int Cin, int Cout, const void* X, const void* Wt,
+                      const float* bias, void* P, uint32_t* relubits, cudaStream_t st);
+int conv_dz(int dtype, int64_t B, int H, int W, int Cout, const void* dP, const uint32_t* relubits, void* dZ,
+            cudaStream_t st);
+int conv_input_grad(int dtype, int64_t B, int H, int W, int Cin, int Cout, const void* dZ, const void* Wt, void* dX,
+                    cudaStream_t st);
+int64_t conv_weight_grad_workspace(int64_t B, int Cin, int Cout);
+int conv_weight_grad(const rad_store* store, int H, int W, int Cin, int Cout, const void* dZ, float* dW, void* workspace,
+                     int64_t workspace_bytes, cudaStream_t st);
+
 // tcgen05 kernels (bf16, aligned)
 bool tc_shape_ok(int64_t B, int64_t D, int64_t H, const void* p0, int64_t ld0, const void* p1,
                  int64_t ld1);
