@@ -510,9 +510,11 @@ tc_gemm_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, const 
     // One thread per keep-bit word: half h = columns 128h..128h+127 of the tile (one store tile),
     // row r of the slab, columns 32*wq..32*wq+31 of that half.  The row's first value is given by
     // the stored row offset; the words before this one in the row are counted with popc.
+    // Eight consecutive lanes take eight consecutive rows of the same word column: with the
+    // 128-byte swizzle their 16-byte zero stores then fall on eight different bank groups.
     const int et = tid - 32 * kFirstExpanderWarp;            // 0..511
     const int h = et >> 8, wi = et & 255;
-    const int r = wi >> 2, wq = wi & 3;
+    const int r = (wi & 7) + ((wi >> 5) << 3), wq = (wi >> 3) & 3;
     int stage = 0, slot = 0;
     uint32_t phase = 0, cphase = 0;
     bool ok = true;
