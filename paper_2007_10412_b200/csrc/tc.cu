@@ -540,17 +540,34 @@ tc_gemm_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, const 
           uint8_t* rowp = sA + h * 16384 + (wq >> 1) * 8192 + r * 128;
           const int j0 = (wq & 1) * 4;
           const uint32_t limit = (uint32_t)p.comp_cap >> 1;
-          if (__popc(word) <= 10) {
-            // sparse word: zero this thread's 32 columns, then drop the kept values in place
+          const uint32_t cnt = __popc(word);
+          // one path per warp: the dense form is right for any word
+          if (__all_sync(0xffffffffu, cnt + (pos & 3u) <= 12u && cnt <= 10u)) {
+            // sparse word: zero this thread's 32 columns, then drop the kept values in place.  The
+            // values are consecutive from `pos`: three aligned 8-byte loads cover them (a word whose
+            // values would pass the end of the staged tile places nothing: the producer has flagged it)
 #pragma unroll
             for (int jj = 0; jj < 4; ++jj)
               *reinterpret_cast<uint4*>(rowp + (((j0 + jj) ^ (r & 7)) << 4)) = make_uint4(0, 0, 0, 0);
-            uint32_t rest = word;
-            while (rest != 0) {
+            uint32_t rest = (pos + cnt <= limit) ? word : 0u;
+            const uint32_t e0 = pos & 3u;
+            const uint2* win = reinterpret_cast<const uint2*>(vals + (min(pos, limit) & ~3u));   // stays inside the ring
+            const uint2 q0 = win[0], q1 = win[1];
+            uint2 q2 = make_uint2(0u, 0u);
+            if (e0 + cnt > 8u) q2 = win[2];
+            // bring the first kept value to bit 0 of s0: drop whole words, then a half word
+            const bool drop = (e0 & 2u) != 0u;
+            const uint32_t w0 = drop ? q0.y : q0.x, w1 = drop ? q1.x : q0.y, w2 = drop ? q1.y : q1.x;
+            const uint32_t w3 = drop ? q2.x : q1.y, w4 = drop ? q2.y : q2.x, w5 = drop ? 0u : q2.y;
+            const uint32_t sh = (e0 & 1u) << 4;
+            const uint32_t sv[5] = {__funnelshift_r(w0, w1, sh), __funnelshift_r(w1, w2, sh), __funnelshift_r(w2, w3, sh),
+                                    __funnelshift_r(w3, w4, sh), __funnelshift_r(w4, w5, sh)};
+#pragma unroll
+            for (int i = 0; i < 10; ++i) {
+              if (rest == 0) break;
               const int b = __ffs(rest) - 1;
               rest &= rest - 1;
-              const unsigned short v = (pos < limit) ? vals[pos] : (unsigned short)0;
-              ++pos;
+              const unsigned short v = (unsigned short)(sv[i >> 1] >> (16 * (i & 1)));
               const int j = j0 + (b >> 3);
               *reinterpret_cast<unsigned short*>(rowp + ((j ^ (r & 7)) << 4) + ((b & 7) << 1)) = v;
             }
