@@ -11,7 +11,7 @@
 // 128x256x16 MMAs.  Operands arrive by TMA (128-byte swizzle, no multicast) through a 3-stage
 // mbarrier ring; for the different-sample dW the A operand is written by sixteen "expander" warps
 // instead.  Warp roles: 0 TMA producer, 1 MMA issuer and tensor-memory owner, 2-5 epilogue,
-// 6 producer of the compressed ring and 7-22 expanders (sparse A only).  Long contractions can be split along K; partial tiles are
+// (2-17 in the dense kernels), 6 producer of the compressed ring and 7-22 expanders (sparse A only).  Long contractions can be split along K; partial tiles are
 // summed in split order by a second kernel, so results are reproducible.
 // Every mbarrier wait is bounded: on expiry the CTA raises RAD_DEV_ETIMEOUT, all roles leave
 // their loops, tensor memory is released and the kernel returns.
@@ -196,7 +196,13 @@ struct SmemCtl {
 constexpr int kIndexBytes = kTileWords * 4;   // keep bits + row offsets of one store tile (1152 B)
 constexpr int kExpanderWarps = 16;            // one thread per keep-bit word of the two halves
 constexpr int kFirstExpanderWarp = 7;        // warp 6 feeds the compressed ring
-template <int AK> __host__ __device__ constexpr int threads_for() { return AK == kASparse ? 32 * (kFirstExpanderWarp + kExpanderWarps) : 192; }
+// Epilogue warps: a warp reads the tensor-memory lanes 32 (warp % 4) .. +31; the dense kernels put
+// four warps on each lane quarter (64 accumulator columns each), since their epilogue is not
+// overlapped with the next tile's MMAs and carries the activation math.
+template <int AK> __host__ __device__ constexpr int epi_warps_for() { return AK == kASparse ? 4 : 16; }
+template <int AK> __host__ __device__ constexpr int threads_for() {
+  return AK == kASparse ? 32 * (kFirstExpanderWarp + kExpanderWarps) : 32 * (2 + epi_warps_for<AK>());
+}
 
 template <int AK, int BKIND, int EPI>
 __global__ void __launch_bounds__(threads_for<AK>(), 1)
@@ -231,7 +237,7 @@ tc_gemm_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, const 
       mbar_init(smem_u32(&ctl->comp_empty[c]), kExpanderWarps);
     }
     mbar_init(smem_u32(&ctl->tmem_full), 1);
-    mbar_init(smem_u32(&ctl->tmem_empty), 128);
+    mbar_init(smem_u32(&ctl->tmem_empty), 32 * epi_warps_for<AK>());
     ctl->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -324,9 +330,11 @@ tc_gemm_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, const 
       }
       unit_phase ^= 1u;
     }
-  } else if (warp < 6) {
-    // ===== epilogue: thread = one accumulator row (tensor-memory lane) =====
+  } else if (warp < 2 + epi_warps_for<AK>()) {
+    // ===== epilogue: thread = one accumulator row (tensor-memory lane) and a range of columns =====
     const int q = warp & 3;                      // lanes 32q .. 32q+31 are the ones this warp may read
+    constexpr int kColsPerWarp = BN / (epi_warps_for<AK>() / 4);
+    const int c_first = ((warp - 2) >> 2) * kColsPerWarp;
     uint32_t unit_phase = 0;
     bool ok = true;
     for (int64_t u = blockIdx.x; u < sched.units && ok; u += gridDim.x) {
@@ -339,7 +347,7 @@ tc_gemm_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, const 
         const int64_t m = w.m0 + h * kHalfM + q * 32 + lane;
         const bool row_ok = m < sched.M;
 #pragma unroll 1
-        for (int c0 = 0; c0 < BN; c0 += 32) {
+        for (int c0 = c_first; c0 < c_first + kColsPerWarp; c0 += 32) {
           const int64_t n = w.n0 + c0;
           if (n >= p.N) break;                  // warp-uniform
           uint32_t r[32];
