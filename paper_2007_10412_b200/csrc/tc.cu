@@ -186,6 +186,118 @@ struct Schedule {
   }
 };
 
+// ---- epilogue of one 32-column chunk of one accumulator row ------------------------------------------
+// r: the 32 float32 accumulators of row m, columns n .. n+31 (as bit patterns).
+template <int EPI>
+__device__ __forceinline__ void epilogue_chunk(const TcParams& p, uint32_t (&r)[32], int64_t m, int64_t n, bool row_ok,
+                                               int32_t split) {
+  const int nvalid = (int)min((int64_t)32, p.N - n);      // multiple of 8
+  if (EPI == kFwd) {
+    float v[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+    if (p.bias != nullptr) {
+#pragma unroll
+      for (int j = 0; j < 32; j += 4) {
+        if (j < nvalid) {
+          const float4 b4 = __ldg(reinterpret_cast<const float4*>(p.bias + n + j));
+          v[j] += b4.x; v[j + 1] += b4.y; v[j + 2] += b4.z; v[j + 3] += b4.w;
+        }
+      }
+    }
+    if (row_ok) {
+      if (p.out_z != nullptr) {
+        float4* dst = reinterpret_cast<float4*>(p.out_z + m * p.ld_z + n);
+#pragma unroll
+        for (int j = 0; j < 32; j += 4)
+          if (j < nvalid) dst[j >> 2] = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+      }
+      if (p.out_zlow != nullptr) {
+        uint4* dst = reinterpret_cast<uint4*>(p.out_zlow + m * p.ld_zlow + n);
+#pragma unroll
+        for (int j = 0; j < 32; j += 8) {
+          if (j < nvalid) {
+            __nv_bfloat162 a = __floats2bfloat162_rn(v[j], v[j + 1]), b = __floats2bfloat162_rn(v[j + 2], v[j + 3]);
+            __nv_bfloat162 c = __floats2bfloat162_rn(v[j + 4], v[j + 5]), d = __floats2bfloat162_rn(v[j + 6], v[j + 7]);
+            dst[j >> 3] = make_uint4(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b),
+                                     *reinterpret_cast<uint32_t*>(&c), *reinterpret_cast<uint32_t*>(&d));
+          }
+        }
+      }
+      if (p.out_act != nullptr) {
+        uint32_t bits = 0;
+        uint4* dst = reinterpret_cast<uint4*>(p.out_act + m * p.ld_act + n);
+#pragma unroll
+        for (int j = 0; j < 32; j += 8) {
+          if (j < nvalid) {
+            uint32_t pk[4];
+#pragma unroll
+            for (int e = 0; e < 8; e += 2) {
+              float a0 = v[j + e], a1 = v[j + e + 1];
+              if (p.act == RAD_ACT_RELU) { a0 = fmaxf(a0, 0.0f); a1 = fmaxf(a1, 0.0f); }
+              else if (p.act == RAD_ACT_GELU) { a0 = gelu_f(a0); a1 = gelu_f(a1); }
+              const __nv_bfloat162 h2 = __floats2bfloat162_rn(a0, a1);
+              pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+              // the bit is taken from the rounded activation, the tensor the backward sees
+              bits |= (__bfloat162float(h2.x) > 0.0f ? 1u : 0u) << (j + e);
+              bits |= (__bfloat162float(h2.y) > 0.0f ? 1u : 0u) << (j + e + 1);
+            }
+            dst[j >> 3] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          }
+        }
+        if (p.relubits != nullptr) p.relubits[m * p.w32 + (n >> 5)] = bits;
+      }
+    }
+  } else if (EPI == kDx) {
+    if (row_ok) {
+      uint32_t bits = 0xffffffffu;
+      if (p.relubits_prev != nullptr) bits = __ldg(p.relubits_prev + m * ((p.N + 31) / 32) + (n >> 5));
+      uint4* dst = reinterpret_cast<uint4*>(p.out_dx + m * p.ld_dx + n);
+#pragma unroll
+      for (int j = 0; j < 32; j += 8) {
+        if (j < nvalid) {
+          float g[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) g[e] = ((bits >> (j + e)) & 1u) ? __uint_as_float(r[j + e]) : 0.0f;
+          if (p.z_prev != nullptr) {
+            const uint4 zq = __ldg(reinterpret_cast<const uint4*>(p.z_prev + m * p.ld_zprev + n + j));
+            const uint32_t zw[4] = {zq.x, zq.y, zq.z, zq.w};
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const float z = __uint_as_float((e & 1) ? (zw[e >> 1] & 0xffff0000u) : (zw[e >> 1] << 16));
+              g[e] *= gelu_grad_f(z);
+            }
+          }
+          uint32_t pk[4];
+#pragma unroll
+          for (int e = 0; e < 8; e += 2) {
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(g[e], g[e + 1]);
+            pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+          }
+          dst[j >> 3] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
+      }
+    }
+  } else {
+    if (row_ok) {
+      float* dst;
+      if (p.splits > 1) {
+        dst = p.partial + ((int64_t)split * p.partial_rows + m) * p.N + n;
+      } else {
+        const int64_t row = (p.row_idx != nullptr) ? (int64_t)__ldg(p.row_idx + m) : m;
+        if (row >= p.dw_rows) { raise_status(p.dev_status, RAD_DEV_EINTERNAL); return; }
+        dst = p.out_dw + row * p.ld_dw + n;
+      }
+      float4* d4 = reinterpret_cast<float4*>(dst);
+#pragma unroll
+      for (int j = 0; j < 32; j += 4)
+        if (j < nvalid)
+          d4[j >> 2] = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
+                                   __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+    }
+  }
+}
+
 // ---- shared memory layout -------------------------------------------------------------------------
 struct SmemCtl {
   uint64_t full[4], empty[4], comp_full[8], comp_empty[8], tmem_full, tmem_empty;
@@ -353,111 +465,7 @@ tc_gemm_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, const 
           uint32_t r[32];
           tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * 256 + c0), r);
           tmem_ld_wait();
-          const int nvalid = (int)min((int64_t)32, p.N - n);      // multiple of 8
-          if (EPI == kFwd) {
-            float v[32];
-#pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-            if (p.bias != nullptr) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 4) {
-                if (j < nvalid) {
-                  const float4 b4 = __ldg(reinterpret_cast<const float4*>(p.bias + n + j));
-                  v[j] += b4.x; v[j + 1] += b4.y; v[j + 2] += b4.z; v[j + 3] += b4.w;
-                }
-              }
-            }
-            if (row_ok) {
-              if (p.out_z != nullptr) {
-                float4* dst = reinterpret_cast<float4*>(p.out_z + m * p.ld_z + n);
-#pragma unroll
-                for (int j = 0; j < 32; j += 4)
-                  if (j < nvalid) dst[j >> 2] = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-              }
-              if (p.out_zlow != nullptr) {
-                uint4* dst = reinterpret_cast<uint4*>(p.out_zlow + m * p.ld_zlow + n);
-#pragma unroll
-                for (int j = 0; j < 32; j += 8) {
-                  if (j < nvalid) {
-                    __nv_bfloat162 a = __floats2bfloat162_rn(v[j], v[j + 1]), b = __floats2bfloat162_rn(v[j + 2], v[j + 3]);
-                    __nv_bfloat162 c = __floats2bfloat162_rn(v[j + 4], v[j + 5]), d = __floats2bfloat162_rn(v[j + 6], v[j + 7]);
-                    dst[j >> 3] = make_uint4(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b),
-                                             *reinterpret_cast<uint32_t*>(&c), *reinterpret_cast<uint32_t*>(&d));
-                  }
-                }
-              }
-              if (p.out_act != nullptr) {
-                uint32_t bits = 0;
-                uint4* dst = reinterpret_cast<uint4*>(p.out_act + m * p.ld_act + n);
-#pragma unroll
-                for (int j = 0; j < 32; j += 8) {
-                  if (j < nvalid) {
-                    uint32_t pk[4];
-#pragma unroll
-                    for (int e = 0; e < 8; e += 2) {
-                      float a0 = v[j + e], a1 = v[j + e + 1];
-                      if (p.act == RAD_ACT_RELU) { a0 = fmaxf(a0, 0.0f); a1 = fmaxf(a1, 0.0f); }
-                      else if (p.act == RAD_ACT_GELU) { a0 = gelu_f(a0); a1 = gelu_f(a1); }
-                      const __nv_bfloat162 h2 = __floats2bfloat162_rn(a0, a1);
-                      pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
-                      // the bit is taken from the rounded activation, the tensor the backward sees
-                      bits |= (__bfloat162float(h2.x) > 0.0f ? 1u : 0u) << (j + e);
-                      bits |= (__bfloat162float(h2.y) > 0.0f ? 1u : 0u) << (j + e + 1);
-                    }
-                    dst[j >> 3] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                  }
-                }
-                if (p.relubits != nullptr) p.relubits[m * p.w32 + (n >> 5)] = bits;
-              }
-            }
-          } else if (EPI == kDx) {
-            if (row_ok) {
-              uint32_t bits = 0xffffffffu;
-              if (p.relubits_prev != nullptr) bits = __ldg(p.relubits_prev + m * ((p.N + 31) / 32) + (n >> 5));
-              uint4* dst = reinterpret_cast<uint4*>(p.out_dx + m * p.ld_dx + n);
-#pragma unroll
-              for (int j = 0; j < 32; j += 8) {
-                if (j < nvalid) {
-                  float g[8];
-#pragma unroll
-                  for (int e = 0; e < 8; ++e) g[e] = ((bits >> (j + e)) & 1u) ? __uint_as_float(r[j + e]) : 0.0f;
-                  if (p.z_prev != nullptr) {
-                    const uint4 zq = __ldg(reinterpret_cast<const uint4*>(p.z_prev + m * p.ld_zprev + n + j));
-                    const uint32_t zw[4] = {zq.x, zq.y, zq.z, zq.w};
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                      const float z = __uint_as_float((e & 1) ? (zw[e >> 1] & 0xffff0000u) : (zw[e >> 1] << 16));
-                      g[e] *= gelu_grad_f(z);
-                    }
-                  }
-                  uint32_t pk[4];
-#pragma unroll
-                  for (int e = 0; e < 8; e += 2) {
-                    const __nv_bfloat162 h2 = __floats2bfloat162_rn(g[e], g[e + 1]);
-                    pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
-                  }
-                  dst[j >> 3] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                }
-              }
-            }
-          } else {
-            if (row_ok) {
-              float* dst;
-              if (p.splits > 1) {
-                dst = p.partial + ((int64_t)w.split * p.partial_rows + m) * p.N + n;
-              } else {
-                const int64_t row = (p.row_idx != nullptr) ? (int64_t)__ldg(p.row_idx + m) : m;
-                if (row >= p.dw_rows) { raise_status(p.dev_status, RAD_DEV_EINTERNAL); continue; }
-                dst = p.out_dw + row * p.ld_dw + n;
-              }
-              float4* d4 = reinterpret_cast<float4*>(dst);
-#pragma unroll
-              for (int j = 0; j < 32; j += 4)
-                if (j < nvalid)
-                  d4[j >> 2] = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
-                                           __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
-            }
-          }
+          epilogue_chunk<EPI>(p, r, m, n, row_ok, w.split);
         }
       }
       tc_fence_before();
@@ -620,6 +628,248 @@ tc_gemm_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, const 
   }
 }
 
+// ---- two-CTA engine (dense operands) -----------------------------------------------------------------
+// A cluster of two CTAs (one SM pair) owns a 256 x 256 output tile.  Each CTA stages 128 rows of
+// the A tile and 128 rows (N) of the B tile per K block and keeps 128 accumulator rows in its own
+// tensor memory; one thread of the even CTA issues tcgen05.mma.cta_group::2, which reads both
+// CTAs' shared memory.  Against the one-CTA tile this halves the operand bytes each SM's shared
+// memory has to deliver per MMA, and a 128 x 256 accumulator takes 256 tensor-memory columns, so
+// two of them alternate: the epilogue of one tile runs under the MMAs of the next.
+// Barriers: full[s] (even CTA; its producer arrives once with the byte count of both CTAs, and
+// both CTAs' TMA complete on it: the odd CTA reloads a stage only after the commit that follows the
+// even CTA's wait on the previous phase, so its bytes never reach an older phase), empty[s] and tmem_full[b] (one per CTA, signalled by the MMA thread's commit to
+// both CTAs), tmem_empty[b] (even CTA; every epilogue warp of the pair arrives).
+constexpr int kStage2Bytes = 2 * 128 * BK * 2;   // 16 KB of A + 16 KB of B per CTA and stage
+constexpr int kStages2 = 6;
+constexpr int kEpiWarps2 = 8;
+constexpr int kThreads2 = 32 * (2 + kEpiWarps2);
+
+struct SmemCtl2 {
+  uint64_t full[kStages2], empty[kStages2], tmem_full[2], tmem_empty[2];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {   // shared::cluster address
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t caddr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(caddr) : "memory");
+}
+// Bounded wait of the pair: on expiry both CTAs' abort flags are raised.
+__device__ __forceinline__ bool mbar_wait2(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t peer_abort) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  while (true) {
+#pragma unroll 1
+    for (int i = 0; i < 32; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag != 0) return false;
+    if (global_timer_ns() - t0 > kWaitLimitNs) {
+      *abort_flag = 1;
+      asm volatile("st.relaxed.cluster.shared::cluster.u32 [%0], %1;" ::"r"(peer_abort), "r"(1u) : "memory");
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t cbar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(cbar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {   // the barrier at this offset in both CTAs
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+// D = f32, A = B = bf16, M = 256 over the pair, N = 256.
+__host__ __device__ constexpr uint32_t make_idesc_pair(bool a_mn, bool b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+         ((256u >> 3) << 17) | ((256u >> 4) << 24);
+}
+
+template <int AK, int BKIND, int EPI>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads2, 1)
+tc_gemm_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  SmemCtl2* ctl = reinterpret_cast<SmemCtl2*>(smem + (size_t)kStages2 * kStage2Bytes);
+  volatile int* abort_flag = &ctl->abort_flag;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t rank = cluster_ctarank();         // 0: issues the MMAs; both stage operands and run epilogues
+  const uint32_t peer_abort = map_to_cta(smem_u32(&ctl->abort_flag), rank ^ 1u);
+  int64_t m_rows = p.M;
+  if (p.M_dev != nullptr) {
+    int64_t md;
+    asm volatile("ld.global.cg.s64 %0, [%1];" : "=l"(md) : "l"(p.M_dev) : "memory");
+    m_rows = md < m_rows ? md : m_rows;
+  }
+  const Schedule sched(m_rows, p.N, p.K, p.splits);
+  const int64_t pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+  if (tid == 0) {
+    for (int s = 0; s < kStages2; ++s) {
+      mbar_init(smem_u32(&ctl->full[s]), 1);
+      mbar_init(smem_u32(&ctl->empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&ctl->tmem_full[b]), 1);
+      mbar_init(smem_u32(&ctl->tmem_empty[b]), 2 * kEpiWarps2);
+    }
+    ctl->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {   // the same warp of both CTAs allocates for the pair: two 128 x 256 accumulators per CTA
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(&ctl->tmem_base)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  cluster_sync_all();        // the peer's barriers are initialised before anything arrives on them
+  tc_fence_after();
+  const uint32_t tmem_base = ctl->tmem_base;
+  const uint32_t smem_base = smem_u32(smem);
+
+  if (warp == 0) {
+    // ===== TMA producer: this CTA's 128 rows of A and 128 rows (N) of B, completing on the even CTA's barrier =====
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int64_t u = pair; u < sched.units && ok; u += npairs) {
+      const Unit w = sched.unit(u);
+      const int m_own = (int)w.m0 + 128 * (int)rank, n_own = (int)w.n0 + 128 * (int)rank;
+      for (int kb = w.kb0; kb < w.kb1; ++kb) {
+        if (lane == 0) {
+          ok = mbar_wait2(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, peer_abort);
+          if (ok) {
+            const uint32_t sA = smem_base + stage * kStage2Bytes;
+            const uint32_t sB = sA + kStage2Bytes / 2;
+            const uint32_t full = map_to_cta(smem_u32(&ctl->full[stage]), 0u);
+            const int k0 = kb * BK;
+            if (rank == 0) mbar_arrive_expect_tx(smem_u32(&ctl->full[stage]), 2 * kStage2Bytes);   // both CTAs' bytes
+            if (AK == kAK) {
+              tma_load_2d_pair(sA, &tmA, k0, m_own, full);                         // 64 (K) x 128 rows
+            } else {
+#pragma unroll
+              for (int c = 0; c < 2; ++c) tma_load_2d_pair(sA + c * 8192, &tmA, m_own + c * 64, k0, full);
+            }
+            if (BKIND == kBK_) {
+              tma_load_2d_pair(sB, &tmB, k0, n_own, full);
+            } else {
+#pragma unroll
+              for (int c = 0; c < 2; ++c) tma_load_2d_pair(sB + c * 8192, &tmB, n_own + c * 64, k0, full);
+            }
+          }
+        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) break;
+        if (++stage == kStages2) { stage = 0; phase ^= 1u; }
+      }
+    }
+    // tail: every commit aimed at this CTA's stage barriers has landed before the CTA may leave
+    if (lane == 0) {
+      for (int i = 0; i < kStages2 && ok; ++i) {
+        ok = mbar_wait2(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, peer_abort);
+        if (++stage == kStages2) { stage = 0; phase ^= 1u; }
+      }
+    }
+  } else if (warp == 1) {
+    // ===== MMA issuer: one thread of the even CTA drives both tensor cores =====
+    if (rank == 0) {
+      constexpr uint32_t idesc = make_idesc_pair(AK != kAK, BKIND == kBMN);
+      int stage = 0, buf = 0;
+      uint32_t phase = 0, buf_phases = 0;          // bit b: phase of accumulator b
+      bool ok = true;
+      for (int64_t u = pair; u < sched.units && ok; u += npairs) {
+        const Unit w = sched.unit(u);
+        if (lane == 0)
+          ok = mbar_wait2(smem_u32(&ctl->tmem_empty[0]) + 8u * buf, ((buf_phases >> buf) & 1u) ^ 1u, abort_flag, peer_abort);
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) break;
+        tc_fence_after();
+        for (int kb = w.kb0; kb < w.kb1; ++kb) {
+          if (lane == 0) {
+            ok = mbar_wait2(smem_u32(&ctl->full[stage]), phase, abort_flag, peer_abort);
+            if (ok) {
+              tc_fence_after();
+              const uint32_t sA = smem_base + stage * kStage2Bytes;
+              const uint32_t sB = sA + kStage2Bytes / 2;
+#pragma unroll
+              for (int k = 0; k < BK / 16; ++k) {
+                const uint64_t adesc = (AK == kAK) ? make_desc(sA + k * 32, 16, 1024) : make_desc(sA + k * 2048, 8192, 1024);
+                const uint64_t bdesc = (BKIND == kBK_) ? make_desc(sB + k * 32, 16, 1024) : make_desc(sB + k * 2048, 8192, 1024);
+                tc_mma_pair(tmem_base + buf * 256, adesc, bdesc, idesc, (kb > w.kb0 || k > 0) ? 1u : 0u);
+              }
+              tc_commit_pair(smem_u32(&ctl->empty[stage]));          // frees the stage in both CTAs
+              if (kb == w.kb1 - 1) tc_commit_pair(smem_u32(&ctl->tmem_full[0]) + 8u * buf);
+            }
+          }
+          ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+          if (!ok) break;
+          if (++stage == kStages2) { stage = 0; phase ^= 1u; }
+        }
+        buf_phases ^= 1u << buf;
+        buf ^= 1;
+      }
+    }
+  } else {
+    // ===== epilogue: thread = one accumulator row of this CTA, 128 columns per warp =====
+    const int q = warp & 3;
+    const int c_first = ((warp - 2) >> 2) * (BN / (kEpiWarps2 / 4));
+    const uint32_t empty_bar = map_to_cta(smem_u32(&ctl->tmem_empty[0]), 0u);     // [b] is 8 bytes further
+    int buf = 0;
+    uint32_t buf_phases = 0;
+    bool ok = true;
+    for (int64_t u = pair; u < sched.units && ok; u += npairs) {
+      const Unit w = sched.unit(u);
+      if (lane == 0) ok = mbar_wait2(smem_u32(&ctl->tmem_full[0]) + 8u * buf, (buf_phases >> buf) & 1u, abort_flag, peer_abort);
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) break;
+      tc_fence_after();
+      const int64_t m = w.m0 + 128 * (int64_t)rank + q * 32 + lane;
+      const bool row_ok = m < sched.M;
+#pragma unroll 1
+      for (int c0 = c_first; c0 < c_first + BN / (kEpiWarps2 / 4); c0 += 32) {
+        const int64_t n = w.n0 + c0;
+        if (n >= p.N) break;                  // warp-uniform
+        uint32_t r[32];
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 256 + c0), r);
+        tmem_ld_wait();
+        epilogue_chunk<EPI>(p, r, m, n, row_ok, w.split);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(empty_bar + 8u * buf);
+      buf_phases ^= 1u << buf;
+      buf ^= 1;
+    }
+  }
+
+  // ===== teardown: neither CTA leaves (or frees tensor memory) while the other may still use it =====
+  tc_fence_before();
+  cluster_sync_all();
+  if (tid == 0 && ctl->abort_flag != 0) raise_status(p.dev_status, RAD_DEV_ETIMEOUT);
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
 // Sum of the K-split partial tiles in split order; rows may be scattered (same-sample).
 __global__ void __launch_bounds__(256) dw_reduce_kernel(const float* partial, int64_t partial_rows, int splits,
                                                         int64_t M, const int64_t* M_dev, int64_t N,
@@ -758,6 +1008,38 @@ int launch(const TcParams& p, const CUtensorMap& ta, const CUtensorMap& tb, int6
   return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
 }
 
+template <int AK, int BKIND, int EPI>
+int launch_pair(const TcParams& p, const CUtensorMap& ta, const CUtensorMap& tb, int64_t max_units, cudaStream_t s) {
+  constexpr size_t smem = (size_t)kStages2 * kStage2Bytes + sizeof(SmemCtl2) + 1024;
+  static_assert(smem <= 227 * 1024, "stage ring too deep");
+  auto kernel = tc_gemm_pair_kernel<AK, BKIND, EPI>;
+  // The kernel is persistent: the grid must not exceed the clusters that can be resident at once
+  // (SM pairs that can host a cluster; fewer than half the SM count on some parts).
+  static int resident_pairs = 0;
+  if (resident_pairs == 0) {
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return RAD_ECUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * (num_sms() / 2));
+    cfg.blockDim = dim3(kThreads2);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n <= 0) {
+      (void)cudaGetLastError();
+      n = num_sms() / 2;
+    }
+    resident_pairs = std::min(n, num_sms() / 2);
+  }
+  const int pairs = (int)std::max<int64_t>(1, std::min<int64_t>(max_units, resident_pairs));
+  count_launch();
+  kernel<<<2 * pairs, kThreads2, smem, s>>>(p, ta, tb);
+  return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
+}
+
 bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
 
 }  // namespace
@@ -774,7 +1056,7 @@ int tc_forward(int act, int64_t B, int64_t D, int64_t H, const void* A, int64_t 
                const float* bias, void* out_act, int64_t ld_act, float* out_z, int64_t ld_z, void* out_zlow,
                int64_t ld_zlow, uint32_t* relubits, int32_t* dev_status, cudaStream_t s) {
   CUtensorMap ta, tb;
-  int rc = make_map(&ta, A, D, B, lda, 256);          // K-major A: box 64 (K) x 256 rows
+  int rc = make_map(&ta, A, D, B, lda, 128);          // K-major A: box 64 (K) x 128 rows (one CTA of the pair)
   if (rc != RAD_OK) return rc;
   rc = make_map(&tb, W, H, D, ldw, 64);               // MN-major B: box 64 (N) x 64 K rows
   if (rc != RAD_OK) return rc;
@@ -784,23 +1066,23 @@ int tc_forward(int act, int64_t B, int64_t D, int64_t H, const void* A, int64_t 
   p.out_act = static_cast<bf16*>(out_act); p.ld_act = ld_act; p.out_z = out_z; p.ld_z = ld_z;
   p.out_zlow = static_cast<bf16*>(out_zlow); p.ld_zlow = ld_zlow; p.relubits = relubits; p.w32 = ceil_div(H, 32);
   p.dev_status = dev_status;
-  return launch<kAK, kBMN, kFwd>(p, ta, tb, ceil_div(B, BM) * ceil_div(H, BN), s);
+  return launch_pair<kAK, kBMN, kFwd>(p, ta, tb, ceil_div(B, BM) * ceil_div(H, BN), s);
 }
 
 int tc_input_grad(int64_t B, int64_t D, int64_t H, const void* dZ, int64_t ldz, const void* W, int64_t ldw,
                   const uint32_t* relubits_prev, const void* z_prev, int64_t ld_zprev, void* dZ_prev, int64_t ldp,
                   int32_t* dev_status, cudaStream_t s) {
   CUtensorMap ta, tb;
-  int rc = make_map(&ta, dZ, H, B, ldz, 256);         // K-major A (K = H)
+  int rc = make_map(&ta, dZ, H, B, ldz, 128);         // K-major A (K = H)
   if (rc != RAD_OK) return rc;
-  rc = make_map(&tb, W, H, D, ldw, 256);              // K-major B: rows d (N), K = H contiguous
+  rc = make_map(&tb, W, H, D, ldw, 128);              // K-major B: rows d (N), K = H contiguous
   if (rc != RAD_OK) return rc;
   TcParams p = {};
   p.M = B; p.N = D; p.K = H; p.splits = 1; p.num_stages = 3;
   p.relubits_prev = relubits_prev; p.z_prev = static_cast<const bf16*>(z_prev); p.ld_zprev = ld_zprev;
   p.out_dx = static_cast<bf16*>(dZ_prev); p.ld_dx = ldp;
   p.dev_status = dev_status;
-  return launch<kAK, kBK_, kDx>(p, ta, tb, ceil_div(B, BM) * ceil_div(D, BN), s);
+  return launch_pair<kAK, kBK_, kDx>(p, ta, tb, ceil_div(B, BM) * ceil_div(D, BN), s);
 }
 
 int64_t tc_weight_grad_workspace(const rad_store* st, int64_t H) {
@@ -828,7 +1110,7 @@ int tc_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H, 
     p.M = mmax; p.M_dev = st->nnz; p.row_idx = st->offsets;
     count_launch();
     zero_f32_kernel<<<grid_z, 256, 0, s>>>(dW, st->D, H, ldw);
-    rc = launch<kAMN, kBMN, kDw>(p, ta, tb, ceil_div(mmax, BM) * ceil_div(H, BN) * d.splits, s);
+    rc = launch_pair<kAMN, kBMN, kDw>(p, ta, tb, ceil_div(mmax, BM) * ceil_div(H, BN) * d.splits, s);
   } else {
     ta = tb;                                           // unused by the sparse-A kernel
     p.M = st->D;
