@@ -157,10 +157,11 @@ struct Unit {
 
 struct Schedule {
   int64_t M, m_tiles, n_tiles, ntiles, units;
-  int32_t kblocks, splits;
-  __device__ Schedule(int64_t M_, int64_t N_, int64_t K_, int32_t splits_) {
+  int32_t kblocks, splits, bm;
+  __device__ Schedule(int64_t M_, int64_t N_, int64_t K_, int32_t splits_, int32_t bm_ = BM) {
     M = M_;
-    m_tiles = (M + BM - 1) / BM;
+    bm = bm_;
+    m_tiles = (M + bm - 1) / bm;
     n_tiles = (N_ + BN - 1) / BN;
     ntiles = m_tiles * n_tiles;
     kblocks = (int32_t)((K_ + BK - 1) / BK);
@@ -176,7 +177,7 @@ struct Schedule {
     const int64_t g = t / per_group, r = t % per_group;
     const int64_t first_m = g * kRasterGroup;
     const int64_t gm = min((int64_t)kRasterGroup, m_tiles - first_m);
-    w.m0 = (first_m + r % gm) * BM;
+    w.m0 = (first_m + r % gm) * bm;
     w.n0 = (r / gm) * BN;
     w.split = (int32_t)s;
     w.kb0 = (int32_t)(s * kblocks / splits);
@@ -314,6 +315,73 @@ constexpr int kFirstExpanderWarp = 7;        // warp 6 feeds the compressed ring
 template <int AK> __host__ __device__ constexpr int epi_warps_for() { return AK == kASparse ? 4 : 16; }
 template <int AK> __host__ __device__ constexpr int threads_for() {
   return AK == kASparse ? 32 * (kFirstExpanderWarp + kExpanderWarps) : 32 * (2 + epi_warps_for<AK>());
+}
+
+// ---- expansion of one keep-bit word into the A_hat tile -------------------------------------------
+// sA: the stage's A tile (four 8 KB blocks of 64 columns, 128-byte rows per K index, 128-byte
+// swizzle); sC: keep bits, row offsets and packed values of store tile h of this K block; the thread
+// owns row r, columns 32 wq .. 32 wq + 31 of that store tile.  limit: staged values per tile.
+__device__ __forceinline__ void expand_word(uint8_t* sA, const uint8_t* sC, int h, int r, int wq, uint32_t limit) {
+  const uint32_t* bits = reinterpret_cast<const uint32_t*>(sC);
+  const unsigned short* rowoff = reinterpret_cast<const unsigned short*>(sC + kBitWords * 4);
+  const unsigned short* vals = reinterpret_cast<const unsigned short*>(sC + kIndexBytes);
+  const uint4 rowbits = *reinterpret_cast<const uint4*>(bits + r * 4);
+  const uint32_t word = wq == 0 ? rowbits.x : wq == 1 ? rowbits.y : wq == 2 ? rowbits.z : rowbits.w;
+  uint32_t pos = rowoff[r];
+  if (wq > 0) pos += __popc(rowbits.x);
+  if (wq > 1) pos += __popc(rowbits.y);
+  if (wq > 2) pos += __popc(rowbits.z);
+  uint8_t* rowp = sA + h * 16384 + (wq >> 1) * 8192 + r * 128;
+  const int j0 = (wq & 1) * 4;
+  const uint32_t cnt = __popc(word);
+  // one path per warp: the dense form is right for any word
+  if (__all_sync(0xffffffffu, cnt + (pos & 3u) <= 12u && cnt <= 10u)) {
+    // sparse word: zero this thread's 32 columns, then drop the kept values in place.  The
+    // values are consecutive from `pos`: three aligned 8-byte loads cover them (a word whose
+    // values would pass the end of the staged tile places nothing: the producer has flagged it)
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj)
+      *reinterpret_cast<uint4*>(rowp + (((j0 + jj) ^ (r & 7)) << 4)) = make_uint4(0, 0, 0, 0);
+    uint32_t rest = (pos + cnt <= limit) ? word : 0u;
+    const uint32_t e0 = pos & 3u;
+    const uint2* win = reinterpret_cast<const uint2*>(vals + (min(pos, limit) & ~3u));   // stays inside the ring
+    const uint2 q0 = win[0], q1 = win[1];
+    uint2 q2 = make_uint2(0u, 0u);
+    if (e0 + cnt > 8u) q2 = win[2];
+    // bring the first kept value to bit 0 of s0: drop whole words, then a half word
+    const bool drop = (e0 & 2u) != 0u;
+    const uint32_t w0 = drop ? q0.y : q0.x, w1 = drop ? q1.x : q0.y, w2 = drop ? q1.y : q1.x;
+    const uint32_t w3 = drop ? q2.x : q1.y, w4 = drop ? q2.y : q2.x, w5 = drop ? 0u : q2.y;
+    const uint32_t sh = (e0 & 1u) << 4;
+    const uint32_t sv[5] = {__funnelshift_r(w0, w1, sh), __funnelshift_r(w1, w2, sh), __funnelshift_r(w2, w3, sh),
+                            __funnelshift_r(w3, w4, sh), __funnelshift_r(w4, w5, sh)};
+#pragma unroll
+    for (int i = 0; i < 10; ++i) {
+      if (rest == 0) break;
+      const int b = __ffs(rest) - 1;
+      rest &= rest - 1;
+      const unsigned short v = (unsigned short)(sv[i >> 1] >> (16 * (i & 1)));
+      const int j = j0 + (b >> 3);
+      *reinterpret_cast<unsigned short*>(rowp + ((j ^ (r & 7)) << 4) + ((b & 7) << 1)) = v;
+    }
+  } else {
+    // dense word: every column's value position follows from a popcount of the bits below
+    // it, so the 32 loads are independent; each 16-byte chunk is written once
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+      uint32_t pk[4];
+#pragma unroll
+      for (int e = 0; e < 8; e += 2) {
+        const int b0 = jj * 8 + e;
+        const uint32_t p0 = pos + __popc(word & ((1u << b0) - 1u));
+        const uint32_t p1 = pos + __popc(word & ((2u << b0) - 1u));
+        const uint32_t v0 = ((word >> b0) & 1u) && p0 < limit ? vals[p0] : 0u;
+        const uint32_t v1 = ((word >> (b0 + 1)) & 1u) && p1 < limit ? vals[p1] : 0u;
+        pk[e >> 1] = v0 | (v1 << 16);
+      }
+      *reinterpret_cast<uint4*>(rowp + (((j0 + jj) ^ (r & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+    }
+  }
 }
 
 template <int AK, int BKIND, int EPI>
@@ -544,67 +612,7 @@ tc_gemm_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, const 
         if (h < w.halves) {
           uint8_t* sA = smem + (size_t)stage * stage_bytes;
           const uint8_t* sC = comp_base + (size_t)slot * comp_slot + (size_t)h * comp_half;
-          const uint32_t* bits = reinterpret_cast<const uint32_t*>(sC);
-          const unsigned short* rowoff = reinterpret_cast<const unsigned short*>(sC + kBitWords * 4);
-          const unsigned short* vals = reinterpret_cast<const unsigned short*>(sC + kIndexBytes);
-          const uint4 rowbits = *reinterpret_cast<const uint4*>(bits + r * 4);
-          const uint32_t word = wq == 0 ? rowbits.x : wq == 1 ? rowbits.y : wq == 2 ? rowbits.z : rowbits.w;
-          uint32_t pos = rowoff[r];
-          if (wq > 0) pos += __popc(rowbits.x);
-          if (wq > 1) pos += __popc(rowbits.y);
-          if (wq > 2) pos += __popc(rowbits.z);
-          uint8_t* rowp = sA + h * 16384 + (wq >> 1) * 8192 + r * 128;
-          const int j0 = (wq & 1) * 4;
-          const uint32_t limit = (uint32_t)p.comp_cap >> 1;
-          const uint32_t cnt = __popc(word);
-          // one path per warp: the dense form is right for any word
-          if (__all_sync(0xffffffffu, cnt + (pos & 3u) <= 12u && cnt <= 10u)) {
-            // sparse word: zero this thread's 32 columns, then drop the kept values in place.  The
-            // values are consecutive from `pos`: three aligned 8-byte loads cover them (a word whose
-            // values would pass the end of the staged tile places nothing: the producer has flagged it)
-#pragma unroll
-            for (int jj = 0; jj < 4; ++jj)
-              *reinterpret_cast<uint4*>(rowp + (((j0 + jj) ^ (r & 7)) << 4)) = make_uint4(0, 0, 0, 0);
-            uint32_t rest = (pos + cnt <= limit) ? word : 0u;
-            const uint32_t e0 = pos & 3u;
-            const uint2* win = reinterpret_cast<const uint2*>(vals + (min(pos, limit) & ~3u));   // stays inside the ring
-            const uint2 q0 = win[0], q1 = win[1];
-            uint2 q2 = make_uint2(0u, 0u);
-            if (e0 + cnt > 8u) q2 = win[2];
-            // bring the first kept value to bit 0 of s0: drop whole words, then a half word
-            const bool drop = (e0 & 2u) != 0u;
-            const uint32_t w0 = drop ? q0.y : q0.x, w1 = drop ? q1.x : q0.y, w2 = drop ? q1.y : q1.x;
-            const uint32_t w3 = drop ? q2.x : q1.y, w4 = drop ? q2.y : q2.x, w5 = drop ? 0u : q2.y;
-            const uint32_t sh = (e0 & 1u) << 4;
-            const uint32_t sv[5] = {__funnelshift_r(w0, w1, sh), __funnelshift_r(w1, w2, sh), __funnelshift_r(w2, w3, sh),
-                                    __funnelshift_r(w3, w4, sh), __funnelshift_r(w4, w5, sh)};
-#pragma unroll
-            for (int i = 0; i < 10; ++i) {
-              if (rest == 0) break;
-              const int b = __ffs(rest) - 1;
-              rest &= rest - 1;
-              const unsigned short v = (unsigned short)(sv[i >> 1] >> (16 * (i & 1)));
-              const int j = j0 + (b >> 3);
-              *reinterpret_cast<unsigned short*>(rowp + ((j ^ (r & 7)) << 4) + ((b & 7) << 1)) = v;
-            }
-          } else {
-            // dense word: every column's value position follows from a popcount of the bits below
-            // it, so the 32 loads are independent; each 16-byte chunk is written once
-#pragma unroll
-            for (int jj = 0; jj < 4; ++jj) {
-              uint32_t pk[4];
-#pragma unroll
-              for (int e = 0; e < 8; e += 2) {
-                const int b0 = jj * 8 + e;
-                const uint32_t p0 = pos + __popc(word & ((1u << b0) - 1u));
-                const uint32_t p1 = pos + __popc(word & ((2u << b0) - 1u));
-                const uint32_t v0 = ((word >> b0) & 1u) && p0 < limit ? vals[p0] : 0u;
-                const uint32_t v1 = ((word >> (b0 + 1)) & 1u) && p1 < limit ? vals[p1] : 0u;
-                pk[e >> 1] = v0 | (v1 << 16);
-              }
-              *reinterpret_cast<uint4*>(rowp + (((j0 + jj) ^ (r & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-            }
-          }
+          expand_word(sA, sC, h, r, wq, (uint32_t)p.comp_cap >> 1);
           fence_proxy_async();
         }
         __syncwarp();
@@ -870,6 +878,279 @@ tc_gemm_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, c
   }
 }
 
+// ---- two-CTA engine, sparse A (different-sample dW) --------------------------------------------------
+// The pair owns a 512 x 256 tile of dW: each CTA rebuilds its own 256 columns of A_hat (two store
+// tiles per K block, as in the one-CTA kernel) and loads half of the dZ tile, so the dZ bytes per
+// SM and the operand reads of each shared memory are halved.  Two MMAs per 16 rows of K, one per
+// 128-row half of each CTA's A tile; the four accumulators fill the pair's tensor memory.
+// Roles per CTA: 0 dZ producer, 1 MMA issuer (even CTA) and tensor-memory owner, 2-5 epilogue,
+// 6 producer of the compressed ring, 7-22 expanders.  full[s] lives in the even CTA: one arrival
+// with the dZ bytes of both CTAs plus one per expander warp of either CTA.
+constexpr int kSpAStageBytes = 256 * BK * 2;           // 32 KB: this CTA's 256 columns of A_hat
+constexpr int kSpBStageBytes = 128 * BK * 2;           // 16 KB: this CTA's 128 columns of dZ
+constexpr int kSpStageBytes = kSpAStageBytes + kSpBStageBytes;
+constexpr int kSpMaxStages = 4;
+constexpr int kSpThreads = 32 * (kFirstExpanderWarp + kExpanderWarps);
+
+struct SmemCtlSp {
+  uint64_t full[kSpMaxStages], empty[kSpMaxStages], comp_full[8], comp_empty[8], tmem_full, tmem_empty;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+// Arrival on a barrier of the even CTA from either CTA (default semantics, as for a local arrival;
+// writes meant for the tensor core are fenced into the async proxy before it).
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t caddr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(caddr) : "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSpThreads, 1)
+tc_sparse_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmB) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int stages = p.num_stages;
+  const int comp_half = kIndexBytes + p.comp_cap;               // index data + values of one store tile
+  const int comp_slot = 2 * comp_half;                           // compressed data of one K block of this CTA
+  uint8_t* comp_base = smem + (size_t)stages * kSpStageBytes;
+  SmemCtlSp* ctl = reinterpret_cast<SmemCtlSp*>(comp_base + (size_t)p.comp_depth * comp_slot);
+  volatile int* abort_flag = &ctl->abort_flag;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t rank = cluster_ctarank();
+  const uint32_t peer_abort = map_to_cta(smem_u32(&ctl->abort_flag), rank ^ 1u);
+  const Schedule sched(p.M, p.N, p.K, p.splits, 512);
+  const int64_t pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+  if (tid == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(smem_u32(&ctl->full[s]), 1 + 2 * kExpanderWarps);
+      mbar_init(smem_u32(&ctl->empty[s]), 1);
+    }
+    for (int c = 0; c < p.comp_depth; ++c) {
+      mbar_init(smem_u32(&ctl->comp_full[c]), 1);
+      mbar_init(smem_u32(&ctl->comp_empty[c]), kExpanderWarps);
+    }
+    mbar_init(smem_u32(&ctl->tmem_full), 1);
+    mbar_init(smem_u32(&ctl->tmem_empty), 8);          // four epilogue warps in each CTA
+    ctl->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(&ctl->tmem_base)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  cluster_sync_all();
+  tc_fence_after();
+  const uint32_t tmem_base = ctl->tmem_base;
+  const uint32_t smem_base = smem_u32(smem);
+  // store tiles (128 columns each) of this CTA's 256 columns that exist, per unit: 0, 1 or 2
+  auto own_halves = [&](const Unit& w) -> int {
+    const int64_t first = (w.m0 + 256 * (int64_t)rank) / kTileCols;
+    return (int)max((int64_t)0, min((int64_t)2, (int64_t)p.ncb - first));
+  };
+
+  if (warp == 0) {
+    // ===== dZ producer: this CTA's 128 columns of the dZ tile =====
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int64_t u = pair; u < sched.units && ok; u += npairs) {
+      const Unit w = sched.unit(u);
+      const int n_own = (int)w.n0 + 128 * (int)rank;
+      for (int kb = w.kb0; kb < w.kb1; ++kb) {
+        if (lane == 0) {
+          ok = mbar_wait2(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, peer_abort);
+          if (ok) {
+            const uint32_t sB = smem_base + stage * kSpStageBytes + kSpAStageBytes;
+            if (rank == 0) mbar_arrive_expect_tx(smem_u32(&ctl->full[stage]), 2 * kSpBStageBytes);   // both CTAs' bytes
+            const uint32_t full = map_to_cta(smem_u32(&ctl->full[stage]), 0u);
+#pragma unroll
+            for (int c = 0; c < 2; ++c) tma_load_2d_pair(sB + c * 8192, &tmB, n_own + c * 64, kb * BK, full);
+          }
+        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) break;
+        if (++stage == stages) { stage = 0; phase ^= 1u; }
+      }
+    }
+    if (lane == 0) {   // every commit aimed at this CTA's stage barriers has landed before the CTA may leave
+      for (int i = 0; i < stages && ok; ++i) {
+        ok = mbar_wait2(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, peer_abort);
+        if (++stage == stages) { stage = 0; phase ^= 1u; }
+      }
+    }
+  } else if (warp == 1) {
+    // ===== MMA issuer (even CTA) =====
+    if (rank == 0) {
+      constexpr uint32_t idesc = make_idesc_pair(true, true);
+      int stage = 0;
+      uint32_t phase = 0, unit_phase = 0;
+      bool ok = true;
+      for (int64_t u = pair; u < sched.units && ok; u += npairs) {
+        const Unit w = sched.unit(u);
+        if (lane == 0) ok = mbar_wait2(smem_u32(&ctl->tmem_empty), unit_phase ^ 1u, abort_flag, peer_abort);
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) break;
+        tc_fence_after();
+        for (int kb = w.kb0; kb < w.kb1; ++kb) {
+          if (lane == 0) {
+            ok = mbar_wait2(smem_u32(&ctl->full[stage]), phase, abort_flag, peer_abort);
+            if (ok) {
+              tc_fence_after();
+              const uint32_t sA = smem_base + stage * kSpStageBytes;
+              const uint32_t sB = sA + kSpAStageBytes;
+#pragma unroll
+              for (int k = 0; k < BK / 16; ++k) {
+                const uint64_t bdesc = make_desc(sB + k * 2048, 8192, 1024);
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+                  tc_mma_pair(tmem_base + h * 256, make_desc(sA + h * 16384 + k * 2048, 8192, 1024), bdesc, idesc,
+                              (kb > w.kb0 || k > 0) ? 1u : 0u);
+              }
+              tc_commit_pair(smem_u32(&ctl->empty[stage]));
+              if (kb == w.kb1 - 1) tc_commit_pair(smem_u32(&ctl->tmem_full));
+            }
+          }
+          ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+          if (!ok) break;
+          if (++stage == stages) { stage = 0; phase ^= 1u; }
+        }
+        unit_phase ^= 1u;
+      }
+    }
+  } else if (warp < 6) {
+    // ===== epilogue: thread = one accumulator row of each of this CTA's two halves =====
+    const int q = warp & 3;
+    const uint32_t empty_bar = map_to_cta(smem_u32(&ctl->tmem_empty), 0u);
+    uint32_t unit_phase = 0;
+    bool ok = true;
+    for (int64_t u = pair; u < sched.units && ok; u += npairs) {
+      const Unit w = sched.unit(u);
+      if (lane == 0) ok = mbar_wait2(smem_u32(&ctl->tmem_full), unit_phase, abort_flag, peer_abort);
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) break;
+      tc_fence_after();
+      for (int h = 0; h < 2; ++h) {
+        const int64_t m = w.m0 + 256 * (int64_t)rank + h * kHalfM + q * 32 + lane;
+        const bool row_ok = m < sched.M;
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          const int64_t n = w.n0 + c0;
+          if (n >= p.N) break;                  // warp-uniform
+          uint32_t r[32];
+          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * 256 + c0), r);
+          tmem_ld_wait();
+          epilogue_chunk<kDw>(p, r, m, n, row_ok, w.split);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_remote(empty_bar);
+      unit_phase ^= 1u;
+    }
+  } else if (warp == 6) {
+    // ===== producer of the compressed ring: keep bits + row offsets (1152 B) and packed values of
+    // this CTA's store tiles of each K block.  It runs ahead of the A/B ring: a slot is free as soon
+    // as the expanders have read it, long before the MMAs of that K block retire. =====
+    int slot = 0;
+    uint32_t cphase = 0;
+    bool ok = true;
+    for (int64_t u = pair; u < sched.units && ok; u += npairs) {
+      const Unit w = sched.unit(u);
+      const int halves = own_halves(w);
+      const int64_t tile_col = (w.m0 + 256 * (int64_t)rank) / kTileCols;
+      uint32_t off_lo = 0, off_mid = 0, off_hi = 0;   // tile offsets of K block (base + lane)
+      for (int kb = w.kb0; kb < w.kb1; ++kb) {
+        if (((kb - w.kb0) & 31) == 0 && halves > 0) {
+          const int kbl = kb + lane;
+          if (kbl < w.kb1) {
+            const int64_t t0 = (int64_t)kbl * p.ncb + tile_col;
+            off_lo = __ldg(p.offsets + t0);
+            off_mid = __ldg(p.offsets + t0 + 1);
+            off_hi = (halves == 2) ? __ldg(p.offsets + t0 + 2) : off_mid;
+          }
+        }
+        const int src = (kb - w.kb0) & 31;
+        const uint32_t o0 = __shfl_sync(0xffffffffu, off_lo, src);
+        const uint32_t o1 = __shfl_sync(0xffffffffu, off_mid, src);
+        const uint32_t o2 = __shfl_sync(0xffffffffu, off_hi, src);
+        if (lane == 0) {
+          ok = mbar_wait2(smem_u32(&ctl->comp_empty[slot]), cphase ^ 1u, abort_flag, peer_abort);
+          if (ok) {
+            const uint32_t cfull = smem_u32(&ctl->comp_full[slot]);
+            const uint32_t sC = smem_u32(comp_base) + slot * comp_slot;
+            const int64_t t0 = (int64_t)kb * p.ncb + tile_col;
+            uint32_t vb0 = halves > 0 ? (o1 - o0) * 2u : 0u, vb1 = halves > 1 ? (o2 - o1) * 2u : 0u;
+            bool bad = false;
+            if (vb0 > (uint32_t)p.comp_cap || (int64_t)o1 > p.values_capacity) { vb0 = 0; bad = true; }
+            if (vb1 > (uint32_t)p.comp_cap || (int64_t)o2 > p.values_capacity) { vb1 = 0; bad = true; }
+            if (bad) raise_status(p.dev_status, RAD_DEV_ECAPACITY);
+            mbar_arrive_expect_tx(cfull, (uint32_t)kIndexBytes * halves + vb0 + vb1);
+            if (halves > 0) {
+              bulk_load(sC, p.keepbits + t0 * kTileWords, kIndexBytes, cfull);
+              if (vb0 != 0) bulk_load(sC + kIndexBytes, p.values + o0, vb0, cfull);
+            }
+            if (halves > 1) {
+              bulk_load(sC + comp_half, p.keepbits + (t0 + 1) * kTileWords, kIndexBytes, cfull);
+              if (vb1 != 0) bulk_load(sC + comp_half + kIndexBytes, p.values + o1, vb1, cfull);
+            }
+          }
+        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) break;
+        if (++slot == p.comp_depth) { slot = 0; cphase ^= 1u; }
+      }
+    }
+  } else {
+    // ===== expanders: rebuild this CTA's A_hat tile (64 K rows x 256 columns, M-major, swizzled) =====
+    // One thread per keep-bit word: half h = columns 128h..128h+127 of the tile (one store tile),
+    // row r of the slab, columns 32*wq..32*wq+31 of that half.  The row's first value is given by
+    // the stored row offset; the words before this one in the row are counted with popc.
+    // Eight consecutive lanes take eight consecutive rows of the same word column: with the
+    // 128-byte swizzle their 16-byte zero stores then fall on eight different bank groups.
+    const int et = tid - 32 * kFirstExpanderWarp;            // 0..511
+    const int h = et >> 8, wi = et & 255;
+    const int r = (wi & 7) + ((wi >> 5) << 3), wq = (wi >> 3) & 3;
+    int stage = 0, slot = 0;
+    uint32_t phase = 0, cphase = 0;
+    bool ok = true;
+    for (int64_t u = pair; u < sched.units && ok; u += npairs) {
+      const Unit w = sched.unit(u);
+      const int halves = own_halves(w);
+      for (int kb = w.kb0; kb < w.kb1; ++kb) {
+        ok = mbar_wait2(smem_u32(&ctl->comp_full[slot]), cphase, abort_flag, peer_abort) &&
+             mbar_wait2(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, peer_abort);     // A tile of this stage is free
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        // columns past the layer's width keep whatever the buffer held: their accumulator rows are never written
+        if (h < halves) {
+          uint8_t* sA = smem + (size_t)stage * kSpStageBytes;
+          const uint8_t* sC = comp_base + (size_t)slot * comp_slot + (size_t)h * comp_half;
+          expand_word(sA, sC, h, r, wq, (uint32_t)p.comp_cap >> 1);
+          fence_proxy_async();
+        }
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive_remote(map_to_cta(smem_u32(&ctl->full[stage]), 0u));
+          mbar_arrive(smem_u32(&ctl->comp_empty[slot]));
+        }
+        if (++stage == stages) { stage = 0; phase ^= 1u; }
+        if (++slot == p.comp_depth) { slot = 0; cphase ^= 1u; }
+      }
+    }
+  }
+
+  // ===== teardown: neither CTA leaves (or frees tensor memory) while the other may still use it =====
+  tc_fence_before();
+  cluster_sync_all();
+  if (tid == 0 && ctl->abort_flag != 0) raise_status(p.dev_status, RAD_DEV_ETIMEOUT);
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
 // Sum of the K-split partial tiles in split order; rows may be scattered (same-sample).
 __global__ void __launch_bounds__(256) dw_reduce_kernel(const float* partial, int64_t partial_rows, int splits,
                                                         int64_t M, const int64_t* M_dev, int64_t N,
@@ -940,10 +1221,9 @@ int num_sms() {
 // (about 1024 tensor-pipe clocks): waves x K blocks per unit, plus what writing and re-reading the
 // float32 partial tiles costs at HBM speed.  Pure function of the shapes, so the workspace query
 // and the launch agree.
-int choose_splits(int64_t m_tiles, int64_t n_tiles, int64_t kblocks) {
-  const int64_t sms = kNumSMsDefault;
+int choose_splits(int64_t m_tiles, int64_t n_tiles, int64_t kblocks, int64_t bm = BM, int64_t sms = kNumSMsDefault) {
   const double kblock_us = 0.55;                                            // 1024 clk at ~1.9 GHz
-  const double partial_us = (double)(m_tiles * BM) * (double)(n_tiles * BN) * 8.0 / 6.5e6;   // per split
+  const double partial_us = (double)(m_tiles * bm) * (double)(n_tiles * BN) * 8.0 / 6.5e6;   // per split
   int best = 1;
   double best_cost = 1e300;
   for (int s = 1; s <= kMaxSplits && s <= kblocks; ++s) {
@@ -975,14 +1255,16 @@ DwPlan plan_dw(const rad_store* st, int64_t H) {
     int64_t cap = (int64_t)(n * pe + 8.0 * std::sqrt(n * pe * (1.0 - pe)) + 16.0);
     cap = std::min<int64_t>(round_up(cap, 8), (int64_t)n) * 2;
     d.comp_cap = (int)round_up(cap, 128);
-    // shared memory: 64 KB per A/B stage plus a ring of compressed slots, at least one deeper than
-    // the A/B ring when it fits
-    const int64_t budget = 227 * 1024 - 2048 - (int64_t)sizeof(SmemCtl);
+    // shared memory: 48 KB per A/B stage plus a ring of compressed slots
+    const int64_t budget = 227 * 1024 - 2048 - (int64_t)sizeof(SmemCtlSp);
     const int64_t slot = 2 * (kIndexBytes + d.comp_cap);
-    d.stages = (3 * 65536 + 3 * slot <= budget) ? 3 : 2;
-    d.comp_depth = (int)std::max<int64_t>(2, std::min<int64_t>(6, (budget - d.stages * 65536) / slot));
+    d.stages = (4 * kSpStageBytes + 3 * slot <= budget) ? 4 : (3 * kSpStageBytes + 2 * slot <= budget) ? 3 : 2;
+    d.comp_depth = (int)std::max<int64_t>(2, std::min<int64_t>(6, (budget - d.stages * kSpStageBytes) / slot));
+    d.splits = choose_splits(ceil_div(m_expect, 512), ceil_div(H, BN), kblocks, 512, kNumSMsDefault / 2);
+    d.bytes = d.splits > 1 ? (int64_t)d.splits * d.partial_rows * H * 4 : 0;
+    return d;
   }
-  d.splits = choose_splits(ceil_div(m_expect, BM), ceil_div(H, BN), kblocks);
+  d.splits = choose_splits(ceil_div(m_expect, BM), ceil_div(H, BN), kblocks, BM, kNumSMsDefault / 2);
   d.bytes = d.splits > 1 ? (int64_t)d.splits * d.partial_rows * H * 4 : 0;
   return d;
 }
@@ -1037,6 +1319,42 @@ int launch_pair(const TcParams& p, const CUtensorMap& ta, const CUtensorMap& tb,
   const int pairs = (int)std::max<int64_t>(1, std::min<int64_t>(max_units, resident_pairs));
   count_launch();
   kernel<<<2 * pairs, kThreads2, smem, s>>>(p, ta, tb);
+  return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
+}
+
+// Clusters of two CTAs of `kernel` that can be resident at once.
+template <typename K>
+int resident_pairs_of(K kernel, int threads, size_t smem) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * (num_sms() / 2));
+  cfg.blockDim = dim3(threads);
+  cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n <= 0) {
+    (void)cudaGetLastError();
+    n = num_sms() / 2;
+  }
+  return std::min(n, num_sms() / 2);
+}
+
+int launch_sparse_pair(const TcParams& p, const CUtensorMap& tb, int64_t max_units, cudaStream_t s) {
+  const size_t smem = (size_t)p.num_stages * kSpStageBytes + (size_t)p.comp_depth * 2 * (kIndexBytes + p.comp_cap) +
+                      sizeof(SmemCtlSp) + 1024;
+  if (smem > 227 * 1024 || p.num_stages > kSpMaxStages || p.comp_depth > 8) return RAD_EUNSUPPORTED;
+  static int resident_pairs = 0;
+  if (resident_pairs == 0) {
+    if (cudaFuncSetAttribute(tc_sparse_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+      return RAD_ECUDA;
+    resident_pairs = resident_pairs_of(tc_sparse_pair_kernel, kSpThreads, 227 * 1024);
+  }
+  const int pairs = (int)std::max<int64_t>(1, std::min<int64_t>(max_units, resident_pairs));
+  count_launch();
+  tc_sparse_pair_kernel<<<2 * pairs, kSpThreads, smem, s>>>(p, tb);
   return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
 }
 
@@ -1116,7 +1434,7 @@ int tc_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H, 
     p.M = st->D;
     p.values = static_cast<const bf16*>(st->values); p.keepbits = st->keepbits; p.offsets = st->offsets;
     p.values_capacity = st->values_capacity; p.ncb = (int32_t)ceil_div(st->D, kTileCols); p.comp_cap = d.comp_cap;
-    rc = launch<kASparse, kBMN, kDw>(p, ta, tb, ceil_div(st->D, BM) * ceil_div(H, BN) * d.splits, s);
+    rc = launch_sparse_pair(p, tb, ceil_div(st->D, 512) * ceil_div(H, BN) * d.splits, s);
   }
   if (rc != RAD_OK) return rc;
   if (d.splits > 1) {
