@@ -6,15 +6,19 @@
 //   dW, diff.    dW = A_hat^T dZ             (A_hat tiles rebuilt in shared memory from keep bits
 //                                             and packed values; Sec. 4.2 / 4.3 "different sample")
 //
-// One CTA per SM, persistent.  A CTA owns a 256 x 256 output tile held as two 128 x 256
-// accumulators that fill all 512 tensor-memory columns; per 64-deep K block it issues eight
-// 128x256x16 MMAs.  Operands arrive by TMA (128-byte swizzle, no multicast) through a 3-stage
-// mbarrier ring; for the different-sample dW the A operand is written by sixteen "expander" warps
-// instead.  Warp roles: 0 TMA producer, 1 MMA issuer and tensor-memory owner, 2-5 epilogue,
-// (2-17 in the dense kernels), 6 producer of the compressed ring and 7-22 expanders (sparse A only).  Long contractions can be split along K; partial tiles are
-// summed in split order by a second kernel, so results are reproducible.
-// Every mbarrier wait is bounded: on expiry the CTA raises RAD_DEV_ETIMEOUT, all roles leave
-// their loops, tensor memory is released and the kernel returns.
+// Every kernel here runs on SM pairs: a cluster of two CTAs, one per SM, persistent, with one
+// thread of the even CTA issuing tcgen05.mma.cta_group::2 on operands that both CTAs stage in their
+// own shared memory (TMA, 128-byte swizzle, no multicast) through an mbarrier ring.
+//   dense kernels    256 x 256 tile per pair; each CTA keeps two alternating 128 x 256 float32
+//                    accumulators in tensor memory, so the epilogue of a tile (bias, activation,
+//                    ReLU bits, GELU', stores) runs under the MMAs of the next one.
+//   sparse-A kernel  512 x 256 tile per pair; sixteen "expander" warps per CTA write the A_hat
+//                    tile of each K block into shared memory instead of TMA.
+// Long dW contractions can be split along K; partial tiles are summed in split order by a second
+// kernel, so results are reproducible.
+// Every mbarrier wait is bounded: on expiry both CTAs of the pair raise their abort flags, all
+// roles leave their loops, the pair meets at a cluster barrier, tensor memory is released, the
+// kernel returns and the launch reports RAD_DEV_ETIMEOUT.
 #include <cuda.h>
 
 #include <algorithm>
@@ -27,8 +31,6 @@ namespace {
 
 constexpr int BM = 256, BN = 256, BK = 64;
 constexpr int kHalfM = 128;
-constexpr int kAStageBytes = BM * BK * 2;      // 32 KB
-constexpr int kBStageBytes = BN * BK * 2;      // 32 KB
 constexpr int kNumSMsDefault = 148;
 constexpr int kMaxSplits = 16;
 constexpr int kRasterGroup = 8;                // m-tiles per raster group
@@ -85,24 +87,6 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 }
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any legitimate wait here
 
-// Bounded wait.  Returns false if the CTA is aborting (this or another role timed out).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_timer_ns();
-  while (true) {
-#pragma unroll 1
-    for (int i = 0; i < 32; ++i)
-      if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag != 0) return false;
-    if (global_timer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
-  }
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
-}
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
@@ -110,15 +94,6 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
-}
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -141,18 +116,11 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
          ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 
-// Instruction descriptor: D = f32, A = B = bf16, M = 128, N = 256, operand major-ness as given.
-__host__ __device__ constexpr uint32_t make_idesc(bool a_mn, bool b_mn) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
-         ((256u >> 3) << 17) | ((128u >> 4) << 24);
-}
-
 // ---- work decomposition ---------------------------------------------------------------------------
 struct Unit {
   int64_t m0, n0;
   int32_t kb0, kb1;    // K blocks [kb0, kb1)
   int32_t split;
-  int32_t halves;      // 1 or 2 active 128-row halves
 };
 
 struct Schedule {
@@ -182,7 +150,6 @@ struct Schedule {
     w.split = (int32_t)s;
     w.kb0 = (int32_t)(s * kblocks / splits);
     w.kb1 = (int32_t)((s + 1) * kblocks / splits);
-    w.halves = (w.m0 + kHalfM < M) ? 2 : 1;
     return w;
   }
 };
@@ -300,23 +267,9 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams& p, uint32_t (&r)[
 }
 
 // ---- shared memory layout -------------------------------------------------------------------------
-struct SmemCtl {
-  uint64_t full[4], empty[4], comp_full[8], comp_empty[8], tmem_full, tmem_empty;
-  uint32_t tmem_base;
-  int abort_flag;
-};
-
 constexpr int kIndexBytes = kTileWords * 4;   // keep bits + row offsets of one store tile (1152 B)
 constexpr int kExpanderWarps = 16;            // one thread per keep-bit word of the two halves
 constexpr int kFirstExpanderWarp = 7;        // warp 6 feeds the compressed ring
-// Epilogue warps: a warp reads the tensor-memory lanes 32 (warp % 4) .. +31; the dense kernels put
-// four warps on each lane quarter (64 accumulator columns each), since their epilogue is not
-// overlapped with the next tile's MMAs and carries the activation math.
-template <int AK> __host__ __device__ constexpr int epi_warps_for() { return AK == kASparse ? 4 : 16; }
-template <int AK> __host__ __device__ constexpr int threads_for() {
-  return AK == kASparse ? 32 * (kFirstExpanderWarp + kExpanderWarps) : 32 * (2 + epi_warps_for<AK>());
-}
-
 // ---- expansion of one keep-bit word into the A_hat tile -------------------------------------------
 // sA: the stage's A tile (four 8 KB blocks of 64 columns, 128-byte rows per K index, 128-byte
 // swizzle); sC: keep bits, row offsets and packed values of store tile h of this K block; the thread
@@ -381,258 +334,6 @@ __device__ __forceinline__ void expand_word(uint8_t* sA, const uint8_t* sC, int 
       }
       *reinterpret_cast<uint4*>(rowp + (((j0 + jj) ^ (r & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
     }
-  }
-}
-
-template <int AK, int BKIND, int EPI>
-__global__ void __launch_bounds__(threads_for<AK>(), 1)
-tc_gemm_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB) {
-  extern __shared__ uint8_t smem_raw[];
-  // 1024-byte alignment for the 128-byte swizzle atoms
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  const int stages = p.num_stages;
-  const int comp_half = (AK == kASparse) ? (kIndexBytes + p.comp_cap) : 0;   // index data + values of one half
-  constexpr int stage_bytes = kAStageBytes + kBStageBytes;      // 64 KB: swizzle atoms stay 1024-byte aligned
-  const int comp_slot = 2 * comp_half;                           // compressed data of one K block (two halves)
-  uint8_t* comp_base = smem + (size_t)stages * stage_bytes;
-  SmemCtl* ctl = reinterpret_cast<SmemCtl*>(comp_base + (size_t)p.comp_depth * comp_slot);
-  volatile int* abort_flag = &ctl->abort_flag;
-
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  // rows of the problem: for the same-sample dW the number of kept columns lives in device memory
-  int64_t m_rows = p.M;
-  if (p.M_dev != nullptr) {
-    int64_t md;
-    asm volatile("ld.global.cg.s64 %0, [%1];" : "=l"(md) : "l"(p.M_dev) : "memory");
-    m_rows = md < m_rows ? md : m_rows;
-  }
-  const Schedule sched(m_rows, p.N, p.K, p.splits);
-  if (tid == 0) {
-    for (int s = 0; s < stages; ++s) {
-      mbar_init(smem_u32(&ctl->full[s]), AK == kASparse ? 1 + kExpanderWarps : 1);
-      mbar_init(smem_u32(&ctl->empty[s]), 1);
-    }
-    for (int c = 0; c < p.comp_depth; ++c) {
-      mbar_init(smem_u32(&ctl->comp_full[c]), 1);
-      mbar_init(smem_u32(&ctl->comp_empty[c]), kExpanderWarps);
-    }
-    mbar_init(smem_u32(&ctl->tmem_full), 1);
-    mbar_init(smem_u32(&ctl->tmem_empty), 32 * epi_warps_for<AK>());
-    ctl->abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (warp == 1) {   // tensor memory: all 512 columns (two 128 x 256 float32 accumulators)
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(smem_u32(&ctl->tmem_base)), "r"(512u) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = ctl->tmem_base;
-  const uint32_t smem_base = smem_u32(smem);
-
-  if (warp == 0) {
-    // ===== TMA producer for the A and B tiles (one lane issues) =====
-    int stage = 0;
-    uint32_t phase = 0;
-    bool ok = true;
-    for (int64_t u = blockIdx.x; u < sched.units && ok; u += gridDim.x) {
-      const Unit w = sched.unit(u);
-      for (int kb = w.kb0; kb < w.kb1; ++kb) {
-        if (lane == 0) {
-          ok = mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag);
-          if (ok) {
-            const uint32_t sA = smem_base + stage * stage_bytes;
-            const uint32_t sB = sA + kAStageBytes;
-            const uint32_t full = smem_u32(&ctl->full[stage]);
-            const int k0 = kb * BK;
-            if (AK == kASparse) {
-              mbar_arrive_expect_tx(full, kBStageBytes);
-            } else {
-              mbar_arrive_expect_tx(full, kAStageBytes + kBStageBytes);
-              if (AK == kAK) {
-                tma_load_2d(sA, &tmA, k0, (int)w.m0, full);                       // 64 (K) x 256 rows
-              } else {
-#pragma unroll
-                for (int c = 0; c < 4; ++c) tma_load_2d(sA + c * 8192, &tmA, (int)w.m0 + c * 64, k0, full);
-              }
-            }
-            if (BKIND == kBK_) {
-              tma_load_2d(sB, &tmB, k0, (int)w.n0, full);
-            } else {
-#pragma unroll
-              for (int c = 0; c < 4; ++c) tma_load_2d(sB + c * 8192, &tmB, (int)w.n0 + c * 64, k0, full);
-            }
-          }
-        }
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-        if (!ok) break;
-        if (++stage == stages) { stage = 0; phase ^= 1u; }
-      }
-    }
-  } else if (warp == 1) {
-    // ===== MMA issuer =====
-    constexpr uint32_t idesc = make_idesc(AK != kAK, BKIND == kBMN);
-    int stage = 0;
-    uint32_t phase = 0, unit_phase = 0;
-    bool ok = true;
-    for (int64_t u = blockIdx.x; u < sched.units && ok; u += gridDim.x) {
-      const Unit w = sched.unit(u);
-      if (lane == 0) ok = mbar_wait(smem_u32(&ctl->tmem_empty), unit_phase ^ 1u, abort_flag);
-      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-      if (!ok) break;
-      tc_fence_after();
-      for (int kb = w.kb0; kb < w.kb1; ++kb) {
-        if (lane == 0) {
-          ok = mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag);
-          if (ok) {
-            tc_fence_after();
-            const uint32_t sA = smem_base + stage * stage_bytes;
-            const uint32_t sB = sA + kAStageBytes;
-#pragma unroll
-            for (int k = 0; k < BK / 16; ++k) {
-              const uint64_t bdesc = (BKIND == kBK_) ? make_desc(sB + k * 32, 16, 1024)
-                                                     : make_desc(sB + k * 2048, 8192, 1024);
-              for (int h = 0; h < w.halves; ++h) {
-                const uint64_t adesc = (AK == kAK) ? make_desc(sA + h * 16384 + k * 32, 16, 1024)
-                                                   : make_desc(sA + h * 16384 + k * 2048, 8192, 1024);
-                tc_mma(tmem_base + h * 256, adesc, bdesc, idesc, (kb > w.kb0 || k > 0) ? 1u : 0u);
-              }
-            }
-            tc_commit(smem_u32(&ctl->empty[stage]));            // frees the stage when the MMAs retire
-            if (kb == w.kb1 - 1) tc_commit(smem_u32(&ctl->tmem_full));
-          }
-        }
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-        if (!ok) break;
-        if (++stage == stages) { stage = 0; phase ^= 1u; }
-      }
-      unit_phase ^= 1u;
-    }
-  } else if (warp < 2 + epi_warps_for<AK>()) {
-    // ===== epilogue: thread = one accumulator row (tensor-memory lane) and a range of columns =====
-    const int q = warp & 3;                      // lanes 32q .. 32q+31 are the ones this warp may read
-    constexpr int kColsPerWarp = BN / (epi_warps_for<AK>() / 4);
-    const int c_first = ((warp - 2) >> 2) * kColsPerWarp;
-    uint32_t unit_phase = 0;
-    bool ok = true;
-    for (int64_t u = blockIdx.x; u < sched.units && ok; u += gridDim.x) {
-      const Unit w = sched.unit(u);
-      ok = mbar_wait(smem_u32(&ctl->tmem_full), unit_phase, abort_flag);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      tc_fence_after();
-      for (int h = 0; h < w.halves; ++h) {
-        const int64_t m = w.m0 + h * kHalfM + q * 32 + lane;
-        const bool row_ok = m < sched.M;
-#pragma unroll 1
-        for (int c0 = c_first; c0 < c_first + kColsPerWarp; c0 += 32) {
-          const int64_t n = w.n0 + c0;
-          if (n >= p.N) break;                  // warp-uniform
-          uint32_t r[32];
-          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * 256 + c0), r);
-          tmem_ld_wait();
-          epilogue_chunk<EPI>(p, r, m, n, row_ok, w.split);
-        }
-      }
-      tc_fence_before();
-      mbar_arrive(smem_u32(&ctl->tmem_empty));
-      unit_phase ^= 1u;
-    }
-  } else if (AK == kASparse && warp == 6) {
-    // ===== producer of the compressed ring: keep bits + row offsets (1152 B) and packed values of
-    // the one or two store tiles of each K block.  It runs ahead of the A/B ring: a slot is free as
-    // soon as the expanders have read it, long before the MMAs of that K block retire. =====
-    int slot = 0;
-    uint32_t cphase = 0;
-    bool ok = true;
-    for (int64_t u = blockIdx.x; u < sched.units && ok; u += gridDim.x) {
-      const Unit w = sched.unit(u);
-      uint32_t off_lo = 0, off_mid = 0, off_hi = 0;   // tile offsets of K block (base + lane)
-      for (int kb = w.kb0; kb < w.kb1; ++kb) {
-        if (((kb - w.kb0) & 31) == 0) {
-          const int kbl = kb + lane;
-          if (kbl < w.kb1) {
-            const int64_t t0 = (int64_t)kbl * p.ncb + w.m0 / kTileCols;
-            off_lo = __ldg(p.offsets + t0);
-            off_mid = __ldg(p.offsets + t0 + 1);
-            off_hi = (w.halves == 2) ? __ldg(p.offsets + t0 + 2) : off_mid;
-          }
-        }
-        const int src = (kb - w.kb0) & 31;
-        const uint32_t o0 = __shfl_sync(0xffffffffu, off_lo, src);
-        const uint32_t o1 = __shfl_sync(0xffffffffu, off_mid, src);
-        const uint32_t o2 = __shfl_sync(0xffffffffu, off_hi, src);
-        if (lane == 0) {
-          ok = mbar_wait(smem_u32(&ctl->comp_empty[slot]), cphase ^ 1u, abort_flag);
-          if (ok) {
-            const uint32_t cfull = smem_u32(&ctl->comp_full[slot]);
-            const uint32_t sC = smem_u32(comp_base) + slot * comp_slot;
-            const int64_t t0 = (int64_t)kb * p.ncb + w.m0 / kTileCols;
-            uint32_t vb0 = (o1 - o0) * 2u, vb1 = (o2 - o1) * 2u;
-            bool bad = false;
-            if (vb0 > (uint32_t)p.comp_cap || (int64_t)o1 > p.values_capacity) { vb0 = 0; bad = true; }
-            if (vb1 > (uint32_t)p.comp_cap || (int64_t)o2 > p.values_capacity) { vb1 = 0; bad = true; }
-            if (bad) raise_status(p.dev_status, RAD_DEV_ECAPACITY);
-            mbar_arrive_expect_tx(cfull, (uint32_t)kIndexBytes * w.halves + vb0 + (w.halves == 2 ? vb1 : 0u));
-            bulk_load(sC, p.keepbits + t0 * kTileWords, kIndexBytes, cfull);
-            if (vb0 != 0) bulk_load(sC + kIndexBytes, p.values + o0, vb0, cfull);
-            if (w.halves == 2) {
-              bulk_load(sC + comp_half, p.keepbits + (t0 + 1) * kTileWords, kIndexBytes, cfull);
-              if (vb1 != 0) bulk_load(sC + comp_half + kIndexBytes, p.values + o1, vb1, cfull);
-            }
-          }
-        }
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-        if (!ok) break;
-        if (++slot == p.comp_depth) { slot = 0; cphase ^= 1u; }
-      }
-    }
-  } else if (AK == kASparse) {
-    // ===== expanders: rebuild the A_hat tile (64 K rows x 256 columns, M-major, swizzled) =====
-    // One thread per keep-bit word: half h = columns 128h..128h+127 of the tile (one store tile),
-    // row r of the slab, columns 32*wq..32*wq+31 of that half.  The row's first value is given by
-    // the stored row offset; the words before this one in the row are counted with popc.
-    // Eight consecutive lanes take eight consecutive rows of the same word column: with the
-    // 128-byte swizzle their 16-byte zero stores then fall on eight different bank groups.
-    const int et = tid - 32 * kFirstExpanderWarp;            // 0..511
-    const int h = et >> 8, wi = et & 255;
-    const int r = (wi & 7) + ((wi >> 5) << 3), wq = (wi >> 3) & 3;
-    int stage = 0, slot = 0;
-    uint32_t phase = 0, cphase = 0;
-    bool ok = true;
-    for (int64_t u = blockIdx.x; u < sched.units && ok; u += gridDim.x) {
-      const Unit w = sched.unit(u);
-      for (int kb = w.kb0; kb < w.kb1; ++kb) {
-        ok = mbar_wait(smem_u32(&ctl->comp_full[slot]), cphase, abort_flag) &&
-             mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag);     // A tile of this stage is free
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        if (h < w.halves) {
-          uint8_t* sA = smem + (size_t)stage * stage_bytes;
-          const uint8_t* sC = comp_base + (size_t)slot * comp_slot + (size_t)h * comp_half;
-          expand_word(sA, sC, h, r, wq, (uint32_t)p.comp_cap >> 1);
-          fence_proxy_async();
-        }
-        __syncwarp();
-        if (lane == 0) {
-          mbar_arrive(smem_u32(&ctl->full[stage]));
-          mbar_arrive(smem_u32(&ctl->comp_empty[slot]));
-        }
-        if (++stage == stages) { stage = 0; phase ^= 1u; }
-        if (++slot == p.comp_depth) { slot = 0; cphase ^= 1u; }
-      }
-    }
-  }
-
-  // ===== teardown =====
-  tc_fence_before();
-  __syncthreads();
-  if (tid == 0 && ctl->abort_flag != 0) raise_status(p.dev_status, RAD_DEV_ETIMEOUT);
-  if (warp == 1) {
-    tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
   }
 }
 
@@ -1267,27 +968,6 @@ DwPlan plan_dw(const rad_store* st, int64_t H) {
   d.splits = choose_splits(ceil_div(m_expect, BM), ceil_div(H, BN), kblocks, BM, kNumSMsDefault / 2);
   d.bytes = d.splits > 1 ? (int64_t)d.splits * d.partial_rows * H * 4 : 0;
   return d;
-}
-
-template <int AK, int BKIND, int EPI>
-int launch(const TcParams& p, const CUtensorMap& ta, const CUtensorMap& tb, int64_t max_units, cudaStream_t s) {
-  const int comp_half = (AK == kASparse) ? (kIndexBytes + p.comp_cap) : 0;
-  const size_t smem = (size_t)p.num_stages * (kAStageBytes + kBStageBytes) + (size_t)p.comp_depth * 2 * comp_half +
-                      sizeof(SmemCtl) + 1024;
-  auto kernel = tc_gemm_kernel<AK, BKIND, EPI>;
-  static bool configured = false;
-  static size_t configured_smem = 0;
-  if (!configured || smem > configured_smem) {
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
-      return RAD_ECUDA;
-    configured = true;
-    configured_smem = 227 * 1024;
-  }
-  if (smem > 227 * 1024) return RAD_EUNSUPPORTED;
-  const int grid = (int)std::max<int64_t>(1, std::min<int64_t>(max_units, num_sms()));
-  count_launch();
-  kernel<<<grid, threads_for<AK>(), smem, s>>>(p, ta, tb);
-  return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
 }
 
 template <int AK, int BKIND, int EPI>
