@@ -397,16 +397,25 @@ def run_ours(args):
     if dominant == "dW":
         ms_k = sum(t for _, t in dw_big) / len(dw_big)
         if args.variant == "different":
-            flops, what = 2.0 * B * 8192 * 8192, "tc_gemm_kernel<sparse A> dW, dense-tile flops 2*B*D*H"
+            flops, what = 2.0 * B * 8192 * 8192, "tc_sparse_pair_kernel (different-sample dW), dense-tile flops 2*B*D*H"
         else:
             k = int(lw.stores[1].nnz[0].item())
-            flops, what = 2.0 * B * k * 8192, "tc_gemm_kernel<MN,MN> dW, flops 2*B*k'*H on kept columns"
+            flops, what = 2.0 * B * k * 8192, "tc_gemm_pair_kernel<MN,MN> (same-sample dW), flops 2*B*k'*H on kept columns"
     else:
         ms_k = sum(t for _, t in fwd_big) / len(fwd_big)
-        flops, what = 2.0 * B * 8192 * 8192, "tc_gemm_kernel forward, flops 2*B*D*H"
+        flops, what = 2.0 * B * 8192 * 8192, "tc_gemm_pair_kernel forward, flops 2*B*D*H"
     achieved = flops / ms_k / 1e9
+    # DRAM bytes per launch from the ncu captures under profiles/ (batch 8192, 8192 x 8192 layer): bytes
+    # read grow with the batch and are scaled by B / 8192, the dW output does not grow.  Only the
+    # default workload has a capture.
+    traffic = None
+    if args.act == "gelu" and abs(args.p - 0.1) < 1e-9:
+        if dominant == "dW" and args.variant == "different":
+            traffic = int(351.5e6 * B / 8192 + 228.4e6)
+        elif dominant != "dW":
+            traffic = int((1095.8e6 + 251.4e6) * B / 8192)
     roofline = dict(bound="tensor", kernel=what, achieved=round(achieved, 1), peak=pk["tflops_sustained"],
-                    unit="TFLOP/s", frac=round(achieved / pk["tflops_sustained"], 4), traffic=None,
+                    unit="TFLOP/s", frac=round(achieved / pk["tflops_sustained"], 4), traffic=traffic,
                     peak_source=pk["source"] + " (sustained cuBLAS bf16)", ms_per_launch=round(ms_k, 4),
                     how="CUDA events around the call on the launching stream, inside the timed steps")
     store_big = [sum(v) / len(v) for (f, l), v in fam.items() if f == "store" and dims[l] == 8192]
@@ -418,7 +427,9 @@ def run_ours(args):
     ms_s = sum(store_big) / len(store_big)
     store_roofline = dict(bound="hbm", kernel="store kernel, one 8192-wide layer input",
                           achieved=round(sbytes / ms_s / 1e6, 1), peak=pk["hbm_gbs"], unit="GB/s",
-                          frac=round(sbytes / ms_s / 1e6 / pk["hbm_gbs"], 4), traffic=None,
+                          frac=round(sbytes / ms_s / 1e6 / pk["hbm_gbs"], 4),
+                          traffic=(int((134.3e6 + 7.0e6) * B / 8192)
+                                   if args.variant == "different" and abs(args.p - 0.1) < 1e-9 else None),
                           ms_per_launch=round(ms_s, 4), algorithmic_bytes=sbytes)
 
     # stored activation bytes versus full backprop (from the whole-net entry point's plan)
