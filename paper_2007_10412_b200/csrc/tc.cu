@@ -291,11 +291,15 @@ __device__ __forceinline__ void expand_word(uint8_t* sA, const uint8_t* sC, int 
   if (__all_sync(0xffffffffu, cnt + (pos & 3u) <= 12u && cnt <= 10u)) {
     // sparse word: zero this thread's 32 columns, then drop the kept values in place.  The
     // values are consecutive from `pos`: three aligned 8-byte loads cover them (a word whose
-    // values would pass the end of the staged tile places nothing: the producer has flagged it)
+    // values would pass the end of the staged tile places nothing: the producer has flagged it).
+    // Byte address of column c of this word in the swizzled row: base ^ (c << 1), because the
+    // 16-byte chunk index (j0 + (c >> 3)) ^ (r & 7) equals (c >> 3) ^ (j0 ^ (r & 7)) for j0 in {0, 4}
+    // and rows are 128-byte aligned.
+    const uint32_t base = smem_u32(rowp) ^ ((uint32_t)(j0 ^ (r & 7)) << 4);
 #pragma unroll
     for (int jj = 0; jj < 4; ++jj)
-      *reinterpret_cast<uint4*>(rowp + (((j0 + jj) ^ (r & 7)) << 4)) = make_uint4(0, 0, 0, 0);
-    uint32_t rest = (pos + cnt <= limit) ? word : 0u;
+      asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(base ^ (uint32_t)(jj << 4)), "r"(0u) : "memory");
+    const uint32_t rest = (pos + cnt <= limit) ? word : 0u;
     const uint32_t e0 = pos & 3u;
     const uint2* win = reinterpret_cast<const uint2*>(vals + (min(pos, limit) & ~3u));   // stays inside the ring
     const uint2 q0 = win[0], q1 = win[1];
@@ -308,14 +312,18 @@ __device__ __forceinline__ void expand_word(uint8_t* sA, const uint8_t* sC, int 
     const uint32_t sh = (e0 & 1u) << 4;
     const uint32_t sv[5] = {__funnelshift_r(w0, w1, sh), __funnelshift_r(w1, w2, sh), __funnelshift_r(w2, w3, sh),
                             __funnelshift_r(w3, w4, sh), __funnelshift_r(w4, w5, sh)};
+    // every lane runs the warp's longest word; a lane that has run out stores nothing.  The word is
+    // bit-reversed so that the next kept column is a leading-zero count away.
+    const uint32_t steps = __reduce_max_sync(0xffffffffu, rest != 0u ? cnt : 0u);
+    uint32_t rw = __brev(rest);
 #pragma unroll
     for (int i = 0; i < 10; ++i) {
-      if (rest == 0) break;
-      const int b = __ffs(rest) - 1;
-      rest &= rest - 1;
-      const unsigned short v = (unsigned short)(sv[i >> 1] >> (16 * (i & 1)));
-      const int j = j0 + (b >> 3);
-      *reinterpret_cast<unsigned short*>(rowp + ((j ^ (r & 7)) << 4) + ((b & 7) << 1)) = v;
+      if ((uint32_t)i >= steps) break;                  // warp-uniform
+      const uint32_t c = (uint32_t)__clz((int)rw);      // 32 once the word is used up
+      const uint32_t v = sv[i >> 1] >> (16 * (i & 1));
+      asm volatile("{\n\t.reg .pred k;\n\tsetp.ne.u32 k, %2, 0;\n\t@k st.shared.b16 [%0], %1;\n\t}"
+                   ::"r"(base ^ (c << 1)), "h"((unsigned short)v), "r"(rw) : "memory");
+      rw &= ~(0x80000000u >> (c & 31u));
     }
   } else {
     // dense word: every column's value position follows from a popcount of the bits below
@@ -372,17 +380,24 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) { 
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t caddr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(caddr) : "memory");
+// Arrival on a barrier of either CTA of the pair (default semantics, as for a local arrival: what
+// the waiter goes on to touch is ordered by tcgen05 or proxy fences issued before the arrival; a
+// cluster-scope release here would drain the SM's outstanding stores every time).
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t caddr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(caddr) : "memory");
 }
-// Bounded wait of the pair: on expiry both CTAs' abort flags are raised.
-__device__ __forceinline__ bool mbar_wait2(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t peer_abort) {
+// Bounded wait of the pair: on expiry both CTAs' abort flags are raised.  sleep_ns > 0: a long wait
+// off the critical path (an epilogue warp waiting for a whole tile) leaves the issue slots to others.
+__device__ __forceinline__ bool mbar_wait2(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t peer_abort,
+                                           uint32_t sleep_ns = 0) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   while (true) {
 #pragma unroll 1
-    for (int i = 0; i < 32; ++i)
+    for (int i = 0; i < 32; ++i) {
       if (mbar_try_wait(bar, parity)) return true;
+      if (sleep_ns != 0) __nanosleep(sleep_ns);
+    }
     if (*abort_flag != 0) return false;
     if (global_timer_ns() - t0 > kWaitLimitNs) {
       *abort_flag = 1;
@@ -546,7 +561,7 @@ tc_gemm_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, c
     bool ok = true;
     for (int64_t u = pair; u < sched.units && ok; u += npairs) {
       const Unit w = sched.unit(u);
-      if (lane == 0) ok = mbar_wait2(smem_u32(&ctl->tmem_full[0]) + 8u * buf, (buf_phases >> buf) & 1u, abort_flag, peer_abort);
+      if (lane == 0) ok = mbar_wait2(smem_u32(&ctl->tmem_full[0]) + 8u * buf, (buf_phases >> buf) & 1u, abort_flag, peer_abort, 200u);
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) break;
       tc_fence_after();
@@ -563,7 +578,7 @@ tc_gemm_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, c
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(empty_bar + 8u * buf);
+      if (lane == 0) mbar_arrive_remote(empty_bar + 8u * buf);
       buf_phases ^= 1u << buf;
       buf ^= 1;
     }
@@ -598,12 +613,6 @@ struct SmemCtlSp {
   uint32_t tmem_base;
   int abort_flag;
 };
-
-// Arrival on a barrier of the even CTA from either CTA (default semantics, as for a local arrival;
-// writes meant for the tensor core are fenced into the async proxy before it).
-__device__ __forceinline__ void mbar_arrive_remote(uint32_t caddr) {
-  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(caddr) : "memory");
-}
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSpThreads, 1)
 tc_sparse_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmB) {
@@ -728,7 +737,7 @@ tc_sparse_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmB)
     bool ok = true;
     for (int64_t u = pair; u < sched.units && ok; u += npairs) {
       const Unit w = sched.unit(u);
-      if (lane == 0) ok = mbar_wait2(smem_u32(&ctl->tmem_full), unit_phase, abort_flag, peer_abort);
+      if (lane == 0) ok = mbar_wait2(smem_u32(&ctl->tmem_full), unit_phase, abort_flag, peer_abort, 1000u);
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) break;
       tc_fence_after();
