@@ -440,6 +440,15 @@ def run_ours(args):
                   preact_bytes=s.preact_bytes, unsampled_bytes=s.unsampled_bytes, held_bytes=held,
                   full_backprop_bytes=s.full_backprop_bytes, ratio=round(s.full_backprop_bytes / held, 3))
 
+    # the same shapes with ReLU (1-bit derivatives instead of kept pre-activations): plan only, not run
+    if args.act != "relu":
+        _, sr = rad.rad_mlp_workspace(dims, B, "bf16", "relu", args.variant, args.p)
+        held_r = sr.value_bytes + sr.index_bytes + sr.relu_bytes + sr.preact_bytes + sr.unsampled_bytes
+        memory["same_shapes_relu"] = dict(value_bytes=sr.value_bytes, index_bytes=sr.index_bytes, relu_bytes=sr.relu_bytes,
+                                          preact_bytes=sr.preact_bytes, unsampled_bytes=sr.unsampled_bytes,
+                                          held_bytes=held_r, full_backprop_bytes=sr.full_backprop_bytes,
+                                          ratio=round(sr.full_backprop_bytes / held_r, 3))
+
     # end to end through rad_mlp_step: the batch comes from pinned host memory every step
     Xh = torch.empty(X.shape, dtype=bf).pin_memory()
     Xh.copy_(X)

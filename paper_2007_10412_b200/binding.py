@@ -269,6 +269,15 @@ def rad_linear_input_grad(dZ, W, relubits_prev=None, z_prev=None, dZ_prev=None, 
                                        _ptr(dev_status), _stream()), "rad_linear_input_grad")
 
 
+def rad_mlp_workspace(dims, B, dtype="f32", act="relu", variant="different", p=0.1):
+    """(workspace bytes, rad_step_stats) of a net shape; allocates nothing."""
+    dims_c = (C.c_int64 * len(dims))(*dims)
+    desc = rad_mlp_desc(len(dims) - 1, ACTS[act], DTYPES[dtype], VARIANTS[variant], dims_c, B, p, 0, 0)
+    nbytes, stats = C.c_int64(0), rad_step_stats()
+    _check(lib().rad_mlp_workspace(C.byref(desc), C.byref(nbytes), C.byref(stats)), "rad_mlp_workspace")
+    return nbytes.value, stats
+
+
 class MLPStep:
     """Owns the workspace and pointer tables of rad_mlp_step for one net shape."""
 
