@@ -88,6 +88,32 @@ def keep_mask(variant: str, B: int, D: int, p, seed: int, layer: int, step: int)
     return np.ascontiguousarray(m)
 
 
+def keep_mask_at(variant: str, rows, cols, p, seed: int, layer: int, step: int) -> np.ndarray:
+    """Keep decisions of the given rows x the given columns (len(rows) x len(cols), boolean): the same
+    counter, key and lane rule as keep_mask, evaluated only where asked, so that single tiles or
+    single columns of a layer too large to expand in full can be checked."""
+    T = keep_threshold(p)
+    rows = np.asarray(rows, dtype=np.uint64).reshape(-1, 1)
+    cols = np.asarray(cols, dtype=np.uint64).reshape(1, -1)
+    if variant == "different":
+        stream = STREAM_DIFFERENT
+    elif variant == "same":
+        rows, stream = np.zeros_like(rows), STREAM_SAME
+    else:
+        raise ValueError(variant)
+    c2 = np.uint64((layer & 0xFFFFFF) | (stream << 24))
+    words = philox4x32_10(cols // np.uint64(LANES_PER_CALL) + np.zeros_like(rows), rows + np.zeros_like(cols), c2,
+                          np.uint64(step & 0xFFFFFFFF), np.uint64(seed & 0xFFFFFFFF),
+                          np.uint64((seed >> 32) & 0xFFFFFFFF))
+    lane = (cols % np.uint64(LANES_PER_CALL)).astype(np.int64) + np.zeros(rows.shape, dtype=np.int64)
+    out = np.zeros(lane.shape, dtype=bool)
+    for j, w in enumerate(words):
+        w = np.broadcast_to(w, lane.shape)
+        out |= (lane == 2 * j) & ((w & np.uint32(0xFFFF)) < T)
+        out |= (lane == 2 * j + 1) & ((w >> np.uint32(16)) < T)
+    return out
+
+
 # --------------------------------------------------------------------------
 # number formats
 # --------------------------------------------------------------------------

@@ -1,0 +1,135 @@
+"""The wide layer of the bench workload (65536 x 8192 x 8192, bf16) through the same calls the bench
+times, checked on sampled outputs the oracle can compute one by one and on properties that hold at
+any size.  Inputs come from the seeded generators; nothing here is compared with a stored value."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import rad as orc
+from workloads import layer_inputs, to_bf16_grid
+
+from gpu_util import rel_err, to_host_f32
+
+pytestmark = pytest.mark.gpu
+
+B, D, H = 65536, 8192, 8192
+P, SEED, LAYER, STEP = 0.1, 5, 1, 3
+TILE_ROWS, TILE_COLS, TILE_WORDS, ALIGN = 64, 128, 288, 8
+
+
+@pytest.fixture(scope="module")
+def wide():
+    import paper_2007_10412_b200 as rad
+    A, dZ = layer_inputs(B, D, H, dtype="bf16", seed=77)
+    rng = np.random.default_rng(78)
+    W = to_bf16_grid(rng.standard_normal((D, H), dtype=np.float32) * np.float32(np.sqrt(2.0 / D)))
+    bias = rng.standard_normal(H, dtype=np.float32)
+    dev = dict(A=torch.from_numpy(A).to(torch.bfloat16).cuda(), dZ=torch.from_numpy(dZ).to(torch.bfloat16).cuda(),
+               W=torch.from_numpy(W).to(torch.bfloat16).cuda(), bias=torch.from_numpy(bias).cuda())
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    st = rad.Store("different", "bf16", B, D, P, seed=SEED, layer=LAYER, step=STEP, relu_bits=False)
+    rad.rad_linear_forward_store(dev["A"], st, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    yield dict(A=A, dZ=dZ, W=W, bias=bias, dev=dev, st=st, status=status, rad=rad)
+    del dev, st
+    torch.cuda.empty_cache()
+
+
+def test_store_sampled_tiles_are_bit_exact(wide):
+    st, A = wide["st"], wide["A"]
+    nslab, ncb = B // TILE_ROWS, D // TILE_COLS
+    ntiles = nslab * ncb
+    rng = np.random.default_rng(1)
+    tiles = [0, 1, ncb - 1, ncb, ntiles - 1, ntiles - ncb] + [int(t) for t in rng.integers(0, ntiles, 10)]
+    offsets = st.offsets.cpu().numpy().view(np.uint32)
+    scale = np.float32(orc.scale_factor(P))
+    for t in tiles:
+        slab, blk = divmod(t, ncb)
+        rows = np.arange(slab * TILE_ROWS, (slab + 1) * TILE_ROWS)
+        cols = np.arange(blk * TILE_COLS, (blk + 1) * TILE_COLS)
+        m = orc.keep_mask_at("different", rows, cols, P, SEED, LAYER, STEP)
+        words = st.keepbits[t * TILE_WORDS:(t + 1) * TILE_WORDS].cpu().numpy().view(np.uint32)
+        assert np.array_equal(words[:256], orc.pack_bits(m).reshape(-1)), t
+        rowoff = np.concatenate([[0], np.cumsum(m.sum(axis=1))[:-1]]).astype(np.uint16)
+        assert np.array_equal(words[256:].view(np.uint16), rowoff), t
+        n = int(m.sum())
+        padded = -(-n // ALIGN) * ALIGN
+        assert int(offsets[t + 1]) - int(offsets[t]) == padded, t
+        ref = orc.round_bf16(A[np.ix_(rows, cols)][m] * scale)
+        got = st.values[int(offsets[t]):int(offsets[t]) + padded].view(torch.int16).cpu().numpy().view(np.uint16)
+        assert np.array_equal(got[:n], orc.bf16_bits(ref)), t
+        assert (got[n:] == 0).all(), t
+
+
+def test_store_counts_hold_together(wide):
+    st = wide["st"]
+    ntiles = (B // TILE_ROWS) * (D // TILE_COLS)
+    words = st.keepbits.view(ntiles, TILE_WORDS)[:, :256].contiguous()
+    # set bits of every keep word, summed per tile on the device (16-bit lookups of a byte table)
+    table = torch.tensor([bin(i).count("1") for i in range(256)], dtype=torch.int32, device="cuda")
+    per_tile = torch.zeros(ntiles, dtype=torch.int64, device="cuda")
+    for sh in (0, 8, 16, 24):
+        per_tile += table[((words >> sh) & 0xFF).long()].sum(dim=1)
+    nnz = st.nnz.cpu().numpy()
+    assert int(per_tile.sum()) == int(nnz[0])
+    offsets = st.offsets.cpu().numpy().view(np.uint32).astype(np.int64)
+    assert offsets[0] == 0 and int(offsets[ntiles]) == int(nnz[1])
+    padded = ((per_tile + (ALIGN - 1)) // ALIGN * ALIGN).cpu().numpy()
+    assert np.array_equal(np.diff(offsets[:ntiles + 1]), padded)
+    # Binomial(B D, p_eff): six standard deviations
+    pe = orc.effective_p(P)
+    assert abs(int(nnz[0]) - B * D * pe) < 6.0 * np.sqrt(B * D * pe * (1.0 - pe))
+
+
+def test_weight_grad_sampled_entries(wide):
+    rad, st, A, dZ = wide["rad"], wide["st"], wide["A"], wide["dZ"]
+    dW = torch.full((D, H), float("nan"), dtype=torch.float32, device="cuda")
+    rad.rad_linear_weight_grad(st, wide["dev"]["dZ"], dW, dev_status=wide["status"])
+    torch.cuda.synchronize()
+    assert wide["status"].item() == 0
+    assert torch.isfinite(dW).all()
+    rng = np.random.default_rng(2)
+    ds = np.concatenate([[0, 127, 128, 255, 256, 511, 512, D - 1], rng.integers(0, D, 16)])
+    hs = np.concatenate([[0, 255, 256, H - 1], rng.integers(0, H, 12)])
+    scale = np.float32(orc.scale_factor(P))
+    m = orc.keep_mask_at("different", np.arange(B), ds, P, SEED, LAYER, STEP)          # B x len(ds)
+    a_hat = np.where(m, orc.round_bf16(A[:, ds] * scale), np.float32(0)).astype(np.float64)
+    ref = a_hat.T @ dZ[:, hs].astype(np.float64)
+    got = to_host_f32(dW[torch.from_numpy(ds).cuda()][:, torch.from_numpy(hs).cuda()])
+    fro, mx = rel_err(got, ref)
+    assert fro <= 2e-2 and mx <= 2e-2, (fro, mx)
+    # float32 accumulation of exact bf16 products: far inside the stated tolerance
+    bound = 1e-4 * (np.abs(a_hat).T @ np.abs(dZ[:, hs]).astype(np.float64))
+    assert (np.abs(got - ref) <= bound + 1e-30).all()
+
+
+def test_forward_and_input_grad_sampled_entries(wide):
+    rad, dev, A, W, bias, dZ = wide["rad"], wide["dev"], wide["A"], wide["W"], wide["bias"], wide["dZ"]
+    act = torch.empty(B, H, dtype=torch.bfloat16, device="cuda")
+    zlow = torch.empty(B, H, dtype=torch.bfloat16, device="cuda")
+    rad.rad_linear_forward(dev["A"], dev["W"], dev["bias"], "gelu", out_act=act, out_zlow=zlow, dev_status=wide["status"])
+    torch.cuda.synchronize()
+    assert wide["status"].item() == 0
+    rng = np.random.default_rng(3)
+    bs = np.concatenate([[0, 127, 128, 255, 256, B - 1], rng.integers(0, B, 18)])
+    hs = np.concatenate([[0, 127, 128, 255, 256, H - 1], rng.integers(0, H, 10)])
+    z = A[bs].astype(np.float64) @ W[:, hs].astype(np.float64) + bias[hs]
+    bi, hi = torch.from_numpy(bs).cuda(), torch.from_numpy(hs).cuda()
+    assert max(rel_err(to_host_f32(zlow[bi][:, hi]), z)) <= 8e-3
+    assert max(rel_err(to_host_f32(act[bi][:, hi]), orc.act_forward(z, "gelu"))) <= 8e-3
+    del act
+    # input gradient with the GELU derivative taken at the stored pre-activation
+    dA = torch.empty(B, D, dtype=torch.bfloat16, device="cuda")
+    db = torch.empty(H, dtype=torch.float32, device="cuda")
+    zprev = dev["A"]                                   # any B x D bf16 tensor serves as the pre-activation
+    rad.rad_linear_input_grad(dev["dZ"], dev["W"], z_prev=zprev, dZ_prev=dA, db=db, dev_status=wide["status"])
+    torch.cuda.synchronize()
+    assert wide["status"].item() == 0
+    ds = np.concatenate([[0, 127, 128, 255, 256, D - 1], rng.integers(0, D, 10)])
+    g = dZ[bs].astype(np.float64) @ W[ds].astype(np.float64).T                       # len(bs) x len(ds)
+    ref = orc.round_bf16((g * orc.gelu_grad(A[np.ix_(bs, ds)].astype(np.float64))).astype(np.float32)).astype(np.float64)
+    got = to_host_f32(dA[bi][:, torch.from_numpy(ds).cuda()])
+    assert max(rel_err(got, ref)) <= 2e-2
+    ref_db = dZ[:, hs].astype(np.float64).sum(axis=0)
+    assert max(rel_err(to_host_f32(db[hi]), ref_db)) <= 1e-5

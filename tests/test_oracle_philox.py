@@ -7,8 +7,10 @@ independent restatement in Python big integers, invertibility of each round
 every counter/key word, and lane uniformity.
 """
 import numpy as np
+import pytest
 
 from oracle import philox as ph
+from oracle import rad as orc
 
 M0, M1, W0, W1 = 0xD2511F53, 0xCD9E8D57, 0x9E3779B9, 0xBB67AE85
 MASK = (1 << 32) - 1
@@ -79,3 +81,15 @@ def test_lane_uniformity_chi_square():
     chi2 = ((hist - expected) ** 2 / expected).sum()
     # 255 degrees of freedom: mean 255, sd ~22.6; 6 sigma band
     assert abs(chi2 - 255.0) < 6 * 22.6
+
+
+@pytest.mark.parametrize("variant", ["different", "same"])
+def test_keep_mask_at_agrees_with_the_full_mask(variant):
+    """The block-wise form is the full mask restricted to the rows and columns asked for."""
+    B, D, p, seed, layer, step = 37, 203, 0.3, 0x1234567890, 5, 9
+    full = orc.keep_mask(variant, B, D, p, seed, layer, step)
+    rows = np.array([0, 3, 36, 17, 17])
+    cols = np.array([202, 0, 7, 8, 9, 100, 64])
+    got = orc.keep_mask_at(variant, rows, cols, p, seed, layer, step)
+    assert np.array_equal(got, full[np.ix_(rows, cols)])
+    assert np.array_equal(orc.keep_mask_at(variant, np.arange(B), np.arange(D), p, seed, layer, step), full)
