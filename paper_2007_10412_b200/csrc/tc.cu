@@ -125,12 +125,13 @@ struct Unit {
 
 struct Schedule {
   int64_t M, m_tiles, n_tiles, ntiles, units;
-  int32_t kblocks, splits, bm;
-  __device__ Schedule(int64_t M_, int64_t N_, int64_t K_, int32_t splits_, int32_t bm_ = BM) {
+  int32_t kblocks, splits, bm, bn;
+  __device__ Schedule(int64_t M_, int64_t N_, int64_t K_, int32_t splits_, int32_t bm_ = BM, int32_t bn_ = BN) {
     M = M_;
     bm = bm_;
+    bn = bn_;
     m_tiles = (M + bm - 1) / bm;
-    n_tiles = (N_ + BN - 1) / BN;
+    n_tiles = (N_ + bn - 1) / bn;
     ntiles = m_tiles * n_tiles;
     kblocks = (int32_t)((K_ + BK - 1) / BK);
     splits = splits_;
@@ -146,7 +147,7 @@ struct Schedule {
     const int64_t first_m = g * kRasterGroup;
     const int64_t gm = min((int64_t)kRasterGroup, m_tiles - first_m);
     w.m0 = (first_m + r % gm) * bm;
-    w.n0 = (r / gm) * BN;
+    w.n0 = (r / gm) * bn;
     w.split = (int32_t)s;
     w.kb0 = (int32_t)(s * kblocks / splits);
     w.kb1 = (int32_t)((s + 1) * kblocks / splits);
@@ -595,18 +596,23 @@ tc_gemm_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, c
 }
 
 // ---- two-CTA engine, sparse A (different-sample dW) --------------------------------------------------
-// The pair owns a 512 x 256 tile of dW: each CTA rebuilds its own 256 columns of A_hat (two store
-// tiles per K block, as in the one-CTA kernel) and loads half of the dZ tile, so the dZ bytes per
-// SM and the operand reads of each shared memory are halved.  Two MMAs per 16 rows of K, one per
-// 128-row half of each CTA's A tile; the four accumulators fill the pair's tensor memory.
+// The pair owns a 256 x 512 tile of dW.  Each CTA rebuilds 128 columns of A_hat (one store tile per
+// K block) in shared memory and loads its half of the dZ tile (two blocks of 128 columns); per 16
+// rows of K two MMAs (M256 N256), one per 256-column half of the tile; the two 128 x 256
+// accumulators of a CTA fill its tensor memory.  A store tile is expanded once per 512 output
+// columns: the wide tile halves the expansion work per flop against a 256-column tile and brings the
+// shared-memory traffic per K block and CTA from about 1540 to about 1200 wavefronts.
 // Roles per CTA: 0 dZ producer, 1 MMA issuer (even CTA) and tensor-memory owner, 2-5 epilogue,
-// 6 producer of the compressed ring, 7-22 expanders.  full[s] lives in the even CTA: one arrival
+// 6 producer of the compressed ring, 7-22 expanders (two groups on alternate K blocks).  full[s] lives in the even CTA: one arrival
 // with the dZ bytes of both CTAs plus one per expander warp of either CTA.
-constexpr int kSpAStageBytes = 256 * BK * 2;           // 32 KB: this CTA's 256 columns of A_hat
-constexpr int kSpBStageBytes = 128 * BK * 2;           // 16 KB: this CTA's 128 columns of dZ
+constexpr int kSpBM = 256, kSpBN = 512;
+constexpr int kSpAStageBytes = 128 * BK * 2;           // 16 KB: this CTA's 128 columns of A_hat
+constexpr int kSpBStageBytes = 256 * BK * 2;           // 32 KB: this CTA's 2 x 128 columns of dZ
 constexpr int kSpStageBytes = kSpAStageBytes + kSpBStageBytes;
 constexpr int kSpMaxStages = 4;
-constexpr int kSpThreads = 32 * (kFirstExpanderWarp + kExpanderWarps);
+constexpr int kSpExpanderWarps = 8;                    // per K block: one thread per keep-bit word of the store tile
+constexpr int kSpExpanderGroups = 2;                   // groups of eight warps take alternate K blocks
+constexpr int kSpThreads = 32 * (kFirstExpanderWarp + kSpExpanderGroups * kSpExpanderWarps);
 
 struct SmemCtlSp {
   uint64_t full[kSpMaxStages], empty[kSpMaxStages], comp_full[8], comp_empty[8], tmem_full, tmem_empty;
@@ -619,8 +625,7 @@ tc_sparse_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmB)
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int stages = p.num_stages;
-  const int comp_half = kIndexBytes + p.comp_cap;               // index data + values of one store tile
-  const int comp_slot = 2 * comp_half;                           // compressed data of one K block of this CTA
+  const int comp_slot = kIndexBytes + p.comp_cap;               // index data + values of this CTA's store tile of one K block
   uint8_t* comp_base = smem + (size_t)stages * kSpStageBytes;
   SmemCtlSp* ctl = reinterpret_cast<SmemCtlSp*>(comp_base + (size_t)p.comp_depth * comp_slot);
   volatile int* abort_flag = &ctl->abort_flag;
@@ -628,16 +633,16 @@ tc_sparse_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmB)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t rank = cluster_ctarank();
   const uint32_t peer_abort = map_to_cta(smem_u32(&ctl->abort_flag), rank ^ 1u);
-  const Schedule sched(p.M, p.N, p.K, p.splits, 512);
+  const Schedule sched(p.M, p.N, p.K, p.splits, kSpBM, kSpBN);
   const int64_t pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
   if (tid == 0) {
     for (int s = 0; s < stages; ++s) {
-      mbar_init(smem_u32(&ctl->full[s]), 1 + 2 * kExpanderWarps);
+      mbar_init(smem_u32(&ctl->full[s]), 1 + 2 * kSpExpanderWarps);
       mbar_init(smem_u32(&ctl->empty[s]), 1);
     }
     for (int c = 0; c < p.comp_depth; ++c) {
       mbar_init(smem_u32(&ctl->comp_full[c]), 1);
-      mbar_init(smem_u32(&ctl->comp_empty[c]), kExpanderWarps);
+      mbar_init(smem_u32(&ctl->comp_empty[c]), kSpExpanderWarps);
     }
     mbar_init(smem_u32(&ctl->tmem_full), 1);
     mbar_init(smem_u32(&ctl->tmem_empty), 8);          // four epilogue warps in each CTA
@@ -654,20 +659,17 @@ tc_sparse_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmB)
   tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
   const uint32_t smem_base = smem_u32(smem);
-  // store tiles (128 columns each) of this CTA's 256 columns that exist, per unit: 0, 1 or 2
-  auto own_halves = [&](const Unit& w) -> int {
-    const int64_t first = (w.m0 + 256 * (int64_t)rank) / kTileCols;
-    return (int)max((int64_t)0, min((int64_t)2, (int64_t)p.ncb - first));
-  };
+  // this CTA's store tile column (128 columns of the layer input) of a unit, and whether it exists
+  auto tile_col_of = [&](const Unit& w) -> int64_t { return (w.m0 + 128 * (int64_t)rank) / kTileCols; };
 
   if (warp == 0) {
-    // ===== dZ producer: this CTA's 128 columns of the dZ tile =====
+    // ===== dZ producer: this CTA's 128 columns of each 256-column half of the dZ tile =====
     int stage = 0;
     uint32_t phase = 0;
     bool ok = true;
     for (int64_t u = pair; u < sched.units && ok; u += npairs) {
       const Unit w = sched.unit(u);
-      const int n_own = (int)w.n0 + 128 * (int)rank;
+      const int n_own = (int)w.n0 + 128 * (int)rank;       // + 256 for the second half
       for (int kb = w.kb0; kb < w.kb1; ++kb) {
         if (lane == 0) {
           ok = mbar_wait2(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, peer_abort);
@@ -676,7 +678,8 @@ tc_sparse_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmB)
             if (rank == 0) mbar_arrive_expect_tx(smem_u32(&ctl->full[stage]), 2 * kSpBStageBytes);   // both CTAs' bytes
             const uint32_t full = map_to_cta(smem_u32(&ctl->full[stage]), 0u);
 #pragma unroll
-            for (int c = 0; c < 2; ++c) tma_load_2d_pair(sB + c * 8192, &tmB, n_own + c * 64, kb * BK, full);
+            for (int c = 0; c < 4; ++c)
+              tma_load_2d_pair(sB + c * 8192, &tmB, n_own + (c >> 1) * 256 + (c & 1) * 64, kb * BK, full);
           }
         }
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -712,10 +715,10 @@ tc_sparse_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmB)
               const uint32_t sB = sA + kSpAStageBytes;
 #pragma unroll
               for (int k = 0; k < BK / 16; ++k) {
-                const uint64_t bdesc = make_desc(sB + k * 2048, 8192, 1024);
+                const uint64_t adesc = make_desc(sA + k * 2048, 8192, 1024);
 #pragma unroll
-                for (int h = 0; h < 2; ++h)
-                  tc_mma_pair(tmem_base + h * 256, make_desc(sA + h * 16384 + k * 2048, 8192, 1024), bdesc, idesc,
+                for (int j = 0; j < 2; ++j)
+                  tc_mma_pair(tmem_base + j * 256, adesc, make_desc(sB + j * 16384 + k * 2048, 8192, 1024), idesc,
                               (kb > w.kb0 || k > 0) ? 1u : 0u);
               }
               tc_commit_pair(smem_u32(&ctl->empty[stage]));
@@ -730,7 +733,7 @@ tc_sparse_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmB)
       }
     }
   } else if (warp < 6) {
-    // ===== epilogue: thread = one accumulator row of each of this CTA's two halves =====
+    // ===== epilogue: thread = one accumulator row (512 columns) =====
     const int q = warp & 3;
     const uint32_t empty_bar = map_to_cta(smem_u32(&ctl->tmem_empty), 0u);
     uint32_t unit_phase = 0;
@@ -741,18 +744,16 @@ tc_sparse_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmB)
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) break;
       tc_fence_after();
-      for (int h = 0; h < 2; ++h) {
-        const int64_t m = w.m0 + 256 * (int64_t)rank + h * kHalfM + q * 32 + lane;
-        const bool row_ok = m < sched.M;
+      const int64_t m = w.m0 + 128 * (int64_t)rank + q * 32 + lane;
+      const bool row_ok = m < sched.M;
 #pragma unroll 1
-        for (int c0 = 0; c0 < BN; c0 += 32) {
-          const int64_t n = w.n0 + c0;
-          if (n >= p.N) break;                  // warp-uniform
-          uint32_t r[32];
-          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * 256 + c0), r);
-          tmem_ld_wait();
-          epilogue_chunk<kDw>(p, r, m, n, row_ok, w.split);
-        }
+      for (int c0 = 0; c0 < kSpBN; c0 += 32) {
+        const int64_t n = w.n0 + c0;
+        if (n >= p.N) break;                  // warp-uniform
+        uint32_t r[32];
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+        tmem_ld_wait();
+        epilogue_chunk<kDw>(p, r, m, n, row_ok, w.split);
       }
       tc_fence_before();
       __syncwarp();
@@ -761,49 +762,42 @@ tc_sparse_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmB)
     }
   } else if (warp == 6) {
     // ===== producer of the compressed ring: keep bits + row offsets (1152 B) and packed values of
-    // this CTA's store tiles of each K block.  It runs ahead of the A/B ring: a slot is free as soon
+    // this CTA's store tile of each K block.  It runs ahead of the A/B ring: a slot is free as soon
     // as the expanders have read it, long before the MMAs of that K block retire. =====
     int slot = 0;
     uint32_t cphase = 0;
     bool ok = true;
     for (int64_t u = pair; u < sched.units && ok; u += npairs) {
       const Unit w = sched.unit(u);
-      const int halves = own_halves(w);
-      const int64_t tile_col = (w.m0 + 256 * (int64_t)rank) / kTileCols;
-      uint32_t off_lo = 0, off_mid = 0, off_hi = 0;   // tile offsets of K block (base + lane)
+      const int64_t tile_col = tile_col_of(w);
+      const bool have = tile_col < p.ncb;
+      uint32_t off_lo = 0, off_hi = 0;                // tile offsets of K block (base + lane)
       for (int kb = w.kb0; kb < w.kb1; ++kb) {
-        if (((kb - w.kb0) & 31) == 0 && halves > 0) {
+        if (((kb - w.kb0) & 31) == 0 && have) {
           const int kbl = kb + lane;
           if (kbl < w.kb1) {
             const int64_t t0 = (int64_t)kbl * p.ncb + tile_col;
             off_lo = __ldg(p.offsets + t0);
-            off_mid = __ldg(p.offsets + t0 + 1);
-            off_hi = (halves == 2) ? __ldg(p.offsets + t0 + 2) : off_mid;
+            off_hi = __ldg(p.offsets + t0 + 1);
           }
         }
         const int src = (kb - w.kb0) & 31;
         const uint32_t o0 = __shfl_sync(0xffffffffu, off_lo, src);
-        const uint32_t o1 = __shfl_sync(0xffffffffu, off_mid, src);
-        const uint32_t o2 = __shfl_sync(0xffffffffu, off_hi, src);
+        const uint32_t o1 = __shfl_sync(0xffffffffu, off_hi, src);
         if (lane == 0) {
           ok = mbar_wait2(smem_u32(&ctl->comp_empty[slot]), cphase ^ 1u, abort_flag, peer_abort);
           if (ok) {
             const uint32_t cfull = smem_u32(&ctl->comp_full[slot]);
             const uint32_t sC = smem_u32(comp_base) + slot * comp_slot;
-            const int64_t t0 = (int64_t)kb * p.ncb + tile_col;
-            uint32_t vb0 = halves > 0 ? (o1 - o0) * 2u : 0u, vb1 = halves > 1 ? (o2 - o1) * 2u : 0u;
-            bool bad = false;
-            if (vb0 > (uint32_t)p.comp_cap || (int64_t)o1 > p.values_capacity) { vb0 = 0; bad = true; }
-            if (vb1 > (uint32_t)p.comp_cap || (int64_t)o2 > p.values_capacity) { vb1 = 0; bad = true; }
-            if (bad) raise_status(p.dev_status, RAD_DEV_ECAPACITY);
-            mbar_arrive_expect_tx(cfull, (uint32_t)kIndexBytes * halves + vb0 + vb1);
-            if (halves > 0) {
-              bulk_load(sC, p.keepbits + t0 * kTileWords, kIndexBytes, cfull);
-              if (vb0 != 0) bulk_load(sC + kIndexBytes, p.values + o0, vb0, cfull);
+            uint32_t vb = have ? (o1 - o0) * 2u : 0u;
+            if (vb > (uint32_t)p.comp_cap || (int64_t)o1 > p.values_capacity) {
+              vb = 0;
+              raise_status(p.dev_status, RAD_DEV_ECAPACITY);
             }
-            if (halves > 1) {
-              bulk_load(sC + comp_half, p.keepbits + (t0 + 1) * kTileWords, kIndexBytes, cfull);
-              if (vb1 != 0) bulk_load(sC + comp_half + kIndexBytes, p.values + o1, vb1, cfull);
+            mbar_arrive_expect_tx(cfull, (have ? (uint32_t)kIndexBytes : 0u) + vb);
+            if (have) {
+              bulk_load(sC, p.keepbits + ((int64_t)kb * p.ncb + tile_col) * kTileWords, kIndexBytes, cfull);
+              if (vb != 0) bulk_load(sC + kIndexBytes, p.values + o0, vb, cfull);
             }
           }
         }
@@ -813,37 +807,42 @@ tc_sparse_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmB)
       }
     }
   } else {
-    // ===== expanders: rebuild this CTA's A_hat tile (64 K rows x 256 columns, M-major, swizzled) =====
-    // One thread per keep-bit word: half h = columns 128h..128h+127 of the tile (one store tile),
-    // row r of the slab, columns 32*wq..32*wq+31 of that half.  The row's first value is given by
-    // the stored row offset; the words before this one in the row are counted with popc.
-    // Eight consecutive lanes take eight consecutive rows of the same word column: with the
-    // 128-byte swizzle their 16-byte zero stores then fall on eight different bank groups.
+    // ===== expanders: rebuild this CTA's A_hat tile (64 K rows x 128 columns, M-major, swizzled) =====
+    // One thread per keep-bit word: row r of the slab, columns 32*wq..32*wq+31 of the store tile.
+    // The row's first value is given by the stored row offset; the words before this one in the row
+    // are counted with popc.  Eight consecutive lanes take eight consecutive rows of the same word
+    // column: with the 128-byte swizzle their 16-byte zero stores then fall on eight different bank
+    // groups.
+    // Two groups of eight warps take alternate K blocks, so the waits, loads and fence of one K
+    // block overlap the stores of the next.
     const int et = tid - 32 * kFirstExpanderWarp;            // 0..511
-    const int h = et >> 8, wi = et & 255;
+    const uint32_t group = (uint32_t)(et >> 8);
+    const int wi = et & 255;
     const int r = (wi & 7) + ((wi >> 5) << 3), wq = (wi >> 3) & 3;
     int stage = 0, slot = 0;
-    uint32_t phase = 0, cphase = 0;
+    uint32_t phase = 0, cphase = 0, turn = 0;
     bool ok = true;
     for (int64_t u = pair; u < sched.units && ok; u += npairs) {
       const Unit w = sched.unit(u);
-      const int halves = own_halves(w);
-      for (int kb = w.kb0; kb < w.kb1; ++kb) {
-        ok = mbar_wait2(smem_u32(&ctl->comp_full[slot]), cphase, abort_flag, peer_abort) &&
-             mbar_wait2(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, peer_abort);     // A tile of this stage is free
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        // columns past the layer's width keep whatever the buffer held: their accumulator rows are never written
-        if (h < halves) {
-          uint8_t* sA = smem + (size_t)stage * kSpStageBytes;
-          const uint8_t* sC = comp_base + (size_t)slot * comp_slot + (size_t)h * comp_half;
-          expand_word(sA, sC, h, r, wq, (uint32_t)p.comp_cap >> 1);
-          fence_proxy_async();
-        }
-        __syncwarp();
-        if (lane == 0) {
-          mbar_arrive_remote(map_to_cta(smem_u32(&ctl->full[stage]), 0u));
-          mbar_arrive(smem_u32(&ctl->comp_empty[slot]));
+      const bool have = tile_col_of(w) < p.ncb;
+      for (int kb = w.kb0; kb < w.kb1; ++kb, turn ^= 1u) {
+        if (turn == group) {
+          ok = mbar_wait2(smem_u32(&ctl->comp_full[slot]), cphase, abort_flag, peer_abort) &&
+               mbar_wait2(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, peer_abort);     // A tile of this stage is free
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          // columns past the layer's width keep whatever the buffer held: their accumulator rows are never written
+          if (have) {
+            uint8_t* sA = smem + (size_t)stage * kSpStageBytes;
+            const uint8_t* sC = comp_base + (size_t)slot * comp_slot;
+            expand_word(sA, sC, 0, r, wq, (uint32_t)p.comp_cap >> 1);
+            fence_proxy_async();
+          }
+          __syncwarp();
+          if (lane == 0) {
+            mbar_arrive_remote(map_to_cta(smem_u32(&ctl->full[stage]), 0u));
+            mbar_arrive(smem_u32(&ctl->comp_empty[slot]));
+          }
         }
         if (++stage == stages) { stage = 0; phase ^= 1u; }
         if (++slot == p.comp_depth) { slot = 0; cphase ^= 1u; }
@@ -931,9 +930,10 @@ int num_sms() {
 // (about 1024 tensor-pipe clocks): waves x K blocks per unit, plus what writing and re-reading the
 // float32 partial tiles costs at HBM speed.  Pure function of the shapes, so the workspace query
 // and the launch agree.
-int choose_splits(int64_t m_tiles, int64_t n_tiles, int64_t kblocks, int64_t bm = BM, int64_t sms = kNumSMsDefault) {
+int choose_splits(int64_t m_tiles, int64_t n_tiles, int64_t kblocks, int64_t bm = BM, int64_t sms = kNumSMsDefault,
+                  int64_t bn = BN) {
   const double kblock_us = 0.55;                                            // 1024 clk at ~1.9 GHz
-  const double partial_us = (double)(m_tiles * bm) * (double)(n_tiles * BN) * 8.0 / 6.5e6;   // per split
+  const double partial_us = (double)(m_tiles * bm) * (double)(n_tiles * bn) * 8.0 / 6.5e6;   // per split
   int best = 1;
   double best_cost = 1e300;
   for (int s = 1; s <= kMaxSplits && s <= kblocks; ++s) {
@@ -967,10 +967,10 @@ DwPlan plan_dw(const rad_store* st, int64_t H) {
     d.comp_cap = (int)round_up(cap, 128);
     // shared memory: 48 KB per A/B stage plus a ring of compressed slots
     const int64_t budget = 227 * 1024 - 2048 - (int64_t)sizeof(SmemCtlSp);
-    const int64_t slot = 2 * (kIndexBytes + d.comp_cap);
+    const int64_t slot = kIndexBytes + d.comp_cap;
     d.stages = (4 * kSpStageBytes + 3 * slot <= budget) ? 4 : (3 * kSpStageBytes + 2 * slot <= budget) ? 3 : 2;
-    d.comp_depth = (int)std::max<int64_t>(2, std::min<int64_t>(6, (budget - d.stages * kSpStageBytes) / slot));
-    d.splits = choose_splits(ceil_div(m_expect, 512), ceil_div(H, BN), kblocks, 512, kNumSMsDefault / 2);
+    d.comp_depth = (int)std::max<int64_t>(2, std::min<int64_t>(8, (budget - d.stages * kSpStageBytes) / slot));
+    d.splits = choose_splits(ceil_div(m_expect, kSpBM), ceil_div(H, kSpBN), kblocks, kSpBM, kNumSMsDefault / 2, kSpBN);
     d.bytes = d.splits > 1 ? (int64_t)d.splits * d.partial_rows * H * 4 : 0;
     return d;
   }
@@ -1032,7 +1032,7 @@ int resident_pairs_of(K kernel, int threads, size_t smem) {
 }
 
 int launch_sparse_pair(const TcParams& p, const CUtensorMap& tb, int64_t max_units, cudaStream_t s) {
-  const size_t smem = (size_t)p.num_stages * kSpStageBytes + (size_t)p.comp_depth * 2 * (kIndexBytes + p.comp_cap) +
+  const size_t smem = (size_t)p.num_stages * kSpStageBytes + (size_t)p.comp_depth * (kIndexBytes + p.comp_cap) +
                       sizeof(SmemCtlSp) + 1024;
   if (smem > 227 * 1024 || p.num_stages > kSpMaxStages || p.comp_depth > 8) return RAD_EUNSUPPORTED;
   static int resident_pairs = 0;
@@ -1123,7 +1123,7 @@ int tc_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H, 
     p.M = st->D;
     p.values = static_cast<const bf16*>(st->values); p.keepbits = st->keepbits; p.offsets = st->offsets;
     p.values_capacity = st->values_capacity; p.ncb = (int32_t)ceil_div(st->D, kTileCols); p.comp_cap = d.comp_cap;
-    rc = launch_sparse_pair(p, tb, ceil_div(st->D, 512) * ceil_div(H, BN) * d.splits, s);
+    rc = launch_sparse_pair(p, tb, ceil_div(st->D, kSpBM) * ceil_div(H, kSpBN) * d.splits, s);
   }
   if (rc != RAD_OK) return rc;
   if (d.splits > 1) {
