@@ -19,10 +19,13 @@ R = diag(sqrt(m / p_eff)) restricted to kept columns.  "different sample"
 draws m per minibatch row, "same sample" draws one m per layer and step
 (Sec. 4.3).
 
-The keep decision for (row b, column d) compares a 16-bit lane of a
-Philox-4x32-10 output with a threshold T = round(p * 2^16) clipped to
-[1, 2^16]; p_eff = T / 2^16 and stored values are scaled by fl32(2^16 / T) so
-the estimator is exactly unbiased for the probability actually sampled.
+The keep decision for (row b, column d) compares one byte of a
+Philox-4x32-10 output with a threshold T = round(p * 2^8) clipped to
+[1, 2^8]; p_eff = T / 2^8 and stored values are scaled by fl32(2^8 / T) so
+the estimator is exactly unbiased for the probability actually sampled.  The
+paper leaves the source of randomness open; one byte per decision lets one
+128-bit generator output decide sixteen entries, and the keep probabilities
+the paper uses (0.05 ... 0.5) move by less than 2 % of their value.
 """
 from dataclasses import dataclass, field
 from typing import List, Optional
@@ -34,37 +37,39 @@ from .philox import philox4x32_10
 
 STREAM_DIFFERENT = 0     # counter stream of per-row masks
 STREAM_SAME = 1          # counter stream of masks shared by the minibatch
-LANE_BITS = 16
-LANES_PER_CALL = 8       # 128 output bits / 16
+LANE_BITS = 8
+LANES_PER_CALL = 16      # 128 output bits / 8
+LANE_RANGE = 1 << LANE_BITS
 
 
 # --------------------------------------------------------------------------
 # mask (Sec. 3.2: E[P] = I; Sec. 4.3: "same sample" / "different sample")
 # --------------------------------------------------------------------------
 def keep_threshold(p) -> int:
-    """T such that a 16-bit lane u is kept iff u < T."""
+    """T such that a byte lane u is kept iff u < T."""
     p32 = float(np.float32(p))
     if not (0.0 < p32 <= 1.0):
         raise ValueError("p must be in (0, 1]")
-    return int(min(max(np.rint(p32 * 65536.0), 1.0), 65536.0))
+    return int(min(max(np.rint(p32 * LANE_RANGE), 1.0), float(LANE_RANGE)))
 
 
 def effective_p(p) -> float:
-    return keep_threshold(p) / 65536.0
+    return keep_threshold(p) / LANE_RANGE
 
 
 def scale_factor(p) -> np.float32:
     """s = fl32(1 / p_eff), one correctly rounded float32 division."""
-    return np.float32(65536.0) / np.float32(keep_threshold(p))
+    return np.float32(LANE_RANGE) / np.float32(keep_threshold(p))
 
 
 def keep_mask(variant: str, B: int, D: int, p, seed: int, layer: int, step: int) -> np.ndarray:
     """Boolean B x D keep mask.
 
-    Counter = (d // 8, row, layer | stream << 24, step), key = (seed low word,
-    seed high word).  Output word j holds the lanes of columns 8*(d//8) + 2j
-    (low half) and 8*(d//8) + 2j + 1 (high half).  For "same" the row field is
-    0 and the single row of decisions is shared by every minibatch element.
+    Counter = (d // 16, row, layer | stream << 24, step), key = (seed low word,
+    seed high word).  The sixteen bytes of the output, words in order and
+    least significant byte first, are the lanes of columns 16*(d//16) + 0..15:
+    column d reads byte d % 4 of word (d % 16) // 4.  For "same" the row field
+    is 0 and the single row of decisions is shared by every minibatch element.
     """
     T = keep_threshold(p)
     groups = (D + LANES_PER_CALL - 1) // LANES_PER_CALL
@@ -80,8 +85,8 @@ def keep_mask(variant: str, B: int, D: int, p, seed: int, layer: int, step: int)
                           np.uint64(seed & 0xFFFFFFFF), np.uint64((seed >> 32) & 0xFFFFFFFF))
     lanes = np.empty(words[0].shape + (LANES_PER_CALL,), dtype=np.uint32)
     for j, w in enumerate(words):
-        lanes[..., 2 * j] = w & np.uint32(0xFFFF)
-        lanes[..., 2 * j + 1] = w >> np.uint32(16)
+        for k in range(4):
+            lanes[..., 4 * j + k] = (w >> np.uint32(8 * k)) & np.uint32(0xFF)
     m = (lanes < T).reshape(lanes.shape[0], groups * LANES_PER_CALL)[:, :D]
     if variant == "same":
         m = np.broadcast_to(m, (B, D))
@@ -109,8 +114,8 @@ def keep_mask_at(variant: str, rows, cols, p, seed: int, layer: int, step: int) 
     out = np.zeros(lane.shape, dtype=bool)
     for j, w in enumerate(words):
         w = np.broadcast_to(w, lane.shape)
-        out |= (lane == 2 * j) & ((w & np.uint32(0xFFFF)) < T)
-        out |= (lane == 2 * j + 1) & ((w >> np.uint32(16)) < T)
+        for k in range(4):
+            out |= (lane == 4 * j + k) & (((w >> np.uint32(8 * k)) & np.uint32(0xFF)) < T)
     return out
 
 

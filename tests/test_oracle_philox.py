@@ -75,8 +75,8 @@ def test_every_input_word_matters():
 def test_lane_uniformity_chi_square():
     n = 1 << 16
     words = ph.philox4x32_10(np.arange(n, dtype=np.uint64), 9, 2, 0, 42, 0)
-    lanes = np.concatenate([w & np.uint32(0xFFFF) for w in words] + [w >> np.uint32(16) for w in words])
-    hist = np.bincount(lanes >> 8, minlength=256).astype(np.float64)
+    lanes = np.concatenate([(w >> np.uint32(8 * k)) & np.uint32(0xFF) for w in words for k in range(4)])
+    hist = np.bincount(lanes, minlength=256).astype(np.float64)
     expected = lanes.size / 256.0
     chi2 = ((hist - expected) ** 2 / expected).sum()
     # 255 degrees of freedom: mean 255, sd ~22.6; 6 sigma band
@@ -93,3 +93,21 @@ def test_keep_mask_at_agrees_with_the_full_mask(variant):
     got = orc.keep_mask_at(variant, rows, cols, p, seed, layer, step)
     assert np.array_equal(got, full[np.ix_(rows, cols)])
     assert np.array_equal(orc.keep_mask_at(variant, np.arange(B), np.arange(D), p, seed, layer, step), full)
+
+
+@pytest.mark.parametrize("variant", ["different", "same"])
+def test_lane_of_a_column_is_its_byte_of_the_128_bit_output(variant):
+    """Column d is decided by byte d % 16 of the generator output for counter d // 16, the output read
+    as sixteen bytes, words in order and least significant byte first; restated here with Python
+    integers, independent of the array code in the oracle."""
+    B, D, p, seed, layer, step = 5, 77, 0.3, 0xABCDEF0123456789, 6, 11
+    T = orc.keep_threshold(p)
+    assert T == 77          # rint(0.3 * 256)
+    full = orc.keep_mask(variant, B, D, p, seed, layer, step)
+    stream = 0 if variant == "different" else 1
+    for b in range(B):
+        for d in range(D):
+            out = bigint_philox([d // 16, b if variant == "different" else 0, layer | stream << 24, step],
+                                [seed & MASK, seed >> 32])
+            octets = b"".join(int(w).to_bytes(4, "little") for w in out)
+            assert bool(full[b, d]) == (octets[d % 16] < T)
