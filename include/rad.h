@@ -60,18 +60,19 @@ typedef enum { RAD_ACT_NONE = 0, RAD_ACT_RELU = 1, RAD_ACT_GELU = 2 } rad_act;
 
 /*
  * The mask (Sec. 3.2: a random P with E[P] = I; Sec. 4.3: "same sample" /
- * "different sample").  Entry (b, d) is kept iff a 16-bit lane of
- * Philox-4x32-10 is below T = clamp(rint(p * 65536), 1, 65536):
+ * "different sample").  Entry (b, d) is kept iff one byte of a
+ * Philox-4x32-10 output is below T = clamp(rint(p * 256), 1, 256):
  *   key     = (seed & 0xffffffff, seed >> 32)
- *   counter = (d / 8, row, layer | stream << 24, step), row = b and stream = 0
+ *   counter = (d / 16, row, layer | stream << 24, step), row = b and stream = 0
  *             for different-sample; row = 0 and stream = 1 for same-sample
- *   lane of column d = 16-bit half (d & 1) of output word (d % 8) / 2.
- * p_eff = T / 65536 is the probability actually sampled and kept values are
- * multiplied by fl32(65536 / T) = 1 / p_eff, so E[A_hat] = A exactly.
+ *   byte of column d = byte d % 4 (least significant first) of output word
+ *             (d % 16) / 4: one 128-bit output decides sixteen columns.
+ * p_eff = T / 256 is the probability actually sampled and kept values are
+ * multiplied by fl32(256 / T) = 1 / p_eff, so E[A_hat] = A exactly.
  */
 uint32_t rad_keep_threshold(float p);   /* T; 0 if p is outside (0, 1]                        */
-float    rad_effective_p(float p);      /* T / 65536                                          */
-float    rad_scale(float p);            /* fl32(65536 / T)                                    */
+float    rad_effective_p(float p);      /* T / 256                                            */
+float    rad_scale(float p);            /* fl32(256 / T)                                      */
 
 /*
  * One layer's compact store: plain data, all buffers device memory of the caller.

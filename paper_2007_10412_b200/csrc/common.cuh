@@ -65,19 +65,39 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
   out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
-// Keep bits of the 8 columns of one counter: bit i set iff the 16-bit lane of column i is < T.
-__device__ __forceinline__ uint32_t philox_keep8(uint32_t group, uint32_t row, uint32_t c2, uint32_t c3,
-                                                 const PhiloxKeys& ks, uint32_t T) {
+// One keep decision per output byte: a 128-bit output decides sixteen consecutive columns, column i
+// of the sixteen reading byte i % 4 of word i / 4; it is kept iff the byte is below T (1..256).
+constexpr uint32_t kLaneRange = 256;
+
+struct KeepThreshold {
+  uint32_t y;    // T - 1 in every byte
+  uint32_t y1;   // y with the top bit of every byte set
+};
+inline KeepThreshold make_keep_threshold(uint32_t T) {
+  KeepThreshold k;
+  k.y = ((T - 1u) & 0xffu) * 0x01010101u;
+  k.y1 = k.y | 0x80808080u;
+  return k;
+}
+
+// Top bit of every byte of the result: byte of x <= byte of y.  The low seven bits are compared by a
+// subtraction that cannot borrow across bytes (the minuend's top bits are set, the subtrahend's
+// cleared); the top bits decide where they differ.
+__device__ __forceinline__ uint32_t bytes_le(uint32_t x, const KeepThreshold& k) {
+  const uint32_t d = k.y1 - (x & 0x7f7f7f7fu);
+  return ((~x & k.y) | (~(x ^ k.y) & d)) & 0x80808080u;
+}
+
+// Keep bits of the 16 columns of one counter, bit i = column i.  The multiplication moves the four
+// flag bits of a word (bits 7, 15, 23, 31) to bits 28..31 (all partial products land on distinct
+// bits, so nothing carries); the funnel shift appends that nibble.
+__device__ __forceinline__ uint32_t philox_keep16(uint32_t group, uint32_t row, uint32_t c2, uint32_t c3,
+                                                  const PhiloxKeys& ks, const KeepThreshold& k) {
   uint32_t w[4];
   philox4x32_10(group, row, c2, c3, ks, w);
-  // lane - T is negative exactly when lane < T (both below 2^17); a funnel shift moves each sign
-  // bit into the mask, last column first
   uint32_t m = 0;
 #pragma unroll
-  for (int j = 3; j >= 0; --j) {
-    m = __funnelshift_l((w[j] >> 16) - T, m, 1);
-    m = __funnelshift_l((w[j] & 0xffffu) - T, m, 1);
-  }
+  for (int j = 3; j >= 0; --j) m = __funnelshift_l(bytes_le(w[j], k) * 0x00204081u, m, 4);
   return m;
 }
 
@@ -120,6 +140,7 @@ inline int64_t round_up(int64_t a, int64_t b) { return ceil_div(a, b) * b; }
 // internal launchers shared across translation units --------------------------------------------
 int check_device();   // RAD_OK on an sm_100 device
 void count_launch(int n = 1);   // host-side tally of kernels this library has launched
+void* tensor_map_encoder();     // cuTensorMapEncodeTiled, or nullptr (tc.cu)
 
 // f32/bf16 CUDA-core kernels (small or unaligned problems)
 int simt_forward(int dtype, int act, int64_t B, int64_t D, int64_t H, const void* A, int64_t lda,

@@ -24,7 +24,7 @@ struct RnnParams {
   int64_t B, T;
   int32_t Hd, w32, ngroups;
   int32_t same;                      // same-sample: the mask does not depend on the row
-  uint32_t T16;                      // keep threshold
+  KeepThreshold keepT;               // keep threshold
   float scale;
   uint32_t c2, step0;
   const float* x;                    // B x T
@@ -68,9 +68,9 @@ __global__ void __launch_bounds__(kRnnThreads) irnn_forward_kernel(const RnnPara
     if (warp == 4) {
       // store of h_{t-1}: keep bits of the step, kept entries scaled and appended to the row's values
       uint32_t m = 0;
-      if (lane < p.ngroups) {
-        const int nvalid = min(8, Hd - lane * 8);
-        m = philox_keep8((uint32_t)lane, mask_row, p.c2, p.step0 + (uint32_t)t, ks, p.T16) & ((1u << nvalid) - 1u);
+      if (lane * 16 < Hd) {                          // one draw decides sixteen units
+        const int nvalid = min(16, Hd - lane * 16);
+        m = philox_keep16((uint32_t)lane, mask_row, p.c2, p.step0 + (uint32_t)t, ks, p.keepT) & (0xffffu >> (16 - nvalid));
       }
       const uint32_t c = __popc(m);
       uint32_t incl = c;
@@ -83,16 +83,15 @@ __global__ void __launch_bounds__(kRnnThreads) irnn_forward_kernel(const RnnPara
       uint32_t pos = off + incl - c;
       if ((int64_t)off + total <= p.cap_row) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i)
-          if ((m >> i) & 1u) p.values[b * p.cap_row + pos++] = hc[lane * 8 + i] * p.scale;
+        for (int i = 0; i < 16; ++i)
+          if ((m >> i) & 1u) p.values[b * p.cap_row + pos++] = hc[lane * 16 + i] * p.scale;
       } else if (lane == 0) {
         raise_status(p.dev_status, RAD_DEV_ECAPACITY);
       }
-      uint32_t kw = m << (8 * (lane & 3));
+      uint32_t kw = m << (16 * (lane & 1));
       kw |= __shfl_xor_sync(0xffffffffu, kw, 1);
-      kw |= __shfl_xor_sync(0xffffffffu, kw, 2);
       const int64_t sb = (t - 1) * p.B + b;
-      if ((lane & 3) == 0 && (lane >> 2) < p.w32) p.keepbits[sb * p.w32 + (lane >> 2)] = kw;
+      if ((lane & 1) == 0 && (lane >> 1) < p.w32) p.keepbits[sb * p.w32 + (lane >> 1)] = kw;
       if (lane == 0) p.offsets[sb] = off;
       off += total;
     } else {
@@ -266,9 +265,9 @@ struct RnnPlan {
 int make_rnn_plan(const rad_irnn_desc* d, RnnPlan* pl) {
   if (d == nullptr || d->B <= 0 || d->T <= 0 || d->Hd <= 0 || d->Hd > kHdMax || d->C <= 0) return RAD_EINVAL;
   if (d->variant != RAD_DIFFERENT_SAMPLE && d->variant != RAD_SAME_SAMPLE) return RAD_EINVAL;
-  const uint32_t T16 = keep_threshold_host(d->p);
-  if (T16 == 0) return RAD_EINVAL;
-  const double pe = T16 / 65536.0, n = (double)d->T * d->Hd;
+  const uint32_t Tk = keep_threshold_host(d->p);
+  if (Tk == 0) return RAD_EINVAL;
+  const double pe = Tk / (double)kLaneRange, n = (double)d->T * d->Hd;
   int64_t cap = (int64_t)(n * pe + 8.0 * std::sqrt(n * pe * (1.0 - pe)) + 16.0);
   cap = std::min<int64_t>(round_up(cap, 4), round_up((int64_t)n, 4));
   pl->cap_row = cap;
@@ -341,11 +340,11 @@ extern "C" int rad_irnn_step(const rad_irnn_desc* d, const float* x, const int32
   if (rc != RAD_OK) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   char* ws = static_cast<char*>(workspace);
-  const uint32_t T16 = keep_threshold_host(d->p);
+  const uint32_t Tk = keep_threshold_host(d->p);
   RnnParams p = {};
   p.B = d->B; p.T = d->T; p.Hd = (int32_t)d->Hd; p.w32 = (int32_t)ceil_div(d->Hd, 32); p.ngroups = (int32_t)ceil_div(d->Hd, 8);
   p.same = d->variant == RAD_SAME_SAMPLE ? 1 : 0;
-  p.T16 = T16; p.scale = 65536.0f / (float)T16;
+  p.keepT = make_keep_threshold(Tk); p.scale = (float)kLaneRange / (float)Tk;
   p.c2 = counter_word2(0, d->variant); p.step0 = d->step0;
   p.x = x; p.W_ih = W_ih; p.b_ih = b_ih; p.W_hh = W_hh; p.b_hh = b_hh;
   p.h_last = reinterpret_cast<float*>(ws + pl.h_last);

@@ -13,64 +13,19 @@
 #include <cmath>
 
 #include "common.cuh"
+#include "store.cuh"
 
 namespace rad {
 
 uint32_t keep_threshold_host(float p) {
   if (!(p > 0.0f) || !(p <= 1.0f)) return 0;
-  double t = rint((double)p * 65536.0);
+  double t = rint((double)p * (double)kLaneRange);
   if (t < 1.0) t = 1.0;
-  if (t > 65536.0) t = 65536.0;
+  if (t > (double)kLaneRange) t = (double)kLaneRange;
   return (uint32_t)t;
 }
 
 namespace {
-
-// ---- look-back status word ---------------------------------------------------------------------
-// bits 63..62 flag, 61..32 padded prefix in granules of 8 elements, 31..0 exact kept count.
-constexpr uint64_t kFlagShift = 62;
-constexpr uint64_t kFlagAggregate = 1, kFlagPrefix = 2, kFlagPoison = 3;
-constexpr uint64_t kValueMask = (1ull << kFlagShift) - 1;
-constexpr int kSpinLimit = 1 << 20;   // bounded wait: about a second with the back-off below
-
-__device__ __forceinline__ uint64_t pack_counts(uint32_t granules, uint32_t exact) {
-  return ((uint64_t)granules << 32) | exact;
-}
-__device__ __forceinline__ uint64_t load_status(const uint64_t* p) {
-  uint64_t v;
-  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ void store_status(uint64_t* p, uint64_t v) {
-  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
-}
-__device__ __forceinline__ uint64_t warp_sum_u64(uint64_t v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
-}
-
-struct StoreParams {
-  const void* A;
-  int64_t lda;
-  int64_t B, D;
-  int32_t ncb;        // column blocks
-  int32_t ntiles;
-  uint32_t T;         // keep threshold
-  float scale;
-  uint32_t c2, c3;    // counter words 2 and 3
-  void* values;
-  int64_t capacity;
-  uint32_t* keepbits;
-  uint32_t* offsets;
-  int64_t* nnz;
-  uint32_t* relubits;
-  int32_t w32;        // relu-bit words per row
-  uint64_t* status;   // ntiles look-back words (zeroed before launch)
-  uint32_t* ticket;   // zeroed before launch
-  int32_t* dev_status;
-  int32_t vec_ok;     // rows are 16-byte aligned: 8-element vector loads allowed
-};
 
 template <typename T> struct Raw8;   // eight consecutive elements of one row
 template <> struct Raw8<float> { float v[8]; };
@@ -159,7 +114,9 @@ __global__ void __launch_bounds__(256) store_different_kernel(const StoreParams 
     const int64_t row = slab * kTileRows + warp * 8 + it * 2 + half;
     if (row < p.B && nvalid > 0) {
       load8<T>(Abase + row * p.lda, col0, nvalid, p.vec_ok != 0, raw[it]);
-      const uint32_t m = philox_keep8((uint32_t)(col0 >> 3), (uint32_t)row, p.c2, p.c3, ks, p.T) & ((1u << nvalid) - 1u);
+      // this lane's eight columns are one half of a sixteen-column draw
+      const uint32_t m16 = philox_keep16((uint32_t)(col0 >> 4), (uint32_t)row, p.c2, p.c3, ks, p.T);
+      const uint32_t m = (m16 >> (8 * (cg & 1))) & ((1u << nvalid) - 1u);
       masks |= m << (8 * it);
       counts |= __popc(m) << (8 * it);
       if (p.relubits != nullptr) relus |= (positive8(raw[it]) & ((1u << nvalid) - 1u)) << (8 * it);
@@ -304,7 +261,7 @@ struct SameParams {
   const void* A;
   int64_t lda;
   int64_t B, D;
-  uint32_t T;
+  KeepThreshold T;
   float scale;
   uint32_t c2, c3;
   void* values;
@@ -322,18 +279,17 @@ __global__ void __launch_bounds__(1024) same_mask_kernel(const SameParams p, con
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) s_running = 0;
   __syncthreads();
-  const int64_t groups = (p.D + 7) / 8;
+  const int64_t groups = (p.D + 15) / 16;
   for (int64_t g0 = 0; g0 < groups; g0 += 1024) {
     const int64_t g = g0 + tid;
     uint32_t m = 0;
     if (g < groups) {
-      const int nvalid = (int)min((int64_t)8, p.D - g * 8);
-      m = philox_keep8((uint32_t)g, 0u, p.c2, p.c3, ks, p.T) & ((1u << nvalid) - 1u);
+      const int nvalid = (int)min((int64_t)16, p.D - g * 16);
+      m = philox_keep16((uint32_t)g, 0u, p.c2, p.c3, ks, p.T) & (0xffffu >> (16 - nvalid));
     }
-    uint32_t kw = m << (8 * (lane & 3));
+    uint32_t kw = m << (16 * (lane & 1));
     kw |= __shfl_xor_sync(0xffffffffu, kw, 1);
-    kw |= __shfl_xor_sync(0xffffffffu, kw, 2);
-    if ((lane & 3) == 0 && g < groups) p.keepbits[g >> 2] = kw;
+    if ((lane & 1) == 0 && g < groups) p.keepbits[g >> 1] = kw;
     const uint32_t c = __popc(m);
     uint32_t incl = c;
 #pragma unroll
@@ -355,8 +311,8 @@ __global__ void __launch_bounds__(1024) same_mask_kernel(const SameParams p, con
     }
     __syncthreads();
     uint32_t pos = s_running + s_warp[warp] + incl - c;
-    for (int i = 0; i < 8; ++i)
-      if ((m >> i) & 1u) p.idx[pos++] = (uint32_t)(g * 8 + i);
+    for (int i = 0; i < 16; ++i)
+      if ((m >> i) & 1u) p.idx[pos++] = (uint32_t)(g * 16 + i);
     __syncthreads();
     if (tid == 1023) s_running = pos;   // last thread's end position is the running total
     __syncthreads();
@@ -409,6 +365,20 @@ __global__ void __launch_bounds__(256) relu_bits_kernel(const T* A, int64_t lda,
   }
 }
 
+// The persistent TMA-fed kernel where the input can be described by a tensor map, else the generic one
+// (same layout, same scratch: a claim counter and one status word per tile or chunk of tiles).
+int launch_store_different(const StoreParams& p, const PhiloxKeys& ks, int dtype, cudaStream_t s) {
+  const int rc = launch_store_pipelined(p, ks, dtype, s);
+  if (rc != RAD_EUNSUPPORTED) return rc;
+  count_launch();
+  if (dtype == RAD_BF16)
+    store_different_kernel<bf16><<<p.ntiles, 256, 0, s>>>(p, ks);
+  else
+    store_different_kernel<float><<<p.ntiles, 256, 0, s>>>(p, ks);
+  RAD_CUDA_TRY(cudaGetLastError());
+  return RAD_OK;
+}
+
 int64_t store_workspace_bytes(int variant, int64_t B, int64_t D) {
   if (variant == RAD_SAME_SAMPLE) return 256;
   const int64_t ntiles = ceil_div(B, kTileRows) * ceil_div(D, kTileCols);
@@ -421,10 +391,10 @@ int64_t store_workspace_bytes(int variant, int64_t B, int64_t D) {
 using namespace rad;
 
 extern "C" uint32_t rad_keep_threshold(float p) { return keep_threshold_host(p); }
-extern "C" float rad_effective_p(float p) { return (float)keep_threshold_host(p) / 65536.0f; }
+extern "C" float rad_effective_p(float p) { return (float)keep_threshold_host(p) / (float)kLaneRange; }
 extern "C" float rad_scale(float p) {
   const uint32_t T = keep_threshold_host(p);
-  return T == 0 ? 0.0f : 65536.0f / (float)T;
+  return T == 0 ? 0.0f : (float)kLaneRange / (float)T;
 }
 
 extern "C" int rad_store_size_query(int32_t variant, int32_t dtype, int64_t B, int64_t D, float p,
@@ -435,7 +405,7 @@ extern "C" int rad_store_size_query(int32_t variant, int32_t dtype, int64_t B, i
   const uint32_t T = keep_threshold_host(p);
   if (T == 0) return RAD_EINVAL;
   if ((double)B * (double)D >= 4294967296.0 * 0.75) return RAD_EINVAL;   // 32-bit tile offsets
-  const double pe = T / 65536.0;
+  const double pe = T / (double)kLaneRange;
   const int64_t w32 = ceil_div(D, 32);
   out->relubits_words = B * w32;
   if (variant == RAD_DIFFERENT_SAMPLE) {
@@ -492,7 +462,7 @@ extern "C" int rad_linear_forward_store(const void* A, int64_t lda, const rad_st
     p.A = A; p.lda = lda; p.B = st->B; p.D = st->D;
     p.ncb = (int32_t)ceil_div(st->D, kTileCols);
     p.ntiles = (int32_t)(ceil_div(st->B, kTileRows) * p.ncb);
-    p.T = T; p.scale = 65536.0f / (float)T;
+    p.T = make_keep_threshold(T); p.scale = (float)kLaneRange / (float)T;
     p.c2 = counter_word2(st->layer, RAD_DIFFERENT_SAMPLE); p.c3 = st->step;
     p.values = st->values; p.capacity = st->values_capacity;
     p.keepbits = st->keepbits; p.offsets = st->offsets; p.nnz = st->nnz;
@@ -502,19 +472,13 @@ extern "C" int rad_linear_forward_store(const void* A, int64_t lda, const rad_st
     p.dev_status = dev_status;
     p.vec_ok = (((uintptr_t)A & 15) == 0 && (lda * esz) % 16 == 0) ? 1 : 0;
     RAD_CUDA_TRY(cudaMemsetAsync(workspace, 0, (size_t)need, s));
-    count_launch();
-    if (st->dtype == RAD_BF16)
-      store_different_kernel<bf16><<<p.ntiles, 256, 0, s>>>(p, ks);
-    else
-      store_different_kernel<float><<<p.ntiles, 256, 0, s>>>(p, ks);
-    RAD_CUDA_TRY(cudaGetLastError());
-    return RAD_OK;
+    return launch_store_different(p, ks, st->dtype, s);
   }
 
   if (st->values_ld <= 0 || st->values_ld % 8 != 0 || st->values_capacity < st->B * st->values_ld)
     return RAD_EINVAL;
   SameParams p;
-  p.A = A; p.lda = lda; p.B = st->B; p.D = st->D; p.T = T; p.scale = 65536.0f / (float)T;
+  p.A = A; p.lda = lda; p.B = st->B; p.D = st->D; p.T = make_keep_threshold(T); p.scale = (float)kLaneRange / (float)T;
   p.c2 = counter_word2(st->layer, RAD_SAME_SAMPLE); p.c3 = st->step;
   p.values = st->values; p.ld = st->values_ld; p.keepbits = st->keepbits; p.idx = st->offsets;
   p.nnz = st->nnz; p.dev_status = dev_status;
@@ -588,7 +552,7 @@ extern "C" int rad_linear_forward_store_static(const void* A, int64_t lda, const
   p.A = A; p.lda = lda; p.B = st->B; p.D = st->D;
   p.ncb = (int32_t)ceil_div(st->D, kTileCols);
   p.ntiles = (int32_t)ntiles;
-  p.T = T; p.scale = 65536.0f / (float)T;
+  p.T = make_keep_threshold(T); p.scale = (float)kLaneRange / (float)T;
   p.c2 = counter_word2(st->layer, RAD_DIFFERENT_SAMPLE); p.c3 = st->step;
   p.values = st->values; p.capacity = st->values_capacity;
   p.keepbits = st->keepbits; p.offsets = st->offsets; p.nnz = st->nnz;
@@ -599,11 +563,5 @@ extern "C" int rad_linear_forward_store_static(const void* A, int64_t lda, const
   p.vec_ok = (((uintptr_t)A & 15) == 0 && (lda * esz) % 16 == 0) ? 1 : 0;
   // the array keeps what the last call left: the counter and this call's status words start at zero
   RAD_CUDA_TRY(cudaMemsetAsync(scratch, 0, 256 + 8 * (size_t)ntiles, s));
-  count_launch();
-  if (st->dtype == RAD_BF16)
-    store_different_kernel<bf16><<<p.ntiles, 256, 0, s>>>(p, ks);
-  else
-    store_different_kernel<float><<<p.ntiles, 256, 0, s>>>(p, ks);
-  RAD_CUDA_TRY(cudaGetLastError());
-  return RAD_OK;
+  return launch_store_different(p, ks, st->dtype, s);
 }

@@ -1,0 +1,58 @@
+// Shared by the two different-sample store kernels: launch parameters and the look-back status word.
+#pragma once
+
+#include "common.cuh"
+
+namespace rad {
+
+// ---- look-back status word ---------------------------------------------------------------------
+// bits 63..62 flag, 61..32 padded prefix in granules of 8 elements, 31..0 exact kept count.
+constexpr uint64_t kFlagShift = 62;
+constexpr uint64_t kFlagAggregate = 1, kFlagPrefix = 2, kFlagPoison = 3;
+constexpr uint64_t kValueMask = (1ull << kFlagShift) - 1;
+constexpr int kSpinLimit = 1 << 20;   // bounded wait: about a second with the back-off below
+
+__device__ __forceinline__ uint64_t pack_counts(uint32_t granules, uint32_t exact) {
+  return ((uint64_t)granules << 32) | exact;
+}
+__device__ __forceinline__ uint64_t load_status(const uint64_t* p) {
+  uint64_t v;
+  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void store_status(uint64_t* p, uint64_t v) {
+  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ uint64_t warp_sum_u64(uint64_t v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+struct StoreParams {
+  const void* A;
+  int64_t lda;
+  int64_t B, D;
+  int32_t ncb;        // column blocks
+  int32_t ntiles;
+  KeepThreshold T;    // keep threshold
+  float scale;
+  uint32_t c2, c3;    // counter words 2 and 3
+  void* values;
+  int64_t capacity;
+  uint32_t* keepbits;
+  uint32_t* offsets;
+  int64_t* nnz;
+  uint32_t* relubits;
+  int32_t w32;        // relu-bit words per row
+  uint64_t* status;   // ntiles look-back words (zeroed before launch)
+  uint32_t* ticket;   // zeroed before launch
+  int32_t* dev_status;
+  int32_t vec_ok;     // rows are 16-byte aligned: 8-element vector loads allowed
+};
+
+// store_pipe.cu: the persistent TMA-fed kernel.  RAD_EUNSUPPORTED (nothing enqueued) when the input does not
+// meet the alignment rules of a tensor map; the caller then takes the generic kernel.
+int launch_store_pipelined(const StoreParams& p, const PhiloxKeys& ks, int dtype, cudaStream_t s);
+
+}  // namespace rad

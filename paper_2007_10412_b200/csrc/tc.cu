@@ -885,21 +885,27 @@ __global__ void __launch_bounds__(256) zero_f32_kernel(float* out, int64_t rows,
 }
 
 // ---- host side -------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+}  // namespace
 
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
+// cuTensorMapEncodeTiled through the runtime's driver entry point table (no link against libcuda).
+void* tensor_map_encoder() {
+  static void* fn = nullptr;
   if (fn == nullptr) {
     void* sym = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
         qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(sym);
+      fn = sym;
   }
   return fn;
 }
+
+namespace {
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() { return reinterpret_cast<EncodeTiledFn>(tensor_map_encoder()); }
 
 // bf16 matrix, `inner` contiguous elements per row, `outer` rows of `ld` elements; box = 64 x box_outer.
 int make_map(CUtensorMap* map, const void* ptr, int64_t inner, int64_t outer, int64_t ld, int box_outer) {
@@ -952,7 +958,7 @@ DwPlan plan_dw(const rad_store* st, int64_t H) {
   const int64_t kblocks = ceil_div(st->B, BK);
   int64_t m_expect;
   if (st->variant == RAD_SAME_SAMPLE) {
-    m_expect = std::max<int64_t>(1, (int64_t)std::llround((double)st->D * keep_threshold_host(st->p) / 65536.0));
+    m_expect = std::max<int64_t>(1, (int64_t)std::llround((double)st->D * keep_threshold_host(st->p) / (double)kLaneRange));
     d.partial_rows = round_up(std::min(st->values_ld, round_up(st->D, 8)), BM);
     d.comp_cap = 0;
     d.stages = 3;
@@ -961,7 +967,7 @@ DwPlan plan_dw(const rad_store* st, int64_t H) {
     m_expect = st->D;
     d.partial_rows = round_up(st->D, BM);
     // per-tile value staging: mean + 8 sigma of Binomial(8192, p_eff), padded, in bytes
-    const double pe = keep_threshold_host(st->p) / 65536.0, n = (double)kTileRows * kTileCols;
+    const double pe = keep_threshold_host(st->p) / (double)kLaneRange, n = (double)kTileRows * kTileCols;
     int64_t cap = (int64_t)(n * pe + 8.0 * std::sqrt(n * pe * (1.0 - pe)) + 16.0);
     cap = std::min<int64_t>(round_up(cap, 8), (int64_t)n) * 2;
     d.comp_cap = (int)round_up(cap, 128);
