@@ -145,6 +145,22 @@ int rad_linear_forward_store(const void* A /* device */, int64_t lda, const rad_
                              int32_t* dev_status /* device or NULL */, void* stream);
 
 /*
+ * Which kernel the different-sample store runs (Sec. 3.2 / 4.2: same operation,
+ * same layout, bit-identical output).  The persistent TMA-fed kernel is made for
+ * many tiles and sparse masks, the generic one-CTA-per-tile kernel for small or
+ * dense problems and for inputs a tensor map cannot describe (A or lda not
+ * 16-byte aligned).  RAD_STORE_KERNEL_AUTO picks by size and keep probability;
+ * the other two values force a kernel where it can run (tests use them to put
+ * both kernels through the same cases).  Host only, process-wide, not
+ * synchronised with calls in flight on other threads.  Returns the previous
+ * setting, or RAD_EINVAL.
+ */
+#define RAD_STORE_KERNEL_AUTO      0
+#define RAD_STORE_KERNEL_GENERIC   1
+#define RAD_STORE_KERNEL_PIPELINED 2
+int rad_set_store_kernel(int32_t which);
+
+/*
  * rad_linear_forward_store without a workspace argument (the paper has no
  * counterpart: this entry point exists for the sake of callers, not of the
  * method).  It is meant for programs that must not allocate device memory

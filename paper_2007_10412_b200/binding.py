@@ -67,7 +67,7 @@ class rad_step_stats(C.Structure):
                                          "unsampled_bytes", "full_backprop_bytes")]
 
 
-EXPORTS = ["rad_keep_threshold", "rad_effective_p", "rad_scale", "rad_store_size_query",
+EXPORTS = ["rad_keep_threshold", "rad_effective_p", "rad_scale", "rad_store_size_query", "rad_set_store_kernel",
            "rad_linear_forward_store", "rad_linear_forward_store_static", "rad_weight_grad_workspace", "rad_linear_weight_grad",
            "rad_linear_forward", "rad_softmax_xent", "rad_input_grad_workspace", "rad_linear_input_grad",
            "rad_mlp_workspace", "rad_mlp_step", "rad_irnn_workspace", "rad_irnn_step", "rad_cnn_workspace", "rad_cnn_step", "rad_launch_count", "rad_strerror", "rad_version"]
@@ -93,6 +93,7 @@ def lib():
         L.rad_version.restype = C.c_char_p
         L.rad_launch_count.restype = C.c_int64
         i32, i64, f32, vp = C.c_int32, C.c_int64, C.c_float, C.c_void_p
+        L.rad_set_store_kernel.argtypes = [i32]
         L.rad_store_size_query.argtypes = [i32, i32, i64, i64, f32, C.POINTER(rad_store_sizes)]
         L.rad_linear_forward_store.argtypes = [vp, i64, C.POINTER(rad_store), vp, i64, vp, vp]
         L.rad_linear_forward_store_static.argtypes = [vp, i64, C.POINTER(rad_store), vp, vp]
@@ -200,6 +201,17 @@ def rad_linear_forward_store(A, store, dev_status=None):
     _check(lib().rad_linear_forward_store(_ptr(A), A.stride(0), C.byref(store.c), _ptr(store.workspace),
                                           store.workspace.numel(), _ptr(dev_status), _stream()),
            "rad_linear_forward_store")
+
+
+STORE_KERNELS = {"auto": 0, "generic": 1, "pipelined": 2}
+
+
+def rad_set_store_kernel(which):
+    """Selects the different-sample store kernel ("auto", "generic", "pipelined"); returns the previous name."""
+    prev = lib().rad_set_store_kernel(STORE_KERNELS[which])
+    if prev < 0:
+        _check(prev, "rad_set_store_kernel")
+    return {v: k for k, v in STORE_KERNELS.items()}[prev]
 
 
 STATIC_STORE_MAX_TILES = 131072

@@ -365,10 +365,18 @@ __global__ void __launch_bounds__(256) relu_bits_kernel(const T* A, int64_t lda,
   }
 }
 
+constexpr int kPipelinedMinTiles = 2048;
+int g_store_kernel = RAD_STORE_KERNEL_AUTO;
+
 // The persistent TMA-fed kernel where the input can be described by a tensor map, else the generic one
 // (same layout, same scratch: a claim counter and one status word per tile or chunk of tiles).
-int launch_store_different(const StoreParams& p, const PhiloxKeys& ks, int dtype, cudaStream_t s) {
-  const int rc = launch_store_pipelined(p, ks, dtype, s);
+int launch_store_different(const StoreParams& p, const PhiloxKeys& ks, int dtype, uint32_t T, cudaStream_t s) {
+  // The pipelined kernel pays off where there are many tiles per SM and most entries are dropped: its
+  // per-entry staging loop is slower than the generic kernel's for dense masks, and a CTA works
+  // through a chunk of tiles one after the other, which only adds latency to a small problem.
+  const bool pipelined = g_store_kernel == RAD_STORE_KERNEL_PIPELINED ||
+                         (g_store_kernel == RAD_STORE_KERNEL_AUTO && p.ntiles >= kPipelinedMinTiles && T <= kLaneRange / 2);
+  const int rc = pipelined ? launch_store_pipelined(p, ks, dtype, s) : RAD_EUNSUPPORTED;
   if (rc != RAD_EUNSUPPORTED) return rc;
   count_launch();
   if (dtype == RAD_BF16)
@@ -389,6 +397,14 @@ int64_t store_workspace_bytes(int variant, int64_t B, int64_t D) {
 }  // namespace rad
 
 using namespace rad;
+
+extern "C" int rad_set_store_kernel(int32_t which) {
+  if (which != RAD_STORE_KERNEL_AUTO && which != RAD_STORE_KERNEL_GENERIC && which != RAD_STORE_KERNEL_PIPELINED)
+    return RAD_EINVAL;
+  const int prev = g_store_kernel;
+  g_store_kernel = which;
+  return prev;
+}
 
 extern "C" uint32_t rad_keep_threshold(float p) { return keep_threshold_host(p); }
 extern "C" float rad_effective_p(float p) { return (float)keep_threshold_host(p) / (float)kLaneRange; }
@@ -472,7 +488,7 @@ extern "C" int rad_linear_forward_store(const void* A, int64_t lda, const rad_st
     p.dev_status = dev_status;
     p.vec_ok = (((uintptr_t)A & 15) == 0 && (lda * esz) % 16 == 0) ? 1 : 0;
     RAD_CUDA_TRY(cudaMemsetAsync(workspace, 0, (size_t)need, s));
-    return launch_store_different(p, ks, st->dtype, s);
+    return launch_store_different(p, ks, st->dtype, T, s);
   }
 
   if (st->values_ld <= 0 || st->values_ld % 8 != 0 || st->values_capacity < st->B * st->values_ld)
@@ -563,5 +579,5 @@ extern "C" int rad_linear_forward_store_static(const void* A, int64_t lda, const
   p.vec_ok = (((uintptr_t)A & 15) == 0 && (lda * esz) % 16 == 0) ? 1 : 0;
   // the array keeps what the last call left: the counter and this call's status words start at zero
   RAD_CUDA_TRY(cudaMemsetAsync(scratch, 0, 256 + 8 * (size_t)ntiles, s));
-  return launch_store_different(p, ks, st->dtype, s);
+  return launch_store_different(p, ks, st->dtype, T, s);
 }

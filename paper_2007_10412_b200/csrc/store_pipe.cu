@@ -2,23 +2,22 @@
 // layer input is sampled, scaled by 1 / p_eff and only the kept entries are held).
 //
 // A CTA claims chunks of kChunk consecutive 64 x 128 tiles in ticket order and runs two phases per
-// chunk, the first phase of the next chunk ahead of the second phase of the current one:
+// chunk, the first phase kAhead chunks ahead of the second:
 //   phase 1  needs no data: every compute thread draws the 32 keep decisions of one keep-bit word
 //            per tile (two Philox calls), writes the word, and the warp totals go to shared memory;
 //   look-back a service warp adds the chunk's padded and exact counts, publishes them, and finds where
-//            the chunk starts in `values` from the chunks before it (decoupled look-back);
+//            the chunk starts in `values` from the chunks before it (decoupled look-back over one
+//            status word per chunk);
 //   phase 2  the tile of A arrives in shared memory by TMA (a second service warp runs a ring of
 //            loads ahead of the compute warps); a warp scan over the counts gives every word its
-//            place in (row, column) order, and each thread walks the set bits of its word, scaling
-//            the kept entries into a staging buffer;
-//   output   a third service warp pads the tile to a multiple of eight entries and sends the staging
-//            buffer to `values` with one bulk copy.
-// The look-back of chunk c+1 therefore has the whole second phase of chunk c to finish in, and no
-// compute thread ever loads from or stores to global memory except for the index words.
+//            place in (row, column) order; each thread walks the set bits of its word and scales the
+//            kept entries into its warp's staging buffer, which the warp then copies to `values`
+//            with coalesced stores.  No compute warp waits for another one in this phase.
+// The look-back of a chunk therefore has kAhead chunk periods to finish in.
 // The layout produced is the one of the generic kernel: the order of tiles in `values` is the tile index.
 //
 // Every wait is bounded (2 s on the global timer).  On expiry the CTA raises RAD_DEV_ETIMEOUT, all
-// roles leave their loops, outstanding loads and bulk copies are waited for, and the kernel returns.
+// roles leave their loops, outstanding loads are waited for, and the kernel returns.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -27,23 +26,26 @@
 namespace rad {
 namespace {
 
-constexpr int kChunk = 4;                       // tiles per claimed chunk
+constexpr int kChunk = 8;                       // tiles per claimed chunk
 constexpr int kComputeWarps = 8;                // 256 threads: one keep-bit word of a tile each
-constexpr int kLoaderWarp = kComputeWarps, kLookbackWarp = kComputeWarps + 1;   // the output warp is the last one
-constexpr int kPipeThreads = (kComputeWarps + 3) * 32;
-constexpr int kSlots = 4;                       // chunk descriptors in flight
+constexpr int kLoaderWarp = kComputeWarps;      // the look-back warp is the last one
+constexpr int kPipeThreads = (kComputeWarps + 2) * 32;
+constexpr int kAhead = 2;                       // chunks between the first and the second phase
+constexpr int kSlots = 8;                       // chunk descriptors in flight
+constexpr int kLookWindows = 8;                 // look-back: 32 status words per window
 constexpr uint32_t kNoChunk = 0xffffffffu;
 constexpr uint64_t kPipeWaitLimitNs = 2000000000ull;
 constexpr int kTileElems = kTileRows * kTileCols;
+constexpr int kWarpElems = kTileElems / kComputeWarps;   // entries of a tile that one warp owns
 
 template <typename T, int S>
 struct PipeSmem {
   alignas(128) T raw[S][kTileElems];            // tiles of A as loaded
-  alignas(128) T outv[2][kTileElems];           // kept values of a tile in (row, column) order
+  alignas(16) T wbuf[kComputeWarps][kWarpElems];   // kept values of a warp's eight rows, in order
   uint64_t full[S], empty[S];                   // raw ring
-  uint64_t staged[2], out_free[2];              // staging buffers
   uint64_t chunk_ready[kSlots], cnt_ready[kSlots], base_ready[kSlots];
   uint32_t chunk_id[kSlots];
+  uint32_t tile_slab[kSlots][kChunk], tile_cb[kSlots][kChunk];   // row slab and column block of each tile
   uint32_t warp_total[kSlots][kChunk][kComputeWarps];
   uint32_t tile_total[kSlots][kChunk];
   int64_t tile_base[kSlots][kChunk];            // first element in `values`; -1: do not write
@@ -74,9 +76,9 @@ __device__ __forceinline__ uint64_t timer_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Bounded wait; false when the CTA is giving up (this wait or another one ran out of time).
-__device__ __forceinline__ bool bar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  if (bar_try_wait(bar, parity)) return true;
+// Bounded wait; false when the CTA is giving up (this wait or another one ran out of time).  The
+// slow path is kept out of line: it is rarely taken and the kernel's code should stay small.
+__device__ __noinline__ bool bar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   const uint64_t t0 = timer_ns();
   while (true) {
 #pragma unroll 1
@@ -89,20 +91,15 @@ __device__ __forceinline__ bool bar_wait(uint64_t* bar, uint32_t parity, volatil
     }
   }
 }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ bool bar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  if (bar_try_wait(bar, parity)) return true;
+  return bar_wait_slow(bar, parity, abort_flag);
+}
 __device__ __forceinline__ void tma_load_tile(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(smem_addr(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_addr(bar)) : "memory");
 }
-__device__ __forceinline__ void bulk_store(void* gdst, const void* ssrc, uint32_t bytes) {
-  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_addr(ssrc)), "r"(bytes)
-               : "memory");
-  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-}
-__device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void bulk_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-
 __device__ __forceinline__ uint32_t warp_inclusive_scan(uint32_t v, int lane) {
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -143,7 +140,7 @@ __device__ __forceinline__ uint32_t positive32(const bf16* src) {
 }
 
 template <typename T, int S>
-__global__ void __launch_bounds__(kPipeThreads) store_pipelined_kernel(const StoreParams p, const PhiloxKeys ks,
+__global__ void __launch_bounds__(kPipeThreads, 3) store_pipelined_kernel(const StoreParams p, const PhiloxKeys ks,
                                                                       const __grid_constant__ CUtensorMap tmA) {
   extern __shared__ unsigned char smem_raw[];
   PipeSmem<T, S>& sm = *reinterpret_cast<PipeSmem<T, S>*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
@@ -154,7 +151,6 @@ __global__ void __launch_bounds__(kPipeThreads) store_pipelined_kernel(const Sto
 
   if (tid == 0) {
     for (int s = 0; s < S; ++s) { bar_init(&sm.full[s], 1); bar_init(&sm.empty[s], kComputeWarps); }
-    for (int b = 0; b < 2; ++b) { bar_init(&sm.staged[b], kComputeWarps); bar_init(&sm.out_free[b], 1); }
     for (int q = 0; q < kSlots; ++q) {
       bar_init(&sm.chunk_ready[q], 1);
       bar_init(&sm.cnt_ready[q], kComputeWarps);
@@ -171,9 +167,8 @@ __global__ void __launch_bounds__(kPipeThreads) store_pipelined_kernel(const Sto
     // 8 * warp + lane / 4 of the tile, columns 32 * (lane % 4) .. + 31.
     // ---------------------------------------------------------------------------------------------
     const int r = warp * 8 + (lane >> 2), wq = lane & 3;
+    const uint32_t nrows = (uint32_t)p.B, ncols = (uint32_t)p.D;   // B * D < 2^32 (checked by the host)
     uint32_t n = 0;                               // tiles this CTA has worked through (ring position)
-    uint32_t m_cur[kChunk], m_nxt[kChunk];
-    uint32_t chunk_cur = kNoChunk, chunk_nxt = kNoChunk;
 
     auto phase1 = [&](uint32_t seq, uint32_t (&m)[kChunk]) -> uint32_t {
       const int slot = seq % kSlots;
@@ -185,18 +180,17 @@ __global__ void __launch_bounds__(kPipeThreads) store_pipelined_kernel(const Sto
         const uint32_t tile = chunk * kChunk + g;
         uint32_t mm = 0;
         if (tile < ntiles) {
-          const uint32_t slab = tile / (uint32_t)p.ncb, cb = tile - slab * (uint32_t)p.ncb;
-          const int64_t row = (int64_t)slab * kTileRows + r;
-          const int64_t col0 = (int64_t)cb * kTileCols + wq * 32;
-          const int64_t nv = p.D - col0;
-          if (row < p.B && nv > 0) {
-            const uint32_t g16 = (uint32_t)(col0 >> 4);
-            const uint32_t lo = philox_keep16(g16, (uint32_t)row, p.c2, p.c3, ks, p.T);
-            const uint32_t hi = philox_keep16(g16 + 1u, (uint32_t)row, p.c2, p.c3, ks, p.T);
+          const uint32_t row = sm.tile_slab[slot][g] * kTileRows + r;
+          const uint32_t col0 = sm.tile_cb[slot][g] * kTileCols + wq * 32;
+          if (row < nrows && col0 < ncols) {
+            const uint32_t g16 = col0 >> 4;
+            const uint32_t lo = philox_keep16(g16, row, p.c2, p.c3, ks, p.T);
+            const uint32_t hi = philox_keep16(g16 + 1u, row, p.c2, p.c3, ks, p.T);
             mm = lo | (hi << 16);
-            if (nv < 32) mm &= (1u << (int)nv) - 1u;
+            const uint32_t nv = ncols - col0;
+            if (nv < 32) mm &= (1u << nv) - 1u;
           }
-          p.keepbits[(int64_t)tile * kTileWords + warp * 32 + lane] = mm;
+          p.keepbits[tile * (uint32_t)kTileWords + (uint32_t)(warp * 32 + lane)] = mm;
         }
         m[g] = mm;
         const uint32_t wt = __reduce_add_sync(0xffffffffu, __popc(mm));
@@ -207,69 +201,109 @@ __global__ void __launch_bounds__(kPipeThreads) store_pipelined_kernel(const Sto
       return chunk;
     };
 
-    uint32_t seq = 0;
-    chunk_nxt = phase1(seq, m_nxt);
-    bool ok = true;
-    while (ok && chunk_nxt != kNoChunk) {
-      chunk_cur = chunk_nxt;
+    // chunks whose first phase is done, oldest first
+    uint32_t mq[kAhead][kChunk], cq[kAhead];
+    uint32_t seq1 = 0, seq2 = 0;                  // chunks handed to the first / second phase so far
+    bool more = true;                             // the loader has not yet said that the work is finished
 #pragma unroll
-      for (int g = 0; g < kChunk; ++g) m_cur[g] = m_nxt[g];
-      const int slot = seq % kSlots;
-      const uint32_t slot_parity = (seq / kSlots) & 1u;
-      ++seq;
-      chunk_nxt = phase1(seq, m_nxt);
-      // phase 2 of chunk_cur; the other warps' totals of its first phase are needed now
-      if (!bar_wait(&sm.cnt_ready[slot], slot_parity, abort_flag)) break;
+    for (int a = 0; a < kAhead; ++a) {
+      cq[a] = kNoChunk;
+#pragma unroll
+      for (int g = 0; g < kChunk; ++g) mq[a][g] = 0;
+    }
+    bool ok = true;
+#pragma unroll 1
+    for (uint32_t it = 0; ok; ++it) {
+      uint32_t m_new[kChunk], c_new = kNoChunk;
+#pragma unroll
+      for (int g = 0; g < kChunk; ++g) m_new[g] = 0;
+      if (more) {
+        c_new = phase1(seq1++, m_new);
+        more = c_new != kNoChunk;
+      }
+      if (it >= (uint32_t)kAhead && cq[0] == kNoChunk) break;     // every claimed chunk is through
+      if (cq[0] != kNoChunk) {
+      const uint32_t chunk_cur = cq[0];
+      const int slot = seq2 % kSlots;
+      const uint32_t slot_parity = (seq2 / kSlots) & 1u;
+      ++seq2;
+      // phase 2 of the oldest chunk: the other warps' totals of its first phase and the chunk's place
+      // in `values` are needed now
+      if (!bar_wait(&sm.cnt_ready[slot], slot_parity, abort_flag) ||
+          !bar_wait(&sm.base_ready[slot], slot_parity, abort_flag))
+        break;
+      T* const wb = sm.wbuf[warp];
 #pragma unroll
       for (int g = 0; g < kChunk; ++g) {
         const uint32_t tile = chunk_cur * kChunk + g;
         if (tile >= ntiles) break;
-        const int s = n % S, b = n & 1;
-        uint32_t mm = m_cur[g];
+        const int s = n % S;
+        const uint32_t mm = mq[0][g];
         const uint32_t cnt = __popc(mm);
         const uint32_t incl = warp_inclusive_scan(cnt, lane);
         const uint32_t wt = sm.warp_total[slot][g][lane & 7];
         const uint32_t wbase = __reduce_add_sync(0xffffffffu, lane < warp ? wt : 0u);
-        uint32_t pos = wbase + incl - cnt;
+        const uint32_t wtotal = __shfl_sync(0xffffffffu, incl, 31);
         if (wq == 0)
-          reinterpret_cast<uint16_t*>(p.keepbits + (int64_t)tile * kTileWords + kBitWords)[r] = (uint16_t)pos;
-        if (!bar_wait(&sm.out_free[b], ((n >> 1) & 1u) ^ 1u, abort_flag) ||
-            !bar_wait(&sm.full[s], (n / S) & 1u, abort_flag)) {
+          reinterpret_cast<uint16_t*>(p.keepbits + (int64_t)tile * kTileWords + kBitWords)[r] =
+              (uint16_t)(wbase + incl - cnt);
+        const int64_t base = sm.tile_base[slot][g];
+        if (!bar_wait(&sm.full[s], (n / S) & 1u, abort_flag)) {
           ok = false;
           break;
         }
         const T* src = sm.raw[s] + r * kTileCols + wq * 32;
-        T* dst = sm.outv[b] + pos;
-        uint32_t rev = __brev(mm);                // leading zeros of rev = index of the lowest set bit
+        // kept entries go to the warp's buffer as they are (bit h of the reversed word is column 31 - h);
+        // scaling waits for the copy to `values`, where every lane has work
+        const T* src_end = src + 31;
+        T* dst = wb + (incl - cnt);
+        uint32_t rev = __brev(mm);
         while (rev != 0) {
-          const int q = __clz(rev);
-          rev &= ~(0x80000000u >> q);
-          *dst++ = from_float<T>(raw_to_float(src[q]) * p.scale);
+          uint32_t h;
+          asm("bfind.u32 %0, %1;" : "=r"(h) : "r"(rev));
+          rev &= ~(1u << h);
+          *dst++ = *(src_end - h);
         }
         if (p.relubits != nullptr) {
-          const uint32_t slab = tile / (uint32_t)p.ncb, cb = tile - slab * (uint32_t)p.ncb;
-          const int64_t row = (int64_t)slab * kTileRows + r;
-          const int word = (int)cb * 4 + wq;
-          if (row < p.B && word < p.w32) {
+          const uint32_t row = sm.tile_slab[slot][g] * kTileRows + r;
+          const uint32_t word = sm.tile_cb[slot][g] * 4 + wq;
+          if (row < nrows && word < (uint32_t)p.w32) {
             uint32_t rb = positive32(src);
-            const int64_t nv = p.D - (int64_t)word * 32;
-            if (nv < 32) rb &= (1u << (int)nv) - 1u;
-            p.relubits[row * p.w32 + word] = rb;
+            const uint32_t nv = ncols - word * 32;
+            if (nv < 32) rb &= (1u << nv) - 1u;
+            p.relubits[(int64_t)row * p.w32 + word] = rb;
           }
         }
-        fence_async_smem();                       // the staging buffer leaves through the async proxy
         __syncwarp();
-        if (lane == 0) {
-          bar_arrive(&sm.staged[b]);
-          bar_arrive(&sm.empty[s]);
+        if (lane == 0) bar_arrive(&sm.empty[s]);   // the tile of A is not read again
+        if (base >= 0) {
+          T* out = static_cast<T*>(p.values) + base + wbase;
+          for (uint32_t i = lane; i < wtotal; i += 32) out[i] = from_float<T>(raw_to_float(wb[i]) * p.scale);
+          if (warp == kComputeWarps - 1) {
+            // zeros up to the next multiple of kValueAlign after the tile's last value
+            const uint32_t total = wbase + wtotal;
+            const uint32_t padded = (total + kValueAlign - 1) / kValueAlign * kValueAlign;
+            if (total + lane < padded) out[wtotal + lane] = from_float<T>(0.0f);
+          }
         }
+        __syncwarp();                             // the staging buffer is rewritten for the next tile
         ++n;
       }
+      }
+#pragma unroll
+      for (int a = 0; a + 1 < kAhead; ++a) {
+        cq[a] = cq[a + 1];
+#pragma unroll
+        for (int g = 0; g < kChunk; ++g) mq[a][g] = mq[a + 1][g];
+      }
+      cq[kAhead - 1] = c_new;
+#pragma unroll
+      for (int g = 0; g < kChunk; ++g) mq[kAhead - 1][g] = m_new[g];
     }
   } else if (warp == kLoaderWarp) {
     // ---------------------------------------------------------------------------------------------
-    // loader: claims chunks one ahead of the loads it issues, so that the compute warps can run the
-    // first phase of the next chunk before the second phase of the current one.
+    // loader: claims chunks kAhead + 1 ahead of the loads it issues, so that the compute warps can run
+    // the first phase of a chunk kAhead chunks before its second phase.
     // ---------------------------------------------------------------------------------------------
     if (lane == 0) {
       uint32_t n = 0, seq_claim = 0;
@@ -279,17 +313,26 @@ __global__ void __launch_bounds__(kPipeThreads) store_pipelined_kernel(const Sto
         const uint32_t id = t < nchunks ? t : kNoChunk;
         const int slot = seq_claim % kSlots;
         sm.chunk_id[slot] = id;
+        if (id != kNoChunk) {
+          uint32_t slab = id * kChunk / (uint32_t)p.ncb, cb = id * kChunk - slab * (uint32_t)p.ncb;
+          for (int g = 0; g < kChunk; ++g) {
+            sm.tile_slab[slot][g] = slab;
+            sm.tile_cb[slot][g] = cb;
+            if (++cb == (uint32_t)p.ncb) { cb = 0; ++slab; }
+          }
+        }
         bar_arrive(&sm.chunk_ready[slot]);
         ++seq_claim;
         if (id == kNoChunk) more = false;
         return id;
       };
-      uint32_t cur = claim();
-      uint32_t nxt = more ? claim() : kNoChunk;
+      uint32_t q[kAhead + 1];                     // claimed, not yet loaded, oldest first
+#pragma unroll
+      for (int a = 0; a <= kAhead; ++a) q[a] = more ? claim() : kNoChunk;
       bool ok = true;
-      while (ok && cur != kNoChunk) {
+      while (ok && q[0] != kNoChunk) {
         for (int g = 0; g < kChunk && ok; ++g) {
-          const uint32_t tile = cur * kChunk + g;
+          const uint32_t tile = q[0] * kChunk + g;
           if (tile >= ntiles) break;
           const int s = n % S;
           if (!bar_wait(&sm.empty[s], ((n / S) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
@@ -298,8 +341,9 @@ __global__ void __launch_bounds__(kPipeThreads) store_pipelined_kernel(const Sto
           tma_load_tile(sm.raw[s], &tmA, (int)(cb * kTileCols), (int)(slab * kTileRows), &sm.full[s]);
           ++n;
         }
-        cur = nxt;
-        nxt = (ok && more) ? claim() : kNoChunk;
+#pragma unroll
+        for (int a = 0; a < kAhead; ++a) q[a] = q[a + 1];
+        q[kAhead] = (ok && more) ? claim() : kNoChunk;
       }
       if (*abort_flag != 0) {
         // loads already issued still write this CTA's shared memory: wait for the last one of each stage
@@ -310,65 +354,89 @@ __global__ void __launch_bounds__(kPipeThreads) store_pipelined_kernel(const Sto
         }
       }
     }
-  } else if (warp == kLookbackWarp) {
+  } else {
     // ---------------------------------------------------------------------------------------------
     // look-back: one status word per chunk (flag, padded prefix in granules of 8, exact count)
     // ---------------------------------------------------------------------------------------------
-    for (uint32_t seq = 0;; ++seq) {
+    // A chunk's counts are published as soon as its first phase is done; its look-back starts one
+    // chunk later, when the chunks before it (other CTAs work at the same pace) have published theirs.
+    struct Counts { uint32_t tot[kChunk], chunk_gran, chunk_exact; };
+    auto publish = [&](uint32_t seq, Counts& c) -> uint32_t {
       const int slot = seq % kSlots;
       const uint32_t par = (seq / kSlots) & 1u;
-      if (!bar_wait(&sm.chunk_ready[slot], par, abort_flag)) break;
+      if (!bar_wait(&sm.chunk_ready[slot], par, abort_flag)) return kNoChunk;
       const uint32_t chunk = sm.chunk_id[slot];
-      if (chunk == kNoChunk) break;
-      if (!bar_wait(&sm.cnt_ready[slot], par, abort_flag)) break;
-      // lane (8 g + w) reads warp w's total of tile g; a butterfly over eight lanes sums a tile
-      static_assert(kChunk * kComputeWarps == 32, "one lane per (tile, warp)");
-      uint32_t t = sm.warp_total[slot][lane >> 3][lane & 7];
-      t += __shfl_xor_sync(0xffffffffu, t, 1);
-      t += __shfl_xor_sync(0xffffffffu, t, 2);
-      t += __shfl_xor_sync(0xffffffffu, t, 4);
-      uint32_t tot[kChunk], gran[kChunk];
-      uint32_t chunk_gran = 0, chunk_exact = 0;
+      if (chunk == kNoChunk) return kNoChunk;
+      if (!bar_wait(&sm.cnt_ready[slot], par, abort_flag)) return kNoChunk;
+      // lane (8 g + w) reads warp w's totals of tiles g and g + 4; a butterfly over eight lanes sums a tile
+      static_assert(kChunk == 8 && kComputeWarps == 8, "two (tile, warp) entries per lane");
+      uint32_t t0 = sm.warp_total[slot][lane >> 3][lane & 7];
+      uint32_t t1 = sm.warp_total[slot][4 + (lane >> 3)][lane & 7];
+#pragma unroll
+      for (int o = 1; o < 8; o <<= 1) {
+        t0 += __shfl_xor_sync(0xffffffffu, t0, o);
+        t1 += __shfl_xor_sync(0xffffffffu, t1, o);
+      }
+      c.chunk_gran = 0;
+      c.chunk_exact = 0;
 #pragma unroll
       for (int g = 0; g < kChunk; ++g) {
-        tot[g] = __shfl_sync(0xffffffffu, t, 8 * g);
-        gran[g] = (tot[g] + kValueAlign - 1) / kValueAlign;
-        chunk_gran += gran[g];
-        chunk_exact += tot[g];
+        c.tot[g] = __shfl_sync(0xffffffffu, g < 4 ? t0 : t1, 8 * (g & 3));
+        c.chunk_gran += (c.tot[g] + kValueAlign - 1) / kValueAlign;
+        c.chunk_exact += c.tot[g];
       }
       if (lane == 0)
         store_status(p.status + chunk, ((chunk == 0 ? kFlagPrefix : kFlagAggregate) << kFlagShift) |
-                                           pack_counts(chunk_gran, chunk_exact));
-      uint64_t excl = 0;
+                                           pack_counts(c.chunk_gran, c.chunk_exact));
+      return chunk;
+    };
+    Counts cur, nxt;
+    uint32_t chunk = publish(0, cur);
+    for (uint32_t seq = 0; chunk != kNoChunk; ++seq) {
+      const int slot = seq % kSlots;
+      const uint32_t chunk_nxt = publish(seq + 1, nxt);
+      if (*abort_flag != 0) break;
+      const uint32_t chunk_gran = cur.chunk_gran, chunk_exact = cur.chunk_exact;
+      // Look-back.  The CTAs of the grid work through their chunks at the same pace, so the nearest
+      // chunk whose prefix is known is typically a few hundred chunks back: every lane fetches
+      // kLookWindows status words at once (all loads in flight together); the windows of 32 are
+      // examined nearest first, every lane adds up what it holds, and one warp sum ends the walk.
+      uint64_t mine = 0;
       bool failed = false;
       if (chunk != 0) {
         int64_t idx = (int64_t)chunk - 1;
         bool done = false;
-        while (!done) {
-          const int64_t j = idx - lane;
-          uint64_t w = kFlagPrefix << kFlagShift;          // before the first chunk: prefix 0
-          if (j >= 0) {
+        while (!done && !failed) {
+          uint64_t w[kLookWindows];
+#pragma unroll
+          for (int k = 0; k < kLookWindows; ++k) {
+            const int64_t j = idx - 32 * k - lane;
+            w[k] = j >= 0 ? load_status(p.status + j) : (kFlagPrefix << kFlagShift);   // before chunk 0: prefix 0
+          }
+#pragma unroll
+          for (int k = 0; k < kLookWindows; ++k) {
+            if (done || failed) break;
+            const int64_t j = idx - 32 * k - lane;
             int spins = 0;
-            w = load_status(p.status + j);
-            while ((w >> kFlagShift) == 0 && spins < kSpinLimit) {
+            while ((w[k] >> kFlagShift) == 0 && spins < kSpinLimit) {
               __nanosleep(spins < 64 ? 32 : 256);
-              w = load_status(p.status + j);
+              w[k] = load_status(p.status + j);
               ++spins;
             }
+            const uint64_t flag = w[k] >> kFlagShift;
+            if (__any_sync(0xffffffffu, flag == 0 || flag == kFlagPoison)) { failed = true; break; }
+            const uint32_t pm = __ballot_sync(0xffffffffu, flag == kFlagPrefix);
+            if (pm != 0) {
+              if (lane <= __ffs(pm) - 1) mine += w[k] & kValueMask;
+              done = true;
+            } else {
+              mine += w[k] & kValueMask;
+            }
           }
-          const uint64_t flag = w >> kFlagShift;
-          if (__any_sync(0xffffffffu, flag == 0 || flag == kFlagPoison)) { failed = true; break; }
-          const uint32_t pm = __ballot_sync(0xffffffffu, flag == kFlagPrefix);
-          uint64_t contrib = w & kValueMask;
-          if (pm != 0) {
-            const int first = __ffs(pm) - 1;
-            if (lane > first) contrib = 0;
-            done = true;
-          }
-          excl += warp_sum_u64(contrib);
-          idx -= 32;
+          idx -= 32 * kLookWindows;
         }
       }
+      const uint64_t excl = warp_sum_u64(mine);
       if (failed) {
         if (lane == 0) {
           store_status(p.status + chunk, kFlagPoison << kFlagShift);   // later chunks stop waiting too
@@ -383,12 +451,12 @@ __global__ void __launch_bounds__(kPipeThreads) store_pipelined_kernel(const Sto
       for (int g = 0; g < kChunk; ++g) {
         const uint32_t tile = chunk * kChunk + g;
         if (tile < ntiles) {
-          const int64_t padded = (int64_t)gran[g] * kValueAlign;
+          const int64_t padded = (int64_t)((cur.tot[g] + kValueAlign - 1) / kValueAlign) * kValueAlign;
           const bool fits = base + padded <= p.capacity;
           over = over || !fits;
           if (lane == 0) {
             if (!failed) p.offsets[tile] = (uint32_t)base;
-            sm.tile_total[slot][g] = tot[g];
+            sm.tile_total[slot][g] = cur.tot[g];
             sm.tile_base[slot][g] = (failed || !fits) ? -1 : base;
           }
           base += padded;
@@ -404,42 +472,9 @@ __global__ void __launch_bounds__(kPipeThreads) store_pipelined_kernel(const Sto
       }
       __syncwarp();
       if (lane == 0) bar_arrive(&sm.base_ready[slot]);
+      chunk = chunk_nxt;
+      cur = nxt;
     }
-  } else {
-    // ---------------------------------------------------------------------------------------------
-    // output: one bulk copy per tile from the staging buffer to `values`
-    // ---------------------------------------------------------------------------------------------
-    uint32_t n = 0;
-    bool ok = true;
-    for (uint32_t seq = 0; ok; ++seq) {
-      const int slot = seq % kSlots;
-      const uint32_t par = (seq / kSlots) & 1u;
-      if (!bar_wait(&sm.chunk_ready[slot], par, abort_flag)) break;
-      const uint32_t chunk = sm.chunk_id[slot];
-      if (chunk == kNoChunk) break;
-      if (!bar_wait(&sm.base_ready[slot], par, abort_flag)) break;
-      for (int g = 0; g < kChunk; ++g) {
-        const uint32_t tile = chunk * kChunk + g;
-        if (tile >= ntiles) break;
-        const int b = n & 1;
-        const uint32_t total = sm.tile_total[slot][g];
-        const int64_t base = sm.tile_base[slot][g];
-        const uint32_t padded = (total + kValueAlign - 1) / kValueAlign * kValueAlign;
-        if (!bar_wait(&sm.staged[b], (n >> 1) & 1u, abort_flag)) { ok = false; break; }
-        if (total + lane < padded) sm.outv[b][total + lane] = from_float<T>(0.0f);
-        fence_async_smem();
-        __syncwarp();
-        if (lane == 0) {
-          if (base >= 0 && padded != 0) {
-            bulk_store(static_cast<T*>(p.values) + base, sm.outv[b], padded * (uint32_t)sizeof(T));
-            bulk_store_wait_read();
-          }
-          bar_arrive(&sm.out_free[b]);
-        }
-        ++n;
-      }
-    }
-    if (lane == 0) bulk_store_wait_all();
   }
   __syncthreads();
   if (tid == 0 && sm.abort_flag != 0) raise_status(p.dev_status, RAD_DEV_ETIMEOUT);
