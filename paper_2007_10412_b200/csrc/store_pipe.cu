@@ -78,12 +78,14 @@ __device__ __forceinline__ uint64_t timer_ns() {
 }
 // Bounded wait; false when the CTA is giving up (this wait or another one ran out of time).  The
 // slow path is kept out of line: it is rarely taken and the kernel's code should stay small.
-__device__ __noinline__ bool bar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __noinline__ bool bar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint32_t sleep_ns) {
   const uint64_t t0 = timer_ns();
   while (true) {
 #pragma unroll 1
-    for (int i = 0; i < 64; ++i)
+    for (int i = 0; i < 64; ++i) {
       if (bar_try_wait(bar, parity)) return true;
+      if (sleep_ns != 0) __nanosleep(sleep_ns);   // a waiting warp leaves the issue slots to the others
+    }
     if (*abort_flag != 0) return false;
     if (timer_ns() - t0 > kPipeWaitLimitNs) {
       *abort_flag = 1;
@@ -91,9 +93,9 @@ __device__ __noinline__ bool bar_wait_slow(uint64_t* bar, uint32_t parity, volat
     }
   }
 }
-__device__ __forceinline__ bool bar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool bar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint32_t sleep_ns = 40) {
   if (bar_try_wait(bar, parity)) return true;
-  return bar_wait_slow(bar, parity, abort_flag);
+  return bar_wait_slow(bar, parity, abort_flag, sleep_ns);
 }
 __device__ __forceinline__ void tma_load_tile(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
   asm volatile(
@@ -335,7 +337,7 @@ __global__ void __launch_bounds__(kPipeThreads, 3) store_pipelined_kernel(const 
           const uint32_t tile = q[0] * kChunk + g;
           if (tile >= ntiles) break;
           const int s = n % S;
-          if (!bar_wait(&sm.empty[s], ((n / S) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          if (!bar_wait(&sm.empty[s], ((n / S) & 1u) ^ 1u, abort_flag, 0)) { ok = false; break; }
           const uint32_t slab = tile / (uint32_t)p.ncb, cb = tile - slab * (uint32_t)p.ncb;
           bar_arrive_expect_tx(&sm.full[s], (uint32_t)(kTileElems * sizeof(T)));
           tma_load_tile(sm.raw[s], &tmA, (int)(cb * kTileCols), (int)(slab * kTileRows), &sm.full[s]);
@@ -364,10 +366,10 @@ __global__ void __launch_bounds__(kPipeThreads, 3) store_pipelined_kernel(const 
     auto publish = [&](uint32_t seq, Counts& c) -> uint32_t {
       const int slot = seq % kSlots;
       const uint32_t par = (seq / kSlots) & 1u;
-      if (!bar_wait(&sm.chunk_ready[slot], par, abort_flag)) return kNoChunk;
+      if (!bar_wait(&sm.chunk_ready[slot], par, abort_flag, 400)) return kNoChunk;
       const uint32_t chunk = sm.chunk_id[slot];
       if (chunk == kNoChunk) return kNoChunk;
-      if (!bar_wait(&sm.cnt_ready[slot], par, abort_flag)) return kNoChunk;
+      if (!bar_wait(&sm.cnt_ready[slot], par, abort_flag, 400)) return kNoChunk;
       // lane (8 g + w) reads warp w's totals of tiles g and g + 4; a butterfly over eight lanes sums a tile
       static_assert(kChunk == 8 && kComputeWarps == 8, "two (tile, warp) entries per lane");
       uint32_t t0 = sm.warp_total[slot][lane >> 3][lane & 7];
