@@ -26,6 +26,10 @@ the estimator is exactly unbiased for the probability actually sampled.  The
 paper leaves the source of randomness open; one byte per decision lets one
 128-bit generator output decide sixteen entries, and the keep probabilities
 the paper uses (0.05 ... 0.5) move by less than 2 % of their value.
+
+Second sampling law, the paper's own (Sec. 3.2, App. A): k = ceil(fraction * d)
+coordinates drawn uniformly WITH replacement, P = (d / k) sum_s e_s e_s^T, so a
+coordinate hit c times is kept with weight c * d / k (`law="replace"`).
 """
 from dataclasses import dataclass, field
 from typing import List, Optional
@@ -37,6 +41,8 @@ from .philox import philox4x32_10
 
 STREAM_DIFFERENT = 0     # counter stream of per-row masks
 STREAM_SAME = 1          # counter stream of masks shared by the minibatch
+STREAM_DIFFERENT_REPLACE = 2   # with-replacement draws, per row
+STREAM_SAME_REPLACE = 3        # with-replacement draws, shared by the minibatch
 LANE_BITS = 8
 LANES_PER_CALL = 16      # 128 output bits / 8
 LANE_RANGE = 1 << LANE_BITS
@@ -120,6 +126,54 @@ def keep_mask_at(variant: str, rows, cols, p, seed: int, layer: int, step: int) 
 
 
 # --------------------------------------------------------------------------
+# the paper's own sampling law (Sec. 3.2: "sampling (with replacement) k out of
+# the d vertices"; App. A: fraction of activations sampled with replacement)
+# --------------------------------------------------------------------------
+def draws_per_row(fraction, D: int) -> int:
+    """k = ceil(fraction * d), at least 1 and at most d.  The fraction arrives as a float32 (0.1 is then
+    a little above one tenth), so the product is taken in float64 and shrunk by 2^-22 before the
+    ceiling: 0.1 * 300 gives 30, not 31."""
+    f32 = float(np.float32(fraction))
+    if not (0.0 < f32 <= 1.0):
+        raise ValueError("fraction must be in (0, 1]")
+    return int(min(max(np.ceil(f32 * D * (1.0 - 2.0 ** -22)), 1.0), float(D)))
+
+
+def replace_scale(fraction, D: int) -> np.float32:
+    """d / k as one float32 division: the weight of a coordinate drawn once."""
+    return np.float32(D) / np.float32(draws_per_row(fraction, D))
+
+
+def multiplicity(variant: str, B: int, D: int, fraction, seed: int, layer: int, step: int) -> np.ndarray:
+    """c[b, d] = how many of the k draws of row b picked column d (B x D, int64).
+
+    Draw j of a row reads 32-bit word j % 4 of the Philox output for counter
+    (j // 4, row, layer | stream << 24, step) and picks column
+    floor(word * D / 2^32).  "same": one set of draws (row field 0) for the whole
+    minibatch.  Every row's multiplicities add up to k.
+    """
+    k = draws_per_row(fraction, D)
+    if variant == "different":
+        rows, stream = np.arange(B, dtype=np.uint64)[:, None], STREAM_DIFFERENT_REPLACE
+    elif variant == "same":
+        rows, stream = np.zeros((1, 1), dtype=np.uint64), STREAM_SAME_REPLACE
+    else:
+        raise ValueError(variant)
+    calls = (k + 3) // 4
+    c0 = np.arange(calls, dtype=np.uint64)[None, :]
+    words = philox4x32_10(c0, rows, np.uint64((layer & 0xFFFFFF) | (stream << 24)), np.uint64(step & 0xFFFFFFFF),
+                          np.uint64(seed & 0xFFFFFFFF), np.uint64((seed >> 32) & 0xFFFFFFFF))
+    draws = np.stack([w.astype(np.uint64) for w in words], axis=-1).reshape(rows.shape[0], calls * 4)[:, :k]
+    cols = (draws * np.uint64(D)) >> np.uint64(32)
+    nrows = cols.shape[0]
+    flat = (np.arange(nrows, dtype=np.uint64)[:, None] * np.uint64(D) + cols).reshape(-1).astype(np.int64)
+    c = np.bincount(flat, minlength=nrows * D).reshape(nrows, D)
+    if variant == "same":
+        c = np.broadcast_to(c, (B, D))
+    return np.ascontiguousarray(c.astype(np.int64))
+
+
+# --------------------------------------------------------------------------
 # number formats
 # --------------------------------------------------------------------------
 def round_bf16(x) -> np.ndarray:
@@ -175,20 +229,33 @@ class Store:
 
 
 def forward_store(A, dtype: str, variant: str, p, seed: int, layer: int, step: int,
-                  mask: Optional[np.ndarray] = None, with_relu_bits: bool = True) -> Store:
+                  mask: Optional[np.ndarray] = None, with_relu_bits: bool = True,
+                  law: str = "bernoulli", counts: Optional[np.ndarray] = None) -> Store:
     """What the forward pass keeps of a layer input A (B x D).
 
     A_hat[b, d] = m[b, d] * round_dtype(fl32(A[b, d] * s)); only the kept
     entries are emitted.  `mask` replaces the Philox mask (test hook for
-    exhaustive enumeration).  The ReLU derivative of the layer that produced A
+    exhaustive enumeration).  law="replace": the paper's k draws with
+    replacement; `T` then holds k and `p` is the fraction.  The ReLU derivative of the layer that produced A
     is (A > 0), one bit per entry (Sec. 4.2; -0.0 and 0.0 give 0).
     """
     A = np.ascontiguousarray(A, dtype=np.float32)
     B, D = A.shape
-    T = keep_threshold(p)
-    s = scale_factor(p)
-    m = keep_mask(variant, B, D, p, seed, layer, step) if mask is None else np.asarray(mask, bool)
-    scaled = A * s                                   # float32 x float32, one rounding
+    if law == "bernoulli":
+        T = keep_threshold(p)
+        s = scale_factor(p)
+        m = keep_mask(variant, B, D, p, seed, layer, step) if mask is None else np.asarray(mask, bool)
+        scaled = A * s                                   # float32 x float32, one rounding
+    elif law == "replace":
+        # `counts` replaces the Philox draws (test hook for exhaustive enumeration).  A coordinate drawn
+        # c times weighs c * d / k: fl32(c * s) first, then one float32 product with the entry.
+        T = draws_per_row(p, D)
+        s = replace_scale(p, D)
+        c = multiplicity(variant, B, D, p, seed, layer, step) if counts is None else np.asarray(counts, np.int64)
+        m = c > 0
+        scaled = A * (c.astype(np.float32) * s)
+    else:
+        raise ValueError(law)
     if dtype == "bf16":
         scaled = round_bf16(scaled)
     elif dtype != "f32":
