@@ -70,6 +70,25 @@ typedef enum { RAD_ACT_NONE = 0, RAD_ACT_RELU = 1, RAD_ACT_GELU = 2 } rad_act;
  * p_eff = T / 256 is the probability actually sampled and kept values are
  * multiplied by fl32(256 / T) = 1 / p_eff, so E[A_hat] = A exactly.
  */
+/*
+ * Second sampling law, the paper's own (Sec. 3.2: "sampling (with replacement) k
+ * out of the d vertices", P = (d / k) sum_s e_s e_s^T; App. A: a fraction of the
+ * activations sampled with replacement).  Per row (different-sample) or once per
+ * layer and step (same-sample), k = ceil(fraction * D) columns are drawn; a column
+ * drawn c > 0 times is kept and its entry is multiplied by fl32(c * fl32(D / k)).
+ *   draw j  = 32-bit word j % 4 of the Philox-4x32-10 output for
+ *             counter (j / 4, row, layer | stream << 24, step), stream = 2
+ *             (different-sample, row = b) or 3 (same-sample, row = 0)
+ *   column  = floor(word * D / 2^32)
+ *   k       = ceil(fraction * D * (1 - 2^-22)) in double, clamped to [1, D]: the
+ *             fraction is a float32, so 0.1 * 300 gives 30 and not 31.
+ * The compact store has the same layout as with the Bernoulli law (a kept entry
+ * carries its weight in its value), so the weight-gradient calls take it as is.
+ */
+typedef enum { RAD_LAW_BERNOULLI = 0, RAD_LAW_REPLACE = 1 } rad_law;
+int64_t rad_draws_per_row(float fraction, int64_t D);   /* k; 0 if the fraction is outside (0, 1] */
+float   rad_replace_scale(float fraction, int64_t D);   /* fl32(D / k)                            */
+
 uint32_t rad_keep_threshold(float p);   /* T; 0 if p is outside (0, 1]                        */
 float    rad_effective_p(float p);      /* T / 256                                            */
 float    rad_scale(float p);            /* fl32(256 / T)                                      */
@@ -115,6 +134,8 @@ typedef struct rad_store {
   uint32_t* offsets;
   int64_t*  nnz;              /* 2 device int64 */
   uint32_t* relubits;         /* or NULL */
+  int32_t   law;              /* rad_law; 0 (Bernoulli keeps) unless set.  RAD_LAW_REPLACE: p is */
+                              /* the fraction of the with-replacement law                         */
 } rad_store;
 
 typedef struct rad_store_sizes {
@@ -129,6 +150,11 @@ typedef struct rad_store_sizes {
 /* Buffer sizes for a store of the given shape (host only, nothing is launched). */
 int rad_store_size_query(int32_t variant, int32_t dtype, int64_t B, int64_t D, float p,
                          rad_store_sizes* out /* host */);
+
+/* The same for a given sampling law (rad_law): capacities follow the number of distinct columns
+ * k draws hit, and the workspace holds the multiplicities (B x D bytes for different-sample). */
+int rad_store_size_query_law(int32_t variant, int32_t dtype, int32_t law, int64_t B, int64_t D, float p,
+                             rad_store_sizes* out /* host */);
 
 /*
  * Forward-pass store of one layer input (Sec. 3.2 "sparsify the input vectors";

@@ -22,6 +22,7 @@ TILE_ROWS, TILE_COLS, VALUE_ALIGN = 64, 128, 8
 
 DTYPES = {"f32": RAD_F32, "bf16": RAD_BF16, torch.float32: RAD_F32, torch.bfloat16: RAD_BF16}
 VARIANTS = {"different": RAD_DIFFERENT_SAMPLE, "same": RAD_SAME_SAMPLE}
+LAWS = {"bernoulli": 0, "replace": 1}
 ACTS = {"none": RAD_ACT_NONE, "relu": RAD_ACT_RELU, "gelu": RAD_ACT_GELU}
 TORCH_DTYPE = {RAD_F32: torch.float32, RAD_BF16: torch.bfloat16}
 
@@ -35,7 +36,7 @@ class rad_store(C.Structure):
                 ("p", C.c_float), ("layer", C.c_uint32), ("step", C.c_uint32), ("seed", C.c_uint64),
                 ("values", C.c_void_p), ("values_capacity", C.c_int64), ("values_ld", C.c_int64),
                 ("keepbits", C.c_void_p), ("offsets", C.c_void_p), ("nnz", C.c_void_p),
-                ("relubits", C.c_void_p)]
+                ("relubits", C.c_void_p), ("law", C.c_int32)]
 
 
 class rad_store_sizes(C.Structure):
@@ -68,6 +69,7 @@ class rad_step_stats(C.Structure):
 
 
 EXPORTS = ["rad_keep_threshold", "rad_effective_p", "rad_scale", "rad_store_size_query", "rad_set_store_kernel",
+           "rad_draws_per_row", "rad_replace_scale", "rad_store_size_query_law",
            "rad_linear_forward_store", "rad_linear_forward_store_static", "rad_weight_grad_workspace", "rad_linear_weight_grad",
            "rad_linear_forward", "rad_softmax_xent", "rad_input_grad_workspace", "rad_linear_input_grad",
            "rad_mlp_workspace", "rad_mlp_step", "rad_irnn_workspace", "rad_irnn_step", "rad_cnn_workspace", "rad_cnn_step", "rad_launch_count", "rad_strerror", "rad_version"]
@@ -94,6 +96,11 @@ def lib():
         L.rad_launch_count.restype = C.c_int64
         i32, i64, f32, vp = C.c_int32, C.c_int64, C.c_float, C.c_void_p
         L.rad_set_store_kernel.argtypes = [i32]
+        L.rad_draws_per_row.restype = i64
+        L.rad_draws_per_row.argtypes = [f32, i64]
+        L.rad_replace_scale.restype = f32
+        L.rad_replace_scale.argtypes = [f32, i64]
+        L.rad_store_size_query_law.argtypes = [i32, i32, i32, i64, i64, f32, C.POINTER(rad_store_sizes)]
         L.rad_store_size_query.argtypes = [i32, i32, i64, i64, f32, C.POINTER(rad_store_sizes)]
         L.rad_linear_forward_store.argtypes = [vp, i64, C.POINTER(rad_store), vp, i64, vp, vp]
         L.rad_linear_forward_store_static.argtypes = [vp, i64, C.POINTER(rad_store), vp, vp]
@@ -164,13 +171,28 @@ def rad_store_size_query(variant, dtype, B, D, p):
     return out
 
 
+def rad_store_size_query_law(variant, dtype, law, B, D, p):
+    out = rad_store_sizes()
+    _check(lib().rad_store_size_query_law(VARIANTS[variant], DTYPES[dtype], LAWS[law], B, D, p, C.byref(out)),
+           "rad_store_size_query_law")
+    return out
+
+
+def rad_draws_per_row(fraction, D):
+    return int(lib().rad_draws_per_row(fraction, D))
+
+
+def rad_replace_scale(fraction, D):
+    return float(lib().rad_replace_scale(fraction, D))
+
+
 class Store:
     """Device buffers of one layer's compact store plus the host struct that describes them."""
 
     def __init__(self, variant, dtype, B, D, p, seed=0, layer=0, step=0, relu_bits=True, capacity="typical",
-                 device="cuda"):
-        self.variant, self.dtype, self.B, self.D, self.p = variant, dtype, B, D, p
-        sz = rad_store_size_query(variant, dtype, B, D, p)
+                 device="cuda", law="bernoulli"):
+        self.variant, self.dtype, self.B, self.D, self.p, self.law = variant, dtype, B, D, p, law
+        sz = rad_store_size_query_law(variant, dtype, law, B, D, p)
         self.sizes = sz
         cap = {"typical": sz.values_typical, "worst": sz.values_worst}.get(capacity, capacity)
         ld = 0
@@ -187,7 +209,7 @@ class Store:
         self.c = rad_store(VARIANTS[variant], DTYPES[dtype], B, D, p, layer, step, seed,
                            self.values.data_ptr(), int(cap), int(ld), self.keepbits.data_ptr(),
                            self.offsets.data_ptr(), self.nnz.data_ptr(),
-                           self.relubits.data_ptr() if relu_bits else None)
+                           self.relubits.data_ptr() if relu_bits else None, LAWS[law])
 
     def held_bytes(self):
         """Bytes this store holds between forward and backward (values as reserved, indices, ReLU bits)."""

@@ -25,6 +25,23 @@ uint32_t keep_threshold_host(float p) {
   return (uint32_t)t;
 }
 
+int64_t draws_per_row_host(float fraction, int64_t D) {
+  if (!(fraction > 0.0f) || !(fraction <= 1.0f) || D <= 0) return 0;
+  double k = ceil((double)fraction * (double)D * (1.0 - ldexp(1.0, -22)));
+  if (k < 1.0) k = 1.0;
+  if (k > (double)D) k = (double)D;
+  return (int64_t)k;
+}
+
+// Expected share of kept entries: p_eff for Bernoulli keeps, 1 - (1 - 1/D)^k for k draws with replacement.
+double store_keep_fraction(const rad_store* st) {
+  if (st->law == RAD_LAW_REPLACE) {
+    const double k = (double)draws_per_row_host(st->p, st->D), D = (double)st->D;
+    return D <= 1.0 ? 1.0 : 1.0 - pow(1.0 - 1.0 / D, k);
+  }
+  return keep_threshold_host(st->p) / (double)kLaneRange;
+}
+
 namespace {
 
 template <typename T> struct Raw8;   // eight consecutive elements of one row
@@ -86,7 +103,9 @@ __device__ __forceinline__ uint32_t transpose4x4_bytes(uint32_t v, int k) {
   return v;
 }
 
-template <typename T>
+// kReplace: keep bits and weights come from the multiplicity matrix (with-replacement law) instead
+// of a Bernoulli draw; everything after the mask is the same.
+template <typename T, bool kReplace>
 __global__ void __launch_bounds__(256) store_different_kernel(const StoreParams p, const PhiloxKeys ks) {
   __shared__ uint32_t s_rowcnt[kTileRows];
   __shared__ uint32_t s_rowoff[kTileRows];
@@ -108,15 +127,26 @@ __global__ void __launch_bounds__(256) store_different_kernel(const StoreParams 
   const T* Abase = static_cast<const T*>(p.A);
 
   Raw8<T> raw[4];
+  uint2 mult[4];                                 // kReplace: the eight multiplicities of an item, a byte each
   uint32_t masks = 0, relus = 0, counts = 0;     // one byte per item: keep bits, ReLU bits, kept count
 #pragma unroll
   for (int it = 0; it < 4; ++it) {
     const int64_t row = slab * kTileRows + warp * 8 + it * 2 + half;
     if (row < p.B && nvalid > 0) {
       load8<T>(Abase + row * p.lda, col0, nvalid, p.vec_ok != 0, raw[it]);
-      // this lane's eight columns are one half of a sixteen-column draw
-      const uint32_t m16 = philox_keep16((uint32_t)(col0 >> 4), (uint32_t)row, p.c2, p.c3, ks, p.T);
-      const uint32_t m = (m16 >> (8 * (cg & 1))) & ((1u << nvalid) - 1u);
+      uint32_t m;
+      if (kReplace) {
+        mult[it] = *reinterpret_cast<const uint2*>(p.counts + row * p.ldc + col0);
+        m = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          m |= ((((i < 4 ? mult[it].x : mult[it].y) >> (8 * (i & 3))) & 0xffu) != 0 ? 1u : 0u) << i;
+        m &= (1u << nvalid) - 1u;
+      } else {
+        // this lane's eight columns are one half of a sixteen-column draw
+        const uint32_t m16 = philox_keep16((uint32_t)(col0 >> 4), (uint32_t)row, p.c2, p.c3, ks, p.T);
+        m = (m16 >> (8 * (cg & 1))) & ((1u << nvalid) - 1u);
+      }
       masks |= m << (8 * it);
       counts |= __popc(m) << (8 * it);
       if (p.relubits != nullptr) relus |= (positive8(raw[it]) & ((1u << nvalid) - 1u)) << (8 * it);
@@ -184,8 +214,14 @@ __global__ void __launch_bounds__(256) store_different_kernel(const StoreParams 
     const uint32_t m = (masks >> (8 * it)) & 0xffu;
     if (m != 0) {
 #pragma unroll
-      for (int i = 0; i < 8; ++i)
-        if ((m >> i) & 1u) s_stage[pos++] = from_float<T>(elem(raw[it], i) * p.scale);
+      for (int i = 0; i < 8; ++i) {
+        if ((m >> i) & 1u) {
+          float w = p.scale;
+          if (kReplace)   // weight of an entry drawn c times: fl32(c * (D / k)), then one product with the entry
+            w = __fmul_rn((float)(((i < 4 ? mult[it].x : mult[it].y) >> (8 * (i & 3))) & 0xffu), p.scale);
+          s_stage[pos++] = from_float<T>(__fmul_rn(elem(raw[it], i), w));
+        }
+      }
     }
   }
   if (tid < (int)(padded - total)) s_stage[total + tid] = from_float<T>(0.0f);
@@ -327,7 +363,7 @@ __global__ void __launch_bounds__(1024) same_mask_kernel(const SameParams p, con
 
 // values[b, j] = A[b, idx[j]] * scale for j < k', zero up to ld.  One warp per row at a time.
 template <typename T>
-__global__ void __launch_bounds__(256) same_gather_kernel(const SameParams p) {
+__global__ void __launch_bounds__(256) same_gather_kernel(const SameParams p, const float* colscale) {
   const int64_t k = min(p.nnz[0], p.ld);
   const int lane = threadIdx.x & 31;
   const int64_t warp0 = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -341,7 +377,7 @@ __global__ void __launch_bounds__(256) same_gather_kernel(const SameParams p) {
       float v = 0.0f;
       if (j < k) {
         const uint32_t col = __ldg(p.idx + j);
-        if (col < (uint32_t)p.D) v = to_float(rowp[col]) * p.scale;
+        if (col < (uint32_t)p.D) v = __fmul_rn(to_float(rowp[col]), colscale != nullptr ? colscale[j] : p.scale);
         else raise_status(p.dev_status, RAD_DEV_EINTERNAL);
       }
       orow[j] = from_float<T>(v);
@@ -365,6 +401,105 @@ __global__ void __launch_bounds__(256) relu_bits_kernel(const T* A, int64_t lda,
   }
 }
 
+// ---- with-replacement law -------------------------------------------------------------------------
+struct ReplaceParams {
+  int64_t B, D, k;
+  uint32_t c2, c3;
+  uint8_t* counts;      // different-sample: B rows of ldc bytes
+  int64_t ldc;
+  int32_t* dev_status;
+};
+
+// One CTA per row: the k draws of the row land in a shared-memory histogram (a byte per column, four to
+// a word), which is then written out as the row of the multiplicity matrix.
+__global__ void __launch_bounds__(128) replace_counts_kernel(const ReplaceParams p, const PhiloxKeys ks) {
+  extern __shared__ uint32_t s_hist[];
+  const int64_t row = blockIdx.x;
+  const int words = (int)(p.ldc / 4);
+  for (int i = threadIdx.x; i < words; i += 128) s_hist[i] = 0;
+  __syncthreads();
+  const int64_t calls = (p.k + 3) / 4;
+  for (int64_t c = threadIdx.x; c < calls; c += 128) {
+    uint32_t w[4];
+    philox4x32_10((uint32_t)c, (uint32_t)row, p.c2, p.c3, ks, w);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (4 * c + j < p.k) {
+        const uint32_t col = __umulhi(w[j], (uint32_t)p.D);
+        const uint32_t old = atomicAdd(&s_hist[col >> 2], 1u << (8 * (col & 3)));
+        if (((old >> (8 * (col & 3))) & 0xffu) == 0xffu) raise_status(p.dev_status, RAD_DEV_EINTERNAL);   // a byte ran over
+      }
+    }
+  }
+  __syncthreads();
+  uint32_t* out = reinterpret_cast<uint32_t*>(p.counts + row * p.ldc);
+  for (int i = threadIdx.x; i < words; i += 128) out[i] = s_hist[i];
+}
+
+struct SameReplaceParams {
+  int64_t D, k;
+  uint32_t c2, c3;
+  float scale;          // D / k
+  uint32_t* hist;       // D words of scratch
+  float* colscale;      // weight of kept column j (D floats of scratch)
+};
+
+// Same-sample: one set of k draws for the layer.  One CTA: histogram in global scratch, then the
+// ascending list of the columns that were hit, their weights and the keep-bit words.
+__global__ void __launch_bounds__(1024) same_replace_mask_kernel(const SameParams p, const SameReplaceParams r,
+                                                                 const PhiloxKeys ks) {
+  __shared__ uint32_t s_warp[32];
+  __shared__ uint32_t s_running;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int64_t i = tid; i < p.D; i += 1024) r.hist[i] = 0;
+  if (tid == 0) s_running = 0;
+  __syncthreads();
+  const int64_t calls = (r.k + 3) / 4;
+  for (int64_t c = tid; c < calls; c += 1024) {
+    uint32_t w[4];
+    philox4x32_10((uint32_t)c, 0u, r.c2, r.c3, ks, w);
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      if (4 * c + j < r.k) atomicAdd(&r.hist[__umulhi(w[j], (uint32_t)p.D)], 1u);
+  }
+  __syncthreads();
+  for (int64_t d0 = 0; d0 < p.D; d0 += 1024) {
+    const int64_t d = d0 + tid;
+    const uint32_t c = d < p.D ? r.hist[d] : 0u;
+    const uint32_t kept = c != 0 ? 1u : 0u;
+    const uint32_t word = __ballot_sync(0xffffffffu, kept != 0);
+    if (lane == 0 && d < p.D) p.keepbits[d >> 5] = word;
+    const uint32_t before = __popc(word & ((1u << lane) - 1u));
+    if (lane == 31) s_warp[warp] = before + kept;
+    __syncthreads();
+    if (warp == 0) {
+      const uint32_t v = s_warp[lane];
+      uint32_t wi = v;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t n = __shfl_up_sync(0xffffffffu, wi, o);
+        if (lane >= o) wi += n;
+      }
+      s_warp[lane] = wi - v;
+    }
+    __syncthreads();
+    const uint32_t pos = s_running + s_warp[warp] + before;
+    if (kept) {
+      p.idx[pos] = (uint32_t)d;
+      r.colscale[pos] = __fmul_rn((float)c, r.scale);
+    }
+    __syncthreads();
+    if (tid == 1023) s_running = pos + kept;   // last thread's end position is the running total
+    __syncthreads();
+  }
+  if (tid == 0) {
+    const int64_t k = s_running;
+    p.nnz[0] = k;
+    p.nnz[1] = k * p.B;
+    if (k > p.ld) raise_status(p.dev_status, RAD_DEV_ECAPACITY);
+  }
+}
+
 constexpr int kPipelinedMinTiles = 2048;
 int g_store_kernel = RAD_STORE_KERNEL_AUTO;
 
@@ -374,24 +509,39 @@ int launch_store_different(const StoreParams& p, const PhiloxKeys& ks, int dtype
   // The pipelined kernel pays off where there are many tiles per SM and most entries are dropped: its
   // per-entry staging loop is slower than the generic kernel's for dense masks, and a CTA works
   // through a chunk of tiles one after the other, which only adds latency to a small problem.
-  const bool pipelined = g_store_kernel == RAD_STORE_KERNEL_PIPELINED ||
+  const bool pipelined = p.counts != nullptr ? false : g_store_kernel == RAD_STORE_KERNEL_PIPELINED ||
                          (g_store_kernel == RAD_STORE_KERNEL_AUTO && p.ntiles >= kPipelinedMinTiles && T <= kLaneRange / 2);
   const int rc = pipelined ? launch_store_pipelined(p, ks, dtype, s) : RAD_EUNSUPPORTED;
   if (rc != RAD_EUNSUPPORTED) return rc;
   count_launch();
-  if (dtype == RAD_BF16)
-    store_different_kernel<bf16><<<p.ntiles, 256, 0, s>>>(p, ks);
-  else
-    store_different_kernel<float><<<p.ntiles, 256, 0, s>>>(p, ks);
+  if (p.counts != nullptr) {
+    if (dtype == RAD_BF16)
+      store_different_kernel<bf16, true><<<p.ntiles, 256, 0, s>>>(p, ks);
+    else
+      store_different_kernel<float, true><<<p.ntiles, 256, 0, s>>>(p, ks);
+  } else if (dtype == RAD_BF16) {
+    store_different_kernel<bf16, false><<<p.ntiles, 256, 0, s>>>(p, ks);
+  } else {
+    store_different_kernel<float, false><<<p.ntiles, 256, 0, s>>>(p, ks);
+  }
   RAD_CUDA_TRY(cudaGetLastError());
   return RAD_OK;
 }
 
-int64_t store_workspace_bytes(int variant, int64_t B, int64_t D) {
-  if (variant == RAD_SAME_SAMPLE) return 256;
+int64_t status_bytes(int64_t B, int64_t D) {
   const int64_t ntiles = ceil_div(B, kTileRows) * ceil_div(D, kTileCols);
   return round_up(ntiles * 8 + 256, 256);
 }
+int64_t counts_ld(int64_t D) { return round_up(D, 16); }
+
+// different-sample: claim counter and look-back status words, then (with-replacement law) the multiplicity
+// matrix; same-sample with replacement: 256 bytes, a histogram word and a weight per column.
+int64_t store_workspace_bytes(int variant, int64_t B, int64_t D, int law = RAD_LAW_BERNOULLI) {
+  if (variant == RAD_SAME_SAMPLE) return law == RAD_LAW_REPLACE ? 256 + round_up(8 * D, 256) : 256;
+  return status_bytes(B, D) + (law == RAD_LAW_REPLACE ? round_up(B * counts_ld(D), 256) : 0);
+}
+
+constexpr int64_t kMaxCountsRowBytes = 200 * 1024;   // a row's histogram has to fit shared memory
 
 }  // namespace
 }  // namespace rad
@@ -413,15 +563,31 @@ extern "C" float rad_scale(float p) {
   return T == 0 ? 0.0f : (float)kLaneRange / (float)T;
 }
 
+extern "C" int64_t rad_draws_per_row(float fraction, int64_t D) { return draws_per_row_host(fraction, D); }
+extern "C" float rad_replace_scale(float fraction, int64_t D) {
+  const int64_t k = draws_per_row_host(fraction, D);
+  return k == 0 ? 0.0f : (float)D / (float)k;
+}
+
 extern "C" int rad_store_size_query(int32_t variant, int32_t dtype, int64_t B, int64_t D, float p,
                                     rad_store_sizes* out) {
+  return rad_store_size_query_law(variant, dtype, RAD_LAW_BERNOULLI, B, D, p, out);
+}
+
+extern "C" int rad_store_size_query_law(int32_t variant, int32_t dtype, int32_t law, int64_t B, int64_t D, float p,
+                                        rad_store_sizes* out) {
   if (out == nullptr || B <= 0 || D <= 0) return RAD_EINVAL;
   if (variant != RAD_DIFFERENT_SAMPLE && variant != RAD_SAME_SAMPLE) return RAD_EINVAL;
   if (dtype != RAD_F32 && dtype != RAD_BF16) return RAD_EINVAL;
+  if (law != RAD_LAW_BERNOULLI && law != RAD_LAW_REPLACE) return RAD_EINVAL;
   const uint32_t T = keep_threshold_host(p);
   if (T == 0) return RAD_EINVAL;
   if ((double)B * (double)D >= 4294967296.0 * 0.75) return RAD_EINVAL;   // 32-bit tile offsets
-  const double pe = T / (double)kLaneRange;
+  rad_store probe = {};
+  probe.law = law; probe.p = p; probe.D = D;
+  // share of kept entries; the count of distinct columns among k draws varies less than a Binomial
+  // of the same mean, so the Binomial band below covers it
+  const double pe = store_keep_fraction(&probe);
   const int64_t w32 = ceil_div(D, 32);
   out->relubits_words = B * w32;
   if (variant == RAD_DIFFERENT_SAMPLE) {
@@ -447,7 +613,7 @@ extern "C" int rad_store_size_query(int32_t variant, int32_t dtype, int64_t B, i
     out->keepbits_words = w32;
     out->offsets_words = D;
   }
-  out->workspace_bytes = store_workspace_bytes(variant, B, D);
+  out->workspace_bytes = store_workspace_bytes(variant, B, D, law);
   return RAD_OK;
 }
 
@@ -461,24 +627,32 @@ extern "C" int rad_linear_forward_store(const void* A, int64_t lda, const rad_st
     return RAD_EINVAL;
   const uint32_t T = keep_threshold_host(st->p);
   if (T == 0) return RAD_EINVAL;
+  if (st->law != RAD_LAW_BERNOULLI && st->law != RAD_LAW_REPLACE) return RAD_EINVAL;
   if ((double)st->B * (double)st->D >= 4294967296.0 * 0.75) return RAD_EINVAL;
   if (((uintptr_t)st->values & 15) != 0) return RAD_EUNSUPPORTED;
+  const bool replace = st->law == RAD_LAW_REPLACE;
+  const int64_t k = replace ? draws_per_row_host(st->p, st->D) : 0;
+  if (replace && st->variant == RAD_DIFFERENT_SAMPLE && counts_ld(st->D) > kMaxCountsRowBytes) return RAD_EUNSUPPORTED;
   int rc = check_device();
   if (rc != RAD_OK) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t esz = st->dtype == RAD_BF16 ? 2 : 4;
   const PhiloxKeys ks = philox_expand_key(st->seed);
   const int64_t w32 = ceil_div(st->D, 32);
+  // Bernoulli: 1 / p_eff; with replacement: D / k, the weight of a column drawn once
+  const float scale = replace ? (float)st->D / (float)k : (float)kLaneRange / (float)T;
+  const int64_t need = store_workspace_bytes(st->variant, st->B, st->D, st->law);
+  if (need > 256 || st->variant == RAD_DIFFERENT_SAMPLE) {
+    if (workspace == nullptr || workspace_bytes < need) return RAD_EWORKSPACE;
+    if (((uintptr_t)workspace & 15) != 0) return RAD_EINVAL;
+  }
 
   if (st->variant == RAD_DIFFERENT_SAMPLE) {
-    const int64_t need = store_workspace_bytes(st->variant, st->B, st->D);
-    if (workspace == nullptr || workspace_bytes < need) return RAD_EWORKSPACE;
-    if (((uintptr_t)workspace & 7) != 0) return RAD_EINVAL;
     StoreParams p;
     p.A = A; p.lda = lda; p.B = st->B; p.D = st->D;
     p.ncb = (int32_t)ceil_div(st->D, kTileCols);
     p.ntiles = (int32_t)(ceil_div(st->B, kTileRows) * p.ncb);
-    p.T = make_keep_threshold(T); p.scale = (float)kLaneRange / (float)T;
+    p.T = make_keep_threshold(T); p.scale = scale;
     p.c2 = counter_word2(st->layer, RAD_DIFFERENT_SAMPLE); p.c3 = st->step;
     p.values = st->values; p.capacity = st->values_capacity;
     p.keepbits = st->keepbits; p.offsets = st->offsets; p.nnz = st->nnz;
@@ -487,24 +661,54 @@ extern "C" int rad_linear_forward_store(const void* A, int64_t lda, const rad_st
     p.status = reinterpret_cast<uint64_t*>(static_cast<char*>(workspace) + 256);
     p.dev_status = dev_status;
     p.vec_ok = (((uintptr_t)A & 15) == 0 && (lda * esz) % 16 == 0) ? 1 : 0;
-    RAD_CUDA_TRY(cudaMemsetAsync(workspace, 0, (size_t)need, s));
+    p.counts = nullptr; p.ldc = 0;
+    RAD_CUDA_TRY(cudaMemsetAsync(workspace, 0, (size_t)status_bytes(st->B, st->D), s));
+    if (replace) {
+      // first the multiplicities of every row, then the generic kernel with the mask and the weights
+      // taken from them
+      ReplaceParams rp;
+      rp.B = st->B; rp.D = st->D; rp.k = k;
+      rp.c2 = counter_word2(st->layer, RAD_DIFFERENT_SAMPLE, RAD_LAW_REPLACE); rp.c3 = st->step;
+      rp.counts = reinterpret_cast<uint8_t*>(static_cast<char*>(workspace) + status_bytes(st->B, st->D));
+      rp.ldc = counts_ld(st->D);
+      rp.dev_status = dev_status;
+      if (rp.ldc > 48 * 1024)
+        RAD_CUDA_TRY(cudaFuncSetAttribute(replace_counts_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)kMaxCountsRowBytes));
+      count_launch();
+      replace_counts_kernel<<<(unsigned)st->B, 128, (size_t)rp.ldc, s>>>(rp, ks);
+      RAD_CUDA_TRY(cudaGetLastError());
+      p.counts = rp.counts; p.ldc = rp.ldc;
+    }
     return launch_store_different(p, ks, st->dtype, T, s);
   }
 
   if (st->values_ld <= 0 || st->values_ld % 8 != 0 || st->values_capacity < st->B * st->values_ld)
     return RAD_EINVAL;
   SameParams p;
-  p.A = A; p.lda = lda; p.B = st->B; p.D = st->D; p.T = make_keep_threshold(T); p.scale = (float)kLaneRange / (float)T;
+  p.A = A; p.lda = lda; p.B = st->B; p.D = st->D; p.T = make_keep_threshold(T); p.scale = scale;
   p.c2 = counter_word2(st->layer, RAD_SAME_SAMPLE); p.c3 = st->step;
   p.values = st->values; p.ld = st->values_ld; p.keepbits = st->keepbits; p.idx = st->offsets;
   p.nnz = st->nnz; p.dev_status = dev_status;
+  const float* colscale = nullptr;
   count_launch(2);
-  same_mask_kernel<<<1, 1024, 0, s>>>(p, ks);
+  if (replace) {
+    SameReplaceParams r;
+    r.D = st->D; r.k = k;
+    r.c2 = counter_word2(st->layer, RAD_SAME_SAMPLE, RAD_LAW_REPLACE); r.c3 = st->step;
+    r.scale = scale;
+    r.hist = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + 256);
+    r.colscale = reinterpret_cast<float*>(static_cast<char*>(workspace) + 256 + 4 * st->D);
+    colscale = r.colscale;
+    same_replace_mask_kernel<<<1, 1024, 0, s>>>(p, r, ks);
+  } else {
+    same_mask_kernel<<<1, 1024, 0, s>>>(p, ks);
+  }
   const int grid = (int)std::min<int64_t>(ceil_div(st->B, 8), 148 * 8);
   if (st->dtype == RAD_BF16)
-    same_gather_kernel<bf16><<<grid, 256, 0, s>>>(p);
+    same_gather_kernel<bf16><<<grid, 256, 0, s>>>(p, colscale);
   else
-    same_gather_kernel<float><<<grid, 256, 0, s>>>(p);
+    same_gather_kernel<float><<<grid, 256, 0, s>>>(p, colscale);
   if (st->relubits != nullptr) {
     const int64_t n = st->B * w32;
     const int g2 = (int)std::min<int64_t>(ceil_div(n, 256), 148 * 16);
@@ -546,7 +750,7 @@ extern "C" int rad_linear_forward_store_static(const void* A, int64_t lda, const
                                                int32_t* dev_status, void* stream) {
   if (A == nullptr || st == nullptr) return RAD_EINVAL;
   if (st->B <= 0 || st->D <= 0 || lda < st->D) return RAD_EINVAL;
-  if (st->variant != RAD_DIFFERENT_SAMPLE) return RAD_EUNSUPPORTED;
+  if (st->variant != RAD_DIFFERENT_SAMPLE || st->law != RAD_LAW_BERNOULLI) return RAD_EUNSUPPORTED;
   if (st->dtype != RAD_F32 && st->dtype != RAD_BF16) return RAD_EINVAL;
   if (st->values == nullptr || st->keepbits == nullptr || st->offsets == nullptr || st->nnz == nullptr)
     return RAD_EINVAL;
@@ -577,6 +781,7 @@ extern "C" int rad_linear_forward_store_static(const void* A, int64_t lda, const
   p.status = reinterpret_cast<uint64_t*>(static_cast<char*>(scratch) + 256);
   p.dev_status = dev_status;
   p.vec_ok = (((uintptr_t)A & 15) == 0 && (lda * esz) % 16 == 0) ? 1 : 0;
+  p.counts = nullptr; p.ldc = 0;
   // the array keeps what the last call left: the counter and this call's status words start at zero
   RAD_CUDA_TRY(cudaMemsetAsync(scratch, 0, 256 + 8 * (size_t)ntiles, s));
   return launch_store_different(p, ks, st->dtype, T, s);

@@ -49,6 +49,10 @@ struct StoreParams {
   uint32_t* ticket;   // zeroed before launch
   int32_t* dev_status;
   int32_t vec_ok;     // rows are 16-byte aligned: 8-element vector loads allowed
+  // with-replacement law: multiplicities, one byte per entry, rows of ldc bytes (ldc a multiple of 16);
+  // nullptr: Bernoulli keeps drawn in the kernel
+  const uint8_t* counts;
+  int64_t ldc;
 };
 
 // store_pipe.cu: the persistent TMA-fed kernel.  RAD_EUNSUPPORTED (nothing enqueued) when the input does not

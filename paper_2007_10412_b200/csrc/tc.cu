@@ -958,7 +958,7 @@ DwPlan plan_dw(const rad_store* st, int64_t H) {
   const int64_t kblocks = ceil_div(st->B, BK);
   int64_t m_expect;
   if (st->variant == RAD_SAME_SAMPLE) {
-    m_expect = std::max<int64_t>(1, (int64_t)std::llround((double)st->D * keep_threshold_host(st->p) / (double)kLaneRange));
+    m_expect = std::max<int64_t>(1, (int64_t)std::llround((double)st->D * store_keep_fraction(st)));
     d.partial_rows = round_up(std::min(st->values_ld, round_up(st->D, 8)), BM);
     d.comp_cap = 0;
     d.stages = 3;
@@ -967,7 +967,7 @@ DwPlan plan_dw(const rad_store* st, int64_t H) {
     m_expect = st->D;
     d.partial_rows = round_up(st->D, BM);
     // per-tile value staging: mean + 8 sigma of Binomial(8192, p_eff), padded, in bytes
-    const double pe = keep_threshold_host(st->p) / (double)kLaneRange, n = (double)kTileRows * kTileCols;
+    const double pe = store_keep_fraction(st), n = (double)kTileRows * kTileCols;
     int64_t cap = (int64_t)(n * pe + 8.0 * std::sqrt(n * pe * (1.0 - pe)) + 16.0);
     cap = std::min<int64_t>(round_up(cap, 8), (int64_t)n) * 2;
     d.comp_cap = (int)round_up(cap, 128);
