@@ -199,9 +199,10 @@ int rad_set_store_kernel(int32_t which);
  * (about 1 MiB), held by every GPU that has loaded the library until the
  * process exits.  The call itself allocates nothing and frees nothing.
  *
- *   - different-sample stores only (the same-sample path of
- *     rad_linear_forward_store needs no scratch; pass it a NULL workspace);
- *     RAD_EUNSUPPORTED otherwise.
+ *   - different-sample stores with Bernoulli keeps only (the same-sample path
+ *     of rad_linear_forward_store needs no scratch; pass it a NULL workspace;
+ *     the with-replacement law needs a B x D byte matrix, far beyond a fixed
+ *     array); RAD_EUNSUPPORTED otherwise.
  *   - ceil(B / 64) * ceil(D / 128) must not exceed RAD_STATIC_STORE_MAX_TILES,
  *     else RAD_ELIMIT and nothing is enqueued.
  *   - The first call on a device looks up the array's device address (with
@@ -288,6 +289,7 @@ typedef struct rad_mlp_desc {
   float    p;
   uint32_t step;
   uint64_t seed;
+  int32_t  law;               /* rad_law of every layer's store; 0 = Bernoulli keeps */
 } rad_mlp_desc;
 
 typedef struct rad_step_stats {   /* bytes held between forward and backward (App. A accounting) */

@@ -358,7 +358,7 @@ class StepResult:
 
 
 def mlp_step(X, labels, Ws, bs, act="relu", dtype="f32", variant=None, p=1.0, seed=0, step=0,
-             masks=None) -> StepResult:
+             masks=None, law="bernoulli") -> StepResult:
     """One forward + backward pass of a fully connected net with softmax cross-entropy.
 
     variant None: exact backprop (dW_l = A_{l-1}^T dZ_l).  Otherwise the input
@@ -384,7 +384,7 @@ def mlp_step(X, labels, Ws, bs, act="relu", dtype="f32", variant=None, p=1.0, se
     for l in range(L):
         if variant is not None:
             stores.append(forward_store(A[l].astype(np.float32), dtype, variant, p, seed, l, step,
-                                        mask=None if masks is None else masks[l]))
+                                        mask=None if masks is None else masks[l], law=law))
         else:
             stores.append(None)
         z = A[l] @ W64[l] + b64[l]

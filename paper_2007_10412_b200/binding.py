@@ -48,7 +48,7 @@ class rad_store_sizes(C.Structure):
 class rad_mlp_desc(C.Structure):
     _fields_ = [("L", C.c_int32), ("act", C.c_int32), ("dtype", C.c_int32), ("variant", C.c_int32),
                 ("dims", C.POINTER(C.c_int64)), ("B", C.c_int64), ("p", C.c_float), ("step", C.c_uint32),
-                ("seed", C.c_uint64)]
+                ("seed", C.c_uint64), ("law", C.c_int32)]
 
 
 class rad_irnn_desc(C.Structure):
@@ -303,10 +303,10 @@ def rad_linear_input_grad(dZ, W, relubits_prev=None, z_prev=None, dZ_prev=None, 
                                        _ptr(dev_status), _stream()), "rad_linear_input_grad")
 
 
-def rad_mlp_workspace(dims, B, dtype="f32", act="relu", variant="different", p=0.1):
+def rad_mlp_workspace(dims, B, dtype="f32", act="relu", variant="different", p=0.1, law="bernoulli"):
     """(workspace bytes, rad_step_stats) of a net shape; allocates nothing."""
     dims_c = (C.c_int64 * len(dims))(*dims)
-    desc = rad_mlp_desc(len(dims) - 1, ACTS[act], DTYPES[dtype], VARIANTS[variant], dims_c, B, p, 0, 0)
+    desc = rad_mlp_desc(len(dims) - 1, ACTS[act], DTYPES[dtype], VARIANTS[variant], dims_c, B, p, 0, 0, LAWS[law])
     nbytes, stats = C.c_int64(0), rad_step_stats()
     _check(lib().rad_mlp_workspace(C.byref(desc), C.byref(nbytes), C.byref(stats)), "rad_mlp_workspace")
     return nbytes.value, stats
@@ -315,10 +315,12 @@ def rad_mlp_workspace(dims, B, dtype="f32", act="relu", variant="different", p=0
 class MLPStep:
     """Owns the workspace and pointer tables of rad_mlp_step for one net shape."""
 
-    def __init__(self, dims, B, dtype="f32", act="relu", variant="different", p=0.1, device="cuda"):
+    def __init__(self, dims, B, dtype="f32", act="relu", variant="different", p=0.1, device="cuda",
+                 law="bernoulli"):
         self.dims, self.B, self.L = list(dims), B, len(dims) - 1
         self._dims = (C.c_int64 * len(dims))(*dims)
-        self.desc = rad_mlp_desc(self.L, ACTS[act], DTYPES[dtype], VARIANTS[variant], self._dims, B, p, 0, 0)
+        self.desc = rad_mlp_desc(self.L, ACTS[act], DTYPES[dtype], VARIANTS[variant], self._dims, B, p, 0, 0,
+                                 LAWS[law])
         nbytes = C.c_int64(0)
         self.stats = rad_step_stats()
         _check(lib().rad_mlp_workspace(C.byref(self.desc), C.byref(nbytes), C.byref(self.stats)),

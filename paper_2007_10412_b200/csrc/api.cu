@@ -53,6 +53,7 @@ int make_plan(const rad_mlp_desc* net, StepPlan* plan) {
   if (net->variant != RAD_DIFFERENT_SAMPLE && net->variant != RAD_SAME_SAMPLE) return RAD_EINVAL;
   if (net->act != RAD_ACT_RELU && net->act != RAD_ACT_GELU) return RAD_EINVAL;
   if (keep_threshold_host(net->p) == 0) return RAD_EINVAL;
+  if (net->law != RAD_LAW_BERNOULLI && net->law != RAD_LAW_REPLACE) return RAD_EINVAL;
   const int64_t B = net->B, es = esize(net->dtype);
   int64_t off = 0;
   auto take = [&](int64_t bytes) { const int64_t at = off; off += round_up(bytes, 256); return at; };
@@ -62,7 +63,7 @@ int make_plan(const rad_mlp_desc* net, StepPlan* plan) {
     const int64_t D = net->dims[l], H = net->dims[l + 1];
     if (D <= 0 || H <= 0) return RAD_EINVAL;
     rad_store_sizes sz;
-    int rc = rad_store_size_query(net->variant, net->dtype, B, D, net->p, &sz);
+    int rc = rad_store_size_query_law(net->variant, net->dtype, net->law, B, D, net->p, &sz);
     if (rc != RAD_OK) return rc;
     LayerPlan& lp = plan->layer[l];
     lp.capacity = sz.values_typical;
@@ -84,6 +85,7 @@ int make_plan(const rad_mlp_desc* net, StepPlan* plan) {
     scratch = max(scratch, column_sums_workspace(B, H));
     rad_store tmp = {};
     tmp.variant = net->variant; tmp.dtype = net->dtype; tmp.B = B; tmp.D = D; tmp.p = net->p;
+    tmp.law = net->law;
     tmp.values_ld = lp.values_ld; tmp.values_capacity = lp.capacity;
     scratch = max(scratch, tc_weight_grad_workspace(&tmp, H));
   }
@@ -227,7 +229,7 @@ extern "C" int rad_mlp_step(const rad_mlp_desc* net, const void* X, const int32_
   char* ws = static_cast<char*>(workspace);
   const int L = net->L;
   const int64_t B = net->B;
-  rad_store st[64];
+  rad_store st[64] = {};
   const void* a_in = X;
   int64_t ld_in = net->dims[0];
   for (int l = 0; l < L; ++l) {
@@ -236,7 +238,7 @@ extern "C" int rad_mlp_step(const rad_mlp_desc* net, const void* X, const int32_
     const LayerPlan& lp = plan.layer[l];
     rad_store& s = st[l];
     s.variant = net->variant; s.dtype = net->dtype; s.B = B; s.D = D; s.p = net->p;
-    s.layer = (uint32_t)l; s.step = net->step; s.seed = net->seed;
+    s.layer = (uint32_t)l; s.step = net->step; s.seed = net->seed; s.law = net->law;
     s.values = ws + lp.values; s.values_capacity = lp.capacity; s.values_ld = lp.values_ld;
     s.keepbits = reinterpret_cast<uint32_t*>(ws + lp.keepbits);
     s.offsets = reinterpret_cast<uint32_t*>(ws + lp.offsets);

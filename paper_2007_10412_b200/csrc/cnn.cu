@@ -135,7 +135,7 @@ extern "C" int rad_cnn_step(const rad_cnn_desc* d, const void* X, const int32_t*
   char* ws = static_cast<char*>(workspace);
   const int64_t B = d->B;
   const int nl = pl.nc + pl.nf;
-  rad_store st[2 * kMaxLayers];
+  rad_store st[2 * kMaxLayers] = {};
   auto make_store = [&](int idx, int64_t D) {
     rad_store& q = st[idx];
     q.variant = d->variant; q.dtype = d->dtype; q.B = B; q.D = D; q.p = d->p;

@@ -11,11 +11,11 @@ from gpu_util import TOL, rel_err, to_dev, to_host_f32
 pytestmark = pytest.mark.gpu
 
 
-def _run(cfg, variant, p, seed, act=None, step=0):
+def _run(cfg, variant, p, seed, act=None, step=0, law="bernoulli"):
     import paper_2007_10412_b200 as rad
     act = act or cfg.act
     X, y, Ws, bs = mlp_inputs(cfg.dims, cfg.batch, cfg.dtype, cfg.x_dist, cfg.data_seed, bias_zero=False)
-    ctx = rad.MLPStep(cfg.dims, cfg.batch, cfg.dtype, act, variant, p)
+    ctx = rad.MLPStep(cfg.dims, cfg.batch, cfg.dtype, act, variant, p, law=law)
     dX = to_dev(X, cfg.dtype)
     dy = torch.from_numpy(y).cuda()
     dWs = [to_dev(W, cfg.dtype) for W in Ws]
@@ -23,8 +23,25 @@ def _run(cfg, variant, p, seed, act=None, step=0):
     ctx(dX, dy, dWs, dbs, seed=seed, step=step)
     torch.cuda.synchronize()
     assert ctx.dev_status.item() == 0
-    ref = orc.mlp_step(X, y, Ws, bs, act=act, dtype=cfg.dtype, variant=variant, p=p, seed=seed, step=step)
+    ref = orc.mlp_step(X, y, Ws, bs, act=act, dtype=cfg.dtype, variant=variant, p=p, seed=seed, step=step, law=law)
     return ctx, ref, (X, y, Ws, bs)
+
+
+@pytest.mark.parametrize("name,variant", [("mlp_small_different", "different"), ("mlp_small_same", "same"),
+                                          ("mlp_wide_cut", "different"), ("mlp_wide_cut", "same")])
+def test_step_with_the_with_replacement_law_matches_oracle(name, variant):
+    """The whole step with the paper's own sampling law (k = ceil(0.1 d) draws with replacement per layer
+    input): loss and bias gradients as in exact backprop, weight gradients from the stores."""
+    cfg = get_config(name)
+    ctx, ref, _ = _run(cfg, variant, 0.1, seed=3, step=2, law="replace")
+    tol = TOL[cfg.dtype]
+    assert abs(ctx.loss.item() - ref.loss) <= (1e-5 if cfg.dtype == "f32" else 2e-3) * abs(ref.loss)
+    nnz = ctx.nnz.cpu().numpy().reshape(-1, 2)
+    for l in range(len(cfg.dims) - 1):
+        assert nnz[l, 0] == (ref.stores[l].nnz if variant == "different" else ref.stores[l].idx.size)
+        for got, want in ((ctx.dW[l], ref.dW[l]), (ctx.db[l], ref.db[l])):
+            fro, mx = rel_err(to_host_f32(got), want)
+            assert fro <= tol and mx <= tol, (l, fro, mx)
 
 
 @pytest.mark.parametrize("name,variant", [("mlp_small_different", "different"), ("mlp_small_same", "same"),
