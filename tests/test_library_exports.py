@@ -3,6 +3,7 @@ import ctypes
 import os
 import re
 
+import numpy as np
 import pytest
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
@@ -53,3 +54,23 @@ def test_host_only_entry_points():
     with pytest.raises(b.RadError):
         b.rad_store_size_query("same", "f32", 150, 784, 0.0)
     assert b.lib().rad_strerror(-4).decode() == "workspace too small"
+
+
+def test_host_only_entry_points_of_the_with_replacement_law_and_the_kernel_choice():
+    from oracle import rad as orc
+    from paper_2007_10412_b200 import binding as b
+    for f, D in [(0.1, 784), (0.1, 300), (0.5, 3), (1.0, 7), (0.05, 8192), (1e-9, 50), (0.3333, 1000)]:
+        assert b.rad_draws_per_row(f, D) == orc.draws_per_row(f, D)
+        assert np.float32(b.rad_replace_scale(f, D)) == orc.replace_scale(f, D)
+    assert b.rad_draws_per_row(0.0, 10) == 0 and b.rad_draws_per_row(1.5, 10) == 0
+    # the workspace of a different-sample store with this law holds a byte per entry on top of the status words
+    plain = b.rad_store_size_query_law("different", "bf16", "bernoulli", 1000, 1160, 0.1)
+    repl = b.rad_store_size_query_law("different", "bf16", "replace", 1000, 1160, 0.1)
+    assert repl.workspace_bytes >= plain.workspace_bytes + 1000 * 1168
+    k = orc.draws_per_row(0.1, 1160)
+    mean = 1000 * 1160 * (1 - (1 - 1 / 1160) ** k)
+    assert mean < repl.values_typical < 1.1 * mean + 16 * 10 * 7 + 2000
+    assert b.rad_set_store_kernel("generic") == "auto"
+    assert b.rad_set_store_kernel("pipelined") == "generic"
+    assert b.rad_set_store_kernel("auto") == "pipelined"
+    assert b.lib().rad_set_store_kernel(7) == -1
