@@ -30,6 +30,11 @@ the paper uses (0.05 ... 0.5) move by less than 2 % of their value.
 Second sampling law, the paper's own (Sec. 3.2, App. A): k = ceil(fraction * d)
 coordinates drawn uniformly WITH replacement, P = (d / k) sum_s e_s e_s^T, so a
 coordinate hit c times is kept with weight c * d / k (`law="replace"`).
+
+Third law (App. A, caption of the fraction sweep: the method "could be modified
+to sample without replacement", and fraction 1.0 is then the exact gradient):
+a uniformly random subset of exactly k = ceil(fraction * d) coordinates, each
+kept with weight d / k (`law="fixed"`).
 """
 from dataclasses import dataclass, field
 from typing import List, Optional
@@ -43,6 +48,8 @@ STREAM_DIFFERENT = 0     # counter stream of per-row masks
 STREAM_SAME = 1          # counter stream of masks shared by the minibatch
 STREAM_DIFFERENT_REPLACE = 2   # with-replacement draws, per row
 STREAM_SAME_REPLACE = 3        # with-replacement draws, shared by the minibatch
+STREAM_DIFFERENT_FIXED = 4     # k distinct columns, per row
+STREAM_SAME_FIXED = 5          # k distinct columns, shared by the minibatch
 LANE_BITS = 8
 LANES_PER_CALL = 16      # 128 output bits / 8
 LANE_RANGE = 1 << LANE_BITS
@@ -174,6 +181,55 @@ def multiplicity(variant: str, B: int, D: int, fraction, seed: int, layer: int, 
 
 
 # --------------------------------------------------------------------------
+# exactly k distinct coordinates, without replacement (App. A, remark under the
+# fraction sweep)
+# --------------------------------------------------------------------------
+def floyd_subset(ts, D: int) -> np.ndarray:
+    """Floyd's subset sampling, vectorised over rows.  ts[:, i] is the i-th draw, an integer in
+    [0, D - k + i]; step i adds ts[:, i] to the subset unless it is already in, in which case it adds
+    D - k + i (never in before).  If every ts[:, i] is uniform on its range, every k-subset of
+    {0, ..., D-1} is equally likely.  Returns the indicator (rows x D, bool)."""
+    ts = np.asarray(ts, dtype=np.int64)
+    rows, k = ts.shape
+    chosen = np.zeros((rows, D), dtype=bool)
+    r = np.arange(rows)
+    for i in range(k):
+        j = D - k + i
+        t = ts[:, i]
+        if (t < 0).any() or (t > j).any():
+            raise ValueError("draw out of range")
+        pick = np.where(chosen[r, t], j, t)
+        chosen[r, pick] = True
+    return chosen
+
+
+def fixed_subset(variant: str, B: int, D: int, fraction, seed: int, layer: int, step: int) -> np.ndarray:
+    """Indicator (B x D, int64, k ones per row) of the k columns a row keeps.
+
+    Draw i of a row reads 32-bit word i % 4 of the Philox output for counter
+    (i // 4, row, layer | stream << 24, step) and becomes floor(word * (D - k + i + 1) / 2^32), the i-th
+    draw of floyd_subset.  "same": one subset (row field 0) for the whole minibatch.
+    """
+    k = draws_per_row(fraction, D)
+    if variant == "different":
+        rows, stream = np.arange(B, dtype=np.uint64)[:, None], STREAM_DIFFERENT_FIXED
+    elif variant == "same":
+        rows, stream = np.zeros((1, 1), dtype=np.uint64), STREAM_SAME_FIXED
+    else:
+        raise ValueError(variant)
+    calls = (k + 3) // 4
+    c0 = np.arange(calls, dtype=np.uint64)[None, :]
+    words = philox4x32_10(c0, rows, np.uint64((layer & 0xFFFFFF) | (stream << 24)), np.uint64(step & 0xFFFFFFFF),
+                          np.uint64(seed & 0xFFFFFFFF), np.uint64((seed >> 32) & 0xFFFFFFFF))
+    draws = np.stack([w.astype(np.uint64) for w in words], axis=-1).reshape(rows.shape[0], calls * 4)[:, :k]
+    span = (np.uint64(D - k + 1) + np.arange(k, dtype=np.uint64))[None, :]
+    chosen = floyd_subset(((draws * span) >> np.uint64(32)).astype(np.int64), D).astype(np.int64)
+    if variant == "same":
+        chosen = np.broadcast_to(chosen, (B, D))
+    return np.ascontiguousarray(chosen)
+
+
+# --------------------------------------------------------------------------
 # number formats
 # --------------------------------------------------------------------------
 def round_bf16(x) -> np.ndarray:
@@ -252,6 +308,13 @@ def forward_store(A, dtype: str, variant: str, p, seed: int, layer: int, step: i
         T = draws_per_row(p, D)
         s = replace_scale(p, D)
         c = multiplicity(variant, B, D, p, seed, layer, step) if counts is None else np.asarray(counts, np.int64)
+        m = c > 0
+        scaled = A * (c.astype(np.float32) * s)
+    elif law == "fixed":
+        # exactly k distinct coordinates per row, weight d / k each; `counts` replaces the Philox subset
+        T = draws_per_row(p, D)
+        s = replace_scale(p, D)
+        c = fixed_subset(variant, B, D, p, seed, layer, step) if counts is None else np.asarray(counts, np.int64)
         m = c > 0
         scaled = A * (c.astype(np.float32) * s)
     else:
