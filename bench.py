@@ -276,11 +276,11 @@ def kernel_sweep(rad, torch, A, dZ, H, ps):
                              dW_ms=round(ms_dw, 4), dW_tflops=round(flops / ms_dw / 1e9, 1), dW_flops=kind,
                              nnz=int(nnz[0])))
             del st, ws
-    # the paper's own law (k = ceil(fraction D) draws with replacement): multiplicity kernel + store, then
-    # the same weight-gradient kernels on the store it leaves
-    for variant in ("different", "same"):
+    # the paper's own law (k = ceil(fraction D) draws with replacement) and the fixed-count law without
+    # replacement: multiplicity kernel + store, then the same weight-gradient kernels on the store it leaves
+    for law, variant in (("replace", "different"), ("replace", "same"), ("fixed", "different"), ("fixed", "same")):
         p = 0.1
-        st = rad.Store(variant, "bf16", B, D, p, relu_bits=False, law="replace")
+        st = rad.Store(variant, "bf16", B, D, p, relu_bits=False, law=law)
         ms_store = timed(lambda: rad.rad_linear_forward_store(A, st, status))
         nnz = st.nnz.cpu().numpy()
         ws = torch.empty(max(rad.rad_weight_grad_workspace(st, H), 256), dtype=torch.uint8, device="cuda")
@@ -292,7 +292,7 @@ def kernel_sweep(rad, torch, A, dZ, H, ps):
         else:
             store_bytes = B * D * 2 + int(nnz[1]) * 2 + 4 * int(nnz[0])
             flops, kind = 2.0 * B * int(nnz[0]) * H, "kept-columns"
-        rows.append(dict(variant=variant, law="replace", p=p, draws_per_row=rad.rad_draws_per_row(p, D),
+        rows.append(dict(variant=variant, law=law, p=p, draws_per_row=rad.rad_draws_per_row(p, D),
                          store_ms=round(ms_store, 4), store_gbs=round(store_bytes / ms_store / 1e6, 1),
                          dW_ms=round(ms_dw, 4), dW_tflops=round(flops / ms_dw / 1e9, 1), dW_flops=kind,
                          nnz=int(nnz[0])))

@@ -84,8 +84,16 @@ typedef enum { RAD_ACT_NONE = 0, RAD_ACT_RELU = 1, RAD_ACT_GELU = 2 } rad_act;
  *             fraction is a float32, so 0.1 * 300 gives 30 and not 31.
  * The compact store has the same layout as with the Bernoulli law (a kept entry
  * carries its weight in its value), so the weight-gradient calls take it as is.
+ *
+ * Third law (App. A, remark under the fraction sweep: sampling without
+ * replacement makes a fraction of 1.0 the exact gradient): a uniformly random
+ * subset of exactly k columns, each kept with weight fl32(D / k), drawn by
+ * Floyd's subset sampling: step i = 0 .. k-1 takes t = floor(word_i * (D - k + i
+ * + 1) / 2^32) and adds t to the subset unless it is already in, in which case
+ * it adds D - k + i; word_i as for the with-replacement law with streams 4
+ * (different-sample) and 5 (same-sample).
  */
-typedef enum { RAD_LAW_BERNOULLI = 0, RAD_LAW_REPLACE = 1 } rad_law;
+typedef enum { RAD_LAW_BERNOULLI = 0, RAD_LAW_REPLACE = 1, RAD_LAW_FIXED = 2 } rad_law;
 int64_t rad_draws_per_row(float fraction, int64_t D);   /* k; 0 if the fraction is outside (0, 1] */
 float   rad_replace_scale(float fraction, int64_t D);   /* fl32(D / k)                            */
 
@@ -134,8 +142,8 @@ typedef struct rad_store {
   uint32_t* offsets;
   int64_t*  nnz;              /* 2 device int64 */
   uint32_t* relubits;         /* or NULL */
-  int32_t   law;              /* rad_law; 0 (Bernoulli keeps) unless set.  RAD_LAW_REPLACE: p is */
-                              /* the fraction of the with-replacement law                         */
+  int32_t   law;              /* rad_law; 0 (Bernoulli keeps) unless set.  For the other two laws */
+                              /* p is the fraction: k = ceil(p * D) draws or kept columns          */
 } rad_store;
 
 typedef struct rad_store_sizes {

@@ -22,7 +22,7 @@ TILE_ROWS, TILE_COLS, VALUE_ALIGN = 64, 128, 8
 
 DTYPES = {"f32": RAD_F32, "bf16": RAD_BF16, torch.float32: RAD_F32, torch.bfloat16: RAD_BF16}
 VARIANTS = {"different": RAD_DIFFERENT_SAMPLE, "same": RAD_SAME_SAMPLE}
-LAWS = {"bernoulli": 0, "replace": 1}
+LAWS = {"bernoulli": 0, "replace": 1, "fixed": 2}
 ACTS = {"none": RAD_ACT_NONE, "relu": RAD_ACT_RELU, "gelu": RAD_ACT_GELU}
 TORCH_DTYPE = {RAD_F32: torch.float32, RAD_BF16: torch.bfloat16}
 

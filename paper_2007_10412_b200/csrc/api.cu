@@ -53,7 +53,7 @@ int make_plan(const rad_mlp_desc* net, StepPlan* plan) {
   if (net->variant != RAD_DIFFERENT_SAMPLE && net->variant != RAD_SAME_SAMPLE) return RAD_EINVAL;
   if (net->act != RAD_ACT_RELU && net->act != RAD_ACT_GELU) return RAD_EINVAL;
   if (keep_threshold_host(net->p) == 0) return RAD_EINVAL;
-  if (net->law != RAD_LAW_BERNOULLI && net->law != RAD_LAW_REPLACE) return RAD_EINVAL;
+  if (net->law != RAD_LAW_BERNOULLI && net->law != RAD_LAW_REPLACE && net->law != RAD_LAW_FIXED) return RAD_EINVAL;
   const int64_t B = net->B, es = esize(net->dtype);
   int64_t off = 0;
   auto take = [&](int64_t bytes) { const int64_t at = off; off += round_up(bytes, 256); return at; };

@@ -104,7 +104,7 @@ __device__ __forceinline__ uint32_t philox_keep16(uint32_t group, uint32_t row, 
 // Host-side twins of the threshold arithmetic (double rint, one float32 division).
 uint32_t keep_threshold_host(float p);
 inline uint32_t counter_word2(uint32_t layer, int variant, int law = RAD_LAW_BERNOULLI) {
-  const uint32_t stream = (variant == RAD_SAME_SAMPLE ? 1u : 0u) + (law == RAD_LAW_REPLACE ? 2u : 0u);
+  const uint32_t stream = (variant == RAD_SAME_SAMPLE ? 1u : 0u) + 2u * (uint32_t)law;   // 0..5
   return (layer & 0xffffffu) | (stream << 24);
 }
 int64_t draws_per_row_host(float fraction, int64_t D);   // k of the with-replacement law; 0: bad fraction

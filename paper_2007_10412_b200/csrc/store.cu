@@ -39,6 +39,7 @@ double store_keep_fraction(const rad_store* st) {
     const double k = (double)draws_per_row_host(st->p, st->D), D = (double)st->D;
     return D <= 1.0 ? 1.0 : 1.0 - pow(1.0 - 1.0 / D, k);
   }
+  if (st->law == RAD_LAW_FIXED) return (double)draws_per_row_host(st->p, st->D) / (double)st->D;
   return keep_threshold_host(st->p) / (double)kLaneRange;
 }
 
@@ -436,10 +437,51 @@ __global__ void __launch_bounds__(128) replace_counts_kernel(const ReplaceParams
   for (int i = threadIdx.x; i < words; i += 128) out[i] = s_hist[i];
 }
 
+// Fixed-count law: one thread per row runs Floyd's subset sampling on a bitmap of its own in shared
+// memory (step i needs the outcome of the steps before it, so a row cannot be split; the rows run side
+// by side); the CTA then writes the rows of the multiplicity matrix, 0 or 1 per entry.
+constexpr int kFixedRows = 64;
+__global__ void __launch_bounds__(128) fixed_counts_kernel(const ReplaceParams p, const PhiloxKeys ks, int rows_per_cta,
+                                                           int words) {
+  extern __shared__ uint32_t s_bits[];            // rows_per_cta x words
+  const int tid = threadIdx.x;
+  for (int i = tid; i < rows_per_cta * words; i += 128) s_bits[i] = 0;
+  __syncthreads();
+  const int64_t row0 = (int64_t)blockIdx.x * rows_per_cta;
+  if (tid < rows_per_cta && row0 + tid < p.B) {
+    uint32_t* bm = s_bits + tid * words;
+    for (int64_t c = 0; 4 * c < p.k; ++c) {
+      uint32_t w[4];
+      philox4x32_10((uint32_t)c, (uint32_t)(row0 + tid), p.c2, p.c3, ks, w);
+#pragma unroll
+      for (int jj = 0; jj < 4; ++jj) {
+        const int64_t i = 4 * c + jj;
+        if (i < p.k) {
+          const uint32_t j = (uint32_t)(p.D - p.k + i);
+          const uint32_t t = __umulhi(w[jj], j + 1u);
+          const uint32_t pick = ((bm[t >> 5] >> (t & 31)) & 1u) ? j : t;
+          bm[pick >> 5] |= 1u << (pick & 31);
+        }
+      }
+    }
+  }
+  __syncthreads();
+  const int quads = (int)(p.ldc / 4);             // four entries, a byte each, per output word
+  for (int r = 0; r < rows_per_cta && row0 + r < p.B; ++r) {
+    uint32_t* out = reinterpret_cast<uint32_t*>(p.counts + (row0 + r) * p.ldc);
+    for (int q = tid; q < quads; q += 128) {
+      const uint32_t nib = (q >> 3) < words ? (s_bits[r * words + (q >> 3)] >> (4 * (q & 7))) & 0xfu : 0u;
+      out[q] = (nib & 1u) | ((nib & 2u) << 7) | ((nib & 4u) << 14) | ((nib & 8u) << 21);
+    }
+  }
+}
+
+constexpr int kSameFixedMaxD = 262144;   // same-sample fixed-count law: the bitmap sits in shared memory
 struct SameReplaceParams {
   int64_t D, k;
   uint32_t c2, c3;
   float scale;          // D / k
+  int32_t fixed;        // 1: k distinct columns by Floyd's sampling instead of k draws with replacement
   uint32_t* hist;       // D words of scratch
   float* colscale;      // weight of kept column j (D floats of scratch)
 };
@@ -454,13 +496,38 @@ __global__ void __launch_bounds__(1024) same_replace_mask_kernel(const SameParam
   for (int64_t i = tid; i < p.D; i += 1024) r.hist[i] = 0;
   if (tid == 0) s_running = 0;
   __syncthreads();
-  const int64_t calls = (r.k + 3) / 4;
-  for (int64_t c = tid; c < calls; c += 1024) {
-    uint32_t w[4];
-    philox4x32_10((uint32_t)c, 0u, r.c2, r.c3, ks, w);
+  if (r.fixed) {
+    // Floyd's subset sampling is sequential: one thread, bitmap in shared memory (D <= kSameFixedMaxD)
+    __shared__ uint32_t s_bits[kSameFixedMaxD / 32];
+    for (int i = tid; i < kSameFixedMaxD / 32; i += 1024) s_bits[i] = 0;
+    __syncthreads();
+    if (tid == 0) {
+      for (int64_t c = 0; 4 * c < r.k; ++c) {
+        uint32_t w[4];
+        philox4x32_10((uint32_t)c, 0u, r.c2, r.c3, ks, w);
 #pragma unroll
-    for (int j = 0; j < 4; ++j)
-      if (4 * c + j < r.k) atomicAdd(&r.hist[__umulhi(w[j], (uint32_t)p.D)], 1u);
+        for (int jj = 0; jj < 4; ++jj) {
+          const int64_t i = 4 * c + jj;
+          if (i < r.k) {
+            const uint32_t j = (uint32_t)(p.D - r.k + i);
+            const uint32_t t = __umulhi(w[jj], j + 1u);
+            const uint32_t pick = ((s_bits[t >> 5] >> (t & 31)) & 1u) ? j : t;
+            s_bits[pick >> 5] |= 1u << (pick & 31);
+          }
+        }
+      }
+    }
+    __syncthreads();
+    for (int64_t i = tid; i < p.D; i += 1024) r.hist[i] = (s_bits[i >> 5] >> (i & 31)) & 1u;
+  } else {
+    const int64_t calls = (r.k + 3) / 4;
+    for (int64_t c = tid; c < calls; c += 1024) {
+      uint32_t w[4];
+      philox4x32_10((uint32_t)c, 0u, r.c2, r.c3, ks, w);
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (4 * c + j < r.k) atomicAdd(&r.hist[__umulhi(w[j], (uint32_t)p.D)], 1u);
+    }
   }
   __syncthreads();
   for (int64_t d0 = 0; d0 < p.D; d0 += 1024) {
@@ -537,8 +604,8 @@ int64_t counts_ld(int64_t D) { return round_up(D, 16); }
 // different-sample: claim counter and look-back status words, then (with-replacement law) the multiplicity
 // matrix; same-sample with replacement: 256 bytes, a histogram word and a weight per column.
 int64_t store_workspace_bytes(int variant, int64_t B, int64_t D, int law = RAD_LAW_BERNOULLI) {
-  if (variant == RAD_SAME_SAMPLE) return law == RAD_LAW_REPLACE ? 256 + round_up(8 * D, 256) : 256;
-  return status_bytes(B, D) + (law == RAD_LAW_REPLACE ? round_up(B * counts_ld(D), 256) : 0);
+  if (variant == RAD_SAME_SAMPLE) return law != RAD_LAW_BERNOULLI ? 256 + round_up(8 * D, 256) : 256;
+  return status_bytes(B, D) + (law != RAD_LAW_BERNOULLI ? round_up(B * counts_ld(D), 256) : 0);
 }
 
 constexpr int64_t kMaxCountsRowBytes = 200 * 1024;   // a row's histogram has to fit shared memory
@@ -579,7 +646,7 @@ extern "C" int rad_store_size_query_law(int32_t variant, int32_t dtype, int32_t 
   if (out == nullptr || B <= 0 || D <= 0) return RAD_EINVAL;
   if (variant != RAD_DIFFERENT_SAMPLE && variant != RAD_SAME_SAMPLE) return RAD_EINVAL;
   if (dtype != RAD_F32 && dtype != RAD_BF16) return RAD_EINVAL;
-  if (law != RAD_LAW_BERNOULLI && law != RAD_LAW_REPLACE) return RAD_EINVAL;
+  if (law != RAD_LAW_BERNOULLI && law != RAD_LAW_REPLACE && law != RAD_LAW_FIXED) return RAD_EINVAL;
   const uint32_t T = keep_threshold_host(p);
   if (T == 0) return RAD_EINVAL;
   if ((double)B * (double)D >= 4294967296.0 * 0.75) return RAD_EINVAL;   // 32-bit tile offsets
@@ -627,12 +694,14 @@ extern "C" int rad_linear_forward_store(const void* A, int64_t lda, const rad_st
     return RAD_EINVAL;
   const uint32_t T = keep_threshold_host(st->p);
   if (T == 0) return RAD_EINVAL;
-  if (st->law != RAD_LAW_BERNOULLI && st->law != RAD_LAW_REPLACE) return RAD_EINVAL;
+  if (st->law != RAD_LAW_BERNOULLI && st->law != RAD_LAW_REPLACE && st->law != RAD_LAW_FIXED) return RAD_EINVAL;
   if ((double)st->B * (double)st->D >= 4294967296.0 * 0.75) return RAD_EINVAL;
   if (((uintptr_t)st->values & 15) != 0) return RAD_EUNSUPPORTED;
-  const bool replace = st->law == RAD_LAW_REPLACE;
+  const bool replace = st->law != RAD_LAW_BERNOULLI;      // mask and weights come from a multiplicity matrix
+  const bool fixed = st->law == RAD_LAW_FIXED;
   const int64_t k = replace ? draws_per_row_host(st->p, st->D) : 0;
   if (replace && st->variant == RAD_DIFFERENT_SAMPLE && counts_ld(st->D) > kMaxCountsRowBytes) return RAD_EUNSUPPORTED;
+  if (fixed && st->variant == RAD_SAME_SAMPLE && st->D > kSameFixedMaxD) return RAD_EUNSUPPORTED;
   int rc = check_device();
   if (rc != RAD_OK) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -668,15 +737,25 @@ extern "C" int rad_linear_forward_store(const void* A, int64_t lda, const rad_st
       // taken from them
       ReplaceParams rp;
       rp.B = st->B; rp.D = st->D; rp.k = k;
-      rp.c2 = counter_word2(st->layer, RAD_DIFFERENT_SAMPLE, RAD_LAW_REPLACE); rp.c3 = st->step;
+      rp.c2 = counter_word2(st->layer, RAD_DIFFERENT_SAMPLE, st->law); rp.c3 = st->step;
       rp.counts = reinterpret_cast<uint8_t*>(static_cast<char*>(workspace) + status_bytes(st->B, st->D));
       rp.ldc = counts_ld(st->D);
       rp.dev_status = dev_status;
-      if (rp.ldc > 48 * 1024)
-        RAD_CUDA_TRY(cudaFuncSetAttribute(replace_counts_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)kMaxCountsRowBytes));
       count_launch();
-      replace_counts_kernel<<<(unsigned)st->B, 128, (size_t)rp.ldc, s>>>(rp, ks);
+      if (fixed) {
+        const int words = (int)ceil_div(st->D, 32);
+        const int rows = (int)std::max<int64_t>(1, std::min<int64_t>(kFixedRows, kMaxCountsRowBytes / (4 * (int64_t)words)));
+        const size_t smem = (size_t)rows * words * 4;
+        if (smem > 48 * 1024)
+          RAD_CUDA_TRY(cudaFuncSetAttribute(fixed_counts_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)kMaxCountsRowBytes));
+        fixed_counts_kernel<<<(unsigned)ceil_div(st->B, rows), 128, smem, s>>>(rp, ks, rows, words);
+      } else {
+        if (rp.ldc > 48 * 1024)
+          RAD_CUDA_TRY(cudaFuncSetAttribute(replace_counts_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)kMaxCountsRowBytes));
+        replace_counts_kernel<<<(unsigned)st->B, 128, (size_t)rp.ldc, s>>>(rp, ks);
+      }
       RAD_CUDA_TRY(cudaGetLastError());
       p.counts = rp.counts; p.ldc = rp.ldc;
     }
@@ -695,8 +774,9 @@ extern "C" int rad_linear_forward_store(const void* A, int64_t lda, const rad_st
   if (replace) {
     SameReplaceParams r;
     r.D = st->D; r.k = k;
-    r.c2 = counter_word2(st->layer, RAD_SAME_SAMPLE, RAD_LAW_REPLACE); r.c3 = st->step;
+    r.c2 = counter_word2(st->layer, RAD_SAME_SAMPLE, st->law); r.c3 = st->step;
     r.scale = scale;
+    r.fixed = fixed ? 1 : 0;
     r.hist = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + 256);
     r.colscale = reinterpret_cast<float*>(static_cast<char*>(workspace) + 256 + 4 * st->D);
     colscale = r.colscale;

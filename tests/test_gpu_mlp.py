@@ -29,11 +29,13 @@ def _run(cfg, variant, p, seed, act=None, step=0, law="bernoulli"):
 
 @pytest.mark.parametrize("name,variant", [("mlp_small_different", "different"), ("mlp_small_same", "same"),
                                           ("mlp_wide_cut", "different"), ("mlp_wide_cut", "same")])
-def test_step_with_the_with_replacement_law_matches_oracle(name, variant):
+@pytest.mark.parametrize("law", ["replace", "fixed"])
+def test_step_with_the_other_sampling_laws_matches_oracle(name, variant, law):
     """The whole step with the paper's own sampling law (k = ceil(0.1 d) draws with replacement per layer
-    input): loss and bias gradients as in exact backprop, weight gradients from the stores."""
+    input) and with the fixed-count law without replacement: loss and bias gradients as in exact backprop,
+    weight gradients from the stores."""
     cfg = get_config(name)
-    ctx, ref, _ = _run(cfg, variant, 0.1, seed=3, step=2, law="replace")
+    ctx, ref, _ = _run(cfg, variant, 0.1, seed=3, step=2, law=law)
     tol = TOL[cfg.dtype]
     assert abs(ctx.loss.item() - ref.loss) <= (1e-5 if cfg.dtype == "f32" else 2e-3) * abs(ref.loss)
     nnz = ctx.nnz.cpu().numpy().reshape(-1, 2)

@@ -1,5 +1,5 @@
-"""The paper's with-replacement sampling law on the GPU against the oracle: multiplicities, store and
-weight gradient (different-sample and same-sample, float32 and bf16)."""
+"""The with-replacement law (the paper's own) and the fixed-count law without replacement on the GPU
+against the oracle: store and weight gradient (different-sample and same-sample, float32 and bf16)."""
 import numpy as np
 import pytest
 import torch
@@ -16,16 +16,22 @@ SHAPES = [(150, 784, "f32"), (150, 300, "bf16"), (7, 5, "f32"), (64, 128, "bf16"
           (257, 1160, "f32"), (1, 1, "f32")]
 
 
+LAWS = ["replace", "fixed"]
+
+
+@pytest.mark.parametrize("law", LAWS)
 @pytest.mark.parametrize("B,D,dtype", SHAPES)
 @pytest.mark.parametrize("f", [0.1, 0.5, 1.0, 0.01])
-def test_different_sample_store_is_bit_exact(B, D, dtype, f):
+def test_different_sample_store_is_bit_exact(B, D, dtype, f, law):
     import paper_2007_10412_b200 as rad
     A, _ = layer_inputs(B, D, 1, dtype=dtype, seed=B + D, relu_like=True)
     seed, layer, step = (1 << 40) + 777, 2, 5
-    ref = orc.forward_store(A, dtype, "different", f, seed, layer, step, law="replace")
+    ref = orc.forward_store(A, dtype, "different", f, seed, layer, step, law=law)
     assert rad.rad_draws_per_row(f, D) == ref.T
     assert np.float32(rad.rad_replace_scale(f, D)) == ref.scale
-    st = rad.Store("different", dtype, B, D, f, seed=seed, layer=layer, step=step, capacity="worst", law="replace")
+    if law == "fixed":
+        assert ref.nnz == B * ref.T                      # exactly k entries per row
+    st = rad.Store("different", dtype, B, D, f, seed=seed, layer=layer, step=step, capacity="worst", law=law)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     rad.rad_linear_forward_store(to_dev(A, dtype), st, status)
     torch.cuda.synchronize()
@@ -39,14 +45,15 @@ def test_different_sample_store_is_bit_exact(B, D, dtype, f):
     assert np.array_equal(u32(st.relubits).reshape(B, -1), ref.relubits)
 
 
+@pytest.mark.parametrize("law", LAWS)
 @pytest.mark.parametrize("B,D,dtype", SHAPES)
 @pytest.mark.parametrize("f", [0.1, 0.5, 1.0])
-def test_same_sample_store_is_bit_exact(B, D, dtype, f):
+def test_same_sample_store_is_bit_exact(B, D, dtype, f, law):
     import paper_2007_10412_b200 as rad
     A, _ = layer_inputs(B, D, 1, dtype=dtype, seed=B + D + 1, relu_like=True)
     seed, layer, step = 99, 1, 3
-    ref = orc.forward_store(A, dtype, "same", f, seed, layer, step, law="replace")
-    st = rad.Store("same", dtype, B, D, f, seed=seed, layer=layer, step=step, capacity="worst", law="replace")
+    ref = orc.forward_store(A, dtype, "same", f, seed, layer, step, law=law)
+    st = rad.Store("same", dtype, B, D, f, seed=seed, layer=layer, step=step, capacity="worst", law=law)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     rad.rad_linear_forward_store(to_dev(A, dtype), st, status)
     torch.cuda.synchronize()
@@ -62,16 +69,17 @@ def test_same_sample_store_is_bit_exact(B, D, dtype, f):
     assert (got[:, k:] == 0).all()
 
 
+@pytest.mark.parametrize("law", LAWS)
 @pytest.mark.parametrize("variant", ["different", "same"])
 @pytest.mark.parametrize("B,D,H,dtype", [(150, 784, 300, "f32"), (328, 640, 520, "bf16"), (130, 264, 72, "bf16")])
-def test_weight_gradient_from_the_store(variant, B, D, H, dtype):
-    """dW_hat = A_hat^T dZ from a with-replacement store through the same weight-gradient call."""
+def test_weight_gradient_from_the_store(variant, B, D, H, dtype, law):
+    """dW_hat = A_hat^T dZ from such a store through the same weight-gradient call."""
     import paper_2007_10412_b200 as rad
     f = 0.2
     A, dZ = layer_inputs(B, D, H, dtype=dtype, seed=B + H)
-    ref = orc.forward_store(A, dtype, variant, f, 5, 0, 1, law="replace")
+    ref = orc.forward_store(A, dtype, variant, f, 5, 0, 1, law=law)
     want = orc.weight_grad(ref, dZ)
-    st = rad.Store(variant, dtype, B, D, f, seed=5, layer=0, step=1, law="replace")
+    st = rad.Store(variant, dtype, B, D, f, seed=5, layer=0, step=1, law=law)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     rad.rad_linear_forward_store(to_dev(A, dtype), st, status)
     dW = torch.empty(D, H, dtype=torch.float32, device="cuda")
@@ -102,3 +110,21 @@ def test_a_layer_of_many_tiles_and_the_typical_capacity():
     # distinct columns per row: D (1 - (1 - 1/D)^k) on average (Sec. 3.2 law), fewer than the k draws
     k = orc.draws_per_row(f, D)
     assert abs(ref.nnz / B - D * (1 - (1 - 1 / D) ** k)) < 3.0 and ref.nnz < B * k
+
+
+@pytest.mark.parametrize("variant", ["different", "same"])
+def test_fixed_count_law_at_fraction_one_is_exact_backprop(variant):
+    """Without replacement a fraction of 1.0 keeps everything with weight 1 (App. A): dW equals A^T dZ."""
+    import paper_2007_10412_b200 as rad
+    B, D, H = 150, 300, 64
+    A, dZ = layer_inputs(B, D, H, dtype="f32", seed=4)
+    st = rad.Store(variant, "f32", B, D, 1.0, seed=8, law="fixed", capacity="worst")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    rad.rad_linear_forward_store(to_dev(A, "f32"), st, status)
+    dW = torch.empty(D, H, dtype=torch.float32, device="cuda")
+    ws = torch.empty(max(rad.rad_weight_grad_workspace(st, H), 256), dtype=torch.uint8, device="cuda")
+    rad.rad_linear_weight_grad(st, to_dev(dZ, "f32"), dW, ws, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0 and st.nnz.cpu().numpy()[0] == (B * D if variant == "different" else D)
+    fro, mx = rel_err(dW.cpu().numpy(), A.astype(np.float64).T @ dZ.astype(np.float64))
+    assert fro <= 1e-5 and mx <= 1e-5
