@@ -35,6 +35,11 @@ Third law (App. A, caption of the fraction sweep: the method "could be modified
 to sample without replacement", and fraction 1.0 is then the exact gradient):
 a uniformly random subset of exactly k = ceil(fraction * d) coordinates, each
 kept with weight d / k (`law="fixed"`).
+
+Random projection (Sec. 3.2 after Eq. 5; App. A "Random Projections for RAD"):
+P = R R^T with R a d x k matrix of independent Rademacher signs scaled by
+1 / sqrt(k).  The forward pass keeps S = A R' (B x k, R' the unscaled signs),
+the backward pass forms dW_hat = R' ((S^T dZ) / k) (`variant="project"`).
 """
 from dataclasses import dataclass, field
 from typing import List, Optional
@@ -50,6 +55,7 @@ STREAM_DIFFERENT_REPLACE = 2   # with-replacement draws, per row
 STREAM_SAME_REPLACE = 3        # with-replacement draws, shared by the minibatch
 STREAM_DIFFERENT_FIXED = 4     # k distinct columns, per row
 STREAM_SAME_FIXED = 5          # k distinct columns, shared by the minibatch
+STREAM_PROJECT = 6             # signs of the Rademacher projection
 LANE_BITS = 8
 LANES_PER_CALL = 16      # 128 output bits / 8
 LANE_RANGE = 1 << LANE_BITS
@@ -230,6 +236,44 @@ def fixed_subset(variant: str, B: int, D: int, fraction, seed: int, layer: int, 
 
 
 # --------------------------------------------------------------------------
+# random projection (Sec. 3.2: "R be a random projection matrix of independent
+# Rademacher random variables"; App. A: scaled so that P = R R^T has E[P] = I)
+# --------------------------------------------------------------------------
+def rademacher(D: int, k: int, seed: int, layer: int, step: int) -> np.ndarray:
+    """The unscaled sign matrix R' (D x k, entries +1 / -1, float64); R = R' / sqrt(k).
+
+    Entry (d, j) reads bit j % 32 of word (j % 128) // 32 of the Philox output for counter
+    (j // 128, d, layer | 6 << 24, step): set means -1.
+    """
+    calls = (k + 127) // 128
+    c0 = np.arange(calls, dtype=np.uint64)[None, :]
+    rows = np.arange(D, dtype=np.uint64)[:, None]
+    words = philox4x32_10(c0, rows, np.uint64((layer & 0xFFFFFF) | (STREAM_PROJECT << 24)),
+                          np.uint64(step & 0xFFFFFFFF), np.uint64(seed & 0xFFFFFFFF),
+                          np.uint64((seed >> 32) & 0xFFFFFFFF))
+    w = np.stack(words, axis=-1)                                   # D x calls x 4
+    bits = (w[..., None] >> np.arange(32, dtype=np.uint32)) & np.uint32(1)     # D x calls x 4 x 32
+    bits = bits.reshape(D, calls * 128)[:, :k]
+    return 1.0 - 2.0 * bits.astype(np.float64)
+
+
+def project_store(A, dtype: str, fraction, seed: int, layer: int, step: int, R=None) -> "Store":
+    """What the forward pass keeps with the projection: S = round_dtype(A R') (B x k), k = ceil(fraction d).
+    `R` replaces the Philox signs (test hook for exhaustive enumeration)."""
+    A = np.ascontiguousarray(A, dtype=np.float32)
+    B, D = A.shape
+    k = draws_per_row(fraction, D)
+    Rm = rademacher(D, k, seed, layer, step) if R is None else np.asarray(R, np.float64)
+    S = (A.astype(np.float64) @ Rm).astype(np.float32)
+    if dtype == "bf16":
+        S = round_bf16(S)
+    elif dtype != "f32":
+        raise ValueError(dtype)
+    return Store("project", dtype, B, D, k, np.float32(1.0) / np.float32(k), np.zeros((0, 0), np.uint32),
+                 S.reshape(-1), R=Rm)
+
+
+# --------------------------------------------------------------------------
 # number formats
 # --------------------------------------------------------------------------
 def round_bf16(x) -> np.ndarray:
@@ -277,6 +321,7 @@ class Store:
     values: np.ndarray                   # float32, canonical order (row-major, ascending column)
     row_ptr: Optional[np.ndarray] = None  # different: int64 B+1
     idx: Optional[np.ndarray] = None      # same: kept columns ascending
+    R: Optional[np.ndarray] = None        # project: the D x k sign matrix (regenerated from the key on the device)
     relubits: Optional[np.ndarray] = None  # uint32 B x ceil(D/32): (A > 0)
 
     @property
@@ -355,6 +400,13 @@ def weight_grad(st: Store, dZ) -> np.ndarray:
     part of the weight matrix is updated).
     """
     dZ = np.asarray(dZ, dtype=np.float64)
+    if st.variant == "project":
+        # dW_hat = R (R^T A^T dZ) with R = R' / sqrt(k): G = (S^T dZ) / k is a tensor of the working type
+        # on the device (float32 product with fl32(1 / k), then one rounding), then R' G
+        k = st.T
+        G = (st.values.reshape(st.B, k).astype(np.float64).T @ dZ).astype(np.float32) * st.scale
+        G = round_bf16(G) if st.dtype == "bf16" else G
+        return st.R @ G.astype(np.float64)
     if st.variant == "same":
         dW = np.zeros((st.D, dZ.shape[1]), dtype=np.float64)
         Ac = st.values.reshape(st.B, st.idx.size).astype(np.float64)
