@@ -297,6 +297,19 @@ def kernel_sweep(rad, torch, A, dZ, H, ps):
                          dW_ms=round(ms_dw, 4), dW_tflops=round(flops / ms_dw / 1e9, 1), dW_flops=kind,
                          nnz=int(nnz[0])))
         del st, ws
+    # random projection (P = R R^T, Rademacher signs, k = ceil(0.1 D) columns): the store is one dense GEMM,
+    # the weight gradient two; TFLOP/s on the flops of those contractions (2 B D k; 2 B k H + 2 D k H)
+    p = 0.1
+    st = rad.Store("project", "bf16", B, D, p, relu_bits=False)
+    k = rad.rad_draws_per_row(p, D)
+    ms_store = timed(lambda: rad.rad_linear_forward_store(A, st, status))
+    ws = torch.empty(max(rad.rad_weight_grad_workspace(st, H), 256), dtype=torch.uint8, device="cuda")
+    ms_dw = timed(lambda: rad.rad_linear_weight_grad(st, dZ, dW, ws, status), n=3)
+    rows.append(dict(variant="project", p=p, k=k, store_ms=round(ms_store, 4),
+                     store_tflops=round(2.0 * B * D * k / ms_store / 1e9, 1), dW_ms=round(ms_dw, 4),
+                     dW_tflops=round((2.0 * B * k * H + 2.0 * D * k * H) / ms_dw / 1e9, 1), dW_flops="projected",
+                     stored_bytes=int(st.c.values_ld) * B * 2))
+    del st, ws
     assert status.item() == 0, f"device status {status.item()}"
     return rows
 

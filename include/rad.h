@@ -48,7 +48,7 @@ extern "C" {
 #define RAD_DEV_EINTERNAL 3    /* an index left its buffer; the access was skipped (a bug)   */
 
 typedef enum { RAD_F32 = 0, RAD_BF16 = 1 } rad_dtype;
-typedef enum { RAD_DIFFERENT_SAMPLE = 0, RAD_SAME_SAMPLE = 1 } rad_variant;
+typedef enum { RAD_DIFFERENT_SAMPLE = 0, RAD_SAME_SAMPLE = 1, RAD_PROJECT = 2 } rad_variant;
 typedef enum { RAD_ACT_NONE = 0, RAD_ACT_RELU = 1, RAD_ACT_GELU = 2 } rad_act;
 
 /* Geometry of the compact store (fixed; part of the data layout). */
@@ -154,6 +154,24 @@ typedef struct rad_store_sizes {
   int64_t keepbits_words, offsets_words, relubits_words;
   int64_t workspace_bytes;    /* scratch rad_linear_forward_store needs                        */
 } rad_store_sizes;
+
+/*
+ * Random-projection variant, variant = RAD_PROJECT (Sec. 3.2 after Eq. 5; App. A "Random
+ * Projections for RAD"): P = R R^T with R a D x k matrix of independent Rademacher signs scaled by
+ * 1 / sqrt(k), k = ceil(p * D) as for the with-replacement law.  The store is the dense block
+ * S = A R' (R' the unscaled signs), rounded to `dtype`:
+ *   values   : B x values_ld row-major, values[b, j] = sum_d A[b, d] R'[d, j] for j < k, zero for
+ *              k <= j < values_ld (values_ld a multiple of 8, at least k; the size query gives k
+ *              rounded up to 64);  nnz[0] = k, nnz[1] = B * k;  keepbits, offsets and law unused.
+ *   R'[d, j] : -1 if bit j % 32 of word (j % 128) / 32 of the Philox-4x32-10 output for counter
+ *              (j / 128, d, layer | 6 << 24, step) is set, else +1.  R' is not stored: both passes
+ *              draw it again into their workspace.
+ * rad_linear_weight_grad forms dW_hat = R' G with G = (S^T dZ) * fl32(1 / k) rounded to `dtype`: two
+ * dense contractions on the same GEMM kernels as the exact paths.
+ * rad_rademacher writes R' (D x ld, row-major, type `dtype`, columns k .. ld-1 zero) to `out`.
+ */
+int rad_rademacher(int32_t dtype, int64_t D, float fraction, int64_t ld, uint64_t seed, uint32_t layer,
+                   uint32_t step, void* out /* device */, void* stream);
 
 /* Buffer sizes for a store of the given shape (host only, nothing is launched). */
 int rad_store_size_query(int32_t variant, int32_t dtype, int64_t B, int64_t D, float p,

@@ -497,7 +497,9 @@ def mlp_step(X, labels, Ws, bs, act="relu", dtype="f32", variant=None, p=1.0, se
     A = [np.asarray(X, dtype=np.float64)]
     Z, stores = [], []
     for l in range(L):
-        if variant is not None:
+        if variant == "project":
+            stores.append(project_store(A[l].astype(np.float32), dtype, p, seed, l, step))
+        elif variant is not None:
             stores.append(forward_store(A[l].astype(np.float32), dtype, variant, p, seed, l, step,
                                         mask=None if masks is None else masks[l], law=law))
         else:

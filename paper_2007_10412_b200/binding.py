@@ -15,13 +15,13 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "librad_b200.so")
 
 RAD_F32, RAD_BF16 = 0, 1
-RAD_DIFFERENT_SAMPLE, RAD_SAME_SAMPLE = 0, 1
+RAD_DIFFERENT_SAMPLE, RAD_SAME_SAMPLE, RAD_PROJECT = 0, 1, 2
 RAD_ACT_NONE, RAD_ACT_RELU, RAD_ACT_GELU = 0, 1, 2
 RAD_DEV_ECAPACITY, RAD_DEV_ETIMEOUT = 1, 2
 TILE_ROWS, TILE_COLS, VALUE_ALIGN = 64, 128, 8
 
 DTYPES = {"f32": RAD_F32, "bf16": RAD_BF16, torch.float32: RAD_F32, torch.bfloat16: RAD_BF16}
-VARIANTS = {"different": RAD_DIFFERENT_SAMPLE, "same": RAD_SAME_SAMPLE}
+VARIANTS = {"different": RAD_DIFFERENT_SAMPLE, "same": RAD_SAME_SAMPLE, "project": RAD_PROJECT}
 LAWS = {"bernoulli": 0, "replace": 1, "fixed": 2}
 ACTS = {"none": RAD_ACT_NONE, "relu": RAD_ACT_RELU, "gelu": RAD_ACT_GELU}
 TORCH_DTYPE = {RAD_F32: torch.float32, RAD_BF16: torch.bfloat16}
@@ -69,7 +69,7 @@ class rad_step_stats(C.Structure):
 
 
 EXPORTS = ["rad_keep_threshold", "rad_effective_p", "rad_scale", "rad_store_size_query", "rad_set_store_kernel",
-           "rad_draws_per_row", "rad_replace_scale", "rad_store_size_query_law",
+           "rad_draws_per_row", "rad_replace_scale", "rad_store_size_query_law", "rad_rademacher",
            "rad_linear_forward_store", "rad_linear_forward_store_static", "rad_weight_grad_workspace", "rad_linear_weight_grad",
            "rad_linear_forward", "rad_softmax_xent", "rad_input_grad_workspace", "rad_linear_input_grad",
            "rad_mlp_workspace", "rad_mlp_step", "rad_irnn_workspace", "rad_irnn_step", "rad_cnn_workspace", "rad_cnn_step", "rad_launch_count", "rad_strerror", "rad_version"]
@@ -100,6 +100,7 @@ def lib():
         L.rad_draws_per_row.argtypes = [f32, i64]
         L.rad_replace_scale.restype = f32
         L.rad_replace_scale.argtypes = [f32, i64]
+        L.rad_rademacher.argtypes = [i32, i64, f32, i64, C.c_uint64, C.c_uint32, C.c_uint32, vp, vp]
         L.rad_store_size_query_law.argtypes = [i32, i32, i32, i64, i64, f32, C.POINTER(rad_store_sizes)]
         L.rad_store_size_query.argtypes = [i32, i32, i64, i64, f32, C.POINTER(rad_store_sizes)]
         L.rad_linear_forward_store.argtypes = [vp, i64, C.POINTER(rad_store), vp, i64, vp, vp]
@@ -178,6 +179,12 @@ def rad_store_size_query_law(variant, dtype, law, B, D, p):
     return out
 
 
+def rad_rademacher(dtype, D, fraction, ld, seed, layer, step, out):
+    """Writes the D x ld sign matrix of the projection variant to `out` (columns beyond k are zero)."""
+    _check(lib().rad_rademacher(DTYPES[dtype], D, fraction, ld, seed, layer, step, _ptr(out), _stream()),
+           "rad_rademacher")
+
+
 def rad_draws_per_row(fraction, D):
     return int(lib().rad_draws_per_row(fraction, D))
 
@@ -196,7 +203,7 @@ class Store:
         self.sizes = sz
         cap = {"typical": sz.values_typical, "worst": sz.values_worst}.get(capacity, capacity)
         ld = 0
-        if variant == "same":
+        if variant in ("same", "project"):
             ld = {"typical": sz.values_ld_typical, "worst": sz.values_ld_worst}.get(capacity, capacity)
             cap = B * ld
         tdt = TORCH_DTYPE[DTYPES[dtype]]

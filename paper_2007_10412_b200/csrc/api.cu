@@ -50,7 +50,8 @@ struct StepPlan {
 int make_plan(const rad_mlp_desc* net, StepPlan* plan) {
   if (net == nullptr || net->dims == nullptr || net->L < 1 || net->L > 64 || net->B <= 0) return RAD_EINVAL;
   if (!valid_dtype(net->dtype)) return RAD_EINVAL;
-  if (net->variant != RAD_DIFFERENT_SAMPLE && net->variant != RAD_SAME_SAMPLE) return RAD_EINVAL;
+  if (net->variant != RAD_DIFFERENT_SAMPLE && net->variant != RAD_SAME_SAMPLE && net->variant != RAD_PROJECT)
+    return RAD_EINVAL;
   if (net->act != RAD_ACT_RELU && net->act != RAD_ACT_GELU) return RAD_EINVAL;
   if (keep_threshold_host(net->p) == 0) return RAD_EINVAL;
   if (net->law != RAD_LAW_BERNOULLI && net->law != RAD_LAW_REPLACE && net->law != RAD_LAW_FIXED) return RAD_EINVAL;
@@ -87,7 +88,8 @@ int make_plan(const rad_mlp_desc* net, StepPlan* plan) {
     tmp.variant = net->variant; tmp.dtype = net->dtype; tmp.B = B; tmp.D = D; tmp.p = net->p;
     tmp.law = net->law;
     tmp.values_ld = lp.values_ld; tmp.values_capacity = lp.capacity;
-    scratch = max(scratch, tc_weight_grad_workspace(&tmp, H));
+    scratch = max(scratch, net->variant == RAD_PROJECT ? project_weight_grad_workspace(&tmp, H)
+                                                       : tc_weight_grad_workspace(&tmp, H));
   }
   st.unsampled_bytes = B * net->dims[net->L] * 4;
   st.full_backprop_bytes += st.unsampled_bytes;
@@ -129,6 +131,11 @@ extern "C" const char* rad_strerror(int code) {
 
 extern "C" int rad_weight_grad_workspace(const rad_store* st, int64_t H, int64_t* bytes) {
   if (st == nullptr || bytes == nullptr || H <= 0 || st->B <= 0 || st->D <= 0) return RAD_EINVAL;
+  if (st->variant == RAD_PROJECT) {
+    if (st->values_ld <= 0) return RAD_EINVAL;
+    *bytes = project_weight_grad_workspace(st, H);
+    return RAD_OK;
+  }
   *bytes = round_up(tc_weight_grad_workspace(st, H), 256);
   return RAD_OK;
 }
@@ -136,6 +143,14 @@ extern "C" int rad_weight_grad_workspace(const rad_store* st, int64_t H, int64_t
 extern "C" int rad_linear_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H, float* dW,
                                       int64_t ldw, void* workspace, int64_t workspace_bytes,
                                       int32_t* dev_status, void* stream) {
+  if (st != nullptr && st->variant == RAD_PROJECT) {
+    if (st->B <= 0 || st->D <= 0 || !valid_dtype(st->dtype) || dZ == nullptr || dW == nullptr || H <= 0 || ldz < H ||
+        ldw < H)
+      return RAD_EINVAL;
+    const int rcp = check_device();
+    return rcp != RAD_OK ? rcp
+                         : project_weight_grad(st, dZ, ldz, H, dW, ldw, workspace, workspace_bytes, dev_status, stream);
+  }
   if (!store_args_ok(st) || dZ == nullptr || dW == nullptr || H <= 0 || ldz < H || ldw < H) return RAD_EINVAL;
   int rc = check_device();
   if (rc != RAD_OK) return rc;

@@ -145,6 +145,17 @@ int check_device();   // RAD_OK on an sm_100 device
 void count_launch(int n = 1);   // host-side tally of kernels this library has launched
 void* tensor_map_encoder();     // cuTensorMapEncodeTiled, or nullptr (tc.cu)
 
+// random-projection variant (project.cu)
+int64_t project_ld(int64_t k);
+bool project_store_ok(const rad_store* st);
+int64_t project_store_workspace(int dtype, int64_t D, int64_t ld);
+int64_t project_weight_grad_workspace(const rad_store* st, int64_t H);
+int project_forward_store(const void* A, int64_t lda, const rad_store* st, void* workspace, int64_t workspace_bytes,
+                          int32_t* dev_status, void* stream);
+int project_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H, float* dW, int64_t ldw,
+                        void* workspace, int64_t workspace_bytes, int32_t* dev_status, void* stream);
+int launch_relu_bits(int dtype, const void* A, int64_t lda, int64_t B, int64_t D, uint32_t* relubits, cudaStream_t s);
+
 // f32/bf16 CUDA-core kernels (small or unaligned problems)
 int simt_forward(int dtype, int act, int64_t B, int64_t D, int64_t H, const void* A, int64_t lda,
                  const void* W, int64_t ldw, const float* bias, void* out_act, int64_t ld_act,

@@ -613,6 +613,19 @@ constexpr int64_t kMaxCountsRowBytes = 200 * 1024;   // a row's histogram has to
 }  // namespace
 }  // namespace rad
 
+namespace rad {
+int launch_relu_bits(int dtype, const void* A, int64_t lda, int64_t B, int64_t D, uint32_t* relubits, cudaStream_t s) {
+  const int64_t w32 = ceil_div(D, 32), n = B * w32;
+  const int g2 = (int)std::min<int64_t>(ceil_div(n, 256), 148 * 16);
+  count_launch();
+  if (dtype == RAD_BF16)
+    relu_bits_kernel<bf16><<<g2, 256, 0, s>>>(static_cast<const bf16*>(A), lda, B, D, w32, relubits);
+  else
+    relu_bits_kernel<float><<<g2, 256, 0, s>>>(static_cast<const float*>(A), lda, B, D, w32, relubits);
+  return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
+}
+}  // namespace rad
+
 using namespace rad;
 
 extern "C" int rad_set_store_kernel(int32_t which) {
@@ -644,8 +657,20 @@ extern "C" int rad_store_size_query(int32_t variant, int32_t dtype, int64_t B, i
 extern "C" int rad_store_size_query_law(int32_t variant, int32_t dtype, int32_t law, int64_t B, int64_t D, float p,
                                         rad_store_sizes* out) {
   if (out == nullptr || B <= 0 || D <= 0) return RAD_EINVAL;
-  if (variant != RAD_DIFFERENT_SAMPLE && variant != RAD_SAME_SAMPLE) return RAD_EINVAL;
   if (dtype != RAD_F32 && dtype != RAD_BF16) return RAD_EINVAL;
+  if (variant == RAD_PROJECT) {
+    // a dense B x ld block (ld: k rounded up to 64 columns, zero beyond k); no index data
+    const int64_t k = draws_per_row_host(p, D);
+    if (k == 0) return RAD_EINVAL;
+    const int64_t ld = project_ld(k);
+    out->values_ld_worst = out->values_ld_typical = ld;
+    out->values_worst = out->values_typical = B * ld;
+    out->keepbits_words = out->offsets_words = 0;
+    out->relubits_words = B * ceil_div(D, 32);
+    out->workspace_bytes = project_store_workspace(dtype, D, ld);
+    return RAD_OK;
+  }
+  if (variant != RAD_DIFFERENT_SAMPLE && variant != RAD_SAME_SAMPLE) return RAD_EINVAL;
   if (law != RAD_LAW_BERNOULLI && law != RAD_LAW_REPLACE && law != RAD_LAW_FIXED) return RAD_EINVAL;
   const uint32_t T = keep_threshold_host(p);
   if (T == 0) return RAD_EINVAL;
@@ -688,8 +713,12 @@ extern "C" int rad_linear_forward_store(const void* A, int64_t lda, const rad_st
                                         int64_t workspace_bytes, int32_t* dev_status, void* stream) {
   if (A == nullptr || st == nullptr) return RAD_EINVAL;
   if (st->B <= 0 || st->D <= 0 || lda < st->D) return RAD_EINVAL;
-  if (st->variant != RAD_DIFFERENT_SAMPLE && st->variant != RAD_SAME_SAMPLE) return RAD_EINVAL;
   if (st->dtype != RAD_F32 && st->dtype != RAD_BF16) return RAD_EINVAL;
+  if (st->variant == RAD_PROJECT) {
+    const int rcp = check_device();
+    return rcp != RAD_OK ? rcp : project_forward_store(A, lda, st, workspace, workspace_bytes, dev_status, stream);
+  }
+  if (st->variant != RAD_DIFFERENT_SAMPLE && st->variant != RAD_SAME_SAMPLE) return RAD_EINVAL;
   if (st->values == nullptr || st->keepbits == nullptr || st->offsets == nullptr || st->nnz == nullptr)
     return RAD_EINVAL;
   const uint32_t T = keep_threshold_host(st->p);

@@ -110,3 +110,19 @@ def test_same_sample_statistics_over_seeds(p):
         else:
             assert err <= 2.0 * var_sum / S + 1e-10 * norm
             assert abs(float(sq[l]) / S - var_sum) <= 0.15 * var_sum
+
+
+@pytest.mark.parametrize("name", ["mlp_small_different", "mlp_wide_cut"])
+def test_step_with_the_projection_variant_matches_oracle(name):
+    """The whole step with P = R R^T (Rademacher projection, k = ceil(0.25 d)): loss and bias gradients as in
+    exact backprop, weight gradients R' ((S^T dZ) / k) from the stored blocks."""
+    cfg = get_config(name)
+    ctx, ref, _ = _run(cfg, "project", 0.25, seed=5, step=1)
+    tol = TOL[cfg.dtype]
+    assert abs(ctx.loss.item() - ref.loss) <= (1e-5 if cfg.dtype == "f32" else 2e-3) * abs(ref.loss)
+    nnz = ctx.nnz.cpu().numpy().reshape(-1, 2)
+    for l in range(len(cfg.dims) - 1):
+        assert nnz[l, 0] == ref.stores[l].T
+        for got, want in ((ctx.dW[l], ref.dW[l]), (ctx.db[l], ref.db[l])):
+            fro, mx = rel_err(to_host_f32(got), want)
+            assert fro <= tol and mx <= tol, (l, fro, mx)
