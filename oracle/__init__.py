@@ -12,9 +12,12 @@ Parity status
     pinned by tests/test_oracle_*.py (p = 1 equals exact backprop, exhaustive
     expectation and variance over all masks, finite differences, torch
     autograd in float64, the memory figures printed in App. A and Table 1).
-  * Philox-4x32-10: pinned for internal consistency (independent big-integer
-    restatement, invertible rounds, uniformity).  Conformance to the known
-    answer vectors distributed with the generator's reference code is
-    "parity unpinned": those vectors are not available offline.
+  * Philox-4x32-10: pinned against the known-answer vectors published with the
+    generator's reference code (tests/golden), an independent big-integer
+    restatement, invertible rounds and uniformity.
+  * the with-replacement law, the fixed-count law and the random projection:
+    pinned by tests/test_oracle_replace.py, test_oracle_fixed.py and
+    test_oracle_project.py (all draw sequences / subsets / sign matrices of
+    tiny layers, closed-form variances, special cases that are exact).
 """
 from . import philox, rad, memory_model, irnn, cnn  # noqa: F401

@@ -1,11 +1,11 @@
 """Pins for the oracle's Philox-4x32-10 (host only).
 
-The generator's published known-answer vectors are not available offline, so
-conformance to them is unpinned.  What is pinned: agreement with an
+Pinned: the generator's published known-answer vectors (tests/golden), agreement with an
 independent restatement in Python big integers, invertibility of each round
 (multiplication by an odd constant is a bijection mod 2^32), sensitivity to
 every counter/key word, and lane uniformity.
 """
+import os
 import numpy as np
 import pytest
 
@@ -35,6 +35,17 @@ def inverse_round(c, k):
     c1 = c[0] ^ ((M1 * c2) >> 32) ^ k[0]
     c3 = c[2] ^ ((M0 * c0) >> 32) ^ k[1]
     return [c0, c1, c2, c3]
+
+
+def test_published_known_answer_vectors():
+    path = os.path.join(os.path.dirname(__file__), "golden", "philox4x32_10_known_answers.txt")
+    rows = [[int(t, 16) for t in line.split()] for line in open(path) if line.strip() and not line.startswith("#")]
+    assert len(rows) == 3
+    for r in rows:
+        ctr, key, want = r[:4], r[4:6], r[6:]
+        got = ph.philox4x32_10(*(np.uint64(v) for v in ctr), *(np.uint64(v) for v in key))
+        assert [int(v) for v in got] == want
+        assert bigint_philox(ctr, key) == want
 
 
 def test_matches_bigint_restatement():
