@@ -41,7 +41,7 @@ constexpr int kWarpElems = kTileElems / kComputeWarps;   // entries of a tile th
 template <typename T, int S>
 struct PipeSmem {
   alignas(128) T raw[S][kTileElems];            // tiles of A as loaded
-  alignas(16) T wbuf[kComputeWarps][kWarpElems];   // kept values of a warp's eight rows, in order
+  alignas(16) T wbuf[kComputeWarps][kWarpElems + 8];   // kept values of a warp's eight rows, in order (from index 0 or 1)
   uint64_t full[S], empty[S];                   // raw ring
   uint64_t chunk_ready[kSlots], cnt_ready[kSlots], base_ready[kSlots];
   uint32_t chunk_id[kSlots];
@@ -141,6 +141,30 @@ __device__ __forceinline__ uint32_t positive32(const bf16* src) {
   return m;
 }
 
+// Copies entries [first, end) of a warp's staging buffer to `out` (same indices), multiplied by `scale`
+// and rounded once to the working type.  out + 0 is 4-byte aligned.
+__device__ __forceinline__ void copy_scaled(const float* wb, float* out, uint32_t first, uint32_t end, float scale,
+                                            int lane) {
+  for (uint32_t i = first + lane; i < end; i += 32) out[i] = __fmul_rn(wb[i], scale);
+}
+// bf16: two entries per lane and step (one 4-byte load, one 4-byte store); a pair that sticks out of
+// [first, end) at either end stores its inner half alone.
+__device__ __forceinline__ void copy_scaled(const bf16* wb, bf16* out, uint32_t first, uint32_t end, float scale,
+                                            int lane) {
+  const uint32_t* wb2 = reinterpret_cast<const uint32_t*>(wb);
+  for (uint32_t pr = lane; 2 * pr < end; pr += 32) {
+    const uint32_t v = wb2[pr];
+    const __nv_bfloat162 h2 = __floats2bfloat162_rn(__fmul_rn(__uint_as_float(v << 16), scale),
+                                                    __fmul_rn(__uint_as_float(v & 0xffff0000u), scale));
+    if (2 * pr >= first && 2 * pr + 1 < end) {
+      reinterpret_cast<__nv_bfloat162*>(out)[pr] = h2;
+    } else {
+      if (2 * pr >= first) out[2 * pr] = h2.x;
+      if (2 * pr + 1 >= first && 2 * pr + 1 < end) out[2 * pr + 1] = h2.y;
+    }
+  }
+}
+
 template <typename T, int S>
 __global__ void __launch_bounds__(kPipeThreads, 3) store_pipelined_kernel(const StoreParams p, const PhiloxKeys ks,
                                                                       const __grid_constant__ CUtensorMap tmA) {
@@ -203,44 +227,19 @@ __global__ void __launch_bounds__(kPipeThreads, 3) store_pipelined_kernel(const 
       return chunk;
     };
 
-    // chunks whose first phase is done, oldest first
-    uint32_t mq[kAhead][kChunk], cq[kAhead];
-    uint32_t seq1 = 0, seq2 = 0;                  // chunks handed to the first / second phase so far
-    bool more = true;                             // the loader has not yet said that the work is finished
-#pragma unroll
-    for (int a = 0; a < kAhead; ++a) {
-      cq[a] = kNoChunk;
-#pragma unroll
-      for (int g = 0; g < kChunk; ++g) mq[a][g] = 0;
-    }
-    bool ok = true;
-#pragma unroll 1
-    for (uint32_t it = 0; ok; ++it) {
-      uint32_t m_new[kChunk], c_new = kNoChunk;
-#pragma unroll
-      for (int g = 0; g < kChunk; ++g) m_new[g] = 0;
-      if (more) {
-        c_new = phase1(seq1++, m_new);
-        more = c_new != kNoChunk;
-      }
-      if (it >= (uint32_t)kAhead && cq[0] == kNoChunk) break;     // every claimed chunk is through
-      if (cq[0] != kNoChunk) {
-      const uint32_t chunk_cur = cq[0];
-      const int slot = seq2 % kSlots;
-      const uint32_t slot_parity = (seq2 / kSlots) & 1u;
-      ++seq2;
-      // phase 2 of the oldest chunk: the other warps' totals of its first phase and the chunk's place
-      // in `values` are needed now
+    // Second phase of one chunk (slot: its descriptor, m: its keep-bit words).  false: a wait gave up.
+    auto phase2 = [&](uint32_t chunk, int slot, uint32_t slot_parity, const uint32_t (&m)[kChunk]) -> bool {
+      // the other warps' totals of the first phase and the chunk's place in `values` are needed now
       if (!bar_wait(&sm.cnt_ready[slot], slot_parity, abort_flag) ||
           !bar_wait(&sm.base_ready[slot], slot_parity, abort_flag))
-        break;
+        return false;
       T* const wb = sm.wbuf[warp];
 #pragma unroll
       for (int g = 0; g < kChunk; ++g) {
-        const uint32_t tile = chunk_cur * kChunk + g;
+        const uint32_t tile = chunk * kChunk + g;
         if (tile >= ntiles) break;
         const int s = n % S;
-        const uint32_t mm = mq[0][g];
+        const uint32_t mm = m[g];
         const uint32_t cnt = __popc(mm);
         const uint32_t incl = warp_inclusive_scan(cnt, lane);
         const uint32_t wt = sm.warp_total[slot][g][lane & 7];
@@ -250,15 +249,14 @@ __global__ void __launch_bounds__(kPipeThreads, 3) store_pipelined_kernel(const 
           reinterpret_cast<uint16_t*>(p.keepbits + (int64_t)tile * kTileWords + kBitWords)[r] =
               (uint16_t)(wbase + incl - cnt);
         const int64_t base = sm.tile_base[slot][g];
-        if (!bar_wait(&sm.full[s], (n / S) & 1u, abort_flag)) {
-          ok = false;
-          break;
-        }
+        if (!bar_wait(&sm.full[s], (n / S) & 1u, abort_flag)) return false;
         const T* src = sm.raw[s] + r * kTileCols + wq * 32;
-        // kept entries go to the warp's buffer as they are (bit h of the reversed word is column 31 - h);
-        // scaling waits for the copy to `values`, where every lane has work
+        // Kept entries go to the warp's buffer as they are (bit h of the reversed word is column 31 - h);
+        // scaling waits for the copy to `values`, where every lane has work.  The buffer is filled from
+        // index `odd` on, so that an entry's index in it and its index in `values` have the same parity.
+        const uint32_t odd = wbase & 1u;
         const T* src_end = src + 31;
-        T* dst = wb + (incl - cnt);
+        T* dst = wb + odd + (incl - cnt);
         uint32_t rev = __brev(mm);
         while (rev != 0) {
           uint32_t h;
@@ -279,18 +277,47 @@ __global__ void __launch_bounds__(kPipeThreads, 3) store_pipelined_kernel(const 
         __syncwarp();
         if (lane == 0) bar_arrive(&sm.empty[s]);   // the tile of A is not read again
         if (base >= 0) {
-          T* out = static_cast<T*>(p.values) + base + wbase;
-          for (uint32_t i = lane; i < wtotal; i += 32) out[i] = from_float<T>(raw_to_float(wb[i]) * p.scale);
+          T* out = static_cast<T*>(p.values) + base + wbase - odd;   // even element index: 4-byte aligned for bf16
+          const uint32_t end = odd + wtotal;
+          copy_scaled(wb, out, odd, end, p.scale, lane);
           if (warp == kComputeWarps - 1) {
             // zeros up to the next multiple of kValueAlign after the tile's last value
             const uint32_t total = wbase + wtotal;
             const uint32_t padded = (total + kValueAlign - 1) / kValueAlign * kValueAlign;
-            if (total + lane < padded) out[wtotal + lane] = from_float<T>(0.0f);
+            if (total + lane < padded) out[end + lane] = from_float<T>(0.0f);
           }
         }
         __syncwarp();                             // the staging buffer is rewritten for the next tile
         ++n;
       }
+      return true;
+    };
+
+    // chunks whose first phase is done, oldest first
+    uint32_t mq[kAhead][kChunk], cq[kAhead];
+    uint32_t seq1 = 0, seq2 = 0;                  // chunks handed to the first / second phase so far
+    bool more = true;                             // the loader has not yet said that the work is finished
+#pragma unroll
+    for (int a = 0; a < kAhead; ++a) {
+      cq[a] = kNoChunk;
+#pragma unroll
+      for (int g = 0; g < kChunk; ++g) mq[a][g] = 0;
+    }
+#pragma unroll 1
+    for (uint32_t it = 0;; ++it) {
+      uint32_t m_new[kChunk], c_new = kNoChunk;
+#pragma unroll
+      for (int g = 0; g < kChunk; ++g) m_new[g] = 0;
+      if (more) {
+        c_new = phase1(seq1++, m_new);
+        more = c_new != kNoChunk;
+      }
+      if (cq[0] != kNoChunk) {
+        const bool ok = phase2(cq[0], seq2 % kSlots, (seq2 / kSlots) & 1u, mq[0]);
+        ++seq2;
+        if (!ok) break;
+      } else if (it >= (uint32_t)kAhead) {
+        break;                                    // every claimed chunk is through
       }
 #pragma unroll
       for (int a = 0; a + 1 < kAhead; ++a) {
