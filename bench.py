@@ -42,7 +42,9 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--variant", default="different", choices=["different", "same"])
+    ap.add_argument("--variant", default="different", choices=["different", "same", "project"])
+    ap.add_argument("--law", default="bernoulli", choices=["bernoulli", "replace", "fixed"],
+                    help="sampling law of the different / same variants")
     ap.add_argument("--p", type=float, default=0.1)
     ap.add_argument("--act", default="gelu", choices=["gelu", "relu"])
     ap.add_argument("--batch", type=int, default=BATCH)
@@ -71,7 +73,7 @@ def time_oracle(args, steps, warmup):
     times = []
     for i in range(warmup + steps):
         t0 = time.perf_counter()
-        r = orc.mlp_step(X, y, Ws, bs, act=args.act, dtype="bf16", variant=args.variant, p=args.p, seed=0, step=i)
+        r = orc.mlp_step(X, y, Ws, bs, act=args.act, dtype="bf16", variant=args.variant, p=args.p, seed=0, step=i, law=args.law)
         dt = time.perf_counter() - t0
         if i >= warmup:
             times.append(dt)
@@ -92,7 +94,7 @@ def run_reference(args):
                 warmup=warmup, ms_per_step=mean * 1e3, higher_is_better=True, scaling="weak", vs_baseline=None,
                 dtype="f64", data="synthetic",
                 config=dict(workload="mlp_wide 8192x4->1000 bf16 grid, oracle on a row slab", dims=list(DIMS),
-                            batch=CPU_SLAB_ROWS, variant=args.variant, p=args.p, act=args.act),
+                            batch=CPU_SLAB_ROWS, variant=args.variant, law=args.law, p=args.p, act=args.act),
                 cpu_baseline=base,
                 e2e=dict(value=base["value"], unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
     print(json.dumps(line))
@@ -164,11 +166,11 @@ class ClockSampler:
 class LayerwiseStep:
     """The launches of rad_mlp_step issued call by call, with CUDA events around each kernel family."""
 
-    def __init__(self, rad, torch, dims, B, act, variant, p):
+    def __init__(self, rad, torch, dims, B, act, variant, p, law="bernoulli"):
         self.rad, self.torch, self.dims, self.B, self.act, self.variant, self.p = rad, torch, dims, B, act, variant, p
         L = self.L = len(dims) - 1
         dev, bf = "cuda", torch.bfloat16
-        self.stores = [rad.Store(variant, "bf16", B, dims[l], p, layer=l, relu_bits=False) for l in range(L)]
+        self.stores = [rad.Store(variant, "bf16", B, dims[l], p, layer=l, relu_bits=False, law=law) for l in range(L)]
         hid = max(dims[1:L]) if L > 1 else 8
         self.acts = [torch.empty(B, hid, dtype=bf, device=dev) for _ in range(2)]
         self.dzs = [torch.empty(B, max(dims[1:]), dtype=bf, device=dev) for _ in range(2)]
@@ -391,7 +393,7 @@ def run_ours(args):
           for l in range(L)]
     bs = [torch.zeros(dims[l + 1], device="cuda") for l in range(L)]
 
-    lw = LayerwiseStep(rad, torch, dims, B, args.act, args.variant, args.p)
+    lw = LayerwiseStep(rad, torch, dims, B, args.act, args.variant, args.p, args.law)
 
     def barrier():
         if world > 1:
@@ -432,6 +434,9 @@ def run_ours(args):
         ms_k = sum(t for _, t in dw_big) / len(dw_big)
         if args.variant == "different":
             flops, what = 2.0 * B * 8192 * 8192, "tc_sparse_pair_kernel (different-sample dW), dense-tile flops 2*B*D*H"
+        elif args.variant == "project":
+            k = int(lw.stores[1].nnz[0].item())
+            flops, what = 2.0 * B * k * 8192 + 2.0 * 8192 * k * 8192, "projection dW: S^T dZ and R' G, flops 2*B*k*H + 2*D*k*H"
         else:
             k = int(lw.stores[1].nnz[0].item())
             flops, what = 2.0 * B * k * 8192, "tc_gemm_pair_kernel<MN,MN> (same-sample dW), flops 2*B*k'*H on kept columns"
@@ -443,7 +448,7 @@ def run_ours(args):
     # read grow with the batch and are scaled by B / 8192, the dW output does not grow.  Only the
     # default workload has a capture.
     traffic = None
-    if args.act == "gelu" and abs(args.p - 0.1) < 1e-9:
+    if args.act == "gelu" and abs(args.p - 0.1) < 1e-9 and args.law == "bernoulli":
         if dominant == "dW" and args.variant == "different":
             traffic = int(351.5e6 * B / 8192 + 228.4e6)
         elif dominant != "dW":
@@ -456,18 +461,29 @@ def run_ours(args):
     nnz1 = lw.stores[1].nnz.cpu().numpy()
     if args.variant == "different":
         sbytes = B * 8192 * 2 + int(nnz1[1]) * 2 + B * 8192 // 8 + 4 * len(lw.stores[1].offsets)
+        if args.law != "bernoulli":
+            sbytes += 2 * B * 8192                     # the multiplicity matrix, written and read once
     else:
         sbytes = B * 8192 * 2 + int(nnz1[1]) * 2 + 4 * int(nnz1[0])
     ms_s = sum(store_big) / len(store_big)
-    store_roofline = dict(bound="hbm", kernel="store kernel, one 8192-wide layer input",
-                          achieved=round(sbytes / ms_s / 1e6, 1), peak=pk["hbm_gbs"], unit="GB/s",
-                          frac=round(sbytes / ms_s / 1e6 / pk["hbm_gbs"], 4),
-                          traffic=(int((134.4e6 + 16.6e6) * B / 8192)
-                                   if args.variant == "different" and abs(args.p - 0.1) < 1e-9 else None),
-                          ms_per_launch=round(ms_s, 4), algorithmic_bytes=sbytes)
+    if args.variant == "project":
+        # the store of this variant is a dense contraction (S = A R'), not a streaming kernel
+        sflops = 2.0 * B * 8192 * int(nnz1[0])
+        store_roofline = dict(bound="tensor", kernel="projection store S = A R', flops 2*B*D*k",
+                              achieved=round(sflops / ms_s / 1e9, 1), peak=pk["tflops_sustained"], unit="TFLOP/s",
+                              frac=round(sflops / ms_s / 1e9 / pk["tflops_sustained"], 4), traffic=None,
+                              ms_per_launch=round(ms_s, 4))
+    else:
+        store_roofline = dict(bound="hbm", kernel="store kernel, one 8192-wide layer input",
+                              achieved=round(sbytes / ms_s / 1e6, 1), peak=pk["hbm_gbs"], unit="GB/s",
+                              frac=round(sbytes / ms_s / 1e6 / pk["hbm_gbs"], 4),
+                              traffic=(int((134.4e6 + 16.6e6) * B / 8192)
+                                       if args.variant == "different" and args.law == "bernoulli" and
+                                       abs(args.p - 0.1) < 1e-9 else None),
+                              ms_per_launch=round(ms_s, 4), algorithmic_bytes=sbytes)
 
     # stored activation bytes versus full backprop (from the whole-net entry point's plan)
-    ctx = rad.MLPStep(dims, B, "bf16", args.act, args.variant, args.p)
+    ctx = rad.MLPStep(dims, B, "bf16", args.act, args.variant, args.p, law=args.law)
     s = ctx.stats
     held = s.value_bytes + s.index_bytes + s.relu_bytes + s.preact_bytes + s.unsampled_bytes
     memory = dict(value_bytes=s.value_bytes, index_bytes=s.index_bytes, relu_bytes=s.relu_bytes,
@@ -476,7 +492,7 @@ def run_ours(args):
 
     # the same shapes with ReLU (1-bit derivatives instead of kept pre-activations): plan only, not run
     if args.act != "relu":
-        _, sr = rad.rad_mlp_workspace(dims, B, "bf16", "relu", args.variant, args.p)
+        _, sr = rad.rad_mlp_workspace(dims, B, "bf16", "relu", args.variant, args.p, args.law)
         held_r = sr.value_bytes + sr.index_bytes + sr.relu_bytes + sr.preact_bytes + sr.unsampled_bytes
         memory["same_shapes_relu"] = dict(value_bytes=sr.value_bytes, index_bytes=sr.index_bytes, relu_bytes=sr.relu_bytes,
                                           preact_bytes=sr.preact_bytes, unsampled_bytes=sr.unsampled_bytes,
@@ -560,7 +576,7 @@ def run_ours(args):
                     ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
                     data="synthetic",
                     config=dict(workload="mlp_wide: 8192->8192x4->1000, bf16, batch 65536 per GPU, N(0,1) inputs",
-                                dims=list(dims), global_batch=world * B, act=args.act, variant=args.variant, p=args.p,
+                                dims=list(dims), global_batch=world * B, act=args.act, variant=args.variant, law=args.law, p=args.p,
                                 parallelism="replicas" if world > 1 else "1 GPU",
                                 l2="inputs larger than L2 (1 GiB activations per layer)"),
                     clocks=clocks, e2e=e2e, gpu_launches=int(launches), roofline=roofline,
