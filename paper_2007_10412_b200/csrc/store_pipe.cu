@@ -3,16 +3,18 @@
 //
 // A CTA claims chunks of kChunk consecutive 64 x 128 tiles in ticket order and runs two phases per
 // chunk, the first phase kAhead chunks ahead of the second:
-//   phase 1  needs no data: every compute thread draws the 32 keep decisions of one keep-bit word
-//            per tile (two Philox calls), writes the word, and the warp totals go to shared memory;
+//   phase 1  needs no data: the eight compute warps work on two tiles side by side, four warps each; a
+//            thread draws the 64 keep decisions of two adjacent keep-bit words of a row (four Philox
+//            calls), writes the words, and the warp totals go to shared memory;
 //   look-back a service warp adds the chunk's padded and exact counts, publishes them, and finds where
 //            the chunk starts in `values` from the chunks before it (decoupled look-back over one
 //            status word per chunk);
 //   phase 2  the tile of A arrives in shared memory by TMA (a second service warp runs a ring of
 //            loads ahead of the compute warps); a warp scan over the counts gives every word its
-//            place in (row, column) order; each thread walks the set bits of its word and scales the
-//            kept entries into its warp's staging buffer, which the warp then copies to `values`
-//            with coalesced stores.  No compute warp waits for another one in this phase.
+//            place in (row, column) order; each thread walks the set bits of its two words and copies
+//            the kept entries into its warp's staging buffer, which the warp then writes to `values`
+//            with coalesced stores, scaling on the way.  No compute warp waits for another one in
+//            this phase.
 // The look-back of a chunk therefore has kAhead chunk periods to finish in.
 // The layout produced is the one of the generic kernel: the order of tiles in `values` is the tile index.
 //
@@ -27,7 +29,9 @@ namespace rad {
 namespace {
 
 constexpr int kChunk = 8;                       // tiles per claimed chunk
-constexpr int kComputeWarps = 8;                // 256 threads: one keep-bit word of a tile each
+constexpr int kComputeWarps = 8;
+constexpr int kWarpsPerTile = 4;                // 128 threads per tile: two keep-bit words (64 columns of a row) each
+constexpr int kTilesPerStep = kComputeWarps / kWarpsPerTile;   // tiles the compute warps work on side by side
 constexpr int kLoaderWarp = kComputeWarps;      // the look-back warp is the last one
 constexpr int kPipeThreads = (kComputeWarps + 2) * 32;
 constexpr int kAhead = 2;                       // chunks between the first and the second phase
@@ -36,17 +40,17 @@ constexpr int kLookWindows = 8;                 // look-back: 32 status words pe
 constexpr uint32_t kNoChunk = 0xffffffffu;
 constexpr uint64_t kPipeWaitLimitNs = 2000000000ull;
 constexpr int kTileElems = kTileRows * kTileCols;
-constexpr int kWarpElems = kTileElems / kComputeWarps;   // entries of a tile that one warp owns
+constexpr int kWarpElems = kTileElems / kWarpsPerTile;   // entries of a tile that one warp owns (16 rows)
 
 template <typename T, int S>
 struct PipeSmem {
   alignas(128) T raw[S][kTileElems];            // tiles of A as loaded
-  alignas(16) T wbuf[kComputeWarps][kWarpElems + 8];   // kept values of a warp's eight rows, in order (from index 0 or 1)
+  alignas(16) T wbuf[kComputeWarps][kWarpElems + 8];   // kept values of a warp's sixteen rows, in order (from index 0 or 1)
   uint64_t full[S], empty[S];                   // raw ring
   uint64_t chunk_ready[kSlots], cnt_ready[kSlots], base_ready[kSlots];
   uint32_t chunk_id[kSlots];
   uint32_t tile_slab[kSlots][kChunk], tile_cb[kSlots][kChunk];   // row slab and column block of each tile
-  uint32_t warp_total[kSlots][kChunk][kComputeWarps];
+  uint32_t warp_total[kSlots][kChunk][kWarpsPerTile];
   uint32_t tile_total[kSlots][kChunk];
   int64_t tile_base[kSlots][kChunk];            // first element in `values`; -1: do not write
   int abort_flag;
@@ -166,7 +170,7 @@ __device__ __forceinline__ void copy_scaled(const bf16* wb, bf16* out, uint32_t 
 }
 
 template <typename T, int S>
-__global__ void __launch_bounds__(kPipeThreads, 3) store_pipelined_kernel(const StoreParams p, const PhiloxKeys ks,
+__global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const StoreParams p, const PhiloxKeys ks,
                                                                       const __grid_constant__ CUtensorMap tmA) {
   extern __shared__ unsigned char smem_raw[];
   PipeSmem<T, S>& sm = *reinterpret_cast<PipeSmem<T, S>*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
@@ -176,7 +180,7 @@ __global__ void __launch_bounds__(kPipeThreads, 3) store_pipelined_kernel(const 
   const uint32_t nchunks = (ntiles + kChunk - 1) / kChunk;
 
   if (tid == 0) {
-    for (int s = 0; s < S; ++s) { bar_init(&sm.full[s], 1); bar_init(&sm.empty[s], kComputeWarps); }
+    for (int s = 0; s < S; ++s) { bar_init(&sm.full[s], 1); bar_init(&sm.empty[s], kWarpsPerTile); }
     for (int q = 0; q < kSlots; ++q) {
       bar_init(&sm.chunk_ready[q], 1);
       bar_init(&sm.cnt_ready[q], kComputeWarps);
@@ -189,38 +193,46 @@ __global__ void __launch_bounds__(kPipeThreads, 3) store_pipelined_kernel(const 
 
   if (warp < kComputeWarps) {
     // ---------------------------------------------------------------------------------------------
-    // compute warps.  Thread (warp, lane) owns keep-bit word warp * 32 + lane of every tile: row
-    // 8 * warp + lane / 4 of the tile, columns 32 * (lane % 4) .. + 31.
+    // compute warps.  Warps 0-3 take the even tiles of a chunk, warps 4-7 the odd ones.  Within a tile
+    // warp v owns rows 16 v .. 16 v + 15 and lane l row 16 v + l / 2, columns 64 (l % 2) .. + 63: keep-bit
+    // words 4 row + 2 (l % 2) and the next one.  Lane order is (row, column) order.
     // ---------------------------------------------------------------------------------------------
-    const int r = warp * 8 + (lane >> 2), wq = lane & 3;
+    const int side = warp / kWarpsPerTile, v = warp % kWarpsPerTile, half = lane & 1;
+    const int r = v * 16 + (lane >> 1);
     const uint32_t nrows = (uint32_t)p.B, ncols = (uint32_t)p.D;   // B * D < 2^32 (checked by the host)
     uint32_t n = 0;                               // tiles this CTA has worked through (ring position)
 
+    // m[2 i], m[2 i + 1]: this thread's two words of its tile in step i of the chunk
     auto phase1 = [&](uint32_t seq, uint32_t (&m)[kChunk]) -> uint32_t {
       const int slot = seq % kSlots;
       if (!bar_wait(&sm.chunk_ready[slot], (seq / kSlots) & 1u, abort_flag)) return kNoChunk;
       const uint32_t chunk = sm.chunk_id[slot];
       if (chunk == kNoChunk) return kNoChunk;
 #pragma unroll
-      for (int g = 0; g < kChunk; ++g) {
+      for (int i = 0; i < kChunk / kTilesPerStep; ++i) {
+        const int g = kTilesPerStep * i + side;
         const uint32_t tile = chunk * kChunk + g;
-        uint32_t mm = 0;
+        uint32_t m0 = 0, m1 = 0;
         if (tile < ntiles) {
           const uint32_t row = sm.tile_slab[slot][g] * kTileRows + r;
-          const uint32_t col0 = sm.tile_cb[slot][g] * kTileCols + wq * 32;
+          const uint32_t col0 = sm.tile_cb[slot][g] * kTileCols + half * 64;
           if (row < nrows && col0 < ncols) {
             const uint32_t g16 = col0 >> 4;
-            const uint32_t lo = philox_keep16(g16, row, p.c2, p.c3, ks, p.T);
-            const uint32_t hi = philox_keep16(g16 + 1u, row, p.c2, p.c3, ks, p.T);
-            mm = lo | (hi << 16);
-            const uint32_t nv = ncols - col0;
-            if (nv < 32) mm &= (1u << nv) - 1u;
+            m0 = philox_keep16(g16, row, p.c2, p.c3, ks, p.T) | (philox_keep16(g16 + 1u, row, p.c2, p.c3, ks, p.T) << 16);
+            m1 = philox_keep16(g16 + 2u, row, p.c2, p.c3, ks, p.T) | (philox_keep16(g16 + 3u, row, p.c2, p.c3, ks, p.T) << 16);
+            const uint32_t nv = ncols - col0;     // valid columns from col0 on
+            if (nv < 64) {
+              m0 &= nv >= 32 ? 0xffffffffu : (1u << nv) - 1u;
+              m1 &= nv <= 32 ? 0u : (1u << (nv - 32)) - 1u;
+            }
           }
-          p.keepbits[tile * (uint32_t)kTileWords + (uint32_t)(warp * 32 + lane)] = mm;
+          *reinterpret_cast<uint2*>(p.keepbits + (tile * (uint32_t)kTileWords + (uint32_t)(r * 4 + half * 2))) =
+              make_uint2(m0, m1);
         }
-        m[g] = mm;
-        const uint32_t wt = __reduce_add_sync(0xffffffffu, __popc(mm));
-        if (lane == 0) sm.warp_total[slot][g][warp] = wt;
+        m[2 * i] = m0;
+        m[2 * i + 1] = m1;
+        const uint32_t wt = __reduce_add_sync(0xffffffffu, __popc(m0) + __popc(m1));
+        if (lane == 0) sm.warp_total[slot][g][v] = wt;
       }
       __syncwarp();
       if (lane == 0) bar_arrive(&sm.cnt_ready[slot]);
@@ -234,44 +246,53 @@ __global__ void __launch_bounds__(kPipeThreads, 3) store_pipelined_kernel(const 
           !bar_wait(&sm.base_ready[slot], slot_parity, abort_flag))
         return false;
       T* const wb = sm.wbuf[warp];
+      const uint32_t valid = min((uint32_t)kChunk, ntiles - chunk * kChunk);   // tiles of this chunk
 #pragma unroll
-      for (int g = 0; g < kChunk; ++g) {
+      for (int i = 0; i < kChunk / kTilesPerStep; ++i) {
+        const int g = kTilesPerStep * i + side;
+        if ((uint32_t)g >= valid) break;
         const uint32_t tile = chunk * kChunk + g;
-        if (tile >= ntiles) break;
-        const int s = n % S;
-        const uint32_t mm = m[g];
-        const uint32_t cnt = __popc(mm);
+        const uint32_t pos = n + g;               // the tile's place in the ring of loads
+        const int s = pos % S;
+        const uint32_t m0 = m[2 * i], m1 = m[2 * i + 1];
+        const uint32_t cnt = __popc(m0) + __popc(m1);
         const uint32_t incl = warp_inclusive_scan(cnt, lane);
-        const uint32_t wt = sm.warp_total[slot][g][lane & 7];
-        const uint32_t wbase = __reduce_add_sync(0xffffffffu, lane < warp ? wt : 0u);
+        const uint32_t wt = sm.warp_total[slot][g][lane & 3];
+        const uint32_t wbase = __reduce_add_sync(0xffffffffu, lane < v ? wt : 0u);
         const uint32_t wtotal = __shfl_sync(0xffffffffu, incl, 31);
-        if (wq == 0)
+        if (half == 0)
           reinterpret_cast<uint16_t*>(p.keepbits + (int64_t)tile * kTileWords + kBitWords)[r] =
               (uint16_t)(wbase + incl - cnt);
         const int64_t base = sm.tile_base[slot][g];
-        if (!bar_wait(&sm.full[s], (n / S) & 1u, abort_flag)) return false;
-        const T* src = sm.raw[s] + r * kTileCols + wq * 32;
-        // Kept entries go to the warp's buffer as they are (bit h of the reversed word is column 31 - h);
+        if (!bar_wait(&sm.full[s], (pos / S) & 1u, abort_flag)) return false;
+        const T* src = sm.raw[s] + r * kTileCols + half * 64;
+        // Kept entries go to the warp's buffer as they are (bit h of a reversed word is column 31 - h);
         // scaling waits for the copy to `values`, where every lane has work.  The buffer is filled from
         // index `odd` on, so that an entry's index in it and its index in `values` have the same parity.
+        // One loop serves both words: it runs as long as the fullest pair of words of the warp.
         const uint32_t odd = wbase & 1u;
         const T* src_end = src + 31;
         T* dst = wb + odd + (incl - cnt);
-        uint32_t rev = __brev(mm);
+        uint32_t rev = __brev(m0), rev_next = __brev(m1);
+        if (rev == 0) { rev = rev_next; rev_next = 0; src_end += 32; }
         while (rev != 0) {
           uint32_t h;
           asm("bfind.u32 %0, %1;" : "=r"(h) : "r"(rev));
           rev &= ~(1u << h);
           *dst++ = *(src_end - h);
+          if (rev == 0) { rev = rev_next; rev_next = 0; src_end += 32; }
         }
         if (p.relubits != nullptr) {
           const uint32_t row = sm.tile_slab[slot][g] * kTileRows + r;
-          const uint32_t word = sm.tile_cb[slot][g] * 4 + wq;
-          if (row < nrows && word < (uint32_t)p.w32) {
-            uint32_t rb = positive32(src);
-            const uint32_t nv = ncols - word * 32;
-            if (nv < 32) rb &= (1u << nv) - 1u;
-            p.relubits[(int64_t)row * p.w32 + word] = rb;
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            const uint32_t word = sm.tile_cb[slot][g] * 4 + half * 2 + j;
+            if (row < nrows && word < (uint32_t)p.w32) {
+              uint32_t rb = positive32(src + 32 * j);
+              const uint32_t nv = ncols - word * 32;
+              if (nv < 32) rb &= (1u << nv) - 1u;
+              p.relubits[(int64_t)row * p.w32 + word] = rb;
+            }
           }
         }
         __syncwarp();
@@ -280,7 +301,7 @@ __global__ void __launch_bounds__(kPipeThreads, 3) store_pipelined_kernel(const 
           T* out = static_cast<T*>(p.values) + base + wbase - odd;   // even element index: 4-byte aligned for bf16
           const uint32_t end = odd + wtotal;
           copy_scaled(wb, out, odd, end, p.scale, lane);
-          if (warp == kComputeWarps - 1) {
+          if (v == kWarpsPerTile - 1) {
             // zeros up to the next multiple of kValueAlign after the tile's last value
             const uint32_t total = wbase + wtotal;
             const uint32_t padded = (total + kValueAlign - 1) / kValueAlign * kValueAlign;
@@ -288,8 +309,8 @@ __global__ void __launch_bounds__(kPipeThreads, 3) store_pipelined_kernel(const 
           }
         }
         __syncwarp();                             // the staging buffer is rewritten for the next tile
-        ++n;
       }
+      n += valid;
       return true;
     };
 
@@ -397,20 +418,16 @@ __global__ void __launch_bounds__(kPipeThreads, 3) store_pipelined_kernel(const 
       const uint32_t chunk = sm.chunk_id[slot];
       if (chunk == kNoChunk) return kNoChunk;
       if (!bar_wait(&sm.cnt_ready[slot], par, abort_flag, 400)) return kNoChunk;
-      // lane (8 g + w) reads warp w's totals of tiles g and g + 4; a butterfly over eight lanes sums a tile
-      static_assert(kChunk == 8 && kComputeWarps == 8, "two (tile, warp) entries per lane");
-      uint32_t t0 = sm.warp_total[slot][lane >> 3][lane & 7];
-      uint32_t t1 = sm.warp_total[slot][4 + (lane >> 3)][lane & 7];
-#pragma unroll
-      for (int o = 1; o < 8; o <<= 1) {
-        t0 += __shfl_xor_sync(0xffffffffu, t0, o);
-        t1 += __shfl_xor_sync(0xffffffffu, t1, o);
-      }
+      // lane (4 g + v) reads warp v's total of tile g; a butterfly over four lanes sums a tile
+      static_assert(kChunk * kWarpsPerTile == 32, "one (tile, warp) entry per lane");
+      uint32_t t = sm.warp_total[slot][lane >> 2][lane & 3];
+      t += __shfl_xor_sync(0xffffffffu, t, 1);
+      t += __shfl_xor_sync(0xffffffffu, t, 2);
       c.chunk_gran = 0;
       c.chunk_exact = 0;
 #pragma unroll
       for (int g = 0; g < kChunk; ++g) {
-        c.tot[g] = __shfl_sync(0xffffffffu, g < 4 ? t0 : t1, 8 * (g & 3));
+        c.tot[g] = __shfl_sync(0xffffffffu, t, 4 * g);
         c.chunk_gran += (c.tot[g] + kValueAlign - 1) / kValueAlign;
         c.chunk_exact += c.tot[g];
       }
@@ -542,6 +559,7 @@ int launch_typed(const StoreParams& p, const PhiloxKeys& ks, const CUtensorMap& 
 int launch_store_pipelined(const StoreParams& p, const PhiloxKeys& ks, int dtype, cudaStream_t s) {
   const size_t esz = dtype == RAD_BF16 ? 2 : 4;
   if (((uintptr_t)p.A & 15) != 0 || ((size_t)p.lda * esz) % 16 != 0) return RAD_EUNSUPPORTED;
+  if (((uintptr_t)p.keepbits & 7) != 0) return RAD_EUNSUPPORTED;   // keep-bit words leave in pairs
   EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(tensor_map_encoder());
   if (fn == nullptr) return RAD_EUNSUPPORTED;
   CUtensorMap map;
@@ -554,8 +572,8 @@ int launch_store_pipelined(const StoreParams& p, const PhiloxKeys& ks, int dtype
                         CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return RAD_EUNSUPPORTED;
-  if (dtype == RAD_BF16) return launch_typed<bf16, 3>(p, ks, map, s);
-  return launch_typed<float, 2>(p, ks, map, s);
+  if (dtype == RAD_BF16) return launch_typed<bf16, 4>(p, ks, map, s);
+  return launch_typed<float, 3>(p, ks, map, s);
 }
 
 }  // namespace rad
