@@ -172,6 +172,9 @@ __device__ __forceinline__ void copy_scaled(const bf16* wb, bf16* out, uint32_t 
 template <typename T, int S>
 __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const StoreParams p, const PhiloxKeys ks,
                                                                       const __grid_constant__ CUtensorMap tmA) {
+  // A stage of the ring must always serve the same half of the compute warps: a waiter tells the phases of
+  // a barrier apart by one parity bit, which only works if it has itself waited for the phase before.
+  static_assert(S % kTilesPerStep == 0, "stages and tiles worked on side by side");
   extern __shared__ unsigned char smem_raw[];
   PipeSmem<T, S>& sm = *reinterpret_cast<PipeSmem<T, S>*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -573,7 +576,7 @@ int launch_store_pipelined(const StoreParams& p, const PhiloxKeys& ks, int dtype
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return RAD_EUNSUPPORTED;
   if (dtype == RAD_BF16) return launch_typed<bf16, 4>(p, ks, map, s);
-  return launch_typed<float, 3>(p, ks, map, s);
+  return launch_typed<float, 4>(p, ks, map, s);
 }
 
 }  // namespace rad
