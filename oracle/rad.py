@@ -19,13 +19,17 @@ R = diag(sqrt(m / p_eff)) restricted to kept columns.  "different sample"
 draws m per minibatch row, "same sample" draws one m per layer and step
 (Sec. 4.3).
 
-The keep decision for (row b, column d) compares one byte of a
-Philox-4x32-10 output with a threshold T = round(p * 2^8) clipped to
-[1, 2^8]; p_eff = T / 2^8 and stored values are scaled by fl32(2^8 / T) so
-the estimator is exactly unbiased for the probability actually sampled.  The
-paper leaves the source of randomness open; one byte per decision lets one
-128-bit generator output decide sixteen entries, and the keep probabilities
-the paper uses (0.05 ... 0.5) move by less than 2 % of their value.
+The keep decision for (row b, column d) compares a byte u with a threshold
+T = round(p * 2^8) clipped to [1, 2^8]: kept iff u < T; p_eff = T / 2^8 and
+stored values are scaled by fl32(2^8 / T), so the estimator is exactly unbiased
+for the probability actually sampled.  The paper leaves the source of
+randomness open.  The bytes of 32 consecutive columns are laid across the
+eight words of two Philox-4x32-10 outputs, one bit plane per word: bit d % 32
+of word i holds (complemented) bit 7 - i of the byte of column d.  A device
+then gets the 32 decisions of a keep-bit word from eight word-wide AND / OR
+steps along the binary digits of T instead of 32 byte compares.  The keep
+probabilities the paper uses (0.05 ... 0.5) move by less than 2 % of their
+value.
 
 Second sampling law, the paper's own (Sec. 3.2, App. A): k = ceil(fraction * d)
 coordinates drawn uniformly WITH replacement, P = (d / k) sum_s e_s e_s^T, so a
@@ -57,7 +61,7 @@ STREAM_DIFFERENT_FIXED = 4     # k distinct columns, per row
 STREAM_SAME_FIXED = 5          # k distinct columns, shared by the minibatch
 STREAM_PROJECT = 6             # signs of the Rademacher projection
 LANE_BITS = 8
-LANES_PER_CALL = 16      # 128 output bits / 8
+COLUMNS_PER_GROUP = 32   # one keep-bit word: two generator outputs (256 bits), eight bit planes of 32 columns
 LANE_RANGE = 1 << LANE_BITS
 
 
@@ -81,32 +85,41 @@ def scale_factor(p) -> np.float32:
     return np.float32(LANE_RANGE) / np.float32(keep_threshold(p))
 
 
-def keep_mask(variant: str, B: int, D: int, p, seed: int, layer: int, step: int) -> np.ndarray:
-    """Boolean B x D keep mask.
+def _decision_bytes(group, rows, stream, seed, layer, step):
+    """Bytes u of the 32 columns of each (row, group): shape rows x groups x 32, uint32 in [0, 256).
 
-    Counter = (d // 16, row, layer | stream << 24, step), key = (seed low word,
-    seed high word).  The sixteen bytes of the output, words in order and
-    least significant byte first, are the lanes of columns 16*(d//16) + 0..15:
-    column d reads byte d % 4 of word (d % 16) // 4.  For "same" the row field
-    is 0 and the single row of decisions is shared by every minibatch element.
+    Outputs of the generator for counters (2 * group, row, layer | stream << 24, step) and
+    (2 * group + 1, ...), key = (seed low word, seed high word), give words w_0 .. w_7 (first
+    output first).  Column c of the group has u = sum_i (1 - bit c of w_i) << (7 - i).
     """
+    c2 = np.uint64((layer & 0xFFFFFF) | (stream << 24))
+    k0, k1 = np.uint64(seed & 0xFFFFFFFF), np.uint64((seed >> 32) & 0xFFFFFFFF)
+    words = []
+    for j in range(2):
+        words.extend(philox4x32_10(np.uint64(2) * group + np.uint64(j), rows, c2, np.uint64(step & 0xFFFFFFFF), k0, k1))
+    shape = np.broadcast(group, rows).shape
+    u = np.zeros(shape + (COLUMNS_PER_GROUP,), dtype=np.uint32)
+    cols = np.arange(COLUMNS_PER_GROUP, dtype=np.uint32)
+    for i, w in enumerate(words):
+        bits = (np.broadcast_to(w, shape)[..., None] >> cols) & np.uint32(1)
+        u |= (np.uint32(1) - bits) << np.uint32(7 - i)
+    return u
+
+
+def keep_mask(variant: str, B: int, D: int, p, seed: int, layer: int, step: int) -> np.ndarray:
+    """Boolean B x D keep mask: column d of row b is kept iff its byte (see _decision_bytes, group d // 32,
+    column d % 32 of the group) is below T.  For "same" the row field of the counter is 0 and the single
+    row of decisions is shared by every minibatch element."""
     T = keep_threshold(p)
-    groups = (D + LANES_PER_CALL - 1) // LANES_PER_CALL
+    groups = (D + COLUMNS_PER_GROUP - 1) // COLUMNS_PER_GROUP
     if variant == "different":
         rows, stream = np.arange(B, dtype=np.uint64)[:, None], STREAM_DIFFERENT
     elif variant == "same":
         rows, stream = np.zeros((1, 1), dtype=np.uint64), STREAM_SAME
     else:
         raise ValueError(variant)
-    c0 = np.arange(groups, dtype=np.uint64)[None, :]
-    c2 = np.uint64((layer & 0xFFFFFF) | (stream << 24))
-    words = philox4x32_10(c0, rows, c2, np.uint64(step & 0xFFFFFFFF),
-                          np.uint64(seed & 0xFFFFFFFF), np.uint64((seed >> 32) & 0xFFFFFFFF))
-    lanes = np.empty(words[0].shape + (LANES_PER_CALL,), dtype=np.uint32)
-    for j, w in enumerate(words):
-        for k in range(4):
-            lanes[..., 4 * j + k] = (w >> np.uint32(8 * k)) & np.uint32(0xFF)
-    m = (lanes < T).reshape(lanes.shape[0], groups * LANES_PER_CALL)[:, :D]
+    u = _decision_bytes(np.arange(groups, dtype=np.uint64)[None, :], rows, stream, seed, layer, step)
+    m = (u < T).reshape(u.shape[0], groups * COLUMNS_PER_GROUP)[:, :D]
     if variant == "same":
         m = np.broadcast_to(m, (B, D))
     return np.ascontiguousarray(m)
@@ -114,7 +127,7 @@ def keep_mask(variant: str, B: int, D: int, p, seed: int, layer: int, step: int)
 
 def keep_mask_at(variant: str, rows, cols, p, seed: int, layer: int, step: int) -> np.ndarray:
     """Keep decisions of the given rows x the given columns (len(rows) x len(cols), boolean): the same
-    counter, key and lane rule as keep_mask, evaluated only where asked, so that single tiles or
+    counter, key and byte rule as keep_mask, evaluated only where asked, so that single tiles or
     single columns of a layer too large to expand in full can be checked."""
     T = keep_threshold(p)
     rows = np.asarray(rows, dtype=np.uint64).reshape(-1, 1)
@@ -125,17 +138,10 @@ def keep_mask_at(variant: str, rows, cols, p, seed: int, layer: int, step: int) 
         rows, stream = np.zeros_like(rows), STREAM_SAME
     else:
         raise ValueError(variant)
-    c2 = np.uint64((layer & 0xFFFFFF) | (stream << 24))
-    words = philox4x32_10(cols // np.uint64(LANES_PER_CALL) + np.zeros_like(rows), rows + np.zeros_like(cols), c2,
-                          np.uint64(step & 0xFFFFFFFF), np.uint64(seed & 0xFFFFFFFF),
-                          np.uint64((seed >> 32) & 0xFFFFFFFF))
-    lane = (cols % np.uint64(LANES_PER_CALL)).astype(np.int64) + np.zeros(rows.shape, dtype=np.int64)
-    out = np.zeros(lane.shape, dtype=bool)
-    for j, w in enumerate(words):
-        w = np.broadcast_to(w, lane.shape)
-        for k in range(4):
-            out |= (lane == 4 * j + k) & (((w >> np.uint32(8 * k)) & np.uint32(0xFF)) < T)
-    return out
+    u = _decision_bytes(cols // np.uint64(COLUMNS_PER_GROUP) + np.zeros_like(rows), rows + np.zeros_like(cols), stream,
+                        seed, layer, step)                                  # rows x cols x 32
+    pick = (cols % np.uint64(COLUMNS_PER_GROUP)).astype(np.int64) + np.zeros(rows.shape, dtype=np.int64)
+    return np.take_along_axis(u, pick[..., None], axis=-1)[..., 0] < T
 
 
 # --------------------------------------------------------------------------

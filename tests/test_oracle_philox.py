@@ -107,9 +107,9 @@ def test_keep_mask_at_agrees_with_the_full_mask(variant):
 
 
 @pytest.mark.parametrize("variant", ["different", "same"])
-def test_lane_of_a_column_is_its_byte_of_the_128_bit_output(variant):
-    """Column d is decided by byte d % 16 of the generator output for counter d // 16, the output read
-    as sixteen bytes, words in order and least significant byte first; restated here with Python
+def test_byte_of_a_column_is_laid_across_the_eight_words_of_two_outputs(variant):
+    """Column d is decided by the byte whose bit 7 - i is the complement of bit d % 32 of word i of the
+    two generator outputs for counters 2 (d // 32) and 2 (d // 32) + 1; restated here with Python
     integers, independent of the array code in the oracle."""
     B, D, p, seed, layer, step = 5, 77, 0.3, 0xABCDEF0123456789, 6, 11
     T = orc.keep_threshold(p)
@@ -117,8 +117,18 @@ def test_lane_of_a_column_is_its_byte_of_the_128_bit_output(variant):
     full = orc.keep_mask(variant, B, D, p, seed, layer, step)
     stream = 0 if variant == "different" else 1
     for b in range(B):
+        row = b if variant == "different" else 0
         for d in range(D):
-            out = bigint_philox([d // 16, b if variant == "different" else 0, layer | stream << 24, step],
-                                [seed & MASK, seed >> 32])
-            octets = b"".join(int(w).to_bytes(4, "little") for w in out)
-            assert bool(full[b, d]) == (octets[d % 16] < T)
+            words = []
+            for j in range(2):
+                words += bigint_philox([2 * (d // 32) + j, row, layer | stream << 24, step], [seed & MASK, seed >> 32])
+            u = sum((1 - ((w >> (d % 32)) & 1)) << (7 - i) for i, w in enumerate(words))
+            assert bool(full[b, d]) == (u < T)
+
+
+def test_decision_bytes_are_uniform():
+    u = orc._decision_bytes(np.arange(64, dtype=np.uint64)[None, :], np.arange(64, dtype=np.uint64)[:, None], 0, 42, 2, 0)
+    hist = np.bincount(u.reshape(-1), minlength=256).astype(np.float64)
+    expected = u.size / 256.0
+    chi2 = ((hist - expected) ** 2 / expected).sum()
+    assert abs(chi2 - 255.0) < 6 * 22.6
