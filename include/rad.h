@@ -60,13 +60,17 @@ typedef enum { RAD_ACT_NONE = 0, RAD_ACT_RELU = 1, RAD_ACT_GELU = 2 } rad_act;
 
 /*
  * The mask (Sec. 3.2: a random P with E[P] = I; Sec. 4.3: "same sample" /
- * "different sample").  Entry (b, d) is kept iff one byte of a
- * Philox-4x32-10 output is below T = clamp(rint(p * 256), 1, 256):
+ * "different sample").  Entry (b, d) is kept iff its byte u is below
+ * T = clamp(rint(p * 256), 1, 256):
  *   key     = (seed & 0xffffffff, seed >> 32)
- *   counter = (d / 16, row, layer | stream << 24, step), row = b and stream = 0
- *             for different-sample; row = 0 and stream = 1 for same-sample
- *   byte of column d = byte d % 4 (least significant first) of output word
- *             (d % 16) / 4: one 128-bit output decides sixteen columns.
+ *   words   = w_0 .. w_3 from the Philox-4x32-10 output for counter
+ *             (2 * (d / 32), row, layer | stream << 24, step), w_4 .. w_7 from the
+ *             output for counter (2 * (d / 32) + 1, ...); row = b and stream = 0
+ *             for different-sample, row = 0 and stream = 1 for same-sample
+ *   u       = sum over i of (1 - bit (d % 32) of w_i) << (7 - i): the bytes of 32
+ *             columns lie across the eight words, one bit plane per word, so a
+ *             keep-bit word follows from eight AND / OR steps along the binary
+ *             digits of T.
  * p_eff = T / 256 is the probability actually sampled and kept values are
  * multiplied by fl32(256 / T) = 1 / p_eff, so E[A_hat] = A exactly.
  */

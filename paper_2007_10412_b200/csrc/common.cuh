@@ -65,40 +65,36 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
   out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
-// One keep decision per output byte: a 128-bit output decides sixteen consecutive columns, column i
-// of the sixteen reading byte i % 4 of word i / 4; it is kept iff the byte is below T (1..256).
+// An entry is kept iff its byte u is below T (1..256).  The bytes of 32 consecutive columns are laid
+// across the eight words w_0 .. w_7 of two generator outputs, one bit plane per word: bit c of w_i is the
+// complement of bit 7 - i of the byte of column c.  Comparing from the least significant digit of T
+// upwards, "u < T so far" becomes (w_i | x) where the digit of T is 1 and (w_i & x) where it is 0, so the 32
+// decisions of a keep-bit word are eight three-input logic operations, no compares.
 constexpr uint32_t kLaneRange = 256;
 
 struct KeepThreshold {
-  uint32_t y;    // T - 1 in every byte
-  uint32_t y1;   // y with the top bit of every byte set
+  uint32_t digit[8];   // digit[i]: all ones if bit 7 - i of T is set (T = 256: all set)
+  uint32_t start;      // decisions before any digit: none kept, or all kept for T = 256
 };
 inline KeepThreshold make_keep_threshold(uint32_t T) {
   KeepThreshold k;
-  k.y = ((T - 1u) & 0xffu) * 0x01010101u;
-  k.y1 = k.y | 0x80808080u;
+  for (int i = 0; i < 8; ++i) k.digit[i] = (T >= kLaneRange || ((T >> (7 - i)) & 1u)) ? 0xffffffffu : 0u;
+  k.start = T >= kLaneRange ? 0xffffffffu : 0u;
   return k;
 }
 
-// Top bit of every byte of the result: byte of x <= byte of y.  The low seven bits are compared by a
-// subtraction that cannot borrow across bytes (the minuend's top bits are set, the subtrahend's
-// cleared); the top bits decide where they differ.
-__device__ __forceinline__ uint32_t bytes_le(uint32_t x, const KeepThreshold& k) {
-  const uint32_t d = k.y1 - (x & 0x7f7f7f7fu);
-  return ((~x & k.y) | (~(x ^ k.y) & d)) & 0x80808080u;
-}
-
-// Keep bits of the 16 columns of one counter, bit i = column i.  The multiplication moves the four
-// flag bits of a word (bits 7, 15, 23, 31) to bits 28..31 (all partial products land on distinct
-// bits, so nothing carries); the funnel shift appends that nibble.
-__device__ __forceinline__ uint32_t philox_keep16(uint32_t group, uint32_t row, uint32_t c2, uint32_t c3,
+// Keep bits of columns 32 * group32 .. + 31 of one row: bit c = column c of the group.
+__device__ __forceinline__ uint32_t philox_keep32(uint32_t group32, uint32_t row, uint32_t c2, uint32_t c3,
                                                   const PhiloxKeys& ks, const KeepThreshold& k) {
-  uint32_t w[4];
-  philox4x32_10(group, row, c2, c3, ks, w);
-  uint32_t m = 0;
+  uint32_t lo[4], hi[4];
+  philox4x32_10(2u * group32, row, c2, c3, ks, lo);
+  philox4x32_10(2u * group32 + 1u, row, c2, c3, ks, hi);
+  uint32_t x = k.start;
 #pragma unroll
-  for (int j = 3; j >= 0; --j) m = __funnelshift_l(bytes_le(w[j], k) * 0x00204081u, m, 4);
-  return m;
+  for (int i = 3; i >= 0; --i) x = (hi[i] & x) | ((hi[i] | x) & k.digit[4 + i]);
+#pragma unroll
+  for (int i = 3; i >= 0; --i) x = (lo[i] & x) | ((lo[i] | x) & k.digit[i]);
+  return x;
 }
 
 // Host-side twins of the threshold arithmetic (double rint, one float32 division).

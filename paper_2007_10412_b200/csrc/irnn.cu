@@ -68,9 +68,9 @@ __global__ void __launch_bounds__(kRnnThreads) irnn_forward_kernel(const RnnPara
     if (warp == 4) {
       // store of h_{t-1}: keep bits of the step, kept entries scaled and appended to the row's values
       uint32_t m = 0;
-      if (lane * 16 < Hd) {                          // one draw decides sixteen units
-        const int nvalid = min(16, Hd - lane * 16);
-        m = philox_keep16((uint32_t)lane, mask_row, p.c2, p.step0 + (uint32_t)t, ks, p.keepT) & (0xffffu >> (16 - nvalid));
+      if (lane * 32 < Hd) {                          // one keep-bit word decides 32 units
+        const int nvalid = min(32, Hd - lane * 32);
+        m = philox_keep32((uint32_t)lane, mask_row, p.c2, p.step0 + (uint32_t)t, ks, p.keepT) & (0xffffffffu >> (32 - nvalid));
       }
       const uint32_t c = __popc(m);
       uint32_t incl = c;
@@ -83,15 +83,13 @@ __global__ void __launch_bounds__(kRnnThreads) irnn_forward_kernel(const RnnPara
       uint32_t pos = off + incl - c;
       if ((int64_t)off + total <= p.cap_row) {
 #pragma unroll
-        for (int i = 0; i < 16; ++i)
-          if ((m >> i) & 1u) p.values[b * p.cap_row + pos++] = hc[lane * 16 + i] * p.scale;
+        for (int i = 0; i < 32; ++i)
+          if ((m >> i) & 1u) p.values[b * p.cap_row + pos++] = hc[lane * 32 + i] * p.scale;
       } else if (lane == 0) {
         raise_status(p.dev_status, RAD_DEV_ECAPACITY);
       }
-      uint32_t kw = m << (16 * (lane & 1));
-      kw |= __shfl_xor_sync(0xffffffffu, kw, 1);
       const int64_t sb = (t - 1) * p.B + b;
-      if ((lane & 1) == 0 && (lane >> 1) < p.w32) p.keepbits[sb * p.w32 + (lane >> 1)] = kw;
+      if (lane < p.w32) p.keepbits[sb * p.w32 + lane] = m;
       if (lane == 0) p.offsets[sb] = off;
       off += total;
     } else {

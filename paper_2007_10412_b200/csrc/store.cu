@@ -144,9 +144,9 @@ __global__ void __launch_bounds__(256) store_different_kernel(const StoreParams 
           m |= ((((i < 4 ? mult[it].x : mult[it].y) >> (8 * (i & 3))) & 0xffu) != 0 ? 1u : 0u) << i;
         m &= (1u << nvalid) - 1u;
       } else {
-        // this lane's eight columns are one half of a sixteen-column draw
-        const uint32_t m16 = philox_keep16((uint32_t)(col0 >> 4), (uint32_t)row, p.c2, p.c3, ks, p.T);
-        m = (m16 >> (8 * (cg & 1))) & ((1u << nvalid) - 1u);
+        // this lane's eight columns are one byte of the keep-bit word that four lanes share
+        m = (philox_keep32((uint32_t)(col0 >> 5), (uint32_t)row, p.c2, p.c3, ks, p.T) >> (8 * (cg & 3))) &
+            ((1u << nvalid) - 1u);
       }
       masks |= m << (8 * it);
       counts |= __popc(m) << (8 * it);
@@ -316,17 +316,15 @@ __global__ void __launch_bounds__(1024) same_mask_kernel(const SameParams p, con
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) s_running = 0;
   __syncthreads();
-  const int64_t groups = (p.D + 15) / 16;
+  const int64_t groups = (p.D + 31) / 32;
   for (int64_t g0 = 0; g0 < groups; g0 += 1024) {
     const int64_t g = g0 + tid;
     uint32_t m = 0;
     if (g < groups) {
-      const int nvalid = (int)min((int64_t)16, p.D - g * 16);
-      m = philox_keep16((uint32_t)g, 0u, p.c2, p.c3, ks, p.T) & (0xffffu >> (16 - nvalid));
+      const int nvalid = (int)min((int64_t)32, p.D - g * 32);
+      m = philox_keep32((uint32_t)g, 0u, p.c2, p.c3, ks, p.T) & (0xffffffffu >> (32 - nvalid));
+      p.keepbits[g] = m;
     }
-    uint32_t kw = m << (16 * (lane & 1));
-    kw |= __shfl_xor_sync(0xffffffffu, kw, 1);
-    if ((lane & 1) == 0 && g < groups) p.keepbits[g >> 1] = kw;
     const uint32_t c = __popc(m);
     uint32_t incl = c;
 #pragma unroll
@@ -348,8 +346,8 @@ __global__ void __launch_bounds__(1024) same_mask_kernel(const SameParams p, con
     }
     __syncthreads();
     uint32_t pos = s_running + s_warp[warp] + incl - c;
-    for (int i = 0; i < 16; ++i)
-      if ((m >> i) & 1u) p.idx[pos++] = (uint32_t)(g * 16 + i);
+    for (int i = 0; i < 32; ++i)
+      if ((m >> i) & 1u) p.idx[pos++] = (uint32_t)(g * 32 + i);
     __syncthreads();
     if (tid == 1023) s_running = pos;   // last thread's end position is the running total
     __syncthreads();

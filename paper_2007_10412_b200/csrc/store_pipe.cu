@@ -5,7 +5,7 @@
 // chunk, the first phase kAhead chunks ahead of the second:
 //   phase 1  needs no data: the eight compute warps work on two tiles side by side, four warps each; a
 //            thread draws the 64 keep decisions of two adjacent keep-bit words of a row (four Philox
-//            calls), writes the words, and the warp totals go to shared memory;
+//            calls, eight logic operations per word), writes the words, and the warp totals go to shared memory;
 //   look-back a service warp adds the chunk's padded and exact counts, publishes them, and finds where
 //            the chunk starts in `values` from the chunks before it (decoupled look-back over one
 //            status word per chunk);
@@ -220,9 +220,9 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
           const uint32_t row = sm.tile_slab[slot][g] * kTileRows + r;
           const uint32_t col0 = sm.tile_cb[slot][g] * kTileCols + half * 64;
           if (row < nrows && col0 < ncols) {
-            const uint32_t g16 = col0 >> 4;
-            m0 = philox_keep16(g16, row, p.c2, p.c3, ks, p.T) | (philox_keep16(g16 + 1u, row, p.c2, p.c3, ks, p.T) << 16);
-            m1 = philox_keep16(g16 + 2u, row, p.c2, p.c3, ks, p.T) | (philox_keep16(g16 + 3u, row, p.c2, p.c3, ks, p.T) << 16);
+            const uint32_t g32 = col0 >> 5;
+            m0 = philox_keep32(g32, row, p.c2, p.c3, ks, p.T);
+            m1 = philox_keep32(g32 + 1u, row, p.c2, p.c3, ks, p.T);
             const uint32_t nv = ncols - col0;     // valid columns from col0 on
             if (nv < 64) {
               m0 &= nv >= 32 ? 0xffffffffu : (1u << nv) - 1u;
