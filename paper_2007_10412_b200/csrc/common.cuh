@@ -83,18 +83,42 @@ inline KeepThreshold make_keep_threshold(uint32_t T) {
   return k;
 }
 
-// Keep bits of columns 32 * group32 .. + 31 of one row: bit c = column c of the group.
-__device__ __forceinline__ uint32_t philox_keep32(uint32_t group32, uint32_t row, uint32_t c2, uint32_t c3,
-                                                  const PhiloxKeys& ks, const KeepThreshold& k) {
-  uint32_t lo[4], hi[4];
-  philox4x32_10(2u * group32, row, c2, c3, ks, lo);
-  philox4x32_10(2u * group32 + 1u, row, c2, c3, ks, hi);
+// The eight AND / OR steps on the words of the two outputs (lo first).
+__device__ __forceinline__ uint32_t keep_word(const uint32_t (&lo)[4], const uint32_t (&hi)[4], const KeepThreshold& k) {
   uint32_t x = k.start;
 #pragma unroll
   for (int i = 3; i >= 0; --i) x = (hi[i] & x) | ((hi[i] | x) & k.digit[4 + i]);
 #pragma unroll
   for (int i = 3; i >= 0; --i) x = (lo[i] & x) | ((lo[i] | x) & k.digit[i]);
   return x;
+}
+
+// Keep bits of columns 32 * group32 .. + 31 of one row: bit c = column c of the group.
+__device__ __forceinline__ uint32_t philox_keep32(uint32_t group32, uint32_t row, uint32_t c2, uint32_t c3,
+                                                  const PhiloxKeys& ks, const KeepThreshold& k) {
+  uint32_t lo[4], hi[4];
+  philox4x32_10(2u * group32, row, c2, c3, ks, lo);
+  philox4x32_10(2u * group32 + 1u, row, c2, c3, ks, hi);
+  return keep_word(lo, hi, k);
+}
+
+// The same word where four adjacent lanes (lane & 3 = 0..3) own a quarter of it each: lanes 0 and 1 make
+// the first output, lanes 2 and 3 the second, and the words cross over by shuffles.  Every lane of the
+// warp has to call it.
+__device__ __forceinline__ uint32_t philox_keep32_shared(uint32_t group32, uint32_t row, uint32_t c2, uint32_t c3,
+                                                         const PhiloxKeys& ks, const KeepThreshold& k, int lane) {
+  const bool second = (lane & 2) != 0;
+  uint32_t mine[4], theirs[4];
+  philox4x32_10(2u * group32 + (second ? 1u : 0u), row, c2, c3, ks, mine);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) theirs[i] = __shfl_xor_sync(0xffffffffu, mine[i], 2);
+  uint32_t lo[4], hi[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    lo[i] = second ? theirs[i] : mine[i];
+    hi[i] = second ? mine[i] : theirs[i];
+  }
+  return keep_word(lo, hi, k);
 }
 
 // Host-side twins of the threshold arithmetic (double rint, one float32 division).

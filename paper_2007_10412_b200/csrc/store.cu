@@ -133,6 +133,9 @@ __global__ void __launch_bounds__(256) store_different_kernel(const StoreParams 
 #pragma unroll
   for (int it = 0; it < 4; ++it) {
     const int64_t row = slab * kTileRows + warp * 8 + it * 2 + half;
+    // four lanes share a keep-bit word and make it together (all lanes take part, valid or not)
+    uint32_t word = 0;
+    if (!kReplace) word = philox_keep32_shared((uint32_t)(col0 >> 5), (uint32_t)row, p.c2, p.c3, ks, p.T, lane);
     if (row < p.B && nvalid > 0) {
       load8<T>(Abase + row * p.lda, col0, nvalid, p.vec_ok != 0, raw[it]);
       uint32_t m;
@@ -144,9 +147,8 @@ __global__ void __launch_bounds__(256) store_different_kernel(const StoreParams 
           m |= ((((i < 4 ? mult[it].x : mult[it].y) >> (8 * (i & 3))) & 0xffu) != 0 ? 1u : 0u) << i;
         m &= (1u << nvalid) - 1u;
       } else {
-        // this lane's eight columns are one byte of the keep-bit word that four lanes share
-        m = (philox_keep32((uint32_t)(col0 >> 5), (uint32_t)row, p.c2, p.c3, ks, p.T) >> (8 * (cg & 3))) &
-            ((1u << nvalid) - 1u);
+        // this lane's eight columns are one byte of the word
+        m = (word >> (8 * (cg & 3))) & ((1u << nvalid) - 1u);
       }
       masks |= m << (8 * it);
       counts |= __popc(m) << (8 * it);
