@@ -102,16 +102,18 @@ __device__ __forceinline__ uint32_t philox_keep32(uint32_t group32, uint32_t row
   return keep_word(lo, hi, k);
 }
 
-// The same word where four adjacent lanes (lane & 3 = 0..3) own a quarter of it each: lanes 0 and 1 make
-// the first output, lanes 2 and 3 the second, and the words cross over by shuffles.  Every lane of the
-// warp has to call it.
+// The same word made by lanes that work together, one generator output each, the words crossing over by
+// shuffles: kPartner = 2: four adjacent lanes own a quarter of the word each, lanes 0 and 1 make the first
+// output, lanes 2 and 3 the second; kPartner = 1: two adjacent lanes, one output each.  Every lane of the
+// warp has to call it; all lanes of a group get the word.
+template <int kPartner = 2>
 __device__ __forceinline__ uint32_t philox_keep32_shared(uint32_t group32, uint32_t row, uint32_t c2, uint32_t c3,
                                                          const PhiloxKeys& ks, const KeepThreshold& k, int lane) {
-  const bool second = (lane & 2) != 0;
+  const bool second = (lane & kPartner) != 0;
   uint32_t mine[4], theirs[4];
   philox4x32_10(2u * group32 + (second ? 1u : 0u), row, c2, c3, ks, mine);
 #pragma unroll
-  for (int i = 0; i < 4; ++i) theirs[i] = __shfl_xor_sync(0xffffffffu, mine[i], 2);
+  for (int i = 0; i < 4; ++i) theirs[i] = __shfl_xor_sync(0xffffffffu, mine[i], kPartner);
   uint32_t lo[4], hi[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
