@@ -477,7 +477,7 @@ def run_ours(args):
         store_roofline = dict(bound="hbm", kernel="store kernel, one 8192-wide layer input",
                               achieved=round(sbytes / ms_s / 1e6, 1), peak=pk["hbm_gbs"], unit="GB/s",
                               frac=round(sbytes / ms_s / 1e6 / pk["hbm_gbs"], 4),
-                              traffic=(int((134.3e6 + 16.6e6) * B / 8192)
+                              traffic=(int((134.3e6 + 16.2e6) * B / 8192)
                                        if args.variant == "different" and args.law == "bernoulli" and
                                        abs(args.p - 0.1) < 1e-9 else None),
                               ms_per_launch=round(ms_s, 4), algorithmic_bytes=sbytes)
