@@ -163,8 +163,9 @@ def replace_scale(fraction, D: int) -> np.float32:
     return np.float32(D) / np.float32(draws_per_row(fraction, D))
 
 
-def multiplicity(variant: str, B: int, D: int, fraction, seed: int, layer: int, step: int) -> np.ndarray:
-    """c[b, d] = how many of the k draws of row b picked column d (B x D, int64).
+def multiplicity(variant: str, B: int, D: int, fraction, seed: int, layer: int, step: int, rows=None) -> np.ndarray:
+    """c[b, d] = how many of the k draws of row b picked column d (B x D, int64).  `rows`: evaluate these
+    minibatch rows only (len(rows) x D), for layers too large to expand in full.
 
     Draw j of a row reads 32-bit word j % 4 of the Philox output for counter
     (j // 4, row, layer | stream << 24, step) and picks column
@@ -172,8 +173,11 @@ def multiplicity(variant: str, B: int, D: int, fraction, seed: int, layer: int, 
     minibatch.  Every row's multiplicities add up to k.
     """
     k = draws_per_row(fraction, D)
+    if rows is not None:
+        B = len(rows)
     if variant == "different":
-        rows, stream = np.arange(B, dtype=np.uint64)[:, None], STREAM_DIFFERENT_REPLACE
+        rows = np.arange(B, dtype=np.uint64) if rows is None else np.asarray(rows, dtype=np.uint64)
+        rows, stream = rows[:, None], STREAM_DIFFERENT_REPLACE
     elif variant == "same":
         rows, stream = np.zeros((1, 1), dtype=np.uint64), STREAM_SAME_REPLACE
     else:
@@ -215,16 +219,20 @@ def floyd_subset(ts, D: int) -> np.ndarray:
     return chosen
 
 
-def fixed_subset(variant: str, B: int, D: int, fraction, seed: int, layer: int, step: int) -> np.ndarray:
-    """Indicator (B x D, int64, k ones per row) of the k columns a row keeps.
+def fixed_subset(variant: str, B: int, D: int, fraction, seed: int, layer: int, step: int, rows=None) -> np.ndarray:
+    """Indicator (B x D, int64, k ones per row) of the k columns a row keeps.  `rows`: evaluate these
+    minibatch rows only.
 
     Draw i of a row reads 32-bit word i % 4 of the Philox output for counter
     (i // 4, row, layer | stream << 24, step) and becomes floor(word * (D - k + i + 1) / 2^32), the i-th
     draw of floyd_subset.  "same": one subset (row field 0) for the whole minibatch.
     """
     k = draws_per_row(fraction, D)
+    if rows is not None:
+        B = len(rows)
     if variant == "different":
-        rows, stream = np.arange(B, dtype=np.uint64)[:, None], STREAM_DIFFERENT_FIXED
+        rows = np.arange(B, dtype=np.uint64) if rows is None else np.asarray(rows, dtype=np.uint64)
+        rows, stream = rows[:, None], STREAM_DIFFERENT_FIXED
     elif variant == "same":
         rows, stream = np.zeros((1, 1), dtype=np.uint64), STREAM_SAME_FIXED
     else:

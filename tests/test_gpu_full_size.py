@@ -133,3 +133,91 @@ def test_forward_and_input_grad_sampled_entries(wide):
     assert max(rel_err(got, ref)) <= 2e-2
     ref_db = dZ[:, hs].astype(np.float64).sum(axis=0)
     assert max(rel_err(to_host_f32(db[hi]), ref_db)) <= 1e-5
+
+
+@pytest.mark.parametrize("law", ["replace", "fixed"])
+def test_other_sampling_laws_sampled_tiles_and_counts(wide, law):
+    """The with-replacement and the fixed-count law at the size the bench sweep times them: sampled store
+    tiles bit for bit against the oracle (multiplicities of the tile's 64 rows over all columns), offsets
+    against the keep-bit population, and the kept count (exactly B k without replacement)."""
+    rad, A = wide["rad"], wide["A"]
+    st = rad.Store("different", "bf16", B, D, P, seed=SEED, layer=LAYER, step=STEP, relu_bits=False, law=law)
+    status = wide["status"]
+    rad.rad_linear_forward_store(wide["dev"]["A"], st, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    nslab, ncb = B // TILE_ROWS, D // TILE_COLS
+    ntiles = nslab * ncb
+    k = orc.draws_per_row(P, D)
+    s = orc.replace_scale(P, D)
+    offsets = st.offsets.cpu().numpy().view(np.uint32).astype(np.int64)
+    nnz = st.nnz.cpu().numpy()
+    count = orc.multiplicity if law == "replace" else orc.fixed_subset
+    rng = np.random.default_rng(4)
+    for t in [0, ncb - 1, ntiles - 1] + [int(t) for t in rng.integers(0, ntiles, 5)]:
+        slab, blk = divmod(t, ncb)
+        rows = np.arange(slab * TILE_ROWS, (slab + 1) * TILE_ROWS)
+        c_rows = count("different", B, D, P, SEED, LAYER, STEP, rows=rows)
+        assert (c_rows.sum(axis=1) == k).all()
+        c = c_rows[:, blk * TILE_COLS:(blk + 1) * TILE_COLS]
+        m = c > 0
+        words = st.keepbits[t * TILE_WORDS:(t + 1) * TILE_WORDS].cpu().numpy().view(np.uint32)
+        assert np.array_equal(words[:256], orc.pack_bits(m).reshape(-1)), t
+        rowoff = np.concatenate([[0], np.cumsum(m.sum(axis=1))[:-1]]).astype(np.uint16)
+        assert np.array_equal(words[256:].view(np.uint16), rowoff), t
+        n = int(m.sum())
+        padded = -(-n // ALIGN) * ALIGN
+        assert offsets[t + 1] - offsets[t] == padded, t
+        tile = A[np.ix_(rows, np.arange(blk * TILE_COLS, (blk + 1) * TILE_COLS))]
+        ref = orc.round_bf16(tile * (c.astype(np.float32) * s))[m]
+        got = st.values[int(offsets[t]):int(offsets[t]) + padded].view(torch.int16).cpu().numpy().view(np.uint16)
+        assert np.array_equal(got[:n], orc.bf16_bits(ref)), t
+        assert (got[n:] == 0).all(), t
+    words = st.keepbits.view(ntiles, TILE_WORDS)[:, :256].contiguous()
+    table = torch.tensor([bin(i).count("1") for i in range(256)], dtype=torch.int32, device="cuda")
+    per_tile = torch.zeros(ntiles, dtype=torch.int64, device="cuda")
+    for sh in (0, 8, 16, 24):
+        per_tile += table[((words >> sh) & 0xFF).long()].sum(dim=1)
+    assert int(per_tile.sum()) == int(nnz[0]) and int(offsets[ntiles]) == int(nnz[1])
+    if law == "fixed":
+        assert int(nnz[0]) == B * k
+    else:
+        mean = B * D * (1.0 - (1.0 - 1.0 / D) ** k)
+        assert abs(int(nnz[0]) - mean) < 6.0 * np.sqrt(mean)      # the distinct count varies less than a Poisson
+    del st
+    torch.cuda.empty_cache()
+
+
+def test_projection_sampled_entries(wide):
+    """The random projection at the bench size: S = A R' on sampled rows and dW_hat = R' ((S^T dZ) / k) on
+    sampled entries against the oracle's definition (S over all rows in float32: bf16 inputs and signs give
+    exact products)."""
+    rad, A, dZ = wide["rad"], wide["A"], wide["dZ"]
+    st = rad.Store("project", "bf16", B, D, P, seed=SEED, layer=LAYER, step=STEP, relu_bits=False)
+    status = wide["status"]
+    rad.rad_linear_forward_store(wide["dev"]["A"], st, status)
+    dW = torch.empty(D, H, dtype=torch.float32, device="cuda")
+    ws = torch.empty(max(rad.rad_weight_grad_workspace(st, H), 256), dtype=torch.uint8, device="cuda")
+    rad.rad_linear_weight_grad(st, wide["dev"]["dZ"], dW, ws, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    k = orc.draws_per_row(P, D)
+    assert st.nnz.cpu().numpy()[0] == k
+    R = orc.rademacher(D, k, SEED, LAYER, STEP).astype(np.float32)
+    S = np.empty((B, k), dtype=np.float32)
+    for b0 in range(0, B, 8192):
+        S[b0:b0 + 8192] = orc.round_bf16(A[b0:b0 + 8192] @ R)
+    ld = st.c.values_ld
+    rng = np.random.default_rng(5)
+    bs = np.concatenate([[0, 127, 128, B - 1], rng.integers(0, B, 28)])
+    got_S = to_host_f32(st.values.view(B, ld)[torch.from_numpy(bs).cuda()])
+    assert (got_S[:, k:] == 0).all()
+    assert max(rel_err(got_S[:, :k], S[bs])) <= 8e-3
+    hs = np.concatenate([[0, 255, 256, H - 1], rng.integers(0, H, 12)])
+    ds = np.concatenate([[0, 255, 256, D - 1], rng.integers(0, D, 12)])
+    G = (S.astype(np.float64).T @ dZ[:, hs].astype(np.float64)).astype(np.float32) * (np.float32(1.0) / np.float32(k))
+    ref = R[ds].astype(np.float64) @ orc.round_bf16(G).astype(np.float64)
+    got = to_host_f32(dW[torch.from_numpy(ds).cuda()][:, torch.from_numpy(hs).cuda()])
+    assert max(rel_err(got, ref)) <= 2e-2
+    del st, dW, ws
+    torch.cuda.empty_cache()

@@ -160,3 +160,12 @@ def test_store_structure_and_rounding():
     c1 = rad.multiplicity("same", B, D, f, 1, 0, 2)[0]
     assert np.array_equal(same.idx, np.flatnonzero(c1))
     assert np.array_equal(same.values.reshape(B, -1), (A * (c1.astype(np.float32) * s))[:, c1 > 0])
+
+
+def test_rows_argument_is_the_full_matrix_restricted_to_those_rows():
+    B, D, f = 40, 150, 0.2
+    rows = np.array([0, 7, 39, 12, 12])
+    assert np.array_equal(rad.multiplicity("different", B, D, f, 3, 1, 2, rows=rows),
+                          rad.multiplicity("different", B, D, f, 3, 1, 2)[rows])
+    assert np.array_equal(rad.fixed_subset("different", B, D, f, 3, 1, 2, rows=rows),
+                          rad.fixed_subset("different", B, D, f, 3, 1, 2)[rows])
