@@ -66,3 +66,17 @@ def test_bad_arguments_are_refused():
     st.workspace = st.workspace[:256]
     with pytest.raises(rad.RadError, match="workspace"):
         rad.rad_linear_forward_store(to_dev(A, "bf16"), st)
+
+
+def test_relu_bits_come_with_the_projected_store():
+    """The 1-bit ReLU derivative of the layer that produced A (Sec. 4.2) is written by the same call."""
+    import paper_2007_10412_b200 as rad
+    B, D = 130, 264
+    A, _ = layer_inputs(B, D, 1, dtype="bf16", seed=6, relu_like=True)
+    st = rad.Store("project", "bf16", B, D, 0.25, seed=2, relu_bits=True)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    rad.rad_linear_forward_store(to_dev(A, "bf16"), st, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    got = st.relubits.cpu().numpy().view(np.uint32).reshape(B, -1)
+    assert np.array_equal(got, orc.pack_bits(A > 0))
