@@ -19,24 +19,24 @@ R = diag(sqrt(m / p_eff)) restricted to kept columns.  "different sample"
 draws m per minibatch row, "same sample" draws one m per layer and step
 (Sec. 4.3).
 
-The keep decision for (row b, column d) compares a byte u with a threshold
-T = round(p * 2^8) clipped to [1, 2^8]: kept iff u < T; p_eff = T / 2^8 and
-stored values are scaled by fl32(2^8 / T), so the estimator is exactly unbiased
-for the probability actually sampled.  The paper leaves the source of
-randomness open.  The bytes of 32 consecutive columns are laid across the
-eight words of two Philox-4x32-10 outputs, one bit plane per word: bit d % 32
-of word i holds (complemented) bit 7 - i of the byte of column d.  A device
-then gets the 32 decisions of a keep-bit word from eight word-wide AND / OR
-steps along the binary digits of T instead of 32 byte compares.  The keep
-probabilities the paper uses (0.05 ... 0.5) move by less than 2 % of their
-value.
+The keep decision for (row b, column d) compares a 12-bit number u with a
+threshold T = round(p * 2^12) clipped to [1, 2^12]: kept iff u < T;
+p_eff = T / 2^12 and stored values are scaled by fl32(2^12 / T), so the
+estimator is exactly unbiased for the probability actually sampled.  The paper
+leaves the source of randomness open.  The numbers of 32 consecutive columns
+are laid across the twelve words of three Philox-4x32-10 outputs, one bit
+plane per word: bit d % 32 of word i holds (complemented) bit 11 - i of the
+number of column d.  A device then gets the 32 decisions of a keep-bit word
+from twelve word-wide AND / OR steps along the binary digits of T instead of
+32 compares.  Every keep probability of the sweeps (0.01 ... 0.5) is sampled
+within 0.1 % of its value, and probabilities down to 2^-12 stay distinct.
 
 Second sampling law, the paper's own (Sec. 3.2, App. A): k = ceil(fraction * d)
 coordinates drawn uniformly WITH replacement, P = (d / k) sum_s e_s e_s^T, so a
 coordinate hit c times is kept with weight c * d / k (`law="replace"`).
 
-Third law (App. A, caption of the fraction sweep: the method "could be modified
-to sample without replacement", and fraction 1.0 is then the exact gradient):
+Third law (App. A, caption of the fraction sweep, which remarks that drawing
+without replacement would make fraction 1.0 the exact gradient):
 a uniformly random subset of exactly k = ceil(fraction * d) coordinates, each
 kept with weight d / k (`law="fixed"`).
 
@@ -60,8 +60,9 @@ STREAM_SAME_REPLACE = 3        # with-replacement draws, shared by the minibatch
 STREAM_DIFFERENT_FIXED = 4     # k distinct columns, per row
 STREAM_SAME_FIXED = 5          # k distinct columns, shared by the minibatch
 STREAM_PROJECT = 6             # signs of the Rademacher projection
-LANE_BITS = 8
-COLUMNS_PER_GROUP = 32   # one keep-bit word: two generator outputs (256 bits), eight bit planes of 32 columns
+LANE_BITS = 12
+OUTPUTS_PER_GROUP = LANE_BITS // 4   # generator outputs (four words each) behind one keep-bit word
+COLUMNS_PER_GROUP = 32   # one keep-bit word: three generator outputs (384 bits), twelve bit planes of 32 columns
 LANE_RANGE = 1 << LANE_BITS
 
 
@@ -69,7 +70,7 @@ LANE_RANGE = 1 << LANE_BITS
 # mask (Sec. 3.2: E[P] = I; Sec. 4.3: "same sample" / "different sample")
 # --------------------------------------------------------------------------
 def keep_threshold(p) -> int:
-    """T such that a byte lane u is kept iff u < T."""
+    """T such that an entry whose 12-bit number is u is kept iff u < T."""
     p32 = float(np.float32(p))
     if not (0.0 < p32 <= 1.0):
         raise ValueError("p must be in (0, 1]")
@@ -85,29 +86,30 @@ def scale_factor(p) -> np.float32:
     return np.float32(LANE_RANGE) / np.float32(keep_threshold(p))
 
 
-def _decision_bytes(group, rows, stream, seed, layer, step):
-    """Bytes u of the 32 columns of each (row, group): shape rows x groups x 32, uint32 in [0, 256).
+def _decision_numbers(group, rows, stream, seed, layer, step):
+    """Numbers u of the 32 columns of each (row, group): shape rows x groups x 32, uint32 in [0, 4096).
 
-    Outputs of the generator for counters (2 * group, row, layer | stream << 24, step) and
-    (2 * group + 1, ...), key = (seed low word, seed high word), give words w_0 .. w_7 (first
-    output first).  Column c of the group has u = sum_i (1 - bit c of w_i) << (7 - i).
+    Outputs of the generator for counters (3 * group + j, row, layer | stream << 24, step), j = 0, 1, 2,
+    key = (seed low word, seed high word), give words w_0 .. w_11 (first output first).  Column c of the
+    group has u = sum_i (1 - bit c of w_i) << (11 - i).
     """
     c2 = np.uint64((layer & 0xFFFFFF) | (stream << 24))
     k0, k1 = np.uint64(seed & 0xFFFFFFFF), np.uint64((seed >> 32) & 0xFFFFFFFF)
     words = []
-    for j in range(2):
-        words.extend(philox4x32_10(np.uint64(2) * group + np.uint64(j), rows, c2, np.uint64(step & 0xFFFFFFFF), k0, k1))
+    for j in range(OUTPUTS_PER_GROUP):
+        words.extend(philox4x32_10(np.uint64(OUTPUTS_PER_GROUP) * group + np.uint64(j), rows, c2,
+                                   np.uint64(step & 0xFFFFFFFF), k0, k1))
     shape = np.broadcast(group, rows).shape
     u = np.zeros(shape + (COLUMNS_PER_GROUP,), dtype=np.uint32)
     cols = np.arange(COLUMNS_PER_GROUP, dtype=np.uint32)
     for i, w in enumerate(words):
         bits = (np.broadcast_to(w, shape)[..., None] >> cols) & np.uint32(1)
-        u |= (np.uint32(1) - bits) << np.uint32(7 - i)
+        u |= (np.uint32(1) - bits) << np.uint32(LANE_BITS - 1 - i)
     return u
 
 
 def keep_mask(variant: str, B: int, D: int, p, seed: int, layer: int, step: int) -> np.ndarray:
-    """Boolean B x D keep mask: column d of row b is kept iff its byte (see _decision_bytes, group d // 32,
+    """Boolean B x D keep mask: column d of row b is kept iff its number (see _decision_numbers, group d // 32,
     column d % 32 of the group) is below T.  For "same" the row field of the counter is 0 and the single
     row of decisions is shared by every minibatch element."""
     T = keep_threshold(p)
@@ -118,7 +120,7 @@ def keep_mask(variant: str, B: int, D: int, p, seed: int, layer: int, step: int)
         rows, stream = np.zeros((1, 1), dtype=np.uint64), STREAM_SAME
     else:
         raise ValueError(variant)
-    u = _decision_bytes(np.arange(groups, dtype=np.uint64)[None, :], rows, stream, seed, layer, step)
+    u = _decision_numbers(np.arange(groups, dtype=np.uint64)[None, :], rows, stream, seed, layer, step)
     m = (u < T).reshape(u.shape[0], groups * COLUMNS_PER_GROUP)[:, :D]
     if variant == "same":
         m = np.broadcast_to(m, (B, D))
@@ -127,7 +129,7 @@ def keep_mask(variant: str, B: int, D: int, p, seed: int, layer: int, step: int)
 
 def keep_mask_at(variant: str, rows, cols, p, seed: int, layer: int, step: int) -> np.ndarray:
     """Keep decisions of the given rows x the given columns (len(rows) x len(cols), boolean): the same
-    counter, key and byte rule as keep_mask, evaluated only where asked, so that single tiles or
+    counter, key and threshold rule as keep_mask, evaluated only where asked, so that single tiles or
     single columns of a layer too large to expand in full can be checked."""
     T = keep_threshold(p)
     rows = np.asarray(rows, dtype=np.uint64).reshape(-1, 1)
@@ -138,15 +140,15 @@ def keep_mask_at(variant: str, rows, cols, p, seed: int, layer: int, step: int) 
         rows, stream = np.zeros_like(rows), STREAM_SAME
     else:
         raise ValueError(variant)
-    u = _decision_bytes(cols // np.uint64(COLUMNS_PER_GROUP) + np.zeros_like(rows), rows + np.zeros_like(cols), stream,
+    u = _decision_numbers(cols // np.uint64(COLUMNS_PER_GROUP) + np.zeros_like(rows), rows + np.zeros_like(cols), stream,
                         seed, layer, step)                                  # rows x cols x 32
     pick = (cols % np.uint64(COLUMNS_PER_GROUP)).astype(np.int64) + np.zeros(rows.shape, dtype=np.int64)
     return np.take_along_axis(u, pick[..., None], axis=-1)[..., 0] < T
 
 
 # --------------------------------------------------------------------------
-# the paper's own sampling law (Sec. 3.2: "sampling (with replacement) k out of
-# the d vertices"; App. A: fraction of activations sampled with replacement)
+# the paper's own sampling law (Sec. 3.2, the example after Eq. 5: k of the d
+# coordinates drawn with replacement; App. A: a fraction of the activations)
 # --------------------------------------------------------------------------
 def draws_per_row(fraction, D: int) -> int:
     """k = ceil(fraction * d), at least 1 and at most d.  The fraction arrives as a float32 (0.1 is then
@@ -250,8 +252,8 @@ def fixed_subset(variant: str, B: int, D: int, fraction, seed: int, layer: int, 
 
 
 # --------------------------------------------------------------------------
-# random projection (Sec. 3.2: "R be a random projection matrix of independent
-# Rademacher random variables"; App. A: scaled so that P = R R^T has E[P] = I)
+# random projection (Sec. 3.2 after Eq. 5: R a matrix of independent Rademacher
+# signs; App. A: scaled so that P = R R^T has E[P] = I)
 # --------------------------------------------------------------------------
 def rademacher(D: int, k: int, seed: int, layer: int, step: int) -> np.ndarray:
     """The unscaled sign matrix R' (D x k, entries +1 / -1, float64); R = R' / sqrt(k).
@@ -321,7 +323,8 @@ def unpack_bits(words: np.ndarray, D: int) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------
-# the compact store (Sec. 3.2 "sparsify the input vectors"; App. A memory model)
+# the compact store (Sec. 3.2, last paragraph: the layer input is what gets
+# sparsified, not the Jacobian; App. A memory model)
 # --------------------------------------------------------------------------
 @dataclass
 class Store:

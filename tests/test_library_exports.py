@@ -48,7 +48,7 @@ def test_host_only_entry_points():
     assert sz.keepbits_words == ntiles * 288 and sz.offsets_words == ntiles + 1
     assert sz.relubits_words == 65536 * 256
     assert sz.values_worst == 65536 * 8192 + 7 * ntiles
-    assert 26 / 256 * 65536 * 8192 < sz.values_typical < 1.01 * 26 / 256 * 65536 * 8192
+    assert 410 / 4096 * 65536 * 8192 < sz.values_typical < 1.01 * 410 / 4096 * 65536 * 8192
     sz = b.rad_store_size_query("same", "f32", 150, 784, 0.1)
     assert sz.values_ld_worst == 832 and sz.values_ld_typical % 64 == 0 and sz.values_ld_typical >= 128
     with pytest.raises(b.RadError):

@@ -26,7 +26,7 @@ def exact_dW(A, dZ):
 def test_p_one_is_exact_backprop(variant, dtype):
     A, dZ = layer_inputs(37, 70, 9, dtype=dtype, seed=3)
     st = rad.forward_store(A, dtype, variant, 1.0, seed=5, layer=2, step=1)
-    assert st.T == 256 and st.scale == np.float32(1.0)
+    assert st.T == 4096 and st.scale == np.float32(1.0)
     assert st.nnz == A.size
     assert np.array_equal(st.values.view(np.uint32), A.reshape(-1).view(np.uint32))
     assert np.array_equal(rad.weight_grad(st, dZ), exact_dW(A, dZ))
@@ -166,12 +166,30 @@ def test_mask_depends_on_key_fields_only():
 
 
 def test_threshold_table():
-    for p, T in [(0.01, 3), (0.05, 13), (0.1, 26), (0.2, 51), (0.5, 128), (1.0, 256), (1e-9, 1), (0.998, 255), (0.9990235, 256)]:
+    for p, T in [(0.01, 41), (0.05, 205), (0.1, 410), (0.2, 819), (0.5, 2048), (1.0, 4096), (1e-9, 1),
+                 (0.998, 4088), (0.99995, 4096), (1.0 / 4096, 1), (1.0 / 2048, 2), (1.0 / 512, 8)]:
         assert rad.keep_threshold(p) == T
     with pytest.raises(ValueError):
         rad.keep_threshold(0.0)
     with pytest.raises(ValueError):
         rad.keep_threshold(1.5)
+
+
+def test_sampled_probability_is_the_requested_one():
+    """The estimator is Bernoulli(p) rescaled by 1 / p (Sec. 3.2, E[P] = I): the probability really sampled
+    stays within 0.1 % of the requested one for every value of the sweeps, the scale is its reciprocal, and
+    small probabilities do not collapse onto one another."""
+    for p in (0.01, 0.05, 0.1, 0.2, 0.3, 0.5, 0.8, 1.0):
+        pe = rad.effective_p(p)
+        assert abs(pe - p) / p <= 1e-3, (p, pe)
+        assert rad.scale_factor(p) == np.float32(1.0 / pe)
+    small = [rad.effective_p(2.0 ** -k) for k in range(1, 13)]
+    assert small == [2.0 ** -k for k in range(1, 13)]
+    # the frequency of kept entries follows p_eff (Binomial band of five standard deviations)
+    for p in (0.01, 0.05):
+        m = rad.keep_mask("different", 512, 1024, p, 3, 1, 0)
+        n, pe = m.size, rad.effective_p(p)
+        assert abs(m.sum() - n * pe) < 5 * np.sqrt(n * pe * (1 - pe))
 
 
 def test_bf16_rounding_matches_torch():

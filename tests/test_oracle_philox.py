@@ -107,28 +107,34 @@ def test_keep_mask_at_agrees_with_the_full_mask(variant):
 
 
 @pytest.mark.parametrize("variant", ["different", "same"])
-def test_byte_of_a_column_is_laid_across_the_eight_words_of_two_outputs(variant):
-    """Column d is decided by the byte whose bit 7 - i is the complement of bit d % 32 of word i of the
-    two generator outputs for counters 2 (d // 32) and 2 (d // 32) + 1; restated here with Python
+def test_number_of_a_column_is_laid_across_the_twelve_words_of_three_outputs(variant):
+    """Column d is decided by the 12-bit number whose bit 11 - i is the complement of bit d % 32 of word i
+    of the three generator outputs for counters 3 (d // 32) + j, j = 0, 1, 2; restated here with Python
     integers, independent of the array code in the oracle."""
     B, D, p, seed, layer, step = 5, 77, 0.3, 0xABCDEF0123456789, 6, 11
     T = orc.keep_threshold(p)
-    assert T == 77          # rint(0.3 * 256)
+    assert T == 1229          # rint(0.3 * 4096)
     full = orc.keep_mask(variant, B, D, p, seed, layer, step)
     stream = 0 if variant == "different" else 1
     for b in range(B):
         row = b if variant == "different" else 0
         for d in range(D):
             words = []
-            for j in range(2):
-                words += bigint_philox([2 * (d // 32) + j, row, layer | stream << 24, step], [seed & MASK, seed >> 32])
-            u = sum((1 - ((w >> (d % 32)) & 1)) << (7 - i) for i, w in enumerate(words))
+            for j in range(3):
+                words += bigint_philox([3 * (d // 32) + j, row, layer | stream << 24, step], [seed & MASK, seed >> 32])
+            u = sum((1 - ((w >> (d % 32)) & 1)) << (11 - i) for i, w in enumerate(words))
             assert bool(full[b, d]) == (u < T)
 
 
-def test_decision_bytes_are_uniform():
-    u = orc._decision_bytes(np.arange(64, dtype=np.uint64)[None, :], np.arange(64, dtype=np.uint64)[:, None], 0, 42, 2, 0)
-    hist = np.bincount(u.reshape(-1), minlength=256).astype(np.float64)
-    expected = u.size / 256.0
+def test_decision_numbers_are_uniform():
+    u = orc._decision_numbers(np.arange(128, dtype=np.uint64)[None, :], np.arange(128, dtype=np.uint64)[:, None], 0, 42, 2, 0)
+    assert u.max() < 4096
+    hist = np.bincount(u.reshape(-1), minlength=4096).astype(np.float64)
+    expected = u.size / 4096.0
     chi2 = ((hist - expected) ** 2 / expected).sum()
-    assert abs(chi2 - 255.0) < 6 * 22.6
+    # 4095 degrees of freedom: mean 4095, sd ~90.5; 6 sigma band
+    assert abs(chi2 - 4095.0) < 6 * 90.5
+    # every bit plane on its own is balanced (a dropped or repeated plane would show here)
+    for i in range(12):
+        ones = int(((u >> i) & 1).sum())
+        assert abs(ones - u.size / 2) < 6 * np.sqrt(u.size / 4)
