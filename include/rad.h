@@ -60,24 +60,25 @@ typedef enum { RAD_ACT_NONE = 0, RAD_ACT_RELU = 1, RAD_ACT_GELU = 2 } rad_act;
 
 /*
  * The mask (Sec. 3.2: a random P with E[P] = I; Sec. 4.3: "same sample" /
- * "different sample").  Entry (b, d) is kept iff its byte u is below
- * T = clamp(rint(p * 256), 1, 256):
+ * "different sample").  Entry (b, d) is kept iff its 12-bit number u is below
+ * T = clamp(rint(p * 4096), 1, 4096):
  *   key     = (seed & 0xffffffff, seed >> 32)
- *   words   = w_0 .. w_3 from the Philox-4x32-10 output for counter
- *             (2 * (d / 32), row, layer | stream << 24, step), w_4 .. w_7 from the
- *             output for counter (2 * (d / 32) + 1, ...); row = b and stream = 0
- *             for different-sample, row = 0 and stream = 1 for same-sample
- *   u       = sum over i of (1 - bit (d % 32) of w_i) << (7 - i): the bytes of 32
- *             columns lie across the eight words, one bit plane per word, so a
- *             keep-bit word follows from eight AND / OR steps along the binary
+ *   words   = w_0 .. w_11: the four words of the Philox-4x32-10 outputs for
+ *             counters (3 * (d / 32) + j, row, layer | stream << 24, step),
+ *             j = 0, 1, 2, first output first; row = b and stream = 0 for
+ *             different-sample, row = 0 and stream = 1 for same-sample
+ *   u       = sum over i of (1 - bit (d % 32) of w_i) << (11 - i): the numbers of
+ *             32 columns lie across the twelve words, one bit plane per word, so
+ *             a keep-bit word follows from twelve AND / OR steps along the binary
  *             digits of T.
- * p_eff = T / 256 is the probability actually sampled and kept values are
- * multiplied by fl32(256 / T) = 1 / p_eff, so E[A_hat] = A exactly.
+ * p_eff = T / 4096 is the probability actually sampled (within 0.1 % of p for
+ * p >= 0.01) and kept values are multiplied by fl32(4096 / T) = 1 / p_eff, so
+ * E[A_hat] = A exactly.
  */
 /*
- * Second sampling law, the paper's own (Sec. 3.2: "sampling (with replacement) k
- * out of the d vertices", P = (d / k) sum_s e_s e_s^T; App. A: a fraction of the
- * activations sampled with replacement).  Per row (different-sample) or once per
+ * Second sampling law, the paper's own (Sec. 3.2, the example after Eq. 5: k of
+ * the d coordinates drawn with replacement, P = (d / k) sum_s e_s e_s^T; App. A: a
+ * fraction of the activations).  Per row (different-sample) or once per
  * layer and step (same-sample), k = ceil(fraction * D) columns are drawn; a column
  * drawn c > 0 times is kept and its entry is multiplied by fl32(c * fl32(D / k)).
  *   draw j  = 32-bit word j % 4 of the Philox-4x32-10 output for
@@ -102,8 +103,8 @@ int64_t rad_draws_per_row(float fraction, int64_t D);   /* k; 0 if the fraction 
 float   rad_replace_scale(float fraction, int64_t D);   /* fl32(D / k)                            */
 
 uint32_t rad_keep_threshold(float p);   /* T; 0 if p is outside (0, 1]                        */
-float    rad_effective_p(float p);      /* T / 256                                            */
-float    rad_scale(float p);            /* fl32(256 / T)                                      */
+float    rad_effective_p(float p);      /* T / 4096                                           */
+float    rad_scale(float p);            /* fl32(4096 / T)                                     */
 
 /*
  * One layer's compact store: plain data, all buffers device memory of the caller.
@@ -187,8 +188,8 @@ int rad_store_size_query_law(int32_t variant, int32_t dtype, int32_t law, int64_
                              rad_store_sizes* out /* host */);
 
 /*
- * Forward-pass store of one layer input (Sec. 3.2 "sparsify the input vectors";
- * Sec. 4.2 sampling of dh/dW).  Reads A (device, B x D, leading dimension lda,
+ * Forward-pass store of one layer input (Sec. 3.2, last paragraph: the layer
+ * input is sparsified, never the Jacobian; Sec. 4.2 sampling of dh/dW).  Reads A (device, B x D, leading dimension lda,
  * type st->dtype), draws the mask, and fills st->keepbits / values / offsets /
  * nnz (and relubits).  `st` is a host struct read during the call.  `workspace`
  * is device scratch of at least rad_store_sizes.workspace_bytes, 256-byte

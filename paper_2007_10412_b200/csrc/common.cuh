@@ -65,62 +65,65 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
   out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
-// An entry is kept iff its byte u is below T (1..256).  The bytes of 32 consecutive columns are laid
-// across the eight words w_0 .. w_7 of two generator outputs, one bit plane per word: bit c of w_i is the
-// complement of bit 7 - i of the byte of column c.  Comparing from the least significant digit of T
-// upwards, "u < T so far" becomes (w_i | x) where the digit of T is 1 and (w_i & x) where it is 0, so the 32
-// decisions of a keep-bit word are eight three-input logic operations, no compares.
-constexpr uint32_t kLaneRange = 256;
+// An entry is kept iff its 12-bit number u is below T (1..4096).  The numbers of 32 consecutive columns are
+// laid across the twelve words w_0 .. w_11 of three generator outputs, one bit plane per word: bit c of w_i
+// is the complement of bit 11 - i of the number of column c.  Comparing from the least significant digit of
+// T upwards, "u < T so far" becomes (w_i | x) where the digit of T is 1 and (w_i & x) where it is 0, so the
+// 32 decisions of a keep-bit word are twelve three-input logic operations, no compares.
+constexpr int kLaneBits = 12;
+constexpr uint32_t kLaneRange = 1u << kLaneBits;
+constexpr int kOutputsPerGroup = kLaneBits / 4;   // generator outputs behind one keep-bit word
 
 struct KeepThreshold {
-  uint32_t digit[8];   // digit[i]: all ones if bit 7 - i of T is set (T = 256: all set)
-  uint32_t start;      // decisions before any digit: none kept, or all kept for T = 256
+  uint32_t digit[kLaneBits];   // digit[i]: all ones if bit 11 - i of T is set (T = 4096: all set)
+  uint32_t start;              // decisions before any digit: none kept, or all kept for T = 4096
 };
 inline KeepThreshold make_keep_threshold(uint32_t T) {
   KeepThreshold k;
-  for (int i = 0; i < 8; ++i) k.digit[i] = (T >= kLaneRange || ((T >> (7 - i)) & 1u)) ? 0xffffffffu : 0u;
+  for (int i = 0; i < kLaneBits; ++i)
+    k.digit[i] = (T >= kLaneRange || ((T >> (kLaneBits - 1 - i)) & 1u)) ? 0xffffffffu : 0u;
   k.start = T >= kLaneRange ? 0xffffffffu : 0u;
   return k;
 }
 
-// The eight AND / OR steps on the words of the two outputs (lo first).
-__device__ __forceinline__ uint32_t keep_word(const uint32_t (&lo)[4], const uint32_t (&hi)[4], const KeepThreshold& k) {
-  uint32_t x = k.start;
+// The AND / OR steps on the four words of output j of a group (planes 4 j .. 4 j + 3), given the
+// decisions x of the planes below them; the outputs are folded in from the last one to the first.
+__device__ __forceinline__ uint32_t keep_fold(uint32_t x, const uint32_t (&w)[4], int j, const KeepThreshold& k) {
 #pragma unroll
-  for (int i = 3; i >= 0; --i) x = (hi[i] & x) | ((hi[i] | x) & k.digit[4 + i]);
-#pragma unroll
-  for (int i = 3; i >= 0; --i) x = (lo[i] & x) | ((lo[i] | x) & k.digit[i]);
+  for (int i = 3; i >= 0; --i) x = (w[i] & x) | ((w[i] | x) & k.digit[4 * j + i]);
   return x;
 }
 
 // Keep bits of columns 32 * group32 .. + 31 of one row: bit c = column c of the group.
 __device__ __forceinline__ uint32_t philox_keep32(uint32_t group32, uint32_t row, uint32_t c2, uint32_t c3,
                                                   const PhiloxKeys& ks, const KeepThreshold& k) {
-  uint32_t lo[4], hi[4];
-  philox4x32_10(2u * group32, row, c2, c3, ks, lo);
-  philox4x32_10(2u * group32 + 1u, row, c2, c3, ks, hi);
-  return keep_word(lo, hi, k);
+  uint32_t x = k.start;
+#pragma unroll
+  for (int j = kOutputsPerGroup - 1; j >= 0; --j) {
+    uint32_t w[4];
+    philox4x32_10((uint32_t)kOutputsPerGroup * group32 + (uint32_t)j, row, c2, c3, ks, w);
+    x = keep_fold(x, w, j, k);
+  }
+  return x;
 }
 
-// The same word made by lanes that work together, one generator output each, the words crossing over by
-// shuffles: kPartner = 2: four adjacent lanes own a quarter of the word each, lanes 0 and 1 make the first
-// output, lanes 2 and 3 the second; kPartner = 1: two adjacent lanes, one output each.  Every lane of the
-// warp has to call it; all lanes of a group get the word.
-template <int kPartner = 2>
-__device__ __forceinline__ uint32_t philox_keep32_shared(uint32_t group32, uint32_t row, uint32_t c2, uint32_t c3,
-                                                         const PhiloxKeys& ks, const KeepThreshold& k, int lane) {
-  const bool second = (lane & kPartner) != 0;
-  uint32_t mine[4], theirs[4];
-  philox4x32_10(2u * group32 + (second ? 1u : 0u), row, c2, c3, ks, mine);
+// The same word made by four adjacent lanes (4 q .. 4 q + 3, which pass the same group and row): lane j of
+// the four makes output j (the fourth lane repeats the last one), the words cross over by shuffles.  Every
+// lane of the warp has to call it; all four lanes get the word.
+__device__ __forceinline__ uint32_t philox_keep32_quad(uint32_t group32, uint32_t row, uint32_t c2, uint32_t c3,
+                                                       const PhiloxKeys& ks, const KeepThreshold& k, int lane) {
+  const int j = min(lane & 3, kOutputsPerGroup - 1);
+  uint32_t mine[4];
+  philox4x32_10((uint32_t)kOutputsPerGroup * group32 + (uint32_t)j, row, c2, c3, ks, mine);
+  uint32_t x = k.start;
 #pragma unroll
-  for (int i = 0; i < 4; ++i) theirs[i] = __shfl_xor_sync(0xffffffffu, mine[i], kPartner);
-  uint32_t lo[4], hi[4];
+  for (int o = kOutputsPerGroup - 1; o >= 0; --o) {
+    uint32_t w[4];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    lo[i] = second ? theirs[i] : mine[i];
-    hi[i] = second ? mine[i] : theirs[i];
+    for (int i = 0; i < 4; ++i) w[i] = __shfl_sync(0xffffffffu, mine[i], (lane & ~3) + o);
+    x = keep_fold(x, w, o, k);
   }
-  return keep_word(lo, hi, k);
+  return x;
 }
 
 // Host-side twins of the threshold arithmetic (double rint, one float32 division).

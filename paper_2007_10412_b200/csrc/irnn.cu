@@ -67,11 +67,11 @@ __global__ void __launch_bounds__(kRnnThreads) irnn_forward_kernel(const RnnPara
     const float* hc = s_h[(t - 1) & 1];
     if (warp == 4) {
       // store of h_{t-1}: keep bits of the step, kept entries scaled and appended to the row's values
-      // one keep-bit word decides 32 units; two lanes make it together (one generator output each, which
-      // keeps this warp off the critical path of the step) and the even lane goes on with it
-      const int wi = lane >> 1;
-      uint32_t m = philox_keep32_shared<1>((uint32_t)wi, mask_row, p.c2, p.step0 + (uint32_t)t, ks, p.keepT, lane);
-      if ((lane & 1) == 0 && wi * 32 < Hd) m &= 0xffffffffu >> (32 - min(32, Hd - wi * 32));
+      // one keep-bit word decides 32 units; four lanes make it together (one generator output each, which
+      // keeps this warp off the critical path of the step) and the first of them goes on with it
+      const int wi = lane >> 2;
+      uint32_t m = philox_keep32_quad((uint32_t)wi, mask_row, p.c2, p.step0 + (uint32_t)t, ks, p.keepT, lane);
+      if ((lane & 3) == 0 && wi * 32 < Hd) m &= 0xffffffffu >> (32 - min(32, Hd - wi * 32));
       else m = 0;
       const uint32_t c = __popc(m);
       uint32_t incl = c;
@@ -90,7 +90,7 @@ __global__ void __launch_bounds__(kRnnThreads) irnn_forward_kernel(const RnnPara
         raise_status(p.dev_status, RAD_DEV_ECAPACITY);
       }
       const int64_t sb = (t - 1) * p.B + b;
-      if ((lane & 1) == 0 && wi < p.w32) p.keepbits[sb * p.w32 + wi] = m;
+      if ((lane & 3) == 0 && wi < p.w32) p.keepbits[sb * p.w32 + wi] = m;
       if (lane == 0) p.offsets[sb] = off;
       off += total;
     } else {

@@ -135,7 +135,7 @@ __global__ void __launch_bounds__(256) store_different_kernel(const StoreParams 
     const int64_t row = slab * kTileRows + warp * 8 + it * 2 + half;
     // four lanes share a keep-bit word and make it together (all lanes take part, valid or not)
     uint32_t word = 0;
-    if (!kReplace) word = philox_keep32_shared((uint32_t)(col0 >> 5), (uint32_t)row, p.c2, p.c3, ks, p.T, lane);
+    if (!kReplace) word = philox_keep32_quad((uint32_t)(col0 >> 5), (uint32_t)row, p.c2, p.c3, ks, p.T, lane);
     if (row < p.B && nvalid > 0) {
       load8<T>(Abase + row * p.lda, col0, nvalid, p.vec_ok != 0, raw[it]);
       uint32_t m;

@@ -36,19 +36,20 @@ def wide():
     torch.cuda.empty_cache()
 
 
-def test_store_sampled_tiles_are_bit_exact(wide):
-    st, A = wide["st"], wide["A"]
+def check_sampled_tiles(st, A, p, n_random=10, seed=1):
+    """Keep bits, row offsets, tile extent and stored values of some tiles of a different-sample store of
+    the wide layer, bit for bit against the oracle's definition evaluated on those tiles alone."""
     nslab, ncb = B // TILE_ROWS, D // TILE_COLS
     ntiles = nslab * ncb
-    rng = np.random.default_rng(1)
-    tiles = [0, 1, ncb - 1, ncb, ntiles - 1, ntiles - ncb] + [int(t) for t in rng.integers(0, ntiles, 10)]
+    rng = np.random.default_rng(seed)
+    tiles = [0, 1, ncb - 1, ncb, ntiles - 1, ntiles - ncb] + [int(t) for t in rng.integers(0, ntiles, n_random)]
     offsets = st.offsets.cpu().numpy().view(np.uint32)
-    scale = np.float32(orc.scale_factor(P))
+    scale = np.float32(orc.scale_factor(p))
     for t in tiles:
         slab, blk = divmod(t, ncb)
         rows = np.arange(slab * TILE_ROWS, (slab + 1) * TILE_ROWS)
         cols = np.arange(blk * TILE_COLS, (blk + 1) * TILE_COLS)
-        m = orc.keep_mask_at("different", rows, cols, P, SEED, LAYER, STEP)
+        m = orc.keep_mask_at("different", rows, cols, p, SEED, LAYER, STEP)
         words = st.keepbits[t * TILE_WORDS:(t + 1) * TILE_WORDS].cpu().numpy().view(np.uint32)
         assert np.array_equal(words[:256], orc.pack_bits(m).reshape(-1)), t
         rowoff = np.concatenate([[0], np.cumsum(m.sum(axis=1))[:-1]]).astype(np.uint16)
@@ -62,11 +63,11 @@ def test_store_sampled_tiles_are_bit_exact(wide):
         assert (got[n:] == 0).all(), t
 
 
-def test_store_counts_hold_together(wide):
-    st = wide["st"]
+def check_counts(st, p):
+    """Identities that tie keep bits, offsets and the kept count together over the whole store."""
     ntiles = (B // TILE_ROWS) * (D // TILE_COLS)
     words = st.keepbits.view(ntiles, TILE_WORDS)[:, :256].contiguous()
-    # set bits of every keep word, summed per tile on the device (16-bit lookups of a byte table)
+    # set bits of every keep word, summed per tile on the device (lookups of a byte table)
     table = torch.tensor([bin(i).count("1") for i in range(256)], dtype=torch.int32, device="cuda")
     per_tile = torch.zeros(ntiles, dtype=torch.int64, device="cuda")
     for sh in (0, 8, 16, 24):
@@ -78,22 +79,23 @@ def test_store_counts_hold_together(wide):
     padded = ((per_tile + (ALIGN - 1)) // ALIGN * ALIGN).cpu().numpy()
     assert np.array_equal(np.diff(offsets[:ntiles + 1]), padded)
     # Binomial(B D, p_eff): six standard deviations
-    pe = orc.effective_p(P)
+    pe = orc.effective_p(p)
     assert abs(int(nnz[0]) - B * D * pe) < 6.0 * np.sqrt(B * D * pe * (1.0 - pe))
 
 
-def test_weight_grad_sampled_entries(wide):
-    rad, st, A, dZ = wide["rad"], wide["st"], wide["A"], wide["dZ"]
+def check_weight_grad_entries(rad, st, A, dZ, dZ_dev, p, status, seed=2):
+    """dW from a different-sample store of the wide layer on sampled (d, h) entries, each summed by the
+    oracle over all 65536 rows from the mask and the rounded scaled values."""
     dW = torch.full((D, H), float("nan"), dtype=torch.float32, device="cuda")
-    rad.rad_linear_weight_grad(st, wide["dev"]["dZ"], dW, dev_status=wide["status"])
+    rad.rad_linear_weight_grad(st, dZ_dev, dW, dev_status=status)
     torch.cuda.synchronize()
-    assert wide["status"].item() == 0
+    assert status.item() == 0
     assert torch.isfinite(dW).all()
-    rng = np.random.default_rng(2)
+    rng = np.random.default_rng(seed)
     ds = np.concatenate([[0, 127, 128, 255, 256, 511, 512, D - 1], rng.integers(0, D, 16)])
     hs = np.concatenate([[0, 255, 256, H - 1], rng.integers(0, H, 12)])
-    scale = np.float32(orc.scale_factor(P))
-    m = orc.keep_mask_at("different", np.arange(B), ds, P, SEED, LAYER, STEP)          # B x len(ds)
+    scale = np.float32(orc.scale_factor(p))
+    m = orc.keep_mask_at("different", np.arange(B), ds, p, SEED, LAYER, STEP)          # B x len(ds)
     a_hat = np.where(m, orc.round_bf16(A[:, ds] * scale), np.float32(0)).astype(np.float64)
     ref = a_hat.T @ dZ[:, hs].astype(np.float64)
     got = to_host_f32(dW[torch.from_numpy(ds).cuda()][:, torch.from_numpy(hs).cuda()])
@@ -102,6 +104,82 @@ def test_weight_grad_sampled_entries(wide):
     # float32 accumulation of exact bf16 products: far inside the stated tolerance
     bound = 1e-4 * (np.abs(a_hat).T @ np.abs(dZ[:, hs]).astype(np.float64))
     assert (np.abs(got - ref) <= bound + 1e-30).all()
+    del dW
+
+
+def test_store_sampled_tiles_are_bit_exact(wide):
+    check_sampled_tiles(wide["st"], wide["A"], P)
+
+
+@pytest.mark.parametrize("p", [0.01, 0.05, 0.5])
+def test_store_and_weight_grad_over_the_p_sweep(wide, p):
+    """The other keep probabilities the bench sweeps: the pipelined store on sampled tiles and count
+    identities; at p = 0.5 also dW, whose expander then takes its dense-word path."""
+    rad, status = wide["rad"], wide["status"]
+    st = rad.Store("different", "bf16", B, D, p, seed=SEED, layer=LAYER, step=STEP, relu_bits=False)
+    rad.rad_linear_forward_store(wide["dev"]["A"], st, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    check_sampled_tiles(st, wide["A"], p, n_random=6, seed=int(p * 1000))
+    check_counts(st, p)
+    if p == 0.5:
+        check_weight_grad_entries(rad, st, wide["A"], wide["dZ"], wide["dev"]["dZ"], p, status, seed=9)
+    del st
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("p", [0.01, 0.1, 0.5])
+def test_same_sample_store_and_weight_grad(wide, p):
+    """Same-sample variant at the size the bench times it (Sec. 4.3: one mask for the whole minibatch): the
+    kept-column list and keep bits in full, sampled rows of the gathered block bit for bit, zero fill beyond
+    the kept count; dW on sampled entries of kept rows, and exactly zero on every row that was not kept."""
+    rad, status, A, dZ = wide["rad"], wide["status"], wide["A"], wide["dZ"]
+    st = rad.Store("same", "bf16", B, D, p, seed=SEED, layer=LAYER, step=STEP, relu_bits=False)
+    rad.rad_linear_forward_store(wide["dev"]["A"], st, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    m = orc.keep_mask_at("same", [0], np.arange(D), p, SEED, LAYER, STEP)[0]
+    idx = np.flatnonzero(m)
+    k = idx.size
+    nnz = st.nnz.cpu().numpy()
+    assert nnz[0] == k and nnz[1] == k * B
+    assert np.array_equal(st.offsets[:k].cpu().numpy().view(np.uint32), idx.astype(np.uint32))
+    assert np.array_equal(st.keepbits.cpu().numpy().view(np.uint32), orc.pack_bits(m[None, :]).reshape(-1))
+    ld = int(st.c.values_ld)
+    rng = np.random.default_rng(6)
+    bs = np.concatenate([[0, 1, 63, 64, 127, 128, B - 1], rng.integers(0, B, 25)])
+    got = st.values.view(B, ld)[torch.from_numpy(bs).cuda()].view(torch.int16).cpu().numpy().view(np.uint16)
+    scale = np.float32(orc.scale_factor(p))
+    ref = orc.bf16_bits(orc.round_bf16(A[np.ix_(bs, idx)] * scale))
+    assert np.array_equal(got[:, :k], ref)
+    assert (got[:, k:] == 0).all()
+    # weight gradient from the store
+    dW = torch.full((D, H), float("nan"), dtype=torch.float32, device="cuda")
+    rad.rad_linear_weight_grad(st, wide["dev"]["dZ"], dW, dev_status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    kept = torch.from_numpy(m).cuda()
+    assert (dW[~kept] == 0).all()                       # rows of columns that were not kept: exactly zero
+    assert torch.isfinite(dW[kept]).all()
+    ds = np.concatenate([idx[[0, 1, k // 2, k - 1]], rng.choice(idx, 12)])
+    hs = np.concatenate([[0, 255, 256, H - 1], rng.integers(0, H, 12)])
+    a_c = orc.round_bf16(A[:, ds] * scale).astype(np.float64)
+    ref = a_c.T @ dZ[:, hs].astype(np.float64)
+    got = to_host_f32(dW[torch.from_numpy(ds).cuda()][:, torch.from_numpy(hs).cuda()])
+    fro, mx = rel_err(got, ref)
+    assert fro <= 2e-2 and mx <= 2e-2, (fro, mx)
+    bound = 1e-4 * (np.abs(a_c).T @ np.abs(dZ[:, hs]).astype(np.float64))
+    assert (np.abs(got - ref) <= bound + 1e-30).all()
+    del st, dW
+    torch.cuda.empty_cache()
+
+
+def test_store_counts_hold_together(wide):
+    check_counts(wide["st"], P)
+
+
+def test_weight_grad_sampled_entries(wide):
+    check_weight_grad_entries(wide["rad"], wide["st"], wide["A"], wide["dZ"], wide["dev"]["dZ"], P, wide["status"])
 
 
 def test_forward_and_input_grad_sampled_entries(wide):

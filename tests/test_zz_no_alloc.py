@@ -46,6 +46,33 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point(dtype):
             assert np.array_equal(g, w)              # integer and byte work: bit exact
 
 
+def test_many_tiles_through_the_built_in_scratch_match_the_oracle():
+    """2145 tiles: the size at which the library switches to its persistent kernel, whose per-chunk words
+    and shared claim counter then live in the built-in array.  Checked against the CPU oracle, not against
+    the other entry point; a small call right after it (the one-CTA-per-tile kernel, same array) must not
+    trip over what the large one left behind."""
+    import paper_2007_10412_b200 as rad
+    from oracle import rad as orc
+    from gpu_util import bits_host, to_dev, u32
+    from layout import bits_of, tile_major
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for (B, D, p, seed) in [(2100, 8200, 0.1, 21), (200, 300, 0.3, 22)]:
+        A, _ = layer_inputs(B, D, 1, dtype="bf16", seed=seed, relu_like=True)
+        ref = orc.forward_store(A, "bf16", "different", p, seed, 2, 5)
+        st = rad.Store("different", "bf16", B, D, p, seed=seed, layer=2, step=5)
+        st.workspace = None
+        rad.rad_linear_forward_store_static(to_dev(A, "bf16"), st, status)
+        torch.cuda.synchronize()
+        assert status.item() == 0
+        kb, vals, offs = tile_major(ref)
+        assert np.array_equal(u32(st.keepbits), kb)
+        assert np.array_equal(u32(st.offsets), offs)
+        nnz = st.nnz.cpu().numpy()
+        assert nnz[0] == ref.nnz and nnz[1] == offs[-1]
+        assert np.array_equal(bits_host(st.values[:int(offs[-1])]), bits_of(vals, "bf16"))
+        assert np.array_equal(u32(st.relubits).reshape(B, -1), ref.relubits)
+
+
 def test_limits_are_reported():
     import paper_2007_10412_b200 as rad
     A = torch.zeros(64, 128, device="cuda")
