@@ -168,6 +168,7 @@ class LayerwiseStep:
 
     def __init__(self, rad, torch, dims, B, act, variant, p, law="bernoulli"):
         self.rad, self.torch, self.dims, self.B, self.act, self.variant, self.p = rad, torch, dims, B, act, variant, p
+        self.law = law
         L = self.L = len(dims) - 1
         dev, bf = "cuda", torch.bfloat16
         self.stores = [rad.Store(variant, "bf16", B, dims[l], p, layer=l, relu_bits=False, law=law) for l in range(L)]
@@ -199,21 +200,34 @@ class LayerwiseStep:
         rad, L, dims = self.rad, self.L, self.dims
         run = self._timed if record else (lambda fam, l, fn: fn())
         a_in = X
+        # different-sample Bernoulli stores of hidden layers come out of the producing GEMM's epilogue; their
+        # index part (key only) is timed with the store family, the GEMM with the forward family
+        fused = self.variant == "different" and self.law == "bernoulli"
         for l in range(L):
-            st = self.stores[l]
-            st.c.seed, st.c.step = seed, step
-            run("store", l, lambda: rad.rad_linear_forward_store(a_in, st, self.status))
+            self.stores[l].c.seed, self.stores[l].c.step = seed, step
+        st0 = self.stores[0]
+        run("store", 0, lambda: rad.rad_linear_forward_store(a_in, st0, self.status))
+        for l in range(L):
             last = l == L - 1
             if last:
                 run("forward", l, lambda: rad.rad_linear_forward(a_in, Ws[l], bs[l], "none", out_z=self.logits,
                                                                  dev_status=self.status))
+                break
+            out = self.acts[l & 1][:, :dims[l + 1]]
+            nxt = self.stores[l + 1]
+            if fused:
+                run("store", l + 1, lambda: rad.rad_store_index(nxt, self.status))
+                run("forward", l, lambda: rad.rad_linear_forward_fill(a_in, Ws[l], bs[l], self.act, out, nxt,
+                                                                      out_zlow=self.preact[l + 1],
+                                                                      relubits=self.relubits[l + 1], index_ready=True,
+                                                                      dev_status=self.status))
             else:
-                out = self.acts[l & 1][:, :dims[l + 1]]
                 run("forward", l, lambda: rad.rad_linear_forward(a_in, Ws[l], bs[l], self.act, out_act=out,
                                                                  out_zlow=self.preact[l + 1],
                                                                  relubits=self.relubits[l + 1],
                                                                  dev_status=self.status))
-                a_in = out
+                run("store", l + 1, lambda: rad.rad_linear_forward_store(out, nxt, self.status))
+            a_in = out
         dz = self.dzs[(L - 1) & 1][:, :dims[L]]
         run("loss", L - 1, lambda: rad.rad_softmax_xent(self.logits, labels, self.loss, dz, self.ws))
         for l in range(L - 1, -1, -1):

@@ -281,6 +281,36 @@ int rad_linear_forward(int32_t dtype, int32_t act, int64_t B, int64_t D, int64_t
                        int32_t* dev_status, void* stream);
 
 /*
+ * Index part of a different-sample store from the key alone (Sec. 3.2: P is drawn independently of the
+ * data).  The keep decision of entry (b, d) depends on (seed, layer, step, b, d) only, so keepbits (keep
+ * words and in-tile row offsets), offsets and nnz of `st` can be written before the layer input exists: no
+ * input is read.  A caller can size `values` exactly from nnz[1] (read it back after the stream has
+ * reached this point), and rad_linear_forward_fill can then place the kept values from the epilogue of the
+ * GEMM that produces the input.  Bernoulli keeps only (RAD_EUNSUPPORTED otherwise); st->values may be NULL
+ * (no capacity check) and st->relubits is not touched.  Bits and layout are those of
+ * rad_linear_forward_store.
+ */
+int rad_store_index(const rad_store* st /* host */, int32_t* dev_status /* device or NULL */, void* stream);
+
+/*
+ * rad_linear_forward of a hidden layer fused with the store of its output as the next layer's input
+ * (Sec. 3: the forward pass is the original graph; Sec. 4.2: what is kept of it is a sample of each layer
+ * input): out_act = act(A W + bias) as rad_linear_forward writes it, and `next` (B x H, same dtype) filled
+ * exactly as rad_linear_forward_store(out_act, next) would fill it, without reading out_act back: the
+ * epilogue that holds a row of activations drops the kept ones into next->values at the places the index
+ * part of `next` gives.  index_ready != 0: the caller has already run rad_store_index on `next` with the
+ * same key; 0: this call runs it first.  next->relubits is ignored (the bits of out_act go to `relubits`).
+ * Shapes the fused kernel does not take (f32, unaligned or tiny layers, same-sample, other laws) run the
+ * two separate calls instead; `workspace` (device, rad_store_sizes.workspace_bytes of `next`) is used only
+ * then.
+ */
+int rad_linear_forward_fill(int32_t dtype, int32_t act, int64_t B, int64_t D, int64_t H,
+                            const void* A, int64_t lda, const void* W, int64_t ldw, const float* bias,
+                            void* out_act, int64_t ld_act, void* out_zlow, int64_t ld_zlow, uint32_t* relubits,
+                            const rad_store* next /* host */, int32_t index_ready,
+                            void* workspace, int64_t workspace_bytes, int32_t* dev_status, void* stream);
+
+/*
  * Loss Jacobian (exact, Sec. 4.2: not a memory bottleneck, never sampled):
  * loss = mean_b CE(softmax(logits_b), label_b), dZ = (softmax - onehot) / B.
  *   logits device float32 B x C; labels device int32[B]; loss device float32[1];
@@ -419,6 +449,25 @@ int rad_cnn_step(const rad_cnn_desc* net /* host */, const void* X, const int32_
                  float* const* dconv_W, float* const* dconv_b, float* const* dfc_W, float* const* dfc_b,
                  float* loss, int64_t* nnz_out, void* workspace, int64_t workspace_bytes,
                  int32_t* dev_status, void* stream);
+
+/*
+ * Device-side waits (the paper has no counterpart: this is failure handling).  Every kernel that waits for
+ * another party (an mbarrier a copy or a tensor-core commit completes, a look-back status word another CTA
+ * publishes) gives up after a time limit, raises RAD_DEV_ETIMEOUT in dev_status, lets its CTAs leave in
+ * order (copies in flight are waited for, tensor memory is released) and returns: the context stays usable.
+ * The limit is an argument of every launch; rad_set_wait_limit_ns changes the value the library passes
+ * (default 2 s; 0 only reads it) and returns the previous one.  Host only, process-wide.
+ *
+ * rad_wait_probe makes one of those waits run out on purpose, without faulting, trapping or hanging
+ * anything: a kernel of one CTA (or one cluster of two) that holds no tensor memory and has no copy in
+ * flight waits, through the same helper the real kernels use, for something that is never signalled, for
+ * `limit_ns` (at most 1 s), then raises RAD_DEV_ETIMEOUT and returns.
+ */
+#define RAD_WAIT_PAIR_BARRIER 0   /* mbarrier wait of the SM-pair GEMM kernels (cluster of two CTAs)     */
+#define RAD_WAIT_PIPE_BARRIER 1   /* mbarrier wait of the persistent store kernel                        */
+#define RAD_WAIT_LOOKBACK     2   /* look-back wait of the store kernels on a status word                */
+uint64_t rad_set_wait_limit_ns(uint64_t limit_ns);
+int rad_wait_probe(int32_t which, uint64_t limit_ns, int32_t* dev_status /* device */, void* stream);
 
 /* Kernels this library has launched since it was loaded (host-side tally; memsets not counted). */
 int64_t rad_launch_count(void);

@@ -71,8 +71,9 @@ class rad_step_stats(C.Structure):
 EXPORTS = ["rad_keep_threshold", "rad_effective_p", "rad_scale", "rad_store_size_query", "rad_set_store_kernel",
            "rad_draws_per_row", "rad_replace_scale", "rad_store_size_query_law", "rad_rademacher",
            "rad_linear_forward_store", "rad_linear_forward_store_static", "rad_weight_grad_workspace", "rad_linear_weight_grad",
-           "rad_linear_forward", "rad_softmax_xent", "rad_input_grad_workspace", "rad_linear_input_grad",
-           "rad_mlp_workspace", "rad_mlp_step", "rad_irnn_workspace", "rad_irnn_step", "rad_cnn_workspace", "rad_cnn_step", "rad_launch_count", "rad_strerror", "rad_version"]
+           "rad_linear_forward", "rad_store_index", "rad_linear_forward_fill", "rad_softmax_xent", "rad_input_grad_workspace", "rad_linear_input_grad",
+           "rad_mlp_workspace", "rad_mlp_step", "rad_irnn_workspace", "rad_irnn_step", "rad_cnn_workspace", "rad_cnn_step", "rad_launch_count", "rad_strerror", "rad_version",
+           "rad_set_wait_limit_ns", "rad_wait_probe"]
 
 _lib = None
 
@@ -109,6 +110,12 @@ def lib():
         L.rad_linear_weight_grad.argtypes = [C.POINTER(rad_store), vp, i64, i64, vp, i64, vp, i64, vp, vp]
         L.rad_linear_forward.argtypes = [i32, i32, i64, i64, i64, vp, i64, vp, i64, vp, vp, i64, vp, i64,
                                          vp, i64, vp, vp, vp]
+        L.rad_store_index.argtypes = [C.POINTER(rad_store), vp, vp]
+        L.rad_set_wait_limit_ns.restype = C.c_uint64
+        L.rad_set_wait_limit_ns.argtypes = [C.c_uint64]
+        L.rad_wait_probe.argtypes = [i32, C.c_uint64, vp, vp]
+        L.rad_linear_forward_fill.argtypes = [i32, i32, i64, i64, i64, vp, i64, vp, i64, vp, vp, i64, vp, i64, vp,
+                                              C.POINTER(rad_store), i32, vp, i64, vp, vp]
         L.rad_softmax_xent.argtypes = [i32, i64, i64, vp, i64, vp, vp, vp, i64, vp, i64, vp]
         L.rad_input_grad_workspace.argtypes = [i64, i64, C.POINTER(i64)]
         L.rad_linear_input_grad.argtypes = [i32, i64, i64, i64, vp, i64, vp, i64, vp, vp, i64, vp, i64, vp,
@@ -281,6 +288,37 @@ def rad_linear_forward(A, W, bias, act, out_act=None, out_z=None, out_zlow=None,
                                     W.stride(0), _ptr(bias), _ptr(out_act), _ld(out_act), _ptr(out_z),
                                     _ld(out_z), _ptr(out_zlow), _ld(out_zlow), _ptr(relubits),
                                     _ptr(dev_status), _stream()), "rad_linear_forward")
+
+
+WAIT_PROBES = {"pair_barrier": 0, "pipe_barrier": 1, "lookback": 2}
+
+
+def rad_set_wait_limit_ns(limit_ns):
+    """Sets the time after which device-side waits give up (0 only reads); returns the previous value."""
+    return int(lib().rad_set_wait_limit_ns(limit_ns))
+
+
+def rad_wait_probe(which, limit_ns, dev_status):
+    """Lets one of the kernels' bounded waits run out on purpose (a tiny kernel; nothing faults or hangs)."""
+    _check(lib().rad_wait_probe(WAIT_PROBES[which], limit_ns, _ptr(dev_status), _stream()), "rad_wait_probe")
+
+
+def rad_store_index(store, dev_status=None):
+    """Keep bits, row offsets, tile offsets and nnz of a different-sample store from its key alone."""
+    _check(lib().rad_store_index(C.byref(store.c), _ptr(dev_status), _stream()), "rad_store_index")
+
+
+def rad_linear_forward_fill(A, W, bias, act, out_act, next_store, out_zlow=None, relubits=None, index_ready=False,
+                            dev_status=None):
+    """Forward of a hidden layer whose epilogue also fills `next_store` from the activations it holds."""
+    B, D = A.shape
+    H = W.shape[1]
+    ws = next_store.workspace
+    _check(lib().rad_linear_forward_fill(DTYPES[A.dtype], ACTS[act], B, D, H, _ptr(A), A.stride(0), _ptr(W),
+                                         W.stride(0), _ptr(bias), _ptr(out_act), _ld(out_act), _ptr(out_zlow),
+                                         _ld(out_zlow), _ptr(relubits), C.byref(next_store.c),
+                                         1 if index_ready else 0, _ptr(ws), 0 if ws is None else ws.numel(),
+                                         _ptr(dev_status), _stream()), "rad_linear_forward_fill")
 
 
 def rad_softmax_xent(logits, labels, loss, dZ, workspace=None):

@@ -20,6 +20,9 @@ int check_device() {
 static int64_t g_launches = 0;
 void count_launch(int n) { g_launches += n; }
 
+static uint64_t g_wait_limit_ns = 2000000000ull;   // 2 s: far beyond any legitimate wait in these kernels
+uint64_t wait_limit_ns() { return g_wait_limit_ns; }
+
 namespace {
 
 bool valid_dtype(int d) { return d == RAD_F32 || d == RAD_BF16; }
@@ -112,6 +115,25 @@ using namespace rad;
 
 extern "C" int64_t rad_launch_count(void) { return g_launches; }
 
+extern "C" uint64_t rad_set_wait_limit_ns(uint64_t limit_ns) {
+  const uint64_t prev = g_wait_limit_ns;
+  if (limit_ns != 0) g_wait_limit_ns = limit_ns;
+  return prev;
+}
+
+extern "C" int rad_wait_probe(int32_t which, uint64_t limit_ns, int32_t* dev_status, void* stream) {
+  if (limit_ns == 0 || limit_ns > 1000000000ull) return RAD_EINVAL;      // a probe waits a second at most
+  const int rc = check_device();
+  if (rc != RAD_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  switch (which) {
+    case RAD_WAIT_PAIR_BARRIER: return launch_wait_probe_pair(limit_ns, dev_status, s);
+    case RAD_WAIT_PIPE_BARRIER: return launch_wait_probe_pipe(limit_ns, dev_status, s);
+    case RAD_WAIT_LOOKBACK:     return launch_wait_probe_lookback(limit_ns, dev_status, s);
+    default: return RAD_EINVAL;
+  }
+}
+
 extern "C" const char* rad_version(void) { return "rad-b200 0.1 (sm_100a)"; }
 
 extern "C" const char* rad_strerror(int code) {
@@ -188,6 +210,41 @@ extern "C" int rad_linear_forward(int32_t dtype, int32_t act, int64_t B, int64_t
                       ld_zlow, relubits, s);
 }
 
+extern "C" int rad_linear_forward_fill(int32_t dtype, int32_t act, int64_t B, int64_t D, int64_t H, const void* A,
+                                       int64_t lda, const void* W, int64_t ldw, const float* bias, void* out_act,
+                                       int64_t ld_act, void* out_zlow, int64_t ld_zlow, uint32_t* relubits,
+                                       const rad_store* next, int32_t index_ready, void* workspace,
+                                       int64_t workspace_bytes, int32_t* dev_status, void* stream) {
+  if (!valid_dtype(dtype) || B <= 0 || D <= 0 || H <= 0 || A == nullptr || W == nullptr || out_act == nullptr)
+    return RAD_EINVAL;
+  if (act != RAD_ACT_NONE && act != RAD_ACT_RELU && act != RAD_ACT_GELU) return RAD_EINVAL;
+  if (lda < D || ldw < H || ld_act < H || (out_zlow != nullptr && ld_zlow < H)) return RAD_EINVAL;
+  if (next == nullptr || next->B != B || next->D != H || next->dtype != dtype) return RAD_EINVAL;
+  int rc = check_device();
+  if (rc != RAD_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const bool fused = dtype == RAD_BF16 && next->variant == RAD_DIFFERENT_SAMPLE && next->law == RAD_LAW_BERNOULLI &&
+                     store_args_ok(next) && tc_shape_ok(B, D, H, A, lda, W, ldw) && ((uintptr_t)bias & 15) == 0 &&
+                     ((uintptr_t)out_act & 15) == 0 && ld_act % 8 == 0 && ((uintptr_t)next->keepbits & 15) == 0 &&
+                     (out_zlow == nullptr || (((uintptr_t)out_zlow & 15) == 0 && ld_zlow % 8 == 0)) &&
+                     (double)B * (double)H < 4294967296.0 * 0.75;
+  if (fused) {
+    if (!index_ready) {
+      rc = launch_store_index(next, true, dev_status, s);
+      if (rc != RAD_OK) return rc;
+    }
+    return tc_forward(act, B, D, H, A, lda, W, ldw, bias, out_act, ld_act, nullptr, 0, out_zlow, ld_zlow, relubits,
+                      dev_status, s, next);
+  }
+  // shapes the fused epilogue does not take: the same results from the two separate calls
+  rc = rad_linear_forward(dtype, act, B, D, H, A, lda, W, ldw, bias, out_act, ld_act, nullptr, 0, out_zlow, ld_zlow,
+                          relubits, dev_status, stream);
+  if (rc != RAD_OK) return rc;
+  rad_store tmp = *next;
+  tmp.relubits = nullptr;                           // the bits of out_act were written by the forward call
+  return rad_linear_forward_store(out_act, ld_act, &tmp, workspace, workspace_bytes, dev_status, stream);
+}
+
 extern "C" int rad_input_grad_workspace(int64_t B, int64_t H, int64_t* bytes) {
   if (bytes == nullptr || B <= 0 || H <= 0) return RAD_EINVAL;
   *bytes = column_sums_workspace(B, H);
@@ -245,38 +302,48 @@ extern "C" int rad_mlp_step(const rad_mlp_desc* net, const void* X, const int32_
   const int L = net->L;
   const int64_t B = net->B;
   rad_store st[64] = {};
-  const void* a_in = X;
-  int64_t ld_in = net->dims[0];
   for (int l = 0; l < L; ++l) {
-    const int64_t D = net->dims[l], H = net->dims[l + 1];
     if (W[l] == nullptr || dW[l] == nullptr || db[l] == nullptr) return RAD_EINVAL;
     const LayerPlan& lp = plan.layer[l];
     rad_store& s = st[l];
-    s.variant = net->variant; s.dtype = net->dtype; s.B = B; s.D = D; s.p = net->p;
+    s.variant = net->variant; s.dtype = net->dtype; s.B = B; s.D = net->dims[l]; s.p = net->p;
     s.layer = (uint32_t)l; s.step = net->step; s.seed = net->seed; s.law = net->law;
     s.values = ws + lp.values; s.values_capacity = lp.capacity; s.values_ld = lp.values_ld;
     s.keepbits = reinterpret_cast<uint32_t*>(ws + lp.keepbits);
     s.offsets = reinterpret_cast<uint32_t*>(ws + lp.offsets);
     s.nnz = nnz_out != nullptr ? nnz_out + 2 * l : reinterpret_cast<int64_t*>(ws + lp.nnz);
-    // the ReLU bits of this layer's input were written by the epilogue of the layer that produced it
+    // the ReLU bits of a hidden layer's input are written by the epilogue of the layer that produces it
     s.relubits = nullptr;
-    rc = rad_linear_forward_store(a_in, ld_in, &s, ws + plan.scratch, plan.scratch_bytes, dev_status, stream);
-    if (rc != RAD_OK) return rc;
-    s.relubits = lp.relubits >= 0 ? reinterpret_cast<uint32_t*>(ws + lp.relubits) : nullptr;
+  }
+  // the network input is stored by the stand-alone kernel; every hidden layer's input is stored from the
+  // epilogue of the GEMM that produces it (or by the same stand-alone call where that kernel does not apply)
+  rc = rad_linear_forward_store(X, net->dims[0], &st[0], ws + plan.scratch, plan.scratch_bytes, dev_status, stream);
+  if (rc != RAD_OK) return rc;
+  const void* a_in = X;
+  int64_t ld_in = net->dims[0];
+  for (int l = 0; l < L; ++l) {
+    const int64_t D = net->dims[l], H = net->dims[l + 1];
     const bool last = (l == L - 1);
-    void* a_out = last ? nullptr : ws + plan.act[l & 1];
+    if (last) {
+      rc = rad_linear_forward(net->dtype, RAD_ACT_NONE, B, D, H, a_in, ld_in, W[l], H, b != nullptr ? b[l] : nullptr,
+                              nullptr, H, reinterpret_cast<float*>(ws + plan.logits), H, nullptr, H, nullptr,
+                              dev_status, stream);
+      if (rc != RAD_OK) return rc;
+      break;
+    }
+    void* a_out = ws + plan.act[l & 1];
     // a GELU net keeps the pre-activation of layer l for the backward of layer l + 1's input
-    void* zlow = (!last && net->act == RAD_ACT_GELU) ? ws + plan.layer[l + 1].preact : nullptr;
-    rc = rad_linear_forward(net->dtype, last ? RAD_ACT_NONE : net->act, B, D, H, a_in, ld_in, W[l], H,
-                            b != nullptr ? b[l] : nullptr, a_out, H,
-                            last ? reinterpret_cast<float*>(ws + plan.logits) : nullptr, H, zlow, H,
-                            (!last && plan.layer[l + 1].relubits >= 0)
-                                ? reinterpret_cast<uint32_t*>(ws + plan.layer[l + 1].relubits) : nullptr,
-                            dev_status, stream);
+    void* zlow = net->act == RAD_ACT_GELU ? ws + plan.layer[l + 1].preact : nullptr;
+    uint32_t* rbits = plan.layer[l + 1].relubits >= 0 ? reinterpret_cast<uint32_t*>(ws + plan.layer[l + 1].relubits) : nullptr;
+    rc = rad_linear_forward_fill(net->dtype, net->act, B, D, H, a_in, ld_in, W[l], H, b != nullptr ? b[l] : nullptr,
+                                 a_out, H, zlow, H, rbits, &st[l + 1], 0, ws + plan.scratch, plan.scratch_bytes,
+                                 dev_status, stream);
     if (rc != RAD_OK) return rc;
     a_in = a_out;
     ld_in = H;
   }
+  for (int l = 1; l < L; ++l)
+    st[l].relubits = plan.layer[l].relubits >= 0 ? reinterpret_cast<uint32_t*>(ws + plan.layer[l].relubits) : nullptr;
   const int64_t C = net->dims[L];
   void* dz = ws + plan.dz[(L - 1) & 1];
   rc = rad_softmax_xent(net->dtype, B, C, reinterpret_cast<const float*>(ws + plan.logits), C, labels, loss, dz,

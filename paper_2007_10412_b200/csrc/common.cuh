@@ -166,6 +166,10 @@ inline int64_t round_up(int64_t a, int64_t b) { return ceil_div(a, b) * b; }
   } while (0)
 
 // internal launchers shared across translation units --------------------------------------------
+uint64_t wait_limit_ns();       // time after which a device-side wait gives up (api.cu; rad_set_wait_limit_ns)
+int launch_wait_probe_pair(uint64_t limit_ns, int32_t* dev_status, cudaStream_t s);      // tc.cu
+int launch_wait_probe_pipe(uint64_t limit_ns, int32_t* dev_status, cudaStream_t s);      // store_pipe.cu
+int launch_wait_probe_lookback(uint64_t limit_ns, int32_t* dev_status, cudaStream_t s);  // store.cu
 int check_device();   // RAD_OK on an sm_100 device
 void count_launch(int n = 1);   // host-side tally of kernels this library has launched
 void* tensor_map_encoder();     // cuTensorMapEncodeTiled, or nullptr (tc.cu)
@@ -212,7 +216,10 @@ bool tc_shape_ok(int64_t B, int64_t D, int64_t H, const void* p0, int64_t ld0, c
 int tc_forward(int act, int64_t B, int64_t D, int64_t H, const void* A, int64_t lda, const void* W,
                int64_t ldw, const float* bias, void* out_act, int64_t ld_act, float* out_z,
                int64_t ld_z, void* out_zlow, int64_t ld_zlow, uint32_t* relubits,
-               int32_t* dev_status, cudaStream_t s);
+               int32_t* dev_status, cudaStream_t s, const rad_store* next = nullptr);
+// store_index.cu: keep bits, row offsets, tile offsets and nnz of a different-sample Bernoulli store from the
+// key alone (no layer input is read)
+int launch_store_index(const rad_store* st, bool check_capacity, int32_t* dev_status, cudaStream_t s);
 int tc_input_grad(int64_t B, int64_t D, int64_t H, const void* dZ, int64_t ldz, const void* W,
                   int64_t ldw, const uint32_t* relubits_prev, const void* z_prev, int64_t ld_zprev,
                   void* dZ_prev, int64_t ldp, int32_t* dev_status, cudaStream_t s);

@@ -45,9 +45,15 @@ __global__ void __launch_bounds__(256) scale_convert_kernel(const float* in, T* 
     out[i] = from_float<T>(__fmul_rn(in[i], scale));
 }
 
-__global__ void project_meta_kernel(uint32_t* idx, int64_t ld, int64_t* nnz, int64_t k, int64_t B) {
-  for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < ld; j += (int64_t)gridDim.x * blockDim.x)
+// idx: the identity list of ld columns; bits: bit j set for j < k (the columns of S that hold data)
+__global__ void project_meta_kernel(uint32_t* idx, uint32_t* bits, int64_t ld, int64_t* nnz, int64_t k, int64_t B) {
+  for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < ld; j += (int64_t)gridDim.x * blockDim.x) {
     if (idx != nullptr) idx[j] = (uint32_t)j;
+    if (bits != nullptr && (j & 31) == 0) {
+      const int64_t nv = k - j;
+      bits[j >> 5] = nv >= 32 ? 0xffffffffu : nv <= 0 ? 0u : (1u << nv) - 1u;
+    }
+  }
   if (nnz != nullptr && blockIdx.x == 0 && threadIdx.x == 0) { nnz[0] = k; nnz[1] = k * B; }
 }
 
@@ -70,11 +76,11 @@ int draw_signs(int dtype, void* out, int64_t D, int64_t k, int64_t ld, uint64_t 
 }
 
 // the stand-in the same-sample weight-gradient path takes: a B x ld block with all of its columns kept
-rad_store as_dense_block(const rad_store* st, uint32_t* idx) {
+rad_store as_dense_block(const rad_store* st, uint32_t* idx, uint32_t* bits) {
   rad_store t = {};
   t.variant = RAD_SAME_SAMPLE; t.dtype = st->dtype; t.B = st->B; t.D = st->values_ld; t.p = 1.0f;
   t.values = st->values; t.values_capacity = st->values_capacity; t.values_ld = st->values_ld;
-  t.keepbits = idx; t.offsets = idx; t.nnz = st->nnz;
+  t.keepbits = bits; t.offsets = idx; t.nnz = st->nnz;
   return t;
 }
 
@@ -92,8 +98,8 @@ int64_t project_store_workspace(int dtype, int64_t D, int64_t ld) { return round
 
 int64_t project_weight_grad_workspace(const rad_store* st, int64_t H) {
   const int64_t ld = st->values_ld, es = esz(st->dtype);
-  rad_store t = as_dense_block(st, nullptr);
-  return round_up(st->D * ld * es, 256) + round_up(ld * 4, 256) + round_up(ld * H * 4, 256) + round_up(ld * H * es, 256) +
+  rad_store t = as_dense_block(st, nullptr, nullptr);
+  return round_up(st->D * ld * es, 256) + round_up(ld * 4, 256) + round_up(ceil_div(ld, 32) * 4, 256) + round_up(ld * H * 4, 256) + round_up(ld * H * es, 256) +
          round_up(tc_weight_grad_workspace(&t, H), 256);
 }
 
@@ -106,7 +112,7 @@ int project_forward_store(const void* A, int64_t lda, const rad_store* st, void*
   int rc = draw_signs(st->dtype, workspace, st->D, k, ld, st->seed, st->layer, st->step, s);
   if (rc != RAD_OK) return rc;
   count_launch();
-  project_meta_kernel<<<1, 32, 0, s>>>(nullptr, 0, st->nnz, k, st->B);
+  project_meta_kernel<<<1, 32, 0, s>>>(nullptr, nullptr, 0, st->nnz, k, st->B);
   // S = A R': B x D times D x ld, stored in the working type
   rc = rad_linear_forward(st->dtype, RAD_ACT_NONE, st->B, st->D, ld, A, lda, workspace, ld, nullptr, st->values, ld,
                           nullptr, 0, nullptr, 0, nullptr, dev_status, stream);
@@ -124,15 +130,16 @@ int project_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_
   char* ws = static_cast<char*>(workspace);
   void* R = ws;                                   ws += round_up(st->D * ld * es, 256);
   uint32_t* idx = reinterpret_cast<uint32_t*>(ws);  ws += round_up(ld * 4, 256);
+  uint32_t* bits = reinterpret_cast<uint32_t*>(ws); ws += round_up(ceil_div(ld, 32) * 4, 256);
   float* G32 = reinterpret_cast<float*>(ws);      ws += round_up(ld * H * 4, 256);
   void* G = ws;                                   ws += round_up(ld * H * es, 256);
   const int64_t inner = workspace_bytes - (ws - static_cast<char*>(workspace));
   int rc = draw_signs(st->dtype, R, st->D, k, ld, st->seed, st->layer, st->step, s);
   if (rc != RAD_OK) return rc;
   count_launch();
-  project_meta_kernel<<<(unsigned)std::min<int64_t>(ceil_div(ld, 256), 1024), 256, 0, s>>>(idx, ld, nullptr, 0, 0);
+  project_meta_kernel<<<(unsigned)std::min<int64_t>(ceil_div(ld, 256), 1024), 256, 0, s>>>(idx, bits, ld, nullptr, k, 0);
   // G32 = S^T dZ (ld x H): the dense block of S goes through the same-sample contraction with every column kept
-  const rad_store t = as_dense_block(st, idx);
+  const rad_store t = as_dense_block(st, idx, bits);
   rc = rad_linear_weight_grad(&t, dZ, ldz, H, G32, H, ws, inner, dev_status, stream);
   if (rc != RAD_OK) return rc;
   // G = (S^T dZ) / k in the working type

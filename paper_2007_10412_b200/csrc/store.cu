@@ -239,15 +239,7 @@ __global__ void __launch_bounds__(256) store_different_kernel(const StoreParams 
       while (!done) {
         const int64_t j = idx - lane;
         uint64_t w = kFlagPrefix << kFlagShift;          // before the first tile: prefix 0
-        if (j >= 0) {
-          int spins = 0;
-          w = load_status(p.status + j);
-          while ((w >> kFlagShift) == 0 && spins < kSpinLimit) {
-            __nanosleep(spins < 64 ? 32 : 256);
-            w = load_status(p.status + j);
-            ++spins;
-          }
-        }
+        if (j >= 0) w = wait_status(p.status + j, p.wait_limit_ns);
         const uint64_t flag = w >> kFlagShift;
         if (__any_sync(0xffffffffu, flag == 0 || flag == kFlagPoison)) { failed = true; break; }
         const uint32_t pm = __ballot_sync(0xffffffffu, flag == kFlagPrefix);
@@ -567,6 +559,14 @@ __global__ void __launch_bounds__(1024) same_replace_mask_kernel(const SameParam
   }
 }
 
+// The look-back's wait on a status word that nobody publishes (a word of the probe's own that stays zero):
+// it gives up after `limit_ns` and the status word reports the timeout, as the store kernels do.
+__device__ uint64_t g_probe_status_word;
+__global__ void wait_probe_lookback_kernel(uint64_t limit_ns, int32_t* dev_status) {
+  const uint64_t w = wait_status(&g_probe_status_word, limit_ns);
+  if ((w >> kFlagShift) == 0) raise_status(dev_status, RAD_DEV_ETIMEOUT);
+}
+
 constexpr int kPipelinedMinTiles = 2048;
 int g_store_kernel = RAD_STORE_KERNEL_AUTO;
 
@@ -614,6 +614,11 @@ constexpr int64_t kMaxCountsRowBytes = 200 * 1024;   // a row's histogram has to
 }  // namespace rad
 
 namespace rad {
+int launch_wait_probe_lookback(uint64_t limit_ns, int32_t* dev_status, cudaStream_t s) {
+  count_launch();
+  wait_probe_lookback_kernel<<<1, 32, 0, s>>>(limit_ns, dev_status);
+  return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
+}
 int launch_relu_bits(int dtype, const void* A, int64_t lda, int64_t B, int64_t D, uint32_t* relubits, cudaStream_t s) {
   const int64_t w32 = ceil_div(D, 32), n = B * w32;
   const int g2 = (int)std::min<int64_t>(ceil_div(n, 256), 148 * 16);
@@ -760,6 +765,7 @@ extern "C" int rad_linear_forward_store(const void* A, int64_t lda, const rad_st
     p.dev_status = dev_status;
     p.vec_ok = (((uintptr_t)A & 15) == 0 && (lda * esz) % 16 == 0) ? 1 : 0;
     p.counts = nullptr; p.ldc = 0;
+    p.wait_limit_ns = wait_limit_ns();
     RAD_CUDA_TRY(cudaMemsetAsync(workspace, 0, (size_t)status_bytes(st->B, st->D), s));
     if (replace) {
       // first the multiplicities of every row, then the generic kernel with the mask and the weights
@@ -891,6 +897,7 @@ extern "C" int rad_linear_forward_store_static(const void* A, int64_t lda, const
   p.dev_status = dev_status;
   p.vec_ok = (((uintptr_t)A & 15) == 0 && (lda * esz) % 16 == 0) ? 1 : 0;
   p.counts = nullptr; p.ldc = 0;
+  p.wait_limit_ns = wait_limit_ns();
   // the array keeps what the last call left: the counter and this call's status words start at zero
   RAD_CUDA_TRY(cudaMemsetAsync(scratch, 0, 256 + 8 * (size_t)ntiles, s));
   return launch_store_different(p, ks, st->dtype, T, s);

@@ -10,7 +10,26 @@ namespace rad {
 constexpr uint64_t kFlagShift = 62;
 constexpr uint64_t kFlagAggregate = 1, kFlagPrefix = 2, kFlagPoison = 3;
 constexpr uint64_t kValueMask = (1ull << kFlagShift) - 1;
-constexpr int kSpinLimit = 1 << 20;   // bounded wait: about a second with the back-off below
+
+// Bounded wait for a status word to get its flag: polls with a back-off of 32 ns, then 256 ns, and gives up
+// (returns the word with flag 0) once `limit_ns` has passed.
+__device__ __forceinline__ uint64_t load_status(const uint64_t* p);
+__device__ __forceinline__ uint64_t wait_status(const uint64_t* p, uint64_t limit_ns) {
+  uint64_t w = load_status(p);
+  if ((w >> kFlagShift) != 0) return w;
+  uint64_t t0;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+  for (int spins = 0;; ++spins) {
+    __nanosleep(spins < 64 ? 32 : 256);
+    w = load_status(p);
+    if ((w >> kFlagShift) != 0) return w;
+    if ((spins & 15) == 15) {
+      uint64_t t;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+      if (t - t0 > limit_ns) return w;
+    }
+  }
+}
 
 __device__ __forceinline__ uint64_t pack_counts(uint32_t granules, uint32_t exact) {
   return ((uint64_t)granules << 32) | exact;
@@ -48,6 +67,7 @@ struct StoreParams {
   uint64_t* status;   // ntiles look-back words (zeroed before launch)
   uint32_t* ticket;   // zeroed before launch
   int32_t* dev_status;
+  uint64_t wait_limit_ns;   // every device-side wait of the launch gives up after this long
   int32_t vec_ok;     // rows are 16-byte aligned: 8-element vector loads allowed
   // with-replacement law: multiplicities, one byte per entry, rows of ldc bytes (ldc a multiple of 16);
   // nullptr: Bernoulli keeps drawn in the kernel

@@ -5,12 +5,13 @@
 // then drops the kept values into place from its epilogue (tc.cu), and a caller learns the exact size of a
 // store before it allocates `values`.
 //
-//   store_index_kernel   one tile (64 x 128 entries) per CTA and turn, one keep-bit word per thread: draw, write
-//                        the word, in-tile row offsets from a CTA scan, exact kept count of the tile into
-//                        offsets[tile]
+//   store_index_kernel   one tile (64 x 128 entries) per warp and turn: draw and write the keep-bit words,
+//                        in-tile row offsets from warp scans, exact kept count of the tile into offsets[tile]
 //   offsets_scan_kernel  one CTA turns the counts into padded exclusive prefixes in place and writes nnz
 //
 // Layout and bits are those of the one-pass store kernels.
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace rad {
@@ -28,82 +29,96 @@ struct IndexParams {
   int32_t* dev_status;
 };
 
-__global__ void __launch_bounds__(256) store_index_kernel(const IndexParams p, const PhiloxKeys ks) {
-  __shared__ uint32_t s_warp[8];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int r = tid >> 2, w = tid & 3;              // row of the tile, keep-bit word of the row
-  for (int64_t tile = blockIdx.x; tile < p.ntiles; tile += gridDim.x) {
-    const int64_t slab = tile / p.ncb;
-    const int cb = (int)(tile - slab * p.ncb);
-    const int64_t row = slab * kTileRows + r;
-    const int64_t col0 = (int64_t)cb * kTileCols + 32 * w;
-    uint32_t m = 0;
-    if (row < p.B && col0 < p.D) {
-      m = philox_keep32((uint32_t)(col0 >> 5), (uint32_t)row, p.c2, p.c3, ks, p.T);
-      const int64_t nv = p.D - col0;
-      if (nv < 32) m &= (1u << nv) - 1u;
-    }
-    p.keepbits[tile * kTileWords + tid] = m;
-    // exclusive prefix over the tile's words in (row, word) order = thread order
-    const uint32_t c = __popc(m);
-    uint32_t incl = c;
+// One warp per tile and turn, no CTA-wide step: lane l draws words l, l + 32, ... of the tile (word t = row
+// t / 4, columns 32 (t % 4) ..), so a warp's stores are contiguous and a warp scan per turn, carried over
+// the eight turns, gives every row its offset in (row, column) order.
+constexpr int kIndexWarps = 4;
+__global__ void __launch_bounds__(32 * kIndexWarps) store_index_kernel(const IndexParams p, const PhiloxKeys ks) {
+  const int lane = threadIdx.x & 31;
+  const uint32_t warp0 = blockIdx.x * kIndexWarps + (threadIdx.x >> 5), nwarps = gridDim.x * kIndexWarps;
+  const uint32_t nrows = (uint32_t)p.B, ncols = (uint32_t)p.D, ncb = (uint32_t)p.ncb;
+  const int w = lane & 3;
+  for (uint32_t tile = warp0; tile < (uint32_t)p.ntiles; tile += nwarps) {
+    const uint32_t slab = tile / ncb, cb = tile - slab * ncb;
+    const uint32_t col0 = cb * kTileCols + 32u * w;
+    uint32_t* tw = p.keepbits + (int64_t)tile * kTileWords;
+    uint32_t base = 0;
+#pragma unroll 2
+    for (int i = 0; i < kBitWords / 32; ++i) {
+      const int r = i * 8 + (lane >> 2);
+      const uint32_t row = slab * kTileRows + r;
+      uint32_t m = 0;
+      if (row < nrows && col0 < ncols) {
+        m = philox_keep32(col0 >> 5, row, p.c2, p.c3, ks, p.T);
+        const uint32_t nv = ncols - col0;
+        if (nv < 32) m &= (1u << nv) - 1u;
+      }
+      tw[i * 32 + lane] = m;
+      const uint32_t c = __popc(m);
+      uint32_t incl = c;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t n = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += n;
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t n = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += n;
+      }
+      if (w == 0) reinterpret_cast<uint16_t*>(tw + kBitWords)[r] = (uint16_t)(base + incl - c);
+      base += __shfl_sync(0xffffffffu, incl, 31);
     }
-    if (lane == 31) s_warp[warp] = incl;
-    __syncthreads();
-    uint32_t before = 0, total = 0;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const uint32_t t = s_warp[i];
-      if (i < warp) before += t;
-      total += t;
-    }
-    if (w == 0) reinterpret_cast<uint16_t*>(p.keepbits + tile * kTileWords + kBitWords)[r] = (uint16_t)(before + incl - c);
-    if (tid == 0) p.offsets[tile] = total;
-    __syncthreads();                                // s_warp is rewritten in the next turn
+    if (lane == 0) p.offsets[tile] = base;
   }
 }
 
 // offsets[t] holds the exact kept count of tile t on entry and the first element of tile t in `values` on
-// exit (every tile padded to a multiple of kValueAlign); offsets[ntiles] = elements used.
+// exit (every tile padded to a multiple of kValueAlign); offsets[ntiles] = elements used.  One CTA: a thread
+// takes 16 consecutive tiles per round (its loads are issued together), 16384 tiles per round.
+constexpr int kScanPer = 16;
 __global__ void __launch_bounds__(1024) offsets_scan_kernel(const IndexParams p) {
-  __shared__ uint64_t s_pad[32], s_exact[32];
+  __shared__ uint32_t s_pad[32], s_exact[32];
+  __shared__ uint64_t s_carry_pad, s_carry_exact;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int64_t per = (p.ntiles + 1023) / 1024;
-  const int64_t t0 = min((int64_t)tid * per, (int64_t)p.ntiles), t1 = min(t0 + per, (int64_t)p.ntiles);
-  uint64_t pad = 0, exact = 0;
-  for (int64_t t = t0; t < t1; ++t) {
-    const uint32_t c = p.offsets[t];
-    exact += c;
-    pad += (c + kValueAlign - 1) / kValueAlign * kValueAlign;
-  }
-  uint64_t ipad = pad, iex = exact;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const uint64_t a = __shfl_up_sync(0xffffffffu, ipad, o), b = __shfl_up_sync(0xffffffffu, iex, o);
-    if (lane >= o) { ipad += a; iex += b; }
-  }
-  if (lane == 31) { s_pad[warp] = ipad; s_exact[warp] = iex; }
+  if (tid == 0) { s_carry_pad = 0; s_carry_exact = 0; }
   __syncthreads();
-  uint64_t base = ipad - pad, all_pad = 0, all_exact = 0;
-  for (int i = 0; i < 32; ++i) {
-    if (i < warp) base += s_pad[i];
-    all_pad += s_pad[i];
-    all_exact += s_exact[i];
-  }
-  for (int64_t t = t0; t < t1; ++t) {
-    const uint32_t c = p.offsets[t];
-    p.offsets[t] = (uint32_t)base;
-    base += (c + kValueAlign - 1) / kValueAlign * kValueAlign;
+  const int64_t ntiles = p.ntiles;
+  for (int64_t r0 = 0; r0 < ntiles; r0 += 1024 * kScanPer) {
+    const int64_t t0 = r0 + (int64_t)tid * kScanPer;
+    uint32_t c[kScanPer];
+#pragma unroll
+    for (int i = 0; i < kScanPer; ++i) c[i] = t0 + i < ntiles ? p.offsets[t0 + i] : 0u;
+    uint32_t pad = 0, exact = 0;                    // a round holds at most 16384 * 8192 entries: 32 bits do
+#pragma unroll
+    for (int i = 0; i < kScanPer; ++i) {
+      exact += c[i];
+      pad += (c[i] + kValueAlign - 1) / kValueAlign * kValueAlign;
+    }
+    uint32_t ipad = pad, iex = exact;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t a = __shfl_up_sync(0xffffffffu, ipad, o), b = __shfl_up_sync(0xffffffffu, iex, o);
+      if (lane >= o) { ipad += a; iex += b; }
+    }
+    if (lane == 31) { s_pad[warp] = ipad; s_exact[warp] = iex; }
+    __syncthreads();
+    uint64_t base = s_carry_pad + (ipad - pad), round_pad = 0, round_exact = 0;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      if (i < warp) base += s_pad[i];
+      round_pad += s_pad[i];
+      round_exact += s_exact[i];
+    }
+#pragma unroll
+    for (int i = 0; i < kScanPer; ++i) {
+      if (t0 + i < ntiles) p.offsets[t0 + i] = (uint32_t)base;
+      base += (c[i] + kValueAlign - 1) / kValueAlign * kValueAlign;
+    }
+    __syncthreads();                                // everyone has read the carry and the warp totals
+    if (tid == 0) { s_carry_pad += round_pad; s_carry_exact += round_exact; }
+    __syncthreads();
   }
   if (tid == 0) {
-    p.offsets[p.ntiles] = (uint32_t)all_pad;
-    p.nnz[0] = (int64_t)all_exact;
-    p.nnz[1] = (int64_t)all_pad;
-    if (p.capacity >= 0 && (int64_t)all_pad > p.capacity) raise_status(p.dev_status, RAD_DEV_ECAPACITY);
+    p.offsets[ntiles] = (uint32_t)s_carry_pad;
+    p.nnz[0] = (int64_t)s_carry_exact;
+    p.nnz[1] = (int64_t)s_carry_pad;
+    if (p.capacity >= 0 && (int64_t)s_carry_pad > p.capacity) raise_status(p.dev_status, RAD_DEV_ECAPACITY);
   }
 }
 
@@ -122,9 +137,9 @@ int launch_store_index(const rad_store* st, bool check_capacity, int32_t* dev_st
   p.capacity = check_capacity ? st->values_capacity : -1;
   p.dev_status = dev_status;
   const PhiloxKeys ks = philox_expand_key(st->seed);
-  const int grid = (int)std::min<int64_t>(p.ntiles, 148 * 8);
+  const int grid = (int)std::min<int64_t>(ceil_div(p.ntiles, kIndexWarps), 148 * 12);
   count_launch(2);
-  store_index_kernel<<<grid, 256, 0, s>>>(p, ks);
+  store_index_kernel<<<grid, 32 * kIndexWarps, 0, s>>>(p, ks);
   offsets_scan_kernel<<<1, 1024, 0, s>>>(p);
   return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
 }

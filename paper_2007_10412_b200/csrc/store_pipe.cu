@@ -38,7 +38,6 @@ constexpr int kAhead = 2;                       // chunks between the first and 
 constexpr int kSlots = 8;                       // chunk descriptors in flight
 constexpr int kLookWindows = 8;                 // look-back: 32 status words per window
 constexpr uint32_t kNoChunk = 0xffffffffu;
-constexpr uint64_t kPipeWaitLimitNs = 2000000000ull;
 constexpr int kTileElems = kTileRows * kTileCols;
 constexpr int kWarpElems = kTileElems / kWarpsPerTile;   // entries of a tile that one warp owns (16 rows)
 
@@ -82,7 +81,11 @@ __device__ __forceinline__ uint64_t timer_ns() {
 }
 // Bounded wait; false when the CTA is giving up (this wait or another one ran out of time).  The
 // slow path is kept out of line: it is rarely taken and the kernel's code should stay small.
-__device__ __noinline__ bool bar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint32_t sleep_ns) {
+struct PipeWait {
+  volatile int* abort_flag;   // the CTA's flag: set by the wait that runs out, seen by all the others
+  uint64_t limit_ns;          // time limit of the launch (a kernel argument)
+};
+__device__ __noinline__ bool bar_wait_slow(uint64_t* bar, uint32_t parity, const PipeWait& wc, uint32_t sleep_ns) {
   const uint64_t t0 = timer_ns();
   while (true) {
 #pragma unroll 1
@@ -90,16 +93,16 @@ __device__ __noinline__ bool bar_wait_slow(uint64_t* bar, uint32_t parity, volat
       if (bar_try_wait(bar, parity)) return true;
       if (sleep_ns != 0) __nanosleep(sleep_ns);   // a waiting warp leaves the issue slots to the others
     }
-    if (*abort_flag != 0) return false;
-    if (timer_ns() - t0 > kPipeWaitLimitNs) {
-      *abort_flag = 1;
+    if (*wc.abort_flag != 0) return false;
+    if (timer_ns() - t0 > wc.limit_ns) {
+      *wc.abort_flag = 1;
       return false;
     }
   }
 }
-__device__ __forceinline__ bool bar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint32_t sleep_ns = 40) {
+__device__ __forceinline__ bool bar_wait(uint64_t* bar, uint32_t parity, const PipeWait& wc, uint32_t sleep_ns = 40) {
   if (bar_try_wait(bar, parity)) return true;
-  return bar_wait_slow(bar, parity, abort_flag, sleep_ns);
+  return bar_wait_slow(bar, parity, wc, sleep_ns);
 }
 __device__ __forceinline__ void tma_load_tile(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
   asm volatile(
@@ -179,6 +182,7 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
   PipeSmem<T, S>& sm = *reinterpret_cast<PipeSmem<T, S>*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   volatile int* abort_flag = &sm.abort_flag;
+  const PipeWait wc = {abort_flag, p.wait_limit_ns};
   const uint32_t ntiles = (uint32_t)p.ntiles;
   const uint32_t nchunks = (ntiles + kChunk - 1) / kChunk;
 
@@ -208,7 +212,7 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
     // m[2 i], m[2 i + 1]: this thread's two words of its tile in step i of the chunk
     auto phase1 = [&](uint32_t seq, uint32_t (&m)[kChunk]) -> uint32_t {
       const int slot = seq % kSlots;
-      if (!bar_wait(&sm.chunk_ready[slot], (seq / kSlots) & 1u, abort_flag)) return kNoChunk;
+      if (!bar_wait(&sm.chunk_ready[slot], (seq / kSlots) & 1u, wc)) return kNoChunk;
       const uint32_t chunk = sm.chunk_id[slot];
       if (chunk == kNoChunk) return kNoChunk;
 #pragma unroll
@@ -245,8 +249,8 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
     // Second phase of one chunk (slot: its descriptor, m: its keep-bit words).  false: a wait gave up.
     auto phase2 = [&](uint32_t chunk, int slot, uint32_t slot_parity, const uint32_t (&m)[kChunk]) -> bool {
       // the other warps' totals of the first phase and the chunk's place in `values` are needed now
-      if (!bar_wait(&sm.cnt_ready[slot], slot_parity, abort_flag) ||
-          !bar_wait(&sm.base_ready[slot], slot_parity, abort_flag))
+      if (!bar_wait(&sm.cnt_ready[slot], slot_parity, wc) ||
+          !bar_wait(&sm.base_ready[slot], slot_parity, wc))
         return false;
       T* const wb = sm.wbuf[warp];
       const uint32_t valid = min((uint32_t)kChunk, ntiles - chunk * kChunk);   // tiles of this chunk
@@ -267,7 +271,7 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
           reinterpret_cast<uint16_t*>(p.keepbits + (int64_t)tile * kTileWords + kBitWords)[r] =
               (uint16_t)(wbase + incl - cnt);
         const int64_t base = sm.tile_base[slot][g];
-        if (!bar_wait(&sm.full[s], (pos / S) & 1u, abort_flag)) return false;
+        if (!bar_wait(&sm.full[s], (pos / S) & 1u, wc)) return false;
         const T* src = sm.raw[s] + r * kTileCols + half * 64;
         // Kept entries go to the warp's buffer as they are (bit h of a reversed word is column 31 - h);
         // scaling waits for the copy to `values`, where every lane has work.  The buffer is filled from
@@ -388,7 +392,7 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
           const uint32_t tile = q[0] * kChunk + g;
           if (tile >= ntiles) break;
           const int s = n % S;
-          if (!bar_wait(&sm.empty[s], ((n / S) & 1u) ^ 1u, abort_flag, 0)) { ok = false; break; }
+          if (!bar_wait(&sm.empty[s], ((n / S) & 1u) ^ 1u, wc, 0)) { ok = false; break; }
           const uint32_t slab = tile / (uint32_t)p.ncb, cb = tile - slab * (uint32_t)p.ncb;
           bar_arrive_expect_tx(&sm.full[s], (uint32_t)(kTileElems * sizeof(T)));
           tma_load_tile(sm.raw[s], &tmA, (int)(cb * kTileCols), (int)(slab * kTileRows), &sm.full[s]);
@@ -403,7 +407,7 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
         const uint32_t first = n > (uint32_t)S ? n - S : 0u;
         for (uint32_t i = first; i < n; ++i) {
           const uint64_t t0 = timer_ns();
-          while (!bar_try_wait(&sm.full[i % S], (i / S) & 1u) && timer_ns() - t0 < kPipeWaitLimitNs) {}
+          while (!bar_try_wait(&sm.full[i % S], (i / S) & 1u) && timer_ns() - t0 < p.wait_limit_ns) {}
         }
       }
     }
@@ -417,10 +421,10 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
     auto publish = [&](uint32_t seq, Counts& c) -> uint32_t {
       const int slot = seq % kSlots;
       const uint32_t par = (seq / kSlots) & 1u;
-      if (!bar_wait(&sm.chunk_ready[slot], par, abort_flag, 400)) return kNoChunk;
+      if (!bar_wait(&sm.chunk_ready[slot], par, wc, 400)) return kNoChunk;
       const uint32_t chunk = sm.chunk_id[slot];
       if (chunk == kNoChunk) return kNoChunk;
-      if (!bar_wait(&sm.cnt_ready[slot], par, abort_flag, 400)) return kNoChunk;
+      if (!bar_wait(&sm.cnt_ready[slot], par, wc, 400)) return kNoChunk;
       // lane (4 g + v) reads warp v's total of tile g; a butterfly over four lanes sums a tile
       static_assert(kChunk * kWarpsPerTile == 32, "one (tile, warp) entry per lane");
       uint32_t t = sm.warp_total[slot][lane >> 2][lane & 3];
@@ -466,12 +470,7 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
           for (int k = 0; k < kLookWindows; ++k) {
             if (done || failed) break;
             const int64_t j = idx - 32 * k - lane;
-            int spins = 0;
-            while ((w[k] >> kFlagShift) == 0 && spins < kSpinLimit) {
-              __nanosleep(spins < 64 ? 32 : 256);
-              w[k] = load_status(p.status + j);
-              ++spins;
-            }
+            if ((w[k] >> kFlagShift) == 0) w[k] = wait_status(p.status + j, p.wait_limit_ns);
             const uint64_t flag = w[k] >> kFlagShift;
             if (__any_sync(0xffffffffu, flag == 0 || flag == kFlagPoison)) { failed = true; break; }
             const uint32_t pm = __ballot_sync(0xffffffffu, flag == kFlagPrefix);
@@ -529,6 +528,24 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
   if (tid == 0 && sm.abort_flag != 0) raise_status(p.dev_status, RAD_DEV_ETIMEOUT);
 }
 
+// The kernel's bounded barrier wait on a barrier nobody arrives at, in one CTA that has no loads in flight:
+// the wait runs out, the abort flag goes up, and the status word reports the timeout on the way out.
+__global__ void wait_probe_pipe_kernel(uint64_t limit_ns, int32_t* dev_status) {
+  __shared__ uint64_t bar;
+  __shared__ int flag;
+  if (threadIdx.x == 0) {
+    bar_init(&bar, 1);
+    flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const PipeWait wc = {&flag, limit_ns};
+  bool ok = true;
+  if (threadIdx.x == 0) ok = bar_wait(&bar, 0u, wc, 100);
+  __syncthreads();
+  if (threadIdx.x == 0 && (!ok || flag != 0)) raise_status(dev_status, RAD_DEV_ETIMEOUT);
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -558,6 +575,12 @@ int launch_typed(const StoreParams& p, const PhiloxKeys& ks, const CUtensorMap& 
 }
 
 }  // namespace
+
+int launch_wait_probe_pipe(uint64_t limit_ns, int32_t* dev_status, cudaStream_t s) {
+  count_launch();
+  wait_probe_pipe_kernel<<<1, 64, 0, s>>>(limit_ns, dev_status);
+  return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
+}
 
 int launch_store_pipelined(const StoreParams& p, const PhiloxKeys& ks, int dtype, cudaStream_t s) {
   const size_t esz = dtype == RAD_BF16 ? 2 : 4;

@@ -37,11 +37,12 @@ constexpr int kRasterGroup = 8;                // m-tiles per raster group
 
 enum AKind { kAK = 0, kAMN = 1, kASparse = 2 };
 enum BKind { kBK_ = 0, kBMN = 1 };
-enum EpiKind { kFwd = 0, kDx = 1, kDw = 2 };
+enum EpiKind { kFwd = 0, kDx = 1, kDw = 2, kDwT = 3 };
 
 struct TcParams {
   int64_t M, N, K;
-  const int64_t* M_dev;      // same-sample dW: M = number of kept columns, read on the device
+  const int64_t* N_dev;      // same-sample dW: N = number of kept columns, read on the device
+  const uint32_t* keep_cols; // same-sample dW: bit d set = column d of the layer input was kept
   int32_t splits;            // K splits (1: epilogue writes final results)
   int32_t num_stages;
   int32_t comp_depth;        // sparse A: depth of the ring of compressed (index + values) buffers
@@ -52,11 +53,14 @@ struct TcParams {
   const float* bias; int32_t act;
   bf16* out_act; int64_t ld_act; float* out_z; int64_t ld_z; bf16* out_zlow; int64_t ld_zlow;
   uint32_t* relubits; int64_t w32;
+  // forward epilogue that also fills the next layer's store (index part already in place)
+  bf16* st_values; const uint32_t* st_keepbits; const uint32_t* st_offsets; int64_t st_capacity; int32_t st_ncb; float st_scale;
   // input-grad epilogue
   const uint32_t* relubits_prev; const bf16* z_prev; int64_t ld_zprev; bf16* out_dx; int64_t ld_dx;
   // dW epilogue
   float* out_dw; int64_t ld_dw; int64_t dw_rows; const uint32_t* row_idx; float* partial; int64_t partial_rows;
   int32_t* dev_status;
+  uint64_t wait_limit_ns;    // every device-side wait of the launch gives up after this long
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------------
@@ -85,7 +89,6 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any legitimate wait here
 
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -195,26 +198,60 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams& p, uint32_t (&r)[
       }
       if (p.out_act != nullptr) {
         uint32_t bits = 0;
+        uint32_t ab[16];                          // the rounded activations, two to a word
         uint4* dst = reinterpret_cast<uint4*>(p.out_act + m * p.ld_act + n);
 #pragma unroll
         for (int j = 0; j < 32; j += 8) {
+#pragma unroll
+          for (int e = 0; e < 8; e += 2) ab[(j + e) >> 1] = 0u;
           if (j < nvalid) {
-            uint32_t pk[4];
 #pragma unroll
             for (int e = 0; e < 8; e += 2) {
               float a0 = v[j + e], a1 = v[j + e + 1];
               if (p.act == RAD_ACT_RELU) { a0 = fmaxf(a0, 0.0f); a1 = fmaxf(a1, 0.0f); }
               else if (p.act == RAD_ACT_GELU) { a0 = gelu_f(a0); a1 = gelu_f(a1); }
               const __nv_bfloat162 h2 = __floats2bfloat162_rn(a0, a1);
-              pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+              ab[(j + e) >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
               // the bit is taken from the rounded activation, the tensor the backward sees
               bits |= (__bfloat162float(h2.x) > 0.0f ? 1u : 0u) << (j + e);
               bits |= (__bfloat162float(h2.y) > 0.0f ? 1u : 0u) << (j + e + 1);
             }
-            dst[j >> 3] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            dst[j >> 3] = make_uint4(ab[j >> 1], ab[(j >> 1) + 1], ab[(j >> 1) + 2], ab[(j >> 1) + 3]);
           }
         }
         if (p.relubits != nullptr) p.relubits[m * p.w32 + (n >> 5)] = bits;
+        if (p.st_values != nullptr) {
+          // This row's 32 activations are one keep-bit word of the next layer's store (Sec. 4.2: the
+          // layer input is what is sampled), whose index part (drawn from the key alone) is in place:
+          // tile offset + row offset + kept entries of the row's earlier words say where they go.
+          const int64_t tile = (m >> 6) * p.st_ncb + (n >> 7);
+          const int rr = (int)(m & 63), wq = (int)((n >> 5) & 3);
+          const uint32_t* tw = p.st_keepbits + tile * kTileWords;
+          const uint4 rowbits = __ldg(reinterpret_cast<const uint4*>(tw + rr * 4));
+          const uint32_t word = wq == 0 ? rowbits.x : wq == 1 ? rowbits.y : wq == 2 ? rowbits.z : rowbits.w;
+          const uint32_t first = __ldg(p.st_offsets + tile);
+          uint64_t pos = (uint64_t)first + __ldg(reinterpret_cast<const unsigned short*>(tw + kBitWords) + rr);
+          if (wq > 0) pos += __popc(rowbits.x);
+          if (wq > 1) pos += __popc(rowbits.y);
+          if (wq > 2) pos += __popc(rowbits.z);
+          const uint64_t cap = (uint64_t)p.st_capacity;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            if ((word >> j) & 1u) {
+              const float a = __uint_as_float((j & 1) ? (ab[j >> 1] & 0xffff0000u) : (ab[j >> 1] << 16));
+              if (pos < cap) p.st_values[pos] = __float2bfloat16_rn(__fmul_rn(a, p.st_scale));
+              ++pos;
+            }
+          }
+          if (rr == 0 && wq == 0) {
+            // zeros between the tile's last value and its padded end
+            const uint4 last = __ldg(reinterpret_cast<const uint4*>(tw + 63 * 4));
+            const uint32_t exact = __ldg(reinterpret_cast<const unsigned short*>(tw + kBitWords) + 63) + __popc(last.x) +
+                                   __popc(last.y) + __popc(last.z) + __popc(last.w);
+            const uint64_t end = min((uint64_t)__ldg(p.st_offsets + tile + 1), cap);
+            for (uint64_t q = (uint64_t)first + exact; q < end; ++q) p.st_values[q] = __float2bfloat16_rn(0.0f);
+          }
+        }
       }
     }
   } else if (EPI == kDx) {
@@ -263,6 +300,29 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams& p, uint32_t (&r)[
         if (j < nvalid)
           d4[j >> 2] = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
                                    __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+    }
+  }
+}
+
+// Same-sample dW, transposed tile: the accumulator row is output column h of dW, the accumulator column is
+// kept column j; r holds dW[idx[n + jj], h] for jj < 32.  For a fixed jj the 32 lanes of a warp write 32
+// consecutive floats of one row of dW (or of the split's partial block, row n + jj).
+__device__ __forceinline__ void epilogue_chunk_dwt(const TcParams& p, const uint32_t (&r)[32], int64_t h, int64_t n,
+                                                   int nvalid, bool row_ok, int32_t split) {
+  if (!row_ok) return;
+  if (p.splits > 1) {
+    float* dst = p.partial + ((int64_t)split * p.partial_rows + n) * p.M + h;
+#pragma unroll
+    for (int jj = 0; jj < 32; ++jj)
+      if (jj < nvalid) dst[(int64_t)jj * p.M] = __uint_as_float(r[jj]);
+  } else {
+#pragma unroll
+    for (int jj = 0; jj < 32; ++jj) {
+      if (jj < nvalid) {
+        const int64_t row = (int64_t)__ldg(p.row_idx + n + jj);
+        if (row < p.dw_rows) p.out_dw[row * p.ld_dw + h] = __uint_as_float(r[jj]);
+        else raise_status(p.dev_status, RAD_DEV_EINTERNAL);
+      }
     }
   }
 }
@@ -387,10 +447,16 @@ __device__ __forceinline__ void cluster_sync_all() {
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t caddr) {
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(caddr) : "memory");
 }
+// What a bounded wait of the pair needs: this CTA's abort flag, the peer's (shared::cluster address) and
+// the time limit of the launch (a kernel argument; rad_set_wait_limit_ns).
+struct PairWait {
+  volatile int* abort_flag;
+  uint32_t peer_abort;
+  uint64_t limit_ns;
+};
 // Bounded wait of the pair: on expiry both CTAs' abort flags are raised.  sleep_ns > 0: a long wait
 // off the critical path (an epilogue warp waiting for a whole tile) leaves the issue slots to others.
-__device__ __forceinline__ bool mbar_wait2(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t peer_abort,
-                                           uint32_t sleep_ns = 0) {
+__device__ __forceinline__ bool mbar_wait2(uint32_t bar, uint32_t parity, const PairWait& wc, uint32_t sleep_ns = 0) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   while (true) {
@@ -399,10 +465,10 @@ __device__ __forceinline__ bool mbar_wait2(uint32_t bar, uint32_t parity, volati
       if (mbar_try_wait(bar, parity)) return true;
       if (sleep_ns != 0) __nanosleep(sleep_ns);
     }
-    if (*abort_flag != 0) return false;
-    if (global_timer_ns() - t0 > kWaitLimitNs) {
-      *abort_flag = 1;
-      asm volatile("st.relaxed.cluster.shared::cluster.u32 [%0], %1;" ::"r"(peer_abort), "r"(1u) : "memory");
+    if (*wc.abort_flag != 0) return false;
+    if (global_timer_ns() - t0 > wc.limit_ns) {
+      *wc.abort_flag = 1;
+      asm volatile("st.relaxed.cluster.shared::cluster.u32 [%0], %1;" ::"r"(wc.peer_abort), "r"(1u) : "memory");
       return false;
     }
   }
@@ -422,10 +488,10 @@ __device__ __forceinline__ void tc_mma_pair(uint32_t tmem_d, uint64_t adesc, uin
       "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
 }
-// D = f32, A = B = bf16, M = 256 over the pair, N = 256.
-__host__ __device__ constexpr uint32_t make_idesc_pair(bool a_mn, bool b_mn) {
+// D = f32, A = B = bf16, M = 256 over the pair, N = n (a multiple of 16, at most 256).
+__host__ __device__ constexpr uint32_t make_idesc_pair(bool a_mn, bool b_mn, uint32_t n = 256u) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
-         ((256u >> 3) << 17) | ((256u >> 4) << 24);
+         ((n >> 3) << 17) | ((256u >> 4) << 24);
 }
 
 template <int AK, int BKIND, int EPI>
@@ -439,13 +505,22 @@ tc_gemm_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, c
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t rank = cluster_ctarank();         // 0: issues the MMAs; both stage operands and run epilogues
   const uint32_t peer_abort = map_to_cta(smem_u32(&ctl->abort_flag), rank ^ 1u);
-  int64_t m_rows = p.M;
-  if (p.M_dev != nullptr) {
-    int64_t md;
-    asm volatile("ld.global.cg.s64 %0, [%1];" : "=l"(md) : "l"(p.M_dev) : "memory");
-    m_rows = md < m_rows ? md : m_rows;
+  const PairWait wc = {abort_flag, peer_abort, p.wait_limit_ns};
+  // Same-sample dW (kDwT): the tile is dW^T, M = H, N = kept columns (known on the device only).  The kept
+  // columns are cut into the fewest tiles of at most 256 and the tile width bn is what one of them needs,
+  // rounded up to the MMA's granule of 16: 105 kept columns cost one tile of 112, not one of 256.
+  int64_t n_cols = p.N;
+  int bn = BN;
+  if (EPI == kDwT) {
+    int64_t nd;
+    asm volatile("ld.global.cg.s64 %0, [%1];" : "=l"(nd) : "l"(p.N_dev) : "memory");
+    n_cols = nd < n_cols ? nd : n_cols;
+    const int64_t nt = max((int64_t)1, (n_cols + BN - 1) / BN);
+    bn = max(16, (int)(((n_cols + nt - 1) / nt + 15) / 16 * 16));
   }
-  const Schedule sched(m_rows, p.N, p.K, p.splits);
+  const Schedule sched(p.M, n_cols, p.K, p.splits, BM, bn);
+  const int boxes_b = (EPI == kDwT) ? (bn / 2 + 63) / 64 : 2;     // 64-column boxes of B this CTA stages per K block
+  const uint32_t stage_tx = 2u * (uint32_t)(kStage2Bytes / 2 + boxes_b * 8192);
   const int64_t pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
   if (tid == 0) {
     for (int s = 0; s < kStages2; ++s) {
@@ -477,16 +552,16 @@ tc_gemm_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, c
     bool ok = true;
     for (int64_t u = pair; u < sched.units && ok; u += npairs) {
       const Unit w = sched.unit(u);
-      const int m_own = (int)w.m0 + 128 * (int)rank, n_own = (int)w.n0 + 128 * (int)rank;
+      const int m_own = (int)w.m0 + 128 * (int)rank, n_own = (int)w.n0 + (bn / 2) * (int)rank;
       for (int kb = w.kb0; kb < w.kb1; ++kb) {
         if (lane == 0) {
-          ok = mbar_wait2(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, peer_abort);
+          ok = mbar_wait2(smem_u32(&ctl->empty[stage]), phase ^ 1u, wc);
           if (ok) {
             const uint32_t sA = smem_base + stage * kStage2Bytes;
             const uint32_t sB = sA + kStage2Bytes / 2;
             const uint32_t full = map_to_cta(smem_u32(&ctl->full[stage]), 0u);
             const int k0 = kb * BK;
-            if (rank == 0) mbar_arrive_expect_tx(smem_u32(&ctl->full[stage]), 2 * kStage2Bytes);   // both CTAs' bytes
+            if (rank == 0) mbar_arrive_expect_tx(smem_u32(&ctl->full[stage]), stage_tx);   // both CTAs' bytes
             if (AK == kAK) {
               tma_load_2d_pair(sA, &tmA, k0, m_own, full);                         // 64 (K) x 128 rows
             } else {
@@ -497,7 +572,8 @@ tc_gemm_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, c
               tma_load_2d_pair(sB, &tmB, k0, n_own, full);
             } else {
 #pragma unroll
-              for (int c = 0; c < 2; ++c) tma_load_2d_pair(sB + c * 8192, &tmB, n_own + c * 64, k0, full);
+              for (int c = 0; c < 2; ++c)
+                if (c < boxes_b) tma_load_2d_pair(sB + c * 8192, &tmB, n_own + c * 64, k0, full);
             }
           }
         }
@@ -509,27 +585,27 @@ tc_gemm_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, c
     // tail: every commit aimed at this CTA's stage barriers has landed before the CTA may leave
     if (lane == 0) {
       for (int i = 0; i < kStages2 && ok; ++i) {
-        ok = mbar_wait2(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, peer_abort);
+        ok = mbar_wait2(smem_u32(&ctl->empty[stage]), phase ^ 1u, wc);
         if (++stage == kStages2) { stage = 0; phase ^= 1u; }
       }
     }
   } else if (warp == 1) {
     // ===== MMA issuer: one thread of the even CTA drives both tensor cores =====
     if (rank == 0) {
-      constexpr uint32_t idesc = make_idesc_pair(AK != kAK, BKIND == kBMN);
+      const uint32_t idesc = make_idesc_pair(AK != kAK, BKIND == kBMN, (uint32_t)bn);
       int stage = 0, buf = 0;
       uint32_t phase = 0, buf_phases = 0;          // bit b: phase of accumulator b
       bool ok = true;
       for (int64_t u = pair; u < sched.units && ok; u += npairs) {
         const Unit w = sched.unit(u);
         if (lane == 0)
-          ok = mbar_wait2(smem_u32(&ctl->tmem_empty[0]) + 8u * buf, ((buf_phases >> buf) & 1u) ^ 1u, abort_flag, peer_abort);
+          ok = mbar_wait2(smem_u32(&ctl->tmem_empty[0]) + 8u * buf, ((buf_phases >> buf) & 1u) ^ 1u, wc);
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         if (!ok) break;
         tc_fence_after();
         for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (lane == 0) {
-            ok = mbar_wait2(smem_u32(&ctl->full[stage]), phase, abort_flag, peer_abort);
+            ok = mbar_wait2(smem_u32(&ctl->full[stage]), phase, wc);
             if (ok) {
               tc_fence_after();
               const uint32_t sA = smem_base + stage * kStage2Bytes;
@@ -555,27 +631,44 @@ tc_gemm_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmA, c
   } else {
     // ===== epilogue: thread = one accumulator row of this CTA, 128 columns per warp =====
     const int q = warp & 3;
-    const int c_first = ((warp - 2) >> 2) * (BN / (kEpiWarps2 / 4));
+    // the two warps of a lane quarter split the tile's 32-column chunks between them
+    const int chunks = (bn + 31) / 32, half_chunks = (chunks + 1) / 2;
+    const int c_first = ((warp - 2) >> 2) * half_chunks * 32;
+    const int c_last = min(c_first + half_chunks * 32, chunks * 32);
     const uint32_t empty_bar = map_to_cta(smem_u32(&ctl->tmem_empty[0]), 0u);     // [b] is 8 bytes further
     int buf = 0;
     uint32_t buf_phases = 0;
     bool ok = true;
+    if (EPI == kDwT && p.keep_cols != nullptr) {
+      // Rows of dW whose column was not kept are zero (Sec. 4.3: only the sampled part of the weight matrix
+      // gets a gradient).  The epilogue warps have nothing to do until the first tile's MMAs retire, so they
+      // write those rows now: row d belongs to CTA d mod grid, a thread writes 16 bytes at a time.
+      const int et = tid - 64;                       // 0 .. 255
+      const int64_t h4 = p.M / 4;
+      for (int64_t d = blockIdx.x; d < p.dw_rows; d += gridDim.x) {
+        if ((__ldg(p.keep_cols + (d >> 5)) >> (d & 31)) & 1u) continue;
+        float4* rowp = reinterpret_cast<float4*>(p.out_dw + d * p.ld_dw);
+        for (int64_t i = et; i < h4; i += 32 * kEpiWarps2) rowp[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
     for (int64_t u = pair; u < sched.units && ok; u += npairs) {
       const Unit w = sched.unit(u);
-      if (lane == 0) ok = mbar_wait2(smem_u32(&ctl->tmem_full[0]) + 8u * buf, (buf_phases >> buf) & 1u, abort_flag, peer_abort, 200u);
+      if (lane == 0) ok = mbar_wait2(smem_u32(&ctl->tmem_full[0]) + 8u * buf, (buf_phases >> buf) & 1u, wc, 200u);
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) break;
       tc_fence_after();
       const int64_t m = w.m0 + 128 * (int64_t)rank + q * 32 + lane;
       const bool row_ok = m < sched.M;
 #pragma unroll 1
-      for (int c0 = c_first; c0 < c_first + BN / (kEpiWarps2 / 4); c0 += 32) {
+      for (int c0 = c_first; c0 < c_last; c0 += 32) {
         const int64_t n = w.n0 + c0;
-        if (n >= p.N) break;                  // warp-uniform
+        if (n >= n_cols) break;               // warp-uniform
         uint32_t r[32];
         tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 256 + c0), r);
         tmem_ld_wait();
-        epilogue_chunk<EPI>(p, r, m, n, row_ok, w.split);
+        // a chunk may reach past the tile's width (bn is a multiple of 16) and past the last kept column
+        if (EPI == kDwT) epilogue_chunk_dwt(p, r, m, n, (int)min((int64_t)min(32, bn - c0), n_cols - n), row_ok, w.split);
+        else epilogue_chunk<(EPI == kDwT ? kDw : EPI)>(p, r, m, n, row_ok, w.split);
       }
       tc_fence_before();
       __syncwarp();
@@ -633,6 +726,7 @@ tc_sparse_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmB)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t rank = cluster_ctarank();
   const uint32_t peer_abort = map_to_cta(smem_u32(&ctl->abort_flag), rank ^ 1u);
+  const PairWait wc = {abort_flag, peer_abort, p.wait_limit_ns};
   const Schedule sched(p.M, p.N, p.K, p.splits, kSpBM, kSpBN);
   const int64_t pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
   if (tid == 0) {
@@ -672,7 +766,7 @@ tc_sparse_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmB)
       const int n_own = (int)w.n0 + 128 * (int)rank;       // + 256 for the second half
       for (int kb = w.kb0; kb < w.kb1; ++kb) {
         if (lane == 0) {
-          ok = mbar_wait2(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, peer_abort);
+          ok = mbar_wait2(smem_u32(&ctl->empty[stage]), phase ^ 1u, wc);
           if (ok) {
             const uint32_t sB = smem_base + stage * kSpStageBytes + kSpAStageBytes;
             if (rank == 0) mbar_arrive_expect_tx(smem_u32(&ctl->full[stage]), 2 * kSpBStageBytes);   // both CTAs' bytes
@@ -689,7 +783,7 @@ tc_sparse_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmB)
     }
     if (lane == 0) {   // every commit aimed at this CTA's stage barriers has landed before the CTA may leave
       for (int i = 0; i < stages && ok; ++i) {
-        ok = mbar_wait2(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, peer_abort);
+        ok = mbar_wait2(smem_u32(&ctl->empty[stage]), phase ^ 1u, wc);
         if (++stage == stages) { stage = 0; phase ^= 1u; }
       }
     }
@@ -702,13 +796,13 @@ tc_sparse_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmB)
       bool ok = true;
       for (int64_t u = pair; u < sched.units && ok; u += npairs) {
         const Unit w = sched.unit(u);
-        if (lane == 0) ok = mbar_wait2(smem_u32(&ctl->tmem_empty), unit_phase ^ 1u, abort_flag, peer_abort);
+        if (lane == 0) ok = mbar_wait2(smem_u32(&ctl->tmem_empty), unit_phase ^ 1u, wc);
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         if (!ok) break;
         tc_fence_after();
         for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (lane == 0) {
-            ok = mbar_wait2(smem_u32(&ctl->full[stage]), phase, abort_flag, peer_abort);
+            ok = mbar_wait2(smem_u32(&ctl->full[stage]), phase, wc);
             if (ok) {
               tc_fence_after();
               const uint32_t sA = smem_base + stage * kSpStageBytes;
@@ -740,7 +834,7 @@ tc_sparse_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmB)
     bool ok = true;
     for (int64_t u = pair; u < sched.units && ok; u += npairs) {
       const Unit w = sched.unit(u);
-      if (lane == 0) ok = mbar_wait2(smem_u32(&ctl->tmem_full), unit_phase, abort_flag, peer_abort, 1000u);
+      if (lane == 0) ok = mbar_wait2(smem_u32(&ctl->tmem_full), unit_phase, wc, 1000u);
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) break;
       tc_fence_after();
@@ -785,7 +879,7 @@ tc_sparse_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmB)
         const uint32_t o0 = __shfl_sync(0xffffffffu, off_lo, src);
         const uint32_t o1 = __shfl_sync(0xffffffffu, off_hi, src);
         if (lane == 0) {
-          ok = mbar_wait2(smem_u32(&ctl->comp_empty[slot]), cphase ^ 1u, abort_flag, peer_abort);
+          ok = mbar_wait2(smem_u32(&ctl->comp_empty[slot]), cphase ^ 1u, wc);
           if (ok) {
             const uint32_t cfull = smem_u32(&ctl->comp_full[slot]);
             const uint32_t sC = smem_u32(comp_base) + slot * comp_slot;
@@ -827,8 +921,8 @@ tc_sparse_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmB)
       const bool have = tile_col_of(w) < p.ncb;
       for (int kb = w.kb0; kb < w.kb1; ++kb, turn ^= 1u) {
         if (turn == group) {
-          ok = mbar_wait2(smem_u32(&ctl->comp_full[slot]), cphase, abort_flag, peer_abort) &&
-               mbar_wait2(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, peer_abort);     // A tile of this stage is free
+          ok = mbar_wait2(smem_u32(&ctl->comp_full[slot]), cphase, wc) &&
+               mbar_wait2(smem_u32(&ctl->empty[stage]), phase ^ 1u, wc);     // A tile of this stage is free
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           // columns past the layer's width keep whatever the buffer held: their accumulator rows are never written
@@ -860,6 +954,26 @@ tc_sparse_pair_kernel(const TcParams p, const __grid_constant__ CUtensorMap tmB)
   }
 }
 
+// The pair kernels' bounded wait on a barrier nobody arrives at, in a cluster of two CTAs that owns no tensor
+// memory and has no loads in flight: both waits run out, both abort flags go up, the pair meets at the
+// cluster barrier as the real kernels do on their way out, and the status word reports the timeout.
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(64, 1) wait_probe_pair_kernel(uint64_t limit_ns, int32_t* dev_status) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  const uint32_t rank = cluster_ctarank();
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  cluster_sync_all();
+  const PairWait wc = {&abort_flag, map_to_cta(smem_u32(&abort_flag), rank ^ 1u), limit_ns};
+  bool ok = true;
+  if (threadIdx.x == 0) ok = mbar_wait2(smem_u32(&bar), 0u, wc, 100u);
+  cluster_sync_all();
+  if (threadIdx.x == 0 && (!ok || abort_flag != 0)) raise_status(dev_status, RAD_DEV_ETIMEOUT);
+}
+
 // Sum of the K-split partial tiles in split order; rows may be scattered (same-sample).
 __global__ void __launch_bounds__(256) dw_reduce_kernel(const float* partial, int64_t partial_rows, int splits,
                                                         int64_t M, const int64_t* M_dev, int64_t N,
@@ -876,12 +990,6 @@ __global__ void __launch_bounds__(256) dw_reduce_kernel(const float* partial, in
     const int64_t row = row_idx != nullptr ? (int64_t)row_idx[m] : m;
     reinterpret_cast<float4*>(out + row * ldw)[c] = acc;
   }
-}
-
-__global__ void __launch_bounds__(256) zero_f32_kernel(float* out, int64_t rows, int64_t cols, int64_t ld) {
-  const int64_t c4 = cols / 4, total = rows * c4;
-  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x)
-    reinterpret_cast<float4*>(out + (i / c4) * ld)[i % c4] = make_float4(0.f, 0.f, 0.f, 0.f);
 }
 
 // ---- host side -------------------------------------------------------------------------------------
@@ -937,8 +1045,8 @@ int num_sms() {
 // float32 partial tiles costs at HBM speed.  Pure function of the shapes, so the workspace query
 // and the launch agree.
 int choose_splits(int64_t m_tiles, int64_t n_tiles, int64_t kblocks, int64_t bm = BM, int64_t sms = kNumSMsDefault,
-                  int64_t bn = BN) {
-  const double kblock_us = 0.55;                                            // 1024 clk at ~1.9 GHz
+                  int64_t bn = BN, double kblock_scale = 1.0) {
+  const double kblock_us = 0.55 * kblock_scale;                             // 1024 clk at ~1.9 GHz for a 256-wide tile
   const double partial_us = (double)(m_tiles * bm) * (double)(n_tiles * bn) * 8.0 / 6.5e6;   // per split
   int best = 1;
   double best_cost = 1e300;
@@ -958,11 +1066,17 @@ DwPlan plan_dw(const rad_store* st, int64_t H) {
   const int64_t kblocks = ceil_div(st->B, BK);
   int64_t m_expect;
   if (st->variant == RAD_SAME_SAMPLE) {
+    // transposed tile: M = H, N = kept columns in tiles of at most 256 (the kernel fits the width to the count)
     m_expect = std::max<int64_t>(1, (int64_t)std::llround((double)st->D * store_keep_fraction(st)));
-    d.partial_rows = round_up(std::min(st->values_ld, round_up(st->D, 8)), BM);
+    d.partial_rows = round_up(std::min(st->values_ld, round_up(st->D, 8)), 16);
     d.comp_cap = 0;
     d.stages = 3;
     d.comp_depth = 0;
+    const int64_t n_tiles = ceil_div(m_expect, BN);
+    const int64_t bn = round_up(ceil_div(m_expect, n_tiles), 16);
+    d.splits = choose_splits(ceil_div(H, BM), n_tiles, kblocks, BM, kNumSMsDefault / 2, bn, (double)bn / BN);
+    d.bytes = d.splits > 1 ? (int64_t)d.splits * d.partial_rows * H * 4 : 0;
+    return d;
   } else {
     m_expect = st->D;
     d.partial_rows = round_up(st->D, BM);
@@ -980,9 +1094,6 @@ DwPlan plan_dw(const rad_store* st, int64_t H) {
     d.bytes = d.splits > 1 ? (int64_t)d.splits * d.partial_rows * H * 4 : 0;
     return d;
   }
-  d.splits = choose_splits(ceil_div(m_expect, BM), ceil_div(H, BN), kblocks, BM, kNumSMsDefault / 2);
-  d.bytes = d.splits > 1 ? (int64_t)d.splits * d.partial_rows * H * 4 : 0;
-  return d;
 }
 
 template <int AK, int BKIND, int EPI>
@@ -1057,6 +1168,12 @@ bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
 
 }  // namespace
 
+int launch_wait_probe_pair(uint64_t limit_ns, int32_t* dev_status, cudaStream_t s) {
+  count_launch();
+  wait_probe_pair_kernel<<<2, 64, 0, s>>>(limit_ns, dev_status);
+  return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
+}
+
 bool tc_shape_ok(int64_t B, int64_t D, int64_t H, const void* p0, int64_t ld0, const void* p1, int64_t ld1) {
   if (B < 64 || D < 64 || H < 64) return false;                    // tiny layers stay on CUDA cores
   if (D % 8 != 0 || H % 8 != 0) return false;
@@ -1067,7 +1184,7 @@ bool tc_shape_ok(int64_t B, int64_t D, int64_t H, const void* p0, int64_t ld0, c
 
 int tc_forward(int act, int64_t B, int64_t D, int64_t H, const void* A, int64_t lda, const void* W, int64_t ldw,
                const float* bias, void* out_act, int64_t ld_act, float* out_z, int64_t ld_z, void* out_zlow,
-               int64_t ld_zlow, uint32_t* relubits, int32_t* dev_status, cudaStream_t s) {
+               int64_t ld_zlow, uint32_t* relubits, int32_t* dev_status, cudaStream_t s, const rad_store* next) {
   CUtensorMap ta, tb;
   int rc = make_map(&ta, A, D, B, lda, 128);          // K-major A: box 64 (K) x 128 rows (one CTA of the pair)
   if (rc != RAD_OK) return rc;
@@ -1079,6 +1196,15 @@ int tc_forward(int act, int64_t B, int64_t D, int64_t H, const void* A, int64_t 
   p.out_act = static_cast<bf16*>(out_act); p.ld_act = ld_act; p.out_z = out_z; p.ld_z = ld_z;
   p.out_zlow = static_cast<bf16*>(out_zlow); p.ld_zlow = ld_zlow; p.relubits = relubits; p.w32 = ceil_div(H, 32);
   p.dev_status = dev_status;
+  p.wait_limit_ns = wait_limit_ns();
+  if (next != nullptr) {
+    // the store of this layer's output (B x H) as the next layer's input; its index part is in place
+    if (out_act == nullptr || next->B != B || next->D != H || next->dtype != RAD_BF16 || !aligned16(next->keepbits))
+      return RAD_EINVAL;
+    p.st_values = static_cast<bf16*>(next->values); p.st_keepbits = next->keepbits; p.st_offsets = next->offsets;
+    p.st_capacity = next->values_capacity; p.st_ncb = (int32_t)ceil_div(H, kTileCols);
+    p.st_scale = (float)kLaneRange / (float)keep_threshold_host(next->p);
+  }
   return launch_pair<kAK, kBMN, kFwd>(p, ta, tb, ceil_div(B, BM) * ceil_div(H, BN), s);
 }
 
@@ -1095,6 +1221,7 @@ int tc_input_grad(int64_t B, int64_t D, int64_t H, const void* dZ, int64_t ldz, 
   p.relubits_prev = relubits_prev; p.z_prev = static_cast<const bf16*>(z_prev); p.ld_zprev = ld_zprev;
   p.out_dx = static_cast<bf16*>(dZ_prev); p.ld_dx = ldp;
   p.dev_status = dev_status;
+  p.wait_limit_ns = wait_limit_ns();
   return launch_pair<kAK, kBK_, kDx>(p, ta, tb, ceil_div(B, BM) * ceil_div(D, BN), s);
 }
 
@@ -1115,15 +1242,17 @@ int tc_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H, 
   p.N = H; p.K = st->B; p.splits = d.splits; p.num_stages = d.stages; p.comp_depth = d.comp_depth;
   p.out_dw = dW; p.ld_dw = ldw; p.dw_rows = st->D; p.partial = static_cast<float*>(workspace); p.partial_rows = d.partial_rows;
   p.dev_status = dev_status;
-  const int grid_z = (int)std::min<int64_t>(ceil_div(st->D * H / 4, 256), 148 * 16);
+  p.wait_limit_ns = wait_limit_ns();
   if (st->variant == RAD_SAME_SAMPLE) {
-    const int64_t mmax = std::min(st->values_ld, round_up(st->D, 8));
-    rc = make_map(&ta, st->values, st->values_ld, st->B, st->values_ld, 64);   // MN-major A: A_c is B x ld
+    // dW[idx, :]^T = dZ^T A_c: A operand dZ (M = h, MN-major), B operand the gathered block A_c (N = kept
+    // column, MN-major), K = minibatch rows; the tile lands transposed and is scattered by kept column
+    const int64_t nmax = std::min(st->values_ld, round_up(st->D, 8));
+    ta = tb;                                           // dZ: box 64 (h) x 64 K rows
+    rc = make_map(&tb, st->values, st->values_ld, st->B, st->values_ld, 64);
     if (rc != RAD_OK) return rc;
-    p.M = mmax; p.M_dev = st->nnz; p.row_idx = st->offsets;
-    count_launch();
-    zero_f32_kernel<<<grid_z, 256, 0, s>>>(dW, st->D, H, ldw);
-    rc = launch_pair<kAMN, kBMN, kDw>(p, ta, tb, ceil_div(mmax, BM) * ceil_div(H, BN) * d.splits, s);
+    p.M = H; p.N = nmax; p.N_dev = st->nnz; p.row_idx = st->offsets; p.keep_cols = st->keepbits;
+    const int64_t n_expect = std::max<int64_t>(1, (int64_t)std::llround((double)st->D * store_keep_fraction(st)));
+    rc = launch_pair<kAMN, kBMN, kDwT>(p, ta, tb, ceil_div(H, BM) * ceil_div(std::min(n_expect, nmax), BN) * d.splits, s);
   } else {
     ta = tb;                                           // unused by the sparse-A kernel
     p.M = st->D;
@@ -1133,10 +1262,11 @@ int tc_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H, 
   }
   if (rc != RAD_OK) return rc;
   if (d.splits > 1) {
-    const int64_t work = p.M * (H / 4);
+    const int64_t rows = st->variant == RAD_SAME_SAMPLE ? p.N : p.M;       // rows of a partial block
+    const int64_t work = rows * (H / 4);
     const int grid = (int)std::max<int64_t>(1, std::min<int64_t>(ceil_div(work, 256), 148 * 16));
     count_launch();
-    dw_reduce_kernel<<<grid, 256, 0, s>>>(p.partial, d.partial_rows, d.splits, p.M, p.M_dev, H, p.row_idx, dW, ldw);
+    dw_reduce_kernel<<<grid, 256, 0, s>>>(p.partial, d.partial_rows, d.splits, rows, p.N_dev, H, p.row_idx, dW, ldw);
   }
   return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
 }

@@ -213,6 +213,42 @@ def test_forward_and_input_grad_sampled_entries(wide):
     assert max(rel_err(to_host_f32(db[hi]), ref_db)) <= 1e-5
 
 
+def test_fused_forward_fills_the_next_store(wide):
+    """The forward GEMM of the wide layer with the next layer's store filled from its epilogue: sampled
+    tiles of that store against the oracle's rule applied to the activations the same call wrote, and the
+    count identities over the whole store."""
+    rad, dev, status = wide["rad"], wide["dev"], wide["status"]
+    act = torch.empty(B, H, dtype=torch.bfloat16, device="cuda")
+    st = rad.Store("different", "bf16", B, H, P, seed=SEED, layer=LAYER + 1, step=STEP, relu_bits=False)
+    st.values.fill_(float("nan"))
+    rad.rad_linear_forward_fill(dev["A"], dev["W"], dev["bias"], "gelu", act, st, dev_status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    check_counts(st, P)
+    nslab, ncb = B // TILE_ROWS, H // TILE_COLS
+    ntiles = nslab * ncb
+    rng = np.random.default_rng(11)
+    offsets = st.offsets.cpu().numpy().view(np.uint32)
+    scale = np.float32(orc.scale_factor(P))
+    for t in [0, ncb - 1, ntiles - 1, ntiles - ncb] + [int(t) for t in rng.integers(0, ntiles, 8)]:
+        slab, blk = divmod(t, ncb)
+        rows = np.arange(slab * TILE_ROWS, (slab + 1) * TILE_ROWS)
+        cols = np.arange(blk * TILE_COLS, (blk + 1) * TILE_COLS)
+        m = orc.keep_mask_at("different", rows, cols, P, SEED, LAYER + 1, STEP)
+        words = st.keepbits[t * TILE_WORDS:(t + 1) * TILE_WORDS].cpu().numpy().view(np.uint32)
+        assert np.array_equal(words[:256], orc.pack_bits(m).reshape(-1)), t
+        n = int(m.sum())
+        padded = -(-n // ALIGN) * ALIGN
+        assert int(offsets[t + 1]) - int(offsets[t]) == padded, t
+        a_tile = to_host_f32(act[slab * TILE_ROWS:(slab + 1) * TILE_ROWS, blk * TILE_COLS:(blk + 1) * TILE_COLS])
+        ref = orc.round_bf16(a_tile[m] * scale)
+        got = st.values[int(offsets[t]):int(offsets[t]) + padded].view(torch.int16).cpu().numpy().view(np.uint16)
+        assert np.array_equal(got[:n], orc.bf16_bits(ref)), t
+        assert (got[n:] == 0).all(), t
+    del st, act
+    torch.cuda.empty_cache()
+
+
 @pytest.mark.parametrize("law", ["replace", "fixed"])
 def test_other_sampling_laws_sampled_tiles_and_counts(wide, law):
     """The with-replacement and the fixed-count law at the size the bench sweep times them: sampled store
