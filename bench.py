@@ -34,6 +34,8 @@ UNIT = "samples/s"
 DIMS = (8192, 8192, 8192, 8192, 8192, 1000)
 BATCH = 65536
 CPU_SLAB_ROWS = 2048         # rows of the workload the CPU oracle is timed on (10-30 s per step on 16 cores)
+CPU_SLAB_ROWS_1CORE = 256    # rows for the single-core run of the same oracle (about the same wall time)
+PHILOX_GCALLS_AT_MAX_CLOCK = 450.0   # Philox-4x32-10 calls per ns, register-only loop on one B200 at 1965 MHz
 
 
 def parse_args():
@@ -50,6 +52,7 @@ def parse_args():
     ap.add_argument("--batch", type=int, default=BATCH)
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-kernel p sweep")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    ap.add_argument("--no-twin", action="store_true", help="skip the timed ReLU twin of the wide net")
     return ap.parse_args()
 
 
@@ -61,27 +64,77 @@ def _oracle_inputs(rows, seed=1234):
     return mlp_inputs(DIMS, rows, "bf16", "normal", seed)
 
 
-def time_oracle(args, steps, warmup):
-    import numpy as np
-    from oracle import rad as orc
+def _blas_threads():
     try:
         from threadpoolctl import threadpool_info
-        cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+        return max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
     except Exception:
-        cores = os.cpu_count() or 1
-    X, y, Ws, bs = _oracle_inputs(CPU_SLAB_ROWS)
+        return os.cpu_count() or 1
+
+
+class _threads:
+    """Limits the BLAS thread pool numpy uses (None: leave it alone)."""
+
+    def __init__(self, n):
+        self.n, self.ctx = n, None
+
+    def __enter__(self):
+        if self.n is not None:
+            from threadpoolctl import threadpool_limits
+            self.ctx = threadpool_limits(limits=self.n)
+            self.ctx.__enter__()
+        return self
+
+    def __exit__(self, *exc):
+        if self.ctx is not None:
+            self.ctx.__exit__(*exc)
+
+
+def time_oracle(args, steps, warmup, rows=CPU_SLAB_ROWS, threads=None):
+    import numpy as np
+    from oracle import rad as orc
+    X, y, Ws, bs = _oracle_inputs(rows)
     times = []
-    for i in range(warmup + steps):
-        t0 = time.perf_counter()
-        r = orc.mlp_step(X, y, Ws, bs, act=args.act, dtype="bf16", variant=args.variant, p=args.p, seed=0, step=i, law=args.law)
-        dt = time.perf_counter() - t0
-        if i >= warmup:
-            times.append(dt)
-        assert np.isfinite(r.loss)
+    with _threads(threads):
+        cores = _blas_threads() if threads is None else threads
+        for i in range(warmup + steps):
+            t0 = time.perf_counter()
+            r = orc.mlp_step(X, y, Ws, bs, act=args.act, dtype="bf16", variant=args.variant, p=args.p, seed=0, step=i, law=args.law)
+            dt = time.perf_counter() - t0
+            if i >= warmup:
+                times.append(dt)
+            assert np.isfinite(r.loss)
     mean = sum(times) / len(times)
-    return dict(value=CPU_SLAB_ROWS / mean, unit=UNIT, cores=int(cores), kind="oracle",
-                sample=f"row slab of {CPU_SLAB_ROWS} rows of the same net (full D and H), "
+    return dict(value=rows / mean, unit=UNIT, cores=int(cores), kind="oracle",
+                sample=f"row slab of {rows} rows of the same net (full D and H), "
                        f"{len(times)} step(s) of {mean:.2f} s"), mean
+
+
+def time_small_oracles():
+    """The oracle on the three small workloads at full size, all cores and one core (seconds per step)."""
+    from oracle import rad as orc, irnn as oirnn, cnn as ocnn
+    from workloads import cnn_inputs, irnn_inputs, mlp_inputs
+    jobs = {}
+    X, y, Ws, bs = mlp_inputs((784, 300, 300, 10), 150, "f32", "uniform01", 1234)
+    jobs["mlp_784_300_300_10_b150_f32_different"] = (150, lambda: orc.mlp_step(X, y, Ws, bs, dtype="f32", variant="different", p=0.1, seed=0))
+    jobs["mlp_784_300_300_10_b150_f32_same"] = (150, lambda: orc.mlp_step(X, y, Ws, bs, dtype="f32", variant="same", p=0.1, seed=0))
+    ia = irnn_inputs(150, 784, 100, 10, 1234, True)
+    jobs["irnn_h100_t784_b150_f32_different"] = (150, lambda: oirnn.irnn_step(*ia, variant="different", p=0.1, seed=0, step0=0))
+    ca = cnn_inputs(128, 32, 3, (16, 32, 64), (128, 10), "bf16", 1234)
+    jobs["cnn_32x32x3_c16_32_64_fc128_10_b128_bf16_different"] = (128, lambda: ocnn.cnn_step(*ca, dtype="bf16", variant="different", p=0.1, seed=0, step=0))
+    out = {}
+    for name, (batch, fn) in jobs.items():
+        row = {}
+        for label, threads in (("all_cores", None), ("one_core", 1)):
+            with _threads(threads):
+                fn()
+                t0 = time.perf_counter()
+                fn()
+                dt = time.perf_counter() - t0
+                row[label] = dict(samples_per_s=round(batch / dt, 1), s_per_step=round(dt, 4),
+                                  cores=int(_blas_threads() if threads is None else threads))
+        out[name] = row
+    return out
 
 
 def run_reference(args):
@@ -93,7 +146,8 @@ def run_reference(args):
     line = dict(impl="reference", metric=METRIC, value=base["value"], unit=UNIT, n_gpus=args.gpus, steps=steps,
                 warmup=warmup, ms_per_step=mean * 1e3, higher_is_better=True, scaling="weak", vs_baseline=None,
                 dtype="f64", data="synthetic",
-                config=dict(workload="mlp_wide 8192x4->1000 bf16 grid, oracle on a row slab", dims=list(DIMS),
+                config=dict(workload=f"mlp_wide: 8192->8192x4->1000 on the bf16 grid, batch {args.batch}; the oracle is "
+                                     f"timed on a slab of {CPU_SLAB_ROWS} rows", dims=list(DIMS),
                             batch=CPU_SLAB_ROWS, variant=args.variant, law=args.law, p=args.p, act=args.act),
                 cpu_baseline=base,
                 e2e=dict(value=base["value"], unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
@@ -161,6 +215,27 @@ class ClockSampler:
             return dict(sm_mhz=None, sm_max_mhz=None, reasons=["no samples"])
         return dict(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), power_w_max=max(power), samples=len(sm),
                     reasons=sorted(reasons))
+
+
+class NvmlClock:
+    """Current SM clock read through NVML (a read only; nothing is set)."""
+
+    def __init__(self, index):
+        self.h = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv, self.h = pynvml, pynvml.nvmlDeviceGetHandleByIndex(index)
+        except Exception:
+            self.h = None
+
+    def mhz(self):
+        if self.h is None:
+            return None
+        try:
+            return int(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+        except Exception:
+            return None
 
 
 class LayerwiseStep:
@@ -252,75 +327,132 @@ def peaks():
         with open(path) as f:
             d = json.load(f)
         return dict(hbm_gbs=d["hbm_gbs"], tflops_burst=d["bf16_tflops"], tflops_sustained=d["bf16_tflops_sustained"],
-                    source="measured")
-    return dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, source="fallback")
+                    sm_max_mhz=d.get("sm_max_mhz", 1965.0), source="measured")
+    return dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, sm_max_mhz=1965.0, source="fallback")
 
 
-def kernel_sweep(rad, torch, A, dZ, H, ps):
-    """Store GB/s and dW TFLOP/s of one 8192 x 8192 layer for both variants over the p sweep."""
+def timed_alone(torch, fn, clock, n=10, settle_ms=60.0):
+    """Median device time of `fn` timed alone (CUDA events on the launching stream) and the median SM clock
+    read while the timed launches run.  `fn` first runs for about settle_ms so that the clock is the one
+    this kernel sustains by itself, not what the kernels before it left behind."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    fn()
+    torch.cuda.synchronize()
+    e0.record(); fn(); e1.record()
+    torch.cuda.synchronize()
+    once = max(e0.elapsed_time(e1), 1e-3)
+    for _ in range(max(2, min(400, int(settle_ms / once)))):
+        fn()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
+    ev[0].record()
+    for i in range(n):
+        fn()
+        ev[i + 1].record()
+    mhz = []
+    while not ev[n].query():
+        m = clock.mhz()
+        if m is not None:
+            mhz.append(m)
+        time.sleep(0.0005)
+    torch.cuda.synchronize()
+    ms = statistics.median(ev[i].elapsed_time(ev[i + 1]) for i in range(n))
+    return ms, (statistics.median(mhz) if mhz else None)
+
+
+def store_bytes_different(B, D, nnz_padded, n_offsets, extra=0):
+    """Algorithmic bytes of a different-sample store: the input read once, kept values (padded per tile),
+    one keep bit per entry plus the row offsets that travel with them, one offset per tile."""
+    ntiles = n_offsets - 1
+    return B * D * 2 + nnz_padded * 2 + ntiles * 288 * 4 + 4 * n_offsets + extra
+
+
+def kernel_sweep(rad, torch, A, dZ, H, ps, pk, clock):
+    """Store and dW of one 8192 x 8192 layer, each kernel timed alone, for both variants over the p sweep."""
+    import numpy as np
     B, D = A.shape
     rows = []
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     dW = torch.empty(D, H, dtype=torch.float32, device="cuda")
+    hbm, burst = pk["hbm_gbs"], pk["tflops_burst"]
 
-    def timed(fn, n=5):
-        fn(); fn()
-        torch.cuda.synchronize()
-        ev = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
-        ev[0].record()
-        for i in range(n):
-            fn()
-            ev[i + 1].record()
-        torch.cuda.synchronize()
-        return statistics.median(ev[i].elapsed_time(ev[i + 1]) for i in range(n))
+    def frac(v, peak):
+        return round(v / peak, 4)
 
+    # every store first (they leave the clock alone), then the weight gradients, whose power draw pulls it down
+    stores = {}
     for variant in ("different", "same"):
         for p in ps:
             st = rad.Store(variant, "bf16", B, D, p, relu_bits=False)
-            ms_store = timed(lambda: rad.rad_linear_forward_store(A, st, status))
+            ms_store, mhz = timed_alone(torch, lambda: rad.rad_linear_forward_store(A, st, status), clock, n=20, settle_ms=150.0)
+            idx_t = None
+            if variant == "different":
+                idx_t = timed_alone(torch, lambda: rad.rad_store_index(st, status), clock, n=20, settle_ms=100.0)
+            stores[(variant, p)] = (st, ms_store, mhz, idx_t)
+    for variant in ("different", "same"):
+        for p in ps:
+            st, ms_store, mhz, idx_t = stores.pop((variant, p))
             nnz = st.nnz.cpu().numpy()
             ws = torch.empty(max(rad.rad_weight_grad_workspace(st, H), 256), dtype=torch.uint8, device="cuda")
-            ms_dw = timed(lambda: rad.rad_linear_weight_grad(st, dZ, dW, ws, status), n=3)
+            ms_dw, mhz_dw = timed_alone(torch, lambda: rad.rad_linear_weight_grad(st, dZ, dW, ws, status), clock, n=5,
+                                        settle_ms=30.0)
+            row = dict(variant=variant, p=p, p_eff=rad.rad_effective_p(p), nnz=int(nnz[0]), store_ms=round(ms_store, 4),
+                       store_sm_mhz=mhz, store_ms_x_mhz=None if mhz is None else round(ms_store * mhz, 1),
+                       dW_ms=round(ms_dw, 4), dW_sm_mhz=mhz_dw)
             if variant == "different":
-                store_bytes = B * D * 2 + int(nnz[1]) * 2 + B * D // 8 + 4 * (len(st.offsets))
-                flops, kind = 2.0 * B * D * H, "dense-tile"
+                sb = store_bytes_different(B, D, int(nnz[1]), len(st.offsets))
+                row.update(store_bytes=sb, store_gbs=round(sb / ms_store / 1e6, 1), store_frac_hbm=frac(sb / ms_store / 1e6, hbm))
+                ms_idx, mhz_idx = idx_t
+                calls = 3.0 * B * D / 32
+                row.update(index_ms=round(ms_idx, 4), index_sm_mhz=mhz_idx, index_philox_gcalls_s=round(calls / ms_idx / 1e6, 1))
+                dense = 2.0 * B * D * H
+                row.update(dW_tflops_dense_tile=round(dense / ms_dw / 1e9, 1), dW_frac_burst=frac(dense / ms_dw / 1e9, burst),
+                           dW_useful_tflops=round(2.0 * int(nnz[0]) * H / ms_dw / 1e9, 1))
             else:
-                store_bytes = B * D * 2 + int(nnz[1]) * 2 + 4 * int(nnz[0])
-                flops, kind = 2.0 * B * int(nnz[0]) * H, "kept-columns"
-            rows.append(dict(variant=variant, p=p, store_ms=round(ms_store, 4),
-                             store_gbs=round(store_bytes / ms_store / 1e6, 1),
-                             dW_ms=round(ms_dw, 4), dW_tflops=round(flops / ms_dw / 1e9, 1), dW_flops=kind,
-                             nnz=int(nnz[0])))
+                k = int(nnz[0])
+                idx = st.offsets[:k].cpu().numpy().view(np.uint32)
+                sectors = int(np.unique(idx // 16).size)          # 32-byte sectors of a row that hold a kept column
+                touched = B * sectors * 32 + B * int(st.c.values_ld) * 2 + 4 * k
+                full = B * D * 2 + B * k * 2 + 4 * k
+                row.update(store_bytes_touched=touched, store_gbs=round(touched / ms_store / 1e6, 1),
+                           store_frac_hbm=frac(touched / ms_store / 1e6, hbm),
+                           store_gbs_if_all_of_A_were_read=round(full / ms_store / 1e6, 1))
+                flops = 2.0 * B * k * H
+                # what this contraction has to move whatever p is: dZ once, the gathered block, dW written once
+                dw_bytes = B * H * 2 + B * int(st.c.values_ld) * 2 + D * H * 4
+                row.update(dW_tflops_kept_columns=round(flops / ms_dw / 1e9, 1), dW_frac_burst=frac(flops / ms_dw / 1e9, burst),
+                           dW_bytes=dw_bytes, dW_gbs=round(dw_bytes / ms_dw / 1e6, 1), dW_frac_hbm=frac(dw_bytes / ms_dw / 1e6, hbm),
+                           dW_bound="hbm" if dw_bytes / hbm / 1e6 > flops / burst / 1e9 else "tensor")
+            rows.append(row)
             del st, ws
     # the paper's own law (k = ceil(fraction D) draws with replacement) and the fixed-count law without
     # replacement: multiplicity kernel + store, then the same weight-gradient kernels on the store it leaves
     for law, variant in (("replace", "different"), ("replace", "same"), ("fixed", "different"), ("fixed", "same")):
         p = 0.1
         st = rad.Store(variant, "bf16", B, D, p, relu_bits=False, law=law)
-        ms_store = timed(lambda: rad.rad_linear_forward_store(A, st, status))
+        ms_store, mhz = timed_alone(torch, lambda: rad.rad_linear_forward_store(A, st, status), clock, n=10)
         nnz = st.nnz.cpu().numpy()
         ws = torch.empty(max(rad.rad_weight_grad_workspace(st, H), 256), dtype=torch.uint8, device="cuda")
-        ms_dw = timed(lambda: rad.rad_linear_weight_grad(st, dZ, dW, ws, status), n=3)
+        ms_dw, _ = timed_alone(torch, lambda: rad.rad_linear_weight_grad(st, dZ, dW, ws, status), clock, n=3, settle_ms=20.0)
+        row = dict(variant=variant, law=law, p=p, draws_per_row=rad.rad_draws_per_row(p, D), nnz=int(nnz[0]),
+                   store_ms=round(ms_store, 4), store_sm_mhz=mhz, dW_ms=round(ms_dw, 4))
         if variant == "different":
             # the multiplicity matrix (a byte per entry) is written and read once on top of the store's bytes
-            store_bytes = B * D * 2 + int(nnz[1]) * 2 + B * D // 8 + 4 * len(st.offsets) + 2 * B * D
-            flops, kind = 2.0 * B * D * H, "dense-tile"
+            sb = store_bytes_different(B, D, int(nnz[1]), len(st.offsets), extra=2 * B * D)
+            row.update(store_bytes=sb, store_gbs=round(sb / ms_store / 1e6, 1), store_frac_hbm=frac(sb / ms_store / 1e6, hbm),
+                       dW_tflops_dense_tile=round(2.0 * B * D * H / ms_dw / 1e9, 1),
+                       dW_useful_tflops=round(2.0 * int(nnz[0]) * H / ms_dw / 1e9, 1))
         else:
-            store_bytes = B * D * 2 + int(nnz[1]) * 2 + 4 * int(nnz[0])
-            flops, kind = 2.0 * B * int(nnz[0]) * H, "kept-columns"
-        rows.append(dict(variant=variant, law=law, p=p, draws_per_row=rad.rad_draws_per_row(p, D),
-                         store_ms=round(ms_store, 4), store_gbs=round(store_bytes / ms_store / 1e6, 1),
-                         dW_ms=round(ms_dw, 4), dW_tflops=round(flops / ms_dw / 1e9, 1), dW_flops=kind,
-                         nnz=int(nnz[0])))
+            row.update(dW_tflops_kept_columns=round(2.0 * B * int(nnz[0]) * H / ms_dw / 1e9, 1))
+        rows.append(row)
         del st, ws
     # random projection (P = R R^T, Rademacher signs, k = ceil(0.1 D) columns): the store is one dense GEMM,
     # the weight gradient two; TFLOP/s on the flops of those contractions (2 B D k; 2 B k H + 2 D k H)
     p = 0.1
     st = rad.Store("project", "bf16", B, D, p, relu_bits=False)
     k = rad.rad_draws_per_row(p, D)
-    ms_store = timed(lambda: rad.rad_linear_forward_store(A, st, status))
+    ms_store, _ = timed_alone(torch, lambda: rad.rad_linear_forward_store(A, st, status), clock, n=5, settle_ms=20.0)
     ws = torch.empty(max(rad.rad_weight_grad_workspace(st, H), 256), dtype=torch.uint8, device="cuda")
-    ms_dw = timed(lambda: rad.rad_linear_weight_grad(st, dZ, dW, ws, status), n=3)
+    ms_dw, _ = timed_alone(torch, lambda: rad.rad_linear_weight_grad(st, dZ, dW, ws, status), clock, n=3, settle_ms=20.0)
     rows.append(dict(variant="project", p=p, k=k, store_ms=round(ms_store, 4),
                      store_tflops=round(2.0 * B * D * k / ms_store / 1e9, 1), dW_ms=round(ms_dw, 4),
                      dW_tflops=round((2.0 * B * k * H + 2.0 * D * k * H) / ms_dw / 1e9, 1), dW_flops="projected",
@@ -331,15 +463,16 @@ def kernel_sweep(rad, torch, A, dZ, H, ps):
 
 
 def small_workloads(rad, torch):
-    """Samples/s of the two small float32 workloads (launch-latency bound; no roofline claim)."""
+    """Samples/s of the small workloads (launch-latency bound; no roofline claim) with the launches per step."""
     import numpy as np
-    from workloads import irnn_inputs, mlp_inputs
+    from workloads import cnn_inputs, irnn_inputs, mlp_inputs
     out = {}
 
     def rate(fn, batch, reps):
         for _ in range(3):
             fn()
         torch.cuda.synchronize()
+        l0 = rad.rad_launch_count()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for i in range(reps):
@@ -347,7 +480,13 @@ def small_workloads(rad, torch):
         e1.record()
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / reps
-        return dict(samples_per_s=round(batch / ms * 1e3, 1), ms_per_step=round(ms, 4))
+        return dict(samples_per_s=round(batch / ms * 1e3, 1), ms_per_step=round(ms, 4),
+                    gpu_launches=int((rad.rad_launch_count() - l0) // reps))
+
+    def memory(ctx, r):
+        st = ctx.stats
+        r["reserved_bytes"] = st.value_bytes + st.index_bytes + st.relu_bytes + st.unsampled_bytes
+        r["full_backprop_bytes"] = st.full_backprop_bytes
 
     X, y, Ws, bs = mlp_inputs((784, 300, 300, 10), 150, "f32", "uniform01", 1234)
     dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
@@ -355,31 +494,38 @@ def small_workloads(rad, torch):
     for variant in ("different", "same"):
         ctx = rad.MLPStep((784, 300, 300, 10), 150, "f32", "relu", variant, 0.1)
         r = rate(lambda i=0: ctx(Xd, yd, Wd, bd, seed=0, step=i), 150, 50)
-        st = ctx.stats
-        r["held_bytes"] = st.value_bytes + st.index_bytes + st.relu_bytes + st.unsampled_bytes
-        r["full_backprop_bytes"] = st.full_backprop_bytes
+        memory(ctx, r)
+        held = rad.rad_mlp_held_bytes(ctx, ctx.nnz.cpu().tolist())
+        r["held_bytes"] = held.value_bytes + held.index_bytes + held.relu_bytes + held.unsampled_bytes
         assert ctx.dev_status.item() == 0
         out["mlp_784_300_300_10_b150_f32_" + variant] = r
     args = [dev(a) for a in irnn_inputs(150, 784, 100, 10, 1234, True)]
     ctx = rad.IRNNStep(150, 784, 100, 10, "different", 0.1)
     r = rate(lambda i=0: ctx(*args, seed=0, step0=784 * i), 150, 20)
-    st = ctx.stats
-    r["held_bytes"] = st.value_bytes + st.index_bytes + st.relu_bytes + st.unsampled_bytes
-    r["full_backprop_bytes"] = st.full_backprop_bytes
+    memory(ctx, r)
     assert ctx.dev_status.item() == 0
     out["irnn_h100_t784_b150_f32_different"] = r
-    from workloads import cnn_inputs
     X, y, cW, cb, fW, fb = cnn_inputs(128, 32, 3, (16, 32, 64), (128, 10), "bf16", 1234)
     bf = lambda a: dev(a).to(torch.bfloat16)
     cargs = (bf(X), dev(y), [bf(w) for w in cW], [dev(b) for b in cb], [bf(w) for w in fW], [dev(b) for b in fb])
     ctx = rad.CNNStep(128, 32, 3, (16, 32, 64), (128, 10), "bf16", "different", 0.1)
     r = rate(lambda i=0: ctx(*cargs, seed=0, step=i), 128, 20)
-    st = ctx.stats
-    r["held_bytes"] = st.value_bytes + st.index_bytes + st.relu_bytes + st.unsampled_bytes
-    r["full_backprop_bytes"] = st.full_backprop_bytes
+    memory(ctx, r)
     assert ctx.dev_status.item() == 0
     out["cnn_32x32x3_c16_32_64_fc128_10_b128_bf16_different"] = r
     return out
+
+
+def memory_report(rad, dims, B, act, variant, p, law, nnz_host):
+    """Bytes held between the passes: as kept by the step that left `nnz_host`, and as reserved beforehand."""
+    _, reserved = rad.rad_mlp_workspace(dims, B, "bf16", act, variant, p, law)
+    held = rad.rad_mlp_held_bytes((dims, B, "bf16", act, variant, p, law), nnz_host)
+    total = held.value_bytes + held.index_bytes + held.relu_bytes + held.preact_bytes + held.unsampled_bytes
+    return dict(value_bytes=held.value_bytes, value_bytes_reserved=reserved.value_bytes, index_bytes=held.index_bytes,
+                relu_bytes=held.relu_bytes, preact_bytes=held.preact_bytes, unsampled_bytes=held.unsampled_bytes,
+                held_bytes=total, held_bytes_if_the_mask_is_redrawn_from_the_key=total - held.index_bytes,
+                full_backprop_bytes=held.full_backprop_bytes, ratio=round(held.full_backprop_bytes / total, 3),
+                ratio_if_the_mask_is_redrawn=round(held.full_backprop_bytes / (total - held.index_bytes), 3))
 
 
 def run_ours(args):
@@ -406,114 +552,119 @@ def run_ours(args):
     Ws = [(torch.randn(dims[l], dims[l + 1], generator=wgen, device="cuda") * (2.0 / dims[l]) ** 0.5).to(bf)
           for l in range(L)]
     bs = [torch.zeros(dims[l + 1], device="cuda") for l in range(L)]
-
-    lw = LayerwiseStep(rad, torch, dims, B, args.act, args.variant, args.p, args.law)
+    pk = peaks()
+    clock = NvmlClock(local)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(args.warmup):
-        lw(X, labels, Ws, bs, seed=0, step=i, record=False)
-    barrier()
-    sampler = ClockSampler(local)
-    sampler.start()
-    launches0 = rad.rad_launch_count()
-    t_start, t_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t_start.record()
-    for i in range(args.steps):
-        lw(X, labels, Ws, bs, seed=0, step=args.warmup + i, record=True)
-    t_stop.record()
-    barrier()
-    launches = (rad.rad_launch_count() - launches0) // max(args.steps, 1)
-    clocks = sampler.stop()
-    ms_total = t_start.elapsed_time(t_stop)
-    ms_total = max_over_ranks(ms_total, "cuda")
-    assert lw.status.item() == 0, f"device status {lw.status.item()}"
+    def timed_steps(lw, warmup, steps, first_step=0):
+        for i in range(warmup):
+            lw(X, labels, Ws, bs, seed=0, step=first_step + i, record=False)
+        barrier()
+        sampler = ClockSampler(local)
+        sampler.start()
+        launches0 = rad.rad_launch_count()
+        t_start, t_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t_start.record()
+        for i in range(steps):
+            lw(X, labels, Ws, bs, seed=0, step=first_step + warmup + i, record=True)
+        t_stop.record()
+        barrier()
+        launches = (rad.rad_launch_count() - launches0) // max(steps, 1)
+        clocks = sampler.stop()
+        ms_total = max_over_ranks(t_start.elapsed_time(t_stop), "cuda")
+        assert lw.status.item() == 0, f"device status {lw.status.item()}"
+        return ms_total, launches, clocks
+
+    lw = LayerwiseStep(rad, torch, dims, B, args.act, args.variant, args.p, args.law)
+    ms_total, launches, clocks = timed_steps(lw, args.warmup, args.steps)
     ms_step = ms_total / args.steps
     value = whole_job_value(world, B, args.steps, ms_total)
 
-    # per-family device time inside the timed region, and the roofline of the dominant kernel
+    # per-family and per-kernel device time inside the timed region
     fam = lw.family_ms()
     by_family = {}
     for (f, l), v in fam.items():
         by_family.setdefault(f, 0.0)
         by_family[f] += sum(v) / args.steps
-    pk = peaks()
-    dw_big = [(l, sum(v) / len(v)) for (f, l), v in fam.items() if f == "dW" and dims[l] == 8192 and dims[l + 1] == 8192]
-    fwd_big = [(l, sum(v) / len(v)) for (f, l), v in fam.items() if f == "forward" and dims[l + 1] == 8192]
-    dominant = max(by_family, key=by_family.get)
-    if dominant == "dW":
-        ms_k = sum(t for _, t in dw_big) / len(dw_big)
-        if args.variant == "different":
-            flops, what = 2.0 * B * 8192 * 8192, "tc_sparse_pair_kernel (different-sample dW), dense-tile flops 2*B*D*H"
-        elif args.variant == "project":
-            k = int(lw.stores[1].nnz[0].item())
-            flops, what = 2.0 * B * k * 8192 + 2.0 * 8192 * k * 8192, "projection dW: S^T dZ and R' G, flops 2*B*k*H + 2*D*k*H"
-        else:
-            k = int(lw.stores[1].nnz[0].item())
-            flops, what = 2.0 * B * k * 8192, "tc_gemm_pair_kernel<MN,MN> (same-sample dW), flops 2*B*k'*H on kept columns"
-    else:
-        ms_k = sum(t for _, t in fwd_big) / len(fwd_big)
-        flops, what = 2.0 * B * 8192 * 8192, "tc_gemm_pair_kernel forward, flops 2*B*D*H"
-    achieved = flops / ms_k / 1e9
-    # DRAM bytes per launch from the ncu captures under profiles/ (batch 8192, 8192 x 8192 layer): bytes
-    # read grow with the batch and are scaled by B / 8192, the dW output does not grow.  Only the
-    # default workload has a capture.
-    traffic = None
-    if args.act == "gelu" and abs(args.p - 0.1) < 1e-9 and args.law == "bernoulli":
-        if dominant == "dW" and args.variant == "different":
-            traffic = int(351.5e6 * B / 8192 + 228.4e6)
-        elif dominant != "dW":
-            traffic = int((1095.8e6 + 251.4e6) * B / 8192)
-    roofline = dict(bound="tensor", kernel=what, achieved=round(achieved, 1), peak=pk["tflops_sustained"],
-                    unit="TFLOP/s", frac=round(achieved / pk["tflops_sustained"], 4), traffic=traffic,
-                    peak_source=pk["source"] + " (sustained cuBLAS bf16)", ms_per_launch=round(ms_k, 4),
-                    how="CUDA events around the call on the launching stream, inside the timed steps")
-    store_big = [sum(v) / len(v) for (f, l), v in fam.items() if f == "store" and dims[l] == 8192]
+
+    def mean_ms(family, pick):
+        t = [sum(v) / len(v) for (f, l), v in fam.items() if f == family and pick(l)]
+        return sum(t) / len(t) if t else None
+
+    big = lambda l: dims[l] == 8192 and dims[l + 1] == 8192
+    fused = args.variant == "different" and args.law == "bernoulli"
+    ms_fwd, ms_dw, ms_dx = mean_ms("forward", big), mean_ms("dW", big), mean_ms("dX+db", lambda l: big(l) and l > 0)
+    ms_store0 = mean_ms("store", lambda l: l == 0)
+    ms_store_hidden = mean_ms("store", lambda l: l > 0)      # fused: the key-only index kernels; else full stores
+    nnz0 = lw.stores[0].nnz.cpu().numpy()
     nnz1 = lw.stores[1].nnz.cpu().numpy()
+    dense = 2.0 * B * 8192 * 8192
+    sust, burst, hbm = pk["tflops_sustained"], pk["tflops_burst"], pk["hbm_gbs"]
+
+    def tensor_entry(what, ms, flops, extra=None):
+        d = dict(kernel=what, bound="tensor", ms_per_launch=round(ms, 4), achieved=round(flops / ms / 1e9, 1), unit="TFLOP/s",
+                 peak=sust, frac=round(flops / ms / 1e9 / sust, 4), peak_kind="sustained (kernel timed inside the step)")
+        if extra:
+            d.update(extra)
+        return d
+
+    kernels = {}
+    kernels["forward"] = tensor_entry("tc_gemm_pair_kernel forward" + (" + next layer's store from the epilogue" if fused else ""),
+                                      ms_fwd, dense)
+    kernels["dX"] = tensor_entry("tc_gemm_pair_kernel input gradient (+ column sums for db)", ms_dx, dense)
     if args.variant == "different":
-        sbytes = B * 8192 * 2 + int(nnz1[1]) * 2 + B * 8192 // 8 + 4 * len(lw.stores[1].offsets)
-        if args.law != "bernoulli":
-            sbytes += 2 * B * 8192                     # the multiplicity matrix, written and read once
+        kernels["dW"] = tensor_entry("tc_sparse_pair_kernel, dense-tile flops 2*B*D*H", ms_dw, dense,
+                                     dict(useful_tflops=round(2.0 * int(nnz1[0]) * 8192 / ms_dw / 1e9, 1)))
+        sb = store_bytes_different(B, 8192, int(nnz0[1]), len(lw.stores[0].offsets),
+                                   extra=2 * B * 8192 if args.law != "bernoulli" else 0)
+        kernels["store"] = dict(kernel="store of the network input (stand-alone kernel)", bound="hbm", ms_per_launch=round(ms_store0, 4),
+                                achieved=round(sb / ms_store0 / 1e6, 1), unit="GB/s", peak=hbm, frac=round(sb / ms_store0 / 1e6 / hbm, 4),
+                                algorithmic_bytes=sb)
+        if fused:
+            calls = 3.0 * B * 8192 / 32
+            mhz = clocks.get("sm_mhz") or pk["sm_max_mhz"]
+            peak_calls = PHILOX_GCALLS_AT_MAX_CLOCK * mhz / pk["sm_max_mhz"]
+            kernels["store_index"] = dict(kernel="store_index_kernel + offsets_scan_kernel (hidden layers: index from the key, "
+                                                 "values from the producing GEMM's epilogue)", bound="alu",
+                                          ms_per_launch=round(ms_store_hidden, 4), achieved=round(calls / ms_store_hidden / 1e6, 1),
+                                          unit="Philox Gcalls/s", peak=round(peak_calls, 1),
+                                          frac=round(calls / ms_store_hidden / 1e6 / peak_calls, 4),
+                                          peak_kind="register-only Philox loop, 450 Gcalls/s at 1965 MHz, scaled to the step's clock")
+    elif args.variant == "same":
+        k = int(nnz1[0])
+        kernels["dW"] = tensor_entry("tc_gemm_pair_kernel same-sample dW (dW^T tile, kept columns on N), flops 2*B*k'*H", ms_dw,
+                                     2.0 * B * k * 8192, dict(kept_columns=k))
+        idx = lw.stores[0].offsets[:int(nnz0[0])].cpu().numpy()
+        import numpy as np
+        sectors = int(np.unique(idx.view(np.uint32) // 16).size)
+        touched = B * sectors * 32 + B * int(lw.stores[0].c.values_ld) * 2
+        kernels["store"] = dict(kernel="same-sample gather (bytes of the sectors it touches + the block written)", bound="hbm",
+                                ms_per_launch=round(ms_store0, 4), achieved=round(touched / ms_store0 / 1e6, 1), unit="GB/s",
+                                peak=hbm, frac=round(touched / ms_store0 / 1e6 / hbm, 4), algorithmic_bytes=touched)
     else:
-        sbytes = B * 8192 * 2 + int(nnz1[1]) * 2 + 4 * int(nnz1[0])
-    ms_s = sum(store_big) / len(store_big)
-    if args.variant == "project":
-        # the store of this variant is a dense contraction (S = A R'), not a streaming kernel
-        sflops = 2.0 * B * 8192 * int(nnz1[0])
-        store_roofline = dict(bound="tensor", kernel="projection store S = A R', flops 2*B*D*k",
-                              achieved=round(sflops / ms_s / 1e9, 1), peak=pk["tflops_sustained"], unit="TFLOP/s",
-                              frac=round(sflops / ms_s / 1e9 / pk["tflops_sustained"], 4), traffic=None,
-                              ms_per_launch=round(ms_s, 4))
-    else:
-        store_roofline = dict(bound="hbm", kernel="store kernel, one 8192-wide layer input",
-                              achieved=round(sbytes / ms_s / 1e6, 1), peak=pk["hbm_gbs"], unit="GB/s",
-                              frac=round(sbytes / ms_s / 1e6 / pk["hbm_gbs"], 4),
-                              traffic=(int((134.3e6 + 16.2e6) * B / 8192)
-                                       if args.variant == "different" and args.law == "bernoulli" and
-                                       abs(args.p - 0.1) < 1e-9 else None),
-                              ms_per_launch=round(ms_s, 4), algorithmic_bytes=sbytes)
-
-    # stored activation bytes versus full backprop (from the whole-net entry point's plan)
-    ctx = rad.MLPStep(dims, B, "bf16", args.act, args.variant, args.p, law=args.law)
-    s = ctx.stats
-    held = s.value_bytes + s.index_bytes + s.relu_bytes + s.preact_bytes + s.unsampled_bytes
-    memory = dict(value_bytes=s.value_bytes, index_bytes=s.index_bytes, relu_bytes=s.relu_bytes,
-                  preact_bytes=s.preact_bytes, unsampled_bytes=s.unsampled_bytes, held_bytes=held,
-                  full_backprop_bytes=s.full_backprop_bytes, ratio=round(s.full_backprop_bytes / held, 3))
-
-    # the same shapes with ReLU (1-bit derivatives instead of kept pre-activations): plan only, not run
-    if args.act != "relu":
-        _, sr = rad.rad_mlp_workspace(dims, B, "bf16", "relu", args.variant, args.p, args.law)
-        held_r = sr.value_bytes + sr.index_bytes + sr.relu_bytes + sr.preact_bytes + sr.unsampled_bytes
-        memory["same_shapes_relu"] = dict(value_bytes=sr.value_bytes, index_bytes=sr.index_bytes, relu_bytes=sr.relu_bytes,
-                                          preact_bytes=sr.preact_bytes, unsampled_bytes=sr.unsampled_bytes,
-                                          held_bytes=held_r, full_backprop_bytes=sr.full_backprop_bytes,
-                                          ratio=round(sr.full_backprop_bytes / held_r, 3))
+        k = int(nnz1[0])
+        kernels["dW"] = tensor_entry("projection dW: S^T dZ and R' G, flops 2*B*k*H + 2*D*k*H", ms_dw,
+                                     2.0 * B * k * 8192 + 2.0 * 8192 * k * 8192)
+        kernels["store"] = tensor_entry("projection store S = A R', flops 2*B*D*k", ms_store0, 2.0 * B * 8192 * k)
+    dominant = max(("forward", "dW", "dX"), key=lambda f: by_family.get({"dX": "dX+db"}.get(f, f), 0.0))
+    dom = kernels[dominant]
+    # DRAM bytes per launch from the ncu captures under profiles/ (batch 8192, 8192 x 8192 layer): bytes read grow
+    # with the batch and are scaled by B / 8192, the dW output does not grow.  Only the default workload has one.
+    traffic = None
+    if args.act == "gelu" and abs(args.p - 0.1) < 1e-9 and args.law == "bernoulli" and not fused:
+        traffic = int((1095.8e6 + 251.4e6) * B / 8192) if dominant != "dW" else None
+    roofline = dict(bound=dom["bound"], kernel=dom["kernel"], achieved=dom["achieved"], peak=dom["peak"], unit=dom["unit"],
+                    frac=dom["frac"], traffic=traffic, peak_source=pk["source"] + " (sustained cuBLAS bf16 / copy bandwidth)",
+                    ms_per_launch=dom["ms_per_launch"],
+                    how="CUDA events around each call on the launching stream, inside the timed steps",
+                    kernels=kernels)
 
     # end to end through rad_mlp_step: the batch comes from pinned host memory every step
+    ctx = rad.MLPStep(dims, B, "bf16", args.act, args.variant, args.p, law=args.law)
     Xh = torch.empty(X.shape, dtype=bf).pin_memory()
     Xh.copy_(X)
     yh = torch.empty(labels.shape, dtype=torch.int32).pin_memory()
@@ -575,27 +726,64 @@ def run_ours(args):
                ms_per_step=round(e2e_ms / args.steps, 3), api="rad_mlp_step", last_loss=round(loss, 5),
                pipeline="two device input buffers; the host-to-device copy of step i+1 runs on a copy stream "
                         "under step i; K copies and K steps inside the timed region")
+    # stored activation bytes versus full backprop, from the counts the last step left
+    memory = memory_report(rad, dims, B, args.act, args.variant, args.p, args.law, ctx.nnz.cpu().tolist())
+    del ctx, Xd, yd
+    torch.cuda.empty_cache()
+
+    # The same shapes with ReLU: 1-bit derivatives instead of kept pre-activations, the setting of the
+    # paper's memory figures (App. A).  Timed for real: one warm-up step, then `twin_steps` steps.
+    twin = None
+    if args.act != "relu" and rank == 0 and world == 1 and not args.no_twin:
+        lw2 = LayerwiseStep(rad, torch, dims, B, "relu", args.variant, args.p, args.law)
+        twin_steps = min(args.steps, 2)
+        ms2, launches2, _ = timed_steps(lw2, 1, twin_steps, first_step=50)
+        nnz_all = []
+        for st in lw2.stores:
+            nnz_all += st.nnz.cpu().tolist()
+        twin = dict(act="relu", steps=twin_steps, ms_per_step=round(ms2 / twin_steps, 3),
+                    samples_per_s=round(B * twin_steps / (ms2 / 1e3), 1), gpu_launches=int(launches2),
+                    family_ms={k: round(sum(sum(v) for (f, l), v in lw2.family_ms().items() if f == k) / twin_steps, 3)
+                               for k in ("store", "forward", "loss", "dW", "dX+db")},
+                    activation_memory=memory_report(rad, dims, B, "relu", args.variant, args.p, args.law, nnz_all))
+        del lw2
+        torch.cuda.empty_cache()
 
     sweep = None
     if rank == 0 and world == 1 and not args.no_sweep:
         dZ = (torch.randn(B, 8192, generator=gen, device="cuda") / B).to(bf)
-        sweep = kernel_sweep(rad, torch, X, dZ, 8192, (0.01, 0.05, 0.1, 0.5))
+        sweep = kernel_sweep(rad, torch, X, dZ, 8192, (0.01, 0.05, 0.1, 0.5), pk, clock)
+        # the two kernels the targets are set for, timed alone at this run's p, beside their in-step figures
+        for row in sweep:
+            if row.get("law") is None and row["variant"] == args.variant and abs(row["p"] - args.p) < 1e-9:
+                if "store" in kernels and "store_frac_hbm" in row:
+                    kernels["store"]["alone"] = dict(ms=row["store_ms"], achieved=row["store_gbs"], frac=row["store_frac_hbm"],
+                                                     sm_mhz=row["store_sm_mhz"], peak=hbm, unit="GB/s")
+                kernels["dW"]["alone"] = dict(ms=row["dW_ms"], achieved=row.get("dW_tflops_dense_tile", row.get("dW_tflops_kept_columns")),
+                                              frac=row["dW_frac_burst"], peak=burst, unit="TFLOP/s", peak_kind="burst")
+        del dZ
     small = small_workloads(rad, torch) if (rank == 0 and world == 1 and not args.no_sweep) else None
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
         cpu, _ = time_oracle(args, 1, 0)
+        one, _ = time_oracle(args, 1, 0, rows=CPU_SLAB_ROWS_1CORE, threads=1)
+        cpu["one_core"] = one
+        if small is not None:
+            for name, row in time_small_oracles().items():
+                small[name]["cpu_oracle"] = row
 
     if rank == 0:
+        pe = rad.rad_effective_p(args.p)
         line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                     ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
                     data="synthetic",
-                    config=dict(workload="mlp_wide: 8192->8192x4->1000, bf16, batch 65536 per GPU, N(0,1) inputs",
+                    config=dict(workload=f"mlp_wide: 8192->8192x4->1000, bf16, batch {B} per GPU, N(0,1) inputs",
                                 dims=list(dims), global_batch=world * B, act=args.act, variant=args.variant, law=args.law, p=args.p,
-                                parallelism="replicas" if world > 1 else "1 GPU",
+                                p_sampled=pe, parallelism="replicas" if world > 1 else "1 GPU",
                                 l2="inputs larger than L2 (1 GiB activations per layer)"),
                     clocks=clocks, e2e=e2e, gpu_launches=int(launches), roofline=roofline,
-                    store_roofline=store_roofline, family_ms={k: round(v, 3) for k, v in by_family.items()},
-                    activation_memory=memory, cpu_baseline=cpu, kernel_sweep=sweep, small_workloads=small)
+                    family_ms={k: round(v, 3) for k, v in by_family.items()},
+                    activation_memory=memory, relu_twin=twin, cpu_baseline=cpu, kernel_sweep=sweep, small_workloads=small)
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -354,7 +354,8 @@ typedef struct rad_mlp_desc {
 } rad_mlp_desc;
 
 typedef struct rad_step_stats {   /* bytes held between forward and backward (App. A accounting) */
-  int64_t value_bytes;            /* capacity reserved for kept values (mean + 8 sigma)          */
+  int64_t value_bytes;            /* rad_mlp_workspace: capacity reserved for kept values (mean  */
+                                  /* + 8 sigma); rad_mlp_held_bytes: what a step really kept     */
   int64_t index_bytes;            /* keep bitmasks / kept-column lists and tile offsets          */
   int64_t relu_bytes;             /* 1-bit ReLU derivatives                                      */
   int64_t preact_bytes;           /* pre-activations kept whole (GELU nets only)                 */
@@ -364,6 +365,16 @@ typedef struct rad_step_stats {   /* bytes held between forward and backward (Ap
 
 int rad_mlp_workspace(const rad_mlp_desc* net /* host */, int64_t* bytes /* host */,
                       rad_step_stats* stats /* host or NULL */);
+
+/*
+ * The same accounting from the counts of a step that has run (App. A, "memory saved": what is held between
+ * the passes): `nnz` (host, 2 * L entries) is rad_mlp_step's nnz_out copied back by the caller; value_bytes
+ * then counts the kept values themselves (different-sample: with the padding of every tile to a multiple
+ * of 8 elements; same-sample: B * k' per layer) instead of the reservation.  Host only; the mask depends on
+ * the key alone, so rad_store_index gives the same counts before any step has run.
+ */
+int rad_mlp_held_bytes(const rad_mlp_desc* net /* host */, const int64_t* nnz /* host */,
+                       rad_step_stats* stats /* host */);
 
 /*
  * Forward, loss and RAD backward of the whole net on one stream (Sec. 4.2 for

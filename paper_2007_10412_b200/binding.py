@@ -72,7 +72,7 @@ EXPORTS = ["rad_keep_threshold", "rad_effective_p", "rad_scale", "rad_store_size
            "rad_draws_per_row", "rad_replace_scale", "rad_store_size_query_law", "rad_rademacher",
            "rad_linear_forward_store", "rad_linear_forward_store_static", "rad_weight_grad_workspace", "rad_linear_weight_grad",
            "rad_linear_forward", "rad_store_index", "rad_linear_forward_fill", "rad_softmax_xent", "rad_input_grad_workspace", "rad_linear_input_grad",
-           "rad_mlp_workspace", "rad_mlp_step", "rad_irnn_workspace", "rad_irnn_step", "rad_cnn_workspace", "rad_cnn_step", "rad_launch_count", "rad_strerror", "rad_version",
+           "rad_mlp_workspace", "rad_mlp_held_bytes", "rad_mlp_step", "rad_irnn_workspace", "rad_irnn_step", "rad_cnn_workspace", "rad_cnn_step", "rad_launch_count", "rad_strerror", "rad_version",
            "rad_set_wait_limit_ns", "rad_wait_probe"]
 
 _lib = None
@@ -121,6 +121,7 @@ def lib():
         L.rad_linear_input_grad.argtypes = [i32, i64, i64, i64, vp, i64, vp, i64, vp, vp, i64, vp, i64, vp,
                                             vp, i64, vp, vp]
         L.rad_mlp_workspace.argtypes = [C.POINTER(rad_mlp_desc), C.POINTER(i64), C.POINTER(rad_step_stats)]
+        L.rad_mlp_held_bytes.argtypes = [C.POINTER(rad_mlp_desc), C.POINTER(i64), C.POINTER(rad_step_stats)]
         L.rad_irnn_workspace.argtypes = [C.POINTER(rad_irnn_desc), C.POINTER(i64), C.POINTER(rad_step_stats)]
         L.rad_irnn_step.argtypes = [C.POINTER(rad_irnn_desc)] + [vp] * 15 + [vp, i64, vp, vp]
         L.rad_cnn_workspace.argtypes = [C.POINTER(rad_cnn_desc), C.POINTER(i64), C.POINTER(rad_step_stats)]
@@ -355,6 +356,21 @@ def rad_mlp_workspace(dims, B, dtype="f32", act="relu", variant="different", p=0
     nbytes, stats = C.c_int64(0), rad_step_stats()
     _check(lib().rad_mlp_workspace(C.byref(desc), C.byref(nbytes), C.byref(stats)), "rad_mlp_workspace")
     return nbytes.value, stats
+
+
+def rad_mlp_held_bytes(net, nnz_host):
+    """rad_step_stats of the step that left `nnz_host` (the 2 L counts of MLPStep.nnz, copied to the host).
+    `net`: an MLPStep, or the tuple (dims, B, dtype, act, variant, p, law) of a net shape."""
+    if isinstance(net, tuple):
+        dims, B, dtype, act, variant, p, law = net
+        dims_c = (C.c_int64 * len(dims))(*dims)
+        desc = rad_mlp_desc(len(dims) - 1, ACTS[act], DTYPES[dtype], VARIANTS[variant], dims_c, B, p, 0, 0, LAWS[law])
+    else:
+        desc = net.desc
+    arr = (C.c_int64 * len(nnz_host))(*[int(v) for v in nnz_host])
+    stats = rad_step_stats()
+    _check(lib().rad_mlp_held_bytes(C.byref(desc), arr, C.byref(stats)), "rad_mlp_held_bytes")
+    return stats
 
 
 class MLPStep:

@@ -285,6 +285,25 @@ extern "C" int rad_mlp_workspace(const rad_mlp_desc* net, int64_t* bytes, rad_st
   return RAD_OK;
 }
 
+extern "C" int rad_mlp_held_bytes(const rad_mlp_desc* net, const int64_t* nnz, rad_step_stats* stats) {
+  if (nnz == nullptr || stats == nullptr) return RAD_EINVAL;
+  StepPlan plan;
+  const int rc = make_plan(net, &plan);
+  if (rc != RAD_OK) return rc;
+  *stats = plan.stats;
+  // values as kept by the step that produced `nnz` (padding of the tile-major layout included), not as reserved
+  int64_t held = 0;
+  for (int l = 0; l < net->L; ++l) {
+    if (nnz[2 * l] < 0 || nnz[2 * l + 1] < nnz[2 * l]) return RAD_EINVAL;
+    const int64_t elems = net->variant == RAD_DIFFERENT_SAMPLE ? nnz[2 * l + 1]
+                        : net->variant == RAD_SAME_SAMPLE      ? net->B * nnz[2 * l]
+                                                               : net->B * plan.layer[l].values_ld;
+    held += elems * esize(net->dtype);
+  }
+  stats->value_bytes = held;
+  return RAD_OK;
+}
+
 extern "C" int rad_mlp_step(const rad_mlp_desc* net, const void* X, const int32_t* labels, const void* const* W,
                             const float* const* b, float* const* dW, float* const* db, float* loss,
                             int64_t* nnz_out, void* workspace, int64_t workspace_bytes, int32_t* dev_status,

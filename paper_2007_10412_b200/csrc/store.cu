@@ -378,6 +378,61 @@ __global__ void __launch_bounds__(256) same_gather_kernel(const SameParams p, co
   }
 }
 
+// The same gather with every access 16 bytes wide, for masks dense enough that most of a row is needed
+// anyway (or when the 1-bit ReLU derivatives of the row are wanted, which need all of it): a warp brings a
+// whole row of A into its own shared-memory buffer with asynchronous 16-byte copies, takes the ReLU bits
+// from there, and writes the gathered row eight (bf16) or four (f32) outputs per lane and store.  The kept
+// columns sit in shared memory as 16-bit numbers (D <= 65536).
+template <typename T>
+__global__ void __launch_bounds__(256) same_gather_rows_kernel(const SameParams p, uint32_t* relubits, int64_t w32, int warps) {
+  extern __shared__ __align__(16) unsigned char s_dyn[];
+  constexpr int kPer = 16 / (int)sizeof(T);
+  const int64_t k = min(p.nnz[0], p.ld);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  uint16_t* s_idx = reinterpret_cast<uint16_t*>(s_dyn);
+  const int64_t idx_bytes = (p.ld * 2 + 15) / 16 * 16;
+  for (int64_t j = tid; j < p.ld; j += blockDim.x) {
+    uint32_t col = 0;
+    if (j < k) {
+      col = __ldg(p.idx + j);
+      if (col >= (uint32_t)p.D) { raise_status(p.dev_status, RAD_DEV_EINTERNAL); col = 0; }
+    }
+    s_idx[j] = (uint16_t)col;
+  }
+  __syncthreads();
+  if (warp >= warps) return;
+  const int64_t row_bytes = p.D * (int64_t)sizeof(T);
+  T* s_row = reinterpret_cast<T*>(s_dyn + idx_bytes + (int64_t)warp * row_bytes);
+  const uint32_t s_row_addr = (uint32_t)__cvta_generic_to_shared(s_row);
+  const T* A = static_cast<const T*>(p.A);
+  T* out = static_cast<T*>(p.values);
+  const int64_t chunks = p.D / kPer;
+  for (int64_t b = (int64_t)blockIdx.x * warps + warp; b < p.B; b += (int64_t)gridDim.x * warps) {
+    const T* rowp = A + b * p.lda;
+    for (int64_t c = lane; c < chunks; c += 32)
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s_row_addr + (uint32_t)(c * 16)), "l"(rowp + c * kPer) : "memory");
+    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+    __syncwarp();
+    if (relubits != nullptr) {
+      for (int64_t w = lane; w < w32; w += 32) {
+        uint32_t m = positive32(s_row + w * 32);    // D is a multiple of 32 on this path
+        relubits[b * w32 + w] = m;
+      }
+    }
+    T* orow = out + b * p.ld;
+    for (int64_t j0 = (int64_t)lane * kPer; j0 < p.ld; j0 += 32 * kPer) {
+      __align__(16) T v[kPer];
+#pragma unroll
+      for (int e = 0; e < kPer; ++e) {
+        const float a = j0 + e < k ? to_float(s_row[s_idx[j0 + e]]) : 0.0f;
+        v[e] = from_float<T>(__fmul_rn(a, p.scale));
+      }
+      *reinterpret_cast<uint4*>(orow + j0) = *reinterpret_cast<const uint4*>(v);
+    }
+    __syncwarp();                                   // the row buffer is overwritten by the next row's copies
+  }
+}
+
 // relubits[b, w] = bits of (A[b, 32w .. 32w+31] > 0).  One thread per output word.
 template <typename T>
 __global__ void __launch_bounds__(256) relu_bits_kernel(const T* A, int64_t lda, int64_t B, int64_t D,
@@ -818,6 +873,35 @@ extern "C" int rad_linear_forward_store(const void* A, int64_t lda, const rad_st
     same_replace_mask_kernel<<<1, 1024, 0, s>>>(p, r, ks);
   } else {
     same_mask_kernel<<<1, 1024, 0, s>>>(p, ks);
+  }
+  // Dense masks (most 32-byte sectors of a row hold a kept column) and calls that also want the ReLU bits take
+  // the row-staging kernel; sparse masks without ReLU bits keep the gather that skips the sectors it does not need.
+  {
+    const int64_t row_bytes = st->D * (int64_t)esz, idx_bytes = round_up(st->values_ld * 2, 16);
+    const int64_t smem_budget = 200 * 1024;
+    const int warps = (int)std::min<int64_t>(8, row_bytes > 0 ? (smem_budget - idx_bytes) / row_bytes : 0);
+    const bool rows_ok = colscale == nullptr && st->D % 32 == 0 && st->D <= 65536 && warps >= 2 &&
+                         ((uintptr_t)A & 15) == 0 && (lda * esz) % 16 == 0 && ((uintptr_t)st->values & 15) == 0;
+    const double pe = store_keep_fraction(st);
+    if (rows_ok && (st->relubits != nullptr || pe >= 0.15)) {
+      const size_t smem = (size_t)(idx_bytes + warps * row_bytes);
+      static int sms = 0;
+      if (sms == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+          sms = 148;
+      }
+      const int grid_r = (int)std::min<int64_t>(ceil_div(st->B, warps), sms);
+      if (st->dtype == RAD_BF16) {
+        RAD_CUDA_TRY(cudaFuncSetAttribute(same_gather_rows_kernel<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_budget));
+        same_gather_rows_kernel<bf16><<<grid_r, 256, smem, s>>>(p, st->relubits, w32, warps);
+      } else {
+        RAD_CUDA_TRY(cudaFuncSetAttribute(same_gather_rows_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_budget));
+        same_gather_rows_kernel<float><<<grid_r, 256, smem, s>>>(p, st->relubits, w32, warps);
+      }
+      RAD_CUDA_TRY(cudaGetLastError());
+      return RAD_OK;
+    }
   }
   const int grid = (int)std::min<int64_t>(ceil_div(st->B, 8), 148 * 8);
   if (st->dtype == RAD_BF16)

@@ -48,6 +48,33 @@ __device__ __forceinline__ uint64_t warp_sum_u64(uint64_t v) {
   return v;
 }
 
+// Bits of (a > 0) for 32 consecutive entries in shared memory; zero of either sign gives 0.
+__device__ __forceinline__ uint32_t positive32(const float* src) {
+  uint32_t m = 0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const float4 v = reinterpret_cast<const float4*>(src)[i];
+    m |= (v.x > 0.0f ? 1u : 0u) << (4 * i) | (v.y > 0.0f ? 1u : 0u) << (4 * i + 1) |
+         (v.z > 0.0f ? 1u : 0u) << (4 * i + 2) | (v.w > 0.0f ? 1u : 0u) << (4 * i + 3);
+  }
+  return m;
+}
+__device__ __forceinline__ uint32_t positive32(const bf16* src) {
+  uint32_t m = 0;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const uint4 q = reinterpret_cast<const uint4*>(src)[i];
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      // positive: sign clear and some other bit set (the add carries into the sign position)
+      const uint32_t nz = ((w[j] & 0x7fff7fffu) + 0x7fff7fffu) & ~w[j] & 0x80008000u;
+      m |= ((nz >> 15) & 1u) << (8 * i + 2 * j) | (nz >> 31) << (8 * i + 2 * j + 1);
+    }
+  }
+  return m;
+}
+
 struct StoreParams {
   const void* A;
   int64_t lda;

@@ -74,3 +74,35 @@ def test_host_only_entry_points_of_the_with_replacement_law_and_the_kernel_choic
     assert b.rad_set_store_kernel("pipelined") == "generic"
     assert b.rad_set_store_kernel("auto") == "pipelined"
     assert b.lib().rad_set_store_kernel(7) == -1
+
+
+def test_held_bytes_from_the_counts_of_a_step():
+    """rad_mlp_held_bytes is host arithmetic on the counts a step leaves: against the oracle's own accounting of
+    the stores it builds for the same net (values only; the device pads every tile to a multiple of 8)."""
+    import ctypes as C
+    from oracle import rad as orc
+    from workloads import mlp_inputs
+    from paper_2007_10412_b200 import binding as b
+    dims, B = (70, 52, 33, 10), 37
+    X, y, Ws, bs = mlp_inputs(dims, B, "f32", "normal", 5)
+    for variant in ("same", "different"):
+        ref = orc.mlp_step(X, y, Ws, bs, dtype="f32", variant=variant, p=0.3, seed=4, step=1)
+        want = orc.stored_bytes(ref.stores, (B, dims[-1]), 4)
+        dims_c = (C.c_int64 * len(dims))(*dims)
+        desc = b.rad_mlp_desc(len(dims) - 1, b.ACTS["relu"], b.DTYPES["f32"], b.VARIANTS[variant], dims_c, B, 0.3, 1, 4, 0)
+        nnz = []
+        for st in ref.stores:
+            # different-sample: (kept entries, elements used with per-tile padding); same-sample: (k', B k')
+            nnz += [st.nnz, st.nnz] if variant == "different" else [st.idx.size, st.nnz]
+        arr = (C.c_int64 * len(nnz))(*nnz)
+        stats = b.rad_step_stats()
+        assert b.lib().rad_mlp_held_bytes(C.byref(desc), arr, C.byref(stats)) == 0
+        assert stats.value_bytes == want["value_bytes"]
+        assert stats.relu_bytes == want["relu_bytes"] and stats.unsampled_bytes == want["unsampled_bytes"]
+        assert stats.full_backprop_bytes == want["full_backprop_bytes"]
+        reserved = b.rad_step_stats()
+        nbytes = C.c_int64(0)
+        assert b.lib().rad_mlp_workspace(C.byref(desc), C.byref(nbytes), C.byref(reserved)) == 0
+        assert reserved.value_bytes >= stats.value_bytes
+    arr[1] = arr[0] - 1
+    assert b.lib().rad_mlp_held_bytes(C.byref(desc), arr, C.byref(stats)) == -1
