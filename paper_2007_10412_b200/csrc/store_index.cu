@@ -69,56 +69,78 @@ __global__ void __launch_bounds__(32 * kIndexWarps) store_index_kernel(const Ind
 }
 
 // offsets[t] holds the exact kept count of tile t on entry and the first element of tile t in `values` on
-// exit (every tile padded to a multiple of kValueAlign); offsets[ntiles] = elements used.  One CTA: a thread
-// takes 16 consecutive tiles per round (its loads are issued together), 16384 tiles per round.
+// exit (every tile padded to a multiple of kValueAlign); offsets[ntiles] = elements used.  One CTA, 16384
+// tiles per round; a thread takes 16 consecutive tiles (four 16-byte loads and stores where `offsets` is
+// 16-byte aligned), adds them up locally, and one warp scan plus one pass over the warp sums places them.
 constexpr int kScanPer = 16;
-__global__ void __launch_bounds__(1024) offsets_scan_kernel(const IndexParams p) {
-  __shared__ uint32_t s_pad[32], s_exact[32];
-  __shared__ uint64_t s_carry_pad, s_carry_exact;
+__global__ void __launch_bounds__(1024) offsets_scan_kernel(const IndexParams p, int vec) {
+  __shared__ uint64_t s_warp[32];                   // padded sum in the high half, exact sum in the low half
+  __shared__ uint64_t s_carry;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) { s_carry_pad = 0; s_carry_exact = 0; }
+  if (tid == 0) s_carry = 0;
   __syncthreads();
   const int64_t ntiles = p.ntiles;
   for (int64_t r0 = 0; r0 < ntiles; r0 += 1024 * kScanPer) {
     const int64_t t0 = r0 + (int64_t)tid * kScanPer;
+    const bool whole = vec != 0 && t0 + kScanPer <= ntiles;
     uint32_t c[kScanPer];
+    if (whole) {
 #pragma unroll
-    for (int i = 0; i < kScanPer; ++i) c[i] = t0 + i < ntiles ? p.offsets[t0 + i] : 0u;
-    uint32_t pad = 0, exact = 0;                    // a round holds at most 16384 * 8192 entries: 32 bits do
+      for (int i = 0; i < kScanPer; i += 4) {
+        const uint4 q = *reinterpret_cast<const uint4*>(p.offsets + t0 + i);
+        c[i] = q.x; c[i + 1] = q.y; c[i + 2] = q.z; c[i + 3] = q.w;
+      }
+    } else {
 #pragma unroll
-    for (int i = 0; i < kScanPer; ++i) {
-      exact += c[i];
-      pad += (c[i] + kValueAlign - 1) / kValueAlign * kValueAlign;
+      for (int i = 0; i < kScanPer; ++i) c[i] = t0 + i < ntiles ? p.offsets[t0 + i] : 0u;
     }
-    uint32_t ipad = pad, iex = exact;
+    // a round holds at most 16384 * 8192 entries: 32 bits each for the padded and the exact sum
+    uint64_t mine = 0;
+#pragma unroll
+    for (int i = 0; i < kScanPer; ++i)
+      mine += ((uint64_t)((c[i] + kValueAlign - 1) / kValueAlign * kValueAlign) << 32) | c[i];
+    uint64_t incl = mine;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t a = __shfl_up_sync(0xffffffffu, ipad, o), b = __shfl_up_sync(0xffffffffu, iex, o);
-      if (lane >= o) { ipad += a; iex += b; }
+      const uint64_t n = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += n;
     }
-    if (lane == 31) { s_pad[warp] = ipad; s_exact[warp] = iex; }
+    if (lane == 31) s_warp[warp] = incl;
     __syncthreads();
-    uint64_t base = s_carry_pad + (ipad - pad), round_pad = 0, round_exact = 0;
+    const uint64_t carry = s_carry;
+    uint64_t before = incl - mine, round_total = 0;
 #pragma unroll
     for (int i = 0; i < 32; ++i) {
-      if (i < warp) base += s_pad[i];
-      round_pad += s_pad[i];
-      round_exact += s_exact[i];
+      const uint64_t t = s_warp[i];
+      if (i < warp) before += t;
+      round_total += t;
     }
+    uint32_t at = (uint32_t)((carry >> 32) + (before >> 32));     // the padded total stays below 2^32
+    uint32_t o[kScanPer];
 #pragma unroll
     for (int i = 0; i < kScanPer; ++i) {
-      if (t0 + i < ntiles) p.offsets[t0 + i] = (uint32_t)base;
-      base += (c[i] + kValueAlign - 1) / kValueAlign * kValueAlign;
+      o[i] = at;
+      at += (c[i] + kValueAlign - 1) / kValueAlign * kValueAlign;
     }
-    __syncthreads();                                // everyone has read the carry and the warp totals
-    if (tid == 0) { s_carry_pad += round_pad; s_carry_exact += round_exact; }
+    if (whole) {
+#pragma unroll
+      for (int i = 0; i < kScanPer; i += 4)
+        *reinterpret_cast<uint4*>(p.offsets + t0 + i) = make_uint4(o[i], o[i + 1], o[i + 2], o[i + 3]);
+    } else {
+#pragma unroll
+      for (int i = 0; i < kScanPer; ++i)
+        if (t0 + i < ntiles) p.offsets[t0 + i] = o[i];
+    }
+    __syncthreads();                                // everyone has read the carry and the warp sums
+    if (tid == 0) s_carry = carry + round_total;
     __syncthreads();
   }
   if (tid == 0) {
-    p.offsets[ntiles] = (uint32_t)s_carry_pad;
-    p.nnz[0] = (int64_t)s_carry_exact;
-    p.nnz[1] = (int64_t)s_carry_pad;
-    if (p.capacity >= 0 && (int64_t)s_carry_pad > p.capacity) raise_status(p.dev_status, RAD_DEV_ECAPACITY);
+    const uint64_t total = s_carry;
+    p.offsets[ntiles] = (uint32_t)(total >> 32);
+    p.nnz[0] = (int64_t)(total & 0xffffffffu);
+    p.nnz[1] = (int64_t)(total >> 32);
+    if (p.capacity >= 0 && (int64_t)(total >> 32) > p.capacity) raise_status(p.dev_status, RAD_DEV_ECAPACITY);
   }
 }
 
@@ -140,7 +162,7 @@ int launch_store_index(const rad_store* st, bool check_capacity, int32_t* dev_st
   const int grid = (int)std::min<int64_t>(ceil_div(p.ntiles, kIndexWarps), 148 * 12);
   count_launch(2);
   store_index_kernel<<<grid, 32 * kIndexWarps, 0, s>>>(p, ks);
-  offsets_scan_kernel<<<1, 1024, 0, s>>>(p);
+  offsets_scan_kernel<<<1, 1024, 0, s>>>(p, ((uintptr_t)p.offsets & 15) == 0 ? 1 : 0);
   return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
 }
 
