@@ -48,7 +48,7 @@ extern "C" {
 #define RAD_DEV_EINTERNAL 3    /* an index left its buffer; the access was skipped (a bug)   */
 
 typedef enum { RAD_F32 = 0, RAD_BF16 = 1 } rad_dtype;
-typedef enum { RAD_DIFFERENT_SAMPLE = 0, RAD_SAME_SAMPLE = 1, RAD_PROJECT = 2 } rad_variant;
+typedef enum { RAD_DIFFERENT_SAMPLE = 0, RAD_SAME_SAMPLE = 1, RAD_PROJECT = 2, RAD_ROWS_SAMPLE = 3 } rad_variant;
 typedef enum { RAD_ACT_NONE = 0, RAD_ACT_RELU = 1, RAD_ACT_GELU = 2 } rad_act;
 
 /* Geometry of the compact store (fixed; part of the data layout). */
@@ -159,6 +159,20 @@ typedef struct rad_store_sizes {
   int64_t keepbits_words, offsets_words, relubits_words;
   int64_t workspace_bytes;    /* scratch rad_linear_forward_store needs                        */
 } rad_store_sizes;
+
+/*
+ * Static-shape variant, variant = RAD_ROWS_SAMPLE with law = RAD_LAW_FIXED (App. A, remark under the fraction
+ * sweep: sampling without replacement): a different sample per minibatch row as with RAD_DIFFERENT_SAMPLE, but
+ * every row keeps exactly k = ceil(p * D) columns, so the store has the same shape whatever the key:
+ *   values   : B x values_ld row-major (values_ld a multiple of 8, at least k; the size query gives k rounded
+ *              up to 8); values[b, j] = A[b, c] * fl32(D / k) for the j-th smallest kept column c of row b,
+ *              zero for k <= j < values_ld.
+ *   keepbits : read as uint16: B x values_ld column numbers, cols[b, j] = c (0 for j >= k); D <= 65536.
+ *   offsets  : unused, may be NULL.   nnz[0] = B * k, nnz[1] = B * values_ld.
+ * The kept set of a row is the one the fixed-count law of RAD_DIFFERENT_SAMPLE keeps for the same key.
+ * rad_linear_weight_grad takes such a store: it rebuilds the index part of the tile-major layout from the key
+ * alone, moves the values into it (both in its workspace) and runs the same contraction.
+ */
 
 /*
  * Random-projection variant, variant = RAD_PROJECT (Sec. 3.2 after Eq. 5; App. A "Random

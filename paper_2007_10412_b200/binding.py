@@ -15,13 +15,13 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "librad_b200.so")
 
 RAD_F32, RAD_BF16 = 0, 1
-RAD_DIFFERENT_SAMPLE, RAD_SAME_SAMPLE, RAD_PROJECT = 0, 1, 2
+RAD_DIFFERENT_SAMPLE, RAD_SAME_SAMPLE, RAD_PROJECT, RAD_ROWS_SAMPLE = 0, 1, 2, 3
 RAD_ACT_NONE, RAD_ACT_RELU, RAD_ACT_GELU = 0, 1, 2
 RAD_DEV_ECAPACITY, RAD_DEV_ETIMEOUT = 1, 2
 TILE_ROWS, TILE_COLS, VALUE_ALIGN = 64, 128, 8
 
 DTYPES = {"f32": RAD_F32, "bf16": RAD_BF16, torch.float32: RAD_F32, torch.bfloat16: RAD_BF16}
-VARIANTS = {"different": RAD_DIFFERENT_SAMPLE, "same": RAD_SAME_SAMPLE, "project": RAD_PROJECT}
+VARIANTS = {"different": RAD_DIFFERENT_SAMPLE, "same": RAD_SAME_SAMPLE, "project": RAD_PROJECT, "rows": RAD_ROWS_SAMPLE}
 LAWS = {"bernoulli": 0, "replace": 1, "fixed": 2}
 ACTS = {"none": RAD_ACT_NONE, "relu": RAD_ACT_RELU, "gelu": RAD_ACT_GELU}
 TORCH_DTYPE = {RAD_F32: torch.float32, RAD_BF16: torch.bfloat16}
@@ -211,13 +211,13 @@ class Store:
         self.sizes = sz
         cap = {"typical": sz.values_typical, "worst": sz.values_worst}.get(capacity, capacity)
         ld = 0
-        if variant in ("same", "project"):
+        if variant in ("same", "project", "rows"):
             ld = {"typical": sz.values_ld_typical, "worst": sz.values_ld_worst}.get(capacity, capacity)
             cap = B * ld
         tdt = TORCH_DTYPE[DTYPES[dtype]]
         self.values = torch.empty(max(int(cap), 8), dtype=tdt, device=device)
         self.keepbits = torch.empty(sz.keepbits_words, dtype=torch.int32, device=device)
-        self.offsets = torch.empty(sz.offsets_words, dtype=torch.int32, device=device)
+        self.offsets = torch.empty(max(sz.offsets_words, 1), dtype=torch.int32, device=device)
         self.nnz = torch.zeros(2, dtype=torch.int64, device=device)
         self.relubits = torch.empty(sz.relubits_words, dtype=torch.int32, device=device) if relu_bits else None
         self.workspace = torch.empty(sz.workspace_bytes, dtype=torch.uint8, device=device)

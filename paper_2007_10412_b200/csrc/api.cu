@@ -28,6 +28,29 @@ namespace {
 bool valid_dtype(int d) { return d == RAD_F32 || d == RAD_BF16; }
 int64_t esize(int dtype) { return dtype == RAD_BF16 ? 2 : 4; }
 
+// Tile-major twin of a static-shape (RAD_ROWS_SAMPLE) store, laid out in a workspace: same key, same mask.
+struct TileTwin { rad_store st; int64_t bytes; };
+TileTwin tile_twin(const rad_store* rows, char* ws) {
+  TileTwin t;
+  const int64_t k = draws_per_row_host(rows->p, rows->D);
+  const int64_t ntiles = ceil_div(rows->B, kTileRows) * ceil_div(rows->D, kTileCols);
+  const int64_t cap = round_up(rows->B * k + ntiles * (kValueAlign - 1), kValueAlign);
+  int64_t off = 0;
+  auto take = [&](int64_t bytes) { const int64_t at = off; off += round_up(bytes, 256); return at; };
+  t.st = *rows;
+  t.st.variant = RAD_DIFFERENT_SAMPLE;
+  t.st.values_capacity = cap;
+  t.st.values_ld = 0;
+  const int64_t v = take(cap * esize(rows->dtype)), kb = take(ntiles * kTileWords * 4), of = take((ntiles + 1) * 4), nz = take(16);
+  t.st.values = ws != nullptr ? ws + v : nullptr;
+  t.st.keepbits = ws != nullptr ? reinterpret_cast<uint32_t*>(ws + kb) : nullptr;
+  t.st.offsets = ws != nullptr ? reinterpret_cast<uint32_t*>(ws + of) : nullptr;
+  t.st.nnz = ws != nullptr ? reinterpret_cast<int64_t*>(ws + nz) : nullptr;
+  t.st.relubits = nullptr;
+  t.bytes = off;
+  return t;
+}
+
 bool store_args_ok(const rad_store* st) {
   if (st == nullptr || st->B <= 0 || st->D <= 0) return false;
   if (st->variant != RAD_DIFFERENT_SAMPLE && st->variant != RAD_SAME_SAMPLE) return false;
@@ -158,6 +181,12 @@ extern "C" int rad_weight_grad_workspace(const rad_store* st, int64_t H, int64_t
     *bytes = project_weight_grad_workspace(st, H);
     return RAD_OK;
   }
+  if (st->variant == RAD_ROWS_SAMPLE) {
+    if (draws_per_row_host(st->p, st->D) == 0) return RAD_EINVAL;
+    const TileTwin t = tile_twin(st, nullptr);
+    *bytes = t.bytes + round_up(tc_weight_grad_workspace(&t.st, H), 256);
+    return RAD_OK;
+  }
   *bytes = round_up(tc_weight_grad_workspace(st, H), 256);
   return RAD_OK;
 }
@@ -172,6 +201,27 @@ extern "C" int rad_linear_weight_grad(const rad_store* st, const void* dZ, int64
     const int rcp = check_device();
     return rcp != RAD_OK ? rcp
                          : project_weight_grad(st, dZ, ldz, H, dW, ldw, workspace, workspace_bytes, dev_status, stream);
+  }
+  if (st != nullptr && st->variant == RAD_ROWS_SAMPLE) {
+    // static-shape store: index part of the tile-major layout from the key alone, values moved into it, then
+    // the same contraction as for a bitmask store
+    if (st->B <= 0 || st->D <= 0 || !valid_dtype(st->dtype) || dZ == nullptr || dW == nullptr || H <= 0 || ldz < H || ldw < H ||
+        !rows_store_ok(st))
+      return RAD_EINVAL;
+    int rcr = check_device();
+    if (rcr != RAD_OK) return rcr;
+    int64_t need = 0;
+    rcr = rad_weight_grad_workspace(st, H, &need);
+    if (rcr != RAD_OK) return rcr;
+    if (workspace == nullptr || workspace_bytes < need || ((uintptr_t)workspace & 255) != 0) return RAD_EWORKSPACE;
+    const TileTwin t = tile_twin(st, static_cast<char*>(workspace));
+    cudaStream_t sr = static_cast<cudaStream_t>(stream);
+    rcr = launch_fixed_index(&t.st, true, dev_status, sr);
+    if (rcr != RAD_OK) return rcr;
+    rcr = rows_to_tiles(st, &t.st, dev_status, sr);
+    if (rcr != RAD_OK) return rcr;
+    return rad_linear_weight_grad(&t.st, dZ, ldz, H, dW, ldw, static_cast<char*>(workspace) + t.bytes, workspace_bytes - t.bytes,
+                                  dev_status, stream);
   }
   if (!store_args_ok(st) || dZ == nullptr || dW == nullptr || H <= 0 || ldz < H || ldw < H) return RAD_EINVAL;
   int rc = check_device();

@@ -220,6 +220,12 @@ int tc_forward(int act, int64_t B, int64_t D, int64_t H, const void* A, int64_t 
 // store_index.cu: keep bits, row offsets, tile offsets and nnz of a different-sample Bernoulli store from the
 // key alone (no layer input is read)
 int launch_store_index(const rad_store* st, bool check_capacity, int32_t* dev_status, cudaStream_t s);
+int launch_offsets_scan(uint32_t* offsets, int64_t ntiles, int64_t* nnz, int64_t capacity, int32_t* dev_status, cudaStream_t s);
+// store_rows.cu: fixed-count law (exactly k columns per row): static-shape store, key-only index, re-tiling
+bool rows_store_ok(const rad_store* st);
+int rows_forward_store(const void* A, int64_t lda, const rad_store* st, int32_t* dev_status, cudaStream_t s);
+int launch_fixed_index(const rad_store* st, bool check_capacity, int32_t* dev_status, cudaStream_t s);
+int rows_to_tiles(const rad_store* rows, const rad_store* tiles, int32_t* dev_status, cudaStream_t s);
 int tc_input_grad(int64_t B, int64_t D, int64_t H, const void* dZ, int64_t ldz, const void* W,
                   int64_t ldw, const uint32_t* relubits_prev, const void* z_prev, int64_t ld_zprev,
                   void* dZ_prev, int64_t ldp, int32_t* dev_status, cudaStream_t s);

@@ -104,10 +104,13 @@ __device__ __forceinline__ uint32_t transpose4x4_bytes(uint32_t v, int k) {
   return v;
 }
 
-// kReplace: keep bits and weights come from the multiplicity matrix (with-replacement law) instead
-// of a Bernoulli draw; everything after the mask is the same.
-template <typename T, bool kReplace>
+// Where the mask comes from: a Bernoulli draw in the kernel; the multiplicity matrix of the with-replacement law
+// (which also gives the weights); or keep bits and tile offsets that are already in place (made from the key
+// alone by an index kernel), in which case only values and ReLU bits are written and nothing waits for anything.
+enum MaskSource { kMaskDraw = 0, kMaskCounts = 1, kMaskIndex = 2 };
+template <typename T, int kMask>
 __global__ void __launch_bounds__(256) store_different_kernel(const StoreParams p, const PhiloxKeys ks) {
+  constexpr bool kReplace = kMask == kMaskCounts;
   __shared__ uint32_t s_rowcnt[kTileRows];
   __shared__ uint32_t s_rowoff[kTileRows];
   __shared__ uint32_t s_tile;
@@ -116,7 +119,7 @@ __global__ void __launch_bounds__(256) store_different_kernel(const StoreParams 
   __shared__ __align__(16) T s_stage[kTileRows * kTileCols];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) s_tile = atomicAdd(p.ticket, 1u);
+  if (tid == 0) s_tile = kMask == kMaskIndex ? blockIdx.x : atomicAdd(p.ticket, 1u);
   __syncthreads();
   const uint32_t tile = s_tile;
   if (tile >= (uint32_t)p.ntiles) return;
@@ -135,7 +138,8 @@ __global__ void __launch_bounds__(256) store_different_kernel(const StoreParams 
     const int64_t row = slab * kTileRows + warp * 8 + it * 2 + half;
     // four lanes share a keep-bit word and make it together (all lanes take part, valid or not)
     uint32_t word = 0;
-    if (!kReplace) word = philox_keep32_quad((uint32_t)(col0 >> 5), (uint32_t)row, p.c2, p.c3, ks, p.T, lane);
+    if (kMask == kMaskDraw) word = philox_keep32_quad((uint32_t)(col0 >> 5), (uint32_t)row, p.c2, p.c3, ks, p.T, lane);
+    if (kMask == kMaskIndex) word = p.keepbits[(int64_t)tile * kTileWords + (warp * 8 + it * 2 + half) * 4 + (cg >> 2)];
     if (row < p.B && nvalid > 0) {
       load8<T>(Abase + row * p.lda, col0, nvalid, p.vec_ok != 0, raw[it]);
       uint32_t m;
@@ -172,7 +176,7 @@ __global__ void __launch_bounds__(256) store_different_kernel(const StoreParams 
     // four lanes make one 32-bit word of keep bits (and of ReLU bits) per item
     const int k = cg & 3;
     const int r = warp * 8 + k * 2 + half;
-    p.keepbits[(int64_t)tile * kTileWords + r * 4 + (cg >> 2)] = transpose4x4_bytes(masks, k);
+    if (kMask != kMaskIndex) p.keepbits[(int64_t)tile * kTileWords + r * 4 + (cg >> 2)] = transpose4x4_bytes(masks, k);
     if (p.relubits != nullptr) {
       const uint32_t rw = transpose4x4_bytes(relus, k);
       const int64_t row = slab * kTileRows + r;
@@ -195,14 +199,15 @@ __global__ void __launch_bounds__(256) store_different_kernel(const StoreParams 
     s_rowoff[2 * lane] = ex;
     s_rowoff[2 * lane + 1] = ex + v0;
     // row offsets travel with the keep bits: the dW kernel finds a row's values without a scan
-    p.keepbits[(int64_t)tile * kTileWords + kBitWords + lane] = ex | ((ex + v0) << 16);
+    if (kMask != kMaskIndex) p.keepbits[(int64_t)tile * kTileWords + kBitWords + lane] = ex | ((ex + v0) << 16);
     const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
     if (lane == 0) {
       s_total = total;
       const uint32_t gran = (total + kValueAlign - 1) / kValueAlign;
       // the first tile knows its prefix at once; the others publish their own count first
-      store_status(p.status + tile, ((tile == 0 ? kFlagPrefix : kFlagAggregate) << kFlagShift) |
-                                        pack_counts(gran, total));
+      if (kMask != kMaskIndex)
+        store_status(p.status + tile, ((tile == 0 ? kFlagPrefix : kFlagAggregate) << kFlagShift) |
+                                          pack_counts(gran, total));
     }
   }
   __syncthreads();
@@ -229,8 +234,19 @@ __global__ void __launch_bounds__(256) store_different_kernel(const StoreParams 
   }
   if (tid < (int)(padded - total)) s_stage[total + tid] = from_float<T>(0.0f);
 
-  // look-back (warp 0): sum the counts of earlier tiles until one with a known prefix is met
-  if (warp == 0) {
+  if (kMask == kMaskIndex) {
+    // the tile's place is known: no look-back
+    if (tid == 0) {
+      const int64_t base = p.offsets[tile];
+      if (base + padded > p.capacity) {
+        raise_status(p.dev_status, RAD_DEV_ECAPACITY);
+        s_base = -1;
+      } else {
+        s_base = base;
+      }
+    }
+  } else if (warp == 0) {
+    // look-back (warp 0): sum the counts of earlier tiles until one with a known prefix is met
     uint64_t excl = 0;
     bool failed = false;
     if (tile != 0) {
@@ -638,13 +654,13 @@ int launch_store_different(const StoreParams& p, const PhiloxKeys& ks, int dtype
   count_launch();
   if (p.counts != nullptr) {
     if (dtype == RAD_BF16)
-      store_different_kernel<bf16, true><<<p.ntiles, 256, 0, s>>>(p, ks);
+      store_different_kernel<bf16, kMaskCounts><<<p.ntiles, 256, 0, s>>>(p, ks);
     else
-      store_different_kernel<float, true><<<p.ntiles, 256, 0, s>>>(p, ks);
+      store_different_kernel<float, kMaskCounts><<<p.ntiles, 256, 0, s>>>(p, ks);
   } else if (dtype == RAD_BF16) {
-    store_different_kernel<bf16, false><<<p.ntiles, 256, 0, s>>>(p, ks);
+    store_different_kernel<bf16, kMaskDraw><<<p.ntiles, 256, 0, s>>>(p, ks);
   } else {
-    store_different_kernel<float, false><<<p.ntiles, 256, 0, s>>>(p, ks);
+    store_different_kernel<float, kMaskDraw><<<p.ntiles, 256, 0, s>>>(p, ks);
   }
   RAD_CUDA_TRY(cudaGetLastError());
   return RAD_OK;
@@ -730,6 +746,20 @@ extern "C" int rad_store_size_query_law(int32_t variant, int32_t dtype, int32_t 
     out->workspace_bytes = project_store_workspace(dtype, D, ld);
     return RAD_OK;
   }
+  if (variant == RAD_ROWS_SAMPLE) {
+    // B x ld values and B x ld 16-bit column numbers (ld: k rounded up to 8 columns); exact, whatever the key
+    const int64_t k = draws_per_row_host(p, D);
+    if (k == 0 || law != RAD_LAW_FIXED) return RAD_EINVAL;
+    if (D > 65536) return RAD_EUNSUPPORTED;
+    const int64_t ld = round_up(k, 8);
+    out->values_ld_worst = out->values_ld_typical = ld;
+    out->values_worst = out->values_typical = B * ld;
+    out->keepbits_words = B * ld / 2;
+    out->offsets_words = 0;
+    out->relubits_words = B * ceil_div(D, 32);
+    out->workspace_bytes = 256;
+    return RAD_OK;
+  }
   if (variant != RAD_DIFFERENT_SAMPLE && variant != RAD_SAME_SAMPLE) return RAD_EINVAL;
   if (law != RAD_LAW_BERNOULLI && law != RAD_LAW_REPLACE && law != RAD_LAW_FIXED) return RAD_EINVAL;
   const uint32_t T = keep_threshold_host(p);
@@ -778,6 +808,10 @@ extern "C" int rad_linear_forward_store(const void* A, int64_t lda, const rad_st
     const int rcp = check_device();
     return rcp != RAD_OK ? rcp : project_forward_store(A, lda, st, workspace, workspace_bytes, dev_status, stream);
   }
+  if (st->variant == RAD_ROWS_SAMPLE) {
+    const int rcr = check_device();
+    return rcr != RAD_OK ? rcr : rows_forward_store(A, lda, st, dev_status, static_cast<cudaStream_t>(stream));
+  }
   if (st->variant != RAD_DIFFERENT_SAMPLE && st->variant != RAD_SAME_SAMPLE) return RAD_EINVAL;
   if (st->values == nullptr || st->keepbits == nullptr || st->offsets == nullptr || st->nnz == nullptr)
     return RAD_EINVAL;
@@ -821,6 +855,21 @@ extern "C" int rad_linear_forward_store(const void* A, int64_t lda, const rad_st
     p.vec_ok = (((uintptr_t)A & 15) == 0 && (lda * esz) % 16 == 0) ? 1 : 0;
     p.counts = nullptr; p.ldc = 0;
     p.wait_limit_ns = wait_limit_ns();
+    if (fixed) {
+      // exactly k columns per row: the index part comes from the key alone (Floyd's sampling, a warp per row),
+      // then one CTA per tile places the values; no multiplicity matrix, no look-back
+      rc = launch_fixed_index(st, true, dev_status, s);
+      if (rc == RAD_OK) {
+        count_launch();
+        if (st->dtype == RAD_BF16)
+          store_different_kernel<bf16, kMaskIndex><<<p.ntiles, 256, 0, s>>>(p, ks);
+        else
+          store_different_kernel<float, kMaskIndex><<<p.ntiles, 256, 0, s>>>(p, ks);
+        RAD_CUDA_TRY(cudaGetLastError());
+        return RAD_OK;
+      }
+      if (rc != RAD_EUNSUPPORTED) return rc;      // rows too long for shared memory: the multiplicity matrix below
+    }
     RAD_CUDA_TRY(cudaMemsetAsync(workspace, 0, (size_t)status_bytes(st->B, st->D), s));
     if (replace) {
       // first the multiplicities of every row, then the generic kernel with the mask and the weights

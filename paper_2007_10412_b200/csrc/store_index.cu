@@ -146,6 +146,16 @@ __global__ void __launch_bounds__(1024) offsets_scan_kernel(const IndexParams p,
 
 }  // namespace
 
+// Exact kept counts per tile in offsets[0 .. ntiles) -> padded exclusive prefixes, offsets[ntiles] and nnz.
+int launch_offsets_scan(uint32_t* offsets, int64_t ntiles, int64_t* nnz, int64_t capacity, int32_t* dev_status,
+                        cudaStream_t s) {
+  IndexParams p = {};
+  p.ntiles = (int32_t)ntiles; p.offsets = offsets; p.nnz = nnz; p.capacity = capacity; p.dev_status = dev_status;
+  count_launch();
+  offsets_scan_kernel<<<1, 1024, 0, s>>>(p, ((uintptr_t)offsets & 15) == 0 ? 1 : 0);
+  return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
+}
+
 // Index part (keep bits, row offsets, tile offsets, nnz) of a different-sample Bernoulli store.
 int launch_store_index(const rad_store* st, bool check_capacity, int32_t* dev_status, cudaStream_t s) {
   const uint32_t T = keep_threshold_host(st->p);
@@ -160,10 +170,11 @@ int launch_store_index(const rad_store* st, bool check_capacity, int32_t* dev_st
   p.dev_status = dev_status;
   const PhiloxKeys ks = philox_expand_key(st->seed);
   const int grid = (int)std::min<int64_t>(ceil_div(p.ntiles, kIndexWarps), 148 * 12);
-  count_launch(2);
+  if (st->law == RAD_LAW_FIXED) return launch_fixed_index(st, check_capacity, dev_status, s);
+  count_launch();
   store_index_kernel<<<grid, 32 * kIndexWarps, 0, s>>>(p, ks);
-  offsets_scan_kernel<<<1, 1024, 0, s>>>(p, ((uintptr_t)p.offsets & 15) == 0 ? 1 : 0);
-  return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
+  if (cudaGetLastError() != cudaSuccess) return RAD_ECUDA;
+  return launch_offsets_scan(p.offsets, p.ntiles, p.nnz, p.capacity, dev_status, s);
 }
 
 }  // namespace rad
@@ -172,7 +183,7 @@ using namespace rad;
 
 extern "C" int rad_store_index(const rad_store* st, int32_t* dev_status, void* stream) {
   if (st == nullptr || st->B <= 0 || st->D <= 0) return RAD_EINVAL;
-  if (st->variant != RAD_DIFFERENT_SAMPLE || st->law != RAD_LAW_BERNOULLI) return RAD_EUNSUPPORTED;
+  if (st->variant != RAD_DIFFERENT_SAMPLE || (st->law != RAD_LAW_BERNOULLI && st->law != RAD_LAW_FIXED)) return RAD_EUNSUPPORTED;
   if (st->keepbits == nullptr || st->offsets == nullptr || st->nnz == nullptr) return RAD_EINVAL;
   if (keep_threshold_host(st->p) == 0) return RAD_EINVAL;
   if ((double)st->B * (double)st->D >= 4294967296.0 * 0.75) return RAD_EINVAL;
