@@ -44,39 +44,53 @@ struct RowsParams {
 
 // Floyd's subset of row `row` into `bm` (words of the row's bitmap in shared memory, zero on entry), by one
 // warp.  `draws`: k words of the warp's own shared memory.
-__device__ __forceinline__ void floyd_row(uint32_t* bm, uint32_t* draws, uint32_t row, int64_t D, int64_t k, uint32_t c2,
+__device__ __forceinline__ void floyd_row(uint32_t* bm, uint32_t* draws, uint32_t row, uint32_t D, uint32_t k, uint32_t c2,
                                           uint32_t c3, const PhiloxKeys& ks, int lane) {
-  const uint32_t first_j = (uint32_t)(D - k);       // step i falls back on column first_j + i
-  for (int64_t c = lane; 4 * c < k; c += 32) {
+  const uint32_t first_j = D - k;                   // step i falls back on column first_j + i
+  for (uint32_t c = lane; 4 * c < k; c += 32) {
     uint32_t w[4];
-    philox4x32_10((uint32_t)c, row, c2, c3, ks, w);
+    philox4x32_10(c, row, c2, c3, ks, w);
 #pragma unroll
     for (int jj = 0; jj < 4; ++jj) {
-      const int64_t i = 4 * c + jj;
-      if (i < k) draws[i] = __umulhi(w[jj], first_j + (uint32_t)i + 1u);
+      const uint32_t i = 4 * c + jj;
+      if (i < k) draws[i] = __umulhi(w[jj], first_j + i + 1u);
     }
   }
   __syncwarp();
-  for (int64_t i0 = 0; i0 < k; i0 += 32) {
-    const int64_t i = i0 + lane;
+  const uint32_t below = (1u << lane) - 1u;
+#pragma unroll 1
+  for (uint32_t i0 = 0; i0 < k; i0 += 32) {
+    const uint32_t i = i0 + lane;
     const bool active = i < k;
-    const uint32_t t = active ? draws[i] : 0xffffffffu - (uint32_t)lane;      // idle lanes match nobody
-    const uint32_t j = first_j + (uint32_t)i;
-    const bool in_before = active && ((bm[t >> 5] >> (t & 31)) & 1u) != 0;
-    const uint32_t same = __match_any_sync(0xffffffffu, t);
-    bool coll = active && (in_before || (same & ((1u << lane) - 1u)) != 0);
-    // a draw equal to the fall-back column of an earlier step of this group is a collision iff that step collided
-    const uint32_t m_lane = t - first_j - (uint32_t)i0;                        // wraps to a large number when t < first_j + i0
-    const bool dep = active && !coll && m_lane < (uint32_t)lane;
-    for (int it = 0; it < 32; ++it) {
-      const uint32_t cm = __ballot_sync(0xffffffffu, coll);
-      const bool now = dep && ((cm >> (m_lane & 31)) & 1u) != 0;
-      if (!__any_sync(0xffffffffu, now && !coll)) break;
-      coll = coll || now;
+    const uint32_t t = active ? draws[i] : 0u;
+    const uint32_t bit = 1u << (t & 31);
+    // in the set after the groups before this one?
+    const bool in_before = active && (bm[t >> 5] & bit) != 0;
+    __syncwarp();
+    // Every draw that is not in yet goes in now.  Two steps of the group with the same draw are rare; one of
+    // them finds the bit already set, and only then the group is matched to tell which step came first.
+    const bool fresh = active && !in_before;
+    const bool lost = fresh && (atomicOr(&bm[t >> 5], bit) & bit) != 0;
+    bool coll = in_before;
+    if (__any_sync(0xffffffffu, lost)) {
+      const uint32_t same = __match_any_sync(0xffffffffu, fresh ? t : 0xffffffffu - (uint32_t)lane);
+      coll = coll || (fresh && (same & below) != 0);
     }
-    if (active) {
-      const uint32_t pick = coll ? j : t;
-      atomicOr(&bm[pick >> 5], 1u << (pick & 31));
+    // a draw equal to the fall-back column of an earlier step of this group is a collision iff that step
+    // collided (its bit is then set twice, which is harmless); settled by iterating to a fixed point
+    const uint32_t m_lane = t - first_j - i0;       // wraps to a large number when t < first_j + i0
+    const bool dep = active && !coll && m_lane < (uint32_t)lane;
+    if (__any_sync(0xffffffffu, dep)) {
+      for (int it = 0; it < 32; ++it) {
+        const uint32_t cm = __ballot_sync(0xffffffffu, coll);
+        const bool now = dep && ((cm >> (m_lane & 31)) & 1u) != 0;
+        if (!__any_sync(0xffffffffu, now && !coll)) break;
+        coll = coll || now;
+      }
+    }
+    if (coll) {
+      const uint32_t j = first_j + i;
+      atomicOr(&bm[j >> 5], 1u << (j & 31));
     }
     __syncwarp();
   }
@@ -101,7 +115,7 @@ __global__ void __launch_bounds__(32 * kRowsWarps) rows_fixed_kernel(const RowsP
     for (int64_t row = (int64_t)blockIdx.x * kRowsWarps + warp; row < p.B; row += (int64_t)gridDim.x * kRowsWarps) {
       for (int i = lane; i < p.words; i += 32) bm[i] = 0;
       __syncwarp();
-      floyd_row(bm, draws, (uint32_t)row, p.D, p.k, p.c2, p.c3, ks, lane);
+      floyd_row(bm, draws, (uint32_t)row, (uint32_t)p.D, (uint32_t)p.k, p.c2, p.c3, ks, lane);
       // ascending list: a lane takes a run of consecutive words, so its kept columns are consecutive in the list
       const int per_lane = (p.words + 31) / 32;
       const int w0 = lane * per_lane, w1 = min(w0 + per_lane, p.words);
@@ -146,7 +160,7 @@ __global__ void __launch_bounds__(32 * kRowsWarps) rows_fixed_kernel(const RowsP
         const int64_t row = slab * kTileRows + r;
         for (int i = lane; i < p.words; i += 32) bm[i] = 0;
         __syncwarp();
-        if (row < p.B) floyd_row(bm, draws, (uint32_t)row, p.D, p.k, p.c2, p.c3, ks, lane);
+        if (row < p.B) floyd_row(bm, draws, (uint32_t)row, (uint32_t)p.D, (uint32_t)p.k, p.c2, p.c3, ks, lane);
         // the row's words go to their tiles (word 4 r + w of tile slab * ncb + block), four words at a time
         for (int cb = lane; cb < p.ncb; cb += 32) {
           uint32_t q[4];
