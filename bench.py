@@ -436,15 +436,33 @@ def kernel_sweep(rad, torch, A, dZ, H, ps, pk, clock):
         row = dict(variant=variant, law=law, p=p, draws_per_row=rad.rad_draws_per_row(p, D), nnz=int(nnz[0]),
                    store_ms=round(ms_store, 4), store_sm_mhz=mhz, dW_ms=round(ms_dw, 4))
         if variant == "different":
-            # the multiplicity matrix (a byte per entry) is written and read once on top of the store's bytes
-            sb = store_bytes_different(B, D, int(nnz[1]), len(st.offsets), extra=2 * B * D)
+            # with replacement: the multiplicity matrix (a byte per entry) is written and read once on top of the
+            # store's bytes; the fixed-count law makes its index from the key alone and needs no such matrix
+            sb = store_bytes_different(B, D, int(nnz[1]), len(st.offsets), extra=2 * B * D if law == "replace" else 0)
             row.update(store_bytes=sb, store_gbs=round(sb / ms_store / 1e6, 1), store_frac_hbm=frac(sb / ms_store / 1e6, hbm),
+                       held_bytes=int(nnz[1]) * 2 + (len(st.keepbits) + len(st.offsets)) * 4,
                        dW_tflops_dense_tile=round(2.0 * B * D * H / ms_dw / 1e9, 1),
                        dW_useful_tflops=round(2.0 * int(nnz[0]) * H / ms_dw / 1e9, 1))
         else:
             row.update(dW_tflops_kept_columns=round(2.0 * B * int(nnz[0]) * H / ms_dw / 1e9, 1))
         rows.append(row)
         del st, ws
+    # the fixed-count law in its static-shape form: B x k values and B x k 16-bit column numbers (k the same for
+    # every row); the weight gradient rebuilds the tile-major index from the key and moves the values into it
+    p = 0.1
+    st = rad.Store("rows", "bf16", B, D, p, relu_bits=False, law="fixed")
+    ms_store, mhz = timed_alone(torch, lambda: rad.rad_linear_forward_store(A, st, status), clock, n=10)
+    ws = torch.empty(max(rad.rad_weight_grad_workspace(st, H), 256), dtype=torch.uint8, device="cuda")
+    ms_dw, _ = timed_alone(torch, lambda: rad.rad_linear_weight_grad(st, dZ, dW, ws, status), clock, n=3, settle_ms=20.0)
+    k, ld = rad.rad_draws_per_row(p, D), int(st.c.values_ld)
+    # bytes: the 32-byte sectors of A that hold a kept column (about 1 - (1 - k/D)^16 of them), values and columns written
+    touched = int(B * D * 2 * (1.0 - (1.0 - k / D) ** 16)) + B * ld * 4
+    rows.append(dict(variant="rows", law="fixed", p=p, kept_per_row=k, store_ms=round(ms_store, 4), store_sm_mhz=mhz,
+                     store_bytes_touched=touched, store_gbs=round(touched / ms_store / 1e6, 1),
+                     store_frac_hbm=frac(touched / ms_store / 1e6, hbm), held_bytes=B * ld * 4,
+                     dW_ms=round(ms_dw, 4), dW_tflops_dense_tile=round(2.0 * B * D * H / ms_dw / 1e9, 1),
+                     dW_useful_tflops=round(2.0 * B * k * H / ms_dw / 1e9, 1)))
+    del st, ws
     # random projection (P = R R^T, Rademacher signs, k = ceil(0.1 D) columns): the store is one dense GEMM,
     # the weight gradient two; TFLOP/s on the flops of those contractions (2 B D k; 2 B k H + 2 D k H)
     p = 0.1
