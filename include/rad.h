@@ -466,6 +466,19 @@ typedef struct rad_cnn_desc {
   uint64_t seed;
 } rad_cnn_desc;
 
+/*
+ * Which kernels the 3x3 convolutions of rad_cnn_step run (same operation either way; Fig. "Convnet activation
+ * sampling").  The tensor-core kernels compute the forward convolution and the filter gradient as implicit
+ * GEMMs (bf16; Cin 16, 32 or 64; Cout a multiple of 8 up to 64); the CUDA-core kernels take every shape.
+ * RAD_CONV_KERNEL_AUTO uses the tensor cores wherever the shape allows, RAD_CONV_KERNEL_SIMT never does;
+ * RAD_CONV_KERNEL_TENSOR is the same as AUTO (shapes the tensor-core kernels cannot take still run on CUDA
+ * cores).  Host only, process-wide.  Returns the previous setting, or RAD_EINVAL.
+ */
+#define RAD_CONV_KERNEL_AUTO   0
+#define RAD_CONV_KERNEL_SIMT   1
+#define RAD_CONV_KERNEL_TENSOR 2
+int rad_set_conv_kernel(int32_t which);
+
 int rad_cnn_workspace(const rad_cnn_desc* net /* host */, int64_t* bytes /* host */,
                       rad_step_stats* stats /* host or NULL */);
 int rad_cnn_step(const rad_cnn_desc* net /* host */, const void* X, const int32_t* labels,

@@ -73,7 +73,7 @@ EXPORTS = ["rad_keep_threshold", "rad_effective_p", "rad_scale", "rad_store_size
            "rad_linear_forward_store", "rad_linear_forward_store_static", "rad_weight_grad_workspace", "rad_linear_weight_grad",
            "rad_linear_forward", "rad_store_index", "rad_linear_forward_fill", "rad_softmax_xent", "rad_input_grad_workspace", "rad_linear_input_grad",
            "rad_mlp_workspace", "rad_mlp_held_bytes", "rad_mlp_step", "rad_irnn_workspace", "rad_irnn_step", "rad_cnn_workspace", "rad_cnn_step", "rad_launch_count", "rad_strerror", "rad_version",
-           "rad_set_wait_limit_ns", "rad_wait_probe"]
+           "rad_set_wait_limit_ns", "rad_wait_probe", "rad_set_conv_kernel"]
 
 _lib = None
 
@@ -97,6 +97,7 @@ def lib():
         L.rad_launch_count.restype = C.c_int64
         i32, i64, f32, vp = C.c_int32, C.c_int64, C.c_float, C.c_void_p
         L.rad_set_store_kernel.argtypes = [i32]
+        L.rad_set_conv_kernel.argtypes = [i32]
         L.rad_draws_per_row.restype = i64
         L.rad_draws_per_row.argtypes = [f32, i64]
         L.rad_replace_scale.restype = f32
@@ -249,6 +250,17 @@ def rad_set_store_kernel(which):
     if prev < 0:
         _check(prev, "rad_set_store_kernel")
     return {v: k for k, v in STORE_KERNELS.items()}[prev]
+
+
+CONV_KERNELS = {"auto": 0, "simt": 1, "tensor": 2}
+
+
+def rad_set_conv_kernel(which):
+    """Selects the kernels of the 3x3 convolutions ("auto", "simt", "tensor"); returns the previous name."""
+    prev = lib().rad_set_conv_kernel(CONV_KERNELS[which])
+    if prev < 0:
+        _check(prev, "rad_set_conv_kernel")
+    return {v: k for k, v in CONV_KERNELS.items()}[prev]
 
 
 STATIC_STORE_MAX_TILES = 131072

@@ -8,7 +8,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(PKG, "_build")
 LIB = os.path.join(PKG, "librad_b200.so")
-SOURCES = ["store.cu", "store_pipe.cu", "store_index.cu", "store_rows.cu", "project.cu", "simt.cu", "loss.cu", "tc.cu", "irnn.cu", "conv.cu", "cnn.cu", "api.cu"]
+SOURCES = ["store.cu", "store_pipe.cu", "store_index.cu", "store_rows.cu", "project.cu", "simt.cu", "loss.cu", "tc.cu", "irnn.cu", "conv.cu", "conv_tc.cu", "cnn.cu", "api.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall", "--expt-relaxed-constexpr"]
 

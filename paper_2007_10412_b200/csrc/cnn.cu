@@ -64,6 +64,7 @@ int make_cnn_plan(const rad_cnn_desc* d, CnnPlan* pl) {
     max_conv_out = std::max<int64_t>(max_conv_out, (int64_t)h * w * co);
     max_act = std::max<int64_t>(max_act, (int64_t)h * w * c);
     scratch = std::max(scratch, conv_weight_grad_workspace(B, c, co));
+    scratch = std::max(scratch, conv_tc_weight_grad_workspace(B, h, w, c, co));
     scratch = std::max(scratch, column_sums_workspace(B * h * w, co));
     h /= 2; w /= 2; c = co;
     max_act = std::max<int64_t>(max_act, (int64_t)h * w * c);
@@ -154,8 +155,14 @@ extern "C" int rad_cnn_step(const rad_cnn_desc* d, const void* X, const int32_t*
     rc = rad_linear_forward_store(a_in, st[l].D, &st[l], ws + pl.scratch, pl.scratch_bytes, dev_status, stream);
     if (rc != RAD_OK) return rc;
     void* a_out = ws + pl.act[l & 1];
-    rc = conv_forward_pool(d->dtype, B, pl.H[l], pl.W[l], pl.Cin[l], pl.Cout[l], a_in, conv_W[l],
-                           conv_b != nullptr ? conv_b[l] : nullptr, a_out, reinterpret_cast<uint32_t*>(ws + pl.relubits[l]), s);
+    // tensor cores where the shape allows (Cin 16 / 32 / 64: the later convolutions), CUDA cores otherwise
+    if (conv_tc_ok(d->dtype, pl.H[l], pl.W[l], pl.Cin[l], pl.Cout[l], a_in, conv_W[l]))
+      rc = conv_tc_forward_pool(B, pl.H[l], pl.W[l], pl.Cin[l], pl.Cout[l], a_in, conv_W[l],
+                                conv_b != nullptr ? conv_b[l] : nullptr, a_out, reinterpret_cast<uint32_t*>(ws + pl.relubits[l]),
+                                dev_status, s);
+    else
+      rc = conv_forward_pool(d->dtype, B, pl.H[l], pl.W[l], pl.Cin[l], pl.Cout[l], a_in, conv_W[l],
+                             conv_b != nullptr ? conv_b[l] : nullptr, a_out, reinterpret_cast<uint32_t*>(ws + pl.relubits[l]), s);
     if (rc != RAD_OK) return rc;
     a_in = a_out;
   }
@@ -200,8 +207,12 @@ extern "C" int rad_cnn_step(const rad_cnn_desc* d, const void* X, const int32_t*
   for (int l = pl.nc - 1; l >= 0; --l) {
     rc = conv_dz(d->dtype, B, pl.H[l], pl.W[l], pl.Cout[l], g, reinterpret_cast<const uint32_t*>(ws + pl.relubits[l]), dz, s);
     if (rc != RAD_OK) return rc;
-    rc = conv_weight_grad(&st[l], pl.H[l], pl.W[l], pl.Cin[l], pl.Cout[l], dz, dconv_W[l], ws + pl.scratch,
-                          pl.scratch_bytes, s);
+    if (conv_tc_ok(d->dtype, pl.H[l], pl.W[l], pl.Cin[l], pl.Cout[l], dz, conv_W[l]))
+      rc = conv_tc_weight_grad(&st[l], pl.H[l], pl.W[l], pl.Cin[l], pl.Cout[l], dz, dconv_W[l], ws + pl.scratch,
+                               pl.scratch_bytes, dev_status, s);
+    else
+      rc = conv_weight_grad(&st[l], pl.H[l], pl.W[l], pl.Cin[l], pl.Cout[l], dz, dconv_W[l], ws + pl.scratch,
+                            pl.scratch_bytes, s);
     if (rc != RAD_OK) return rc;
     rc = column_sums(d->dtype, B * pl.H[l] * pl.W[l], pl.Cout[l], dz, pl.Cout[l], dconv_b[l], ws + pl.scratch,
                      pl.scratch_bytes, s);

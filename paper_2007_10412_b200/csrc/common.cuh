@@ -210,6 +210,14 @@ int64_t conv_weight_grad_workspace(int64_t B, int Cin, int Cout);
 int conv_weight_grad(const rad_store* store, int H, int W, int Cin, int Cout, const void* dZ, float* dW, void* workspace,
                      int64_t workspace_bytes, cudaStream_t st);
 
+// 3x3 convolutions on the tensor cores (conv_tc.cu)
+bool conv_tc_ok(int dtype, int H, int W, int Cin, int Cout, const void* X, const void* Wt);
+int conv_tc_forward_pool(int64_t B, int H, int W, int Cin, int Cout, const void* X, const void* Wt, const float* bias, void* P,
+                         uint32_t* relubits, int32_t* dev_status, cudaStream_t st);
+int64_t conv_tc_weight_grad_workspace(int64_t B, int H, int W, int Cin, int Cout);
+int conv_tc_weight_grad(const rad_store* store, int H, int W, int Cin, int Cout, const void* dZ, float* dW, void* workspace,
+                        int64_t workspace_bytes, int32_t* dev_status, cudaStream_t st);
+
 // tcgen05 kernels (bf16, aligned)
 bool tc_shape_ok(int64_t B, int64_t D, int64_t H, const void* p0, int64_t ld0, const void* p1,
                  int64_t ld1);
