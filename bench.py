@@ -531,6 +531,23 @@ def small_workloads(rad, torch):
     memory(ctx, r)
     assert ctx.dev_status.item() == 0
     out["cnn_32x32x3_c16_32_64_fc128_10_b128_bf16_different"] = r
+    # the same net with the convolutions of blocks 2 and 3 on CUDA cores instead of tensor cores, and both at a
+    # batch large enough to leave the launch-bound regime
+    conv = {}
+    for batch in (128, 4096):
+        Xb, yb, _, _, _, _ = cnn_inputs(batch, 32, 3, (16, 32, 64), (128, 10), "bf16", 1234)
+        bargs = (bf(Xb), dev(yb)) + cargs[2:]
+        for kern in ("tensor", "simt"):
+            prev = rad.rad_set_conv_kernel(kern)
+            try:
+                c2 = rad.CNNStep(batch, 32, 3, (16, 32, 64), (128, 10), "bf16", "different", 0.1)
+                rr = rate(lambda i=0: c2(*bargs, seed=0, step=i), batch, 10)
+                assert c2.dev_status.item() == 0
+            finally:
+                rad.rad_set_conv_kernel(prev)
+            conv[f"b{batch}_{kern}"] = dict(ms_per_step=rr["ms_per_step"], samples_per_s=rr["samples_per_s"])
+            del c2
+    out["cnn_32x32x3_c16_32_64_fc128_10_b128_bf16_different"]["conv_kernels"] = conv
     return out
 
 
