@@ -690,8 +690,11 @@ def run_ours(args):
     # DRAM bytes per launch from the ncu captures under profiles/ (batch 8192, 8192 x 8192 layer): bytes read grow
     # with the batch and are scaled by B / 8192, the dW output does not grow.  Only the default workload has one.
     traffic = None
-    if args.act == "gelu" and abs(args.p - 0.1) < 1e-9 and args.law == "bernoulli" and not fused:
-        traffic = int((1095.8e6 + 251.4e6) * B / 8192) if dominant != "dW" else None
+    if args.act == "gelu" and abs(args.p - 0.1) < 1e-9 and args.law == "bernoulli" and args.variant == "different":
+        if dominant == "forward":
+            traffic = int((1080.2e6 + 263.0e6) * B / 8192)
+        elif dominant == "dW":
+            traffic = int(631.7e6 * B / 8192 + 236.0e6)
     roofline = dict(bound=dom["bound"], kernel=dom["kernel"], achieved=dom["achieved"], peak=dom["peak"], unit=dom["unit"],
                     frac=dom["frac"], traffic=traffic, peak_source=pk["source"] + " (sustained cuBLAS bf16 / copy bandwidth)",
                     ms_per_launch=dom["ms_per_launch"],
