@@ -33,7 +33,7 @@ constexpr int BM = 256, BN = 256, BK = 64;
 constexpr int kHalfM = 128;
 constexpr int kNumSMsDefault = 148;
 constexpr int kMaxSplits = 16;
-constexpr int kRasterGroup = 8;                // m-tiles per raster group
+constexpr int kRasterGroup = 16;               // m-tiles per raster group (16 x 4 MB of A panels stay in L2 beside the B panels in flight)
 
 enum AKind { kAK = 0, kAMN = 1, kASparse = 2 };
 enum BKind { kBK_ = 0, kBMN = 1 };
