@@ -53,6 +53,8 @@ def parse_args():
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-kernel p sweep")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     ap.add_argument("--no-twin", action="store_true", help="skip the timed ReLU twin of the wide net")
+    ap.add_argument("--small-only", action="store_true",
+                    help="run only the small workloads (MNIST-shaped MLP, IRNN, CNN) and print their figures")
     return ap.parse_args()
 
 
@@ -827,9 +829,21 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_small_only():
+    import torch
+    import paper_2007_10412_b200 as rad
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    print(json.dumps(dict(small_workloads=small_workloads(rad, torch))))
+
+
 def main():
     args = parse_args()
-    if args.impl == "reference":
+    if args.small_only:
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_small_only()
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
