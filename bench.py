@@ -279,7 +279,7 @@ class LayerwiseStep:
         a_in = X
         # different-sample Bernoulli stores of hidden layers come out of the producing GEMM's epilogue; their
         # index part (key only) is timed with the store family, the GEMM with the forward family
-        fused = self.variant == "different" and self.law == "bernoulli"
+        fused = self.variant == "different" and self.law in ("bernoulli", "fixed")
         for l in range(L):
             self.stores[l].c.seed, self.stores[l].c.step = seed, step
         st0 = self.stores[0]
@@ -633,7 +633,7 @@ def run_ours(args):
         return sum(t) / len(t) if t else None
 
     big = lambda l: dims[l] == 8192 and dims[l + 1] == 8192
-    fused = args.variant == "different" and args.law == "bernoulli"
+    fused = args.variant == "different" and args.law in ("bernoulli", "fixed")
     ms_fwd, ms_dw, ms_dx = mean_ms("forward", big), mean_ms("dW", big), mean_ms("dX+db", lambda l: big(l) and l > 0)
     ms_store0 = mean_ms("store", lambda l: l == 0)
     ms_store_hidden = mean_ms("store", lambda l: l > 0)      # fused: the key-only index kernels; else full stores
@@ -661,7 +661,7 @@ def run_ours(args):
         kernels["store"] = dict(kernel="store of the network input (stand-alone kernel)", bound="hbm", ms_per_launch=round(ms_store0, 4),
                                 achieved=round(sb / ms_store0 / 1e6, 1), unit="GB/s", peak=hbm, frac=round(sb / ms_store0 / 1e6 / hbm, 4),
                                 algorithmic_bytes=sb)
-        if fused:
+        if fused and args.law == "bernoulli":
             calls = 3.0 * B * 8192 / 32
             mhz = clocks.get("sm_mhz") or pk["sm_max_mhz"]
             peak_calls = PHILOX_GCALLS_AT_MAX_CLOCK * mhz / pk["sm_max_mhz"]

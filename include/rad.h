@@ -300,7 +300,7 @@ int rad_linear_forward(int32_t dtype, int32_t act, int64_t B, int64_t D, int64_t
  * words and in-tile row offsets), offsets and nnz of `st` can be written before the layer input exists: no
  * input is read.  A caller can size `values` exactly from nnz[1] (read it back after the stream has
  * reached this point), and rad_linear_forward_fill can then place the kept values from the epilogue of the
- * GEMM that produces the input.  Bernoulli keeps only (RAD_EUNSUPPORTED otherwise); st->values may be NULL
+ * GEMM that produces the input.  Bernoulli keeps and the fixed-count law (RAD_EUNSUPPORTED otherwise); st->values may be NULL
  * (no capacity check) and st->relubits is not touched.  Bits and layout are those of
  * rad_linear_forward_store.
  */
@@ -314,7 +314,8 @@ int rad_store_index(const rad_store* st /* host */, int32_t* dev_status /* devic
  * epilogue that holds a row of activations drops the kept ones into next->values at the places the index
  * part of `next` gives.  index_ready != 0: the caller has already run rad_store_index on `next` with the
  * same key; 0: this call runs it first.  next->relubits is ignored (the bits of out_act go to `relubits`).
- * Shapes the fused kernel does not take (f32, unaligned or tiny layers, same-sample, other laws) run the
+ * Different-sample stores under the Bernoulli or the fixed-count law are filled this way; shapes the fused
+ * kernel does not take (f32, unaligned or tiny layers, same-sample, the with-replacement law) run the
  * two separate calls instead; `workspace` (device, rad_store_sizes.workspace_bytes of `next`) is used only
  * then.
  */

@@ -260,6 +260,24 @@ extern "C" int rad_linear_forward(int32_t dtype, int32_t act, int64_t B, int64_t
                       ld_zlow, relubits, s);
 }
 
+namespace rad {
+namespace {
+// Whether the forward GEMM can fill `next` from its epilogue: tensor-core shapes, a different-sample store under a
+// law whose index can be made from the key alone.
+bool fill_can_fuse(int dtype, int64_t B, int64_t D, int64_t H, const void* A, int64_t lda, const void* W, int64_t ldw,
+                   const float* bias, const void* out_act, int64_t ld_act, const void* out_zlow, int64_t ld_zlow,
+                   const rad_store* next) {
+  return dtype == RAD_BF16 && next->variant == RAD_DIFFERENT_SAMPLE &&
+         (next->law == RAD_LAW_BERNOULLI || (next->law == RAD_LAW_FIXED && H <= 65536)) && store_args_ok(next) &&
+         tc_shape_ok(B, D, H, A, lda, W, ldw) && ((uintptr_t)bias & 15) == 0 && ((uintptr_t)out_act & 15) == 0 &&
+         ld_act % 8 == 0 && ((uintptr_t)next->keepbits & 15) == 0 &&
+         (out_zlow == nullptr || (((uintptr_t)out_zlow & 15) == 0 && ld_zlow % 8 == 0)) &&
+         (double)B * (double)H < 4294967296.0 * 0.75;
+}
+
+}  // namespace
+}  // namespace rad
+
 extern "C" int rad_linear_forward_fill(int32_t dtype, int32_t act, int64_t B, int64_t D, int64_t H, const void* A,
                                        int64_t lda, const void* W, int64_t ldw, const float* bias, void* out_act,
                                        int64_t ld_act, void* out_zlow, int64_t ld_zlow, uint32_t* relubits,
@@ -273,19 +291,15 @@ extern "C" int rad_linear_forward_fill(int32_t dtype, int32_t act, int64_t B, in
   int rc = check_device();
   if (rc != RAD_OK) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const bool fused = dtype == RAD_BF16 && next->variant == RAD_DIFFERENT_SAMPLE && next->law == RAD_LAW_BERNOULLI &&
-                     store_args_ok(next) && tc_shape_ok(B, D, H, A, lda, W, ldw) && ((uintptr_t)bias & 15) == 0 &&
-                     ((uintptr_t)out_act & 15) == 0 && ld_act % 8 == 0 && ((uintptr_t)next->keepbits & 15) == 0 &&
-                     (out_zlow == nullptr || (((uintptr_t)out_zlow & 15) == 0 && ld_zlow % 8 == 0)) &&
-                     (double)B * (double)H < 4294967296.0 * 0.75;
-  if (fused) {
-    if (!index_ready) {
-      rc = launch_store_index(next, true, dev_status, s);
-      if (rc != RAD_OK) return rc;
-    }
+  bool fused = fill_can_fuse(dtype, B, D, H, A, lda, W, ldw, bias, out_act, ld_act, out_zlow, ld_zlow, next);
+  if (fused && !index_ready) {
+    rc = launch_store_index(next, true, dev_status, s);
+    if (rc == RAD_EUNSUPPORTED) fused = false;        // rows too long for the fixed-count index: the separate calls below
+    else if (rc != RAD_OK) return rc;
+  }
+  if (fused)
     return tc_forward(act, B, D, H, A, lda, W, ldw, bias, out_act, ld_act, nullptr, 0, out_zlow, ld_zlow, relubits,
                       dev_status, s, next);
-  }
   // shapes the fused epilogue does not take: the same results from the two separate calls
   rc = rad_linear_forward(dtype, act, B, D, H, A, lda, W, ldw, bias, out_act, ld_act, nullptr, 0, out_zlow, ld_zlow,
                           relubits, dev_status, stream);
@@ -405,8 +419,8 @@ extern "C" int rad_mlp_step(const rad_mlp_desc* net, const void* X, const int32_
     void* zlow = net->act == RAD_ACT_GELU ? ws + plan.layer[l + 1].preact : nullptr;
     uint32_t* rbits = plan.layer[l + 1].relubits >= 0 ? reinterpret_cast<uint32_t*>(ws + plan.layer[l + 1].relubits) : nullptr;
     rc = rad_linear_forward_fill(net->dtype, net->act, B, D, H, a_in, ld_in, W[l], H, b != nullptr ? b[l] : nullptr,
-                                 a_out, H, zlow, H, rbits, &st[l + 1], 0, ws + plan.scratch, plan.scratch_bytes,
-                                 dev_status, stream);
+                                 a_out, H, zlow, H, rbits, &st[l + 1], 0, ws + plan.scratch,
+                                 plan.scratch_bytes, dev_status, stream);
     if (rc != RAD_OK) return rc;
     a_in = a_out;
     ld_in = H;

@@ -1203,7 +1203,8 @@ int tc_forward(int act, int64_t B, int64_t D, int64_t H, const void* A, int64_t 
       return RAD_EINVAL;
     p.st_values = static_cast<bf16*>(next->values); p.st_keepbits = next->keepbits; p.st_offsets = next->offsets;
     p.st_capacity = next->values_capacity; p.st_ncb = (int32_t)ceil_div(H, kTileCols);
-    p.st_scale = (float)kLaneRange / (float)keep_threshold_host(next->p);
+    p.st_scale = next->law == RAD_LAW_FIXED ? (float)H / (float)draws_per_row_host(next->p, H)
+                                            : (float)kLaneRange / (float)keep_threshold_host(next->p);
   }
   return launch_pair<kAK, kBMN, kFwd>(p, ta, tb, ceil_div(B, BM) * ceil_div(H, BN), s);
 }

@@ -105,6 +105,13 @@ def test_fused_store_matches_the_oracle_store_of_the_written_activations(B, D, H
     _check_fill(B, D, H, "bf16", act, "different", p)
 
 
+@pytest.mark.parametrize("f", [0.1, 0.5])
+def test_fused_store_under_the_fixed_count_law(f):
+    """Exactly k columns per row: the index of that law also comes from the key alone, so the same epilogue fills it."""
+    _check_fill(328, 640, 520, "bf16", "relu", "different", f, law="fixed")
+    _check_fill(200, 128, 1160, "bf16", "gelu", "different", f, law="fixed", index_ready=True, relu=False)
+
+
 def test_fused_store_with_the_index_made_beforehand():
     _check_fill(520, 384, 648, "bf16", "gelu", "different", 0.2, index_ready=True, relu=False)
 
