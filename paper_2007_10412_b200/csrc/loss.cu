@@ -31,6 +31,46 @@ __global__ void __launch_bounds__(256) xent_rows_kernel(const float* logits, int
   if (lane == 0) row_loss[b] = (y >= 0 && y < C) ? (logf(sum) + mx - z[y]) : 0.0f;
 }
 
+// Rows and mean in one launch for small batches (the small nets are bound by their launch count): one CTA, a
+// warp takes rows w, w + 32, ..., then the same fixed-order mean as below over the row losses in shared memory.
+constexpr int kXentSmallRows = 2048;
+template <typename T>
+__global__ void __launch_bounds__(1024) xent_small_kernel(const float* logits, int64_t ldl, const int32_t* labels, int64_t B,
+                                                          int64_t C, T* dZ, int64_t ldz, float* loss) {
+  __shared__ float s_row[kXentSmallRows];
+  __shared__ float s[1024];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int64_t b = warp; b < B; b += 32) {
+    const float* z = logits + b * ldl;
+    float mx = -INFINITY;
+    for (int64_t c = lane; c < C; c += 32) mx = fmaxf(mx, z[c]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float sum = 0.0f;
+    for (int64_t c = lane; c < C; c += 32) sum += expf(z[c] - mx);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    const int32_t y = labels[b];
+    const float inv = 1.0f / sum, invB = 1.0f / (float)B;
+    for (int64_t c = lane; c < C; c += 32) {
+      float g = expf(z[c] - mx) * inv;
+      if (c == y) g -= 1.0f;
+      dZ[b * ldz + c] = from_float<T>(g * invB);
+    }
+    if (lane == 0) s_row[b] = (y >= 0 && y < C) ? (logf(sum) + mx - z[y]) : 0.0f;
+  }
+  __syncthreads();
+  float acc = 0.0f;
+  for (int64_t i = threadIdx.x; i < B; i += 1024) acc += s_row[i];
+  s[threadIdx.x] = acc;
+  __syncthreads();
+  for (int o = 512; o > 0; o >>= 1) {
+    if ((int)threadIdx.x < o) s[threadIdx.x] += s[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *loss = s[0] / (float)B;
+}
+
 // Fixed-order mean of the per-row losses (one CTA).
 __global__ void __launch_bounds__(1024) mean_kernel(const float* row_loss, int64_t B, float* loss) {
   __shared__ float s[1024];
@@ -61,6 +101,15 @@ extern "C" int rad_softmax_xent(int32_t dtype, int64_t B, int64_t C, const float
   int rc = check_device();
   if (rc != RAD_OK) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (B <= kXentSmallRows) {
+    count_launch();
+    if (dtype == RAD_BF16)
+      xent_small_kernel<bf16><<<1, 1024, 0, s>>>(logits, ldl, labels, B, C, static_cast<bf16*>(dZ), ldz, loss);
+    else
+      xent_small_kernel<float><<<1, 1024, 0, s>>>(logits, ldl, labels, B, C, static_cast<float*>(dZ), ldz, loss);
+    RAD_CUDA_TRY(cudaGetLastError());
+    return RAD_OK;
+  }
   float* rows = static_cast<float*>(workspace);
   const unsigned grid = (unsigned)ceil_div(B, 8);
   count_launch(2);

@@ -245,6 +245,22 @@ __global__ void __launch_bounds__(256) colsum_final_kernel(const float* partial,
   for (int64_t c = 0; c < chunks; ++c) s += partial[c * H + h];
   db[h] = s;
 }
+// Both stages in one launch for few rows (the small nets are bound by their launch count): the same chunk sums,
+// added in the same order, by the thread that owns the column.
+constexpr int kColSmallChunks = 2;
+template <typename T>
+__global__ void __launch_bounds__(256) colsum_small_kernel(const T* dZ, int64_t ldz, int64_t B, int64_t H, float* db) {
+  const int64_t h = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (h >= H) return;
+  float total = 0.0f;
+  for (int64_t b0 = 0; b0 < B; b0 += kColChunkRows) {
+    const int64_t b1 = min(B, b0 + kColChunkRows);
+    float s = 0.0f;
+    for (int64_t b = b0; b < b1; ++b) s += to_float(dZ[b * ldz + h]);
+    total += s;
+  }
+  db[h] = total;
+}
 
 }  // namespace
 
@@ -326,6 +342,14 @@ int column_sums(int dtype, int64_t B, int64_t H, const void* dZ, int64_t ldz, fl
                 int64_t workspace_bytes, cudaStream_t s) {
   if (workspace == nullptr || workspace_bytes < column_sums_workspace(B, H)) return RAD_EWORKSPACE;
   const int64_t chunks = ceil_div(B, kColChunkRows);
+  if (chunks <= kColSmallChunks) {
+    count_launch();
+    if (dtype == RAD_BF16)
+      colsum_small_kernel<bf16><<<(unsigned)ceil_div(H, 256), 256, 0, s>>>(static_cast<const bf16*>(dZ), ldz, B, H, db);
+    else
+      colsum_small_kernel<float><<<(unsigned)ceil_div(H, 256), 256, 0, s>>>(static_cast<const float*>(dZ), ldz, B, H, db);
+    return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
+  }
   dim3 grid((unsigned)ceil_div(H, 256), (unsigned)chunks);
   float* partial = static_cast<float*>(workspace);
   count_launch(2);
