@@ -44,7 +44,7 @@ constexpr int kWarpElems = kTileElems / kWarpsPerTile;   // entries of a tile th
 template <typename T, int S>
 struct PipeSmem {
   alignas(128) T raw[S][kTileElems];            // tiles of A as loaded
-  alignas(16) T wbuf[kComputeWarps][kWarpElems + 8];   // kept values of a warp's sixteen rows, in order (from index 0 or 1)
+  alignas(16) T wbuf[kComputeWarps][kWarpElems + 8];   // kept values of a warp's sixteen rows, in order (from index 0 .. 7)
   uint64_t full[S], empty[S];                   // raw ring
   uint64_t chunk_ready[kSlots], cnt_ready[kSlots], base_ready[kSlots];
   uint32_t chunk_id[kSlots];
@@ -121,27 +121,55 @@ __device__ __forceinline__ uint32_t warp_inclusive_scan(uint32_t v, int lane) {
 __device__ __forceinline__ float raw_to_float(float v) { return v; }
 __device__ __forceinline__ float raw_to_float(bf16 v) { return __bfloat162float(v); }
 
-// Copies entries [first, end) of a warp's staging buffer to `out` (same indices), multiplied by `scale`
-// and rounded once to the working type.  out + 0 is 4-byte aligned.
-__device__ __forceinline__ void copy_scaled(const float* wb, float* out, uint32_t first, uint32_t end, float scale,
-                                            int lane) {
-  for (uint32_t i = first + lane; i < end; i += 32) out[i] = __fmul_rn(wb[i], scale);
+// One entry of the working type at a 32-bit shared-memory address.
+__device__ __forceinline__ uint32_t lds_elem(uint32_t a, const bf16*) {
+  uint16_t v;
+  asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a));
+  return v;
 }
-// bf16: two entries per lane and step (one 4-byte load, one 4-byte store); a pair that sticks out of
-// [first, end) at either end stores its inner half alone.
-__device__ __forceinline__ void copy_scaled(const bf16* wb, bf16* out, uint32_t first, uint32_t end, float scale,
-                                            int lane) {
-  const uint32_t* wb2 = reinterpret_cast<const uint32_t*>(wb);
-  for (uint32_t pr = lane; 2 * pr < end; pr += 32) {
-    const uint32_t v = wb2[pr];
-    const __nv_bfloat162 h2 = __floats2bfloat162_rn(__fmul_rn(__uint_as_float(v << 16), scale),
-                                                    __fmul_rn(__uint_as_float(v & 0xffff0000u), scale));
-    if (2 * pr >= first && 2 * pr + 1 < end) {
-      reinterpret_cast<__nv_bfloat162*>(out)[pr] = h2;
+__device__ __forceinline__ uint32_t lds_elem(uint32_t a, const float*) {
+  uint32_t v;
+  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ void sts_elem(uint32_t a, uint32_t v, const bf16*) {
+  asm volatile("st.shared.u16 [%0], %1;" ::"r"(a), "h"((uint16_t)v) : "memory");
+}
+__device__ __forceinline__ void sts_elem(uint32_t a, uint32_t v, const float*) {
+  asm volatile("st.shared.b32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t scale_pair(uint32_t v, float scale) {
+  const __nv_bfloat162 h2 = __floats2bfloat162_rn(__fmul_rn(__uint_as_float(v << 16), scale),
+                                                  __fmul_rn(__uint_as_float(v & 0xffff0000u), scale));
+  return *reinterpret_cast<const uint32_t*>(&h2);
+}
+
+// Copies entries [first, end) of a warp's staging buffer to `out` (same indices), multiplied by `scale`
+// and rounded once to the working type.  wb + 0 and out + 0 are 16-byte aligned and first < 16 bytes' worth
+// of entries: whole 16-byte vectors go as such, the entries before the first and after the last whole
+// vector one by one (lanes 0-7 and 8-15).
+template <typename T>
+__device__ __forceinline__ void copy_scaled(const T* wb, T* out, uint32_t first, uint32_t end, float scale, int lane) {
+  constexpr uint32_t kVec = 16 / sizeof(T);
+  const uint32_t v0 = first == 0 ? 0u : kVec, v1 = end & ~(kVec - 1);
+  const uint32_t head_end = min(v0, end), tail = max(v1, head_end);
+  {
+    const uint32_t i = lane < 8 ? first + lane : tail + (lane - 8);
+    const uint32_t lim = lane < 8 ? head_end : (lane < 16 ? end : 0u);
+    if (i < lim) out[i] = from_float<T>(__fmul_rn(raw_to_float(wb[i]), scale));
+  }
+  for (uint32_t i = v0 + kVec * lane; i < v1; i += 32 * kVec) {
+    uint4 q = *reinterpret_cast<const uint4*>(wb + i);
+    if constexpr (sizeof(T) == 2) {
+      q.x = scale_pair(q.x, scale); q.y = scale_pair(q.y, scale);
+      q.z = scale_pair(q.z, scale); q.w = scale_pair(q.w, scale);
     } else {
-      if (2 * pr >= first) out[2 * pr] = h2.x;
-      if (2 * pr + 1 >= first && 2 * pr + 1 < end) out[2 * pr + 1] = h2.y;
+      q.x = __float_as_uint(__fmul_rn(__uint_as_float(q.x), scale));
+      q.y = __float_as_uint(__fmul_rn(__uint_as_float(q.y), scale));
+      q.z = __float_as_uint(__fmul_rn(__uint_as_float(q.z), scale));
+      q.w = __float_as_uint(__fmul_rn(__uint_as_float(q.w), scale));
     }
+    *reinterpret_cast<uint4*>(out + i) = q;
   }
 }
 
@@ -248,19 +276,21 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
         const T* src = sm.raw[s] + r * kTileCols + half * 64;
         // Kept entries go to the warp's buffer as they are (bit h of a reversed word is column 31 - h);
         // scaling waits for the copy to `values`, where every lane has work.  The buffer is filled from
-        // index `odd` on, so that an entry's index in it and its index in `values` have the same parity.
-        // One loop serves both words: it runs as long as the fullest pair of words of the warp.
-        const uint32_t odd = wbase & 1u;
-        const T* src_end = src + 31;
-        T* dst = wb + odd + (incl - cnt);
+        // index `lead` on, so that an entry's index in it and its index in `values` agree modulo a 16-byte
+        // vector.  One loop serves both words: it runs as long as the fullest pair of words of the warp.
+        constexpr uint32_t kVec = 16 / sizeof(T), kElem = sizeof(T);
+        const uint32_t lead = wbase & (kVec - 1);
+        uint32_t sa = smem_addr(src) + 31 * kElem;          // column 31 of the word being walked
+        uint32_t da = smem_addr(wb) + (lead + incl - cnt) * kElem;
         uint32_t rev = __brev(m0), rev_next = __brev(m1);
-        if (rev == 0) { rev = rev_next; rev_next = 0; src_end += 32; }
+        if (rev == 0) { rev = rev_next; rev_next = 0; sa += 32 * kElem; }
         while (rev != 0) {
           uint32_t h;
           asm("bfind.u32 %0, %1;" : "=r"(h) : "r"(rev));
-          rev &= ~(1u << h);
-          *dst++ = *(src_end - h);
-          if (rev == 0) { rev = rev_next; rev_next = 0; src_end += 32; }
+          rev ^= 1u << h;
+          sts_elem(da, lds_elem(sa - h * kElem, src), src);
+          da += kElem;
+          if (rev == 0) { rev = rev_next; rev_next = 0; sa += 32 * kElem; }
         }
         if (p.relubits != nullptr) {
           const uint32_t row = sm.tile_slab[slot][g] * kTileRows + r;
@@ -278,9 +308,9 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
         __syncwarp();
         if (lane == 0) bar_arrive(&sm.empty[s]);   // the tile of A is not read again
         if (base >= 0) {
-          T* out = static_cast<T*>(p.values) + base + wbase - odd;   // even element index: 4-byte aligned for bf16
-          const uint32_t end = odd + wtotal;
-          copy_scaled(wb, out, odd, end, p.scale, lane);
+          T* out = static_cast<T*>(p.values) + base + wbase - lead;   // a multiple of 16 bytes from `values`
+          const uint32_t end = lead + wtotal;
+          copy_scaled(wb, out, lead, end, p.scale, lane);
           if (v == kWarpsPerTile - 1) {
             // zeros up to the next multiple of kValueAlign after the tile's last value
             const uint32_t total = wbase + wtotal;
@@ -559,6 +589,7 @@ int launch_store_pipelined(const StoreParams& p, const PhiloxKeys& ks, int dtype
   const size_t esz = dtype == RAD_BF16 ? 2 : 4;
   if (((uintptr_t)p.A & 15) != 0 || ((size_t)p.lda * esz) % 16 != 0) return RAD_EUNSUPPORTED;
   if (((uintptr_t)p.keepbits & 7) != 0) return RAD_EUNSUPPORTED;   // keep-bit words leave in pairs
+  if (((uintptr_t)p.values & 15) != 0) return RAD_EUNSUPPORTED;    // kept values leave in 16-byte vectors
   EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(tensor_map_encoder());
   if (fn == nullptr) return RAD_EUNSUPPORTED;
   CUtensorMap map;
