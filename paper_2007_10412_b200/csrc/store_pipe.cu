@@ -1,24 +1,24 @@
 // Different-sample store as a persistent, software-pipelined kernel (Sec. 3.2 / 4.2 of the paper: the
 // layer input is sampled, scaled by 1 / p_eff and only the kept entries are held).
 //
-// A CTA claims chunks of kChunk consecutive 64 x 128 tiles in ticket order and runs two phases per
-// chunk, the first phase kAhead chunks ahead of the second:
-//   phase 1  needs no data: the eight compute warps work on two tiles side by side, four warps each; a
-//            thread draws the 64 keep decisions of two adjacent keep-bit words of a row (four Philox
-//            calls, eight logic operations per word), writes the words, and the warp totals go to shared memory;
-//   look-back a service warp adds the chunk's padded and exact counts, publishes them, and finds where
-//            the chunk starts in `values` from the chunks before it (decoupled look-back over one
-//            status word per chunk);
-//   phase 2  the tile of A arrives in shared memory by TMA (a second service warp runs a ring of
-//            loads ahead of the compute warps); a warp scan over the counts gives every word its
-//            place in (row, column) order; each thread walks the set bits of its two words and copies
-//            the kept entries into its warp's staging buffer, which the warp then writes to `values`
-//            with coalesced stores, scaling on the way.  No compute warp waits for another one in
-//            this phase.
-// The look-back of a chunk therefore has kAhead chunk periods to finish in.
+// A CTA claims chunks of kChunk consecutive 64 x 128 tiles in ticket order.  Its warps have four roles:
+//   drawing    four warps that need no data: a thread draws the 64 keep decisions of two adjacent keep-bit
+//              words of a row (six Philox calls), writes the words to `keepbits`, and the warp's kept count
+//              per tile goes to shared memory.  They run kAhead + 1 chunks ahead of the loads, and their
+//              multiplies fill the issue slots that the other warps leave while they wait for memory;
+//   look-back  one warp adds the chunk's padded and exact counts, publishes them, and finds where the chunk
+//              starts in `values` from the chunks before it (decoupled look-back over one status word per
+//              chunk);
+//   loader     one warp claims chunks and runs a ring of TMA loads of the tiles of A;
+//   compaction eight warps, two tiles side by side, four warps each: a thread reads its two words back, a
+//              warp scan over the counts gives every word its place in (row, column) order; each thread
+//              walks the set bits of its two words and copies the kept entries into its warp's staging
+//              buffer, which the warp then writes to `values` in 16-byte vectors, scaling on the way.  No
+//              compaction warp waits for another one.
+// The look-back of a chunk has about kAhead chunk periods to finish in.
 // The layout produced is the one of the generic kernel: the order of tiles in `values` is the tile index.
 //
-// Every wait is bounded (2 s on the global timer).  On expiry the CTA raises RAD_DEV_ETIMEOUT, all
+// Every wait is bounded (a kernel argument, 2 s on the global timer unless the caller sets it).  On expiry the CTA raises RAD_DEV_ETIMEOUT, all
 // roles leave their loops, outstanding loads are waited for, and the kernel returns.
 #include <cuda.h>
 
@@ -32,8 +32,9 @@ constexpr int kChunk = 8;                       // tiles per claimed chunk
 constexpr int kComputeWarps = 8;
 constexpr int kWarpsPerTile = 4;                // 128 threads per tile: two keep-bit words (64 columns of a row) each
 constexpr int kTilesPerStep = kComputeWarps / kWarpsPerTile;   // tiles the compute warps work on side by side
-constexpr int kLoaderWarp = kComputeWarps;      // the look-back warp is the last one
-constexpr int kPipeThreads = (kComputeWarps + 2) * 32;
+constexpr int kDrawWarps = kWarpsPerTile;       // one per quarter of a tile
+constexpr int kLoaderWarp = kComputeWarps + kDrawWarps;   // the look-back warp is the last one
+constexpr int kPipeThreads = (kComputeWarps + kDrawWarps + 2) * 32;
 constexpr int kAhead = 2;                       // chunks between the first and the second phase
 constexpr int kSlots = 8;                       // chunk descriptors in flight
 constexpr int kLookWindows = 8;                 // look-back: 32 status words per window
@@ -191,7 +192,7 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
     for (int s = 0; s < S; ++s) { bar_init(&sm.full[s], 1); bar_init(&sm.empty[s], kWarpsPerTile); }
     for (int q = 0; q < kSlots; ++q) {
       bar_init(&sm.chunk_ready[q], 1);
-      bar_init(&sm.cnt_ready[q], kComputeWarps);
+      bar_init(&sm.cnt_ready[q], kDrawWarps);
       bar_init(&sm.base_ready[q], 1);
     }
     sm.abort_flag = 0;
@@ -201,7 +202,7 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
 
   if (warp < kComputeWarps) {
     // ---------------------------------------------------------------------------------------------
-    // compute warps.  Warps 0-3 take the even tiles of a chunk, warps 4-7 the odd ones.  Within a tile
+    // compaction warps.  Warps 0-3 take the even tiles of a chunk, warps 4-7 the odd ones.  Within a tile
     // warp v owns rows 16 v .. 16 v + 15 and lane l row 16 v + l / 2, columns 64 (l % 2) .. + 63: keep-bit
     // words 4 row + 2 (l % 2) and the next one.  Lane order is (row, column) order.
     // ---------------------------------------------------------------------------------------------
@@ -209,52 +210,29 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
     const int r = v * 16 + (lane >> 1);
     const uint32_t nrows = (uint32_t)p.B, ncols = (uint32_t)p.D;   // B * D < 2^32 (checked by the host)
     uint32_t n = 0;                               // tiles this CTA has worked through (ring position)
-
-    // m[2 i], m[2 i + 1]: this thread's two words of its tile in step i of the chunk
-    auto phase1 = [&](uint32_t seq, uint32_t (&m)[kChunk]) -> uint32_t {
+#pragma unroll 1
+    for (uint32_t seq = 0;; ++seq) {
       const int slot = seq % kSlots;
-      if (!bar_wait(&sm.chunk_ready[slot], (seq / kSlots) & 1u, wc)) return kNoChunk;
+      const uint32_t slot_parity = (seq / kSlots) & 1u;
+      if (!bar_wait(&sm.chunk_ready[slot], slot_parity, wc)) break;
       const uint32_t chunk = sm.chunk_id[slot];
-      if (chunk == kNoChunk) return kNoChunk;
+      if (chunk == kNoChunk) break;
+      // the keep-bit words and totals of the chunk, then its place in `values`
+      if (!bar_wait(&sm.cnt_ready[slot], slot_parity, wc)) break;
+      const uint32_t valid = min((uint32_t)kChunk, ntiles - chunk * kChunk);   // tiles of this chunk
+      // this thread's two words of its tile in each step of the chunk, as the drawing warps left them
+      uint2 mw[kChunk / kTilesPerStep];
 #pragma unroll
       for (int i = 0; i < kChunk / kTilesPerStep; ++i) {
-        const int g = kTilesPerStep * i + side;
-        const uint32_t tile = chunk * kChunk + g;
-        uint32_t m0 = 0, m1 = 0;
-        if (tile < ntiles) {
-          const uint32_t row = sm.tile_slab[slot][g] * kTileRows + r;
-          const uint32_t col0 = sm.tile_cb[slot][g] * kTileCols + half * 64;
-          if (row < nrows && col0 < ncols) {
-            const uint32_t g32 = col0 >> 5;
-            m0 = philox_keep32(g32, row, p.c2, p.c3, ks, p.T);
-            m1 = philox_keep32(g32 + 1u, row, p.c2, p.c3, ks, p.T);
-            const uint32_t nv = ncols - col0;     // valid columns from col0 on
-            if (nv < 64) {
-              m0 &= nv >= 32 ? 0xffffffffu : (1u << nv) - 1u;
-              m1 &= nv <= 32 ? 0u : (1u << (nv - 32)) - 1u;
-            }
-          }
-          *reinterpret_cast<uint2*>(p.keepbits + (tile * (uint32_t)kTileWords + (uint32_t)(r * 4 + half * 2))) =
-              make_uint2(m0, m1);
-        }
-        m[2 * i] = m0;
-        m[2 * i + 1] = m1;
-        const uint32_t wt = __reduce_add_sync(0xffffffffu, __popc(m0) + __popc(m1));
-        if (lane == 0) sm.warp_total[slot][g][v] = wt;
+        const uint32_t g = kTilesPerStep * i + side;
+        mw[i] = make_uint2(0u, 0u);
+        if (g < valid)
+          mw[i] = __ldcg(reinterpret_cast<const uint2*>(
+              p.keepbits + ((chunk * kChunk + g) * (uint32_t)kTileWords + (uint32_t)(r * 4 + half * 2))));
       }
-      __syncwarp();
-      if (lane == 0) bar_arrive(&sm.cnt_ready[slot]);
-      return chunk;
-    };
-
-    // Second phase of one chunk (slot: its descriptor, m: its keep-bit words).  false: a wait gave up.
-    auto phase2 = [&](uint32_t chunk, int slot, uint32_t slot_parity, const uint32_t (&m)[kChunk]) -> bool {
-      // the other warps' totals of the first phase and the chunk's place in `values` are needed now
-      if (!bar_wait(&sm.cnt_ready[slot], slot_parity, wc) ||
-          !bar_wait(&sm.base_ready[slot], slot_parity, wc))
-        return false;
+      if (!bar_wait(&sm.base_ready[slot], slot_parity, wc)) break;
+      bool ok = true;
       T* const wb = sm.wbuf[warp];
-      const uint32_t valid = min((uint32_t)kChunk, ntiles - chunk * kChunk);   // tiles of this chunk
 #pragma unroll
       for (int i = 0; i < kChunk / kTilesPerStep; ++i) {
         const int g = kTilesPerStep * i + side;
@@ -262,7 +240,7 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
         const uint32_t tile = chunk * kChunk + g;
         const uint32_t pos = n + g;               // the tile's place in the ring of loads
         const int s = pos % S;
-        const uint32_t m0 = m[2 * i], m1 = m[2 * i + 1];
+        const uint32_t m0 = mw[i].x, m1 = mw[i].y;
         const uint32_t cnt = __popc(m0) + __popc(m1);
         const uint32_t incl = warp_inclusive_scan(cnt, lane);
         const uint32_t wt = sm.warp_total[slot][g][lane & 3];
@@ -272,7 +250,7 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
           reinterpret_cast<uint16_t*>(p.keepbits + (int64_t)tile * kTileWords + kBitWords)[r] =
               (uint16_t)(wbase + incl - cnt);
         const int64_t base = sm.tile_base[slot][g];
-        if (!bar_wait(&sm.full[s], (pos / S) & 1u, wc)) return false;
+        if (!bar_wait(&sm.full[s], (pos / S) & 1u, wc)) { ok = false; break; }
         const T* src = sm.raw[s] + r * kTileCols + half * 64;
         // Kept entries go to the warp's buffer as they are (bit h of a reversed word is column 31 - h);
         // scaling waits for the copy to `values`, where every lane has work.  The buffer is filled from
@@ -320,45 +298,51 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
         }
         __syncwarp();                             // the staging buffer is rewritten for the next tile
       }
+      if (!ok) break;
       n += valid;
-      return true;
-    };
-
-    // chunks whose first phase is done, oldest first
-    uint32_t mq[kAhead][kChunk], cq[kAhead];
-    uint32_t seq1 = 0, seq2 = 0;                  // chunks handed to the first / second phase so far
-    bool more = true;                             // the loader has not yet said that the work is finished
-#pragma unroll
-    for (int a = 0; a < kAhead; ++a) {
-      cq[a] = kNoChunk;
-#pragma unroll
-      for (int g = 0; g < kChunk; ++g) mq[a][g] = 0;
     }
+  } else if (warp < kComputeWarps + kDrawWarps) {
+    // ---------------------------------------------------------------------------------------------
+    // drawing warps: the keep decisions need no data, so they run ahead of the loads, as far as the
+    // loader has claimed chunks.  Warp v draws rows 16 v .. 16 v + 15 of every tile of a chunk, a lane the
+    // two words it would own as a compaction lane (six Philox calls), writes them to `keepbits`, and
+    // leaves the warp's kept count per tile in shared memory.
+    // ---------------------------------------------------------------------------------------------
+    const int v = warp - kComputeWarps, half = lane & 1;
+    const int r = v * 16 + (lane >> 1);
+    const uint32_t nrows = (uint32_t)p.B, ncols = (uint32_t)p.D;
 #pragma unroll 1
-    for (uint32_t it = 0;; ++it) {
-      uint32_t m_new[kChunk], c_new = kNoChunk;
-#pragma unroll
-      for (int g = 0; g < kChunk; ++g) m_new[g] = 0;
-      if (more) {
-        c_new = phase1(seq1++, m_new);
-        more = c_new != kNoChunk;
+    for (uint32_t seq = 0;; ++seq) {
+      const int slot = seq % kSlots;
+      if (!bar_wait(&sm.chunk_ready[slot], (seq / kSlots) & 1u, wc)) break;
+      const uint32_t chunk = sm.chunk_id[slot];
+      if (chunk == kNoChunk) break;
+#pragma unroll 2
+      for (int g = 0; g < kChunk; ++g) {
+        const uint32_t tile = chunk * kChunk + g;
+        uint32_t m0 = 0, m1 = 0;
+        if (tile < ntiles) {
+          const uint32_t row = sm.tile_slab[slot][g] * kTileRows + r;
+          const uint32_t col0 = sm.tile_cb[slot][g] * kTileCols + half * 64;
+          if (row < nrows && col0 < ncols) {
+            const uint32_t g32 = col0 >> 5;
+            m0 = philox_keep32(g32, row, p.c2, p.c3, ks, p.T);
+            m1 = philox_keep32(g32 + 1u, row, p.c2, p.c3, ks, p.T);
+            const uint32_t nv = ncols - col0;     // valid columns from col0 on
+            if (nv < 64) {
+              m0 &= nv >= 32 ? 0xffffffffu : (1u << nv) - 1u;
+              m1 &= nv <= 32 ? 0u : (1u << (nv - 32)) - 1u;
+            }
+          }
+          *reinterpret_cast<uint2*>(p.keepbits + (tile * (uint32_t)kTileWords + (uint32_t)(r * 4 + half * 2))) =
+              make_uint2(m0, m1);
+        }
+        const uint32_t wt = __reduce_add_sync(0xffffffffu, __popc(m0) + __popc(m1));
+        if (lane == 0) sm.warp_total[slot][g][v] = wt;
       }
-      if (cq[0] != kNoChunk) {
-        const bool ok = phase2(cq[0], seq2 % kSlots, (seq2 / kSlots) & 1u, mq[0]);
-        ++seq2;
-        if (!ok) break;
-      } else if (it >= (uint32_t)kAhead) {
-        break;                                    // every claimed chunk is through
-      }
-#pragma unroll
-      for (int a = 0; a + 1 < kAhead; ++a) {
-        cq[a] = cq[a + 1];
-#pragma unroll
-        for (int g = 0; g < kChunk; ++g) mq[a][g] = mq[a + 1][g];
-      }
-      cq[kAhead - 1] = c_new;
-#pragma unroll
-      for (int g = 0; g < kChunk; ++g) mq[kAhead - 1][g] = m_new[g];
+      __threadfence_block();                      // the words are read back by the compaction warps
+      __syncwarp();
+      if (lane == 0) bar_arrive(&sm.cnt_ready[slot]);
     }
   } else if (warp == kLoaderWarp) {
     // ---------------------------------------------------------------------------------------------
