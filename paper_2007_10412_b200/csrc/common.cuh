@@ -77,12 +77,21 @@ constexpr int kOutputsPerGroup = kLaneBits / 4;   // generator outputs behind on
 struct KeepThreshold {
   uint32_t digit[kLaneBits];   // digit[i]: all ones if bit 11 - i of T is set (T = 4096: all set)
   uint32_t start;              // decisions before any digit: none kept, or all kept for T = 4096
+  int32_t outputs;             // generator outputs that can change a decision: the planes below the lowest set
+                               // bit of T leave "none kept" as it is, so outputs made of such planes only are
+                               // not drawn (T = 2048: one output instead of three; T = 4096: none)
 };
 inline KeepThreshold make_keep_threshold(uint32_t T) {
   KeepThreshold k;
   for (int i = 0; i < kLaneBits; ++i)
     k.digit[i] = (T >= kLaneRange || ((T >> (kLaneBits - 1 - i)) & 1u)) ? 0xffffffffu : 0u;
   k.start = T >= kLaneRange ? 0xffffffffu : 0u;
+  k.outputs = 0;
+  if (T > 0 && T < kLaneRange) {
+    int lowest = 0;                                // lowest set bit of T = plane kLaneBits - 1 - lowest
+    while (((T >> lowest) & 1u) == 0) ++lowest;
+    k.outputs = (kLaneBits - 1 - lowest) / 4 + 1;
+  }
   return k;
 }
 
@@ -103,6 +112,22 @@ __device__ __forceinline__ uint32_t philox_keep32(uint32_t group32, uint32_t row
     uint32_t w[4];
     philox4x32_10((uint32_t)kOutputsPerGroup * group32 + (uint32_t)j, row, c2, c3, ks, w);
     x = keep_fold(x, w, j, k);
+  }
+  return x;
+}
+// The same word from the first k.outputs generator outputs only (see KeepThreshold): for thresholds with
+// trailing zero digits.  A caller that draws several words at once tests k.outputs once and takes this
+// form for all of them, so that the calls of the usual form stay in one piece and overlap.
+__device__ __forceinline__ uint32_t philox_keep32_few(uint32_t group32, uint32_t row, uint32_t c2, uint32_t c3,
+                                                      const PhiloxKeys& ks, const KeepThreshold& k) {
+  uint32_t x = k.start;
+#pragma unroll
+  for (int j = kOutputsPerGroup - 1; j >= 0; --j) {
+    if (j < k.outputs) {
+      uint32_t w[4];
+      philox4x32_10((uint32_t)kOutputsPerGroup * group32 + (uint32_t)j, row, c2, c3, ks, w);
+      x = keep_fold(x, w, j, k);
+    }
   }
   return x;
 }

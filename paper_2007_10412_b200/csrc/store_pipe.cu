@@ -22,6 +22,8 @@
 // roles leave their loops, outstanding loads are waited for, and the kernel returns.
 #include <cuda.h>
 
+#include <type_traits>
+
 #include "common.cuh"
 #include "store.cuh"
 
@@ -311,6 +313,10 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
     const int v = warp - kComputeWarps, half = lane & 1;
     const int r = v * 16 + (lane >> 1);
     const uint32_t nrows = (uint32_t)p.B, ncols = (uint32_t)p.D;
+    // kFew: the threshold has trailing zero digits and needs fewer generator outputs per word.  The two
+    // forms are two loops, so that the usual one stays free of tests and its calls overlap.
+    auto draw = [&](auto few) {
+    constexpr bool kFew = decltype(few)::value;
 #pragma unroll 1
     for (uint32_t seq = 0;; ++seq) {
       const int slot = seq % kSlots;
@@ -326,8 +332,13 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
           const uint32_t col0 = sm.tile_cb[slot][g] * kTileCols + half * 64;
           if (row < nrows && col0 < ncols) {
             const uint32_t g32 = col0 >> 5;
-            m0 = philox_keep32(g32, row, p.c2, p.c3, ks, p.T);
-            m1 = philox_keep32(g32 + 1u, row, p.c2, p.c3, ks, p.T);
+            if constexpr (kFew) {
+              m0 = philox_keep32_few(g32, row, p.c2, p.c3, ks, p.T);
+              m1 = philox_keep32_few(g32 + 1u, row, p.c2, p.c3, ks, p.T);
+            } else {
+              m0 = philox_keep32(g32, row, p.c2, p.c3, ks, p.T);
+              m1 = philox_keep32(g32 + 1u, row, p.c2, p.c3, ks, p.T);
+            }
             const uint32_t nv = ncols - col0;     // valid columns from col0 on
             if (nv < 64) {
               m0 &= nv >= 32 ? 0xffffffffu : (1u << nv) - 1u;
@@ -344,6 +355,8 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
       __syncwarp();
       if (lane == 0) bar_arrive(&sm.cnt_ready[slot]);
     }
+    };
+    if (p.T.outputs == kOutputsPerGroup) draw(std::false_type{}); else draw(std::true_type{});
   } else if (warp == kLoaderWarp) {
     // ---------------------------------------------------------------------------------------------
     // loader: claims chunks kAhead + 1 ahead of the loads it issues, so that the compute warps can run

@@ -37,7 +37,9 @@ def store_kernel(request):
 # slab and column block
 @pytest.mark.parametrize("store_kernel", ["generic", "pipelined"], indirect=True)
 @pytest.mark.parametrize("B,D,dtype", SHAPES + [(1000, 1160, "bf16"), (449, 2200, "f32")])
-@pytest.mark.parametrize("p", [0.1, 0.5, 1.0, 0.01])
+# thresholds with trailing zero digits need fewer generator outputs per word: 0.5 -> one, 416/4096 -> two,
+# 1.0 -> none
+@pytest.mark.parametrize("p", [0.1, 0.5, 1.0, 0.01, 416 / 4096])
 def test_different_sample_store_is_bit_exact(B, D, dtype, p, store_kernel):
     import paper_2007_10412_b200 as rad
     A, _ = layer_inputs(B, D, 1, dtype=dtype, seed=B + D, relu_like=True)
