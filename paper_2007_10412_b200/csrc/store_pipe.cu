@@ -222,27 +222,26 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
       // the keep-bit words and totals of the chunk, then its place in `values`
       if (!bar_wait(&sm.cnt_ready[slot], slot_parity, wc)) break;
       const uint32_t valid = min((uint32_t)kChunk, ntiles - chunk * kChunk);   // tiles of this chunk
-      // this thread's two words of its tile in each step of the chunk, as the drawing warps left them
-      uint2 mw[kChunk / kTilesPerStep];
-#pragma unroll
-      for (int i = 0; i < kChunk / kTilesPerStep; ++i) {
-        const uint32_t g = kTilesPerStep * i + side;
-        mw[i] = make_uint2(0u, 0u);
-        if (g < valid)
-          mw[i] = __ldcg(reinterpret_cast<const uint2*>(
-              p.keepbits + ((chunk * kChunk + g) * (uint32_t)kTileWords + (uint32_t)(r * 4 + half * 2))));
-      }
+      // this thread's two words of its tile in a step of the chunk, as the drawing warps left them, are
+      // asked for one step ahead
+      auto keep_words = [&](uint32_t g) {
+        return g < valid ? __ldcg(reinterpret_cast<const uint2*>(p.keepbits + ((chunk * kChunk + g) * (uint32_t)kTileWords +
+                                                                              (uint32_t)(r * 4 + half * 2))))
+                         : make_uint2(0u, 0u);
+      };
+      uint2 mw = keep_words((uint32_t)side);
       if (!bar_wait(&sm.base_ready[slot], slot_parity, wc)) break;
       bool ok = true;
       T* const wb = sm.wbuf[warp];
-#pragma unroll
+#pragma unroll 1
       for (int i = 0; i < kChunk / kTilesPerStep; ++i) {
         const int g = kTilesPerStep * i + side;
         if ((uint32_t)g >= valid) break;
         const uint32_t tile = chunk * kChunk + g;
         const uint32_t pos = n + g;               // the tile's place in the ring of loads
         const int s = pos % S;
-        const uint32_t m0 = mw[i].x, m1 = mw[i].y;
+        const uint32_t m0 = mw.x, m1 = mw.y;
+        mw = keep_words((uint32_t)g + kTilesPerStep);
         const uint32_t cnt = __popc(m0) + __popc(m1);
         const uint32_t incl = warp_inclusive_scan(cnt, lane);
         const uint32_t wt = sm.warp_total[slot][g][lane & 3];
@@ -254,23 +253,30 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
         const int64_t base = sm.tile_base[slot][g];
         if (!bar_wait(&sm.full[s], (pos / S) & 1u, wc)) { ok = false; break; }
         const T* src = sm.raw[s] + r * kTileCols + half * 64;
-        // Kept entries go to the warp's buffer as they are (bit h of a reversed word is column 31 - h);
-        // scaling waits for the copy to `values`, where every lane has work.  The buffer is filled from
-        // index `lead` on, so that an entry's index in it and its index in `values` agree modulo a 16-byte
-        // vector.  One loop serves both words: it runs as long as the fullest pair of words of the warp.
+        // Kept entries go to the warp's buffer as they are; scaling waits for the copy to `values`, where
+        // every lane has work.  The buffer is filled from index `lead` on, so that an entry's index in it
+        // and its index in `values` agree modulo a 16-byte vector.  One loop serves both words and takes two
+        // entries a turn: it runs half as long as the fullest pair of words of the warp.  Clearing the
+        // lowest set bit (x & (x - 1)) is the only step one turn waits for from the turn before; the
+        // columns come off it by a population count.
         constexpr uint32_t kVec = 16 / sizeof(T), kElem = sizeof(T);
         const uint32_t lead = wbase & (kVec - 1);
-        uint32_t sa = smem_addr(src) + 31 * kElem;          // column 31 of the word being walked
+        uint32_t sa = smem_addr(src);                       // column 0 of the word being walked
         uint32_t da = smem_addr(wb) + (lead + incl - cnt) * kElem;
-        uint32_t rev = __brev(m0), rev_next = __brev(m1);
-        if (rev == 0) { rev = rev_next; rev_next = 0; sa += 32 * kElem; }
-        while (rev != 0) {
-          uint32_t h;
-          asm("bfind.u32 %0, %1;" : "=r"(h) : "r"(rev));
-          rev ^= 1u << h;
-          sts_elem(da, lds_elem(sa - h * kElem, src), src);
-          da += kElem;
-          if (rev == 0) { rev = rev_next; rev_next = 0; sa += 32 * kElem; }
+        uint32_t x = m0, x_next = m1;
+        if (x == 0) { x = x_next; x_next = 0; sa += 32 * kElem; }
+        while (x != 0) {
+          const uint32_t below0 = x - 1u;                   // ones below the lowest set bit
+          const uint32_t c0 = __popc(~x & below0);          // its column
+          const uint32_t x1 = x & below0;
+          const uint32_t below1 = x1 - 1u;
+          const uint32_t c1 = __popc(~x1 & below1);         // 32 if there is no second one
+          const uint32_t v0 = lds_elem(sa + c0 * kElem, src);
+          sts_elem(da, v0, src);
+          if (x1 != 0) sts_elem(da + kElem, lds_elem(sa + c1 * kElem, src), src);
+          da += x1 != 0 ? 2 * kElem : kElem;
+          x = x1 & below1;
+          if (x == 0) { x = x_next; x_next = 0; sa += 32 * kElem; }
         }
         if (p.relubits != nullptr) {
           const uint32_t row = sm.tile_slab[slot][g] * kTileRows + r;
