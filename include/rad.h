@@ -48,7 +48,8 @@ extern "C" {
 #define RAD_DEV_EINTERNAL 3    /* an index left its buffer; the access was skipped (a bug)   */
 
 typedef enum { RAD_F32 = 0, RAD_BF16 = 1 } rad_dtype;
-typedef enum { RAD_DIFFERENT_SAMPLE = 0, RAD_SAME_SAMPLE = 1, RAD_PROJECT = 2, RAD_ROWS_SAMPLE = 3 } rad_variant;
+typedef enum { RAD_DIFFERENT_SAMPLE = 0, RAD_SAME_SAMPLE = 1, RAD_PROJECT = 2, RAD_ROWS_SAMPLE = 3,
+               RAD_REDRAWN_SAMPLE = 4 } rad_variant;
 typedef enum { RAD_ACT_NONE = 0, RAD_ACT_RELU = 1, RAD_ACT_GELU = 2 } rad_act;
 
 /* Geometry of the compact store (fixed; part of the data layout). */
@@ -172,6 +173,18 @@ typedef struct rad_store_sizes {
  * The kept set of a row is the one the fixed-count law of RAD_DIFFERENT_SAMPLE keeps for the same key.
  * rad_linear_weight_grad takes such a store: it rebuilds the index part of the tile-major layout from the key
  * alone, moves the values into it (both in its workspace) and runs the same contraction.
+ */
+
+/*
+ * Redrawn-mask variant, variant = RAD_REDRAWN_SAMPLE (Sec. 3.2: the random matrix is independent of the data, so
+ * what is held for the backward pass need not include it): the same key, mask, `values`, `offsets` and nnz as
+ * RAD_DIFFERENT_SAMPLE under the same law (Bernoulli keeps or the fixed-count law), but the keep bits and row
+ * offsets are not held between the passes.  `keepbits` is unused and may be NULL.  rad_linear_forward_store and
+ * rad_linear_forward_fill build the index part of the tile-major layout in their workspace; rad_linear_weight_grad
+ * draws it again from the key into its workspace (one pass that reads no activation) and runs the same
+ * contraction, so dW_hat is the one of RAD_DIFFERENT_SAMPLE bit for bit.  Per layer 4 bytes per tile (`offsets`)
+ * are held instead of 1156; the workspaces grow by the index of one layer (rad_store_size_query,
+ * rad_weight_grad_workspace).
  */
 
 /*

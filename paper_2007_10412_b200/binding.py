@@ -15,13 +15,14 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "librad_b200.so")
 
 RAD_F32, RAD_BF16 = 0, 1
-RAD_DIFFERENT_SAMPLE, RAD_SAME_SAMPLE, RAD_PROJECT, RAD_ROWS_SAMPLE = 0, 1, 2, 3
+RAD_DIFFERENT_SAMPLE, RAD_SAME_SAMPLE, RAD_PROJECT, RAD_ROWS_SAMPLE, RAD_REDRAWN_SAMPLE = 0, 1, 2, 3, 4
 RAD_ACT_NONE, RAD_ACT_RELU, RAD_ACT_GELU = 0, 1, 2
 RAD_DEV_ECAPACITY, RAD_DEV_ETIMEOUT = 1, 2
 TILE_ROWS, TILE_COLS, VALUE_ALIGN = 64, 128, 8
 
 DTYPES = {"f32": RAD_F32, "bf16": RAD_BF16, torch.float32: RAD_F32, torch.bfloat16: RAD_BF16}
-VARIANTS = {"different": RAD_DIFFERENT_SAMPLE, "same": RAD_SAME_SAMPLE, "project": RAD_PROJECT, "rows": RAD_ROWS_SAMPLE}
+VARIANTS = {"different": RAD_DIFFERENT_SAMPLE, "same": RAD_SAME_SAMPLE, "project": RAD_PROJECT, "rows": RAD_ROWS_SAMPLE,
+            "redrawn": RAD_REDRAWN_SAMPLE}
 LAWS = {"bernoulli": 0, "replace": 1, "fixed": 2}
 ACTS = {"none": RAD_ACT_NONE, "relu": RAD_ACT_RELU, "gelu": RAD_ACT_GELU}
 TORCH_DTYPE = {RAD_F32: torch.float32, RAD_BF16: torch.bfloat16}
@@ -223,7 +224,8 @@ class Store:
         self.relubits = torch.empty(sz.relubits_words, dtype=torch.int32, device=device) if relu_bits else None
         self.workspace = torch.empty(sz.workspace_bytes, dtype=torch.uint8, device=device)
         self.c = rad_store(VARIANTS[variant], DTYPES[dtype], B, D, p, layer, step, seed,
-                           self.values.data_ptr(), int(cap), int(ld), self.keepbits.data_ptr(),
+                           self.values.data_ptr(), int(cap), int(ld),
+                           self.keepbits.data_ptr() if sz.keepbits_words > 0 else None,
                            self.offsets.data_ptr(), self.nnz.data_ptr(),
                            self.relubits.data_ptr() if relu_bits else None, LAWS[law])
 

@@ -51,6 +51,30 @@ TileTwin tile_twin(const rad_store* rows, char* ws) {
   return t;
 }
 
+// Full different-sample twin of a RAD_REDRAWN_SAMPLE store for the backward pass: keep bits, row offsets, tile
+// offsets and counts are drawn again into the workspace, the values are the held ones.
+TileTwin redrawn_twin(const rad_store* held, char* ws) {
+  TileTwin t;
+  const int64_t ntiles = ceil_div(held->B, kTileRows) * ceil_div(held->D, kTileCols);
+  int64_t off = 0;
+  auto take = [&](int64_t bytes) { const int64_t at = off; off += round_up(bytes, 256); return at; };
+  t.st = *held;
+  t.st.variant = RAD_DIFFERENT_SAMPLE;
+  const int64_t kb = take(redrawn_index_bytes(held->B, held->D)), of = take((ntiles + 1) * 4), nz = take(16);
+  t.st.keepbits = ws != nullptr ? reinterpret_cast<uint32_t*>(ws + kb) : reinterpret_cast<uint32_t*>(256);
+  t.st.offsets = ws != nullptr ? reinterpret_cast<uint32_t*>(ws + of) : reinterpret_cast<uint32_t*>(256);
+  t.st.nnz = ws != nullptr ? reinterpret_cast<int64_t*>(ws + nz) : reinterpret_cast<int64_t*>(256);
+  t.st.relubits = nullptr;
+  t.bytes = off;
+  return t;
+}
+bool redrawn_args_ok(const rad_store* st) {
+  return st != nullptr && st->B > 0 && st->D > 0 && valid_dtype(st->dtype) && st->values != nullptr &&
+         st->offsets != nullptr && st->nnz != nullptr && keep_threshold_host(st->p) != 0 &&
+         (st->law == RAD_LAW_BERNOULLI || st->law == RAD_LAW_FIXED) &&
+         (double)st->B * (double)st->D < 4294967296.0 * 0.75;
+}
+
 bool store_args_ok(const rad_store* st) {
   if (st == nullptr || st->B <= 0 || st->D <= 0) return false;
   if (st->variant != RAD_DIFFERENT_SAMPLE && st->variant != RAD_SAME_SAMPLE) return false;
@@ -76,7 +100,8 @@ struct StepPlan {
 int make_plan(const rad_mlp_desc* net, StepPlan* plan) {
   if (net == nullptr || net->dims == nullptr || net->L < 1 || net->L > 64 || net->B <= 0) return RAD_EINVAL;
   if (!valid_dtype(net->dtype)) return RAD_EINVAL;
-  if (net->variant != RAD_DIFFERENT_SAMPLE && net->variant != RAD_SAME_SAMPLE && net->variant != RAD_PROJECT)
+  if (net->variant != RAD_DIFFERENT_SAMPLE && net->variant != RAD_SAME_SAMPLE && net->variant != RAD_PROJECT &&
+      net->variant != RAD_REDRAWN_SAMPLE)
     return RAD_EINVAL;
   if (net->act != RAD_ACT_RELU && net->act != RAD_ACT_GELU) return RAD_EINVAL;
   if (keep_threshold_host(net->p) == 0) return RAD_EINVAL;
@@ -114,8 +139,10 @@ int make_plan(const rad_mlp_desc* net, StepPlan* plan) {
     tmp.variant = net->variant; tmp.dtype = net->dtype; tmp.B = B; tmp.D = D; tmp.p = net->p;
     tmp.law = net->law;
     tmp.values_ld = lp.values_ld; tmp.values_capacity = lp.capacity;
-    scratch = max(scratch, net->variant == RAD_PROJECT ? project_weight_grad_workspace(&tmp, H)
-                                                       : tc_weight_grad_workspace(&tmp, H));
+    int64_t dw_scratch = 0;
+    rc = rad_weight_grad_workspace(&tmp, H, &dw_scratch);
+    if (rc != RAD_OK) return rc;
+    scratch = max(scratch, dw_scratch);
   }
   st.unsampled_bytes = B * net->dims[net->L] * 4;
   st.full_backprop_bytes += st.unsampled_bytes;
@@ -187,6 +214,11 @@ extern "C" int rad_weight_grad_workspace(const rad_store* st, int64_t H, int64_t
     *bytes = t.bytes + round_up(tc_weight_grad_workspace(&t.st, H), 256);
     return RAD_OK;
   }
+  if (st->variant == RAD_REDRAWN_SAMPLE) {
+    const TileTwin t = redrawn_twin(st, nullptr);
+    *bytes = t.bytes + round_up(tc_weight_grad_workspace(&t.st, H), 256);
+    return RAD_OK;
+  }
   *bytes = round_up(tc_weight_grad_workspace(st, H), 256);
   return RAD_OK;
 }
@@ -220,6 +252,21 @@ extern "C" int rad_linear_weight_grad(const rad_store* st, const void* dZ, int64
     if (rcr != RAD_OK) return rcr;
     rcr = rows_to_tiles(st, &t.st, dev_status, sr);
     if (rcr != RAD_OK) return rcr;
+    return rad_linear_weight_grad(&t.st, dZ, ldz, H, dW, ldw, static_cast<char*>(workspace) + t.bytes, workspace_bytes - t.bytes,
+                                  dev_status, stream);
+  }
+  if (st != nullptr && st->variant == RAD_REDRAWN_SAMPLE) {
+    // the index part from the key alone, into the workspace; then the contraction of a different-sample store
+    if (!redrawn_args_ok(st) || dZ == nullptr || dW == nullptr || H <= 0 || ldz < H || ldw < H) return RAD_EINVAL;
+    int rcd = check_device();
+    if (rcd != RAD_OK) return rcd;
+    int64_t need = 0;
+    rcd = rad_weight_grad_workspace(st, H, &need);
+    if (rcd != RAD_OK) return rcd;
+    if (workspace == nullptr || workspace_bytes < need || ((uintptr_t)workspace & 255) != 0) return RAD_EWORKSPACE;
+    const TileTwin t = redrawn_twin(st, static_cast<char*>(workspace));
+    rcd = launch_store_index(&t.st, false, dev_status, static_cast<cudaStream_t>(stream));
+    if (rcd != RAD_OK) return rcd;
     return rad_linear_weight_grad(&t.st, dZ, ldz, H, dW, ldw, static_cast<char*>(workspace) + t.bytes, workspace_bytes - t.bytes,
                                   dev_status, stream);
   }
@@ -288,6 +335,18 @@ extern "C" int rad_linear_forward_fill(int32_t dtype, int32_t act, int64_t B, in
   if (act != RAD_ACT_NONE && act != RAD_ACT_RELU && act != RAD_ACT_GELU) return RAD_EINVAL;
   if (lda < D || ldw < H || ld_act < H || (out_zlow != nullptr && ld_zlow < H)) return RAD_EINVAL;
   if (next == nullptr || next->B != B || next->D != H || next->dtype != dtype) return RAD_EINVAL;
+  if (next->variant == RAD_REDRAWN_SAMPLE) {
+    // the index part goes to the head of the workspace, then as for a different-sample store
+    if (!redrawn_args_ok(next) || index_ready) return RAD_EINVAL;
+    const int64_t head = redrawn_index_bytes(B, H);
+    if (workspace == nullptr || workspace_bytes < head) return RAD_EWORKSPACE;
+    if (((uintptr_t)workspace & 255) != 0) return RAD_EINVAL;
+    rad_store full = *next;
+    full.variant = RAD_DIFFERENT_SAMPLE;
+    full.keepbits = static_cast<uint32_t*>(workspace);
+    return rad_linear_forward_fill(dtype, act, B, D, H, A, lda, W, ldw, bias, out_act, ld_act, out_zlow, ld_zlow, relubits,
+                                   &full, 0, static_cast<char*>(workspace) + head, workspace_bytes - head, dev_status, stream);
+  }
   int rc = check_device();
   if (rc != RAD_OK) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -359,7 +418,7 @@ extern "C" int rad_mlp_held_bytes(const rad_mlp_desc* net, const int64_t* nnz, r
   int64_t held = 0;
   for (int l = 0; l < net->L; ++l) {
     if (nnz[2 * l] < 0 || nnz[2 * l + 1] < nnz[2 * l]) return RAD_EINVAL;
-    const int64_t elems = net->variant == RAD_DIFFERENT_SAMPLE ? nnz[2 * l + 1]
+    const int64_t elems = (net->variant == RAD_DIFFERENT_SAMPLE || net->variant == RAD_REDRAWN_SAMPLE) ? nnz[2 * l + 1]
                         : net->variant == RAD_SAME_SAMPLE      ? net->B * nnz[2 * l]
                                                                : net->B * plan.layer[l].values_ld;
     held += elems * esize(net->dtype);
@@ -392,7 +451,7 @@ extern "C" int rad_mlp_step(const rad_mlp_desc* net, const void* X, const int32_
     s.variant = net->variant; s.dtype = net->dtype; s.B = B; s.D = net->dims[l]; s.p = net->p;
     s.layer = (uint32_t)l; s.step = net->step; s.seed = net->seed; s.law = net->law;
     s.values = ws + lp.values; s.values_capacity = lp.capacity; s.values_ld = lp.values_ld;
-    s.keepbits = reinterpret_cast<uint32_t*>(ws + lp.keepbits);
+    s.keepbits = net->variant == RAD_REDRAWN_SAMPLE ? nullptr : reinterpret_cast<uint32_t*>(ws + lp.keepbits);
     s.offsets = reinterpret_cast<uint32_t*>(ws + lp.offsets);
     s.nnz = nnz_out != nullptr ? nnz_out + 2 * l : reinterpret_cast<int64_t*>(ws + lp.nnz);
     // the ReLU bits of a hidden layer's input are written by the epilogue of the layer that produces it

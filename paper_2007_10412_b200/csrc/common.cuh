@@ -183,6 +183,11 @@ __device__ __forceinline__ float gelu_grad_f(float z) {
 
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 inline int64_t round_up(int64_t a, int64_t b) { return ceil_div(a, b) * b; }
+// Bytes of the index part (keep bits + row offsets, 256-byte rounded) of a tile-major store of B x D entries:
+// what a RAD_REDRAWN_SAMPLE store keeps in a workspace instead of holding it.
+inline int64_t redrawn_index_bytes(int64_t B, int64_t D) {
+  return round_up(ceil_div(B, kTileRows) * ceil_div(D, kTileCols) * kTileWords * 4, 256);
+}
 
 #define RAD_CUDA_TRY(expr)                          \
   do {                                              \

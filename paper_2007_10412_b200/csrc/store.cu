@@ -760,6 +760,15 @@ extern "C" int rad_store_size_query_law(int32_t variant, int32_t dtype, int32_t 
     out->workspace_bytes = 256;
     return RAD_OK;
   }
+  if (variant == RAD_REDRAWN_SAMPLE) {
+    // the different-sample store without its keep bits; the index of one layer lives in the workspace
+    if (law != RAD_LAW_BERNOULLI && law != RAD_LAW_FIXED) return RAD_EINVAL;
+    const int rc = rad_store_size_query_law(RAD_DIFFERENT_SAMPLE, dtype, law, B, D, p, out);
+    if (rc != RAD_OK) return rc;
+    out->workspace_bytes = redrawn_index_bytes(B, D) + round_up(out->workspace_bytes, 256);
+    out->keepbits_words = 0;
+    return RAD_OK;
+  }
   if (variant != RAD_DIFFERENT_SAMPLE && variant != RAD_SAME_SAMPLE) return RAD_EINVAL;
   if (law != RAD_LAW_BERNOULLI && law != RAD_LAW_REPLACE && law != RAD_LAW_FIXED) return RAD_EINVAL;
   const uint32_t T = keep_threshold_host(p);
@@ -811,6 +820,18 @@ extern "C" int rad_linear_forward_store(const void* A, int64_t lda, const rad_st
   if (st->variant == RAD_ROWS_SAMPLE) {
     const int rcr = check_device();
     return rcr != RAD_OK ? rcr : rows_forward_store(A, lda, st, dev_status, static_cast<cudaStream_t>(stream));
+  }
+  if (st->variant == RAD_REDRAWN_SAMPLE) {
+    // the index part goes to the head of the workspace, the different-sample store does the rest
+    if (st->law != RAD_LAW_BERNOULLI && st->law != RAD_LAW_FIXED) return RAD_EINVAL;
+    const int64_t head = redrawn_index_bytes(st->B, st->D);
+    if (workspace == nullptr || workspace_bytes < head) return RAD_EWORKSPACE;
+    if (((uintptr_t)workspace & 255) != 0) return RAD_EINVAL;
+    rad_store full = *st;
+    full.variant = RAD_DIFFERENT_SAMPLE;
+    full.keepbits = static_cast<uint32_t*>(workspace);
+    return rad_linear_forward_store(A, lda, &full, static_cast<char*>(workspace) + head, workspace_bytes - head, dev_status,
+                                    stream);
   }
   if (st->variant != RAD_DIFFERENT_SAMPLE && st->variant != RAD_SAME_SAMPLE) return RAD_EINVAL;
   if (st->values == nullptr || st->keepbits == nullptr || st->offsets == nullptr || st->nnz == nullptr)

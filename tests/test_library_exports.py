@@ -54,6 +54,14 @@ def test_host_only_entry_points():
     with pytest.raises(b.RadError):
         b.rad_store_size_query("same", "f32", 150, 784, 0.0)
     assert b.lib().rad_strerror(-4).decode() == "workspace too small"
+    # held without its keep bits: same values and offsets, no keep-bit words, the index of one layer in the workspace
+    full = b.rad_store_size_query("different", "bf16", 65536, 8192, 0.1)
+    held = b.rad_store_size_query("redrawn", "bf16", 65536, 8192, 0.1)
+    assert held.keepbits_words == 0 and held.offsets_words == full.offsets_words
+    assert held.values_typical == full.values_typical and held.values_worst == full.values_worst
+    assert held.workspace_bytes >= full.workspace_bytes + ntiles * 288 * 4
+    with pytest.raises(b.RadError):
+        b.rad_store_size_query_law("redrawn", "bf16", "replace", 1000, 1160, 0.1)
 
 
 def test_host_only_entry_points_of_the_with_replacement_law_and_the_kernel_choice():
