@@ -292,7 +292,13 @@ class LayerwiseStep:
                 break
             out = self.acts[l & 1][:, :dims[l + 1]]
             nxt = self.stores[l + 1]
-            if fused:
+            if self.variant == "redrawn":
+                # the index part goes to the store's workspace inside the call and is not held
+                run("forward", l, lambda: rad.rad_linear_forward_fill(a_in, Ws[l], bs[l], self.act, out, nxt,
+                                                                      out_zlow=self.preact[l + 1],
+                                                                      relubits=self.relubits[l + 1],
+                                                                      dev_status=self.status))
+            elif fused:
                 run("store", l + 1, lambda: rad.rad_store_index(nxt, self.status))
                 run("forward", l, lambda: rad.rad_linear_forward_fill(a_in, Ws[l], bs[l], self.act, out, nxt,
                                                                       out_zlow=self.preact[l + 1],
@@ -788,6 +794,21 @@ def run_ours(args):
                     activation_memory=memory_report(rad, dims, B, "relu", args.variant, args.p, args.law, nnz_all))
         del lw2
         torch.cuda.empty_cache()
+        if args.variant == "different" and args.law in ("bernoulli", "fixed"):
+            # the same twin holding no keep bits: every index is drawn again from the key in the backward pass
+            lw3 = LayerwiseStep(rad, torch, dims, B, "relu", "redrawn", args.p, args.law)
+            ms3, launches3, _ = timed_steps(lw3, 1, twin_steps, first_step=60)
+            nnz_all = []
+            for st in lw3.stores:
+                nnz_all += st.nnz.cpu().tolist()
+            twin["mask_redrawn"] = dict(
+                variant="redrawn", steps=twin_steps, ms_per_step=round(ms3 / twin_steps, 3),
+                samples_per_s=round(B * twin_steps / (ms3 / 1e3), 1), gpu_launches=int(launches3),
+                family_ms={k: round(sum(sum(v) for (f, l), v in lw3.family_ms().items() if f == k) / twin_steps, 3)
+                           for k in ("store", "forward", "loss", "dW", "dX+db")},
+                activation_memory=memory_report(rad, dims, B, "relu", "redrawn", args.p, args.law, nnz_all))
+            del lw3
+            torch.cuda.empty_cache()
 
     sweep = None
     if rank == 0 and world == 1 and not args.no_sweep:
