@@ -700,7 +700,7 @@ def run_ours(args):
     traffic = None
     if args.act == "gelu" and abs(args.p - 0.1) < 1e-9 and args.law == "bernoulli" and args.variant == "different":
         if dominant == "forward":
-            traffic = int((1080.2e6 + 263.0e6) * B / 8192)
+            traffic = int((1263.5e6 + 269.8e6) * B / 8192)
         elif dominant == "dW":
             traffic = int(631.7e6 * B / 8192 + 236.0e6)
     roofline = dict(bound=dom["bound"], kernel=dom["kernel"], achieved=dom["achieved"], peak=dom["peak"], unit=dom["unit"],
