@@ -641,6 +641,24 @@ __global__ void wait_probe_lookback_kernel(uint64_t limit_ns, int32_t* dev_statu
 constexpr int kPipelinedMinTiles = 2048;
 int g_store_kernel = RAD_STORE_KERNEL_AUTO;
 
+// Values (and ReLU bits) into a store whose index part is in place: the persistent kernel's loader and
+// compaction warps where they apply (many tiles, aligned input), else one CTA per tile.  p.ticket: 256 bytes.
+int launch_store_fill(const StoreParams& p, const PhiloxKeys& ks, int dtype, double keep_fraction, cudaStream_t s) {
+  if (g_store_kernel == RAD_STORE_KERNEL_PIPELINED ||
+      (g_store_kernel == RAD_STORE_KERNEL_AUTO && p.ntiles >= kPipelinedMinTiles && keep_fraction <= 0.5)) {
+    RAD_CUDA_TRY(cudaMemsetAsync(p.ticket, 0, 256, s));
+    const int rc = launch_store_pipelined(p, ks, dtype, s, true);
+    if (rc != RAD_EUNSUPPORTED) return rc;
+  }
+  count_launch();
+  if (dtype == RAD_BF16)
+    store_different_kernel<bf16, kMaskIndex><<<p.ntiles, 256, 0, s>>>(p, ks);
+  else
+    store_different_kernel<float, kMaskIndex><<<p.ntiles, 256, 0, s>>>(p, ks);
+  RAD_CUDA_TRY(cudaGetLastError());
+  return RAD_OK;
+}
+
 // The persistent TMA-fed kernel where the input can be described by a tensor map, else the generic one
 // (same layout, same scratch: a claim counter and one status word per tile or chunk of tiles).
 int launch_store_different(const StoreParams& p, const PhiloxKeys& ks, int dtype, uint32_t T, cudaStream_t s) {
@@ -880,15 +898,7 @@ extern "C" int rad_linear_forward_store(const void* A, int64_t lda, const rad_st
       // exactly k columns per row: the index part comes from the key alone (Floyd's sampling, a warp per row),
       // then one CTA per tile places the values; no multiplicity matrix, no look-back
       rc = launch_fixed_index(st, true, dev_status, s);
-      if (rc == RAD_OK) {
-        count_launch();
-        if (st->dtype == RAD_BF16)
-          store_different_kernel<bf16, kMaskIndex><<<p.ntiles, 256, 0, s>>>(p, ks);
-        else
-          store_different_kernel<float, kMaskIndex><<<p.ntiles, 256, 0, s>>>(p, ks);
-        RAD_CUDA_TRY(cudaGetLastError());
-        return RAD_OK;
-      }
+      if (rc == RAD_OK) return launch_store_fill(p, ks, st->dtype, store_keep_fraction(st), s);
       if (rc != RAD_EUNSUPPORTED) return rc;      // rows too long for shared memory: the multiplicity matrix below
     }
     RAD_CUDA_TRY(cudaMemsetAsync(workspace, 0, (size_t)status_bytes(st->B, st->D), s));

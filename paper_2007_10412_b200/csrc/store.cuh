@@ -104,6 +104,6 @@ struct StoreParams {
 
 // store_pipe.cu: the persistent TMA-fed kernel.  RAD_EUNSUPPORTED (nothing enqueued) when the input does not
 // meet the alignment rules of a tensor map; the caller then takes the generic kernel.
-int launch_store_pipelined(const StoreParams& p, const PhiloxKeys& ks, int dtype, cudaStream_t s);
+int launch_store_pipelined(const StoreParams& p, const PhiloxKeys& ks, int dtype, cudaStream_t s, bool fill = false);
 
 }  // namespace rad

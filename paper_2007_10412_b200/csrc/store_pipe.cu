@@ -176,7 +176,10 @@ __device__ __forceinline__ void copy_scaled(const T* wb, T* out, uint32_t first,
   }
 }
 
-template <typename T, int S>
+// kFill: the index part of the store (keep bits, row offsets, tile offsets, nnz) is in place already, made
+// from the key alone under whatever law; only the loader and the compaction warps work, a tile's place in
+// `values` and a warp's place in the tile are read instead of computed, and nothing waits for a look-back.
+template <typename T, int S, bool kFill>
 __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const StoreParams p, const PhiloxKeys ks,
                                                                       const __grid_constant__ CUtensorMap tmA) {
   // A stage of the ring must always serve the same half of the compute warps: a waiter tells the phases of
@@ -220,17 +223,27 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
       const uint32_t chunk = sm.chunk_id[slot];
       if (chunk == kNoChunk) break;
       // the keep-bit words and totals of the chunk, then its place in `values`
-      if (!bar_wait(&sm.cnt_ready[slot], slot_parity, wc)) break;
+      if (!kFill && !bar_wait(&sm.cnt_ready[slot], slot_parity, wc)) break;
       const uint32_t valid = min((uint32_t)kChunk, ntiles - chunk * kChunk);   // tiles of this chunk
       // this thread's two words of its tile in a step of the chunk, as the drawing warps left them, are
-      // asked for one step ahead
+      // asked for one step ahead (kFill: with the warp's first row offset and the tile's bounds in `values`)
+      struct Ahead { uint2 m; uint32_t wbase, first, end; };
       auto keep_words = [&](uint32_t g) {
-        return g < valid ? __ldcg(reinterpret_cast<const uint2*>(p.keepbits + ((chunk * kChunk + g) * (uint32_t)kTileWords +
-                                                                              (uint32_t)(r * 4 + half * 2))))
-                         : make_uint2(0u, 0u);
+        Ahead a = {make_uint2(0u, 0u), 0u, 0u, 0u};
+        if (g < valid) {
+          const uint32_t tile = chunk * kChunk + g;
+          const uint32_t* tw = p.keepbits + tile * (uint32_t)kTileWords;
+          a.m = __ldcg(reinterpret_cast<const uint2*>(tw + (uint32_t)(r * 4 + half * 2)));
+          if (kFill) {
+            a.wbase = __ldcg(reinterpret_cast<const uint16_t*>(tw + kBitWords) + 16 * v);
+            a.first = __ldcg(p.offsets + tile);
+            a.end = __ldcg(p.offsets + tile + 1);
+          }
+        }
+        return a;
       };
-      uint2 mw = keep_words((uint32_t)side);
-      if (!bar_wait(&sm.base_ready[slot], slot_parity, wc)) break;
+      Ahead mw = keep_words((uint32_t)side);
+      if (!kFill && !bar_wait(&sm.base_ready[slot], slot_parity, wc)) break;
       bool ok = true;
       T* const wb = sm.wbuf[warp];
 #pragma unroll 1
@@ -240,17 +253,26 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
         const uint32_t tile = chunk * kChunk + g;
         const uint32_t pos = n + g;               // the tile's place in the ring of loads
         const int s = pos % S;
-        const uint32_t m0 = mw.x, m1 = mw.y;
+        const uint32_t m0 = mw.m.x, m1 = mw.m.y;
+        const Ahead here = mw;
         mw = keep_words((uint32_t)g + kTilesPerStep);
         const uint32_t cnt = __popc(m0) + __popc(m1);
         const uint32_t incl = warp_inclusive_scan(cnt, lane);
-        const uint32_t wt = sm.warp_total[slot][g][lane & 3];
-        const uint32_t wbase = __reduce_add_sync(0xffffffffu, lane < v ? wt : 0u);
         const uint32_t wtotal = __shfl_sync(0xffffffffu, incl, 31);
-        if (half == 0)
-          reinterpret_cast<uint16_t*>(p.keepbits + (int64_t)tile * kTileWords + kBitWords)[r] =
-              (uint16_t)(wbase + incl - cnt);
-        const int64_t base = sm.tile_base[slot][g];
+        uint32_t wbase;
+        int64_t base;
+        if (kFill) {
+          wbase = here.wbase;
+          base = (int64_t)here.end <= p.capacity ? (int64_t)here.first : -1;
+          if (base < 0 && v == 0 && lane == 0) raise_status(p.dev_status, RAD_DEV_ECAPACITY);
+        } else {
+          const uint32_t wt = sm.warp_total[slot][g][lane & 3];
+          wbase = __reduce_add_sync(0xffffffffu, lane < v ? wt : 0u);
+          if (half == 0)
+            reinterpret_cast<uint16_t*>(p.keepbits + (int64_t)tile * kTileWords + kBitWords)[r] =
+                (uint16_t)(wbase + incl - cnt);
+          base = sm.tile_base[slot][g];
+        }
         if (!bar_wait(&sm.full[s], (pos / S) & 1u, wc)) { ok = false; break; }
         const T* src = sm.raw[s] + r * kTileCols + half * 64;
         // Kept entries go to the warp's buffer as they are; scaling waits for the copy to `values`, where
@@ -362,7 +384,9 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
       if (lane == 0) bar_arrive(&sm.cnt_ready[slot]);
     }
     };
-    if (p.T.outputs == kOutputsPerGroup) draw(std::false_type{}); else draw(std::true_type{});
+    if (!kFill) {
+      if (p.T.outputs == kOutputsPerGroup) draw(std::false_type{}); else draw(std::true_type{});
+    }
   } else if (warp == kLoaderWarp) {
     // ---------------------------------------------------------------------------------------------
     // loader: claims chunks kAhead + 1 ahead of the loads it issues, so that the compute warps can run
@@ -450,7 +474,7 @@ __global__ void __launch_bounds__(kPipeThreads, 2) store_pipelined_kernel(const 
       return chunk;
     };
     Counts cur, nxt;
-    uint32_t chunk = publish(0, cur);
+    uint32_t chunk = kFill ? kNoChunk : publish(0, cur);
     for (uint32_t seq = 0; chunk != kNoChunk; ++seq) {
       const int slot = seq % kSlots;
       const uint32_t chunk_nxt = publish(seq + 1, nxt);
@@ -556,14 +580,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-template <typename T, int S>
+template <typename T, int S, bool kFill>
 int launch_typed(const StoreParams& p, const PhiloxKeys& ks, const CUtensorMap& map, cudaStream_t s) {
   static int grid_cap[64] = {};                   // resident CTAs per device, found once
   int dev = 0;
   RAD_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return RAD_EUNSUPPORTED;
   const size_t smem = sizeof(PipeSmem<T, S>) + 128;
-  auto kernel = store_pipelined_kernel<T, S>;
+  auto kernel = store_pipelined_kernel<T, S, kFill>;
   if (grid_cap[dev] == 0) {
     RAD_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int per_sm = 0, sms = 0;
@@ -588,7 +612,8 @@ int launch_wait_probe_pipe(uint64_t limit_ns, int32_t* dev_status, cudaStream_t 
   return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
 }
 
-int launch_store_pipelined(const StoreParams& p, const PhiloxKeys& ks, int dtype, cudaStream_t s) {
+// fill: values (and ReLU bits) only, into an index part that is already in place; p.ticket must be zero.
+int launch_store_pipelined(const StoreParams& p, const PhiloxKeys& ks, int dtype, cudaStream_t s, bool fill) {
   const size_t esz = dtype == RAD_BF16 ? 2 : 4;
   if (((uintptr_t)p.A & 15) != 0 || ((size_t)p.lda * esz) % 16 != 0) return RAD_EUNSUPPORTED;
   if (((uintptr_t)p.keepbits & 7) != 0) return RAD_EUNSUPPORTED;   // keep-bit words leave in pairs
@@ -605,8 +630,9 @@ int launch_store_pipelined(const StoreParams& p, const PhiloxKeys& ks, int dtype
                         CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return RAD_EUNSUPPORTED;
-  if (dtype == RAD_BF16) return launch_typed<bf16, 4>(p, ks, map, s);
-  return launch_typed<float, 4>(p, ks, map, s);
+  if (fill) return dtype == RAD_BF16 ? launch_typed<bf16, 4, true>(p, ks, map, s) : launch_typed<float, 4, true>(p, ks, map, s);
+  if (dtype == RAD_BF16) return launch_typed<bf16, 4, false>(p, ks, map, s);
+  return launch_typed<float, 4, false>(p, ks, map, s);
 }
 
 }  // namespace rad

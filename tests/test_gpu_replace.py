@@ -19,10 +19,23 @@ SHAPES = [(150, 784, "f32"), (150, 300, "bf16"), (7, 5, "f32"), (64, 128, "bf16"
 LAWS = ["replace", "fixed"]
 
 
+@pytest.fixture
+def store_kernel(request):
+    """Forces one of the different-sample store kernels for the test, then restores the automatic choice."""
+    import paper_2007_10412_b200 as rad
+    prev = rad.rad_set_store_kernel(request.param)
+    yield request.param
+    rad.rad_set_store_kernel(prev)
+
+
+# "pipelined": where the index part comes from the key alone (fixed-count law), the values are placed by the
+# persistent kernel's loader and compaction warps instead of one CTA per tile; the last two shapes span several
+# chunks with a ragged last chunk, slab and column block
+@pytest.mark.parametrize("store_kernel", ["auto", "pipelined"], indirect=True)
 @pytest.mark.parametrize("law", LAWS)
-@pytest.mark.parametrize("B,D,dtype", SHAPES)
+@pytest.mark.parametrize("B,D,dtype", SHAPES + [(1000, 1160, "bf16"), (449, 2200, "f32")])
 @pytest.mark.parametrize("f", [0.1, 0.5, 1.0, 0.01])
-def test_different_sample_store_is_bit_exact(B, D, dtype, f, law):
+def test_different_sample_store_is_bit_exact(B, D, dtype, f, law, store_kernel):
     import paper_2007_10412_b200 as rad
     A, _ = layer_inputs(B, D, 1, dtype=dtype, seed=B + D, relu_like=True)
     seed, layer, step = (1 << 40) + 777, 2, 5
