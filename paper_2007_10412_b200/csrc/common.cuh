@@ -264,6 +264,9 @@ bool rows_store_ok(const rad_store* st);
 int rows_forward_store(const void* A, int64_t lda, const rad_store* st, int32_t* dev_status, cudaStream_t s);
 int launch_fixed_index(const rad_store* st, bool check_capacity, int32_t* dev_status, cudaStream_t s);
 int rows_to_tiles(const rad_store* rows, const rad_store* tiles, int32_t* dev_status, cudaStream_t s);
+int64_t replace_extras_ld(int64_t D, int64_t k);
+int launch_replace_index(const rad_store* st, uint32_t* extras, bool check_capacity, int32_t* dev_status, cudaStream_t s);
+int launch_replace_extras(const void* A, int64_t lda, const rad_store* st, const uint32_t* extras, cudaStream_t s);
 int tc_input_grad(int64_t B, int64_t D, int64_t H, const void* dZ, int64_t ldz, const void* W,
                   int64_t ldw, const uint32_t* relubits_prev, const void* z_prev, int64_t ld_zprev,
                   void* dZ_prev, int64_t ldp, int32_t* dev_status, cudaStream_t s);

@@ -901,6 +901,19 @@ extern "C" int rad_linear_forward_store(const void* A, int64_t lda, const rad_st
       if (rc == RAD_OK) return launch_store_fill(p, ks, st->dtype, store_keep_fraction(st), s);
       if (rc != RAD_EUNSUPPORTED) return rc;      // rows too long for shared memory: the multiplicity matrix below
     }
+    if (replace && !fixed) {
+      // the same road for k draws with replacement: index part from the key alone, values placed with the
+      // weight of one draw, the few entries drawn more than once written again with theirs (their list takes
+      // the place of the multiplicity matrix in the workspace)
+      uint32_t* extras = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + status_bytes(st->B, st->D));
+      rc = launch_replace_index(st, extras, true, dev_status, s);
+      if (rc == RAD_OK) {
+        rc = launch_store_fill(p, ks, st->dtype, store_keep_fraction(st), s);
+        if (rc != RAD_OK) return rc;
+        return launch_replace_extras(A, lda, st, extras, s);
+      }
+      if (rc != RAD_EUNSUPPORTED) return rc;      // many draws or long rows: the multiplicity matrix below
+    }
     RAD_CUDA_TRY(cudaMemsetAsync(workspace, 0, (size_t)status_bytes(st->B, st->D), s));
     if (replace) {
       // first the multiplicities of every row, then the generic kernel with the mask and the weights

@@ -17,6 +17,15 @@
 //                                     part of a bitmask store, from the key alone
 //   rows_to_tiles_kernel<T>           places the values of a static-shape store into the tile-major layout
 //                                     whose index part the kernel above has written (weight gradient)
+//
+// The with-replacement law (Sec. 3.2: k draws per row, an entry drawn c times weighs c d / k) takes the same
+// road to a bitmask store without a B x D multiplicity matrix in HBM:
+//   replace_index_kernel              a warp's k draws set bits in the bitmap of its row in shared memory; a
+//                                     draw that finds its bit set is a repeat.  The row's keep bits go to the
+//                                     tile-major layout as above, and the few columns drawn more than once go,
+//                                     with their counts, to a short list per row
+//   replace_extras_kernel<T>          after the values have been placed with the weight of a single draw: the
+//                                     listed entries are written again with their own weight
 #include <algorithm>
 
 #include "common.cuh"
@@ -242,6 +251,117 @@ __global__ void __launch_bounds__(256) tile_padding_kernel(const uint32_t* keepb
   }
 }
 
+// With-replacement law, index part.  One CTA per slab of 64 rows; warp w takes rows w, w + 8, ...  A draw sets
+// its column's bit in the row's bitmap (shared memory, the row's keep-bit words); a draw that finds the bit set
+// is a repeat and goes to the warp's short list of repeats.  A column drawn c times is on that list c - 1 times.
+// extras: `extras_ld` words per row: word 0 = entries that follow, each (column | count << 16), count >= 2.
+__global__ void __launch_bounds__(32 * kRowsWarps) replace_index_kernel(const RowsParams p, const PhiloxKeys ks, uint32_t* extras,
+                                                                        int32_t extras_ld) {
+  extern __shared__ __align__(16) uint32_t s_dyn[];
+  __shared__ uint32_t s_nrep[kRowsWarps], s_nex[kRowsWarps];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int per_warp = p.words + p.draws_stride;            // bitmap, then up to k repeats as 16-bit columns
+  uint32_t* bm = s_dyn + warp * per_warp;
+  uint16_t* rep = reinterpret_cast<uint16_t*>(bm + p.words);
+  uint8_t* s_cnt = reinterpret_cast<uint8_t*>(s_dyn + kRowsWarps * per_warp);   // [64 rows][ncb] kept per (row, block)
+  for (int64_t slab = blockIdx.x; slab * kTileRows < p.B; slab += gridDim.x) {
+    for (int r = warp; r < kTileRows; r += kRowsWarps) {
+      const int64_t row = slab * kTileRows + r;
+      for (int i = lane; i < p.words; i += 32) bm[i] = 0;
+      if (lane == 0) { s_nrep[warp] = 0; s_nex[warp] = 0; }
+      __syncwarp();
+      if (row < p.B) {
+        for (uint32_t c = lane; 4 * (int64_t)c < p.k; c += 32) {
+          uint32_t w[4];
+          philox4x32_10(c, (uint32_t)row, p.c2, p.c3, ks, w);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            if (4 * (int64_t)c + j < p.k) {
+              const uint32_t col = __umulhi(w[j], (uint32_t)p.D);
+              const uint32_t bit = 1u << (col & 31);
+              if (atomicOr(&bm[col >> 5], bit) & bit) rep[atomicAdd(&s_nrep[warp], 1u)] = (uint16_t)col;   // fewer than k
+            }
+          }
+        }
+        __syncwarp();
+        // repeats of one column are counted together; the first of them on the list writes the entry
+        const uint32_t n = s_nrep[warp];
+        uint32_t* ex = extras + row * extras_ld;
+        for (uint32_t j = lane; j < n; j += 32) {
+          const uint32_t col = rep[j];
+          uint32_t cnt = 0;
+          bool first = true;
+          for (uint32_t i = 0; i < n; ++i) {
+            const bool same = rep[i] == col;
+            cnt += same ? 1u : 0u;
+            first = first && !(same && i < j);
+          }
+          if (first) {
+            const uint32_t slot = atomicAdd(&s_nex[warp], 1u) + 1u;
+            if ((int)slot < extras_ld) ex[slot] = col | ((cnt + 1u) << 16);
+            else raise_status(p.dev_status, RAD_DEV_EINTERNAL);
+          }
+        }
+        __syncwarp();
+        if (lane == 0) ex[0] = min(s_nex[warp], (uint32_t)(extras_ld - 1));
+      }
+      __syncwarp();
+      for (int cb = lane; cb < p.ncb; cb += 32) {
+        uint32_t q[4];
+#pragma unroll
+        for (int w = 0; w < 4; ++w) q[w] = 4 * cb + w < p.words ? bm[4 * cb + w] : 0u;
+        *reinterpret_cast<uint4*>(p.keepbits + (slab * p.ncb + cb) * kTileWords + r * 4) = make_uint4(q[0], q[1], q[2], q[3]);
+        s_cnt[r * p.ncb + cb] = (uint8_t)(__popc(q[0]) + __popc(q[1]) + __popc(q[2]) + __popc(q[3]));   // at most 128
+      }
+      __syncwarp();
+    }
+    __syncthreads();
+    // in-tile row offsets: prefix down the 64 rows of each column block
+    for (int cb = tid; cb < p.ncb; cb += 32 * kRowsWarps) {
+      uint32_t* tw = p.keepbits + (slab * p.ncb + cb) * kTileWords;
+      uint32_t run = 0;
+      for (int r = 0; r < kTileRows; r += 2) {
+        const uint32_t c0 = s_cnt[r * p.ncb + cb], c1 = s_cnt[(r + 1) * p.ncb + cb];
+        tw[kBitWords + (r >> 1)] = run | ((run + c0) << 16);
+        run += c0 + c1;
+      }
+      p.offsets[slab * p.ncb + cb] = run;
+    }
+    __syncthreads();
+  }
+}
+
+// The entries drawn more than once, written again with their own weight fl32(c * (D / k)) (one product with the
+// entry, as for every other value).  A warp per row; the entry's place follows from the index part.
+template <typename T>
+__global__ void __launch_bounds__(256) replace_extras_kernel(const T* A, int64_t lda, int64_t B, int32_t ncb, const uint32_t* extras,
+                                                             int32_t extras_ld, const uint32_t* keepbits, const uint32_t* offsets,
+                                                             T* values, int64_t capacity, float scale) {
+  const int lane = threadIdx.x & 31;
+  for (int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5); row < B; row += (int64_t)gridDim.x * 8) {
+    const uint32_t* ex = extras + row * extras_ld;
+    const uint32_t n = ex[0];
+    const int64_t slab = row >> 6;
+    const int r = (int)(row & 63);
+    for (uint32_t j = lane; j < n; j += 32) {
+      const uint32_t e = ex[1 + j];
+      const uint32_t col = e & 0xffffu, c = e >> 16;
+      const int64_t tile = slab * ncb + (col >> 7);
+      const uint32_t* tw = keepbits + tile * kTileWords;
+      const uint4 q = *reinterpret_cast<const uint4*>(tw + r * 4);
+      const uint32_t wq = (col & 127u) >> 5, bit = col & 31u;
+      const uint32_t word = wq == 0 ? q.x : wq == 1 ? q.y : wq == 2 ? q.z : q.w;
+      uint32_t rank = __popc(word & ((1u << bit) - 1u));
+      if (wq > 0) rank += __popc(q.x);
+      if (wq > 1) rank += __popc(q.y);
+      if (wq > 2) rank += __popc(q.z);
+      const uint32_t rowoff = reinterpret_cast<const uint16_t*>(tw + kBitWords)[r];
+      if ((int64_t)offsets[tile + 1] <= capacity)       // a tile that does not fit is left out as a whole
+        values[(int64_t)offsets[tile] + rowoff + rank] = from_float<T>(__fmul_rn(to_float(A[row * lda + col]), __fmul_rn((float)c, scale)));
+    }
+  }
+}
+
 constexpr int64_t kRowsSmemBudget = 200 * 1024;
 
 // shared memory of rows_fixed_kernel, or -1 if a row does not fit
@@ -312,6 +432,55 @@ int launch_fixed_index(const rad_store* st, bool check_capacity, int32_t* dev_st
   int rc = launch_rows_fixed<false>(p, st->dtype, st->seed, smem, (int)std::min<int64_t>(slabs, 148 * 8), s);
   if (rc != RAD_OK) return rc;
   return launch_offsets_scan(st->offsets, slabs * p.ncb, st->nnz, check_capacity ? st->values_capacity : -1, dev_status, s);
+}
+
+// Words per row of the list of entries drawn more than once (first word: their number).  k draws hit at most
+// k / 2 columns twice or more; the list takes the place of the row of the multiplicity matrix, so it has to fit
+// in D bytes.  0: the law's index cannot be made this way (too many draws for the list, or a row's histogram
+// does not fit shared memory).
+int64_t replace_extras_ld(int64_t D, int64_t k) {
+  const int64_t words = ceil_div(D, 32), ncb = ceil_div(D, kTileCols);
+  if (D > 65536 || k / 2 + 1 > D / 4) return 0;
+  if (kRowsWarps * (words + round_up(k, 4)) * 4 + round_up(kTileRows * ncb, 16) > kRowsSmemBudget) return 0;
+  return D / 4;
+}
+
+// Index part of a tile-major store under the with-replacement law, from the key alone, plus the list of entries
+// drawn more than once (`extras`: B x replace_extras_ld words).  RAD_EUNSUPPORTED where that does not apply.
+int launch_replace_index(const rad_store* st, uint32_t* extras, bool check_capacity, int32_t* dev_status, cudaStream_t s) {
+  const int64_t k = draws_per_row_host(st->p, st->D);
+  if (k <= 0) return RAD_EINVAL;
+  const int64_t ld = replace_extras_ld(st->D, k);
+  if (ld == 0 || ((uintptr_t)st->keepbits & 15) != 0) return RAD_EUNSUPPORTED;
+  RowsParams p = rows_params(st, k);
+  p.c2 = counter_word2(st->layer, RAD_DIFFERENT_SAMPLE, RAD_LAW_REPLACE);
+  p.keepbits = st->keepbits; p.offsets = st->offsets; p.nnz = st->nnz; p.dev_status = dev_status;
+  const int64_t slabs = ceil_div(st->B, kTileRows);
+  const int64_t smem = kRowsWarps * ((int64_t)p.words + p.draws_stride) * 4 + round_up(kTileRows * p.ncb, 16);
+  const PhiloxKeys ks = philox_expand_key(st->seed);
+  count_launch();
+  RAD_CUDA_TRY(cudaFuncSetAttribute(replace_index_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRowsSmemBudget));
+  replace_index_kernel<<<(int)std::min<int64_t>(slabs, 148 * 8), 32 * kRowsWarps, (size_t)smem, s>>>(p, ks, extras, (int32_t)ld);
+  if (cudaGetLastError() != cudaSuccess) return RAD_ECUDA;
+  return launch_offsets_scan(st->offsets, slabs * p.ncb, st->nnz, check_capacity ? st->values_capacity : -1, dev_status, s);
+}
+
+// The listed entries written again with their own weight (after the values have been placed with D / k).
+int launch_replace_extras(const void* A, int64_t lda, const rad_store* st, const uint32_t* extras, cudaStream_t s) {
+  const int64_t k = draws_per_row_host(st->p, st->D);
+  const int64_t ld = replace_extras_ld(st->D, k);
+  if (ld == 0) return RAD_EUNSUPPORTED;
+  const int32_t ncb = (int32_t)ceil_div(st->D, kTileCols);
+  const float scale = (float)st->D / (float)k;
+  const int grid = (int)std::min<int64_t>(ceil_div(st->B, 8), 148 * 64);   // short dependent chains: many warps in flight
+  count_launch();
+  if (st->dtype == RAD_BF16)
+    replace_extras_kernel<bf16><<<grid, 256, 0, s>>>(static_cast<const bf16*>(A), lda, st->B, ncb, extras, (int32_t)ld, st->keepbits,
+                                                     st->offsets, static_cast<bf16*>(st->values), st->values_capacity, scale);
+  else
+    replace_extras_kernel<float><<<grid, 256, 0, s>>>(static_cast<const float*>(A), lda, st->B, ncb, extras, (int32_t)ld, st->keepbits,
+                                                      st->offsets, static_cast<float*>(st->values), st->values_capacity, scale);
+  return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
 }
 
 // Values of the tile-major store `tiles` (index part in place) from the static-shape store `rows` of the same key.
