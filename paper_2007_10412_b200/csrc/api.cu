@@ -201,6 +201,44 @@ extern "C" const char* rad_strerror(int code) {
   }
 }
 
+namespace rad {
+namespace {
+// rad_linear_weight_grad for a bitmask or column-list store (index held or drawn again); where the contraction
+// runs on the CUDA cores and passes over dZ anyway, it also leaves the bias gradient in `db` (*db_written says
+// whether it did).
+int weight_grad_and_bias(const rad_store* st, const void* dZ, int64_t ldz, int64_t H, float* dW, int64_t ldw, void* workspace,
+                         int64_t workspace_bytes, int32_t* dev_status, void* stream, float* db, bool* db_written) {
+  if (db_written != nullptr) *db_written = false;
+  if (st != nullptr && st->variant == RAD_REDRAWN_SAMPLE) {
+    // the index part from the key alone, into the workspace; then the contraction of a different-sample store
+    if (!redrawn_args_ok(st) || dZ == nullptr || dW == nullptr || H <= 0 || ldz < H || ldw < H) return RAD_EINVAL;
+    int rcd = check_device();
+    if (rcd != RAD_OK) return rcd;
+    int64_t need = 0;
+    rcd = rad_weight_grad_workspace(st, H, &need);
+    if (rcd != RAD_OK) return rcd;
+    if (workspace == nullptr || workspace_bytes < need || ((uintptr_t)workspace & 255) != 0) return RAD_EWORKSPACE;
+    const TileTwin t = redrawn_twin(st, static_cast<char*>(workspace));
+    rcd = launch_store_index(&t.st, false, dev_status, static_cast<cudaStream_t>(stream));
+    if (rcd != RAD_OK) return rcd;
+    return weight_grad_and_bias(&t.st, dZ, ldz, H, dW, ldw, static_cast<char*>(workspace) + t.bytes, workspace_bytes - t.bytes,
+                                dev_status, stream, db, db_written);
+  }
+  if (!store_args_ok(st) || dZ == nullptr || dW == nullptr || H <= 0 || ldz < H || ldw < H) return RAD_EINVAL;
+  int rc = check_device();
+  if (rc != RAD_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (st->dtype == RAD_BF16 && tc_shape_ok(st->B, st->D, H, dZ, ldz, st->values, 8) &&
+      ((uintptr_t)dW & 15) == 0 && ldw % 4 == 0) {
+    if (workspace_bytes < tc_weight_grad_workspace(st, H) || (workspace == nullptr && tc_weight_grad_workspace(st, H) > 0))
+      return RAD_EWORKSPACE;
+    return tc_weight_grad(st, dZ, ldz, H, dW, ldw, workspace, workspace_bytes, dev_status, s);
+  }
+  return simt_weight_grad(st, dZ, ldz, H, dW, ldw, dev_status, s, db, db_written);
+}
+}  // namespace
+}  // namespace rad
+
 extern "C" int rad_weight_grad_workspace(const rad_store* st, int64_t H, int64_t* bytes) {
   if (st == nullptr || bytes == nullptr || H <= 0 || st->B <= 0 || st->D <= 0) return RAD_EINVAL;
   if (st->variant == RAD_PROJECT) {
@@ -255,32 +293,7 @@ extern "C" int rad_linear_weight_grad(const rad_store* st, const void* dZ, int64
     return rad_linear_weight_grad(&t.st, dZ, ldz, H, dW, ldw, static_cast<char*>(workspace) + t.bytes, workspace_bytes - t.bytes,
                                   dev_status, stream);
   }
-  if (st != nullptr && st->variant == RAD_REDRAWN_SAMPLE) {
-    // the index part from the key alone, into the workspace; then the contraction of a different-sample store
-    if (!redrawn_args_ok(st) || dZ == nullptr || dW == nullptr || H <= 0 || ldz < H || ldw < H) return RAD_EINVAL;
-    int rcd = check_device();
-    if (rcd != RAD_OK) return rcd;
-    int64_t need = 0;
-    rcd = rad_weight_grad_workspace(st, H, &need);
-    if (rcd != RAD_OK) return rcd;
-    if (workspace == nullptr || workspace_bytes < need || ((uintptr_t)workspace & 255) != 0) return RAD_EWORKSPACE;
-    const TileTwin t = redrawn_twin(st, static_cast<char*>(workspace));
-    rcd = launch_store_index(&t.st, false, dev_status, static_cast<cudaStream_t>(stream));
-    if (rcd != RAD_OK) return rcd;
-    return rad_linear_weight_grad(&t.st, dZ, ldz, H, dW, ldw, static_cast<char*>(workspace) + t.bytes, workspace_bytes - t.bytes,
-                                  dev_status, stream);
-  }
-  if (!store_args_ok(st) || dZ == nullptr || dW == nullptr || H <= 0 || ldz < H || ldw < H) return RAD_EINVAL;
-  int rc = check_device();
-  if (rc != RAD_OK) return rc;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (st->dtype == RAD_BF16 && tc_shape_ok(st->B, st->D, H, dZ, ldz, st->values, 8) &&
-      ((uintptr_t)dW & 15) == 0 && ldw % 4 == 0) {
-    if (workspace_bytes < tc_weight_grad_workspace(st, H) || (workspace == nullptr && tc_weight_grad_workspace(st, H) > 0))
-      return RAD_EWORKSPACE;
-    return tc_weight_grad(st, dZ, ldz, H, dW, ldw, workspace, workspace_bytes, dev_status, s);
-  }
-  return simt_weight_grad(st, dZ, ldz, H, dW, ldw, dev_status, s);
+  return weight_grad_and_bias(st, dZ, ldz, H, dW, ldw, workspace, workspace_bytes, dev_status, stream, nullptr, nullptr);
 }
 
 extern "C" int rad_linear_forward(int32_t dtype, int32_t act, int64_t B, int64_t D, int64_t H, const void* A,
@@ -360,11 +373,14 @@ extern "C" int rad_linear_forward_fill(int32_t dtype, int32_t act, int64_t B, in
     return tc_forward(act, B, D, H, A, lda, W, ldw, bias, out_act, ld_act, nullptr, 0, out_zlow, ld_zlow, relubits,
                       dev_status, s, next);
   // shapes the fused epilogue does not take: the same results from the two separate calls
+  // Where the forward runs on the CUDA cores its ReLU bits would be one more launch: there they come from the
+  // store kernels, which look at every entry anyway (not from the projection store, which does not).
+  const bool bits_from_store = next->variant != RAD_PROJECT && !(dtype == RAD_BF16 && tc_shape_ok(B, D, H, A, lda, W, ldw));
   rc = rad_linear_forward(dtype, act, B, D, H, A, lda, W, ldw, bias, out_act, ld_act, nullptr, 0, out_zlow, ld_zlow,
-                          relubits, dev_status, stream);
+                          bits_from_store ? nullptr : relubits, dev_status, stream);
   if (rc != RAD_OK) return rc;
   rad_store tmp = *next;
-  tmp.relubits = nullptr;                           // the bits of out_act were written by the forward call
+  tmp.relubits = bits_from_store ? relubits : nullptr;
   return rad_linear_forward_store(out_act, ld_act, &tmp, workspace, workspace_bytes, dev_status, stream);
 }
 
@@ -493,14 +509,20 @@ extern "C" int rad_mlp_step(const rad_mlp_desc* net, const void* X, const int32_
   if (rc != RAD_OK) return rc;
   for (int l = L - 1; l >= 0; --l) {
     const int64_t D = net->dims[l], H = net->dims[l + 1];
-    rc = rad_linear_weight_grad(&st[l], dz, H, H, dW[l], H, ws + plan.scratch, plan.scratch_bytes, dev_status,
-                                stream);
+    bool db_done = false;
+    if (net->variant == RAD_DIFFERENT_SAMPLE || net->variant == RAD_SAME_SAMPLE || net->variant == RAD_REDRAWN_SAMPLE)
+      rc = weight_grad_and_bias(&st[l], dz, H, H, dW[l], H, ws + plan.scratch, plan.scratch_bytes, dev_status, stream, db[l],
+                                &db_done);
+    else
+      rc = rad_linear_weight_grad(&st[l], dz, H, H, dW[l], H, ws + plan.scratch, plan.scratch_bytes, dev_status, stream);
     if (rc != RAD_OK) return rc;
     void* dz_prev = l > 0 ? ws + plan.dz[(l - 1) & 1] : nullptr;
-    rc = rad_linear_input_grad(net->dtype, B, D, H, dz, H, W[l], H, st[l].relubits,
-                               plan.layer[l].preact >= 0 ? ws + plan.layer[l].preact : nullptr, D, dz_prev, D,
-                               db[l], ws + plan.scratch, plan.scratch_bytes, dev_status, stream);
-    if (rc != RAD_OK) return rc;
+    if (dz_prev != nullptr || !db_done) {
+      rc = rad_linear_input_grad(net->dtype, B, D, H, dz, H, W[l], H, st[l].relubits,
+                                 plan.layer[l].preact >= 0 ? ws + plan.layer[l].preact : nullptr, D, dz_prev, D,
+                                 db_done ? nullptr : db[l], ws + plan.scratch, plan.scratch_bytes, dev_status, stream);
+      if (rc != RAD_OK) return rc;
+    }
     dz = dz_prev;
   }
   return RAD_OK;

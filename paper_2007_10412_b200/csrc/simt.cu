@@ -144,6 +144,7 @@ struct SparseDwParams {
   int64_t B, D, H; int32_t ncb, nslabs;
   const void* dZ; int64_t ldz;
   float* dW; int64_t ldw;
+  float* db;                 // or NULL: column sums of dZ (the bias gradient), from the CTAs of column block 0
 };
 
 template <typename T>
@@ -159,6 +160,7 @@ __global__ void __launch_bounds__(256) sparse_dw_kernel(const SparseDwParams p) 
   // 128 x 32 outputs over 256 threads: 4 columns d x 4 outputs h each
   const int td = (tid >> 3) * 4, th = (tid & 7) * 4;
   float acc[4][4] = {};
+  float db_acc = 0.0f;
   for (int slab = 0; slab < p.nslabs; ++slab) {
     const int64_t tile = (int64_t)slab * p.ncb + cb;
     const uint32_t word = p.keepbits[tile * kTileWords + tid];    // row tid/4, word tid%4
@@ -192,6 +194,12 @@ __global__ void __launch_bounds__(256) sparse_dw_kernel(const SparseDwParams p) 
       sZ[rr][hh] = (row < p.B && h < p.H) ? to_float(dZ[row * p.ldz + h]) : 0.0f;
     }
     __syncthreads();
+    if (p.db != nullptr && cb == 0 && tid < kSparseBN) {
+      // the dZ block is in shared memory anyway: its column sums, slab after slab in row order
+      float sum = 0.0f;
+      for (int rr = 0; rr < kTileRows; ++rr) sum += sZ[rr][tid];
+      db_acc += sum;
+    }
 #pragma unroll 4
     for (int rr = 0; rr < kTileRows; ++rr) {
       float a[4], z[4];
@@ -206,6 +214,7 @@ __global__ void __launch_bounds__(256) sparse_dw_kernel(const SparseDwParams p) 
     }
     __syncthreads();
   }
+  if (p.db != nullptr && cb == 0 && tid < kSparseBN && h0 + tid < p.H) p.db[h0 + tid] = db_acc;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int64_t d = (int64_t)cb * kTileCols + td + i;
@@ -305,8 +314,9 @@ int simt_input_grad(int dtype, int64_t B, int64_t D, int64_t H, const void* dZ, 
 }
 
 int simt_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H, float* dW,
-                     int64_t ldw, int32_t* dev_status, cudaStream_t s) {
+                     int64_t ldw, int32_t* dev_status, cudaStream_t s, float* db, bool* db_written) {
   (void)dev_status;
+  if (db_written != nullptr) *db_written = false;
   if (st->variant == RAD_SAME_SAMPLE) {
     const int g = (int)std::min<int64_t>(ceil_div(st->D * H, 256), 148 * 16);
     count_launch();
@@ -325,6 +335,8 @@ int simt_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H
   p.B = st->B; p.D = st->D; p.H = H;
   p.ncb = (int32_t)ceil_div(st->D, kTileCols); p.nslabs = (int32_t)ceil_div(st->B, kTileRows);
   p.dZ = dZ; p.ldz = ldz; p.dW = dW; p.ldw = ldw;
+  p.db = db;
+  if (db_written != nullptr) *db_written = db != nullptr;
   dim3 grid((unsigned)p.ncb, (unsigned)ceil_div(H, kSparseBN));
   count_launch();
   if (st->dtype == RAD_BF16)
