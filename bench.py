@@ -841,7 +841,7 @@ def run_ours(args):
                     config=dict(workload=f"mlp_wide: 8192->8192x4->1000, bf16, batch {B} per GPU, N(0,1) inputs",
                                 dims=list(dims), global_batch=world * B, act=args.act, variant=args.variant, law=args.law, p=args.p,
                                 p_sampled=pe, parallelism="replicas" if world > 1 else "1 GPU",
-                                l2="inputs larger than L2 (1 GiB activations per layer)"),
+                                l2="inputs larger than L2 (1 GiB activations per layer)", sm_pairs=rad.rad_sm_pairs()),
                     clocks=clocks, e2e=e2e, gpu_launches=int(launches), roofline=roofline,
                     family_ms={k: round(v, 3) for k, v in by_family.items()},
                     activation_memory=memory, relu_twin=twin, cpu_baseline=cpu, kernel_sweep=sweep, small_workloads=small)

@@ -524,6 +524,11 @@ int rad_wait_probe(int32_t which, uint64_t limit_ns, int32_t* dev_status /* devi
 /* Kernels this library has launched since it was loaded (host-side tally; memsets not counted). */
 int64_t rad_launch_count(void);
 
+/* Clusters of two CTAs (SM pairs) the tensor-core kernels keep resident on the current device: the width the
+ * K splits of a weight gradient are planned for.  74 on a B200 whose 148 SMs all pair up, fewer on a part with an
+ * odd SM count in some GPC; 74 where there is no device to ask. */
+int32_t rad_sm_pairs(void);
+
 const char* rad_strerror(int code);
 const char* rad_version(void);
 

@@ -73,7 +73,7 @@ EXPORTS = ["rad_keep_threshold", "rad_effective_p", "rad_scale", "rad_store_size
            "rad_draws_per_row", "rad_replace_scale", "rad_store_size_query_law", "rad_rademacher",
            "rad_linear_forward_store", "rad_linear_forward_store_static", "rad_weight_grad_workspace", "rad_linear_weight_grad",
            "rad_linear_forward", "rad_store_index", "rad_linear_forward_fill", "rad_softmax_xent", "rad_input_grad_workspace", "rad_linear_input_grad",
-           "rad_mlp_workspace", "rad_mlp_held_bytes", "rad_mlp_step", "rad_irnn_workspace", "rad_irnn_step", "rad_cnn_workspace", "rad_cnn_step", "rad_launch_count", "rad_strerror", "rad_version",
+           "rad_mlp_workspace", "rad_mlp_held_bytes", "rad_mlp_step", "rad_irnn_workspace", "rad_irnn_step", "rad_cnn_workspace", "rad_cnn_step", "rad_launch_count", "rad_sm_pairs", "rad_strerror", "rad_version",
            "rad_set_wait_limit_ns", "rad_wait_probe", "rad_set_conv_kernel"]
 
 _lib = None
@@ -169,6 +169,11 @@ def rad_scale(p):
 
 def rad_launch_count():
     return int(lib().rad_launch_count())
+
+
+def rad_sm_pairs():
+    """SM pairs the tensor-core kernels keep resident on the current device (74 where there is none to ask)."""
+    return int(lib().rad_sm_pairs())
 
 
 def rad_version():

@@ -164,6 +164,7 @@ int make_plan(const rad_mlp_desc* net, StepPlan* plan) {
 using namespace rad;
 
 extern "C" int64_t rad_launch_count(void) { return g_launches; }
+extern "C" int32_t rad_sm_pairs(void) { return sm_pairs(); }
 
 extern "C" uint64_t rad_set_wait_limit_ns(uint64_t limit_ns) {
   const uint64_t prev = g_wait_limit_ns;

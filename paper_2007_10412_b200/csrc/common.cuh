@@ -275,5 +275,6 @@ int tc_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H, 
                    int64_t ldw, void* workspace, int64_t workspace_bytes, int32_t* dev_status,
                    cudaStream_t s);
 int64_t tc_weight_grad_workspace(const rad_store* st, int64_t H);
+int sm_pairs();   // SM pairs the dW plans count on (see rad_sm_pairs)
 
 }  // namespace rad

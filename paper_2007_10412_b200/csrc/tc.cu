@@ -1061,6 +1061,46 @@ int choose_splits(int64_t m_tiles, int64_t n_tiles, int64_t kblocks, int64_t bm 
 
 struct DwPlan { int splits; int64_t partial_rows; int64_t bytes; int comp_cap; int stages; int comp_depth; };
 
+// Clusters of two CTAs of `kernel` that can be resident at once.
+template <typename K>
+int resident_pairs_of(K kernel, int threads, size_t smem) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * (num_sms() / 2));
+  cfg.blockDim = dim3(threads);
+  cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n <= 0) {
+    (void)cudaGetLastError();
+    n = num_sms() / 2;
+  }
+  return std::min(n, num_sms() / 2);
+}
+
+// SM pairs the K splits of a dW contraction are planned for: what the device can really keep resident (a part
+// whose SM count per GPC is odd somewhere hosts fewer two-CTA clusters than half its SMs, and a plan for 74
+// pairs on 72 runs an extra wave), or half the default SM count where there is no device to ask (size queries
+// on a host without one).  Found once, so that workspace queries and launches agree.
+int planning_pairs() {
+  static int pairs = 0;
+  if (pairs == 0) {
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess && major == 10 &&
+        cudaFuncSetAttribute(tc_sparse_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess) {
+      pairs = resident_pairs_of(tc_sparse_pair_kernel, kSpThreads, 227 * 1024);
+    } else {
+      (void)cudaGetLastError();
+      pairs = kNumSMsDefault / 2;
+    }
+  }
+  return pairs;
+}
+
 DwPlan plan_dw(const rad_store* st, int64_t H) {
   DwPlan d;
   const int64_t kblocks = ceil_div(st->B, BK);
@@ -1074,7 +1114,7 @@ DwPlan plan_dw(const rad_store* st, int64_t H) {
     d.comp_depth = 0;
     const int64_t n_tiles = ceil_div(m_expect, BN);
     const int64_t bn = round_up(ceil_div(m_expect, n_tiles), 16);
-    d.splits = choose_splits(ceil_div(H, BM), n_tiles, kblocks, BM, kNumSMsDefault / 2, bn, (double)bn / BN);
+    d.splits = choose_splits(ceil_div(H, BM), n_tiles, kblocks, BM, planning_pairs(), bn, (double)bn / BN);
     d.bytes = d.splits > 1 ? (int64_t)d.splits * d.partial_rows * H * 4 : 0;
     return d;
   } else {
@@ -1090,7 +1130,7 @@ DwPlan plan_dw(const rad_store* st, int64_t H) {
     const int64_t slot = kIndexBytes + d.comp_cap;
     d.stages = (4 * kSpStageBytes + 3 * slot <= budget) ? 4 : (3 * kSpStageBytes + 2 * slot <= budget) ? 3 : 2;
     d.comp_depth = (int)std::max<int64_t>(2, std::min<int64_t>(8, (budget - d.stages * kSpStageBytes) / slot));
-    d.splits = choose_splits(ceil_div(m_expect, kSpBM), ceil_div(H, kSpBN), kblocks, kSpBM, kNumSMsDefault / 2, kSpBN);
+    d.splits = choose_splits(ceil_div(m_expect, kSpBM), ceil_div(H, kSpBN), kblocks, kSpBM, planning_pairs(), kSpBN);
     d.bytes = d.splits > 1 ? (int64_t)d.splits * d.partial_rows * H * 4 : 0;
     return d;
   }
@@ -1126,26 +1166,6 @@ int launch_pair(const TcParams& p, const CUtensorMap& ta, const CUtensorMap& tb,
   count_launch();
   kernel<<<2 * pairs, kThreads2, smem, s>>>(p, ta, tb);
   return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
-}
-
-// Clusters of two CTAs of `kernel` that can be resident at once.
-template <typename K>
-int resident_pairs_of(K kernel, int threads, size_t smem) {
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(2 * (num_sms() / 2));
-  cfg.blockDim = dim3(threads);
-  cfg.dynamicSmemBytes = smem;
-  cudaLaunchAttribute attr;
-  attr.id = cudaLaunchAttributeClusterDimension;
-  attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
-  cfg.attrs = &attr;
-  cfg.numAttrs = 1;
-  int n = 0;
-  if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n <= 0) {
-    (void)cudaGetLastError();
-    n = num_sms() / 2;
-  }
-  return std::min(n, num_sms() / 2);
 }
 
 int launch_sparse_pair(const TcParams& p, const CUtensorMap& tb, int64_t max_units, cudaStream_t s) {
@@ -1225,6 +1245,8 @@ int tc_input_grad(int64_t B, int64_t D, int64_t H, const void* dZ, int64_t ldz, 
   p.wait_limit_ns = wait_limit_ns();
   return launch_pair<kAK, kBK_, kDx>(p, ta, tb, ceil_div(B, BM) * ceil_div(D, BN), s);
 }
+
+int sm_pairs() { return planning_pairs(); }
 
 int64_t tc_weight_grad_workspace(const rad_store* st, int64_t H) {
   if (st->dtype != RAD_BF16 || st->D % 8 != 0 || H % 8 != 0 || st->B < 64 || st->D < 64 || H < 64) return 0;

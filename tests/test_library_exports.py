@@ -54,6 +54,7 @@ def test_host_only_entry_points():
     with pytest.raises(b.RadError):
         b.rad_store_size_query("same", "f32", 150, 784, 0.0)
     assert b.lib().rad_strerror(-4).decode() == "workspace too small"
+    assert 1 <= b.rad_sm_pairs() <= 74
     # held without its keep bits: same values and offsets, no keep-bit words, the index of one layer in the workspace
     full = b.rad_store_size_query("different", "bf16", 65536, 8192, 0.1)
     held = b.rad_store_size_query("redrawn", "bf16", 65536, 8192, 0.1)
