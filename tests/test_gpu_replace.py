@@ -141,3 +141,30 @@ def test_fixed_count_law_at_fraction_one_is_exact_backprop(variant):
     assert status.item() == 0 and st.nnz.cpu().numpy()[0] == (B * D if variant == "different" else D)
     fro, mx = rel_err(dW.cpu().numpy(), A.astype(np.float64).T @ dZ.astype(np.float64))
     assert fro <= 1e-5 and mx <= 1e-5
+
+
+@pytest.mark.parametrize("store_kernel", ["auto", "pipelined"], indirect=True)
+@pytest.mark.parametrize("law,variant", [("fixed", "different"), ("replace", "different"), ("bernoulli", "redrawn")])
+def test_a_short_values_buffer_is_reported_and_nothing_is_written_past_it(law, variant, store_kernel):
+    """The routes that place values into an index made from the key alone: with room for a part of the tiles
+    only, the call reports it, the counts stay exact, the tiles that fit hold the oracle's values and nothing
+    is written past the declared capacity."""
+    import paper_2007_10412_b200 as rad
+    B, D, f, dtype = 1000, 1160, 0.1, "bf16"
+    A, _ = layer_inputs(B, D, 1, dtype=dtype, seed=5)
+    ref = orc.forward_store(A, dtype, "different", f, 9, 1, 2, law=law, with_relu_bits=False)
+    _, vals, offs = tile_major(ref)
+    declared = int(offs[len(offs) // 2]) + 8            # about half of the tiles fit
+    st = rad.Store(variant, dtype, B, D, f, seed=9, layer=1, step=2, relu_bits=False, capacity="worst", law=law)
+    st.c.values_capacity = declared
+    st.values.fill_(float("nan"))
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    rad.rad_linear_forward_store(to_dev(A, dtype), st, status)
+    torch.cuda.synchronize()
+    assert status.item() == rad.RAD_DEV_ECAPACITY
+    nnz = st.nnz.cpu().numpy()
+    assert nnz[0] == ref.nnz and nnz[1] == offs[-1]
+    got = bits_host(st.values)
+    fits = int(max(o for o in offs if o <= declared))
+    assert np.array_equal(got[:fits], bits_of(vals, dtype)[:fits])
+    assert torch.isnan(st.values[declared:].float()).all()
