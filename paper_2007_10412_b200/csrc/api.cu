@@ -1,6 +1,8 @@
 // C ABI entry points that route to the kernels, and the whole-net step (Sec. 4.2 for arbitrary
 // depth: every layer input is stored through its own mask, dW_l comes from store l, the rest of
 // backprop is exact).
+#include <nvtx3/nvToolsExt.h>
+
 #include "common.cuh"
 
 namespace rad {
@@ -24,6 +26,14 @@ static uint64_t g_wait_limit_ns = 2000000000ull;   // 2 s: far beyond any legiti
 uint64_t wait_limit_ns() { return g_wait_limit_ns; }
 
 namespace {
+
+// Named range on the host timeline for a profiler that is attached (header-only NVTX: a no-op otherwise).
+struct TraceRange {
+  explicit TraceRange(const char* name) { nvtxRangePushA(name); }
+  ~TraceRange() { nvtxRangePop(); }
+  TraceRange(const TraceRange&) = delete;
+  TraceRange& operator=(const TraceRange&) = delete;
+};
 
 bool valid_dtype(int d) { return d == RAD_F32 || d == RAD_BF16; }
 int64_t esize(int dtype) { return dtype == RAD_BF16 ? 2 : 4; }
@@ -476,11 +486,16 @@ extern "C" int rad_mlp_step(const rad_mlp_desc* net, const void* X, const int32_
   }
   // the network input is stored by the stand-alone kernel; every hidden layer's input is stored from the
   // epilogue of the GEMM that produces it (or by the same stand-alone call where that kernel does not apply)
-  rc = rad_linear_forward_store(X, net->dims[0], &st[0], ws + plan.scratch, plan.scratch_bytes, dev_status, stream);
+  TraceRange step_range("rad_mlp_step");
+  {
+    TraceRange r("store input");
+    rc = rad_linear_forward_store(X, net->dims[0], &st[0], ws + plan.scratch, plan.scratch_bytes, dev_status, stream);
+  }
   if (rc != RAD_OK) return rc;
   const void* a_in = X;
   int64_t ld_in = net->dims[0];
   for (int l = 0; l < L; ++l) {
+    TraceRange r("forward layer");
     const int64_t D = net->dims[l], H = net->dims[l + 1];
     const bool last = (l == L - 1);
     if (last) {
@@ -509,6 +524,7 @@ extern "C" int rad_mlp_step(const rad_mlp_desc* net, const void* X, const int32_
                         C, ws + plan.scratch, plan.scratch_bytes, stream);
   if (rc != RAD_OK) return rc;
   for (int l = L - 1; l >= 0; --l) {
+    TraceRange r("backward layer");
     const int64_t D = net->dims[l], H = net->dims[l + 1];
     bool db_done = false;
     if (net->variant == RAD_DIFFERENT_SAMPLE || net->variant == RAD_SAME_SAMPLE || net->variant == RAD_REDRAWN_SAMPLE)

@@ -18,7 +18,8 @@ namespace rad {
 namespace {
 
 constexpr int kHdMax = 128;          // hidden units per CTA row (one thread each)
-constexpr int kRnnThreads = 160;     // 4 unit warps + 1 helper warp
+constexpr int kRnnThreads = 160;     // backward: 4 unit warps + 1 helper warp
+constexpr int kRnnFwdThreads = 192;  // forward: 4 unit warps, the store warp, the warp that draws the masks
 
 struct RnnParams {
   int64_t B, T;
@@ -42,14 +43,14 @@ struct RnnParams {
   int32_t* dev_status;
 };
 
-__global__ void __launch_bounds__(kRnnThreads) irnn_forward_kernel(const RnnParams p, const PhiloxKeys ks) {
+__global__ void __launch_bounds__(kRnnFwdThreads) irnn_forward_kernel(const RnnParams p, const PhiloxKeys ks) {
   extern __shared__ float sm[];
   float* s_x = sm;                                   // T inputs of this row
   __shared__ __align__(16) float s_h[2][kHdMax];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int64_t b = blockIdx.x;
   const int Hd = p.Hd;
-  for (int64_t t = tid; t < p.T; t += kRnnThreads) s_x[t] = p.x[b * p.T + t];
+  for (int64_t t = tid; t < p.T; t += kRnnFwdThreads) s_x[t] = p.x[b * p.T + t];
   if (tid < kHdMax) { s_h[0][tid] = 0.0f; s_h[1][tid] = 0.0f; }
   // unit j keeps column j of W_hh in registers (zero beyond Hd)
   float wcol[kHdMax];
@@ -60,20 +61,33 @@ __global__ void __launch_bounds__(kRnnThreads) irnn_forward_kernel(const RnnPara
     for (int k = 0; k < kHdMax; ++k) wcol[k] = (k < Hd && j < Hd) ? p.W_hh[(int64_t)k * Hd + j] : 0.0f;
     if (j < Hd) { bias = p.b_ih[j] + p.b_hh[j]; wih = p.W_ih[j]; }
   }
-  __syncthreads();
-  uint32_t off = 0;                                  // helper warp: values of this row so far
+  // The keep decisions need no data: the sixth warp draws the words of step t + 2 while step t runs (one
+  // keep-bit word decides 32 units; four lanes make it together, one generator output each).
+  __shared__ uint32_t s_mask[4][8];
   const uint32_t mask_row = p.same ? 0u : (uint32_t)b;
+  auto draw = [&](int64_t t) {
+    const uint32_t m = philox_keep32_quad((uint32_t)(lane >> 2), mask_row, p.c2, p.step0 + (uint32_t)t, ks, p.keepT, lane);
+    if ((lane & 3) == 0) s_mask[t & 3][lane >> 2] = m;
+  };
+  if (warp == 5) {
+    draw(1);
+    if (p.T >= 2) draw(2);
+  }
+  __syncthreads();
+  uint32_t off = 0;                                  // store warp: values of this row so far
   for (int64_t t = 1; t <= p.T; ++t) {
     const float* hc = s_h[(t - 1) & 1];
-    if (warp == 4) {
+    if (warp == 5) {
+      if (t + 2 <= p.T) draw(t + 2);
+    } else if (warp == 4) {
       // store of h_{t-1}: keep bits of the step, kept entries scaled and appended to the row's values
-      // one keep-bit word decides 32 units; four lanes make it together (one generator output each, which
-      // keeps this warp off the critical path of the step) and the first of them goes on with it
-      const int wi = lane >> 2;
-      uint32_t m = philox_keep32_quad((uint32_t)wi, mask_row, p.c2, p.step0 + (uint32_t)t, ks, p.keepT, lane);
-      if ((lane & 3) == 0 && wi * 32 < Hd) m &= 0xffffffffu >> (32 - min(32, Hd - wi * 32));
-      else m = 0;
-      const uint32_t c = __popc(m);
+      // four lanes share a keep-bit word and place eight of its units each
+      const int wi = lane >> 2, q = lane & 3;
+      uint32_t m = s_mask[t & 3][wi];
+      const bool word_ok = wi * 32 < Hd;
+      m = word_ok ? m & (0xffffffffu >> (32 - min(32, Hd - wi * 32))) : 0u;
+      // the word's count enters the scan once (first lane of the four); every lane then places a quarter of it
+      const uint32_t c = q == 0 ? __popc(m) : 0u;
       uint32_t incl = c;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
@@ -81,16 +95,25 @@ __global__ void __launch_bounds__(kRnnThreads) irnn_forward_kernel(const RnnPara
         if (lane >= o) incl += n;
       }
       const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
-      uint32_t pos = off + incl - c;
+      const uint32_t word_pos = __shfl_sync(0xffffffffu, off + incl - c, lane & ~3);
       if ((int64_t)off + total <= p.cap_row) {
+        // units 8 q .. 8 q + 7 of the word: loaded whether kept or not (two 16-byte loads instead of up to
+        // eight dependent ones), stored where kept
+        const uint32_t sub = (m >> (8 * q)) & 0xffu;
+        if (sub != 0) {
+          const float4 lo = *reinterpret_cast<const float4*>(hc + wi * 32 + 8 * q);
+          const float4 hi = *reinterpret_cast<const float4*>(hc + wi * 32 + 8 * q + 4);
+          const float v[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+          float* out = p.values + b * p.cap_row + word_pos + __popc(m & ((1u << (8 * q)) - 1u));
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if ((m >> i) & 1u) p.values[b * p.cap_row + pos++] = hc[wi * 32 + i] * p.scale;
+          for (int i = 0; i < 8; ++i)
+            if ((sub >> i) & 1u) *out++ = v[i] * p.scale;
+        }
       } else if (lane == 0) {
         raise_status(p.dev_status, RAD_DEV_ECAPACITY);
       }
       const int64_t sb = (t - 1) * p.B + b;
-      if ((lane & 3) == 0 && wi < p.w32) p.keepbits[sb * p.w32 + wi] = m;
+      if (q == 0 && wi < p.w32) p.keepbits[sb * p.w32 + wi] = m;
       if (lane == 0) p.offsets[sb] = off;
       off += total;
     } else {
@@ -128,8 +151,8 @@ __global__ void __launch_bounds__(kRnnThreads) irnn_backward_kernel(const RnnPar
   uint32_t* s_rl = s_keep + p.T * p.w32;              // T x w32 ReLU bits
   uint32_t* s_off = s_rl + p.T * p.w32;               // T value offsets
   __shared__ __align__(16) float s_dz[kHdMax];
-  __shared__ uint32_t s_kidx[kRing][kHdMax];
-  __shared__ float s_kval[kRing][kHdMax];
+  __shared__ __align__(16) uint32_t s_kidx[kRing][kHdMax];
+  __shared__ __align__(16) float s_kval[kRing][kHdMax];
   __shared__ uint32_t s_kcnt[kRing];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int64_t b = blockIdx.x;
@@ -193,10 +216,7 @@ __global__ void __launch_bounds__(kRnnThreads) irnn_backward_kernel(const RnnPar
   __syncthreads();
   for (int64_t t = p.T; t >= 1; --t) {
     const int slot = (int)(t % kRing);
-    if (warp == 4) {
-      prefetch(t - (kRing - 1));
-      asm volatile("cp.async.wait_group %0;" ::"n"(kRing - 2) : "memory");    // step t - 1 has landed
-    } else {
+    if (warp < 4) {
       // dz_t = dh_t * relu'(h_t); exact gradients of the input weights and biases
       const uint32_t rbits = warp < p.w32 ? s_rl[(t - 1) * p.w32 + warp] : 0u;
       const float dz = ((rbits >> lane) & 1u) ? dh : 0.0f;
@@ -222,11 +242,27 @@ __global__ void __launch_bounds__(kRnnThreads) irnn_backward_kernel(const RnnPar
       if (k < Hd) {
         const float dzj = s_dz[k];
         const uint32_t cnt = s_kcnt[slot];
-        for (uint32_t n = 0; n < cnt; ++n) {
+        uint32_t n = 0;
+        // four kept units at a time: their rows of dW_hh are different, so the four updates do not wait
+        // for one another
+        for (; n + 4 <= cnt; n += 4) {
+          const uint4 id = *reinterpret_cast<const uint4*>(&s_kidx[slot][n]);
+          const float4 hv = *reinterpret_cast<const float4*>(&s_kval[slot][n]);
+          float* c0 = s_dw + id.x * S + k; float* c1 = s_dw + id.y * S + k;
+          float* c2 = s_dw + id.z * S + k; float* c3 = s_dw + id.w * S + k;
+          const float x0 = *c0, x1 = *c1, x2 = *c2, x3 = *c3;
+          *c0 = fmaf(hv.x, dzj, x0); *c1 = fmaf(hv.y, dzj, x1);
+          *c2 = fmaf(hv.z, dzj, x2); *c3 = fmaf(hv.w, dzj, x3);
+        }
+        for (; n < cnt; ++n) {
           float* cell = s_dw + s_kidx[slot][n] * S + k;
           *cell = fmaf(s_kval[slot][n], dzj, *cell);
         }
       }
+    } else {
+      // beside the long phase of the step: the list of a later step (its ring slot was read a step ago)
+      prefetch(t - (kRing - 1));
+      asm volatile("cp.async.wait_group %0;" ::"n"(kRing - 2) : "memory");    // step t - 1 has landed
     }
     __syncthreads();
   }
@@ -365,7 +401,7 @@ extern "C" int rad_irnn_step(const rad_irnn_desc* d, const float* x, const int32
   RAD_CUDA_TRY(cudaFuncSetAttribute(irnn_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)std::max<size_t>(smem_f, 1024)));
   RAD_CUDA_TRY(cudaFuncSetAttribute(irnn_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_b));
   count_launch();
-  irnn_forward_kernel<<<(unsigned)d->B, kRnnThreads, smem_f, s>>>(p, ks);
+  irnn_forward_kernel<<<(unsigned)d->B, kRnnFwdThreads, smem_f, s>>>(p, ks);
   RAD_CUDA_TRY(cudaGetLastError());
 
   // output layer on the last hidden state: sampled like any other layer input (layer index 1)
