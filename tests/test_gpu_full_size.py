@@ -182,6 +182,30 @@ def test_weight_grad_sampled_entries(wide):
     check_weight_grad_entries(wide["rad"], wide["st"], wide["A"], wide["dZ"], wide["dev"]["dZ"], P, wide["status"])
 
 
+def test_store_without_held_keep_bits_at_full_size(wide):
+    """The variant that holds no keep bits, through the pipelined store with its index in the workspace and the
+    index drawn again for dW: the same offsets, counts and values as the store that holds its index (which the
+    tests above check against the oracle), dW on the oracle's sampled entries and identical to the other dW."""
+    rad, dev, status = wide["rad"], wide["dev"], wide["status"]
+    held = rad.Store("redrawn", "bf16", B, D, P, seed=SEED, layer=LAYER, step=STEP, relu_bits=False)
+    assert held.keepbits.numel() == 0
+    rad.rad_linear_forward_store(dev["A"], held, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    full = wide["st"]
+    assert torch.equal(held.offsets, full.offsets) and torch.equal(held.nnz, full.nnz)
+    used = int(full.nnz.cpu()[1])
+    assert torch.equal(held.values[:used].view(torch.int16), full.values[:used].view(torch.int16))
+    check_weight_grad_entries(rad, held, wide["A"], wide["dZ"], dev["dZ"], P, status)
+    dW_a = torch.empty(D, H, dtype=torch.float32, device="cuda")
+    dW_b = torch.empty(D, H, dtype=torch.float32, device="cuda")
+    rad.rad_linear_weight_grad(held, dev["dZ"], dW_a, dev_status=status)
+    rad.rad_linear_weight_grad(full, dev["dZ"], dW_b, dev_status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0 and torch.equal(dW_a, dW_b)
+    del dW_a, dW_b, held
+
+
 def test_forward_and_input_grad_sampled_entries(wide):
     rad, dev, A, W, bias, dZ = wide["rad"], wide["dev"], wide["A"], wide["W"], wide["bias"], wide["dZ"]
     act = torch.empty(B, H, dtype=torch.bfloat16, device="cuda")
