@@ -433,7 +433,7 @@ def kernel_sweep(rad, torch, A, dZ, H, ps, pk, clock):
             rows.append(row)
             del st, ws
     # the paper's own law (k = ceil(fraction D) draws with replacement) and the fixed-count law without
-    # replacement: multiplicity kernel + store, then the same weight-gradient kernels on the store it leaves
+    # replacement: index from the key alone + fill, then the same weight-gradient kernels on the store it leaves
     for law, variant in (("replace", "different"), ("replace", "same"), ("fixed", "different"), ("fixed", "same")):
         p = 0.1
         st = rad.Store(variant, "bf16", B, D, p, relu_bits=False, law=law)
@@ -444,9 +444,8 @@ def kernel_sweep(rad, torch, A, dZ, H, ps, pk, clock):
         row = dict(variant=variant, law=law, p=p, draws_per_row=rad.rad_draws_per_row(p, D), nnz=int(nnz[0]),
                    store_ms=round(ms_store, 4), store_sm_mhz=mhz, dW_ms=round(ms_dw, 4))
         if variant == "different":
-            # with replacement: the multiplicity matrix (a byte per entry) is written and read once on top of the
-            # store's bytes; the fixed-count law makes its index from the key alone and needs no such matrix
-            sb = store_bytes_different(B, D, int(nnz[1]), len(st.offsets), extra=2 * B * D if law == "replace" else 0)
+            # both laws make their index from the key alone: the algorithmic bytes are those of any bitmask store
+            sb = store_bytes_different(B, D, int(nnz[1]), len(st.offsets))
             row.update(store_bytes=sb, store_gbs=round(sb / ms_store / 1e6, 1), store_frac_hbm=frac(sb / ms_store / 1e6, hbm),
                        held_bytes=int(nnz[1]) * 2 + (len(st.keepbits) + len(st.offsets)) * 4,
                        dW_tflops_dense_tile=round(2.0 * B * D * H / ms_dw / 1e9, 1),
