@@ -219,7 +219,10 @@ extern "C" int rad_cnn_step(const rad_cnn_desc* d, const void* X, const int32_t*
     if (rc != RAD_OK) return rc;
     if (l > 0) {
       void* g_prev = ws + pl.grad[(l - 1) & 1];
-      rc = conv_input_grad(d->dtype, B, pl.H[l], pl.W[l], pl.Cin[l], pl.Cout[l], dz, conv_W[l], g_prev, s);
+      if (conv_tc_dx_ok(d->dtype, pl.H[l], pl.W[l], pl.Cin[l], pl.Cout[l], dz, conv_W[l], g_prev))
+        rc = conv_tc_input_grad(B, pl.H[l], pl.W[l], pl.Cin[l], pl.Cout[l], dz, conv_W[l], g_prev, dev_status, s);
+      else
+        rc = conv_input_grad(d->dtype, B, pl.H[l], pl.W[l], pl.Cin[l], pl.Cout[l], dz, conv_W[l], g_prev, s);
       if (rc != RAD_OK) return rc;
       g = g_prev;
     }

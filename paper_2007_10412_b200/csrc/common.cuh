@@ -248,6 +248,9 @@ int conv_tc_forward_pool(int64_t B, int H, int W, int Cin, int Cout, const void*
 int64_t conv_tc_weight_grad_workspace(int64_t B, int H, int W, int Cin, int Cout);
 int conv_tc_weight_grad(const rad_store* store, int H, int W, int Cin, int Cout, const void* dZ, float* dW, void* workspace,
                         int64_t workspace_bytes, int32_t* dev_status, cudaStream_t st);
+bool conv_tc_dx_ok(int dtype, int H, int W, int Cin, int Cout, const void* dZ, const void* Wt, const void* dX);
+int conv_tc_input_grad(int64_t B, int H, int W, int Cin, int Cout, const void* dZ, const void* Wt, void* dX, int32_t* dev_status,
+                       cudaStream_t st);
 
 // tcgen05 kernels (bf16, aligned)
 bool tc_shape_ok(int64_t B, int64_t D, int64_t H, const void* p0, int64_t ld0, const void* p1,

@@ -12,6 +12,11 @@
 //                    MN-major (the contraction index is the slow index of both tensors).  A_hat is the sampled
 //                    conv input, expanded from its compact store into a zero-filled NHWC buffer of one layer
 //                    (held only while this layer's gradient is formed).  Partial tiles are summed in split order.
+//   input gradient   dX[pixel, ci] = sum over (tap, co) of dZ[pixel - tap, co] W[tap, ci, co] (the transposed
+//                    convolution, exact): M = input pixels in raster order, N = Cin (padded to 64), K = 9 Cout taken
+//                    64 at a time; the A tile is the patch matrix of dZ with the taps mirrored, K-major as in the
+//                    forward pass; B is K-major too (for a tap and an input channel the output channels are
+//                    contiguous in the filter tensor); the epilogue rounds and writes 64 bytes per row and chunk.
 //
 // One CTA (no cluster), eight warps: all of them write operand tiles with the 128-byte swizzle the tensor core
 // expects (16-byte chunk c of row r lands at chunk c ^ (r & 7)), thread 0 issues tcgen05.mma.cta_group::1
@@ -36,7 +41,7 @@ struct ConvTcParams {
   const bf16* X;            // forward: conv input; filter gradient: A_hat (zero where dropped), both NHWC dense
   const bf16* Wt;           // 3 x 3 x Cin x Cout
   const float* bias;
-  bf16* P;                  // pooled output
+  bf16* P;                  // pooled output; input gradient: dX, B x H x W x Cin
   uint32_t* relubits;
   const bf16* dZ;           // B x H x W x Cout
   float* partial;           // splits x (9 Cin) x Cout
@@ -120,9 +125,12 @@ __device__ __forceinline__ uint4 cv_load_pixel(const bf16* T, int64_t b, int y, 
   return __ldg(reinterpret_cast<const uint4*>(T + ((b * H + y) * W + x) * C + c0));
 }
 
-// kDw false: forward tile `blockIdx.x` (128 output pixels); true: filter-gradient unit (m tile, split) = blockIdx
-template <bool kDw>
+// kCvFwd: forward tile `blockIdx.x` (128 output pixels); kCvDw: filter-gradient unit (m tile, split) = blockIdx;
+// kCvDx: input-gradient tile `blockIdx.x` (128 input pixels in raster order)
+enum { kCvFwd = 0, kCvDw = 1, kCvDx = 2 };
+template <int kMode>
 __global__ void __launch_bounds__(kCvThreads) conv_tc_kernel(const ConvTcParams p) {
+  constexpr bool kDw = kMode == kCvDw, kDx = kMode == kCvDx;
   extern __shared__ uint8_t cv_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(cv_raw) + 1023) & ~(uintptr_t)1023);
   CvCtl* ctl = reinterpret_cast<CvCtl*>(smem + 2 * kCvStageBytes);
@@ -149,7 +157,7 @@ __global__ void __launch_bounds__(kCvThreads) conv_tc_kernel(const ConvTcParams 
   // what this CTA contracts over
   const int mtile = kDw ? (int)blockIdx.x : 0, split = kDw ? (int)blockIdx.y : 0;
   const int64_t tile = kDw ? 0 : blockIdx.x;
-  const int nkb = kDw ? p.kblocks_per_split : (ktaps + kCvK - 1) / kCvK;
+  const int nkb = kDw ? p.kblocks_per_split : ((kDx ? 9 * Cout : ktaps) + kCvK - 1) / kCvK;
   const int64_t kb0 = kDw ? (int64_t)split * p.kblocks_per_split : 0;
   bool ok = true;
   for (int kb = 0; kb < nkb; ++kb) {
@@ -159,7 +167,30 @@ __global__ void __launch_bounds__(kCvThreads) conv_tc_kernel(const ConvTcParams 
     // the MMAs of two K blocks ago have read this stage
     if (kb >= 2) ok = cv_wait(cv_smem(&ctl->done[s]), ((kb >> 1) - 1) & 1, abort_flag, p.wait_limit_ns);
     if (!__syncthreads_and(ok ? 1 : 0)) { ok = false; break; }
-    if (!kDw) {
+    if (kDx) {
+      // A: K-major patch tile of dZ, row m = input pixel tile * 128 + m, k = (tap, co): the output pixel that
+      // reached this input pixel through tap (ty, tx) lies at (y - ty + 1, x - tx + 1)
+      for (int c = tid; c < kCvM * 8; c += kCvThreads) {
+        const int m = c >> 3, cc = c & 7;
+        const int k0 = kb * kCvK + cc * 8, tap = k0 / Cout, co0 = k0 - tap * Cout;
+        const int64_t pix = tile * kCvM + m;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (tap < 9 && pix < npix) {
+          const int x = (int)(pix % W), y = (int)((pix / W) % H);
+          const int64_t b = pix / ((int64_t)W * H);
+          v = cv_load_pixel(p.dZ, b, y - tap / 3 + 1, x - tap % 3 + 1, H, W, Cout, co0);
+        }
+        *reinterpret_cast<uint4*>(sA + m * 128 + ((cc ^ (m & 7)) << 4)) = v;
+      }
+      // B: K-major, row n = input channel, k = (tap, co): W[tap, n, co0 .. co0 + 7] is contiguous
+      for (int c = tid; c < kCvN * 8; c += kCvThreads) {
+        const int n = c >> 3, cc = c & 7;
+        const int k0 = kb * kCvK + cc * 8, tap = k0 / Cout, co0 = k0 - tap * Cout;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (tap < 9 && n < Cin) v = __ldg(reinterpret_cast<const uint4*>(p.Wt + ((int64_t)tap * Cin + n) * Cout + co0));
+        *reinterpret_cast<uint4*>(sB + n * 128 + ((cc ^ (n & 7)) << 4)) = v;
+      }
+    } else if (!kDw) {
       // A: K-major patch tile, row m = window (tile * 32 + m / 4), pixel m % 4 of it; 8 chunks of 8 k per row
       for (int c = tid; c < kCvM * 8; c += kCvThreads) {
         const int m = c >> 3, cc = c & 7;
@@ -209,12 +240,13 @@ __global__ void __launch_bounds__(kCvThreads) conv_tc_kernel(const ConvTcParams 
     __syncthreads();
     if (tid == 0) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      constexpr uint32_t idesc = cv_idesc(kDw, true);
+      constexpr uint32_t idesc = cv_idesc(kDw, !kDx);
       const uint32_t a0 = cv_smem(sA), b0 = cv_smem(sB);
 #pragma unroll
       for (int k = 0; k < kCvK / 16; ++k) {
         const uint64_t adesc = kDw ? cv_desc(a0 + k * 2048, 8192, 1024) : cv_desc(a0 + k * 32, 16, 1024);
-        cv_mma(tmem, adesc, cv_desc(b0 + k * 2048, 8192, 1024), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+        const uint64_t bdesc = kDx ? cv_desc(b0 + k * 32, 16, 1024) : cv_desc(b0 + k * 2048, 8192, 1024);
+        cv_mma(tmem, adesc, bdesc, idesc, (kb > 0 || k > 0) ? 1u : 0u);
       }
       cv_commit(cv_smem(&ctl->done[s]));
     }
@@ -228,7 +260,25 @@ __global__ void __launch_bounds__(kCvThreads) conv_tc_kernel(const ConvTcParams 
     const int m = q * 32 + lane;
     uint32_t r[32];
     cv_tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(chunk * 32), r);
-    if (!kDw) {
+    if (kDx) {
+      // row m = input pixel, columns = input channels: rounded once, 64 bytes per row and chunk
+      const int64_t pix = tile * kCvM + m;
+      if (pix < npix) {
+        bf16* dst = p.P + pix * Cin + chunk * 32;
+#pragma unroll
+        for (int j = 0; j < 32; j += 8) {
+          if (chunk * 32 + j < Cin) {
+            uint32_t w[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(r[j + 2 * e]), __uint_as_float(r[j + 2 * e + 1]));
+              w[e] = *reinterpret_cast<const uint32_t*>(&h2);
+            }
+            *reinterpret_cast<uint4*>(dst + j) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+    } else if (!kDw) {
       // rows 4 w .. 4 w + 3 are the 2 x 2 window w: bias, ReLU, derivative bits, rounded average
       const int64_t win = tile * 32 + (m >> 2);
       const bool win_ok = win < npix / 4;
@@ -333,10 +383,31 @@ int conv_tc_forward_pool(int64_t B, int H, int W, int Cin, int Cout, const void*
   p.B = B; p.H = H; p.W = W; p.Cin = Cin; p.Cout = Cout;
   p.X = static_cast<const bf16*>(X); p.Wt = static_cast<const bf16*>(Wt); p.bias = bias;
   p.P = static_cast<bf16*>(P); p.relubits = relubits; p.dev_status = dev_status; p.wait_limit_ns = wait_limit_ns();
-  RAD_CUDA_TRY(cudaFuncSetAttribute(conv_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCvSmem));
+  RAD_CUDA_TRY(cudaFuncSetAttribute(conv_tc_kernel<kCvFwd>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCvSmem));
   const int64_t windows = B * (H / 2) * (W / 2);
   count_launch();
-  conv_tc_kernel<false><<<(unsigned)ceil_div(windows, 32), kCvThreads, kCvSmem, st>>>(p);
+  conv_tc_kernel<kCvFwd><<<(unsigned)ceil_div(windows, 32), kCvThreads, kCvSmem, st>>>(p);
+  return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
+}
+
+// Shapes the input-gradient kernel takes: as above with the channel counts in each other's roles (K runs over
+// (tap, co) in chunks of eight output channels, N over the input channels).
+bool conv_tc_dx_ok(int dtype, int H, int W, int Cin, int Cout, const void* dZ, const void* Wt, const void* dX) {
+  (void)H; (void)W;
+  if (g_conv_kernel == RAD_CONV_KERNEL_SIMT) return false;
+  return dtype == RAD_BF16 && (Cout == 16 || Cout == 32 || Cout == 64) && Cin % 8 == 0 && Cin >= 8 && Cin <= kCvN &&
+         ((uintptr_t)dZ & 15) == 0 && ((uintptr_t)Wt & 15) == 0 && ((uintptr_t)dX & 15) == 0;
+}
+
+int conv_tc_input_grad(int64_t B, int H, int W, int Cin, int Cout, const void* dZ, const void* Wt, void* dX, int32_t* dev_status,
+                       cudaStream_t st) {
+  ConvTcParams p = {};
+  p.B = B; p.H = H; p.W = W; p.Cin = Cin; p.Cout = Cout;
+  p.dZ = static_cast<const bf16*>(dZ); p.Wt = static_cast<const bf16*>(Wt); p.P = static_cast<bf16*>(dX);
+  p.dev_status = dev_status; p.wait_limit_ns = wait_limit_ns();
+  RAD_CUDA_TRY(cudaFuncSetAttribute(conv_tc_kernel<kCvDx>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCvSmem));
+  count_launch();
+  conv_tc_kernel<kCvDx><<<(unsigned)ceil_div(B * H * W, kCvM), kCvThreads, kCvSmem, st>>>(p);
   return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
 }
 
@@ -376,9 +447,9 @@ int conv_tc_weight_grad(const rad_store* store, int H, int W, int Cin, int Cout,
   p.X = dense; p.dZ = static_cast<const bf16*>(dZ); p.partial = partial; p.dev_status = dev_status;
   p.wait_limit_ns = wait_limit_ns();
   const int splits = conv_tc_splits(B * H * W, &p.kblocks_per_split);
-  RAD_CUDA_TRY(cudaFuncSetAttribute(conv_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCvSmem));
+  RAD_CUDA_TRY(cudaFuncSetAttribute(conv_tc_kernel<kCvDw>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCvSmem));
   count_launch(2);
-  conv_tc_kernel<true><<<dim3((unsigned)ceil_div(9 * Cin, kCvM), (unsigned)splits), kCvThreads, kCvSmem, st>>>(p);
+  conv_tc_kernel<kCvDw><<<dim3((unsigned)ceil_div(9 * Cin, kCvM), (unsigned)splits), kCvThreads, kCvSmem, st>>>(p);
   const int64_t n = (int64_t)9 * Cin * Cout;
   conv_tc_reduce_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(partial, splits, n, dW);
   return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
