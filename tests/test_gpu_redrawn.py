@@ -58,8 +58,10 @@ def test_store_and_weight_grad_without_held_keep_bits(B, D, H, dtype, p, law):
     assert full.held_bytes()["index_bytes"] == 4 * (len(offs) + 288 * (len(offs) - 1))
 
 
-@pytest.mark.parametrize("name,act", [("mlp_small_different", "relu"), ("mlp_wide_cut", "relu"), ("mlp_wide_cut", "gelu")])
-def test_step_without_held_keep_bits_equals_the_step_that_holds_them(name, act):
+@pytest.mark.parametrize("name,act,law", [("mlp_small_different", "relu", "bernoulli"), ("mlp_wide_cut", "relu", "bernoulli"),
+                                          ("mlp_wide_cut", "gelu", "bernoulli"), ("mlp_wide_cut", "relu", "fixed"),
+                                          ("mlp_small_different", "relu", "fixed")])
+def test_step_without_held_keep_bits_equals_the_step_that_holds_them(name, act, law):
     """rad_mlp_step with variant "redrawn": the hidden layers' stores come out of the forward epilogue with
     their index in the scratch area, the backward pass draws every index again; loss and all gradients equal
     those of the different-sample step bit for bit, the oracle's within tolerance, and the index bytes held
@@ -71,7 +73,7 @@ def test_step_without_held_keep_bits_equals_the_step_that_holds_them(name, act):
     dWs, dbs = [to_dev(W, cfg.dtype) for W in Ws], [to_dev(b, "f32") for b in bs]
     out = {}
     for variant in ("different", "redrawn"):
-        ctx = rad.MLPStep(cfg.dims, cfg.batch, cfg.dtype, act, variant, 0.1)
+        ctx = rad.MLPStep(cfg.dims, cfg.batch, cfg.dtype, act, variant, 0.1, law=law)
         ctx.workspace.fill_(0x5A)
         ctx(dX, dy, dWs, dbs, seed=11, step=3)
         torch.cuda.synchronize()
@@ -81,7 +83,7 @@ def test_step_without_held_keep_bits_equals_the_step_that_holds_them(name, act):
     assert torch.equal(a.loss, b.loss) and torch.equal(a.nnz, b.nnz)
     for l in range(len(cfg.dims) - 1):
         assert torch.equal(a.dW[l], b.dW[l]) and torch.equal(a.db[l], b.db[l]), l
-    ref = orc.mlp_step(X, y, Ws, bs, act=act, dtype=cfg.dtype, variant="different", p=0.1, seed=11, step=3)
+    ref = orc.mlp_step(X, y, Ws, bs, act=act, dtype=cfg.dtype, variant="different", p=0.1, seed=11, step=3, law=law)
     for l in range(len(cfg.dims) - 1):
         fro, mx = rel_err(to_host_f32(b.dW[l]), ref.dW[l])
         assert fro <= TOL[cfg.dtype] and mx <= TOL[cfg.dtype], (l, fro, mx)
