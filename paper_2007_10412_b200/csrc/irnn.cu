@@ -150,7 +150,7 @@ __global__ void __launch_bounds__(kRnnThreads) irnn_backward_kernel(const RnnPar
   uint32_t* s_keep = reinterpret_cast<uint32_t*>(s_dw + ((Hd * S + 3) & ~3));   // T x w32 keep bits of the row
   uint32_t* s_rl = s_keep + p.T * p.w32;              // T x w32 ReLU bits
   uint32_t* s_off = s_rl + p.T * p.w32;               // T value offsets
-  __shared__ __align__(16) float s_dz[kHdMax];
+  __shared__ __align__(16) float s_dz[2][kHdMax];
   __shared__ __align__(16) uint32_t s_kidx[kRing][kHdMax];
   __shared__ __align__(16) float s_kval[kRing][kHdMax];
   __shared__ uint32_t s_kcnt[kRing];
@@ -166,7 +166,7 @@ __global__ void __launch_bounds__(kRnnThreads) irnn_backward_kernel(const RnnPar
     s_rl[i] = p.relubits[at];
   }
   for (int i = tid; i < Hd * S; i += kRnnThreads) s_dw[i] = 0.0f;
-  if (tid < kHdMax) s_dz[tid] = 0.0f;
+  if (tid < kHdMax) { s_dz[0][tid] = 0.0f; s_dz[1][tid] = 0.0f; }
   const int k = tid;                                  // unit k: row k of W_hh in registers
   float wrow[kHdMax];
   float dh = 0.0f, dwih = 0.0f, dbs = 0.0f, dwih_c = 0.0f, dbs_c = 0.0f;
@@ -213,34 +213,37 @@ __global__ void __launch_bounds__(kRnnThreads) irnn_backward_kernel(const RnnPar
     for (int d = 0; d < kRing - 1; ++d) prefetch(p.T - d);
     asm volatile("cp.async.wait_group %0;" ::"n"(kRing - 2) : "memory");      // step T has landed
   }
+  // dz_t = dh_t * relu'(h_t) and the exact gradients of the input weights and biases, by the thread of unit k;
+  // the two buffers of dz alternate, so a step needs one barrier: the dz of step t - 1 is written at the end of
+  // step t while the other threads may still read the dz of step t
+  auto make_dz = [&](int64_t t) {
+    const uint32_t rbits = warp < p.w32 ? s_rl[(t - 1) * p.w32 + warp] : 0u;
+    const float dz = ((rbits >> lane) & 1u) ? dh : 0.0f;
+    s_dz[t & 1][k] = dz;
+    // compensated sums: T terms of one sign would otherwise drift past the float32 tolerance
+    const float yi = fmaf(s_x[t - 1], dz, -dwih_c), ti = dwih + yi;
+    dwih_c = (ti - dwih) - yi; dwih = ti;
+    const float yb = dz - dbs_c, tb = dbs + yb;
+    dbs_c = (tb - dbs) - yb; dbs = tb;
+  };
+  if (warp < 4) make_dz(p.T);
   __syncthreads();
   for (int64_t t = p.T; t >= 1; --t) {
     const int slot = (int)(t % kRing);
     if (warp < 4) {
-      // dz_t = dh_t * relu'(h_t); exact gradients of the input weights and biases
-      const uint32_t rbits = warp < p.w32 ? s_rl[(t - 1) * p.w32 + warp] : 0u;
-      const float dz = ((rbits >> lane) & 1u) ? dh : 0.0f;
-      s_dz[k] = dz;
-      // compensated sums: T terms of one sign would otherwise drift past the float32 tolerance
-      const float yi = fmaf(s_x[t - 1], dz, -dwih_c), ti = dwih + yi;
-      dwih_c = (ti - dwih) - yi; dwih = ti;
-      const float yb = dz - dbs_c, tb = dbs + yb;
-      dbs_c = (tb - dbs) - yb; dbs = tb;
-    }
-    __syncthreads();
-    if (warp < 4) {
+      const float* dzv = s_dz[t & 1];
       // dh_{t-1}[k] = sum_j dz[j] W_hh[k][j]
       float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
 #pragma unroll
       for (int jj = 0; jj < kHdMax; jj += 4) {
-        const float4 d4 = *reinterpret_cast<const float4*>(s_dz + jj);
+        const float4 d4 = *reinterpret_cast<const float4*>(dzv + jj);
         a0 = fmaf(d4.x, wrow[jj], a0); a1 = fmaf(d4.y, wrow[jj + 1], a1);
         a2 = fmaf(d4.z, wrow[jj + 2], a2); a3 = fmaf(d4.w, wrow[jj + 3], a3);
       }
       dh = (a0 + a1) + (a2 + a3);
       // dW_hh[kept unit d, j] += h_hat_{t-1}[d] * dz[j]: thread j owns column j of every row
       if (k < Hd) {
-        const float dzj = s_dz[k];
+        const float dzj = dzv[k];
         const uint32_t cnt = s_kcnt[slot];
         uint32_t n = 0;
         // four kept units at a time: their rows of dW_hh are different, so the four updates do not wait
@@ -259,8 +262,9 @@ __global__ void __launch_bounds__(kRnnThreads) irnn_backward_kernel(const RnnPar
           *cell = fmaf(s_kval[slot][n], dzj, *cell);
         }
       }
+      if (t > 1) make_dz(t - 1);
     } else {
-      // beside the long phase of the step: the list of a later step (its ring slot was read a step ago)
+      // beside the unit warps: the list of a later step (its ring slot was read a step ago)
       prefetch(t - (kRing - 1));
       asm volatile("cp.async.wait_group %0;" ::"n"(kRing - 2) : "memory");    // step t - 1 has landed
     }
