@@ -709,14 +709,20 @@ def run_ours(args):
         kernels["store"] = tensor_entry("projection store S = A R', flops 2*B*D*k", ms_store0, 2.0 * B * 8192 * k)
     dominant = max(("forward", "dW", "dX"), key=lambda f: by_family.get({"dX": "dX+db"}.get(f, f), 0.0))
     dom = kernels[dominant]
-    # DRAM bytes per launch from the ncu captures under profiles/ (batch 8192, 8192 x 8192 layer): bytes read grow
-    # with the batch and are scaled by B / 8192, the dW output does not grow.  Only the default workload has one.
+    # DRAM bytes per launch from the ncu captures under profiles/ (8192 x 8192 layer).  Two captures: one pass of
+    # dram__bytes_read.sum + dram__bytes_write.sum over this very command at batch 65536, and the full set at batch
+    # 8192; bytes read grow a little faster than the batch (the panels of a wave fall out of L2 sooner), so the
+    # full-size figure serves from batch 32768 up and the small one, scaled by B / 8192, below.  The dW output does
+    # not grow with the batch.  Only the default workload has a capture.
     traffic = None
     if args.act == "gelu" and abs(args.p - 0.1) < 1e-9 and args.law == "bernoulli" and args.variant == "different":
+        big = B >= 32768
         if dominant == "forward":
-            traffic = int((1263.5e6 + 269.8e6) * B / 8192)
+            traffic = int((15.37e9 + 2.25e9) * B / 65536) if big else int((1263.5e6 + 269.8e6) * B / 8192)
         elif dominant == "dW":
-            traffic = int(631.7e6 * B / 8192 + 236.0e6)
+            traffic = int(5.27e9 * B / 65536 + 0.25e9) if big else int(631.7e6 * B / 8192 + 236.0e6)
+        elif dominant == "dX":
+            traffic = int((17.68e9 + 1.07e9) * B / 65536) if big else None
     roofline = dict(bound=dom["bound"], kernel=dom["kernel"], achieved=dom["achieved"], peak=dom["peak"], unit=dom["unit"],
                     frac=dom["frac"], traffic=traffic, peak_source=pk["source"] + " (sustained cuBLAS bf16 / copy bandwidth)",
                     ms_per_launch=dom["ms_per_launch"],
