@@ -217,9 +217,20 @@ namespace {
 // rad_linear_weight_grad for a bitmask or column-list store (index held or drawn again); where the contraction
 // runs on the CUDA cores and passes over dZ anyway, it also leaves the bias gradient in `db` (*db_written says
 // whether it did).
+// Does the input gradient of these operands run on the tensor cores?
+bool input_grad_on_tc(int32_t dtype, int64_t B, int64_t D, int64_t H, const void* dZ, int64_t ldz, const void* W,
+                      int64_t ldw, const void* z_prev, int64_t ld_zprev, const void* dZ_prev, int64_t ldp) {
+  return dtype == RAD_BF16 && tc_shape_ok(B, D, H, dZ, ldz, W, ldw) && ((uintptr_t)dZ_prev & 15) == 0 && ldp % 8 == 0 &&
+         (z_prev == nullptr || (((uintptr_t)z_prev & 15) == 0 && ld_zprev % 8 == 0));
+}
+
+// ig (optional): the input gradient of the same layer; where both contractions run on CUDA cores they share one
+// launch and *ig_done is set, otherwise the caller runs rad_linear_input_grad as usual.
 int weight_grad_and_bias(const rad_store* st, const void* dZ, int64_t ldz, int64_t H, float* dW, int64_t ldw, void* workspace,
-                         int64_t workspace_bytes, int32_t* dev_status, void* stream, float* db, bool* db_written) {
+                         int64_t workspace_bytes, int32_t* dev_status, void* stream, float* db, bool* db_written,
+                         const SimtInputGrad* ig = nullptr, bool* ig_done = nullptr) {
   if (db_written != nullptr) *db_written = false;
+  if (ig_done != nullptr) *ig_done = false;
   if (st != nullptr && st->variant == RAD_REDRAWN_SAMPLE) {
     // the index part from the key alone, into the workspace; then the contraction of a different-sample store
     if (!redrawn_args_ok(st) || dZ == nullptr || dW == nullptr || H <= 0 || ldz < H || ldw < H) return RAD_EINVAL;
@@ -233,7 +244,7 @@ int weight_grad_and_bias(const rad_store* st, const void* dZ, int64_t ldz, int64
     rcd = launch_store_index(&t.st, false, dev_status, static_cast<cudaStream_t>(stream));
     if (rcd != RAD_OK) return rcd;
     return weight_grad_and_bias(&t.st, dZ, ldz, H, dW, ldw, static_cast<char*>(workspace) + t.bytes, workspace_bytes - t.bytes,
-                                dev_status, stream, db, db_written);
+                                dev_status, stream, db, db_written, ig, ig_done);
   }
   if (!store_args_ok(st) || dZ == nullptr || dW == nullptr || H <= 0 || ldz < H || ldw < H) return RAD_EINVAL;
   int rc = check_device();
@@ -245,6 +256,9 @@ int weight_grad_and_bias(const rad_store* st, const void* dZ, int64_t ldz, int64
       return RAD_EWORKSPACE;
     return tc_weight_grad(st, dZ, ldz, H, dW, ldw, workspace, workspace_bytes, dev_status, s);
   }
+  if (ig != nullptr && ig->dZ_prev != nullptr && st->variant == RAD_DIFFERENT_SAMPLE &&
+      !input_grad_on_tc(st->dtype, st->B, st->D, H, dZ, ldz, ig->W, ig->ldw, ig->z_prev, ig->ld_zprev, ig->dZ_prev, ig->ldp))
+    return simt_weight_grad(st, dZ, ldz, H, dW, ldw, dev_status, s, db, db_written, ig, ig_done);
   return simt_weight_grad(st, dZ, ldz, H, dW, ldw, dev_status, s, db, db_written);
 }
 }  // namespace
@@ -419,8 +433,7 @@ extern "C" int rad_linear_input_grad(int32_t dtype, int64_t B, int64_t D, int64_
     if (rc != RAD_OK) return rc;
   }
   if (dZ_prev == nullptr) return RAD_OK;
-  if (dtype == RAD_BF16 && tc_shape_ok(B, D, H, dZ, ldz, W, ldw) && ((uintptr_t)dZ_prev & 15) == 0 &&
-      ldp % 8 == 0 && (z_prev == nullptr || (((uintptr_t)z_prev & 15) == 0 && ld_zprev % 8 == 0)))
+  if (input_grad_on_tc(dtype, B, D, H, dZ, ldz, W, ldw, z_prev, ld_zprev, dZ_prev, ldp))
     return tc_input_grad(B, D, H, dZ, ldz, W, ldw, relubits_prev, z_prev, ld_zprev, dZ_prev, ldp, dev_status, s);
   return simt_input_grad(dtype, B, D, H, dZ, ldz, W, ldw, relubits_prev, z_prev, ld_zprev, dZ_prev, ldp, s);
 }
@@ -526,18 +539,20 @@ extern "C" int rad_mlp_step(const rad_mlp_desc* net, const void* X, const int32_
   for (int l = L - 1; l >= 0; --l) {
     TraceRange r("backward layer");
     const int64_t D = net->dims[l], H = net->dims[l + 1];
-    bool db_done = false;
+    bool db_done = false, dx_done = false;
+    void* dz_prev = l > 0 ? ws + plan.dz[(l - 1) & 1] : nullptr;
+    const void* z_prev = plan.layer[l].preact >= 0 ? ws + plan.layer[l].preact : nullptr;
+    const SimtInputGrad ig = {W[l], H, st[l].relubits, z_prev, D, dz_prev, D};
     if (net->variant == RAD_DIFFERENT_SAMPLE || net->variant == RAD_SAME_SAMPLE || net->variant == RAD_REDRAWN_SAMPLE)
       rc = weight_grad_and_bias(&st[l], dz, H, H, dW[l], H, ws + plan.scratch, plan.scratch_bytes, dev_status, stream, db[l],
-                                &db_done);
+                                &db_done, dz_prev != nullptr ? &ig : nullptr, &dx_done);
     else
       rc = rad_linear_weight_grad(&st[l], dz, H, H, dW[l], H, ws + plan.scratch, plan.scratch_bytes, dev_status, stream);
     if (rc != RAD_OK) return rc;
-    void* dz_prev = l > 0 ? ws + plan.dz[(l - 1) & 1] : nullptr;
-    if (dz_prev != nullptr || !db_done) {
-      rc = rad_linear_input_grad(net->dtype, B, D, H, dz, H, W[l], H, st[l].relubits,
-                                 plan.layer[l].preact >= 0 ? ws + plan.layer[l].preact : nullptr, D, dz_prev, D,
-                                 db_done ? nullptr : db[l], ws + plan.scratch, plan.scratch_bytes, dev_status, stream);
+    if ((dz_prev != nullptr && !dx_done) || !db_done) {
+      rc = rad_linear_input_grad(net->dtype, B, D, H, dz, H, W[l], H, st[l].relubits, z_prev, D,
+                                 dx_done ? nullptr : dz_prev, D, db_done ? nullptr : db[l], ws + plan.scratch,
+                                 plan.scratch_bytes, dev_status, stream);
       if (rc != RAD_OK) return rc;
     }
     dz = dz_prev;

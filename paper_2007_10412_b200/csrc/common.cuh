@@ -223,9 +223,18 @@ int simt_forward(int dtype, int act, int64_t B, int64_t D, int64_t H, const void
 int simt_input_grad(int dtype, int64_t B, int64_t D, int64_t H, const void* dZ, int64_t ldz,
                     const void* W, int64_t ldw, const uint32_t* relubits_prev, const void* z_prev,
                     int64_t ld_zprev, void* dZ_prev, int64_t ldp, cudaStream_t s);
+// The operands of an input gradient dZ_prev = (dZ W^T) * act'(.) that go with a dW of the same layer.
+struct SimtInputGrad {
+  const void* W; int64_t ldw;
+  const uint32_t* relubits_prev; const void* z_prev; int64_t ld_zprev;
+  void* dZ_prev; int64_t ldp;
+};
+// db: also the column sums of dZ, where the kernel can.  ig: also the input gradient, in the same launch, where
+// the kernel can (*ig_done says whether it did).
 int simt_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H, float* dW,
                      int64_t ldw, int32_t* dev_status, cudaStream_t s,
-                     float* db = nullptr, bool* db_written = nullptr);   // db: also the column sums of dZ, where the kernel can
+                     float* db = nullptr, bool* db_written = nullptr,
+                     const SimtInputGrad* ig = nullptr, bool* ig_done = nullptr);
 int column_sums(int dtype, int64_t B, int64_t H, const void* dZ, int64_t ldz, float* db,
                 void* workspace, int64_t workspace_bytes, cudaStream_t s);
 int64_t column_sums_workspace(int64_t B, int64_t H);

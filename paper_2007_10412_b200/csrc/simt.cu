@@ -33,13 +33,13 @@ struct GemmParams {
   float* out_f32; int64_t ld_f32;
 };
 
+// One 64 x 64 tile of C by one CTA of 256 threads; (bx, by) = tile column and row.
 template <typename T, int EPI>
-__global__ void __launch_bounds__(256) gemm_kernel(const GemmParams p) {
-  __shared__ float sA[kBK][kBM + 4];
-  __shared__ float sB[kBK][kBN + 4];
+__device__ __forceinline__ void gemm_body(const GemmParams& p, int64_t bx, int64_t by, float (*sA)[kBM + 4],
+                                          float (*sB)[kBN + 4]) {
   int64_t M = p.M;
   if (p.M_dev != nullptr) M = min(M, *p.M_dev);
-  const int64_t m0 = (int64_t)blockIdx.y * kBM, n0 = (int64_t)blockIdx.x * kBN;
+  const int64_t m0 = by * kBM, n0 = bx * kBN;
   if (m0 >= M) return;
   const int tid = threadIdx.x;
   const int tm = (tid >> 4) * 4, tn = (tid & 15) * 4;
@@ -105,6 +105,13 @@ __global__ void __launch_bounds__(256) gemm_kernel(const GemmParams p) {
   }
 }
 
+template <typename T, int EPI>
+__global__ void __launch_bounds__(256) gemm_kernel(const GemmParams p) {
+  __shared__ float sA[kBK][kBM + 4];
+  __shared__ float sB[kBK][kBN + 4];
+  gemm_body<T, EPI>(p, blockIdx.x, blockIdx.y, sA, sB);
+}
+
 template <int EPI>
 int launch_gemm(int dtype, const GemmParams& p, int64_t Mgrid, cudaStream_t s) {
   dim3 grid((unsigned)ceil_div(p.N, kBN), (unsigned)ceil_div(Mgrid, kBM));
@@ -148,13 +155,10 @@ struct SparseDwParams {
 };
 
 template <typename T>
-__global__ void __launch_bounds__(256) sparse_dw_kernel(const SparseDwParams p) {
-  __shared__ float sAh[kTileRows][kTileCols + 1];
-  __shared__ float sZ[kTileRows][kSparseBN + 1];
-  __shared__ uint32_t s_scan[256];
+__device__ __forceinline__ void sparse_dw_body(const SparseDwParams& p, int cb, int64_t by, float (*sAh)[kTileCols + 1],
+                                               float (*sZ)[kSparseBN + 1], uint32_t* s_scan) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int cb = blockIdx.x;
-  const int64_t h0 = (int64_t)blockIdx.y * kSparseBN;
+  const int64_t h0 = by * kSparseBN;
   const T* vals = static_cast<const T*>(p.values);
   const T* dZ = static_cast<const T*>(p.dZ);
   // 128 x 32 outputs over 256 threads: 4 columns d x 4 outputs h each
@@ -224,6 +228,34 @@ __global__ void __launch_bounds__(256) sparse_dw_kernel(const SparseDwParams p) 
       const int64_t h = h0 + th + j;
       if (h < p.H) p.dW[d * p.ldw + h] = acc[i][j];
     }
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) sparse_dw_kernel(const SparseDwParams p) {
+  __shared__ float sAh[kTileRows][kTileCols + 1];
+  __shared__ float sZ[kTileRows][kSparseBN + 1];
+  __shared__ uint32_t s_scan[256];
+  sparse_dw_body<T>(p, (int)blockIdx.x, blockIdx.y, sAh, sZ, s_scan);
+}
+
+// dW of a layer and the gradient of its input in one launch: both read the same dZ and neither reads the
+// other's result, so the first `dw_blocks` CTAs are those of sparse_dw_kernel and the rest those of the
+// input-gradient GEMM, each doing exactly what it does in a launch of its own (the nets that run on CUDA
+// cores are bound by their launch count).
+constexpr int kDwDxSmemA = kTileRows * (kTileCols + 1) * 4, kDwDxSmemZ = kTileRows * (kSparseBN + 1) * 4;
+static_assert(kDwDxSmemA + kDwDxSmemZ + 1024 >= 2 * kBK * (kBM + 4) * 4 && kBM == kBN, "the GEMM's tiles fit the same buffer");
+template <typename T>
+__global__ void __launch_bounds__(256) dw_dx_kernel(const SparseDwParams d, const GemmParams g, int dw_blocks, int gx) {
+  __shared__ __align__(16) unsigned char raw[kDwDxSmemA + kDwDxSmemZ + 1024];
+  if ((int)blockIdx.x < dw_blocks) {
+    sparse_dw_body<T>(d, (int)(blockIdx.x % d.ncb), blockIdx.x / d.ncb, reinterpret_cast<float(*)[kTileCols + 1]>(raw),
+                      reinterpret_cast<float(*)[kSparseBN + 1]>(raw + kDwDxSmemA),
+                      reinterpret_cast<uint32_t*>(raw + kDwDxSmemA + kDwDxSmemZ));
+  } else {
+    const int b = (int)blockIdx.x - dw_blocks;
+    gemm_body<T, kEpiInputGrad>(g, b % gx, b / gx, reinterpret_cast<float(*)[kBM + 4]>(raw),
+                                reinterpret_cast<float(*)[kBN + 4]>(raw + kBK * (kBM + 4) * 4));
   }
 }
 
@@ -300,23 +332,32 @@ int simt_forward(int dtype, int act, int64_t B, int64_t D, int64_t H, const void
   return RAD_OK;
 }
 
+namespace {
+GemmParams input_grad_params(int64_t B, int64_t D, int64_t H, const void* dZ, int64_t ldz, const SimtInputGrad& ig) {
+  GemmParams p = {};
+  p.A = dZ; p.sam = ldz; p.sak = 1;          // (b, h)
+  p.Bm = ig.W; p.sbk = 1; p.sbn = ig.ldw;    // Bm(h, d) = W[d, h]
+  p.M = B; p.N = D; p.K = H;
+  p.relubits = ig.relubits_prev; p.w32 = ceil_div(D, 32);
+  p.z_prev = ig.z_prev; p.ld_zprev = ig.ld_zprev;
+  p.out_low = ig.dZ_prev; p.ld_low = ig.ldp;
+  return p;
+}
+}  // namespace
+
 int simt_input_grad(int dtype, int64_t B, int64_t D, int64_t H, const void* dZ, int64_t ldz,
                     const void* W, int64_t ldw, const uint32_t* relubits_prev, const void* z_prev,
                     int64_t ld_zprev, void* dZ_prev, int64_t ldp, cudaStream_t s) {
-  GemmParams p = {};
-  p.A = dZ; p.sam = ldz; p.sak = 1;          // (b, h)
-  p.Bm = W; p.sbk = 1; p.sbn = ldw;          // Bm(h, d) = W[d, h]
-  p.M = B; p.N = D; p.K = H;
-  p.relubits = relubits_prev; p.w32 = ceil_div(D, 32);
-  p.z_prev = z_prev; p.ld_zprev = ld_zprev;
-  p.out_low = dZ_prev; p.ld_low = ldp;
-  return launch_gemm<kEpiInputGrad>(dtype, p, B, s);
+  const SimtInputGrad ig = {W, ldw, relubits_prev, z_prev, ld_zprev, dZ_prev, ldp};
+  return launch_gemm<kEpiInputGrad>(dtype, input_grad_params(B, D, H, dZ, ldz, ig), B, s);
 }
 
 int simt_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H, float* dW,
-                     int64_t ldw, int32_t* dev_status, cudaStream_t s, float* db, bool* db_written) {
+                     int64_t ldw, int32_t* dev_status, cudaStream_t s, float* db, bool* db_written,
+                     const SimtInputGrad* ig, bool* ig_done) {
   (void)dev_status;
   if (db_written != nullptr) *db_written = false;
+  if (ig_done != nullptr) *ig_done = false;
   if (st->variant == RAD_SAME_SAMPLE) {
     const int g = (int)std::min<int64_t>(ceil_div(st->D * H, 256), 148 * 16);
     count_launch();
@@ -339,6 +380,18 @@ int simt_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H
   if (db_written != nullptr) *db_written = db != nullptr;
   dim3 grid((unsigned)p.ncb, (unsigned)ceil_div(H, kSparseBN));
   count_launch();
+  if (ig != nullptr && ig_done != nullptr) {
+    const GemmParams g = input_grad_params(st->B, st->D, H, dZ, ldz, *ig);
+    const int64_t gx = ceil_div(g.N, kBN), gy = ceil_div(g.M, kBM), dw_blocks = (int64_t)grid.x * grid.y;
+    if (dw_blocks + gx * gy <= 0x7fffffff) {
+      if (st->dtype == RAD_BF16)
+        dw_dx_kernel<bf16><<<(unsigned)(dw_blocks + gx * gy), 256, 0, s>>>(p, g, (int)dw_blocks, (int)gx);
+      else
+        dw_dx_kernel<float><<<(unsigned)(dw_blocks + gx * gy), 256, 0, s>>>(p, g, (int)dw_blocks, (int)gx);
+      *ig_done = true;
+      return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
+    }
+  }
   if (st->dtype == RAD_BF16)
     sparse_dw_kernel<bf16><<<grid, 256, 0, s>>>(p);
   else

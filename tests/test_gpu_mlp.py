@@ -126,3 +126,60 @@ def test_step_with_the_projection_variant_matches_oracle(name):
         for got, want in ((ctx.dW[l], ref.dW[l]), (ctx.db[l], ref.db[l])):
             fro, mx = rel_err(to_host_f32(got), want)
             assert fro <= tol and mx <= tol, (l, fro, mx)
+
+
+@pytest.mark.parametrize("name,variant,act,launches", [("mlp_small_different", "different", "relu", 10),
+                                                       ("mlp_small_different", "redrawn", "relu", None),
+                                                       ("mlp_small_different", "different", "gelu", 10)])
+def test_small_net_step_equals_the_layer_calls_and_counts_its_launches(name, variant, act, launches):
+    """On the nets that run on CUDA cores a layer's dW and the gradient of its input share one launch inside
+    rad_mlp_step (Sec. 4.2: both are contractions of the same dZ).  The step's weight gradients and loss equal,
+    bit for bit, those of the same step made of the public layer calls, one launch per contraction; the bias
+    gradients agree to rounding (the step sums them in the dW kernel); and the MNIST-shaped net takes ten launches."""
+    import paper_2007_10412_b200 as rad
+    cfg = get_config(name)
+    dims, B, L = cfg.dims, cfg.batch, len(cfg.dims) - 1
+    X, y, Ws, bs = mlp_inputs(dims, B, cfg.dtype, cfg.x_dist, cfg.data_seed, bias_zero=False)
+    dX, dy = to_dev(X, cfg.dtype), torch.from_numpy(y).cuda()
+    dWs, dbs = [to_dev(W, cfg.dtype) for W in Ws], [to_dev(b, "f32") for b in bs]
+    ctx = rad.MLPStep(dims, B, cfg.dtype, act, variant, 0.1)
+    ctx(dX, dy, dWs, dbs, seed=21, step=5)                      # first call: one-time setup outside the count
+    torch.cuda.synchronize()
+    n0 = rad.rad_launch_count()
+    ctx(dX, dy, dWs, dbs, seed=21, step=5)
+    torch.cuda.synchronize()
+    assert ctx.dev_status.item() == 0
+    if launches is not None:
+        assert rad.rad_launch_count() - n0 == launches
+    # the same step, call by call
+    tdt = dX.dtype
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    stores = [rad.Store("different", cfg.dtype, B, dims[l], 0.1, seed=21, layer=l, step=5, relu_bits=False) for l in range(L)]
+    rbits = [None] + [torch.empty(B * ((dims[l] + 31) // 32), dtype=torch.int32, device="cuda") if act == "relu" else None
+                      for l in range(1, L)]
+    pre = [None] + [torch.empty(B, dims[l], dtype=tdt, device="cuda") if act == "gelu" else None for l in range(1, L)]
+    a = dX
+    rad.rad_linear_forward_store(a, stores[0], status)
+    for l in range(L - 1):
+        out = torch.empty(B, dims[l + 1], dtype=tdt, device="cuda")
+        rad.rad_linear_forward(a, dWs[l], dbs[l], act, out_act=out, out_zlow=pre[l + 1], relubits=rbits[l + 1], dev_status=status)
+        rad.rad_linear_forward_store(out, stores[l + 1], status)
+        a = out
+    logits = torch.empty(B, dims[L], dtype=torch.float32, device="cuda")
+    rad.rad_linear_forward(a, dWs[L - 1], dbs[L - 1], "none", out_z=logits, dev_status=status)
+    loss = torch.zeros(1, dtype=torch.float32, device="cuda")
+    dz = torch.empty(B, dims[L], dtype=tdt, device="cuda")
+    rad.rad_softmax_xent(logits, dy, loss, dz)
+    for l in range(L - 1, -1, -1):
+        dW = torch.full((dims[l], dims[l + 1]), float("nan"), dtype=torch.float32, device="cuda")
+        db = torch.empty(dims[l + 1], dtype=torch.float32, device="cuda")
+        rad.rad_linear_weight_grad(stores[l], dz, dW, dev_status=status)
+        dzp = torch.empty(B, dims[l], dtype=tdt, device="cuda") if l > 0 else None
+        rad.rad_linear_input_grad(dz, dWs[l], relubits_prev=rbits[l], z_prev=pre[l], dZ_prev=dzp, db=db, dev_status=status)
+        torch.cuda.synchronize()
+        assert status.item() == 0
+        assert torch.equal(dW, ctx.dW[l]), l
+        fro, mx = rel_err(to_host_f32(ctx.db[l]), to_host_f32(db).astype(np.float64))
+        assert fro <= 1e-5 and mx <= 1e-5, (l, fro, mx)
+        dz = dzp
+    assert torch.equal(loss, ctx.loss)
