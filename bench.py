@@ -340,10 +340,12 @@ def peaks():
     return dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, sm_max_mhz=1965.0, source="fallback")
 
 
-def timed_alone(torch, fn, clock, n=10, settle_ms=60.0):
+def timed_alone(torch, fn, clock, n=10, settle_ms=60.0, idle_ms=0.0):
     """Median device time of `fn` timed alone (CUDA events on the launching stream) and the median SM clock
     read while the timed launches run.  `fn` first runs for about settle_ms so that the clock is the one
-    this kernel sustains by itself, not what the kernels before it left behind."""
+    this kernel sustains by itself, not what the kernels before it left behind.  idle_ms > 0: the device then
+    rests that long and the timed launches are a burst after one more untimed launch (what a burst peak is
+    compared with: the power cap answers within tens of milliseconds to the contractions before it)."""
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     fn()
     torch.cuda.synchronize()
@@ -351,6 +353,10 @@ def timed_alone(torch, fn, clock, n=10, settle_ms=60.0):
     torch.cuda.synchronize()
     once = max(e0.elapsed_time(e1), 1e-3)
     for _ in range(max(2, min(400, int(settle_ms / once)))):
+        fn()
+    if idle_ms > 0.0:
+        torch.cuda.synchronize()
+        time.sleep(idle_ms / 1e3)
         fn()
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
     ev[0].record()
@@ -390,6 +396,11 @@ def sweep_stores(rad, torch, A, ps, clock):
             if variant == "different":
                 idx_t = timed_alone(torch, lambda: rad.rad_store_index(st, status), clock, n=20, settle_ms=100.0)
             stores[(variant, p)] = (st, ms_store, mhz, idx_t)
+    # the other sampling laws at fraction 0.1, and the static-shape form of the fixed-count law
+    for law, variant in (("replace", "different"), ("replace", "same"), ("fixed", "different"), ("fixed", "same"), ("fixed", "rows")):
+        st = rad.Store(variant, "bf16", B, D, 0.1, relu_bits=False, law=law)
+        ms_store, mhz = timed_alone(torch, lambda: rad.rad_linear_forward_store(A, st, status), clock, n=10, settle_ms=100.0)
+        stores[(variant, law)] = (st, ms_store, mhz, None)
     assert status.item() == 0, f"device status {status.item()}"
     return stores
 
@@ -413,7 +424,7 @@ def kernel_sweep(rad, torch, A, dZ, H, ps, pk, clock, stores):
             nnz = st.nnz.cpu().numpy()
             ws = torch.empty(max(rad.rad_weight_grad_workspace(st, H), 256), dtype=torch.uint8, device="cuda")
             ms_dw, mhz_dw = timed_alone(torch, lambda: rad.rad_linear_weight_grad(st, dZ, dW, ws, status), clock, n=5,
-                                        settle_ms=30.0)
+                                        settle_ms=30.0, idle_ms=150.0)
             row = dict(variant=variant, p=p, p_eff=rad.rad_effective_p(p), nnz=int(nnz[0]), store_ms=round(ms_store, 4),
                        store_sm_mhz=mhz, store_ms_x_mhz=None if mhz is None else round(ms_store * mhz, 1),
                        dW_ms=round(ms_dw, 4), dW_sm_mhz=mhz_dw)
@@ -447,11 +458,10 @@ def kernel_sweep(rad, torch, A, dZ, H, ps, pk, clock, stores):
     # replacement: index from the key alone + fill, then the same weight-gradient kernels on the store it leaves
     for law, variant in (("replace", "different"), ("replace", "same"), ("fixed", "different"), ("fixed", "same")):
         p = 0.1
-        st = rad.Store(variant, "bf16", B, D, p, relu_bits=False, law=law)
-        ms_store, mhz = timed_alone(torch, lambda: rad.rad_linear_forward_store(A, st, status), clock, n=10)
+        st, ms_store, mhz, _ = stores.pop((variant, law))
         nnz = st.nnz.cpu().numpy()
         ws = torch.empty(max(rad.rad_weight_grad_workspace(st, H), 256), dtype=torch.uint8, device="cuda")
-        ms_dw, _ = timed_alone(torch, lambda: rad.rad_linear_weight_grad(st, dZ, dW, ws, status), clock, n=3, settle_ms=20.0)
+        ms_dw, _ = timed_alone(torch, lambda: rad.rad_linear_weight_grad(st, dZ, dW, ws, status), clock, n=3, settle_ms=20.0, idle_ms=150.0)
         row = dict(variant=variant, law=law, p=p, draws_per_row=rad.rad_draws_per_row(p, D), nnz=int(nnz[0]),
                    store_ms=round(ms_store, 4), store_sm_mhz=mhz, dW_ms=round(ms_dw, 4))
         if variant == "different":
@@ -468,10 +478,9 @@ def kernel_sweep(rad, torch, A, dZ, H, ps, pk, clock, stores):
     # the fixed-count law in its static-shape form: B x k values and B x k 16-bit column numbers (k the same for
     # every row); the weight gradient rebuilds the tile-major index from the key and moves the values into it
     p = 0.1
-    st = rad.Store("rows", "bf16", B, D, p, relu_bits=False, law="fixed")
-    ms_store, mhz = timed_alone(torch, lambda: rad.rad_linear_forward_store(A, st, status), clock, n=10)
+    st, ms_store, mhz, _ = stores.pop(("rows", "fixed"))
     ws = torch.empty(max(rad.rad_weight_grad_workspace(st, H), 256), dtype=torch.uint8, device="cuda")
-    ms_dw, _ = timed_alone(torch, lambda: rad.rad_linear_weight_grad(st, dZ, dW, ws, status), clock, n=3, settle_ms=20.0)
+    ms_dw, _ = timed_alone(torch, lambda: rad.rad_linear_weight_grad(st, dZ, dW, ws, status), clock, n=3, settle_ms=20.0, idle_ms=150.0)
     k, ld = rad.rad_draws_per_row(p, D), int(st.c.values_ld)
     # bytes: the 32-byte sectors of A that hold a kept column (about 1 - (1 - k/D)^16 of them), values and columns written
     touched = int(B * D * 2 * (1.0 - (1.0 - k / D) ** 16)) + B * ld * 4
@@ -488,7 +497,7 @@ def kernel_sweep(rad, torch, A, dZ, H, ps, pk, clock, stores):
     k = rad.rad_draws_per_row(p, D)
     ms_store, _ = timed_alone(torch, lambda: rad.rad_linear_forward_store(A, st, status), clock, n=5, settle_ms=20.0)
     ws = torch.empty(max(rad.rad_weight_grad_workspace(st, H), 256), dtype=torch.uint8, device="cuda")
-    ms_dw, _ = timed_alone(torch, lambda: rad.rad_linear_weight_grad(st, dZ, dW, ws, status), clock, n=3, settle_ms=20.0)
+    ms_dw, _ = timed_alone(torch, lambda: rad.rad_linear_weight_grad(st, dZ, dW, ws, status), clock, n=3, settle_ms=20.0, idle_ms=150.0)
     rows.append(dict(variant="project", p=p, k=k, store_ms=round(ms_store, 4),
                      store_tflops=round(2.0 * B * D * k / ms_store / 1e9, 1), dW_ms=round(ms_dw, 4),
                      dW_tflops=round((2.0 * B * k * H + 2.0 * D * k * H) / ms_dw / 1e9, 1), dW_flops="projected",
