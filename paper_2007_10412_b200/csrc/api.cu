@@ -256,7 +256,7 @@ int weight_grad_and_bias(const rad_store* st, const void* dZ, int64_t ldz, int64
       return RAD_EWORKSPACE;
     return tc_weight_grad(st, dZ, ldz, H, dW, ldw, workspace, workspace_bytes, dev_status, s);
   }
-  if (ig != nullptr && ig->dZ_prev != nullptr && st->variant == RAD_DIFFERENT_SAMPLE &&
+  if (ig != nullptr && ig->dZ_prev != nullptr && (st->variant == RAD_DIFFERENT_SAMPLE || st->variant == RAD_SAME_SAMPLE) &&
       !input_grad_on_tc(st->dtype, st->B, st->D, H, dZ, ldz, ig->W, ig->ldw, ig->z_prev, ig->ld_zprev, ig->dZ_prev, ig->ldp))
     return simt_weight_grad(st, dZ, ldz, H, dW, ldw, dev_status, s, db, db_written, ig, ig_done);
   return simt_weight_grad(st, dZ, ldz, H, dW, ldw, dev_status, s, db, db_written);

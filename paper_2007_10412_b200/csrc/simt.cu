@@ -31,6 +31,7 @@ struct GemmParams {
   // scatter-rows epilogue (same-sample dW): row m goes to row idx[m] of out_f32
   const uint32_t* row_idx;
   float* out_f32; int64_t ld_f32;
+  float* db;                   // or NULL: column sums of Bm over k (the bias gradient), from the CTAs of tile row 0
 };
 
 // One 64 x 64 tile of C by one CTA of 256 threads; (bx, by) = tile column and row.
@@ -40,8 +41,10 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, int64_t bx, int64
   int64_t M = p.M;
   if (p.M_dev != nullptr) M = min(M, *p.M_dev);
   const int64_t m0 = by * kBM, n0 = bx * kBN;
-  if (m0 >= M) return;
+  const bool sums = EPI == kEpiScatterRows && p.db != nullptr && by == 0;
+  if (m0 >= M && !sums) return;
   const int tid = threadIdx.x;
+  float colsum = 0.0f;
   const int tm = (tid >> 4) * 4, tn = (tid & 15) * 4;
   const T* A = static_cast<const T*>(p.A);
   const T* Bm = static_cast<const T*>(p.Bm);
@@ -62,6 +65,11 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, int64_t bx, int64
       sB[kk][nn] = (n < p.N && k < p.K) ? to_float(Bm[k * p.sbk + n * p.sbn]) : 0.0f;
     }
     __syncthreads();
+    if (sums && tid < kBN) {
+      // the block of Bm is in shared memory anyway: its column sums, row after row (rows past K hold zeros)
+#pragma unroll
+      for (int kk = 0; kk < kBK; ++kk) colsum += sB[kk][tid];
+    }
 #pragma unroll
     for (int kk = 0; kk < kBK; ++kk) {
       float a[4], b[4];
@@ -74,6 +82,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, int64_t bx, int64
     }
     __syncthreads();
   }
+  if (sums && tid < kBN && n0 + tid < p.N) p.db[n0 + tid] = colsum;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int64_t m = m0 + tm + i;
@@ -305,6 +314,28 @@ __global__ void __launch_bounds__(256) colsum_small_kernel(const T* dZ, int64_t 
 
 }  // namespace
 
+// The same for a same-sample store (Sec. 4.3): the first CTAs scatter A_c^T dZ into the kept rows of dW (and
+// leave the bias gradient), the next ones make the input gradient, the last ones write zeros to the rows of dW
+// whose column was not kept (bit d of keep_cols clear), which the scatter never touches.
+template <typename T>
+__global__ void __launch_bounds__(256) same_dw_dx_kernel(const GemmParams w, const GemmParams g, int dw_blocks, int gxw,
+                                                         int dx_blocks, int gxg, const uint32_t* keep_cols, int64_t D, int64_t H) {
+  __shared__ float sA[kBK][kBM + 4];
+  __shared__ float sB[kBK][kBN + 4];
+  const int b = (int)blockIdx.x;
+  if (b < dw_blocks) {
+    gemm_body<T, kEpiScatterRows>(w, b % gxw, b / gxw, sA, sB);
+  } else if (b < dw_blocks + dx_blocks) {
+    gemm_body<T, kEpiInputGrad>(g, (b - dw_blocks) % gxg, (b - dw_blocks) / gxg, sA, sB);
+  } else {
+    const int nz = (int)gridDim.x - dw_blocks - dx_blocks;
+    for (int64_t d = b - dw_blocks - dx_blocks; d < D; d += nz) {
+      if ((keep_cols[d >> 5] >> (d & 31)) & 1u) continue;
+      for (int64_t h = threadIdx.x; h < H; h += 256) w.out_f32[d * w.ld_f32 + h] = 0.0f;
+    }
+  }
+}
+
 int simt_forward(int dtype, int act, int64_t B, int64_t D, int64_t H, const void* A, int64_t lda,
                  const void* W, int64_t ldw, const float* bias, void* out_act, int64_t ld_act,
                  float* out_z, int64_t ld_z, void* out_zlow, int64_t ld_zlow, uint32_t* relubits,
@@ -359,16 +390,37 @@ int simt_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H
   if (db_written != nullptr) *db_written = false;
   if (ig_done != nullptr) *ig_done = false;
   if (st->variant == RAD_SAME_SAMPLE) {
-    const int g = (int)std::min<int64_t>(ceil_div(st->D * H, 256), 148 * 16);
-    count_launch();
-    zero_rows_kernel<<<g, 256, 0, s>>>(dW, ldw, st->D, H);
     GemmParams p = {};
     p.A = st->values; p.sam = 1; p.sak = st->values_ld;     // A(j, b) = values[b, j]
     p.Bm = dZ; p.sbk = ldz; p.sbn = 1;
     p.M = min(st->values_ld, st->D); p.N = H; p.K = st->B;
     p.M_dev = st->nnz;
     p.row_idx = st->offsets; p.out_f32 = dW; p.ld_f32 = ldw;
-    return launch_gemm<kEpiScatterRows>(st->dtype, p, p.M, s);
+    p.db = db;
+    if (db_written != nullptr) *db_written = db != nullptr;
+    const int64_t gxw = ceil_div(p.N, kBN), dw_blocks = gxw * std::max<int64_t>(1, ceil_div(p.M, kBM));
+    if (st->keepbits != nullptr) {
+      // one launch: scatter, zeros for the rows not kept and, where asked for, the input gradient
+      const bool with_dx = ig != nullptr && ig_done != nullptr;
+      const GemmParams g = with_dx ? input_grad_params(st->B, st->D, H, dZ, ldz, *ig) : GemmParams{};
+      const int64_t gxg = with_dx ? ceil_div(g.N, kBN) : 1, dx_blocks = with_dx ? gxg * ceil_div(g.M, kBM) : 0;
+      const int64_t nz = std::min<int64_t>(st->D, 148 * 4);
+      if (dw_blocks + dx_blocks + nz <= 0x7fffffff) {
+        count_launch();
+        if (st->dtype == RAD_BF16)
+          same_dw_dx_kernel<bf16><<<(unsigned)(dw_blocks + dx_blocks + nz), 256, 0, s>>>(p, g, (int)dw_blocks, (int)gxw, (int)dx_blocks,
+                                                                                          (int)gxg, st->keepbits, st->D, H);
+        else
+          same_dw_dx_kernel<float><<<(unsigned)(dw_blocks + dx_blocks + nz), 256, 0, s>>>(p, g, (int)dw_blocks, (int)gxw, (int)dx_blocks,
+                                                                                           (int)gxg, st->keepbits, st->D, H);
+        if (with_dx) *ig_done = true;
+        return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
+      }
+    }
+    const int g = (int)std::min<int64_t>(ceil_div(st->D * H, 256), 148 * 16);
+    count_launch();
+    zero_rows_kernel<<<g, 256, 0, s>>>(dW, ldw, st->D, H);
+    return launch_gemm<kEpiScatterRows>(st->dtype, p, std::max<int64_t>(p.M, 1), s);
   }
   SparseDwParams p;
   p.values = st->values; p.keepbits = st->keepbits; p.offsets = st->offsets;

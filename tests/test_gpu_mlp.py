@@ -130,12 +130,14 @@ def test_step_with_the_projection_variant_matches_oracle(name):
 
 @pytest.mark.parametrize("name,variant,act,launches", [("mlp_small_different", "different", "relu", 10),
                                                        ("mlp_small_different", "redrawn", "relu", None),
-                                                       ("mlp_small_different", "different", "gelu", 10)])
+                                                       ("mlp_small_different", "different", "gelu", 10),
+                                                       ("mlp_small_same", "same", "relu", 15)])
 def test_small_net_step_equals_the_layer_calls_and_counts_its_launches(name, variant, act, launches):
     """On the nets that run on CUDA cores a layer's dW and the gradient of its input share one launch inside
     rad_mlp_step (Sec. 4.2: both are contractions of the same dZ).  The step's weight gradients and loss equal,
     bit for bit, those of the same step made of the public layer calls, one launch per contraction; the bias
-    gradients agree to rounding (the step sums them in the dW kernel); and the MNIST-shaped net takes ten launches."""
+    gradients agree to rounding (the step sums them in the dW kernel); and the MNIST-shaped net takes ten launches
+    (fifteen with same-sample stores, whose store is three kernels)."""
     import paper_2007_10412_b200 as rad
     cfg = get_config(name)
     dims, B, L = cfg.dims, cfg.batch, len(cfg.dims) - 1
@@ -154,7 +156,8 @@ def test_small_net_step_equals_the_layer_calls_and_counts_its_launches(name, var
     # the same step, call by call
     tdt = dX.dtype
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    stores = [rad.Store("different", cfg.dtype, B, dims[l], 0.1, seed=21, layer=l, step=5, relu_bits=False) for l in range(L)]
+    stores = [rad.Store("same" if variant == "same" else "different", cfg.dtype, B, dims[l], 0.1, seed=21, layer=l, step=5,
+                        relu_bits=False) for l in range(L)]
     rbits = [None] + [torch.empty(B * ((dims[l] + 31) // 32), dtype=torch.int32, device="cuda") if act == "relu" else None
                       for l in range(1, L)]
     pre = [None] + [torch.empty(B, dims[l], dtype=tdt, device="cuda") if act == "gelu" else None for l in range(1, L)]
