@@ -293,8 +293,8 @@ int rad_linear_weight_grad(const rad_store* st /* host */, const void* dZ /* dev
                            int32_t* dev_status, void* stream);
 
 /*
- * Exact forward of one layer (never sampled: Sec. 3, the original graph is used
- * for the forward pass): Z = A W + bias, out = act(Z).
+ * Exact forward of one layer (Sec. 3: sampling changes only what the backward pass
+ * reads, the forward pass computes the unsampled network): Z = A W + bias, out = act(Z).
  *   A device B x D (dtype), W device D x H (dtype), bias device float32[H] or NULL.
  *   out_act  device B x H (dtype) or NULL: act(Z) rounded to dtype.
  *   out_z    device B x H float32 or NULL: Z before the activation (the softmax input).

@@ -214,9 +214,6 @@ extern "C" const char* rad_strerror(int code) {
 
 namespace rad {
 namespace {
-// rad_linear_weight_grad for a bitmask or column-list store (index held or drawn again); where the contraction
-// runs on the CUDA cores and passes over dZ anyway, it also leaves the bias gradient in `db` (*db_written says
-// whether it did).
 // Does the input gradient of these operands run on the tensor cores?
 bool input_grad_on_tc(int32_t dtype, int64_t B, int64_t D, int64_t H, const void* dZ, int64_t ldz, const void* W,
                       int64_t ldw, const void* z_prev, int64_t ld_zprev, const void* dZ_prev, int64_t ldp) {
@@ -224,6 +221,9 @@ bool input_grad_on_tc(int32_t dtype, int64_t B, int64_t D, int64_t H, const void
          (z_prev == nullptr || (((uintptr_t)z_prev & 15) == 0 && ld_zprev % 8 == 0));
 }
 
+// rad_linear_weight_grad for a bitmask or column-list store (index held or drawn again); where the contraction
+// runs on the CUDA cores and passes over dZ anyway, it also leaves the bias gradient in `db` (*db_written says
+// whether it did).
 // ig (optional): the input gradient of the same layer; where both contractions run on CUDA cores they share one
 // launch and *ig_done is set, otherwise the caller runs rad_linear_input_grad as usual.
 int weight_grad_and_bias(const rad_store* st, const void* dZ, int64_t ldz, int64_t H, float* dW, int64_t ldw, void* workspace,
