@@ -34,10 +34,15 @@ struct GemmParams {
   float* db;                   // or NULL: column sums of Bm over k (the bias gradient), from the CTAs of tile row 0
 };
 
-// One 64 x 64 tile of C by one CTA of 256 threads; (bx, by) = tile column and row.
+// One 64 x 64 tile of C by one CTA of 256 threads; (bx, by) = tile column and row.  The K loop is double
+// buffered: the next 16 rows of K travel from global memory to registers while the current ones are
+// multiplied out of shared memory, one barrier per step (these GEMMs serve the small nets, where a CTA's time
+// is the latency of its loads).  Every output is one chain of fused multiply-adds over k in ascending order.
+constexpr int kLdS = kBM + 4;                      // floats per k row of a staged operand (16-byte multiples)
+constexpr int kGemmSmemFloats = 4 * kBK * kLdS;    // A and B, two buffers each
+static_assert(kBM == kBN && (kLdS * 4) % 16 == 0, "both operands share the staging layout");
 template <typename T, int EPI>
-__device__ __forceinline__ void gemm_body(const GemmParams& p, int64_t bx, int64_t by, float (*sA)[kBM + 4],
-                                          float (*sB)[kBN + 4]) {
+__device__ __forceinline__ void gemm_body(const GemmParams& p, int64_t bx, int64_t by, float* smem) {
   int64_t M = p.M;
   if (p.M_dev != nullptr) M = min(M, *p.M_dev);
   const int64_t m0 = by * kBM, n0 = bx * kBN;
@@ -49,38 +54,60 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, int64_t bx, int64
   const T* A = static_cast<const T*>(p.A);
   const T* Bm = static_cast<const T*>(p.Bm);
   float acc[4][4] = {};
-  for (int64_t k0 = 0; k0 < p.K; k0 += kBK) {
-    // 64 x 16 elements of each operand, 4 per thread; whichever index is contiguous in memory
-    // is made the fast thread index
-    for (int i = tid; i < kBM * kBK; i += 256) {
+  // 64 x 16 elements of each operand per step, 4 per thread; whichever index is contiguous in memory is made
+  // the fast thread index
+  float ra[4], rb[4];
+  auto fetch = [&](int64_t k0) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int i = tid + j * 256;
       int mm, kk;
       if (p.sak == 1) { kk = i % kBK; mm = i / kBK; } else { mm = i % kBM; kk = i / kBM; }
       const int64_t m = m0 + mm, k = k0 + kk;
-      sA[kk][mm] = (m < M && k < p.K) ? to_float(A[m * p.sam + k * p.sak]) : 0.0f;
-    }
-    for (int i = tid; i < kBN * kBK; i += 256) {
-      int nn, kk;
+      ra[j] = (m < M && k < p.K) ? to_float(A[m * p.sam + k * p.sak]) : 0.0f;
+      int nn;
       if (p.sbk == 1) { kk = i % kBK; nn = i / kBK; } else { nn = i % kBN; kk = i / kBN; }
-      const int64_t n = n0 + nn, k = k0 + kk;
-      sB[kk][nn] = (n < p.N && k < p.K) ? to_float(Bm[k * p.sbk + n * p.sbn]) : 0.0f;
+      const int64_t n = n0 + nn, kb = k0 + kk;
+      rb[j] = (n < p.N && kb < p.K) ? to_float(Bm[kb * p.sbk + n * p.sbn]) : 0.0f;
     }
-    __syncthreads();
+  };
+  auto stash = [&](int buf) {
+    float* sA = smem + buf * 2 * kBK * kLdS;
+    float* sB = sA + kBK * kLdS;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int i = tid + j * 256;
+      if (p.sak == 1) sA[(i % kBK) * kLdS + i / kBK] = ra[j]; else sA[(i / kBM) * kLdS + i % kBM] = ra[j];
+      if (p.sbk == 1) sB[(i % kBK) * kLdS + i / kBK] = rb[j]; else sB[(i / kBN) * kLdS + i % kBN] = rb[j];
+    }
+  };
+  fetch(0);
+  stash(0);
+  __syncthreads();
+  int buf = 0;
+  for (int64_t k0 = 0; k0 < p.K; k0 += kBK) {
+    const bool more = k0 + kBK < p.K;
+    if (more) fetch(k0 + kBK);
+    const float* sA = smem + buf * 2 * kBK * kLdS;
+    const float* sB = sA + kBK * kLdS;
     if (sums && tid < kBN) {
       // the block of Bm is in shared memory anyway: its column sums, row after row (rows past K hold zeros)
 #pragma unroll
-      for (int kk = 0; kk < kBK; ++kk) colsum += sB[kk][tid];
+      for (int kk = 0; kk < kBK; ++kk) colsum += sB[kk * kLdS + tid];
     }
 #pragma unroll
     for (int kk = 0; kk < kBK; ++kk) {
-      float a[4], b[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) { a[i] = sA[kk][tm + i]; b[i] = sB[kk][tn + i]; }
+      const float4 a4 = *reinterpret_cast<const float4*>(sA + kk * kLdS + tm);
+      const float4 b4 = *reinterpret_cast<const float4*>(sB + kk * kLdS + tn);
+      const float a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
     }
+    if (more) stash(buf ^ 1);
     __syncthreads();
+    buf ^= 1;
   }
   if (sums && tid < kBN && n0 + tid < p.N) p.db[n0 + tid] = colsum;
 #pragma unroll
@@ -116,9 +143,8 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, int64_t bx, int64
 
 template <typename T, int EPI>
 __global__ void __launch_bounds__(256) gemm_kernel(const GemmParams p) {
-  __shared__ float sA[kBK][kBM + 4];
-  __shared__ float sB[kBK][kBN + 4];
-  gemm_body<T, EPI>(p, blockIdx.x, blockIdx.y, sA, sB);
+  __shared__ __align__(16) float smem[kGemmSmemFloats];
+  gemm_body<T, EPI>(p, blockIdx.x, blockIdx.y, smem);
 }
 
 template <int EPI>
@@ -253,7 +279,7 @@ __global__ void __launch_bounds__(256) sparse_dw_kernel(const SparseDwParams p) 
 // input-gradient GEMM, each doing exactly what it does in a launch of its own (the nets that run on CUDA
 // cores are bound by their launch count).
 constexpr int kDwDxSmemA = kTileRows * (kTileCols + 1) * 4, kDwDxSmemZ = kTileRows * (kSparseBN + 1) * 4;
-static_assert(kDwDxSmemA + kDwDxSmemZ + 1024 >= 2 * kBK * (kBM + 4) * 4 && kBM == kBN, "the GEMM's tiles fit the same buffer");
+static_assert(kDwDxSmemA + kDwDxSmemZ + 1024 >= kGemmSmemFloats * 4, "the GEMM's tiles fit the same buffer");
 template <typename T>
 __global__ void __launch_bounds__(256) dw_dx_kernel(const SparseDwParams d, const GemmParams g, int dw_blocks, int gx) {
   __shared__ __align__(16) unsigned char raw[kDwDxSmemA + kDwDxSmemZ + 1024];
@@ -263,8 +289,7 @@ __global__ void __launch_bounds__(256) dw_dx_kernel(const SparseDwParams d, cons
                       reinterpret_cast<uint32_t*>(raw + kDwDxSmemA + kDwDxSmemZ));
   } else {
     const int b = (int)blockIdx.x - dw_blocks;
-    gemm_body<T, kEpiInputGrad>(g, b % gx, b / gx, reinterpret_cast<float(*)[kBM + 4]>(raw),
-                                reinterpret_cast<float(*)[kBN + 4]>(raw + kBK * (kBM + 4) * 4));
+    gemm_body<T, kEpiInputGrad>(g, b % gx, b / gx, reinterpret_cast<float*>(raw));
   }
 }
 
@@ -320,13 +345,12 @@ __global__ void __launch_bounds__(256) colsum_small_kernel(const T* dZ, int64_t 
 template <typename T>
 __global__ void __launch_bounds__(256) same_dw_dx_kernel(const GemmParams w, const GemmParams g, int dw_blocks, int gxw,
                                                          int dx_blocks, int gxg, const uint32_t* keep_cols, int64_t D, int64_t H) {
-  __shared__ float sA[kBK][kBM + 4];
-  __shared__ float sB[kBK][kBN + 4];
+  __shared__ __align__(16) float smem[kGemmSmemFloats];
   const int b = (int)blockIdx.x;
   if (b < dw_blocks) {
-    gemm_body<T, kEpiScatterRows>(w, b % gxw, b / gxw, sA, sB);
+    gemm_body<T, kEpiScatterRows>(w, b % gxw, b / gxw, smem);
   } else if (b < dw_blocks + dx_blocks) {
-    gemm_body<T, kEpiInputGrad>(g, (b - dw_blocks) % gxg, (b - dw_blocks) / gxg, sA, sB);
+    gemm_body<T, kEpiInputGrad>(g, (b - dw_blocks) % gxg, (b - dw_blocks) / gxg, smem);
   } else {
     const int nz = (int)gridDim.x - dw_blocks - dx_blocks;
     for (int64_t d = b - dw_blocks - dx_blocks; d < D; d += nz) {
