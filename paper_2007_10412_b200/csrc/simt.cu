@@ -320,6 +320,27 @@ __global__ void __launch_bounds__(256) colsum_final_kernel(const float* partial,
   for (int64_t c = 0; c < chunks; ++c) s += partial[c * H + h];
   db[h] = s;
 }
+// First stage for a narrow matrix (at most 64 columns, e.g. the bias gradient of a convolution: B H W rows, 16
+// columns), where one thread per column would leave most of a CTA idle: the CTA's threads are R row lanes x HP
+// columns (HP the power of two that holds H); a lane sums every R-th row of the CTA's slab, then the column's
+// lanes are added in lane order.  Second stage as above.
+template <typename T>
+__global__ void __launch_bounds__(256) colsum_narrow_partial_kernel(const T* dZ, int64_t ldz, int64_t B, int H, int HP,
+                                                                    int64_t rows_per_block, float* partial) {
+  __shared__ float s[256];
+  const int c = threadIdx.x & (HP - 1), r = threadIdx.x / HP, R = 256 / HP;
+  const int64_t b0 = (int64_t)blockIdx.x * rows_per_block, b1 = min(B, b0 + rows_per_block);
+  float sum = 0.0f;
+  if (c < H)
+    for (int64_t b = b0 + r; b < b1; b += R) sum += to_float(dZ[b * ldz + c]);
+  s[threadIdx.x] = sum;
+  __syncthreads();
+  if (r == 0 && c < H) {
+    float t = 0.0f;
+    for (int i = 0; i < R; ++i) t += s[i * HP + c];
+    partial[(int64_t)blockIdx.x * H + c] = t;
+  }
+}
 // Both stages in one launch for few rows (the small nets are bound by their launch count): the same chunk sums,
 // added in the same order, by the thread that owns the column.
 constexpr int kColSmallChunks = 2;
@@ -491,9 +512,23 @@ int column_sums(int dtype, int64_t B, int64_t H, const void* dZ, int64_t ldz, fl
       colsum_small_kernel<float><<<(unsigned)ceil_div(H, 256), 256, 0, s>>>(static_cast<const float*>(dZ), ldz, B, H, db);
     return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
   }
-  dim3 grid((unsigned)ceil_div(H, 256), (unsigned)chunks);
   float* partial = static_cast<float*>(workspace);
   count_launch(2);
+  if (H <= 64) {
+    // no more slabs than the chunk count the workspace was sized for
+    const int64_t slabs = std::min<int64_t>(chunks, 2 * 148);
+    const int64_t rows_per_block = ceil_div(B, slabs), nblocks = ceil_div(B, rows_per_block);
+    const int HP = H <= 16 ? 16 : H <= 32 ? 32 : 64;
+    if (dtype == RAD_BF16)
+      colsum_narrow_partial_kernel<bf16><<<(unsigned)nblocks, 256, 0, s>>>(static_cast<const bf16*>(dZ), ldz, B, (int)H, HP,
+                                                                          rows_per_block, partial);
+    else
+      colsum_narrow_partial_kernel<float><<<(unsigned)nblocks, 256, 0, s>>>(static_cast<const float*>(dZ), ldz, B, (int)H, HP,
+                                                                           rows_per_block, partial);
+    colsum_final_kernel<<<1, 256, 0, s>>>(partial, nblocks, H, db);
+    return cudaGetLastError() == cudaSuccess ? RAD_OK : RAD_ECUDA;
+  }
+  dim3 grid((unsigned)ceil_div(H, 256), (unsigned)chunks);
   if (dtype == RAD_BF16)
     colsum_partial_kernel<bf16><<<grid, 256, 0, s>>>(static_cast<const bf16*>(dZ), ldz, B, H, partial);
   else
