@@ -32,17 +32,21 @@ struct GemmParams {
   const uint32_t* row_idx;
   float* out_f32; int64_t ld_f32;
   float* db;                   // or NULL: column sums of Bm over k (the bias gradient), from the CTAs of tile row 0
+  int tile;                    // 64 or 32: rows and columns of C per CTA
 };
 
-// One 64 x 64 tile of C by one CTA of 256 threads; (bx, by) = tile column and row.  The K loop is double
+// One TS x TS tile of C (TS = 64, or 32 where 64 would leave most SMs without a CTA) by one CTA of 256 threads,
+// TS/16 x TS/16 outputs per thread; (bx, by) = tile column and row.  The K loop is double
 // buffered: the next 16 rows of K travel from global memory to registers while the current ones are
 // multiplied out of shared memory, one barrier per step (these GEMMs serve the small nets, where a CTA's time
 // is the latency of its loads).  Every output is one chain of fused multiply-adds over k in ascending order.
-constexpr int kLdS = kBM + 4;                      // floats per k row of a staged operand (16-byte multiples)
-constexpr int kGemmSmemFloats = 4 * kBK * kLdS;    // A and B, two buffers each
-static_assert(kBM == kBN && (kLdS * 4) % 16 == 0, "both operands share the staging layout");
-template <typename T, int EPI>
+constexpr int kGemmSmemFloats = 4 * kBK * (kBM + 4);    // A and B, two buffers each, of the larger tile
+static_assert(kBM == kBN, "both operands share the staging layout");
+template <typename T, int EPI, int TS>
 __device__ __forceinline__ void gemm_body(const GemmParams& p, int64_t bx, int64_t by, float* smem) {
+  constexpr int kBM = TS, kBN = TS, TM = TS / 16;
+  constexpr int kLdS = TS + 4;                       // floats per k row of a staged operand (16-byte multiples)
+  static_assert((kLdS * 4) % 16 == 0 && (TM == 4 || TM == 2), "vector reads of the staged operands");
   int64_t M = p.M;
   if (p.M_dev != nullptr) M = min(M, *p.M_dev);
   const int64_t m0 = by * kBM, n0 = bx * kBN;
@@ -50,16 +54,16 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, int64_t bx, int64
   if (m0 >= M && !sums) return;
   const int tid = threadIdx.x;
   float colsum = 0.0f;
-  const int tm = (tid >> 4) * 4, tn = (tid & 15) * 4;
+  const int tm = (tid >> 4) * TM, tn = (tid & 15) * TM;
   const T* A = static_cast<const T*>(p.A);
   const T* Bm = static_cast<const T*>(p.Bm);
-  float acc[4][4] = {};
-  // 64 x 16 elements of each operand per step, 4 per thread; whichever index is contiguous in memory is made
+  float acc[TM][TM] = {};
+  // TS x 16 elements of each operand per step, TS/16 per thread; whichever index is contiguous in memory is made
   // the fast thread index
-  float ra[4], rb[4];
+  float ra[TM], rb[TM];
   auto fetch = [&](int64_t k0) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int j = 0; j < TM; ++j) {
       const int i = tid + j * 256;
       int mm, kk;
       if (p.sak == 1) { kk = i % kBK; mm = i / kBK; } else { mm = i % kBM; kk = i / kBM; }
@@ -75,7 +79,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, int64_t bx, int64
     float* sA = smem + buf * 2 * kBK * kLdS;
     float* sB = sA + kBK * kLdS;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int j = 0; j < TM; ++j) {
       const int i = tid + j * 256;
       if (p.sak == 1) sA[(i % kBK) * kLdS + i / kBK] = ra[j]; else sA[(i / kBM) * kLdS + i % kBM] = ra[j];
       if (p.sbk == 1) sB[(i % kBK) * kLdS + i / kBK] = rb[j]; else sB[(i / kBN) * kLdS + i % kBN] = rb[j];
@@ -97,13 +101,22 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, int64_t bx, int64
     }
 #pragma unroll
     for (int kk = 0; kk < kBK; ++kk) {
-      const float4 a4 = *reinterpret_cast<const float4*>(sA + kk * kLdS + tm);
-      const float4 b4 = *reinterpret_cast<const float4*>(sB + kk * kLdS + tn);
-      const float a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
+      float a[TM], b[TM];
+      if (TM == 4) {
+        const float4 a4 = *reinterpret_cast<const float4*>(sA + kk * kLdS + tm);
+        const float4 b4 = *reinterpret_cast<const float4*>(sB + kk * kLdS + tn);
+        a[0] = a4.x; a[1] = a4.y; a[TM - 2] = a4.z; a[TM - 1] = a4.w;
+        b[0] = b4.x; b[1] = b4.y; b[TM - 2] = b4.z; b[TM - 1] = b4.w;
+      } else {
+        const float2 a2 = *reinterpret_cast<const float2*>(sA + kk * kLdS + tm);
+        const float2 b2 = *reinterpret_cast<const float2*>(sB + kk * kLdS + tn);
+        a[0] = a2.x; a[1] = a2.y;
+        b[0] = b2.x; b[1] = b2.y;
+      }
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
+      for (int i = 0; i < TM; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        for (int j = 0; j < TM; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
     }
     if (more) stash(buf ^ 1);
     __syncthreads();
@@ -111,11 +124,11 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, int64_t bx, int64
   }
   if (sums && tid < kBN && n0 + tid < p.N) p.db[n0 + tid] = colsum;
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
+  for (int i = 0; i < TM; ++i) {
     const int64_t m = m0 + tm + i;
     if (m >= M) continue;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int j = 0; j < TM; ++j) {
       const int64_t n = n0 + tn + j;
       if (n >= p.N) continue;
       float v = acc[i][j];
@@ -141,15 +154,25 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, int64_t bx, int64
   }
 }
 
+// The tile a GEMM of M x N outputs runs with, and the body for it.
+inline int pick_tile(int64_t M, int64_t N) { return ceil_div(M, 64) * ceil_div(N, 64) < 64 ? 32 : 64; }
+template <typename T, int EPI>
+__device__ __forceinline__ void gemm_tile(const GemmParams& p, int64_t bx, int64_t by, float* smem) {
+  if (p.tile == 32) gemm_body<T, EPI, 32>(p, bx, by, smem);
+  else gemm_body<T, EPI, 64>(p, bx, by, smem);
+}
+
 template <typename T, int EPI>
 __global__ void __launch_bounds__(256) gemm_kernel(const GemmParams p) {
   __shared__ __align__(16) float smem[kGemmSmemFloats];
-  gemm_body<T, EPI>(p, blockIdx.x, blockIdx.y, smem);
+  gemm_tile<T, EPI>(p, blockIdx.x, blockIdx.y, smem);
 }
 
 template <int EPI>
-int launch_gemm(int dtype, const GemmParams& p, int64_t Mgrid, cudaStream_t s) {
-  dim3 grid((unsigned)ceil_div(p.N, kBN), (unsigned)ceil_div(Mgrid, kBM));
+int launch_gemm(int dtype, const GemmParams& p0, int64_t Mgrid, cudaStream_t s) {
+  GemmParams p = p0;
+  p.tile = pick_tile(Mgrid, p.N);
+  dim3 grid((unsigned)ceil_div(p.N, p.tile), (unsigned)ceil_div(Mgrid, p.tile));
   if (grid.x == 0 || grid.y == 0) return RAD_OK;
   count_launch();
   if (dtype == RAD_BF16)
@@ -289,7 +312,7 @@ __global__ void __launch_bounds__(256) dw_dx_kernel(const SparseDwParams d, cons
                       reinterpret_cast<uint32_t*>(raw + kDwDxSmemA + kDwDxSmemZ));
   } else {
     const int b = (int)blockIdx.x - dw_blocks;
-    gemm_body<T, kEpiInputGrad>(g, b % gx, b / gx, reinterpret_cast<float*>(raw));
+    gemm_tile<T, kEpiInputGrad>(g, b % gx, b / gx, reinterpret_cast<float*>(raw));
   }
 }
 
@@ -369,9 +392,9 @@ __global__ void __launch_bounds__(256) same_dw_dx_kernel(const GemmParams w, con
   __shared__ __align__(16) float smem[kGemmSmemFloats];
   const int b = (int)blockIdx.x;
   if (b < dw_blocks) {
-    gemm_body<T, kEpiScatterRows>(w, b % gxw, b / gxw, smem);
+    gemm_tile<T, kEpiScatterRows>(w, b % gxw, b / gxw, smem);
   } else if (b < dw_blocks + dx_blocks) {
-    gemm_body<T, kEpiInputGrad>(g, (b - dw_blocks) % gxg, (b - dw_blocks) / gxg, smem);
+    gemm_tile<T, kEpiInputGrad>(g, (b - dw_blocks) % gxg, (b - dw_blocks) / gxg, smem);
   } else {
     const int nz = (int)gridDim.x - dw_blocks - dx_blocks;
     for (int64_t d = b - dw_blocks - dx_blocks; d < D; d += nz) {
@@ -443,12 +466,14 @@ int simt_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H
     p.row_idx = st->offsets; p.out_f32 = dW; p.ld_f32 = ldw;
     p.db = db;
     if (db_written != nullptr) *db_written = db != nullptr;
-    const int64_t gxw = ceil_div(p.N, kBN), dw_blocks = gxw * std::max<int64_t>(1, ceil_div(p.M, kBM));
+    p.tile = pick_tile(p.M, p.N);
+    const int64_t gxw = ceil_div(p.N, p.tile), dw_blocks = gxw * std::max<int64_t>(1, ceil_div(p.M, p.tile));
     if (st->keepbits != nullptr) {
       // one launch: scatter, zeros for the rows not kept and, where asked for, the input gradient
       const bool with_dx = ig != nullptr && ig_done != nullptr;
-      const GemmParams g = with_dx ? input_grad_params(st->B, st->D, H, dZ, ldz, *ig) : GemmParams{};
-      const int64_t gxg = with_dx ? ceil_div(g.N, kBN) : 1, dx_blocks = with_dx ? gxg * ceil_div(g.M, kBM) : 0;
+      GemmParams g = with_dx ? input_grad_params(st->B, st->D, H, dZ, ldz, *ig) : GemmParams{};
+      g.tile = with_dx ? pick_tile(g.M, g.N) : 64;
+      const int64_t gxg = with_dx ? ceil_div(g.N, g.tile) : 1, dx_blocks = with_dx ? gxg * ceil_div(g.M, g.tile) : 0;
       const int64_t nz = std::min<int64_t>(st->D, 148 * 4);
       if (dw_blocks + dx_blocks + nz <= 0x7fffffff) {
         count_launch();
@@ -478,8 +503,9 @@ int simt_weight_grad(const rad_store* st, const void* dZ, int64_t ldz, int64_t H
   dim3 grid((unsigned)p.ncb, (unsigned)ceil_div(H, kSparseBN));
   count_launch();
   if (ig != nullptr && ig_done != nullptr) {
-    const GemmParams g = input_grad_params(st->B, st->D, H, dZ, ldz, *ig);
-    const int64_t gx = ceil_div(g.N, kBN), gy = ceil_div(g.M, kBM), dw_blocks = (int64_t)grid.x * grid.y;
+    GemmParams g = input_grad_params(st->B, st->D, H, dZ, ldz, *ig);
+    g.tile = pick_tile(g.M, g.N);
+    const int64_t gx = ceil_div(g.N, g.tile), gy = ceil_div(g.M, g.tile), dw_blocks = (int64_t)grid.x * grid.y;
     if (dw_blocks + gx * gy <= 0x7fffffff) {
       if (st->dtype == RAD_BF16)
         dw_dx_kernel<bf16><<<(unsigned)(dw_blocks + gx * gy), 256, 0, s>>>(p, g, (int)dw_blocks, (int)gx);
