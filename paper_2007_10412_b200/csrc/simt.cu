@@ -40,11 +40,15 @@ struct GemmParams {
 // buffered: the next 16 rows of K travel from global memory to registers while the current ones are
 // multiplied out of shared memory, one barrier per step (these GEMMs serve the small nets, where a CTA's time
 // is the latency of its loads).  Every output is one chain of fused multiply-adds over k in ascending order.
-constexpr int kGemmSmemFloats = 4 * kBK * (kBM + 4);    // A and B, two buffers each, of the larger tile
+// K rows per step: the small tile takes four times as many, so that its steps, which are bound by the latency
+// of their loads, are a quarter as many.
+constexpr int gemm_bk(int ts) { return ts == 32 ? 64 : 16; }
+constexpr int kGemmSmemFloats = 4 * gemm_bk(32) * (32 + 4) > 4 * gemm_bk(64) * (64 + 4) ? 4 * gemm_bk(32) * (32 + 4)
+                                                                                         : 4 * gemm_bk(64) * (64 + 4);
 static_assert(kBM == kBN, "both operands share the staging layout");
 template <typename T, int EPI, int TS>
 __device__ __forceinline__ void gemm_body(const GemmParams& p, int64_t bx, int64_t by, float* smem) {
-  constexpr int kBM = TS, kBN = TS, TM = TS / 16;
+  constexpr int kBM = TS, kBN = TS, TM = TS / 16, kBK = gemm_bk(TS), NF = TS * kBK / 256;
   constexpr int kLdS = TS + 4;                       // floats per k row of a staged operand (16-byte multiples)
   static_assert((kLdS * 4) % 16 == 0 && (TM == 4 || TM == 2), "vector reads of the staged operands");
   int64_t M = p.M;
@@ -58,12 +62,12 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, int64_t bx, int64
   const T* A = static_cast<const T*>(p.A);
   const T* Bm = static_cast<const T*>(p.Bm);
   float acc[TM][TM] = {};
-  // TS x 16 elements of each operand per step, TS/16 per thread; whichever index is contiguous in memory is made
+  // TS x kBK elements of each operand per step; whichever index is contiguous in memory is made
   // the fast thread index
-  float ra[TM], rb[TM];
+  float ra[NF], rb[NF];
   auto fetch = [&](int64_t k0) {
 #pragma unroll
-    for (int j = 0; j < TM; ++j) {
+    for (int j = 0; j < NF; ++j) {
       const int i = tid + j * 256;
       int mm, kk;
       if (p.sak == 1) { kk = i % kBK; mm = i / kBK; } else { mm = i % kBM; kk = i / kBM; }
@@ -79,7 +83,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, int64_t bx, int64
     float* sA = smem + buf * 2 * kBK * kLdS;
     float* sB = sA + kBK * kLdS;
 #pragma unroll
-    for (int j = 0; j < TM; ++j) {
+    for (int j = 0; j < NF; ++j) {
       const int i = tid + j * 256;
       if (p.sak == 1) sA[(i % kBK) * kLdS + i / kBK] = ra[j]; else sA[(i / kBM) * kLdS + i % kBM] = ra[j];
       if (p.sbk == 1) sB[(i % kBK) * kLdS + i / kBK] = rb[j]; else sB[(i / kBN) * kLdS + i % kBN] = rb[j];
