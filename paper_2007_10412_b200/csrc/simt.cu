@@ -242,16 +242,14 @@ __device__ __forceinline__ void sparse_dw_body(const SparseDwParams& p, int cb, 
     __syncthreads();
     uint32_t wbase = 0;
     for (int w = 0; w < warp; ++w) wbase += s_scan[w];
-    uint32_t pos = wbase + incl - cnt;
-    const int64_t base = p.offsets[tile];
+    const int64_t base = p.offsets[tile] + (wbase + incl - cnt);
     const int r = tid >> 2, c0 = (tid & 3) * 32;
-#pragma unroll 4
+    // every kept entry's place follows from the word alone, so the loads do not wait for one another
+#pragma unroll 16
     for (int b = 0; b < 32; ++b) {
+      const int64_t at = base + __popc(word & ((1u << b) - 1u));
       float v = 0.0f;
-      if ((word >> b) & 1u) {                       // a store that overflowed is never read past
-        const int64_t at = base + pos++;
-        if (at < p.capacity) v = to_float(vals[at]);
-      }
+      if (((word >> b) & 1u) != 0 && at < p.capacity) v = to_float(vals[at]);   // a store that overflowed is never read past
       sAh[r][c0 + b] = v;
     }
     for (int i = tid; i < kTileRows * kSparseBN; i += 256) {
