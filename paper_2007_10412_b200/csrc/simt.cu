@@ -334,6 +334,7 @@ __global__ void __launch_bounds__(256) colsum_partial_kernel(const T* dZ, int64_
   if (h >= H) return;
   const int64_t b0 = (int64_t)blockIdx.y * kColChunkRows, b1 = min(B, b0 + kColChunkRows);
   float s = 0.0f;
+#pragma unroll 8
   for (int64_t b = b0; b < b1; ++b) s += to_float(dZ[b * ldz + h]);
   partial[(int64_t)blockIdx.y * H + h] = s;
 }
@@ -342,7 +343,8 @@ __global__ void __launch_bounds__(256) colsum_final_kernel(const float* partial,
   const int64_t h = (int64_t)blockIdx.x * 256 + threadIdx.x;
   if (h >= H) return;
   float s = 0.0f;
-  for (int64_t c = 0; c < chunks; ++c) s += partial[c * H + h];
+#pragma unroll 8
+  for (int64_t c = 0; c < chunks; ++c) s += partial[c * H + h];      // loads in flight together, added in order
   db[h] = s;
 }
 // First stage for a narrow matrix (at most 64 columns, e.g. the bias gradient of a convolution: B H W rows, 16
@@ -357,6 +359,7 @@ __global__ void __launch_bounds__(256) colsum_narrow_partial_kernel(const T* dZ,
   const int64_t b0 = (int64_t)blockIdx.x * rows_per_block, b1 = min(B, b0 + rows_per_block);
   float sum = 0.0f;
   if (c < H)
+#pragma unroll 8
     for (int64_t b = b0 + r; b < b1; b += R) sum += to_float(dZ[b * ldz + c]);
   s[threadIdx.x] = sum;
   __syncthreads();
@@ -377,6 +380,7 @@ __global__ void __launch_bounds__(256) colsum_small_kernel(const T* dZ, int64_t 
   for (int64_t b0 = 0; b0 < B; b0 += kColChunkRows) {
     const int64_t b1 = min(B, b0 + kColChunkRows);
     float s = 0.0f;
+#pragma unroll 8
     for (int64_t b = b0; b < b1; ++b) s += to_float(dZ[b * ldz + h]);
     total += s;
   }
