@@ -9,7 +9,7 @@
 namespace rad {
 namespace {
 
-constexpr int kBM = 64, kBN = 64, kBK = 16;
+constexpr int kBM = 64, kBN = 64;      // the larger of the two tiles
 
 enum Epilogue { kEpiForward = 0, kEpiInputGrad = 1, kEpiScatterRows = 2 };
 
