@@ -125,3 +125,26 @@ def test_softmax_xent_matches_oracle(B, C, dtype):
     torch.cuda.synchronize()
     assert abs(loss.item() - loss_ref) <= 1e-5 * abs(loss_ref)
     assert max(rel_err(to_host_f32(dz), dz_ref)) <= (1e-5 if dtype == "f32" else 8e-3)
+
+
+@pytest.mark.parametrize("B,H,dtype", [(700, 10, "f32"), (700, 40, "bf16"), (5000, 64, "bf16"), (40000, 16, "bf16"),
+                                       (700, 300, "f32"), (700, 301, "bf16"), (2100, 1000, "bf16"), (130, 1000, "bf16")])
+def test_bias_gradient_alone_on_every_column_sum_route(B, H, dtype):
+    """db = sum over the minibatch of dZ (Sec. 4.2: exact, never sampled), asked for without the input gradient:
+    few rows (one launch), narrow matrices (row lanes x columns), wide bf16 matrices (16-byte loads) and the
+    plain two-stage route, against float64 sums of the same numbers."""
+    import paper_2007_10412_b200 as rad
+    rng = np.random.default_rng(B + H)
+    dZ = rng.standard_normal((B, H), dtype=np.float32)
+    if dtype == "bf16":
+        from workloads import to_bf16_grid
+        dZ = to_bf16_grid(dZ)
+    W = torch.zeros(8, H, dtype=torch.float32 if dtype == "f32" else torch.bfloat16, device="cuda")
+    db = torch.full((H,), float("nan"), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    rad.rad_linear_input_grad(to_dev(dZ, dtype), W, db=db, dev_status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    want = dZ.astype(np.float64).sum(axis=0)
+    bound = 2e-6 * np.abs(dZ.astype(np.float64)).sum(axis=0)
+    assert (np.abs(to_host_f32(db).astype(np.float64) - want) <= bound).all()
