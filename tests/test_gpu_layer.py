@@ -18,6 +18,7 @@ LAYERS = [
     (328, 640, 520, "bf16"),    # aligned bf16: tensor-core kernels
     (328, 392, 200, "bf16"),
     (1024, 256, 512, "bf16"),
+    (900, 520, 600, "f32"),     # float32 with enough tiles for the CUDA-core GEMM's larger tile
 ]
 
 
