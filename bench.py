@@ -479,6 +479,19 @@ def kernel_sweep(rad, torch, A, dZ, H, ps, pk, clock, stores):
             row.update(dW_tflops_kept_columns=round(2.0 * B * int(nnz[0]) * H / ms_dw / 1e9, 1))
         rows.append(row)
         del st, ws
+    # the same-sample contraction against the kept-column count (fixed-count law: the count is exact): its time
+    # follows the number of 256-column tiles, not their width
+    for k in (416, 512, 768, 832, 1024, 2048):
+        st = rad.Store("same", "bf16", B, D, k / D, relu_bits=False, law="fixed")
+        rad.rad_linear_forward_store(A, st, status)
+        ws = torch.empty(max(rad.rad_weight_grad_workspace(st, H), 256), dtype=torch.uint8, device="cuda")
+        ms_dw, mhz_dw = timed_alone(torch, lambda: rad.rad_linear_weight_grad(st, dZ, dW, ws, status), clock, n=5, settle_ms=20.0,
+                                    idle_ms=150.0)
+        kk = int(st.nnz.cpu().numpy()[0])
+        tf = 2.0 * B * kk * H / ms_dw / 1e9
+        rows.append(dict(variant="same", law="fixed", kept_columns=kk, tiles=-(-kk // 256), dW_ms=round(ms_dw, 4), dW_sm_mhz=mhz_dw,
+                         dW_tflops_kept_columns=round(tf, 1), dW_frac_burst=frac(tf, burst)))
+        del st, ws
     # the fixed-count law in its static-shape form: B x k values and B x k 16-bit column numbers (k the same for
     # every row); the weight gradient rebuilds the tile-major index from the key and moves the values into it
     p = 0.1
